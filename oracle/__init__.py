@@ -1,0 +1,169 @@
+"""CPU fp64 oracle for paged-KV rollout attention (see rollart_oracle.c for what it computes).
+
+TEST INFRASTRUCTURE ONLY.  Nothing in the product package imports this; only the tests,
+the smoke check and the bench's CPU-baseline leg do.  Arrays are numpy; bf16 data travels
+as uint16 bit patterns.  Every function here is pinned by tests/test_oracle_pins.py.
+"""
+from __future__ import annotations
+
+import ctypes
+from typing import Optional, Sequence
+
+import numpy as np
+
+from .build import build as _build
+
+_lib = None
+
+_STATUS = {1: "bad argument", 2: "page id out of range", 3: "length out of range"}
+
+
+class OracleError(ValueError):
+    pass
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        L = ctypes.CDLL(_build())
+        L.oracle_num_threads.restype = ctypes.c_int
+        for name in ("oracle_kv_append", "oracle_attend", "oracle_lse_combine"):
+            getattr(L, name).restype = ctypes.c_int
+        _lib = L
+    return _lib
+
+
+def num_threads() -> int:
+    return int(lib().oracle_num_threads())
+
+
+def _p(a: Optional[np.ndarray]):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _c(a, dtype) -> np.ndarray:
+    a = np.ascontiguousarray(a, dtype=dtype)
+    return a
+
+
+def _check(rc: int):
+    if rc != 0:
+        raise OracleError(_STATUS.get(rc, f"status {rc}"))
+
+
+def _pool_dims(pool: np.ndarray):
+    assert pool.dtype == np.uint16 and pool.ndim == 4 and pool.flags.c_contiguous
+    return pool.shape  # num_pages, Hkv, P, D
+
+
+def kv_append(k_pool: np.ndarray, v_pool: np.ndarray, page_table: np.ndarray, seq_lens: np.ndarray,
+              new_indptr: np.ndarray, k_new: np.ndarray, v_new: np.ndarray,
+              traj_ids: Optional[np.ndarray] = None) -> np.ndarray:
+    """In-place append into the uint16 pools (Sec. 6.1: each trajectory appends to its own
+    context).  seq_lens = lengths before.  Returns the lengths after (a new array)."""
+    num_pages, Hkv, P, D = _pool_dims(k_pool)
+    assert v_pool.shape == k_pool.shape and v_pool.dtype == np.uint16 and v_pool.flags.c_contiguous
+    page_table = _c(page_table, np.int32)
+    seq_lens = _c(seq_lens, np.int32)
+    new_indptr = _c(new_indptr, np.int32)
+    n_items = len(new_indptr) - 1
+    tid = None if traj_ids is None else _c(traj_ids, np.int32)
+    k_new = _c(k_new, np.uint16)
+    v_new = _c(v_new, np.uint16)
+    total_new = int(new_indptr[-1]) if n_items >= 0 else 0
+    assert k_new.size == total_new * Hkv * D and v_new.size == k_new.size
+    out = seq_lens.copy()
+    rc = lib().oracle_kv_append(
+        _p(k_pool), _p(v_pool), ctypes.c_int32(num_pages), ctypes.c_int32(P), ctypes.c_int32(Hkv), ctypes.c_int32(D),
+        _p(page_table), ctypes.c_int32(page_table.shape[1]), _p(seq_lens), ctypes.c_int32(len(seq_lens)),
+        _p(tid), _p(new_indptr), ctypes.c_int32(n_items), _p(k_new), _p(v_new), _p(out))
+    _check(rc)
+    return out
+
+
+def attend_rows(k_pool: np.ndarray, v_pool: np.ndarray, page_table: np.ndarray,
+                row_traj, row_count, q: np.ndarray, sm_scale: float, row_begin=None):
+    """out [n_rows][Hq][D] fp64 and lse [n_rows][Hq] fp64 for query rows that each see keys
+    row_begin[r] <= j < row_count[r] of trajectory row_traj[r]."""
+    num_pages, Hkv, P, D = _pool_dims(k_pool)
+    page_table = _c(page_table, np.int32)
+    row_traj = _c(row_traj, np.int32)
+    row_count = _c(row_count, np.int32)
+    rb = None if row_begin is None else _c(row_begin, np.int32)
+    q = _c(q, np.uint16)
+    n_rows = len(row_traj)
+    assert q.ndim == 3 and q.shape[0] == n_rows and q.shape[2] == D
+    Hq = q.shape[1]
+    out = np.empty((n_rows, Hq, D), dtype=np.float64)
+    lse = np.empty((n_rows, Hq), dtype=np.float64)
+    rc = lib().oracle_attend(
+        _p(k_pool), _p(v_pool), ctypes.c_int32(num_pages), ctypes.c_int32(P), ctypes.c_int32(Hkv), ctypes.c_int32(D),
+        _p(page_table), ctypes.c_int32(page_table.shape[1]), ctypes.c_int32(page_table.shape[0]),
+        ctypes.c_int64(n_rows), _p(row_traj), _p(rb), _p(row_count),
+        _p(q), ctypes.c_int32(Hq), ctypes.c_float(sm_scale), _p(out), _p(lse))
+    _check(rc)
+    return out, lse
+
+
+def decode_attn(k_pool, v_pool, page_table, seq_lens, q, sm_scale, traj_ids=None):
+    """One query token per item, seeing all seq_lens[t] keys of its trajectory (lengths AFTER the
+    append, so the token sees itself).  Sec. 3.1: the decode phase reads the whole context."""
+    seq_lens = _c(seq_lens, np.int32)
+    n = q.shape[0]
+    tid = np.arange(n, dtype=np.int32) if traj_ids is None else _c(traj_ids, np.int32)
+    return attend_rows(k_pool, v_pool, page_table, tid, seq_lens[tid], q, sm_scale)
+
+
+def chunk_row_counts(seq_lens, q_indptr, traj_ids=None):
+    """(row_traj, row_count): row j of an n-row chunk that ends trajectory t's L tokens sees
+    L - n + j + 1 keys (the whole prior context and the chunk causally)."""
+    seq_lens = _c(seq_lens, np.int32)
+    q_indptr = _c(q_indptr, np.int32)
+    n_items = len(q_indptr) - 1
+    tid = np.arange(n_items, dtype=np.int32) if traj_ids is None else _c(traj_ids, np.int32)
+    row_traj = np.empty(int(q_indptr[-1]), dtype=np.int32)
+    row_count = np.empty(int(q_indptr[-1]), dtype=np.int32)
+    for i in range(n_items):
+        a, b = int(q_indptr[i]), int(q_indptr[i + 1])
+        n = b - a
+        L = int(seq_lens[tid[i]])
+        if n > L:
+            raise OracleError("chunk longer than its trajectory")
+        row_traj[a:b] = tid[i]
+        row_count[a:b] = L - n + np.arange(n) + 1
+    return row_traj, row_count
+
+
+def obs_chunk_attn(k_pool, v_pool, page_table, seq_lens, q_indptr, q, sm_scale, traj_ids=None,
+                   rows: Optional[Sequence[int]] = None):
+    """Attention of newly arrived observation tokens (Sec. 2.1: many-turn tasks re-process a
+    growing history; with the prefix cached only the new tokens are computed).  `rows` selects a
+    subset of the chunk rows (indices into q) to evaluate."""
+    row_traj, row_count = chunk_row_counts(seq_lens, q_indptr, traj_ids)
+    if rows is not None:
+        rows = np.asarray(rows, dtype=np.int64)
+        return attend_rows(k_pool, v_pool, page_table, row_traj[rows], row_count[rows], q[rows], sm_scale)
+    return attend_rows(k_pool, v_pool, page_table, row_traj, row_count, q, sm_scale)
+
+
+def lse_combine(parts_out: np.ndarray, parts_lse: np.ndarray):
+    """Merge partial results over disjoint key ranges: parts_out [S][...][D], parts_lse [S][...]."""
+    parts_out = _c(parts_out, np.float64)
+    parts_lse = _c(parts_lse, np.float64)
+    S = parts_out.shape[0]
+    D = parts_out.shape[-1]
+    inner = parts_lse.shape[1:]
+    n = int(np.prod(inner)) if inner else 1
+    po = parts_out.reshape(S, n, D)
+    pl = parts_lse.reshape(S, n)
+    out = np.empty((n, D), dtype=np.float64)
+    lse = np.empty(n, dtype=np.float64)
+    for i in range(n):
+        a = np.ascontiguousarray(po[:, i, :])
+        b = np.ascontiguousarray(pl[:, i])
+        one = ctypes.c_double()
+        rc = lib().oracle_lse_combine(ctypes.c_int32(S), ctypes.c_int32(D), _p(a), _p(b),
+                                      out[i].ctypes.data_as(ctypes.c_void_p), ctypes.byref(one))
+        _check(rc)
+        lse[i] = one.value
+    return out.reshape(*inner, D), lse.reshape(inner)

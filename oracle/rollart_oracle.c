@@ -1,0 +1,180 @@
+/*
+ * CPU oracle for paged-KV rollout attention.  TEST INFRASTRUCTURE ONLY: the
+ * product (the CUDA library) never links, loads or calls anything in this file;
+ * only the tests, the smoke check and the bench's CPU-baseline leg do.
+ *
+ * What it computes.  The paper treats the rollout engine step as a black box
+ * ("a decode or prefill step for a batch of requests", Sec. 6.1, inference
+ * worker event loop) acting on trajectories whose context grows by one
+ * (observation, action) pair per turn (Sec. 6.1, EnvManager) and whose decode
+ * phase is bound by reading that whole context per generated token (Sec. 3.1).
+ * The paper prints no formula for the step; the operation has a plain
+ * definition, which is written out here and nothing more:
+ *
+ *   append : the r-th new row of trajectory t goes to logical position
+ *            pos = len_before[t] + r, i.e. physical page table[t][pos / P],
+ *            slot pos % P, for every kv head, as a bit copy.
+ *   attend : query row with c visible keys, q head hq, kv head h = hq / g:
+ *            s_j = scale * <q, k_j>, j in [j0, c);  m = max_j s_j;
+ *            w_j = exp(s_j - m);  Z = sum_j w_j;
+ *            out = sum_j w_j v_j / Z;   lse = m + ln Z.
+ *   combine: parts (out_s, lse_s) over disjoint key ranges merge as
+ *            M = max_s lse_s; a_s = exp(lse_s - M); out = sum a_s out_s / sum a_s;
+ *            lse = M + ln sum a_s.
+ *
+ * Everything floating point is fp64; bf16 inputs convert exactly.  No blocking,
+ * no online softmax, no reordering: two passes over the keys, in index order.
+ * Parity status: every function here is pinned by tests/test_oracle_pins.py
+ * (closed forms, invariants, an independent dense routine, brute force).
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+enum { ORACLE_OK = 0, ORACLE_BAD_ARG = 1, ORACLE_BAD_PAGE = 2, ORACLE_BAD_LENGTH = 3 };
+
+static double bf16_to_f64(uint16_t bits) {
+    uint32_t w = (uint32_t)bits << 16;
+    float f;
+    memcpy(&f, &w, sizeof f);
+    return (double)f;
+}
+
+int oracle_num_threads(void) {
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+/* Append.  seq_lens holds lengths BEFORE the call, indexed by trajectory; item i appends rows
+ * new_indptr[i]..new_indptr[i+1] of k_new/v_new ([total_new][Hkv][D]) to trajectory
+ * traj_ids[i] (identity when traj_ids is NULL).  seq_lens_out (nullable, indexed by
+ * trajectory) receives len + n for the trajectories named; others are left untouched. */
+int oracle_kv_append(uint16_t *k_pool, uint16_t *v_pool, int32_t num_pages, int32_t P, int32_t Hkv, int32_t D,
+                     const int32_t *page_table, int32_t max_pages, const int32_t *seq_lens, int32_t num_traj,
+                     const int32_t *traj_ids, const int32_t *new_indptr, int32_t n_items,
+                     const uint16_t *k_new, const uint16_t *v_new, int32_t *seq_lens_out) {
+    if (P <= 0 || Hkv <= 0 || D <= 0 || n_items < 0) return ORACLE_BAD_ARG;
+    for (int32_t i = 0; i < n_items; ++i) {
+        int32_t t = traj_ids ? traj_ids[i] : i;
+        if (t < 0 || t >= num_traj) return ORACLE_BAD_ARG;
+        int32_t n = new_indptr[i + 1] - new_indptr[i];
+        int32_t len = seq_lens[t];
+        if (n < 0 || len < 0) return ORACLE_BAD_LENGTH;
+        for (int32_t r = 0; r < n; ++r) {
+            int64_t pos = (int64_t)len + r;
+            int64_t lp = pos / P;
+            if (lp >= max_pages) return ORACLE_BAD_LENGTH;
+            int32_t pg = page_table[(int64_t)t * max_pages + lp];
+            if (pg < 0 || pg >= num_pages) return ORACLE_BAD_PAGE;
+            int64_t slot = pos % P;
+            int64_t row = (int64_t)new_indptr[i] + r;
+            for (int32_t h = 0; h < Hkv; ++h) {
+                int64_t dst = (((int64_t)pg * Hkv + h) * P + slot) * D;
+                int64_t src = (row * Hkv + h) * D;
+                memcpy(k_pool + dst, k_new + src, (size_t)D * sizeof(uint16_t));
+                memcpy(v_pool + dst, v_new + src, (size_t)D * sizeof(uint16_t));
+            }
+        }
+        if (seq_lens_out) seq_lens_out[t] = len + n;
+    }
+    return ORACLE_OK;
+}
+
+/* Attention of n_rows query rows.  Row r belongs to trajectory row_traj[r] and sees keys
+ * row_begin[r] <= j < row_count[r] of that trajectory (row_begin NULL = 0).  q is
+ * [n_rows][Hq][D] bf16; out is [n_rows][Hq][D] fp64, lse [n_rows][Hq] fp64 (natural log).
+ * An empty key range gives out = 0, lse = -inf. */
+int oracle_attend(const uint16_t *k_pool, const uint16_t *v_pool, int32_t num_pages, int32_t P, int32_t Hkv, int32_t D,
+                  const int32_t *page_table, int32_t max_pages, int32_t num_traj,
+                  int64_t n_rows, const int32_t *row_traj, const int32_t *row_begin, const int32_t *row_count,
+                  const uint16_t *q, int32_t Hq, float sm_scale, double *out, double *lse) {
+    if (P <= 0 || Hkv <= 0 || D <= 0 || Hq <= 0 || Hq % Hkv != 0 || n_rows < 0) return ORACLE_BAD_ARG;
+    const int32_t g = Hq / Hkv;
+    const double scale = (double)sm_scale;
+    int status = ORACLE_OK;
+    /* validate first, so the parallel region has nothing to report */
+    for (int64_t r = 0; r < n_rows; ++r) {
+        int32_t t = row_traj[r];
+        if (t < 0 || t >= num_traj) return ORACLE_BAD_ARG;
+        int32_t c = row_count[r], j0 = row_begin ? row_begin[r] : 0;
+        if (c < 0 || j0 < 0) return ORACLE_BAD_LENGTH;
+        if (c > 0 && (int64_t)(c - 1) / P >= max_pages) return ORACLE_BAD_LENGTH;
+        for (int64_t lp = j0 / P; c > j0 && lp * P < c; ++lp) {
+            int32_t pg = page_table[(int64_t)t * max_pages + lp];
+            if (pg < 0 || pg >= num_pages) return ORACLE_BAD_PAGE;
+        }
+    }
+    const int64_t n_work = n_rows * Hq;
+#pragma omp parallel
+    {
+        double *s = NULL;
+        size_t s_cap = 0;
+        double *qd = (double *)malloc((size_t)D * sizeof(double));
+        double *acc = (double *)malloc((size_t)D * sizeof(double));
+#pragma omp for schedule(dynamic, 1)
+        for (int64_t w = 0; w < n_work; ++w) {
+            int64_t r = w / Hq;
+            int32_t hq = (int32_t)(w % Hq);
+            int32_t h = hq / g;
+            int32_t t = row_traj[r];
+            int32_t c = row_count[r], j0 = row_begin ? row_begin[r] : 0;
+            double *o = out + (r * Hq + hq) * D;
+            for (int32_t d = 0; d < D; ++d) o[d] = 0.0;
+            if (c <= j0) { lse[r * Hq + hq] = -INFINITY; continue; }
+            size_t n = (size_t)(c - j0);
+            if (n > s_cap) { free(s); s = (double *)malloc(n * sizeof(double)); s_cap = n; }
+            const uint16_t *qp = q + (r * Hq + hq) * D;
+            for (int32_t d = 0; d < D; ++d) qd[d] = bf16_to_f64(qp[d]);
+            double m = -INFINITY;
+            for (int32_t j = j0; j < c; ++j) {
+                int32_t pg = page_table[(int64_t)t * max_pages + j / P];
+                const uint16_t *kp = k_pool + (((int64_t)pg * Hkv + h) * P + j % P) * D;
+                double dot = 0.0;
+                for (int32_t d = 0; d < D; ++d) dot += qd[d] * bf16_to_f64(kp[d]);
+                double sj = scale * dot;
+                s[j - j0] = sj;
+                if (sj > m) m = sj;
+            }
+            double Z = 0.0;
+            for (int32_t d = 0; d < D; ++d) acc[d] = 0.0;
+            for (int32_t j = j0; j < c; ++j) {
+                int32_t pg = page_table[(int64_t)t * max_pages + j / P];
+                const uint16_t *vp = v_pool + (((int64_t)pg * Hkv + h) * P + j % P) * D;
+                double wj = exp(s[j - j0] - m);
+                Z += wj;
+                for (int32_t d = 0; d < D; ++d) acc[d] += wj * bf16_to_f64(vp[d]);
+            }
+            for (int32_t d = 0; d < D; ++d) o[d] = acc[d] / Z;
+            lse[r * Hq + hq] = m + log(Z);
+        }
+        free(s); free(qd); free(acc);
+    }
+    return status;
+}
+
+/* Merge n_parts partial results of ONE (row, head): parts_out [n_parts][D], parts_lse [n_parts].
+ * Parts with lse = -inf (empty ranges) contribute nothing; all empty gives out = 0, lse = -inf. */
+int oracle_lse_combine(int32_t n_parts, int32_t D, const double *parts_out, const double *parts_lse,
+                       double *out, double *lse) {
+    if (n_parts < 0 || D <= 0) return ORACLE_BAD_ARG;
+    double M = -INFINITY;
+    for (int32_t s = 0; s < n_parts; ++s) if (parts_lse[s] > M) M = parts_lse[s];
+    for (int32_t d = 0; d < D; ++d) out[d] = 0.0;
+    if (M == -INFINITY) { *lse = -INFINITY; return ORACLE_OK; }
+    double A = 0.0;
+    for (int32_t s = 0; s < n_parts; ++s) {
+        double a = exp(parts_lse[s] - M);
+        A += a;
+        for (int32_t d = 0; d < D; ++d) out[d] += a * parts_out[(int64_t)s * D + d];
+    }
+    for (int32_t d = 0; d < D; ++d) out[d] /= A;
+    *lse = M + log(A);
+    return ORACLE_OK;
+}
