@@ -1,0 +1,173 @@
+/*
+ * rollart.h -- C ABI of the B200 (sm_100a) paged-KV rollout-attention library.
+ *
+ * Scope.  The rollout stage of agentic RL advances many independent trajectories; each one
+ * appends tokens to its own growing context (an observation from the environment, then the
+ * tokens of the next action) and the inference worker repeatedly "executes a decode or prefill
+ * step for a batch of requests" (paper Sec. 6.1, trajectory-level rollout; Sec. 3.1: decoding is
+ * memory-bandwidth bound, observation prefill compute bound).  This library is the attention
+ * part of that engine step over a paged bf16 KV cache:
+ *
+ *   rollart_kv_append       write the new tokens' K/V rows into the trajectories' pages
+ *   rollart_decode_attn     one new query token per trajectory attends to its whole context
+ *   rollart_obs_chunk_attn  a chunk of new observation tokens attends to the cached prefix and,
+ *                           causally, to itself
+ *
+ * The paper gives no formula for the step; the operation is standard scaled-dot-product softmax
+ * attention with grouped query heads, defined precisely below.
+ *
+ * Conventions.
+ *   - Plain C99 types only.  Pointers marked [device] are CUDA device pointers in the context's
+ *     device; [host] are ordinary host pointers.  `stream` is a cudaStream_t passed as void*
+ *     (NULL = the legacy default stream).
+ *   - The caller owns every buffer it passes.  The library owns only what rollart_create
+ *     allocates (one workspace, one status word, one pinned host word).
+ *   - kv_append / decode_attn / obs_chunk_attn enqueue work on `stream` and return without
+ *     synchronising and without allocating.  Errors the host can see (bad shapes, NULL pointers,
+ *     workspace too small) are returned at once and nothing is enqueued.  Errors only the device
+ *     can see (a page id outside the pool, a length that overruns its page-table row) make the
+ *     kernel skip that access and record a code in the device status word, which
+ *     rollart_check() fetches; a kernel never traps and every in-kernel wait is bounded.
+ *   - A context is not thread safe; use one per host thread / stream.
+ *   - head_dim must be 128; page_size 16, 32 or 64; num_q_heads a multiple of num_kv_heads with
+ *     at most 16 query heads per kv head.  Anything else returns ROLLART_ERR_UNSUPPORTED.
+ *
+ * Data layout.
+ *   pools       bf16 [num_pages][num_kv_heads][page_size][head_dim], K and V in separate pools,
+ *               both 16-byte aligned (a (page, head) tile is one contiguous block)
+ *   page_table  int32 [num_traj][max_pages_per_traj] row major; entry i of row t is the physical
+ *               page of logical page i.  Entries at or beyond ceil(len/page_size) are never read.
+ *   seq_lens    int32 [num_traj], tokens
+ *   Token at logical position pos of trajectory t, kv head h:
+ *               pool[page_table[t][pos / page_size]][h][pos % page_size][0..head_dim)
+ *   Query head hq reads kv head hq / (num_q_heads / num_kv_heads).
+ *   Slots that hold no live token (page tails, unowned pages) may contain anything, including
+ *   NaN and Inf bit patterns; results never depend on them.
+ */
+#ifndef ROLLART_H_
+#define ROLLART_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    ROLLART_OK = 0,
+    ROLLART_ERR_INVALID_ARG = 1, /* NULL pointer, negative count, overlapping in/out buffers   */
+    ROLLART_ERR_UNSUPPORTED = 2, /* head_dim, page_size or group size outside the supported set */
+    ROLLART_ERR_WORKSPACE = 3,   /* the context's workspace is too small for this call         */
+    ROLLART_ERR_CUDA = 4,        /* a CUDA runtime/driver call failed (see rollart_last_error) */
+    ROLLART_ERR_BOUNDS = 5,      /* device saw a page id / length / trajectory id out of range */
+    ROLLART_ERR_TIMEOUT = 6      /* a bounded in-kernel wait ran out                           */
+} rollart_status;
+
+typedef struct rollart_ctx rollart_ctx; /* opaque */
+
+typedef struct {
+    void *k_pool; /* [device] bf16 [num_pages][num_kv_heads][page_size][head_dim] */
+    void *v_pool; /* [device] same shape */
+    int32_t num_pages;
+    int32_t page_size;
+    int32_t num_kv_heads;
+    int32_t head_dim;
+} rollart_kv_pool;
+
+typedef struct {
+    const int32_t *page_table; /* [device] int32 [num_traj][max_pages_per_traj] */
+    int32_t max_pages_per_traj;
+    const int32_t *seq_lens; /* [device] int32 [num_traj] */
+    int32_t num_traj;
+} rollart_trajs;
+
+/* Bytes of workspace that calls with at most max_items items (trajectories per call),
+ * these head counts and contexts up to max_seq_len tokens need.  Pure host arithmetic. */
+size_t rollart_workspace_size(int32_t max_items, int32_t num_q_heads, int32_t num_kv_heads, int32_t max_seq_len);
+
+/* Creates a context on CUDA device `device` and allocates its workspace (workspace_bytes, may
+ * be 0 if only kv_append is used).  *out [host] receives the context.  The only call that
+ * allocates device memory; rollart_destroy frees it. */
+rollart_status rollart_create(rollart_ctx **out, int device, size_t workspace_bytes);
+rollart_status rollart_destroy(rollart_ctx *ctx);
+
+/*
+ * KV append (Sec. 6.1: every turn the trajectory's history grows by the observation and the
+ * generated action; the engine step writes the new tokens' K/V into the cache before attending).
+ *
+ *   trajs->seq_lens   lengths BEFORE the append.
+ *   traj_ids          [device] int32 [n_items], trajectory of item i; NULL = identity (item i is
+ *                     trajectory i).  A trajectory may appear at most once per call.
+ *   new_indptr        [device] int32 [n_items+1], item i appends rows new_indptr[i] ..
+ *                     new_indptr[i+1]-1 of k_new / v_new; new_indptr[0] = 0,
+ *                     new_indptr[n_items] = total_new (the host passes total_new as well).
+ *   k_new, v_new      [device] bf16 [total_new][num_kv_heads][head_dim], 16-byte aligned.
+ *   seq_lens_out      [device] int32 [num_traj] or NULL; entry traj_ids[i] receives len + n_i,
+ *                     other entries are left alone.  Must not overlap trajs->seq_lens.
+ *
+ * Row r of item i lands at logical position len + r.  The pages covering the new positions must
+ * already be present in the page table (page allocation is the caller's).  The copy is bit exact;
+ * no other byte of the pools changes.  Device-side errors (ROLLART_ERR_BOUNDS): trajectory id out
+ * of range, negative length, position beyond max_pages_per_traj * page_size, page id outside
+ * [0, num_pages): the offending row is skipped.
+ */
+rollart_status rollart_kv_append(rollart_ctx *ctx, const rollart_kv_pool *pool, const rollart_trajs *trajs,
+                                 const int32_t *traj_ids, const int32_t *new_indptr, int32_t n_items,
+                                 int32_t total_new, const void *k_new, const void *v_new, int32_t *seq_lens_out,
+                                 void *stream);
+
+/*
+ * Decode attention (Sec. 3.1: the decoding phase is bound by reading the whole context once per
+ * generated token).  For item i with trajectory t = traj_ids[i], L = seq_lens[t] (lengths AFTER
+ * the append: the query attends to its own K/V), query head hq, kv head h = hq / g:
+ *
+ *   s_j = sm_scale * <q[i][hq], K_t[j][h]>,  j = 0..L-1
+ *   out[i][hq] = sum_j softmax(s)_j * V_t[j][h]          (bf16, round to nearest even)
+ *   lse[i][hq] = log sum_j exp(s_j)                       (fp32, natural log; optional)
+ *
+ *   q, out            [device] bf16 [n_items][num_q_heads][head_dim], 16-byte aligned.
+ *   lse               [device] fp32 [n_items][num_q_heads] or NULL.
+ *   max_seq_len       [host value] an upper bound on every L of this call; sizes the schedule and
+ *                     the workspace check.  A longer trajectory is reported as ROLLART_ERR_BOUNDS.
+ *   L = 0 gives out = 0 and lse = -inf.
+ * Arithmetic: bf16 operands, fp32 scores, softmax and accumulation; softmax weights are rounded
+ * to bf16 before they multiply V.  The schedule (how contexts are split over thread blocks and
+ * merged with a log-sum-exp combine) is a fixed function of the lengths, so reruns are bit
+ * identical.
+ */
+rollart_status rollart_decode_attn(rollart_ctx *ctx, const rollart_kv_pool *pool, const rollart_trajs *trajs,
+                                   const int32_t *traj_ids, int32_t n_items, int32_t max_seq_len, const void *q,
+                                   int32_t num_q_heads, float sm_scale, void *out, float *lse, void *stream);
+
+/*
+ * Observation-chunk attention (Sec. 2.1 / 3.1: many-turn tasks keep re-entering generation with
+ * a longer history; with the prefix cached only the newly arrived observation tokens are
+ * computed, a dense compute-bound block).  Item i owns query rows q_indptr[i] .. q_indptr[i+1]-1;
+ * they are the LAST n_i tokens of trajectory t = traj_ids[i] (already appended; L = seq_lens[t]).
+ * Row j (0-based within the chunk) sees keys 0 .. L - n_i + j: the whole prior context, and the
+ * chunk causally including itself.  Same formula, layout of q/out/lse ([total_q][...]) and
+ * arithmetic as rollart_decode_attn; n_i = 1 is exactly a decode step.  n_i > L is a
+ * ROLLART_ERR_BOUNDS device error for that item.
+ */
+rollart_status rollart_obs_chunk_attn(rollart_ctx *ctx, const rollart_kv_pool *pool, const rollart_trajs *trajs,
+                                      const int32_t *traj_ids, const int32_t *q_indptr, int32_t n_items,
+                                      int32_t total_q, int32_t max_seq_len, const void *q, int32_t num_q_heads,
+                                      float sm_scale, void *out, float *lse, void *stream);
+
+/* Synchronises `stream`, then returns and clears the device status word: ROLLART_OK, or the
+ * first device-side error recorded since the last check (ROLLART_ERR_BOUNDS / _TIMEOUT), or
+ * ROLLART_ERR_CUDA if the stream itself reports an error. */
+rollart_status rollart_check(rollart_ctx *ctx, void *stream);
+
+/* [host] NUL-terminated description of the last non-OK status returned for this context; valid
+ * until the next call on it.  Never NULL. */
+const char *rollart_last_error(rollart_ctx *ctx);
+
+/* Number of kernels the library has launched through this context since it was created. */
+int64_t rollart_launch_count(rollart_ctx *ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ROLLART_H_ */

@@ -1,0 +1,94 @@
+// KV append: scatter the new tokens' K/V rows into the trajectories' pages (bit copy).
+//
+// One thread moves 16 bytes of a K row and the matching 16 bytes of the V row.  A (token, kv head)
+// row is 256 B, so 16 consecutive threads cover it and a warp covers two heads of one token;
+// both the source ([token][head][d]) and each destination row are contiguous, so every 16-lane
+// group reads and writes one fully used 256 B segment.  The kernel is bound by HBM traffic for
+// observation chunks and by launch latency for single decode tokens.
+#include "rollart_internal.cuh"
+
+namespace rollart {
+
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kVecPerRow = kRowBytes / 16;  // 16
+
+// item whose row range [indptr[i], indptr[i+1]) holds `row`; indptr is non-decreasing
+__device__ __forceinline__ int find_item(const int32_t *__restrict__ indptr, int n_items, int row) {
+    int lo = 0, hi = n_items;  // invariant: indptr[lo] <= row < indptr[hi]
+    while (hi - lo > 1) {
+        int mid = (lo + hi) >> 1;
+        if (__ldg(indptr + mid) <= row) lo = mid; else hi = mid;
+    }
+    return lo;
+}
+
+__global__ void __launch_bounds__(kThreads)
+kv_append_kernel(__nv_bfloat16 *__restrict__ k_pool, __nv_bfloat16 *__restrict__ v_pool, int num_pages, int page_size,
+                 int num_kv_heads, const int32_t *__restrict__ page_table, int max_pages,
+                 const int32_t *__restrict__ seq_lens, int num_traj, const int32_t *__restrict__ traj_ids,
+                 const int32_t *__restrict__ new_indptr, int n_items, int total_new,
+                 const uint4 *__restrict__ k_new, const uint4 *__restrict__ v_new, int32_t *__restrict__ seq_lens_out,
+                 DeviceStatus *status) {
+    const long long gid = static_cast<long long>(blockIdx.x) * kThreads + threadIdx.x;
+
+    // lengths after the append, one thread per item
+    if (seq_lens_out != nullptr && gid < n_items) {
+        const int i = static_cast<int>(gid);
+        const int t = traj_ids ? __ldg(traj_ids + i) : i;
+        if (t < 0 || t >= num_traj) {
+            report(status, ROLLART_ERR_BOUNDS, t, 1);
+        } else {
+            const int n = __ldg(new_indptr + i + 1) - __ldg(new_indptr + i);
+            seq_lens_out[t] = __ldg(seq_lens + t) + n;
+        }
+    }
+
+    const long long n_vec = static_cast<long long>(total_new) * num_kv_heads * kVecPerRow;
+    if (gid >= n_vec) return;
+    const int c = static_cast<int>(gid % kVecPerRow);
+    const long long rh = gid / kVecPerRow;
+    const int h = static_cast<int>(rh % num_kv_heads);
+    const int row = static_cast<int>(rh / num_kv_heads);
+
+    const int i = find_item(new_indptr, n_items, row);
+    const int t = traj_ids ? __ldg(traj_ids + i) : i;
+    if (t < 0 || t >= num_traj) { report(status, ROLLART_ERR_BOUNDS, t, 1); return; }
+    const int len = __ldg(seq_lens + t);
+    if (len < 0) { report(status, ROLLART_ERR_BOUNDS, len, 1); return; }
+    const long long pos = static_cast<long long>(len) + (row - __ldg(new_indptr + i));
+    const long long lp = pos / page_size;
+    if (lp >= max_pages) { report(status, ROLLART_ERR_BOUNDS, static_cast<int>(lp), 1); return; }
+    const int pg = __ldg(page_table + static_cast<long long>(t) * max_pages + lp);
+    if (pg < 0 || pg >= num_pages) { report(status, ROLLART_ERR_BOUNDS, pg, 1); return; }
+    const int slot = static_cast<int>(pos - lp * page_size);
+
+    const long long dst = ((static_cast<long long>(pg) * num_kv_heads + h) * page_size + slot) * kVecPerRow + c;
+    const uint4 kv = __ldg(k_new + gid);
+    const uint4 vv = __ldg(v_new + gid);
+    reinterpret_cast<uint4 *>(k_pool)[dst] = kv;
+    reinterpret_cast<uint4 *>(v_pool)[dst] = vv;
+}
+
+}  // namespace
+
+cudaError_t launch_kv_append(const rollart_kv_pool &pool, const rollart_trajs &trajs, const int32_t *traj_ids,
+                             const int32_t *new_indptr, int n_items, int total_new, const void *k_new,
+                             const void *v_new, int32_t *seq_lens_out, DeviceStatus *status, cudaStream_t stream,
+                             int64_t *launches) {
+    const long long n_vec = static_cast<long long>(total_new) * pool.num_kv_heads * kVecPerRow;
+    const long long n_thr = n_vec > n_items ? n_vec : n_items;
+    if (n_thr == 0) return cudaSuccess;
+    const long long blocks = (n_thr + kThreads - 1) / kThreads;
+    if (blocks > 0x7FFFFFFFLL) return cudaErrorInvalidValue;
+    kv_append_kernel<<<static_cast<unsigned>(blocks), kThreads, 0, stream>>>(
+        static_cast<__nv_bfloat16 *>(pool.k_pool), static_cast<__nv_bfloat16 *>(pool.v_pool), pool.num_pages,
+        pool.page_size, pool.num_kv_heads, trajs.page_table, trajs.max_pages_per_traj, trajs.seq_lens, trajs.num_traj,
+        traj_ids, new_indptr, n_items, total_new, static_cast<const uint4 *>(k_new), static_cast<const uint4 *>(v_new),
+        seq_lens_out, status);
+    ++*launches;
+    return cudaGetLastError();
+}
+
+}  // namespace rollart

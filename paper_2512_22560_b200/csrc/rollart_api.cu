@@ -1,0 +1,271 @@
+// C ABI of librollart: context, argument validation, dispatch to the kernel launchers.
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "rollart_internal.cuh"
+
+using namespace rollart;
+
+struct rollart_ctx {
+    int device;
+    int sm_count;
+    void *workspace;
+    size_t workspace_bytes;
+    DeviceStatus *d_status;
+    DeviceStatus *h_status;  // pinned
+    int64_t launches;
+    char err[320];
+};
+
+namespace {
+
+rollart_status fail(rollart_ctx *ctx, rollart_status st, const char *fmt, ...) {
+    if (ctx) {
+        va_list ap;
+        va_start(ap, fmt);
+        vsnprintf(ctx->err, sizeof ctx->err, fmt, ap);
+        va_end(ap);
+    }
+    return st;
+}
+
+rollart_status cuda_fail(rollart_ctx *ctx, cudaError_t e, const char *what) {
+    return fail(ctx, ROLLART_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
+}
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+rollart_status check_pool(rollart_ctx *ctx, const rollart_kv_pool *pool) {
+    if (!pool || !pool->k_pool || !pool->v_pool) return fail(ctx, ROLLART_ERR_INVALID_ARG, "pool or pool pointers NULL");
+    if (pool->num_pages <= 0 || pool->num_kv_heads <= 0)
+        return fail(ctx, ROLLART_ERR_INVALID_ARG, "num_pages and num_kv_heads must be positive");
+    if (pool->head_dim != kHeadDim) return fail(ctx, ROLLART_ERR_UNSUPPORTED, "head_dim %d (only 128)", pool->head_dim);
+    if (pool->page_size != 16 && pool->page_size != 32 && pool->page_size != 64)
+        return fail(ctx, ROLLART_ERR_UNSUPPORTED, "page_size %d (only 16, 32, 64)", pool->page_size);
+    if (!aligned16(pool->k_pool) || !aligned16(pool->v_pool))
+        return fail(ctx, ROLLART_ERR_INVALID_ARG, "pools must be 16-byte aligned");
+    return ROLLART_OK;
+}
+
+rollart_status check_trajs(rollart_ctx *ctx, const rollart_trajs *t) {
+    if (!t || !t->page_table || !t->seq_lens) return fail(ctx, ROLLART_ERR_INVALID_ARG, "trajs or its pointers NULL");
+    if (t->num_traj <= 0 || t->max_pages_per_traj <= 0)
+        return fail(ctx, ROLLART_ERR_INVALID_ARG, "num_traj and max_pages_per_traj must be positive");
+    return ROLLART_OK;
+}
+
+rollart_status check_heads(rollart_ctx *ctx, const rollart_kv_pool *pool, int num_q_heads) {
+    if (num_q_heads <= 0 || num_q_heads % pool->num_kv_heads != 0)
+        return fail(ctx, ROLLART_ERR_INVALID_ARG, "num_q_heads %d is not a positive multiple of num_kv_heads %d",
+                    num_q_heads, pool->num_kv_heads);
+    if (num_q_heads / pool->num_kv_heads > kMaxGroup)
+        return fail(ctx, ROLLART_ERR_UNSUPPORTED, "%d query heads per kv head (at most %d)",
+                    num_q_heads / pool->num_kv_heads, kMaxGroup);
+    return ROLLART_OK;
+}
+
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = true;
+    explicit DeviceGuard(int dev) {
+        if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+        if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+    }
+    ~DeviceGuard() {
+        int cur = -1;
+        if (prev >= 0 && cudaGetDevice(&cur) == cudaSuccess && cur != prev) cudaSetDevice(prev);
+    }
+};
+
+AttnCall make_call(rollart_ctx *ctx, const rollart_kv_pool *pool, const rollart_trajs *trajs, const int32_t *traj_ids,
+                   const int32_t *q_indptr, int n_items, int total_q, int max_seq_len, const void *q, int num_q_heads,
+                   float sm_scale, void *out, float *lse) {
+    AttnCall c;
+    c.pool = PoolView{static_cast<const __nv_bfloat16 *>(pool->k_pool), static_cast<const __nv_bfloat16 *>(pool->v_pool),
+                      pool->num_pages, pool->page_size, pool->num_kv_heads};
+    c.trajs = TrajView{trajs->page_table, trajs->seq_lens, trajs->max_pages_per_traj, trajs->num_traj};
+    c.traj_ids = traj_ids;
+    c.q_indptr = q_indptr;
+    c.n_items = n_items;
+    c.total_q = total_q;
+    c.max_seq_len = max_seq_len;
+    c.q = static_cast<const __nv_bfloat16 *>(q);
+    c.num_q_heads = num_q_heads;
+    c.sm_scale = sm_scale;
+    c.out = static_cast<__nv_bfloat16 *>(out);
+    c.lse = lse;
+    c.workspace = ctx->workspace;
+    c.workspace_bytes = ctx->workspace_bytes;
+    c.status = ctx->d_status;
+    c.sm_count = ctx->sm_count;
+    return c;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t rollart_workspace_size(int32_t max_items, int32_t num_q_heads, int32_t num_kv_heads, int32_t max_seq_len) {
+    if (max_items <= 0 || num_q_heads <= 0 || num_kv_heads <= 0 || max_seq_len < 0) return 0;
+    return decode_workspace_bytes(max_items, num_q_heads, num_kv_heads, max_seq_len, /*sm_count=*/0);
+}
+
+rollart_status rollart_create(rollart_ctx **out, int device, size_t workspace_bytes) {
+    if (!out) return ROLLART_ERR_INVALID_ARG;
+    *out = nullptr;
+    int n = 0;
+    if (cudaGetDeviceCount(&n) != cudaSuccess || device < 0 || device >= n) return ROLLART_ERR_CUDA;
+    DeviceGuard guard(device);
+    if (!guard.ok) return ROLLART_ERR_CUDA;
+    rollart_ctx *ctx = new (std::nothrow) rollart_ctx();
+    if (!ctx) return ROLLART_ERR_CUDA;
+    std::memset(ctx, 0, sizeof *ctx);
+    ctx->device = device;
+    cudaDeviceProp prop;
+    cudaError_t e = cudaGetDeviceProperties(&prop, device);
+    if (e == cudaSuccess && prop.major != 10) {
+        // the kernels are sm_100a binaries; refuse loudly rather than fail at the first launch
+        delete ctx;
+        return ROLLART_ERR_UNSUPPORTED;
+    }
+    if (e == cudaSuccess) ctx->sm_count = prop.multiProcessorCount;
+    if (e == cudaSuccess) e = cudaMalloc(&ctx->d_status, sizeof(DeviceStatus));
+    if (e == cudaSuccess) e = cudaMemset(ctx->d_status, 0, sizeof(DeviceStatus));
+    if (e == cudaSuccess) e = cudaMallocHost(&ctx->h_status, sizeof(DeviceStatus));
+    if (e == cudaSuccess && workspace_bytes) e = cudaMalloc(&ctx->workspace, workspace_bytes);
+    if (e == cudaSuccess && workspace_bytes) e = cudaMemset(ctx->workspace, 0, workspace_bytes);
+    if (e == cudaSuccess) e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        if (ctx->workspace) cudaFree(ctx->workspace);
+        if (ctx->d_status) cudaFree(ctx->d_status);
+        if (ctx->h_status) cudaFreeHost(ctx->h_status);
+        delete ctx;
+        return ROLLART_ERR_CUDA;
+    }
+    ctx->workspace_bytes = workspace_bytes;
+    std::snprintf(ctx->err, sizeof ctx->err, "ok");
+    *out = ctx;
+    return ROLLART_OK;
+}
+
+rollart_status rollart_destroy(rollart_ctx *ctx) {
+    if (!ctx) return ROLLART_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    cudaDeviceSynchronize();
+    if (ctx->workspace) cudaFree(ctx->workspace);
+    if (ctx->d_status) cudaFree(ctx->d_status);
+    if (ctx->h_status) cudaFreeHost(ctx->h_status);
+    delete ctx;
+    return ROLLART_OK;
+}
+
+rollart_status rollart_kv_append(rollart_ctx *ctx, const rollart_kv_pool *pool, const rollart_trajs *trajs,
+                                 const int32_t *traj_ids, const int32_t *new_indptr, int32_t n_items,
+                                 int32_t total_new, const void *k_new, const void *v_new, int32_t *seq_lens_out,
+                                 void *stream) {
+    if (!ctx) return ROLLART_ERR_INVALID_ARG;
+    rollart_status st;
+    if ((st = check_pool(ctx, pool)) != ROLLART_OK) return st;
+    if ((st = check_trajs(ctx, trajs)) != ROLLART_OK) return st;
+    if (n_items < 0 || total_new < 0) return fail(ctx, ROLLART_ERR_INVALID_ARG, "negative n_items or total_new");
+    if (n_items == 0) return ROLLART_OK;
+    if (!new_indptr) return fail(ctx, ROLLART_ERR_INVALID_ARG, "new_indptr NULL");
+    if (total_new > 0 && (!k_new || !v_new)) return fail(ctx, ROLLART_ERR_INVALID_ARG, "k_new or v_new NULL");
+    if (!aligned16(k_new) || !aligned16(v_new)) return fail(ctx, ROLLART_ERR_INVALID_ARG, "k_new/v_new must be 16-byte aligned");
+    if (seq_lens_out) {
+        const char *a = reinterpret_cast<const char *>(trajs->seq_lens);
+        const char *b = reinterpret_cast<const char *>(seq_lens_out);
+        size_t bytes = sizeof(int32_t) * static_cast<size_t>(trajs->num_traj);
+        if (a < b + bytes && b < a + bytes) return fail(ctx, ROLLART_ERR_INVALID_ARG, "seq_lens_out overlaps seq_lens");
+    }
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return fail(ctx, ROLLART_ERR_CUDA, "cannot select device %d", ctx->device);
+    cudaError_t e = launch_kv_append(*pool, *trajs, traj_ids, new_indptr, n_items, total_new, k_new, v_new, seq_lens_out,
+                                     ctx->d_status, static_cast<cudaStream_t>(stream), &ctx->launches);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "kv_append launch");
+    return ROLLART_OK;
+}
+
+static rollart_status attn_common(rollart_ctx *ctx, const rollart_kv_pool *pool, const rollart_trajs *trajs,
+                                  int32_t n_items, int32_t total_q, int32_t max_seq_len, const void *q,
+                                  int32_t num_q_heads, void *out) {
+    rollart_status st;
+    if ((st = check_pool(ctx, pool)) != ROLLART_OK) return st;
+    if ((st = check_trajs(ctx, trajs)) != ROLLART_OK) return st;
+    if ((st = check_heads(ctx, pool, num_q_heads)) != ROLLART_OK) return st;
+    if (n_items < 0 || total_q < 0 || max_seq_len < 0)
+        return fail(ctx, ROLLART_ERR_INVALID_ARG, "negative n_items, total_q or max_seq_len");
+    if (total_q > 0 && (!q || !out)) return fail(ctx, ROLLART_ERR_INVALID_ARG, "q or out NULL");
+    if (!aligned16(q) || !aligned16(out)) return fail(ctx, ROLLART_ERR_INVALID_ARG, "q/out must be 16-byte aligned");
+    if (static_cast<int64_t>(max_seq_len) > static_cast<int64_t>(trajs->max_pages_per_traj) * pool->page_size)
+        return fail(ctx, ROLLART_ERR_INVALID_ARG, "max_seq_len %d exceeds the page-table row capacity %lld", max_seq_len,
+                    static_cast<long long>(trajs->max_pages_per_traj) * pool->page_size);
+    return ROLLART_OK;
+}
+
+rollart_status rollart_decode_attn(rollart_ctx *ctx, const rollart_kv_pool *pool, const rollart_trajs *trajs,
+                                   const int32_t *traj_ids, int32_t n_items, int32_t max_seq_len, const void *q,
+                                   int32_t num_q_heads, float sm_scale, void *out, float *lse, void *stream) {
+    if (!ctx) return ROLLART_ERR_INVALID_ARG;
+    rollart_status st = attn_common(ctx, pool, trajs, n_items, n_items, max_seq_len, q, num_q_heads, out);
+    if (st != ROLLART_OK) return st;
+    if (n_items == 0) return ROLLART_OK;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return fail(ctx, ROLLART_ERR_CUDA, "cannot select device %d", ctx->device);
+    AttnCall c = make_call(ctx, pool, trajs, traj_ids, nullptr, n_items, n_items, max_seq_len, q, num_q_heads, sm_scale,
+                           out, lse);
+    bool too_small = false;
+    cudaError_t e = launch_decode_attn(c, static_cast<cudaStream_t>(stream), &ctx->launches, &too_small);
+    if (too_small)
+        return fail(ctx, ROLLART_ERR_WORKSPACE, "workspace of %zu bytes is too small (need %zu)", ctx->workspace_bytes,
+                    decode_workspace_bytes(n_items, num_q_heads, pool->num_kv_heads, max_seq_len, ctx->sm_count));
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "decode_attn launch");
+    return ROLLART_OK;
+}
+
+rollart_status rollart_obs_chunk_attn(rollart_ctx *ctx, const rollart_kv_pool *pool, const rollart_trajs *trajs,
+                                      const int32_t *traj_ids, const int32_t *q_indptr, int32_t n_items,
+                                      int32_t total_q, int32_t max_seq_len, const void *q, int32_t num_q_heads,
+                                      float sm_scale, void *out, float *lse, void *stream) {
+    if (!ctx) return ROLLART_ERR_INVALID_ARG;
+    rollart_status st = attn_common(ctx, pool, trajs, n_items, total_q, max_seq_len, q, num_q_heads, out);
+    if (st != ROLLART_OK) return st;
+    if (n_items == 0 || total_q == 0) return ROLLART_OK;
+    if (!q_indptr) return fail(ctx, ROLLART_ERR_INVALID_ARG, "q_indptr NULL");
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return fail(ctx, ROLLART_ERR_CUDA, "cannot select device %d", ctx->device);
+    AttnCall c = make_call(ctx, pool, trajs, traj_ids, q_indptr, n_items, total_q, max_seq_len, q, num_q_heads, sm_scale,
+                           out, lse);
+    bool too_small = false;
+    cudaError_t e = launch_chunk_attn(c, static_cast<cudaStream_t>(stream), &ctx->launches, &too_small);
+    if (too_small) return fail(ctx, ROLLART_ERR_WORKSPACE, "workspace of %zu bytes is too small", ctx->workspace_bytes);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "obs_chunk_attn launch");
+    return ROLLART_OK;
+}
+
+rollart_status rollart_check(rollart_ctx *ctx, void *stream) {
+    if (!ctx) return ROLLART_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return fail(ctx, ROLLART_ERR_CUDA, "cannot select device %d", ctx->device);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    cudaError_t e = cudaMemcpyAsync(ctx->h_status, ctx->d_status, sizeof(DeviceStatus), cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess) e = cudaMemsetAsync(ctx->d_status, 0, sizeof(DeviceStatus), s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "rollart_check");
+    const DeviceStatus hs = *ctx->h_status;
+    if (hs.code == 0) return ROLLART_OK;
+    static const char *const where[] = {"?", "kv_append", "decode_attn", "obs_chunk_attn", "combine"};
+    const char *w = (hs.where >= 0 && hs.where < 5) ? where[hs.where] : "?";
+    if (hs.code == ROLLART_ERR_TIMEOUT)
+        return fail(ctx, ROLLART_ERR_TIMEOUT, "%s: a bounded wait ran out (detail %d)", w, hs.detail);
+    return fail(ctx, static_cast<rollart_status>(hs.code), "%s: index out of range on the device (detail %d)", w, hs.detail);
+}
+
+const char *rollart_last_error(rollart_ctx *ctx) { return ctx ? ctx->err : "context is NULL"; }
+
+int64_t rollart_launch_count(rollart_ctx *ctx) { return ctx ? ctx->launches : 0; }
+
+}  // extern "C"

@@ -1,0 +1,74 @@
+// Internal declarations shared by the translation units of librollart (not part of the ABI).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "rollart.h"
+
+namespace rollart {
+
+constexpr int kHeadDim = 128;
+constexpr int kMaxGroup = 16;      // query heads per kv head
+constexpr int kRowBytes = kHeadDim * 2;
+
+// Device status word: 0 = ok, else the first rollart_status a kernel recorded.
+// status[1] carries a detail value (the offending index) for the error text.
+struct DeviceStatus {
+    int code;
+    int detail;
+    int where;
+    int pad;
+};
+
+__device__ __forceinline__ void report(DeviceStatus *st, int code, int detail, int where) {
+    if (atomicCAS(&st->code, 0, code) == 0) {
+        st->detail = detail;
+        st->where = where;
+    }
+}
+
+struct PoolView {
+    const __nv_bfloat16 *k;
+    const __nv_bfloat16 *v;
+    int num_pages, page_size, num_kv_heads;
+};
+
+struct TrajView {
+    const int32_t *page_table;
+    const int32_t *seq_lens;
+    int max_pages, num_traj;
+};
+
+// ---- launchers (each enqueues on `stream`, returns the cudaError of the launch, and adds the
+//      number of kernels it launched to *launches) ----
+cudaError_t launch_kv_append(const rollart_kv_pool &pool, const rollart_trajs &trajs, const int32_t *traj_ids,
+                             const int32_t *new_indptr, int n_items, int total_new, const void *k_new,
+                             const void *v_new, int32_t *seq_lens_out, DeviceStatus *status, cudaStream_t stream,
+                             int64_t *launches);
+
+struct AttnCall {
+    PoolView pool;
+    TrajView trajs;
+    const int32_t *traj_ids;  // nullable
+    const int32_t *q_indptr;  // NULL for decode (one row per item)
+    int n_items;
+    int total_q;              // rows of q/out
+    int max_seq_len;
+    const __nv_bfloat16 *q;
+    int num_q_heads;
+    float sm_scale;
+    __nv_bfloat16 *out;
+    float *lse;               // nullable
+    void *workspace;
+    size_t workspace_bytes;
+    DeviceStatus *status;
+    int sm_count;
+};
+
+size_t decode_workspace_bytes(int max_items, int num_q_heads, int num_kv_heads, int max_seq_len, int sm_count);
+// returns cudaSuccess, or cudaErrorInvalidValue with *too_small = true if the workspace cannot hold the call
+cudaError_t launch_decode_attn(const AttnCall &c, cudaStream_t stream, int64_t *launches, bool *too_small);
+cudaError_t launch_chunk_attn(const AttnCall &c, cudaStream_t stream, int64_t *launches, bool *too_small);
+
+}  // namespace rollart

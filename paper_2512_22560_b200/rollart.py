@@ -1,0 +1,213 @@
+"""Thin ctypes binding of librollart.so: argument marshalling only.
+
+Every step of the path runs in the library's CUDA kernels; PyTorch supplies device memory and
+streams.  There is no CPU or eager fallback: if the shared library is missing or cannot be
+loaded, importing the entry points raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "librollart.so")
+
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_BOUNDS, ERR_TIMEOUT = range(7)
+_NAMES = ["OK", "ERR_INVALID_ARG", "ERR_UNSUPPORTED", "ERR_WORKSPACE", "ERR_CUDA", "ERR_BOUNDS", "ERR_TIMEOUT"]
+
+EXPORTS = (
+    "rollart_workspace_size", "rollart_create", "rollart_destroy", "rollart_kv_append", "rollart_decode_attn",
+    "rollart_obs_chunk_attn", "rollart_check", "rollart_last_error", "rollart_launch_count",
+)
+
+
+class RollartError(RuntimeError):
+    def __init__(self, status: int, message: str):
+        super().__init__(f"rollart {_NAMES[status] if 0 <= status < len(_NAMES) else status}: {message}")
+        self.status = status
+
+
+class _KVPool(ctypes.Structure):
+    _fields_ = [("k_pool", ctypes.c_void_p), ("v_pool", ctypes.c_void_p), ("num_pages", ctypes.c_int32),
+                ("page_size", ctypes.c_int32), ("num_kv_heads", ctypes.c_int32), ("head_dim", ctypes.c_int32)]
+
+
+class _Trajs(ctypes.Structure):
+    _fields_ = [("page_table", ctypes.c_void_p), ("max_pages_per_traj", ctypes.c_int32),
+                ("seq_lens", ctypes.c_void_p), ("num_traj", ctypes.c_int32)]
+
+
+_lib = None
+
+
+def load_library() -> ctypes.CDLL:
+    """Loads librollart.so from the package directory; raises if it has not been built."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2512_22560_b200.build` "
+                          "(there is no fallback path)")
+    L = ctypes.CDLL(LIB_PATH)
+    vp, i32, i64, f32 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_float
+    L.rollart_workspace_size.restype = ctypes.c_size_t
+    L.rollart_workspace_size.argtypes = [i32, i32, i32, i32]
+    L.rollart_create.restype = ctypes.c_int
+    L.rollart_create.argtypes = [ctypes.POINTER(vp), ctypes.c_int, ctypes.c_size_t]
+    L.rollart_destroy.restype = ctypes.c_int
+    L.rollart_destroy.argtypes = [vp]
+    L.rollart_kv_append.restype = ctypes.c_int
+    L.rollart_kv_append.argtypes = [vp, ctypes.POINTER(_KVPool), ctypes.POINTER(_Trajs), vp, vp, i32, i32, vp, vp, vp, vp]
+    L.rollart_decode_attn.restype = ctypes.c_int
+    L.rollart_decode_attn.argtypes = [vp, ctypes.POINTER(_KVPool), ctypes.POINTER(_Trajs), vp, i32, i32, vp, i32, f32,
+                                      vp, vp, vp]
+    L.rollart_obs_chunk_attn.restype = ctypes.c_int
+    L.rollart_obs_chunk_attn.argtypes = [vp, ctypes.POINTER(_KVPool), ctypes.POINTER(_Trajs), vp, vp, i32, i32, i32, vp,
+                                         i32, f32, vp, vp, vp]
+    L.rollart_check.restype = ctypes.c_int
+    L.rollart_check.argtypes = [vp, vp]
+    L.rollart_last_error.restype = ctypes.c_char_p
+    L.rollart_last_error.argtypes = [vp]
+    L.rollart_launch_count.restype = i64
+    L.rollart_launch_count.argtypes = [vp]
+    _lib = L
+    return L
+
+
+def workspace_size(max_items: int, num_q_heads: int, num_kv_heads: int, max_seq_len: int) -> int:
+    return int(load_library().rollart_workspace_size(max_items, num_q_heads, num_kv_heads, max_seq_len))
+
+
+def _ptr(t: Optional[torch.Tensor], dtype=None, device=None) -> Optional[int]:
+    if t is None:
+        return None
+    if not t.is_cuda or not t.is_contiguous():
+        raise ValueError("expected a contiguous CUDA tensor")
+    if dtype is not None and t.dtype != dtype:
+        raise ValueError(f"expected dtype {dtype}, got {t.dtype}")
+    if device is not None and t.device.index != device:
+        raise ValueError(f"tensor on cuda:{t.device.index}, context on cuda:{device}")
+    return t.data_ptr()
+
+
+class Context:
+    """Owns one rollart_ctx (workspace + device status word) on one CUDA device."""
+
+    def __init__(self, device: int = 0, workspace_bytes: int = 0):
+        self._lib = load_library()
+        self.device = int(device)
+        self._h = ctypes.c_void_p()
+        st = self._lib.rollart_create(ctypes.byref(self._h), self.device, workspace_bytes)
+        if st != OK:
+            self._h = ctypes.c_void_p()
+            raise RollartError(st, f"rollart_create(device={device}, workspace_bytes={workspace_bytes}) failed")
+        self.workspace_bytes = int(workspace_bytes)
+
+    def close(self):
+        if getattr(self, "_h", None) is not None and self._h.value:
+            self._lib.rollart_destroy(self._h)
+            self._h = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # -- helpers ---------------------------------------------------------------------------------
+    def _raise(self, st: int):
+        raise RollartError(st, self._lib.rollart_last_error(self._h).decode())
+
+    def _stream(self, stream) -> int:
+        if stream is None:
+            stream = torch.cuda.current_stream(self.device)
+        return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
+
+    def _pool(self, k_pool: torch.Tensor, v_pool: torch.Tensor) -> _KVPool:
+        if k_pool.dim() != 4 or k_pool.shape != v_pool.shape:
+            raise ValueError("pools must be [num_pages][num_kv_heads][page_size][head_dim] with equal shapes")
+        n, h, p, d = k_pool.shape
+        return _KVPool(_ptr(k_pool, torch.bfloat16, self.device), _ptr(v_pool, torch.bfloat16, self.device), n, p, h, d)
+
+    def _trajs(self, page_table: torch.Tensor, seq_lens: torch.Tensor) -> _Trajs:
+        if page_table.dim() != 2 or seq_lens.dim() != 1 or page_table.shape[0] != seq_lens.shape[0]:
+            raise ValueError("page_table must be [num_traj][max_pages], seq_lens [num_traj]")
+        return _Trajs(_ptr(page_table, torch.int32, self.device), page_table.shape[1],
+                      _ptr(seq_lens, torch.int32, self.device), page_table.shape[0])
+
+    # -- the three calls ---------------------------------------------------------------------------
+    def kv_append(self, k_pool, v_pool, page_table, seq_lens, new_indptr, k_new, v_new, traj_ids=None,
+                  seq_lens_out=None, stream=None) -> None:
+        pool = self._pool(k_pool, v_pool)
+        trajs = self._trajs(page_table, seq_lens)
+        n_items = new_indptr.shape[0] - 1
+        total_new = k_new.shape[0]
+        if k_new.shape != v_new.shape or tuple(k_new.shape[1:]) != (pool.num_kv_heads, pool.head_dim):
+            raise ValueError("k_new/v_new must be [total_new][num_kv_heads][head_dim]")
+        if traj_ids is not None and traj_ids.shape[0] != n_items:
+            raise ValueError("traj_ids must have one entry per item")
+        if seq_lens_out is not None and seq_lens_out.shape != seq_lens.shape:
+            raise ValueError("seq_lens_out must have the shape of seq_lens")
+        st = self._lib.rollart_kv_append(
+            self._h, ctypes.byref(pool), ctypes.byref(trajs), _ptr(traj_ids, torch.int32, self.device),
+            _ptr(new_indptr, torch.int32, self.device), n_items, total_new, _ptr(k_new, torch.bfloat16, self.device),
+            _ptr(v_new, torch.bfloat16, self.device), _ptr(seq_lens_out, torch.int32, self.device), self._stream(stream))
+        if st != OK:
+            self._raise(st)
+
+    def decode_attn(self, k_pool, v_pool, page_table, seq_lens, q, sm_scale, max_seq_len, out, lse=None,
+                    traj_ids=None, stream=None) -> None:
+        pool = self._pool(k_pool, v_pool)
+        trajs = self._trajs(page_table, seq_lens)
+        if q.dim() != 3 or q.shape != out.shape:
+            raise ValueError("q and out must be [n_items][num_q_heads][head_dim]")
+        n_items, hq, _ = q.shape
+        if traj_ids is not None and traj_ids.shape[0] != n_items:
+            raise ValueError("traj_ids must have one entry per item")
+        if lse is not None and tuple(lse.shape) != (n_items, hq):
+            raise ValueError("lse must be [n_items][num_q_heads]")
+        st = self._lib.rollart_decode_attn(
+            self._h, ctypes.byref(pool), ctypes.byref(trajs), _ptr(traj_ids, torch.int32, self.device), n_items,
+            int(max_seq_len), _ptr(q, torch.bfloat16, self.device), hq, float(sm_scale),
+            _ptr(out, torch.bfloat16, self.device), _ptr(lse, torch.float32, self.device), self._stream(stream))
+        if st != OK:
+            self._raise(st)
+
+    def obs_chunk_attn(self, k_pool, v_pool, page_table, seq_lens, q_indptr, q, sm_scale, max_seq_len, out, lse=None,
+                       traj_ids=None, stream=None) -> None:
+        pool = self._pool(k_pool, v_pool)
+        trajs = self._trajs(page_table, seq_lens)
+        if q.dim() != 3 or q.shape != out.shape:
+            raise ValueError("q and out must be [total_q][num_q_heads][head_dim]")
+        total_q, hq, _ = q.shape
+        n_items = q_indptr.shape[0] - 1
+        if traj_ids is not None and traj_ids.shape[0] != n_items:
+            raise ValueError("traj_ids must have one entry per item")
+        if lse is not None and tuple(lse.shape) != (total_q, hq):
+            raise ValueError("lse must be [total_q][num_q_heads]")
+        st = self._lib.rollart_obs_chunk_attn(
+            self._h, ctypes.byref(pool), ctypes.byref(trajs), _ptr(traj_ids, torch.int32, self.device),
+            _ptr(q_indptr, torch.int32, self.device), n_items, total_q, int(max_seq_len),
+            _ptr(q, torch.bfloat16, self.device), hq, float(sm_scale), _ptr(out, torch.bfloat16, self.device),
+            _ptr(lse, torch.float32, self.device), self._stream(stream))
+        if st != OK:
+            self._raise(st)
+
+    def check(self, stream=None) -> None:
+        """Synchronises the stream and raises if a kernel recorded a device-side error."""
+        st = self._lib.rollart_check(self._h, self._stream(stream))
+        if st != OK:
+            self._raise(st)
+
+    def status(self, stream=None) -> int:
+        return int(self._lib.rollart_check(self._h, self._stream(stream)))
+
+    def last_error(self) -> str:
+        return self._lib.rollart_last_error(self._h).decode()
+
+    @property
+    def launch_count(self) -> int:
+        return int(self._lib.rollart_launch_count(self._h))

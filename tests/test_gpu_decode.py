@@ -1,0 +1,156 @@
+"""Decode attention on the GPU vs the fp64 oracle (|err| <= 1e-2 + 2e-2 |ref|), through the C ABI."""
+import dataclasses
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from harness import (DeviceBatch, assert_attn_close, assert_lse_close, dev_i32, make_ctx, oracle_append)
+from paper_2512_22560_b200 import rollart
+from paper_2512_22560_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+
+def run_decode_case(batch, device, poison=True, with_lse=True, max_seq_len=None):
+    """append + decode on the GPU and in the oracle for every decode trajectory of `batch`."""
+    spec = batch.spec
+    if poison:
+        W.poison_dead_slots(batch, batch.seq_lens_before)
+    ids = batch.decode_ids
+    rows = batch.decode_rows()
+    msl = int(batch.seq_lens_after.max()) if max_seq_len is None else max_seq_len
+    ctx = make_ctx(spec, len(ids), msl)
+    db = DeviceBatch(batch, device)
+    db.append(ctx)
+    q = db.q_new[torch.from_numpy(rows).to(device)].contiguous()
+    out = torch.full_like(q, float("nan"))
+    lse = torch.full((len(ids), spec.num_q_heads), float("nan"), device=device) if with_lse else None
+    ctx.decode_attn(db.k_pool, db.v_pool, db.page_table, db.lens_after, q, spec.sm_scale, msl, out, lse=lse,
+                    traj_ids=dev_i32(ids, device))
+    ctx.check()
+    kp, vp, after = oracle_append(batch)
+    ref_o, ref_l = oracle.decode_attn(kp, vp, batch.page_table, after, W.bf16_to_u16(batch.q_new[rows]), spec.sm_scale,
+                                      traj_ids=ids)
+    st = assert_attn_close(out, ref_o, spec.name)
+    if with_lse:
+        assert_lse_close(lse, ref_l, spec.name)
+    ctx.close()
+    return out, st
+
+
+def test_cfg0_tiny_decode_full(cuda_device):
+    run_decode_case(W.make_batch(W.CONFIGS[0]), cuda_device)
+
+
+@pytest.mark.parametrize("i,T,div", [(1, 16, 4), (2, 12, 16), (3, 4, 16), (4, 10, 8)])
+def test_shrunk_configs(cuda_device, i, T, div):
+    run_decode_case(W.make_batch(W.shrink(W.CONFIGS[i], T, div, 16), seed=200 + i), cuda_device)
+
+
+@pytest.mark.parametrize("P", [16, 32, 64])
+@pytest.mark.parametrize("hq,hkv", [(1, 1), (4, 2), (6, 2), (7, 1), (16, 2), (16, 1), (5, 5)])
+def test_edge_lengths_groups_and_page_sizes(cuda_device, P, hq, hkv):
+    lens = [0, 1, 2, P - 2, P - 1, P, 62, 63, 64, 65, 127, 128, 129, 191, 193, 255, 257, 700]
+    spec = dataclasses.replace(W.CONFIGS[0], page_size=P, num_traj=len(lens), num_q_heads=hq, num_kv_heads=hkv,
+                               name=f"edge_p{P}_{hq}_{hkv}")
+    batch = W.make_layout(spec, seed=31)
+    batch.seq_lens_before = np.array(lens, np.int32)
+    pages = (batch.seq_lens_before + 1 + P - 1) // P
+    batch.page_table, batch.num_pages = W.build_page_table(pages.astype(np.int64), 0.3, np.random.default_rng(8))
+    W.fill_tensors(batch)
+    run_decode_case(batch, cuda_device)
+
+
+def test_zero_length_trajectory_gives_zero_and_minus_inf(cuda_device):
+    spec = dataclasses.replace(W.CONFIGS[0], num_traj=3, name="zero")
+    batch = W.make_batch(spec, seed=4)
+    db = DeviceBatch(batch, cuda_device)
+    ctx = make_ctx(spec, 3, 600)
+    lens = dev_i32([0, 5, 0], cuda_device)
+    q = db.q_new[:3].contiguous()
+    out = torch.full_like(q, float("nan"))
+    lse = torch.full((3, spec.num_q_heads), float("nan"), device=cuda_device)
+    ctx.decode_attn(db.k_pool, db.v_pool, db.page_table, lens, q, 0.1, 600, out, lse=lse)
+    ctx.check()
+    assert torch.all(out[0] == 0) and torch.all(out[2] == 0)
+    assert torch.all(torch.isneginf(lse[0])) and torch.all(torch.isneginf(lse[2]))
+    assert torch.all(torch.isfinite(out[1])) and torch.all(torch.isfinite(lse[1]))
+
+
+def test_needles_give_order_one_outputs(cuda_device):
+    spec = W.shrink(W.CONFIGS[2], 6, 8)
+    batch = W.make_batch(spec, seed=77)
+    P = spec.page_size
+    pos = {}
+    for t in range(spec.num_traj):
+        L = int(batch.seq_lens_before[t])
+        pos[t] = sorted({0, L - 1, min(L - 1, P - 1), (L // P) * P if L % P else L - P, L // 2, min(L - 1, 64), L})
+    W.plant_needles(batch, pos)      # position L is the appended token itself
+    out, st = run_decode_case(batch, cuda_device)
+    assert st["rms_ref"] > 0.2
+
+
+def test_rerun_is_bit_identical_and_schedule_change_stays_close(cuda_device):
+    batch = W.make_batch(W.shrink(W.CONFIGS[3], 3, 8), seed=5)
+    a, _ = run_decode_case(batch, cuda_device, poison=False)
+    batch2 = W.make_batch(W.shrink(W.CONFIGS[3], 3, 8), seed=5)
+    b, _ = run_decode_case(batch2, cuda_device, poison=False)
+    assert torch.equal(a.view(torch.int16), b.view(torch.int16))
+    # a different host bound changes how contexts are split; results stay within a few bf16 ulps
+    batch3 = W.make_batch(W.shrink(W.CONFIGS[3], 3, 8), seed=5)
+    c, _ = run_decode_case(batch3, cuda_device, poison=False, max_seq_len=5 * int(batch.seq_lens_after.max()))
+    assert torch.allclose(a.float(), c.float(), atol=2e-3, rtol=2e-2)
+
+
+def test_shared_prefix_pages(cuda_device):
+    spec = dataclasses.replace(W.CONFIGS[0], num_traj=2, name="shared")
+    batch = W.make_batch(spec, seed=6)
+    batch.seq_lens_before[:] = [100, 90]
+    batch.page_table[1, :4] = batch.page_table[0, :4]          # 64 shared prefix tokens
+    run_decode_case(batch, cuda_device, poison=False)
+
+
+def test_device_side_errors(cuda_device):
+    batch = W.make_batch(W.shrink(W.CONFIGS[0], 4, 2), seed=13)
+    spec = batch.spec
+    db = DeviceBatch(batch, cuda_device)
+    ctx = make_ctx(spec, 4, 400)
+    db.append(ctx)
+    q = db.q_new.contiguous()
+    out = torch.zeros_like(q)
+    table = db.page_table.clone()
+    table[1, 0] = -3
+    ctx.decode_attn(db.k_pool, db.v_pool, table, db.lens_after, q, 0.1, 400, out)
+    assert ctx.status() == rollart.ERR_BOUNDS and "decode_attn" in ctx.last_error()
+    # a trajectory longer than the host bound is reported too
+    ctx.decode_attn(db.k_pool, db.v_pool, db.page_table, db.lens_after, q, 0.1, 16, out)
+    assert ctx.status() == rollart.ERR_BOUNDS
+    # and the context still computes correctly afterwards
+    ctx.decode_attn(db.k_pool, db.v_pool, db.page_table, db.lens_after, q, spec.sm_scale, 400, out)
+    ctx.check()
+    kp, vp, after = oracle_append(batch)
+    ref, _ = oracle.decode_attn(kp, vp, batch.page_table, after, W.bf16_to_u16(batch.q_new), spec.sm_scale)
+    assert_attn_close(out, ref)
+
+
+def test_host_side_validation(cuda_device):
+    batch = W.make_batch(W.shrink(W.CONFIGS[3], 2, 16), seed=14)
+    spec = batch.spec
+    db = DeviceBatch(batch, cuda_device)
+    q = db.q_new.contiguous()
+    out = torch.zeros_like(q)
+    small = rollart.Context(0, 1024)
+    with pytest.raises(rollart.RollartError) as e:
+        small.decode_attn(db.k_pool, db.v_pool, db.page_table, db.lens_before, q, 0.1, 8000, out)
+    assert e.value.status == rollart.ERR_WORKSPACE
+    ctx = make_ctx(spec, 2, 8000)
+    with pytest.raises(rollart.RollartError) as e:       # 64 q heads over 4 kv heads is fine, 3 kv heads is not
+        ctx.decode_attn(db.k_pool[:, :3].contiguous(), db.v_pool[:, :3].contiguous(), db.page_table, db.lens_before, q,
+                        0.1, 8000, out)
+    assert e.value.status == rollart.ERR_INVALID_ARG
+    with pytest.raises(rollart.RollartError) as e:       # bound larger than a page-table row can hold
+        ctx.decode_attn(db.k_pool, db.v_pool, db.page_table, db.lens_before, q, 0.1, 10 ** 7, out)
+    assert e.value.status == rollart.ERR_INVALID_ARG
