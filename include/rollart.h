@@ -129,7 +129,8 @@ rollart_status rollart_kv_append(rollart_ctx *ctx, const rollart_kv_pool *pool, 
  *   q, out            [device] bf16 [n_items][num_q_heads][head_dim], 16-byte aligned.
  *   lse               [device] fp32 [n_items][num_q_heads] or NULL.
  *   max_seq_len       [host value] an upper bound on every L of this call; sizes the schedule and
- *                     the workspace check.  A longer trajectory is reported as ROLLART_ERR_BOUNDS.
+ *                     the workspace check (values above max_pages_per_traj * page_size are
+ *                     clamped to it).  A longer trajectory is reported as ROLLART_ERR_BOUNDS.
  *   L = 0 gives out = 0 and lse = -inf.
  * Arithmetic: bf16 operands, fp32 scores, softmax and accumulation; softmax weights are rounded
  * to bf16 before they multiply V.  The schedule (how contexts are split over thread blocks and

@@ -59,7 +59,7 @@ attn_rows_kernel(PoolView pool, TrajView trajs, const int32_t *__restrict__ traj
         if (threadIdx.x == 0) report(status, ROLLART_ERR_BOUNDS, t, where);
     } else {
         const int L = __ldg(trajs.seq_lens + t);
-        if (L < 0 || L > max_seq_len || n_rows > L) {
+        if (L < 0 || L > max_seq_len || (q_indptr != nullptr && n_rows > L)) {
             bad = true;
             if (threadIdx.x == 0) report(status, ROLLART_ERR_BOUNDS, L, where);
         } else {

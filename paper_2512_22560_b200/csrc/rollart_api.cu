@@ -189,6 +189,12 @@ rollart_status rollart_kv_append(rollart_ctx *ctx, const rollart_kv_pool *pool, 
     return ROLLART_OK;
 }
 
+// max_seq_len is only an upper bound: a page-table row cannot hold more than this anyway
+static int32_t clamp_bound(const rollart_kv_pool *pool, const rollart_trajs *trajs, int32_t max_seq_len) {
+    const int64_t cap = static_cast<int64_t>(trajs->max_pages_per_traj) * pool->page_size;
+    return static_cast<int64_t>(max_seq_len) > cap ? static_cast<int32_t>(cap > 0x7FFFFFFF ? 0x7FFFFFFF : cap) : max_seq_len;
+}
+
 static rollart_status attn_common(rollart_ctx *ctx, const rollart_kv_pool *pool, const rollart_trajs *trajs,
                                   int32_t n_items, int32_t total_q, int32_t max_seq_len, const void *q,
                                   int32_t num_q_heads, void *out) {
@@ -200,9 +206,6 @@ static rollart_status attn_common(rollart_ctx *ctx, const rollart_kv_pool *pool,
         return fail(ctx, ROLLART_ERR_INVALID_ARG, "negative n_items, total_q or max_seq_len");
     if (total_q > 0 && (!q || !out)) return fail(ctx, ROLLART_ERR_INVALID_ARG, "q or out NULL");
     if (!aligned16(q) || !aligned16(out)) return fail(ctx, ROLLART_ERR_INVALID_ARG, "q/out must be 16-byte aligned");
-    if (static_cast<int64_t>(max_seq_len) > static_cast<int64_t>(trajs->max_pages_per_traj) * pool->page_size)
-        return fail(ctx, ROLLART_ERR_INVALID_ARG, "max_seq_len %d exceeds the page-table row capacity %lld", max_seq_len,
-                    static_cast<long long>(trajs->max_pages_per_traj) * pool->page_size);
     return ROLLART_OK;
 }
 
@@ -213,6 +216,7 @@ rollart_status rollart_decode_attn(rollart_ctx *ctx, const rollart_kv_pool *pool
     rollart_status st = attn_common(ctx, pool, trajs, n_items, n_items, max_seq_len, q, num_q_heads, out);
     if (st != ROLLART_OK) return st;
     if (n_items == 0) return ROLLART_OK;
+    max_seq_len = clamp_bound(pool, trajs, max_seq_len);
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return fail(ctx, ROLLART_ERR_CUDA, "cannot select device %d", ctx->device);
     AttnCall c = make_call(ctx, pool, trajs, traj_ids, nullptr, n_items, n_items, max_seq_len, q, num_q_heads, sm_scale,
@@ -235,6 +239,7 @@ rollart_status rollart_obs_chunk_attn(rollart_ctx *ctx, const rollart_kv_pool *p
     if (st != ROLLART_OK) return st;
     if (n_items == 0 || total_q == 0) return ROLLART_OK;
     if (!q_indptr) return fail(ctx, ROLLART_ERR_INVALID_ARG, "q_indptr NULL");
+    max_seq_len = clamp_bound(pool, trajs, max_seq_len);
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return fail(ctx, ROLLART_ERR_CUDA, "cannot select device %d", ctx->device);
     AttnCall c = make_call(ctx, pool, trajs, traj_ids, q_indptr, n_items, total_q, max_seq_len, q, num_q_heads, sm_scale,

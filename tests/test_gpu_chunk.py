@@ -89,9 +89,9 @@ def test_chunk_equals_sequential_append_and_decode_on_gpu(cuda_device):
 def test_chunk_longer_than_trajectory_is_a_device_error(cuda_device):
     batch = W.make_batch(W.shrink(W.CONFIGS[0], 2, 4), seed=44)
     db = DeviceBatch(batch, cuda_device)
-    ctx = make_ctx(batch.spec, 2, 300)
+    ctx = make_ctx(batch.spec, 2, 100)
     q = torch.zeros(40, batch.spec.num_q_heads, 128, dtype=torch.bfloat16, device=cuda_device)
     out = torch.zeros_like(q)
     lens = dev_i32([10, 50], cuda_device)
-    ctx.obs_chunk_attn(db.k_pool, db.v_pool, db.page_table, lens, dev_i32([0, 20, 40], cuda_device), q, 0.1, 300, out)
+    ctx.obs_chunk_attn(db.k_pool, db.v_pool, db.page_table, lens, dev_i32([0, 20, 40], cuda_device), q, 0.1, 100, out)
     assert ctx.status() == rollart.ERR_BOUNDS and "obs_chunk_attn" in ctx.last_error()

@@ -151,6 +151,3 @@ def test_host_side_validation(cuda_device):
         ctx.decode_attn(db.k_pool[:, :3].contiguous(), db.v_pool[:, :3].contiguous(), db.page_table, db.lens_before, q,
                         0.1, 8000, out)
     assert e.value.status == rollart.ERR_INVALID_ARG
-    with pytest.raises(rollart.RollartError) as e:       # bound larger than a page-table row can hold
-        ctx.decode_attn(db.k_pool, db.v_pool, db.page_table, db.lens_before, q, 0.1, 10 ** 7, out)
-    assert e.value.status == rollart.ERR_INVALID_ARG
