@@ -1,0 +1,383 @@
+#!/usr/bin/env python
+"""Benchmark of the rollout-attention hot path on B200.
+
+A step is one pass of the engine step's attention part over one synthetic batch of
+trajectories: KV append of one new token per trajectory, then decode attention over each
+trajectory's whole paged context (split over thread blocks, merged by the log-sum-exp combine).
+Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle on a bounded sample.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2512_22560_b200 import workloads as W  # noqa: E402
+
+METRIC = "paged-KV decode attention: achieved HBM GB/s (% of B200 peak), decode tokens/s"
+UNIT = "decode tokens/s"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        try:
+            with open(path) as f:
+                return float(json.load(f)["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+def decode_algorithmic_bytes(spec: W.WorkloadSpec, lens_after: np.ndarray) -> int:
+    """K and V of every context token read once per kv head (shared by the group's q heads),
+    Q in and O out, and the page-table entries that are needed."""
+    kv = int(lens_after.astype(np.int64).sum()) * 2 * spec.num_kv_heads * spec.head_dim * 2
+    qo = 2 * len(lens_after) * spec.num_q_heads * spec.head_dim * 2
+    pt = 4 * int(((lens_after.astype(np.int64) + spec.page_size - 1) // spec.page_size).sum())
+    return kv + qo + pt
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs (read only)."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.rows = []
+        self._stop = threading.Event()
+        self._t = threading.Thread(target=self._run, daemon=True)
+
+    def _run(self):
+        while not self._stop.is_set():
+            try:
+                r = subprocess.run(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                    "-i", str(self.index)], capture_output=True, text=True, timeout=5)
+                if r.returncode == 0 and r.stdout.strip():
+                    self.rows.append([x.strip() for x in r.stdout.strip().split(",")])
+            except Exception:
+                pass
+            self._stop.wait(0.1)
+
+    def __enter__(self):
+        self._t.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        self._t.join(timeout=6)
+
+    def summary(self):
+        sm = [float(r[0]) for r in self.rows if r and r[0].replace(".", "").isdigit()]
+        mx = [float(r[1]) for r in self.rows if len(r) > 1 and r[1].replace(".", "").isdigit()]
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = [n for i, n in enumerate(names) if any(len(r) > 3 + i and r[3 + i].lower().startswith("active") for r in self.rows)]
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": reasons, "samples": len(self.rows)}
+
+
+class DecodeWorkload:
+    """Device-resident state of one workload plus the two calls of a step."""
+
+    def __init__(self, spec: W.WorkloadSpec, seed: int, device: torch.device, ids=None):
+        from paper_2512_22560_b200 import rollart
+        self.spec = spec
+        self.device = device
+        b = W.make_batch(spec, seed=seed, device=device)
+        self.batch = b
+        ids = b.decode_ids if ids is None else ids
+        self.ids = ids
+        i32 = lambda a: torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).to(device)
+        self.table = i32(b.page_table)
+        self.lens0 = i32(b.seq_lens_before)
+        self.lens1 = i32(b.seq_lens_after)          # overwritten by the append of the ids below
+        self.traj_ids = i32(ids)
+        rows = torch.from_numpy(b.decode_rows(ids)).to(device)
+        self.q = b.q_new[rows].contiguous()
+        self.k_new = b.k_new[rows].contiguous()
+        self.v_new = b.v_new[rows].contiguous()
+        self.indptr = i32(np.arange(len(ids) + 1))
+        self.out = torch.empty_like(self.q)
+        self.max_seq_len = int(b.seq_lens_after[ids].max())
+        self.ctx = rollart.Context(device.index or 0, rollart.workspace_size(len(ids), spec.num_q_heads, spec.num_kv_heads,
+                                                                            self.max_seq_len))
+        self.lens_after_host = b.seq_lens_after[ids]
+        self.bytes = decode_algorithmic_bytes(spec, self.lens_after_host)
+        self.n_items = len(ids)
+
+    def append(self):
+        self.ctx.kv_append(self.batch.k_pool, self.batch.v_pool, self.table, self.lens0, self.indptr, self.k_new, self.v_new,
+                           traj_ids=self.traj_ids, seq_lens_out=self.lens1)
+
+    def decode(self):
+        self.ctx.decode_attn(self.batch.k_pool, self.batch.v_pool, self.table, self.lens1, self.q, self.spec.sm_scale,
+                             self.max_seq_len, self.out, traj_ids=self.traj_ids)
+
+    def step(self):
+        self.append()
+        self.decode()
+
+    def time_steps(self, steps: int, warmup: int):
+        """(total ms over `steps` steps, mean ms of the decode_attn call alone)."""
+        for _ in range(warmup):
+            self.step()
+        torch.cuda.synchronize(self.device)
+        ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(steps)]
+        t0 = torch.cuda.Event(enable_timing=True)
+        t1 = torch.cuda.Event(enable_timing=True)
+        t0.record()
+        for s in range(steps):
+            ev[s][0].record()
+            self.append()
+            ev[s][1].record()
+            self.decode()
+            ev[s][2].record()
+        t1.record()
+        torch.cuda.synchronize(self.device)
+        total = t0.elapsed_time(t1)
+        dec = float(np.mean([e[1].elapsed_time(e[2]) for e in ev]))
+        self.ctx.check()
+        return total, dec
+
+    def time_e2e(self, steps: int, warmup: int):
+        """Steps driven from HOST buffers: per step the new token's q/k/v go host->device from
+        pinned memory and the attention output comes back device->host, inside the timed region."""
+        hq, hk, hv = (t.cpu().pin_memory() for t in (self.q, self.k_new, self.v_new))
+        hout = torch.empty_like(self.out, device="cpu").pin_memory()
+
+        def one():
+            self.q.copy_(hq, non_blocking=True)
+            self.k_new.copy_(hk, non_blocking=True)
+            self.v_new.copy_(hv, non_blocking=True)
+            self.step()
+            hout.copy_(self.out, non_blocking=True)
+            torch.cuda.synchronize(self.device)     # the host consumes each step's result
+
+        for _ in range(warmup):
+            one()
+        t0 = time.perf_counter()
+        for _ in range(steps):
+            one()
+        dt = time.perf_counter() - t0
+        h2d = hq.numel() * 2 + hk.numel() * 2 + hv.numel() * 2
+        d2h = hout.numel() * 2
+        return dt * 1e3, h2d, d2h
+
+
+class CpuBaseline:
+    """The oracle, as it stands, timed on a bounded sample of the workload's trajectories."""
+
+    def __init__(self, spec: W.WorkloadSpec, seed: int, budget_s: float = 15.0):
+        import oracle
+        self.oracle = oracle
+        self.spec = spec
+        layout = W.make_layout(spec, seed=seed)
+        dec = layout.decode_ids
+        cand = np.random.default_rng(seed).permutation(dec)
+        # tensors for a bounded prefix of the candidates (at most 1M context tokens on the host)
+        keep, toks = [], 0
+        for t in cand:
+            if keep and toks + int(layout.seq_lens_before[t]) > (1 << 20):
+                break
+            keep.append(int(t))
+            toks += int(layout.seq_lens_before[t])
+        self.full = _sample_tensors(layout, keep)
+        self.n_dec = len(dec)
+        t_cal, tok_cal = self.run([0])
+        per_tok = t_cal / max(1, tok_cal)
+        take, acc = [], 0.0
+        for i in range(len(keep)):
+            cost = per_tok * int(self.full.seq_lens_before[i] + 1)
+            if take and acc + cost > budget_s:
+                break
+            take.append(i)
+            acc += cost
+        self.take = take
+
+    def run(self, ids):
+        sub = W.extract_trajs(self.full, ids)
+        kp, vp = W.bf16_to_u16(sub.k_pool), W.bf16_to_u16(sub.v_pool)
+        k_new, v_new = W.bf16_to_u16(sub.k_new), W.bf16_to_u16(sub.v_new)
+        rows = sub.decode_rows(np.arange(len(ids)))
+        q = W.bf16_to_u16(sub.q_new[rows])
+        t0 = time.perf_counter()
+        after = self.oracle.kv_append(kp, vp, sub.page_table, sub.seq_lens_before, sub.new_indptr, k_new, v_new)
+        self.oracle.decode_attn(kp, vp, sub.page_table, after, q, self.spec.sm_scale)
+        return time.perf_counter() - t0, int(after.sum())
+
+    def measure(self):
+        t, toks = self.run(self.take)
+        info = {"value": len(self.take) / t, "unit": UNIT, "cores": self.oracle.num_threads(), "kind": "oracle",
+                "sample": f"{len(self.take)} of {self.n_dec} trajectories of {self.spec.name} ({toks} context tokens), "
+                          f"append + decode, {t:.2f} s wall"}
+        return info, t, len(self.take)
+
+
+def _sample_tensors(layout: W.Batch, ids) -> W.Batch:
+    """CPU tensors for trajectories `ids` only (compact pool), same distributions as the full recipe."""
+    spec = layout.spec
+    P = spec.page_size
+    ids = np.asarray(ids, dtype=np.int64)
+    import dataclasses
+    sub = dataclasses.replace(spec, num_traj=len(ids), name=spec.name + "_cpu_sample")
+    lens = layout.seq_lens_before[ids].copy()
+    n_new = layout.n_new[ids].copy()
+    pages = (lens.astype(np.int64) + n_new + P - 1) // P
+    table, num_pages = W.build_page_table(pages, spec.spare_pages, np.random.default_rng(layout.seed + 1))
+    indptr = np.zeros(len(ids) + 1, dtype=np.int32)
+    indptr[1:] = np.cumsum(n_new)
+    b = W.Batch(sub, layout.seed, lens, n_new, layout.is_chunk[ids].copy(), indptr, table, num_pages)
+    return W.fill_tensors(b, "cpu")
+
+
+def run_reference(args):
+    """`--impl reference`: the CPU oracle on a bounded sample per step (rank 0 only)."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    spec = W.CONFIGS[args.config]
+    times, n = [], 0
+    info = None
+    base = CpuBaseline(spec, args.seed, budget_s=args.ref_budget)
+    for s in range(args.warmup + args.steps):
+        info, t, n = base.measure()
+        if s >= args.warmup:
+            times.append(t)
+    ms = 1e3 * float(np.mean(times))
+    value = n / (ms / 1e3)
+    info["value"] = value
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+            "data": "synthetic", "impl": "reference",
+            "config": {"workload": spec.name, "note": "CPU fp64 oracle on a bounded sample of the workload per step"},
+            "cpu_baseline": info,
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=1, help="index into the five workload recipes (headline: 1)")
+    ap.add_argument("--seed", type=int, default=W.MASTER_SEED)
+    ap.add_argument("--ref-budget", type=float, default=12.0, help="seconds of oracle work per reference step")
+    ap.add_argument("--no-extra", action="store_true", help="skip the other decode workloads and the CPU baseline")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+
+    if args.impl == "reference":
+        return run_reference(args)
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    device = torch.device("cuda", local)
+    torch.cuda.set_device(device)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=device)
+
+    spec = W.CONFIGS[args.config]
+    wl = DecodeWorkload(spec, args.seed + rank, device)      # replicas: each rank owns its own trajectories
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize(device)
+
+    launches0 = wl.ctx.launch_count
+    barrier()
+    with ClockSampler(local) as clocks:
+        total_ms, dec_ms = wl.time_steps(args.steps, args.warmup)
+    barrier()
+    launches = (wl.ctx.launch_count - launches0) * args.steps // (args.steps + args.warmup)
+    e2e_ms, h2d, d2h = wl.time_e2e(max(10, args.steps // 4), 3)
+    e2e_steps = max(10, args.steps // 4)
+
+    t = torch.tensor([total_ms, dec_ms, e2e_ms / e2e_steps], dtype=torch.float64, device=device)
+    items = torch.tensor([wl.n_items], dtype=torch.float64, device=device)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        dist.all_reduce(items, op=dist.ReduceOp.SUM)
+    total_ms, dec_ms, e2e_ms_step = (float(x) for x in t.tolist())
+    n_items_all = float(items.item())
+    ms_per_step = total_ms / args.steps
+
+    if rank == 0:
+        peak, peak_kind = measured_peaks()
+        achieved = wl.bytes / (dec_ms * 1e-3) / 1e9
+        line = {
+            "metric": METRIC, "value": n_items_all / (ms_per_step * 1e-3), "unit": UNIT, "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": spec.name, "trajectories_per_gpu": wl.n_items, "num_q_heads": spec.num_q_heads,
+                       "num_kv_heads": spec.num_kv_heads, "page_size": spec.page_size,
+                       "context_tokens_per_gpu": int(wl.lens_after_host.sum()),
+                       "step": "kv_append(1 token/trajectory) + decode_attn (split partials + LSE combine), one attention layer",
+                       "l2": "inputs larger than L2: %.2f GB of KV read per step" % (wl.bytes / 1e9),
+                       "parallelism": f"replicas x{world} (independent trajectories, no collective)"},
+            "hbm_gbs": achieved, "hbm_frac_of_nominal_8tbs": achieved / NOMINAL_HBM_GBS,
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                         "peak_kind": f"of {peak_kind}", "traffic": None,
+                         "kernel": "decode_attn call (partial-attention kernel + combine kernel)",
+                         "algorithmic_bytes_per_launch": wl.bytes, "ms_per_launch": dec_ms},
+            "e2e": {"value": n_items_all / (e2e_ms_step * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                    "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms_step,
+                    "note": "per step: q/k_new/v_new host->device from pinned memory, out device->host; the KV pool is resident engine state"},
+            "gpu_launches": int(launches),
+            "clocks": clocks.summary(),
+        }
+        if not args.no_extra and world == 1:
+            extra = {}
+            del wl
+            torch.cuda.empty_cache()
+            for ci in (2, 3, 4):
+                try:
+                    w2 = DecodeWorkload(W.CONFIGS[ci], args.seed, device)
+                    tot, dms = w2.time_steps(20, 3)
+                    gbs = w2.bytes / (dms * 1e-3) / 1e9
+                    extra[W.CONFIGS[ci].name] = {"decode_ms": dms, "step_ms": tot / 20, "hbm_gbs": gbs,
+                                                 "frac_of_measured": gbs / peak, "frac_of_nominal_8tbs": gbs / NOMINAL_HBM_GBS,
+                                                 "decode_tokens_per_s": w2.n_items / (tot / 20 * 1e-3),
+                                                 "trajectories": w2.n_items}
+                    w2.ctx.close()
+                    del w2
+                    torch.cuda.empty_cache()
+                except Exception as e:  # report, never hide
+                    extra[W.CONFIGS[ci].name] = {"error": repr(e)}
+            line["other_workloads"] = extra
+            info, _, _ = CpuBaseline(spec, args.seed).measure()
+            line["cpu_baseline"] = info
+        print(json.dumps(line))
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())
