@@ -1,8 +1,8 @@
-// Row-at-a-time attention on CUDA cores: one thread block per (query row, kv head, key split).
+// Row-at-a-time attention on CUDA cores: one thread block per (query row, kv head).
 //
 // This is the plain path: every query row streams its keys itself, all g query heads of the
 // group sharing each K/V read, with fp32 FMA dot products and warp-shuffle reductions.  It serves
-// observation chunks (one row per chunk token) and is the fallback shape for decode.
+// observation chunks (one block per chunk token and kv head).
 #include "rollart_internal.cuh"
 
 namespace rollart {
@@ -13,9 +13,6 @@ constexpr int kThreads = 128;
 constexpr int kWarps = kThreads / 32;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
-
-// Workspace slot of one partial result: O[16][128] fp32, m[16], l[16] (log2 domain max, sum).
-constexpr size_t kSlotFloats = kMaxGroup * kHeadDim + 2 * kMaxGroup;
 
 __device__ __forceinline__ int find_item(const int32_t *__restrict__ indptr, int n_items, int row) {
     int lo = 0, hi = n_items;
@@ -36,12 +33,11 @@ template <int G>
 __global__ void __launch_bounds__(kThreads)
 attn_rows_kernel(PoolView pool, TrajView trajs, const int32_t *__restrict__ traj_ids, const int32_t *__restrict__ q_indptr,
                  int n_items, int max_seq_len, const __nv_bfloat16 *__restrict__ q, int num_q_heads, float scale_log2,
-                 __nv_bfloat16 *__restrict__ out, float *__restrict__ lse, float *__restrict__ ws, int keys_per_split,
-                 int nsplit, DeviceStatus *status, int where) {
+                 __nv_bfloat16 *__restrict__ out, float *__restrict__ lse, DeviceStatus *status, int where) {
     __shared__ float sm_acc[kWarps][G][kHeadDim];
     __shared__ float sm_m[kWarps][G], sm_l[kWarps][G];
 
-    const int row = blockIdx.x, h = blockIdx.y, split = blockIdx.z;
+    const int row = blockIdx.x, h = blockIdx.y;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     int item = row, n_rows = 1, j_in_chunk = 0;
@@ -67,8 +63,8 @@ attn_rows_kernel(PoolView pool, TrajView trajs, const int32_t *__restrict__ traj
             if (L == 0) count = 0;
         }
     }
-    const int begin = split * keys_per_split;
-    const int end = bad ? 0 : min(count, begin + keys_per_split);
+    const int begin = 0;
+    const int end = bad ? 0 : count;
 
     // q: lane owns dims 4*lane .. 4*lane+3 of every head of the group
     float qf[G][4];
@@ -129,8 +125,6 @@ attn_rows_kernel(PoolView pool, TrajView trajs, const int32_t *__restrict__ traj
 
     // thread d merges the four warps for dim d of every head, in warp order
     const int d = threadIdx.x;
-    const long long slot = (static_cast<long long>(row) * pool.num_kv_heads + h) * nsplit + split;
-    float *ws_o = ws ? ws + slot * kSlotFloats : nullptr;
 #pragma unroll
     for (int r = 0; r < G; ++r) {
         float M = sm_m[0][r];
@@ -145,60 +139,26 @@ attn_rows_kernel(PoolView pool, TrajView trajs, const int32_t *__restrict__ traj
                 lsum += sm_l[w][r] * a;
             }
         }
-        if (nsplit == 1) {
-            const long long oi = (static_cast<long long>(row) * num_q_heads + h * G + r) * kHeadDim + d;
-            out[oi] = __float2bfloat16_rn(lsum > 0.f ? o / lsum : 0.f);
-            if (lse != nullptr && d == 0)
-                lse[static_cast<long long>(row) * num_q_heads + h * G + r] = lsum > 0.f ? (M + log2f(lsum)) * kLn2 : -INFINITY;
-        } else {
-            ws_o[r * kHeadDim + d] = o;
-            if (d == 0) {
-                ws_o[kMaxGroup * kHeadDim + r] = M;
-                ws_o[kMaxGroup * kHeadDim + kMaxGroup + r] = lsum;
-            }
-        }
+        const long long oi = (static_cast<long long>(row) * num_q_heads + h * G + r) * kHeadDim + d;
+        out[oi] = __float2bfloat16_rn(lsum > 0.f ? o / lsum : 0.f);
+        if (lse != nullptr && d == 0)
+            lse[static_cast<long long>(row) * num_q_heads + h * G + r] = lsum > 0.f ? (M + log2f(lsum)) * kLn2 : -INFINITY;
     }
-}
-
-// Cross-split log-sum-exp combine: one block per (row, q head), thread d owns dim d.
-__global__ void __launch_bounds__(kHeadDim)
-combine_rows_kernel(const float *__restrict__ ws, int num_kv_heads, int group, int nsplit, int num_q_heads,
-                    __nv_bfloat16 *__restrict__ out, float *__restrict__ lse) {
-    const int row = blockIdx.x, hq = blockIdx.y, d = threadIdx.x;
-    const int h = hq / group, r = hq % group;
-    const float *base = ws + (static_cast<long long>(row) * num_kv_heads + h) * nsplit * kSlotFloats;
-    float M = -INFINITY;
-    for (int s = 0; s < nsplit; ++s) M = fmaxf(M, __ldg(base + s * kSlotFloats + kMaxGroup * kHeadDim + r));
-    float o = 0.f, lsum = 0.f;
-    if (M != -INFINITY) {
-        for (int s = 0; s < nsplit; ++s) {
-            const float *p = base + s * kSlotFloats;
-            const float a = exp2f(__ldg(p + kMaxGroup * kHeadDim + r) - M);
-            o += __ldg(p + r * kHeadDim + d) * a;
-            lsum += __ldg(p + kMaxGroup * kHeadDim + kMaxGroup + r) * a;
-        }
-    }
-    out[(static_cast<long long>(row) * num_q_heads + hq) * kHeadDim + d] = __float2bfloat16_rn(lsum > 0.f ? o / lsum : 0.f);
-    if (lse != nullptr && d == 0)
-        lse[static_cast<long long>(row) * num_q_heads + hq] = lsum > 0.f ? (M + log2f(lsum)) * kLn2 : -INFINITY;
 }
 
 template <int G>
-cudaError_t launch_rows_g(const AttnCall &c, int keys_per_split, int nsplit, int where, cudaStream_t stream,
-                          int64_t *launches) {
-    dim3 grid(c.total_q, c.pool.num_kv_heads, nsplit);
-    attn_rows_kernel<G><<<grid, kThreads, 0, stream>>>(
-        c.pool, c.trajs, c.traj_ids, c.q_indptr, c.n_items, c.max_seq_len, c.q, c.num_q_heads, c.sm_scale * kLog2e, c.out,
-        c.lse, nsplit > 1 ? static_cast<float *>(c.workspace) : nullptr, keys_per_split, nsplit, c.status, where);
+cudaError_t launch_rows_g(const AttnCall &c, int where, cudaStream_t stream, int64_t *launches) {
+    dim3 grid(c.total_q, c.pool.num_kv_heads);
+    attn_rows_kernel<G><<<grid, kThreads, 0, stream>>>(c.pool, c.trajs, c.traj_ids, c.q_indptr, c.n_items, c.max_seq_len, c.q,
+                                                       c.num_q_heads, c.sm_scale * kLog2e, c.out, c.lse, c.status, where);
     ++*launches;
     return cudaGetLastError();
 }
 
-cudaError_t launch_rows(const AttnCall &c, int keys_per_split, int nsplit, int where, cudaStream_t stream,
-                        int64_t *launches) {
+cudaError_t launch_rows(const AttnCall &c, int where, cudaStream_t stream, int64_t *launches) {
     const int g = c.num_q_heads / c.pool.num_kv_heads;
     switch (g) {
-#define ROLLART_CASE(G) case G: return launch_rows_g<G>(c, keys_per_split, nsplit, where, stream, launches);
+#define ROLLART_CASE(G) case G: return launch_rows_g<G>(c, where, stream, launches);
         ROLLART_CASE(1) ROLLART_CASE(2) ROLLART_CASE(3) ROLLART_CASE(4) ROLLART_CASE(5) ROLLART_CASE(6)
         ROLLART_CASE(7) ROLLART_CASE(8) ROLLART_CASE(9) ROLLART_CASE(10) ROLLART_CASE(11) ROLLART_CASE(12)
         ROLLART_CASE(13) ROLLART_CASE(14) ROLLART_CASE(15) ROLLART_CASE(16)
@@ -209,42 +169,9 @@ cudaError_t launch_rows(const AttnCall &c, int keys_per_split, int nsplit, int w
 
 }  // namespace
 
-size_t decode_workspace_bytes(int max_items, int num_q_heads, int num_kv_heads, int max_seq_len, int sm_count) {
-    (void)num_q_heads; (void)max_seq_len; (void)sm_count;
-    // one slot per (item, kv head) plus one per extra split; the schedule never makes more than
-    // 2048 extra splits in total
-    const size_t slots = static_cast<size_t>(max_items) * num_kv_heads + 2048;
-    return slots * kSlotFloats * sizeof(float);
-}
-
-cudaError_t launch_decode_attn(const AttnCall &c, cudaStream_t stream, int64_t *launches, bool *too_small) {
-    // enough blocks to fill the machine several times over, splits of at least 64 keys
-    const long long units = static_cast<long long>(c.n_items) * c.pool.num_kv_heads;
-    long long want = (1184 + units - 1) / units;
-    if (want > 64) want = 64;
-    if (want < 1) want = 1;
-    int keys_per_split = static_cast<int>((static_cast<long long>(c.max_seq_len) + want - 1) / want);
-    keys_per_split = ((keys_per_split + 63) / 64) * 64;
-    if (keys_per_split < 64) keys_per_split = 64;
-    int nsplit = (c.max_seq_len + keys_per_split - 1) / keys_per_split;
-    if (nsplit < 1) nsplit = 1;
-    if (nsplit > 1) {
-        const size_t need = static_cast<size_t>(units) * nsplit * kSlotFloats * sizeof(float);
-        if (need > c.workspace_bytes || c.workspace == nullptr) { *too_small = true; return cudaErrorInvalidValue; }
-    }
-    cudaError_t e = launch_rows(c, keys_per_split, nsplit, 2, stream, launches);
-    if (e != cudaSuccess || nsplit == 1) return e;
-    dim3 grid(c.n_items, c.num_q_heads);
-    combine_rows_kernel<<<grid, kHeadDim, 0, stream>>>(static_cast<const float *>(c.workspace), c.pool.num_kv_heads,
-                                                       c.num_q_heads / c.pool.num_kv_heads, nsplit, c.num_q_heads, c.out,
-                                                       c.lse);
-    ++*launches;
-    return cudaGetLastError();
-}
-
 cudaError_t launch_chunk_attn(const AttnCall &c, cudaStream_t stream, int64_t *launches, bool *too_small) {
     (void)too_small;
-    return launch_rows(c, c.max_seq_len > 0 ? c.max_seq_len : 1, 1, 3, stream, launches);
+    return launch_rows(c, 3, stream, launches);
 }
 
 }  // namespace rollart

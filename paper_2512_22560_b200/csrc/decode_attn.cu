@@ -1,0 +1,646 @@
+// Decode attention: split-KV flash decoding over a paged bf16 KV cache, one persistent thread
+// block per SM.
+//
+// Schedule.  Every (item, kv head) owns ceil(L / 64) key tiles.  All tiles of the call are laid
+// on one line, ordered (item, kv head, tile), and the line is cut into gridDim.x equal spans, one
+// per thread block.  A block therefore reads the same number of bytes as every other block
+// whatever the length mix, and a span that crosses an (item, head) boundary simply starts a new
+// "piece".  A piece that covers its (item, head) entirely writes the final bf16 output; otherwise
+// it writes an un-normalised fp32 partial (O, m, l) into a workspace slot, and the combine kernel
+// merges the slots of that (item, head) with the log-sum-exp rule.  The cut is a fixed function
+// of the lengths, so reruns are bit identical.
+//
+// Data path.  A producer warp walks the block's span and brings each 64-key tile of K and V
+// (32 KB) into a ring of shared-memory stages with TMA tensor copies, one box per (page, head)
+// (or per half row), 128-byte swizzled so that ldmatrix reads are bank-conflict free; the page
+// ids come from the page table just ahead of the copy.  Eight consumer warps in two groups take
+// alternate tiles; each warp owns 16 keys of a tile and computes, for all (up to 16) query heads
+// of the GQA group at once, S = Q K^T and O += P V with bf16 mma.sync (fp32 accumulate) and an
+// online softmax in registers.  One K/V read serves the whole group.  HBM traffic is the KV
+// bytes once, plus Q, O and the few partial slots.
+#include <cuda.h>
+
+#include "rollart_internal.cuh"
+
+namespace rollart {
+
+namespace {
+
+constexpr int kTile = 64;                 // keys per stage
+constexpr int kStages = 6;
+constexpr int kConsumerWarps = 8;         // two groups of four
+constexpr int kThreads = (kConsumerWarps + 1) * 32;
+constexpr int kMaxItems = 1024;           // items per launch (prefix table lives in shared memory)
+constexpr int kTensorBytes = kTile * kRowBytes;      // 16 KB of K (or V) per stage
+constexpr int kStageBytes = 2 * kTensorBytes;
+constexpr int kQBytes = kMaxGroup * kRowBytes;       // 4 KB
+constexpr int kMergeStride = kHeadDim + 8;           // floats per merge-buffer row (padded)
+constexpr uint32_t kSpinLimit = 1u << 22;
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+constexpr size_t kSlotFloats = kMaxGroup * kHeadDim + 2 * kMaxGroup;
+
+// shared-memory map (offsets from a 1024-byte aligned base)
+constexpr int kOffStages = 0;
+constexpr int kOffQ = kOffStages + kStages * kStageBytes;
+constexpr int kOffMerge = kOffQ + 2 * kQBytes;
+constexpr int kOffMl = kOffMerge + kMaxGroup * kMergeStride * 4;
+constexpr int kOffLens = kOffMl + kConsumerWarps * kMaxGroup * 2 * 4;
+constexpr int kOffPrefix = kOffLens + kMaxItems * 4;
+constexpr int kOffBars = kOffPrefix + (kMaxItems + 32) * 4;
+constexpr int kNumBars = 2 * kStages + 4;
+constexpr int kOffAbort = kOffBars + kNumBars * 8;
+constexpr int kSmemBytes = kOffAbort + 16 + 1024;    // + slack for the 1024-byte alignment
+
+struct DecodeParams {
+    const int32_t *page_table;
+    const int32_t *seq_lens;
+    const int32_t *traj_ids;
+    int max_pages, num_traj, num_pages, page_size, num_kv_heads, num_q_heads, group;
+    int n_items, item_offset, max_seq_len;
+    int four_d;                 // tensor maps are 4-D (one box per page) instead of 2-D (two boxes)
+    const __nv_bfloat16 *q;
+    __nv_bfloat16 *out;
+    float *lse;
+    float scale_log2;
+    int2 *info;                 // per (item, kv head): first and last block of its pieces
+    float *slots;
+    DeviceStatus *status;
+};
+
+// ------------------------------------------------------------------------------------------
+// PTX wrappers
+// ------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait.  Gives up when the limit runs out or another warp has already given up; the
+// caller carries on (with garbage data) so that every barrier sequence still completes.
+__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, DeviceStatus *status,
+                                          int where) {
+    for (uint32_t it = 0; it < kSpinLimit; ++it) {
+        if (mbar_try_wait(bar, parity)) return;
+        if ((it & 1023u) == 1023u && *abort_flag) return;
+    }
+    if (*abort_flag == 0) {
+        *abort_flag = 1;
+        report(status, ROLLART_ERR_TIMEOUT, where, 2);
+    }
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int x, int y) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1, int c2, int c3) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+}
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void consumer_bar() { asm volatile("bar.sync 1, %0;" ::"n"(kConsumerWarps * 32) : "memory"); }
+
+__device__ __forceinline__ void ldmatrix_x4(uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3, uint32_t addr) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3, uint32_t addr) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t *>(&v);
+}
+
+// ------------------------------------------------------------------------------------------
+// The walk over a block's span of the tile line: the same code runs in the producer and in the
+// consumers, so both see the same sequence of pieces.
+// ------------------------------------------------------------------------------------------
+struct Piece {
+    int item, head, tile0, tile1, ntiles, len;
+};
+
+__device__ __forceinline__ Piece piece_at(const int *prefix, const int *lens, int n_items, int hkv, int p, int p_end) {
+    int lo = 0, hi = n_items;                     // largest item with prefix[item] * hkv <= p
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (prefix[mid] * hkv <= p) lo = mid; else hi = mid;
+    }
+    Piece pc;
+    pc.item = lo;
+    pc.ntiles = max(1, prefix[lo + 1] - prefix[lo]);
+    const int rem = p - prefix[lo] * hkv;
+    pc.head = rem / pc.ntiles;
+    pc.tile0 = rem - pc.head * pc.ntiles;
+    pc.tile1 = min(pc.ntiles, pc.tile0 + (p_end - p));
+    pc.len = lens[lo];
+    return pc;
+}
+
+// ------------------------------------------------------------------------------------------
+// Kernel
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kThreads, 1)
+decode_splitkv_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__ CUtensorMap vmap,
+                      const DecodeParams prm) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    int *s_lens = reinterpret_cast<int *>(smem + kOffLens);
+    int *s_prefix = reinterpret_cast<int *>(smem + kOffPrefix);
+    float *s_merge = reinterpret_cast<float *>(smem + kOffMerge);
+    float *s_ml = reinterpret_cast<float *>(smem + kOffMl);
+    volatile int *s_abort = reinterpret_cast<volatile int *>(smem + kOffAbort);
+    const uint32_t bars = smem_u32(smem + kOffBars);
+    auto bar_full = [&](int s) { return bars + 8u * s; };
+    auto bar_empty = [&](int s) { return bars + 8u * (kStages + s); };
+    auto bar_qfull = [&](int s) { return bars + 8u * (2 * kStages + s); };
+    auto bar_qempty = [&](int s) { return bars + 8u * (2 * kStages + 2 + s); };
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int hkv = prm.num_kv_heads, P = prm.page_size, g = prm.group;
+
+    // ---- lengths -> tiles per item -> exclusive prefix (shared memory) ----
+    for (int i = threadIdx.x; i < prm.n_items; i += kThreads) {
+        const int t = prm.traj_ids ? __ldg(prm.traj_ids + i) : i + prm.item_offset;
+        int L = 0;
+        if (t < 0 || t >= prm.num_traj) {
+            report(prm.status, ROLLART_ERR_BOUNDS, t, 2);
+        } else {
+            L = __ldg(prm.seq_lens + t);
+            if (L < 0 || L > prm.max_seq_len) { report(prm.status, ROLLART_ERR_BOUNDS, L, 2); L = 0; }
+        }
+        s_lens[i] = L;
+    }
+    // zero both Q buffers once: rows >= g are never written by the copies and must read as 0
+    for (int i = threadIdx.x; i < 2 * kQBytes / 16; i += kThreads)
+        reinterpret_cast<uint4 *>(smem + kOffQ)[i] = make_uint4(0, 0, 0, 0);
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) { mbar_init(bar_full(s), 1); mbar_init(bar_empty(s), kConsumerWarps / 2); }
+        for (int s = 0; s < 2; ++s) { mbar_init(bar_qfull(s), 1); mbar_init(bar_qempty(s), kConsumerWarps); }
+        *s_abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    if (warp == 0) {
+        const int per = (prm.n_items + 31) / 32;
+        const int a = min(prm.n_items, lane * per), b = min(prm.n_items, a + per);
+        int sum = 0;
+        for (int i = a; i < b; ++i) sum += (s_lens[i] + kTile - 1) / kTile;
+        int incl = sum;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int v = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += v;
+        }
+        int run = incl - sum;
+        for (int i = a; i < b; ++i) { s_prefix[i] = run; run += (s_lens[i] + kTile - 1) / kTile; }
+        if (lane == 31) s_prefix[prm.n_items] = incl;
+    }
+    fence_proxy_async();      // the zeroed Q rows are ordered before the bulk copies that land beside them
+    __syncthreads();
+
+    const int total = s_prefix[prm.n_items] * hkv;
+    const int span = max(1, (total + static_cast<int>(gridDim.x) - 1) / static_cast<int>(gridDim.x));
+    const int p_begin = min(total, static_cast<int>(blockIdx.x) * span);
+    const int p_end = min(total, p_begin + span);
+    if (p_begin >= p_end) return;
+
+    if (warp == kConsumerWarps) {
+        // =============================== producer warp ===============================
+        const int pages_per_tile = kTile / P;
+        const uint32_t page_bytes = static_cast<uint32_t>(P) * kRowBytes;
+        int n = 0, pcount = 0;
+        for (int p = p_begin; p < p_end; ++pcount) {
+            const Piece pc = piece_at(s_prefix, s_lens, prm.n_items, hkv, p, p_end);
+            const int t = prm.traj_ids ? __ldg(prm.traj_ids + pc.item) : pc.item + prm.item_offset;
+            const int32_t *table_row = prm.page_table + static_cast<long long>(t) * prm.max_pages;
+            // Q rows of this (item, kv head): g contiguous rows of 256 B
+            const int qs = pcount & 1;
+            mbar_wait(bar_qempty(qs), ((pcount >> 1) & 1) ^ 1, s_abort, prm.status, 1);
+            if (lane == 0 && !*s_abort) {
+                mbar_arrive_expect_tx(bar_qfull(qs), static_cast<uint32_t>(g) * kRowBytes);
+                bulk_load(smem_u32(smem + kOffQ + qs * kQBytes),
+                          prm.q + (static_cast<long long>(pc.item) * prm.num_q_heads + pc.head * g) * kHeadDim,
+                          static_cast<uint32_t>(g) * kRowBytes, bar_qfull(qs));
+            }
+            for (int tile = pc.tile0; tile < pc.tile1; ++tile, ++n) {
+                const int stage = n % kStages;
+                // page ids of this tile, one lane per page
+                const int lp = tile * pages_per_tile + lane;
+                int pg = -1;
+                if (lane < pages_per_tile && lp * P < pc.len) {
+                    pg = __ldg(table_row + lp);
+                    if (pg < 0 || pg >= prm.num_pages) { report(prm.status, ROLLART_ERR_BOUNDS, pg, 2); pg = -1; }
+                }
+                const uint32_t nvalid = __popc(__ballot_sync(0xffffffffu, pg >= 0));
+                mbar_wait(bar_empty(stage), ((n / kStages) & 1) ^ 1, s_abort, prm.status, 2);
+                if (*s_abort) continue;
+                if (lane == 0) mbar_arrive_expect_tx(bar_full(stage), nvalid * 2u * page_bytes);
+                __syncwarp();
+                if (pg >= 0) {
+                    const uint32_t kdst = smem_u32(smem + kOffStages + stage * kStageBytes) + lane * page_bytes;
+                    const uint32_t vdst = kdst + kTensorBytes;
+                    const int unit = pg * hkv + pc.head;          // (page, head) tile index
+                    if (prm.four_d) {
+                        tma_load_4d(kdst, &kmap, bar_full(stage), 0, 0, 0, unit);
+                        tma_load_4d(vdst, &vmap, bar_full(stage), 0, 0, 0, unit);
+                    } else {
+                        const int row = unit * P;
+                        tma_load_2d(kdst, &kmap, bar_full(stage), 0, row);
+                        tma_load_2d(kdst + page_bytes / 2, &kmap, bar_full(stage), 64, row);
+                        tma_load_2d(vdst, &vmap, bar_full(stage), 0, row);
+                        tma_load_2d(vdst + page_bytes / 2, &vmap, bar_full(stage), 64, row);
+                    }
+                }
+            }
+            p += pc.tile1 - pc.tile0;
+        }
+        // every copy this warp issued has been waited for by the consumers unless the block gave up;
+        // in that case wait (bounded) for the copies still in flight before the block exits
+        if (*s_abort && lane == 0) {
+            for (int k = 0; k < kStages && k < n; ++k) {
+                const int m = n - 1 - k;
+                for (uint32_t it = 0; it < kSpinLimit; ++it)
+                    if (mbar_try_wait(bar_full(m % kStages), (m / kStages) & 1)) break;
+            }
+        }
+        return;
+    }
+
+    // ================================= consumer warps =================================
+    const int grp = warp >> 2, wq = warp & 3;
+    const int qrow = lane >> 2, qcol = lane & 3;          // fragment row / column-pair of this lane
+    // byte offset of this warp's 16 keys inside a K (or V) stage image, and ldmatrix lane offsets
+    const int key0 = wq * 16;
+    const uint32_t warp_off = static_cast<uint32_t>((key0 / P) * P * kRowBytes + (key0 % P) * 128);
+    const uint32_t half_off = static_cast<uint32_t>(P) * 128;      // second 64 dims of a page image
+    const int lm = lane >> 3, lr = lane & 7;
+    // K: matrices (keys 0-7 | 8-15) x (dim chunk even | odd)
+    const uint32_t k_lane_off = static_cast<uint32_t>(((lm >> 1) * 8 + lr) * 128);
+    const int k_chunk_lo = lm & 1;
+    // V (transposed load): matrices (keys 0-7 | 8-15) x (dim chunk even | odd of the pair)
+    const uint32_t v_lane_off = static_cast<uint32_t>(((lm & 1) * 8 + lr) * 128);
+    const int v_chunk_lo = lm >> 1;
+
+    int n = 0, pcount = 0;
+    for (int p = p_begin; p < p_end; ++pcount) {
+        const Piece pc = piece_at(s_prefix, s_lens, prm.n_items, hkv, p, p_end);
+        const int qs = pcount & 1;
+        mbar_wait(bar_qfull(qs), (pcount >> 1) & 1, s_abort, prm.status, 3);
+        uint32_t qa[8][4];
+        {
+            const uint32_t qbase = smem_u32(smem + kOffQ + qs * kQBytes) + ((lm & 1) * 8 + lr) * kRowBytes + (lm >> 1) * 16;
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks) ldmatrix_x4(qa[ks][0], qa[ks][1], qa[ks][2], qa[ks][3], qbase + ks * 32);
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_qempty(qs));
+
+        float o[16][4];
+#pragma unroll
+        for (int j = 0; j < 16; ++j) o[j][0] = o[j][1] = o[j][2] = o[j][3] = 0.f;
+        float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
+
+        for (int tile = pc.tile0; tile < pc.tile1; ++tile, ++n) {
+            if ((n & 1) != grp) continue;
+            const int stage = n % kStages;
+            mbar_wait(bar_full(stage), (n / kStages) & 1, s_abort, prm.status, 4);
+            const uint32_t kbase = smem_u32(smem + kOffStages + stage * kStageBytes) + warp_off;
+            const uint32_t vbase = kbase + kTensorBytes;
+            const int valid = min(16, pc.len - tile * kTile - key0);   // live keys among this warp's 16
+            if (valid > 0) {
+                if (valid < 16) {
+                    // dead slots may hold anything (NaN included): zero their V rows so that 0 * v stays 0
+                    for (int idx = lane; idx < (16 - valid) * 16; idx += 32) {
+                        const int r = valid + (idx >> 4), c = idx & 15;
+                        const uint32_t a = vbase + (c >> 3) * half_off + r * 128 + (c & 7) * 16;
+                        asm volatile("st.shared.v4.b32 [%0], {%1,%1,%1,%1};" ::"r"(a), "r"(0) : "memory");
+                    }
+                    __syncwarp();
+                }
+                float s[2][4];
+#pragma unroll
+                for (int nt = 0; nt < 2; ++nt) s[nt][0] = s[nt][1] = s[nt][2] = s[nt][3] = 0.f;
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks) {
+                    const int chunk = ks * 2 + k_chunk_lo;
+                    uint32_t b0, b1, b2, b3;
+                    ldmatrix_x4(b0, b1, b2, b3, kbase + (chunk >> 3) * half_off + k_lane_off + (((chunk & 7) ^ lr) << 4));
+                    mma_bf16(s[0], qa[ks], b0, b1);
+                    mma_bf16(s[1], qa[ks], b2, b3);
+                }
+#pragma unroll
+                for (int nt = 0; nt < 2; ++nt)
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const int col = nt * 8 + qcol * 2 + (e & 1);
+                        s[nt][e] = col < valid ? s[nt][e] * prm.scale_log2 : -INFINITY;
+                    }
+                float r0 = fmaxf(fmaxf(s[0][0], s[0][1]), fmaxf(s[1][0], s[1][1]));
+                float r1 = fmaxf(fmaxf(s[0][2], s[0][3]), fmaxf(s[1][2], s[1][3]));
+                r0 = fmaxf(r0, __shfl_xor_sync(0xffffffffu, r0, 1));
+                r0 = fmaxf(r0, __shfl_xor_sync(0xffffffffu, r0, 2));
+                r1 = fmaxf(r1, __shfl_xor_sync(0xffffffffu, r1, 1));
+                r1 = fmaxf(r1, __shfl_xor_sync(0xffffffffu, r1, 2));
+                const float n0 = fmaxf(m0, r0), n1 = fmaxf(m1, r1);
+                if (__any_sync(0xffffffffu, n0 > m0 || n1 > m1)) {
+                    const float c0 = exp2f(m0 - n0), c1 = exp2f(m1 - n1);     // exp2(-inf) = 0 on the first tile
+                    l0 *= c0; l1 *= c1;
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) { o[j][0] *= c0; o[j][1] *= c0; o[j][2] *= c1; o[j][3] *= c1; }
+                    m0 = n0; m1 = n1;
+                }
+                uint32_t pa[4];
+                {
+                    const float p00 = exp2f(s[0][0] - m0), p01 = exp2f(s[0][1] - m0);
+                    const float p02 = exp2f(s[0][2] - m1), p03 = exp2f(s[0][3] - m1);
+                    const float p10 = exp2f(s[1][0] - m0), p11 = exp2f(s[1][1] - m0);
+                    const float p12 = exp2f(s[1][2] - m1), p13 = exp2f(s[1][3] - m1);
+                    l0 += (p00 + p01) + (p10 + p11);
+                    l1 += (p02 + p03) + (p12 + p13);
+                    pa[0] = pack_bf16(p00, p01); pa[1] = pack_bf16(p02, p03);
+                    pa[2] = pack_bf16(p10, p11); pa[3] = pack_bf16(p12, p13);
+                }
+#pragma unroll
+                for (int pr = 0; pr < 8; ++pr) {
+                    const int chunk = pr * 2 + v_chunk_lo;
+                    uint32_t b0, b1, b2, b3;
+                    ldmatrix_x4_trans(b0, b1, b2, b3, vbase + (chunk >> 3) * half_off + v_lane_off + (((chunk & 7) ^ lr) << 4));
+                    mma_bf16(o[2 * pr], pa, b0, b1);
+                    mma_bf16(o[2 * pr + 1], pa, b2, b3);
+                }
+                if (valid < 16) fence_proxy_async();   // our zero stores precede the next copy into this stage
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_empty(stage));
+        }
+
+        // ---- merge the eight warps of the block (fixed order), then write the piece ----
+        l0 += __shfl_xor_sync(0xffffffffu, l0, 1); l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
+        l1 += __shfl_xor_sync(0xffffffffu, l1, 1); l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
+        if (qcol == 0) {
+            s_ml[(warp * kMaxGroup + qrow) * 2] = m0;       s_ml[(warp * kMaxGroup + qrow) * 2 + 1] = l0;
+            s_ml[(warp * kMaxGroup + qrow + 8) * 2] = m1;   s_ml[(warp * kMaxGroup + qrow + 8) * 2 + 1] = l1;
+        }
+        consumer_bar();
+        float M0 = -INFINITY, M1 = -INFINITY;
+#pragma unroll
+        for (int w = 0; w < kConsumerWarps; ++w) {
+            M0 = fmaxf(M0, s_ml[(w * kMaxGroup + qrow) * 2]);
+            M1 = fmaxf(M1, s_ml[(w * kMaxGroup + qrow + 8) * 2]);
+        }
+        const float f0 = m0 == -INFINITY ? 0.f : exp2f(m0 - M0);
+        const float f1 = m1 == -INFINITY ? 0.f : exp2f(m1 - M1);
+#pragma unroll 1
+        for (int r = 0; r < kConsumerWarps; ++r) {
+            if (warp == r) {
+                float *row0 = s_merge + qrow * kMergeStride + qcol * 2;
+                float *row1 = row0 + 8 * kMergeStride;
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                    float2 a = make_float2(o[j][0] * f0, o[j][1] * f0);
+                    float2 b = make_float2(o[j][2] * f1, o[j][3] * f1);
+                    if (r > 0) {
+                        const float2 pa0 = *reinterpret_cast<float2 *>(row0 + j * 8);
+                        const float2 pb0 = *reinterpret_cast<float2 *>(row1 + j * 8);
+                        a.x += pa0.x; a.y += pa0.y; b.x += pb0.x; b.y += pb0.y;
+                    }
+                    *reinterpret_cast<float2 *>(row0 + j * 8) = a;
+                    *reinterpret_cast<float2 *>(row1 + j * 8) = b;
+                }
+            }
+            consumer_bar();
+        }
+        {
+            // thread -> (row, 8 dims): 16 rows x 16 chunks = 256 consumer threads
+            const int row = threadIdx.x >> 4, c8 = (threadIdx.x & 15) * 8;
+            if (row < g) {
+                float M = -INFINITY;
+#pragma unroll
+                for (int w = 0; w < kConsumerWarps; ++w) M = fmaxf(M, s_ml[(w * kMaxGroup + row) * 2]);
+                float lsum = 0.f;
+#pragma unroll
+                for (int w = 0; w < kConsumerWarps; ++w) {
+                    const float mw = s_ml[(w * kMaxGroup + row) * 2];
+                    if (mw != -INFINITY) lsum += s_ml[(w * kMaxGroup + row) * 2 + 1] * exp2f(mw - M);
+                }
+                const float *src = s_merge + row * kMergeStride + c8;
+                const float4 x = *reinterpret_cast<const float4 *>(src), y = *reinterpret_cast<const float4 *>(src + 4);
+                const bool whole = pc.tile0 == 0 && pc.tile1 == pc.ntiles;
+                const int bh = pc.item * hkv + pc.head;
+                if (whole) {
+                    const float inv = lsum > 0.f ? 1.f / lsum : 0.f;
+                    uint4 packed;
+                    packed.x = pack_bf16(x.x * inv, x.y * inv); packed.y = pack_bf16(x.z * inv, x.w * inv);
+                    packed.z = pack_bf16(y.x * inv, y.y * inv); packed.w = pack_bf16(y.z * inv, y.w * inv);
+                    const long long oi = (static_cast<long long>(pc.item) * prm.num_q_heads + pc.head * g + row) * kHeadDim + c8;
+                    *reinterpret_cast<uint4 *>(prm.out + oi) = packed;
+                    if (prm.lse != nullptr && c8 == 0)
+                        prm.lse[static_cast<long long>(pc.item) * prm.num_q_heads + pc.head * g + row] =
+                            lsum > 0.f ? (M + log2f(lsum)) * kLn2 : -INFINITY;
+                } else {
+                    float *slot = prm.slots + static_cast<size_t>(bh + blockIdx.x) * kSlotFloats;
+                    *reinterpret_cast<float4 *>(slot + row * kHeadDim + c8) = x;
+                    *reinterpret_cast<float4 *>(slot + row * kHeadDim + c8 + 4) = y;
+                    if (c8 == 0) { slot[kMaxGroup * kHeadDim + row] = M; slot[kMaxGroup * kHeadDim + kMaxGroup + row] = lsum; }
+                }
+            }
+            if (threadIdx.x == 0 && pc.tile0 == 0) {
+                // the block that starts an (item, head) records which blocks hold its pieces
+                const int first = p / span, last = (p + pc.ntiles - 1) / span;
+                prm.info[pc.item * hkv + pc.head] = make_int2(first, last);
+            }
+        }
+        consumer_bar();     // merge buffers are reused by the next piece
+        p += pc.tile1 - pc.tile0;
+    }
+}
+
+// Cross-split log-sum-exp combine.  One block per (item, kv head); thread d owns dim d.
+__global__ void __launch_bounds__(kHeadDim)
+combine_pieces_kernel(const DecodeParams prm) {
+    const int bh = blockIdx.x, item = bh / prm.num_kv_heads, head = bh % prm.num_kv_heads, d = threadIdx.x;
+    const int g = prm.group;
+    const int t = prm.traj_ids ? __ldg(prm.traj_ids + item) : item + prm.item_offset;
+    int L = 0;
+    if (t >= 0 && t < prm.num_traj) {
+        L = __ldg(prm.seq_lens + t);
+        if (L < 0 || L > prm.max_seq_len) L = 0;
+    }
+    const long long obase = (static_cast<long long>(item) * prm.num_q_heads + head * g) * kHeadDim + d;
+    if (L == 0) {
+        for (int r = 0; r < g; ++r) {
+            prm.out[obase + r * kHeadDim] = __float2bfloat16_rn(0.f);
+            if (prm.lse != nullptr && d == 0) prm.lse[static_cast<long long>(item) * prm.num_q_heads + head * g + r] = -INFINITY;
+        }
+        return;
+    }
+    const int2 fl = prm.info[bh];
+    if (fl.x == fl.y) return;          // a single piece: the decode kernel wrote the final result
+    for (int r = 0; r < g; ++r) {
+        float M = -INFINITY;
+        for (int i = fl.x; i <= fl.y; ++i)
+            M = fmaxf(M, __ldg(prm.slots + static_cast<size_t>(bh + i) * kSlotFloats + kMaxGroup * kHeadDim + r));
+        float acc = 0.f, lsum = 0.f;
+        if (M != -INFINITY) {
+            for (int i = fl.x; i <= fl.y; ++i) {
+                const float *slot = prm.slots + static_cast<size_t>(bh + i) * kSlotFloats;
+                const float mi = __ldg(slot + kMaxGroup * kHeadDim + r);
+                if (mi == -INFINITY) continue;
+                const float a = exp2f(mi - M);
+                acc += __ldg(slot + r * kHeadDim + d) * a;
+                lsum += __ldg(slot + kMaxGroup * kHeadDim + kMaxGroup + r) * a;
+            }
+        }
+        prm.out[obase + r * kHeadDim] = __float2bfloat16_rn(lsum > 0.f ? acc / lsum : 0.f);
+        if (prm.lse != nullptr && d == 0)
+            prm.lse[static_cast<long long>(item) * prm.num_q_heads + head * g + r] = lsum > 0.f ? (M + log2f(lsum)) * kLn2 : -INFINITY;
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// Host side: tensor maps
+// ------------------------------------------------------------------------------------------
+using EncodeTiledFn = CUresult (*)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = [] {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess)
+            p = nullptr;
+        return reinterpret_cast<EncodeTiledFn>(p);
+    }();
+    return fn;
+}
+
+bool encode_pool_map(CUtensorMap *map, const void *pool, int num_pages, int hkv, int P, bool four_d) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    const cuuint64_t units = static_cast<cuuint64_t>(num_pages) * hkv;
+    const cuuint32_t ones[4] = {1, 1, 1, 1};
+    CUresult r;
+    if (four_d) {
+        // dims: 64 elements (128 B) | slot | half of the row | (page, head); one box = one (page, head) tile,
+        // landing as [half][slot][128 B]
+        const cuuint64_t dims[4] = {64, static_cast<cuuint64_t>(P), 2, units};
+        const cuuint64_t strides[3] = {kRowBytes, 128, static_cast<cuuint64_t>(P) * kRowBytes};
+        const cuuint32_t box[4] = {64, static_cast<cuuint32_t>(P), 2, 1};
+        r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(pool), dims, strides, box, ones,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    } else {
+        const cuuint64_t dims[2] = {kHeadDim, units * P};
+        const cuuint64_t strides[1] = {kRowBytes};
+        const cuuint32_t box[2] = {64, static_cast<cuuint32_t>(P)};
+        r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(pool), dims, strides, box, ones,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    }
+    return r == CUDA_SUCCESS;
+}
+
+size_t info_bytes(int items, int hkv) { return (static_cast<size_t>(items) * hkv * sizeof(int2) + 255) & ~size_t(255); }
+
+}  // namespace
+
+size_t decode_workspace_bytes(int max_items, int num_q_heads, int num_kv_heads, int max_seq_len, int sm_count) {
+    (void)num_q_heads; (void)max_seq_len; (void)sm_count;
+    // per launch (at most kMaxItems items): one (first,last) record and one partial slot per
+    // (item, kv head), plus one slot per thread block (at most 1024 blocks)
+    const int items = max_items < kMaxItems ? max_items : kMaxItems;
+    const size_t slots = static_cast<size_t>(items) * num_kv_heads + 1024;
+    return info_bytes(items, num_kv_heads) + slots * kSlotFloats * sizeof(float);
+}
+
+cudaError_t launch_decode_attn(const AttnCall &c, cudaStream_t stream, int64_t *launches, bool *too_small) {
+    const int hkv = c.pool.num_kv_heads;
+    const int chunk_items = c.n_items < kMaxItems ? c.n_items : kMaxItems;
+    const size_t need = decode_workspace_bytes(chunk_items, c.num_q_heads, hkv, c.max_seq_len, c.sm_count);
+    if (c.workspace == nullptr || need > c.workspace_bytes) { *too_small = true; return cudaErrorInvalidValue; }
+    // the tile line of one launch must fit an int
+    const long long tiles_bound = (static_cast<long long>(c.max_seq_len) + kTile - 1) / kTile * hkv;
+    int per_launch = chunk_items;
+    while (per_launch > 1 && tiles_bound * per_launch > 0x3FFFFFFFLL) per_launch /= 2;
+
+    cudaError_t e = cudaFuncSetAttribute(decode_splitkv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    if (e != cudaSuccess) return e;
+    if (c.tma == nullptr) return cudaErrorInvalidValue;
+    TmaCache &tc = *c.tma;
+    if (!tc.valid || tc.k != c.pool.k || tc.v != c.pool.v || tc.num_pages != c.pool.num_pages || tc.hkv != hkv ||
+        tc.page_size != c.pool.page_size) {
+        CUtensorMap *km = reinterpret_cast<CUtensorMap *>(tc.kmap), *vm = reinterpret_cast<CUtensorMap *>(tc.vmap);
+        bool four = encode_pool_map(km, c.pool.k, c.pool.num_pages, hkv, c.pool.page_size, true) &&
+                    encode_pool_map(vm, c.pool.v, c.pool.num_pages, hkv, c.pool.page_size, true);
+        if (!four) {
+            if (!encode_pool_map(km, c.pool.k, c.pool.num_pages, hkv, c.pool.page_size, false) ||
+                !encode_pool_map(vm, c.pool.v, c.pool.num_pages, hkv, c.pool.page_size, false))
+                return cudaErrorInvalidValue;
+        }
+        tc.four_d = four ? 1 : 0;
+        tc.k = c.pool.k; tc.v = c.pool.v; tc.num_pages = c.pool.num_pages; tc.hkv = hkv; tc.page_size = c.pool.page_size;
+        tc.valid = true;
+    }
+
+    const int grid = c.sm_count > 0 ? (c.sm_count < 1024 ? c.sm_count : 1024) : 148;
+    for (int base = 0; base < c.n_items; base += per_launch) {
+        const int n = c.n_items - base < per_launch ? c.n_items - base : per_launch;
+        DecodeParams prm;
+        prm.page_table = c.trajs.page_table; prm.seq_lens = c.trajs.seq_lens;
+        prm.traj_ids = c.traj_ids ? c.traj_ids + base : nullptr;
+        prm.max_pages = c.trajs.max_pages; prm.num_traj = c.trajs.num_traj; prm.num_pages = c.pool.num_pages;
+        prm.page_size = c.pool.page_size; prm.num_kv_heads = hkv; prm.num_q_heads = c.num_q_heads;
+        prm.group = c.num_q_heads / hkv;
+        prm.n_items = n; prm.item_offset = base; prm.max_seq_len = c.max_seq_len; prm.four_d = tc.four_d;
+        prm.q = c.q + static_cast<long long>(base) * c.num_q_heads * kHeadDim;
+        prm.out = c.out + static_cast<long long>(base) * c.num_q_heads * kHeadDim;
+        prm.lse = c.lse ? c.lse + static_cast<long long>(base) * c.num_q_heads : nullptr;
+        prm.scale_log2 = c.sm_scale * kLog2e;
+        prm.info = static_cast<int2 *>(c.workspace);
+        prm.slots = reinterpret_cast<float *>(static_cast<char *>(c.workspace) + info_bytes(chunk_items, hkv));
+        prm.status = c.status;
+        decode_splitkv_kernel<<<grid, kThreads, kSmemBytes, stream>>>(*reinterpret_cast<CUtensorMap *>(tc.kmap),
+                                                                      *reinterpret_cast<CUtensorMap *>(tc.vmap), prm);
+        ++*launches;
+        e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+        combine_pieces_kernel<<<n * hkv, kHeadDim, 0, stream>>>(prm);
+        ++*launches;
+        e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+    }
+    return cudaSuccess;
+}
+
+}  // namespace rollart

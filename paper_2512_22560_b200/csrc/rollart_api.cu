@@ -16,6 +16,7 @@ struct rollart_ctx {
     DeviceStatus *d_status;
     DeviceStatus *h_status;  // pinned
     int64_t launches;
+    TmaCache tma;
     char err[320];
 };
 
@@ -100,6 +101,7 @@ AttnCall make_call(rollart_ctx *ctx, const rollart_kv_pool *pool, const rollart_
     c.workspace_bytes = ctx->workspace_bytes;
     c.status = ctx->d_status;
     c.sm_count = ctx->sm_count;
+    c.tma = &ctx->tma;
     return c;
 }
 

@@ -47,6 +47,16 @@ cudaError_t launch_kv_append(const rollart_kv_pool &pool, const rollart_trajs &t
                              const void *v_new, int32_t *seq_lens_out, DeviceStatus *status, cudaStream_t stream,
                              int64_t *launches);
 
+// Host-side cache of the TMA tensor maps describing the K and V pools (re-encoded when the pools change).
+struct TmaCache {
+    bool valid;
+    const void *k;
+    const void *v;
+    int num_pages, hkv, page_size, four_d;
+    alignas(64) unsigned char kmap[128];
+    alignas(64) unsigned char vmap[128];
+};
+
 struct AttnCall {
     PoolView pool;
     TrajView trajs;
@@ -64,6 +74,7 @@ struct AttnCall {
     size_t workspace_bytes;
     DeviceStatus *status;
     int sm_count;
+    TmaCache *tma;
 };
 
 size_t decode_workspace_bytes(int max_items, int num_q_heads, int num_kv_heads, int max_seq_len, int sm_count);
