@@ -156,6 +156,49 @@ rollart_status rollart_obs_chunk_attn(rollart_ctx *ctx, const rollart_kv_pool *p
                                       int32_t total_q, int32_t max_seq_len, const void *q, int32_t num_q_heads,
                                       float sm_scale, void *out, float *lse, void *stream);
 
+/*
+ * Decode attention for callers that cannot allocate device memory.  The paper has no counterpart
+ * to this call; it exists for the way the library gets embedded.
+ *
+ * Who needs it: a serving engine that has already handed every byte of device memory to its own
+ * KV-cache pool, a plug-in running inside someone else's process under a "no cudaMalloc after
+ * start-up" rule, or a latency-critical loop in which an allocation (which synchronises the
+ * device and may fail) is not acceptable.  Such a caller cannot use rollart_create, because that
+ * is where the regular path allocates its workspace.
+ *
+ * What it does: exactly what rollart_decode_attn does (same kernels, same arithmetic, same
+ * meaning of every shared argument), without a context.  The partial results, the piece records
+ * and a status word live in a fixed array of about 19.2 MB that is part of the library image:
+ * every GPU that loads the library holds that memory until the process exits, whether or not
+ * this call is ever used.  The call performs no cudaMalloc / cudaFree and calls nothing that does.
+ *
+ *   device          CUDA device that owns every [device] pointer of the call.
+ *   device_status   [device] int32[4] or NULL.  Cleared on `stream` at the start of the call;
+ *                   afterwards word 0 holds 0 or the first device-side rollart_status
+ *                   (ROLLART_ERR_BOUNDS / ROLLART_ERR_TIMEOUT), word 1 the offending value.  With
+ *                   NULL, device-side errors are recorded inside the fixed array and not reported.
+ *   err_buf/err_len [host] optional buffer that receives a NUL-terminated description whenever
+ *                   the return value is not ROLLART_OK.
+ *
+ * Limits: n_items * num_kv_heads <= 2048 and n_items <= 1024 per call.  A larger call returns
+ * ROLLART_ERR_WORKSPACE with a message that states the limit, and launches nothing; split the
+ * batch and call again.
+ *
+ * Sharing: all calls on one GPU, from every thread and stream, use the same array, and it keeps
+ * what the previous call left in it.  The call itself clears the one word that has to start at
+ * zero; nothing else is read before it is written.  Two calls whose kernels overlap on the GPU
+ * (different streams without an ordering between them) race on the array and give wrong
+ * results: keep these calls on one stream, or order the streams with events.
+ *
+ * First call on a device: it looks up the device address of the array (cudaGetSymbolAddress,
+ * with that device current) and raises the kernel's shared-memory limit.  Make this first call
+ * before starting any stream capture; later calls only enqueue work on `stream`.
+ */
+rollart_status rollart_decode_attn_noalloc(int device, const rollart_kv_pool *pool, const rollart_trajs *trajs,
+                                           const int32_t *traj_ids, int32_t n_items, int32_t max_seq_len, const void *q,
+                                           int32_t num_q_heads, float sm_scale, void *out, float *lse,
+                                           int32_t *device_status, void *stream, char *err_buf, size_t err_len);
+
 /* Synchronises `stream`, then returns and clears the device status word: ROLLART_OK, or the
  * first device-side error recorded since the last check (ROLLART_ERR_BOUNDS / _TIMEOUT), or
  * ROLLART_ERR_CUDA if the stream itself reports an error. */

@@ -20,6 +20,10 @@
 // bytes once, plus Q, O and the few partial slots.
 #include <cuda.h>
 
+#include <cstdarg>
+#include <cstdio>
+#include <mutex>
+
 #include "rollart_internal.cuh"
 
 namespace rollart {
@@ -644,3 +648,181 @@ cudaError_t launch_decode_attn(const AttnCall &c, cudaStream_t stream, int64_t *
 }
 
 }  // namespace rollart
+
+// ==========================================================================================
+// Decode attention without any allocation (rollart_decode_attn_noalloc).
+//
+// The regular entry point keeps its partial slots, piece records and status word in memory that
+// rollart_create obtained with cudaMalloc.  This variant keeps them in the fixed device array
+// below instead, so a caller that must not (or cannot) allocate device memory can still run the
+// same two kernels.  The array is part of the loaded module: every GPU that loads the library
+// holds these bytes until the process exits.
+// ==========================================================================================
+namespace rollart {
+namespace {
+
+constexpr int kStaticMaxUnits = 2048;   // n_items * num_kv_heads per call
+constexpr int kStaticMaxGrid = 256;     // thread blocks of the decode kernel in this variant
+constexpr size_t kStaticStatusBytes = 256;
+constexpr size_t kStaticInfoBytes = static_cast<size_t>(kStaticMaxUnits) * sizeof(int2);
+constexpr size_t kStaticSlotBytes = static_cast<size_t>(kStaticMaxUnits + kStaticMaxGrid) * kSlotFloats * sizeof(float);
+constexpr size_t kStaticBytes = kStaticStatusBytes + kStaticInfoBytes + kStaticSlotBytes;   // about 19.2 MB
+
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticBytes];
+
+constexpr int kMaxDevices = 64;
+struct StaticSetup {
+    bool done;
+    unsigned char *scratch;   // device address of g_static_scratch on this device
+    int sm_count;
+};
+StaticSetup g_static_setup[kMaxDevices];
+std::mutex g_static_mutex;   // guards the per-device set-up
+
+void write_err(char *buf, size_t len, const char *fmt, ...) {
+    if (!buf || len == 0) return;
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(buf, len, fmt, ap);
+    va_end(ap);
+}
+
+}  // namespace
+}  // namespace rollart
+
+extern "C" rollart_status rollart_decode_attn_noalloc(int device, const rollart_kv_pool *pool, const rollart_trajs *trajs,
+                                                      const int32_t *traj_ids, int32_t n_items, int32_t max_seq_len,
+                                                      const void *q, int32_t num_q_heads, float sm_scale, void *out,
+                                                      float *lse, int32_t *device_status, void *stream, char *err_buf,
+                                                      size_t err_len) {
+    using namespace rollart;
+    write_err(err_buf, err_len, "ok");
+    if (!pool || !trajs || !pool->k_pool || !pool->v_pool || !trajs->page_table || !trajs->seq_lens) {
+        write_err(err_buf, err_len, "pool, trajs or one of their pointers is NULL");
+        return ROLLART_ERR_INVALID_ARG;
+    }
+    if (n_items < 0 || max_seq_len < 0 || pool->num_pages <= 0 || pool->num_kv_heads <= 0 || trajs->num_traj <= 0 ||
+        trajs->max_pages_per_traj <= 0 || (n_items > 0 && (!q || !out))) {
+        write_err(err_buf, err_len, "negative or zero size, or q/out NULL");
+        return ROLLART_ERR_INVALID_ARG;
+    }
+    if (pool->head_dim != kHeadDim || (pool->page_size != 16 && pool->page_size != 32 && pool->page_size != 64)) {
+        write_err(err_buf, err_len, "head_dim %d / page_size %d unsupported (128; 16, 32 or 64)", pool->head_dim, pool->page_size);
+        return ROLLART_ERR_UNSUPPORTED;
+    }
+    const int hkv = pool->num_kv_heads;
+    if (num_q_heads <= 0 || num_q_heads % hkv != 0) {
+        write_err(err_buf, err_len, "num_q_heads %d is not a positive multiple of num_kv_heads %d", num_q_heads, hkv);
+        return ROLLART_ERR_INVALID_ARG;
+    }
+    if (num_q_heads / hkv > kMaxGroup) {
+        write_err(err_buf, err_len, "%d query heads per kv head (at most %d)", num_q_heads / hkv, kMaxGroup);
+        return ROLLART_ERR_UNSUPPORTED;
+    }
+    const uintptr_t align_bits = reinterpret_cast<uintptr_t>(pool->k_pool) | reinterpret_cast<uintptr_t>(pool->v_pool) |
+                                 reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(out);
+    if (align_bits & 15u) {
+        write_err(err_buf, err_len, "pools, q and out must be 16-byte aligned");
+        return ROLLART_ERR_INVALID_ARG;
+    }
+    if (n_items == 0) return ROLLART_OK;
+    // the fixed scratch bounds the call
+    if (n_items > kMaxItems || static_cast<long long>(n_items) * hkv > kStaticMaxUnits) {
+        write_err(err_buf, err_len,
+                  "call too large for the fixed scratch: n_items %d x num_kv_heads %d = %lld (at most %d, and at most %d items)",
+                  n_items, hkv, static_cast<long long>(n_items) * hkv, kStaticMaxUnits, kMaxItems);
+        return ROLLART_ERR_WORKSPACE;
+    }
+    const long long cap = static_cast<long long>(trajs->max_pages_per_traj) * pool->page_size;
+    if (max_seq_len > cap) max_seq_len = static_cast<int32_t>(cap > 0x7FFFFFFF ? 0x7FFFFFFF : cap);
+    if ((static_cast<long long>(max_seq_len) + kTile - 1) / kTile * hkv * n_items > 0x3FFFFFFFLL) {
+        write_err(err_buf, err_len, "n_items x num_kv_heads x max_seq_len too large for one launch");
+        return ROLLART_ERR_WORKSPACE;
+    }
+    if (device < 0 || device >= kMaxDevices) {
+        write_err(err_buf, err_len, "device %d out of range", device);
+        return ROLLART_ERR_INVALID_ARG;
+    }
+
+    int prev = -1;
+    cudaError_t e = cudaGetDevice(&prev);
+    if (e == cudaSuccess && prev != device) e = cudaSetDevice(device);
+    if (e != cudaSuccess) {
+        write_err(err_buf, err_len, "cannot select device %d: %s", device, cudaGetErrorString(e));
+        return ROLLART_ERR_CUDA;
+    }
+    rollart_status result = ROLLART_OK;
+    do {
+        StaticSetup &su = g_static_setup[device];
+        std::lock_guard<std::mutex> lock(g_static_mutex);
+        if (!su.done) {
+            // once per device, with that device current: the array's name is only a host-side handle,
+            // the kernels need the address it has on this device
+            void *ptr = nullptr;
+            e = cudaGetSymbolAddress(&ptr, g_static_scratch);
+            int major = 0, sms = 0;
+            if (e == cudaSuccess) e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, device);
+            if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device);
+            if (e == cudaSuccess)
+                e = cudaFuncSetAttribute(decode_splitkv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+            if (e != cudaSuccess || ptr == nullptr) {
+                write_err(err_buf, err_len, "set-up on device %d failed: %s", device, cudaGetErrorString(e));
+                result = ROLLART_ERR_CUDA;
+                break;
+            }
+            if (major != 10) {
+                write_err(err_buf, err_len, "device %d is not an sm_100 GPU", device);
+                result = ROLLART_ERR_UNSUPPORTED;
+                break;
+            }
+            su.scratch = static_cast<unsigned char *>(ptr);
+            su.sm_count = sms;
+            su.done = true;
+        }
+        CUtensorMap kmap, vmap;
+        bool four = encode_pool_map(&kmap, pool->k_pool, pool->num_pages, hkv, pool->page_size, true) &&
+                    encode_pool_map(&vmap, pool->v_pool, pool->num_pages, hkv, pool->page_size, true);
+        if (!four && (!encode_pool_map(&kmap, pool->k_pool, pool->num_pages, hkv, pool->page_size, false) ||
+                      !encode_pool_map(&vmap, pool->v_pool, pool->num_pages, hkv, pool->page_size, false))) {
+            write_err(err_buf, err_len, "cannot describe the pools to the copy engine (tensor map encode failed)");
+            result = ROLLART_ERR_CUDA;
+            break;
+        }
+        cudaStream_t s = static_cast<cudaStream_t>(stream);
+        DeviceStatus *status = device_status ? reinterpret_cast<DeviceStatus *>(device_status)
+                                             : reinterpret_cast<DeviceStatus *>(su.scratch);
+        // the status word must start at zero; slots and piece records are written before they are read
+        e = cudaMemsetAsync(status, 0, sizeof(DeviceStatus), s);
+        if (e != cudaSuccess) {
+            write_err(err_buf, err_len, "clearing the status word failed: %s", cudaGetErrorString(e));
+            result = ROLLART_ERR_CUDA;
+            break;
+        }
+        DecodeParams prm;
+        prm.page_table = trajs->page_table; prm.seq_lens = trajs->seq_lens; prm.traj_ids = traj_ids;
+        prm.max_pages = trajs->max_pages_per_traj; prm.num_traj = trajs->num_traj; prm.num_pages = pool->num_pages;
+        prm.page_size = pool->page_size; prm.num_kv_heads = hkv; prm.num_q_heads = num_q_heads;
+        prm.group = num_q_heads / hkv;
+        prm.n_items = n_items; prm.item_offset = 0; prm.max_seq_len = max_seq_len; prm.four_d = four ? 1 : 0;
+        prm.q = static_cast<const __nv_bfloat16 *>(q);
+        prm.out = static_cast<__nv_bfloat16 *>(out);
+        prm.lse = lse;
+        prm.scale_log2 = sm_scale * kLog2e;
+        prm.info = reinterpret_cast<int2 *>(su.scratch + kStaticStatusBytes);
+        prm.slots = reinterpret_cast<float *>(su.scratch + kStaticStatusBytes + kStaticInfoBytes);
+        prm.status = status;
+        const int grid = su.sm_count < kStaticMaxGrid ? su.sm_count : kStaticMaxGrid;
+        decode_splitkv_kernel<<<grid, kThreads, kSmemBytes, s>>>(kmap, vmap, prm);
+        e = cudaGetLastError();
+        if (e == cudaSuccess) {
+            combine_pieces_kernel<<<n_items * hkv, kHeadDim, 0, s>>>(prm);
+            e = cudaGetLastError();
+        }
+        if (e != cudaSuccess) {
+            write_err(err_buf, err_len, "kernel launch failed: %s", cudaGetErrorString(e));
+            result = ROLLART_ERR_CUDA;
+        }
+    } while (false);
+    if (prev >= 0 && prev != device) cudaSetDevice(prev);
+    return result;
+}

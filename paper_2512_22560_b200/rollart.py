@@ -21,6 +21,7 @@ _NAMES = ["OK", "ERR_INVALID_ARG", "ERR_UNSUPPORTED", "ERR_WORKSPACE", "ERR_CUDA
 EXPORTS = (
     "rollart_workspace_size", "rollart_create", "rollart_destroy", "rollart_kv_append", "rollart_decode_attn",
     "rollart_obs_chunk_attn", "rollart_check", "rollart_last_error", "rollart_launch_count",
+    "rollart_decode_attn_noalloc",
 )
 
 
@@ -67,6 +68,9 @@ def load_library() -> ctypes.CDLL:
     L.rollart_obs_chunk_attn.restype = ctypes.c_int
     L.rollart_obs_chunk_attn.argtypes = [vp, ctypes.POINTER(_KVPool), ctypes.POINTER(_Trajs), vp, vp, i32, i32, i32, vp,
                                          i32, f32, vp, vp, vp]
+    L.rollart_decode_attn_noalloc.restype = ctypes.c_int
+    L.rollart_decode_attn_noalloc.argtypes = [ctypes.c_int, ctypes.POINTER(_KVPool), ctypes.POINTER(_Trajs), vp, i32, i32,
+                                              vp, i32, f32, vp, vp, vp, vp, ctypes.c_char_p, ctypes.c_size_t]
     L.rollart_check.restype = ctypes.c_int
     L.rollart_check.argtypes = [vp, vp]
     L.rollart_last_error.restype = ctypes.c_char_p
@@ -91,6 +95,44 @@ def _ptr(t: Optional[torch.Tensor], dtype=None, device=None) -> Optional[int]:
     if device is not None and t.device.index != device:
         raise ValueError(f"tensor on cuda:{t.device.index}, context on cuda:{device}")
     return t.data_ptr()
+
+
+def decode_attn_noalloc(k_pool, v_pool, page_table, seq_lens, q, sm_scale, max_seq_len, out, lse=None, traj_ids=None,
+                        device_status=None, stream=None) -> None:
+    """rollart_decode_attn_noalloc: decode attention for callers that must not allocate device
+    memory.  No Context is involved; the scratch is a fixed array inside the library (limits:
+    n_items * num_kv_heads <= 2048, n_items <= 1024).  `device_status` is an optional int32[4]
+    CUDA tensor that receives the device-side status.  Calls that overlap on the GPU race on the
+    shared array: keep them on one stream."""
+    lib = load_library()
+    dev = k_pool.device.index
+    if k_pool.dim() != 4 or k_pool.shape != v_pool.shape:
+        raise ValueError("pools must be [num_pages][num_kv_heads][page_size][head_dim] with equal shapes")
+    n, h, p, d = k_pool.shape
+    pool = _KVPool(_ptr(k_pool, torch.bfloat16, dev), _ptr(v_pool, torch.bfloat16, dev), n, p, h, d)
+    if page_table.dim() != 2 or seq_lens.dim() != 1 or page_table.shape[0] != seq_lens.shape[0]:
+        raise ValueError("page_table must be [num_traj][max_pages], seq_lens [num_traj]")
+    trajs = _Trajs(_ptr(page_table, torch.int32, dev), page_table.shape[1], _ptr(seq_lens, torch.int32, dev),
+                   page_table.shape[0])
+    if q.dim() != 3 or q.shape != out.shape:
+        raise ValueError("q and out must be [n_items][num_q_heads][head_dim]")
+    n_items, hq, _ = q.shape
+    if traj_ids is not None and traj_ids.shape[0] != n_items:
+        raise ValueError("traj_ids must have one entry per item")
+    if lse is not None and tuple(lse.shape) != (n_items, hq):
+        raise ValueError("lse must be [n_items][num_q_heads]")
+    if device_status is not None and (device_status.numel() < 4):
+        raise ValueError("device_status must hold 4 int32")
+    if stream is None:
+        stream = torch.cuda.current_stream(dev)
+    sptr = stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
+    buf = ctypes.create_string_buffer(320)
+    st = lib.rollart_decode_attn_noalloc(
+        dev, ctypes.byref(pool), ctypes.byref(trajs), _ptr(traj_ids, torch.int32, dev), n_items, int(max_seq_len),
+        _ptr(q, torch.bfloat16, dev), hq, float(sm_scale), _ptr(out, torch.bfloat16, dev), _ptr(lse, torch.float32, dev),
+        _ptr(device_status, torch.int32, dev), sptr, buf, len(buf))
+    if st != OK:
+        raise RollartError(st, buf.value.decode())
 
 
 class Context:
