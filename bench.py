@@ -337,13 +337,13 @@ def main():
             "config": {"workload": spec.name, "trajectories_per_gpu": wl.n_items, "num_q_heads": spec.num_q_heads,
                        "num_kv_heads": spec.num_kv_heads, "page_size": spec.page_size,
                        "context_tokens_per_gpu": int(wl.lens_after_host.sum()),
-                       "step": "kv_append(1 token/trajectory) + decode_attn (split partials + LSE combine), one attention layer",
+                       "step": "kv_append(1 token/trajectory) + decode_attn (split-KV partials + last-arriver LSE combine), one attention layer",
                        "l2": "inputs larger than L2: %.2f GB of KV read per step" % (wl.bytes / 1e9),
                        "parallelism": f"replicas x{world} (independent trajectories, no collective)"},
             "hbm_gbs": achieved, "hbm_frac_of_nominal_8tbs": achieved / NOMINAL_HBM_GBS,
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                          "peak_kind": f"of {peak_kind}", "traffic": None,
-                         "kernel": "decode_attn call (partial-attention kernel + combine kernel)",
+                         "kernel": "decode_splitkv_kernel (the decode_attn call: partial attention with the split combine fused in)",
                          "algorithmic_bytes_per_launch": wl.bytes, "ms_per_launch": dec_ms},
             "e2e": {"value": n_items_all / (e2e_ms_step * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms_step,

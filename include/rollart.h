@@ -167,7 +167,7 @@ rollart_status rollart_obs_chunk_attn(rollart_ctx *ctx, const rollart_kv_pool *p
  * is where the regular path allocates its workspace.
  *
  * What it does: exactly what rollart_decode_attn does (same kernels, same arithmetic, same
- * meaning of every shared argument), without a context.  The partial results, the piece records
+ * meaning of every shared argument), without a context.  The partial results, the ticket counters
  * and a status word live in a fixed array of about 19.2 MB that is part of the library image:
  * every GPU that loads the library holds that memory until the process exits, whether or not
  * this call is ever used.  The call performs no cudaMalloc / cudaFree and calls nothing that does.
@@ -185,8 +185,8 @@ rollart_status rollart_obs_chunk_attn(rollart_ctx *ctx, const rollart_kv_pool *p
  * batch and call again.
  *
  * Sharing: all calls on one GPU, from every thread and stream, use the same array, and it keeps
- * what the previous call left in it.  The call itself clears the one word that has to start at
- * zero; nothing else is read before it is written.  Two calls whose kernels overlap on the GPU
+ * what the previous call left in it.  The call itself clears the words that have to start at
+ * zero (status and ticket counters); nothing else is read before it is written.  Two calls whose kernels overlap on the GPU
  * (different streams without an ordering between them) race on the array and give wrong
  * results: keep these calls on one stream, or order the streams with events.
  *

@@ -6,9 +6,10 @@
 // per thread block.  A block therefore reads the same number of bytes as every other block
 // whatever the length mix, and a span that crosses an (item, head) boundary simply starts a new
 // "piece".  A piece that covers its (item, head) entirely writes the final bf16 output; otherwise
-// it writes an un-normalised fp32 partial (O, m, l) into a workspace slot, and the combine kernel
-// merges the slots of that (item, head) with the log-sum-exp rule.  The cut is a fixed function
-// of the lengths, so reruns are bit identical.
+// it writes an un-normalised fp32 partial (O, m, l) into a workspace slot and takes a ticket; the
+// block that takes the last ticket of an (item, head) merges all its slots, in block order, with
+// the log-sum-exp rule (cross-split combine) and writes the output.  The cut and the merge order
+// are fixed functions of the lengths, so reruns are bit identical.
 //
 // Data path.  A producer warp walks the block's span and brings each 64-key tile of K and V
 // (32 KB) into a ring of shared-memory stages with TMA tensor copies, one box per (page, head)
@@ -53,7 +54,7 @@ constexpr int kOffLens = kOffMl + kConsumerWarps * kMaxGroup * 2 * 4;
 constexpr int kOffPrefix = kOffLens + kMaxItems * 4;
 constexpr int kOffBars = kOffPrefix + (kMaxItems + 32) * 4;
 constexpr int kNumBars = 2 * kStages + 4;
-constexpr int kOffAbort = kOffBars + kNumBars * 8;
+constexpr int kOffAbort = kOffBars + kNumBars * 8;   // abort flag, then the last-arriver flag
 constexpr int kSmemBytes = kOffAbort + 16 + 1024;    // + slack for the 1024-byte alignment
 
 struct DecodeParams {
@@ -67,7 +68,7 @@ struct DecodeParams {
     __nv_bfloat16 *out;
     float *lse;
     float scale_log2;
-    int2 *info;                 // per (item, kv head): first and last block of its pieces
+    int *tickets;               // per (item, kv head): pieces that have arrived; 0 between calls
     float *slots;
     DeviceStatus *status;
 };
@@ -144,6 +145,22 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     return *reinterpret_cast<uint32_t *>(&v);
 }
 
+// One round of the end-of-piece merge: this warp adds (or, in the first round, stores) its two
+// 8-dim accumulator tiles of one 16-dim column slice into the shared buffer.
+__device__ __forceinline__ void merge_slice(const float (&a)[4], const float (&b)[4], float f0, float f1, float *row0,
+                                            float *row1, bool add) {
+    float2 a0 = make_float2(a[0] * f0, a[1] * f0), a1 = make_float2(a[2] * f1, a[3] * f1);
+    float2 b0 = make_float2(b[0] * f0, b[1] * f0), b1 = make_float2(b[2] * f1, b[3] * f1);
+    if (add) {
+        const float2 x0 = *reinterpret_cast<float2 *>(row0), x1 = *reinterpret_cast<float2 *>(row1);
+        const float2 y0 = *reinterpret_cast<float2 *>(row0 + 8), y1 = *reinterpret_cast<float2 *>(row1 + 8);
+        a0.x += x0.x; a0.y += x0.y; a1.x += x1.x; a1.y += x1.y;
+        b0.x += y0.x; b0.y += y0.y; b1.x += y1.x; b1.y += y1.y;
+    }
+    *reinterpret_cast<float2 *>(row0) = a0; *reinterpret_cast<float2 *>(row1) = a1;
+    *reinterpret_cast<float2 *>(row0 + 8) = b0; *reinterpret_cast<float2 *>(row1 + 8) = b1;
+}
+
 // ------------------------------------------------------------------------------------------
 // The walk over a block's span of the tile line: the same code runs in the producer and in the
 // consumers, so both see the same sequence of pieces.
@@ -182,6 +199,7 @@ decode_splitkv_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
     float *s_merge = reinterpret_cast<float *>(smem + kOffMerge);
     float *s_ml = reinterpret_cast<float *>(smem + kOffMl);
     volatile int *s_abort = reinterpret_cast<volatile int *>(smem + kOffAbort);
+    volatile int *s_last = s_abort + 1;
     const uint32_t bars = smem_u32(smem + kOffBars);
     auto bar_full = [&](int s) { return bars + 8u * s; };
     auto bar_empty = [&](int s) { return bars + 8u * (kStages + s); };
@@ -231,6 +249,17 @@ decode_splitkv_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
     fence_proxy_async();      // the zeroed Q rows are ordered before the bulk copies that land beside them
     __syncthreads();
 
+    if (blockIdx.x == 0) {
+        // trajectories without keys have no tile and no piece: their result is out = 0, lse = -inf
+        for (int i = 0; i < prm.n_items; ++i) {
+            if (s_lens[i] != 0) continue;
+            uint4 *o = reinterpret_cast<uint4 *>(prm.out + static_cast<long long>(i) * prm.num_q_heads * kHeadDim);
+            for (int k = threadIdx.x; k < prm.num_q_heads * kHeadDim / 8; k += kThreads) o[k] = make_uint4(0, 0, 0, 0);
+            if (prm.lse != nullptr)
+                for (int k = threadIdx.x; k < prm.num_q_heads; k += kThreads)
+                    prm.lse[static_cast<long long>(i) * prm.num_q_heads + k] = -INFINITY;
+        }
+    }
     const int total = s_prefix[prm.n_items] * hkv;
     const int span = max(1, (total + static_cast<int>(gridDim.x) - 1) / static_cast<int>(gridDim.x));
     const int p_begin = min(total, static_cast<int>(blockIdx.x) * span);
@@ -425,27 +454,30 @@ decode_splitkv_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
         const float f1 = m1 == -INFINITY ? 0.f : exp2f(m1 - M1);
 #pragma unroll 1
         for (int r = 0; r < kConsumerWarps; ++r) {
-            if (warp == r) {
-                float *row0 = s_merge + qrow * kMergeStride + qcol * 2;
-                float *row1 = row0 + 8 * kMergeStride;
-#pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                    float2 a = make_float2(o[j][0] * f0, o[j][1] * f0);
-                    float2 b = make_float2(o[j][2] * f1, o[j][3] * f1);
-                    if (r > 0) {
-                        const float2 pa0 = *reinterpret_cast<float2 *>(row0 + j * 8);
-                        const float2 pb0 = *reinterpret_cast<float2 *>(row1 + j * 8);
-                        a.x += pa0.x; a.y += pa0.y; b.x += pb0.x; b.y += pb0.y;
-                    }
-                    *reinterpret_cast<float2 *>(row0 + j * 8) = a;
-                    *reinterpret_cast<float2 *>(row1 + j * 8) = b;
-                }
+            // in round r this warp handles the 16-dim column slice (warp + r) mod 8, so all warps work in
+            // every round and each slice receives the warps in a fixed order
+            const int c = (warp + r) & 7;
+            float *row0 = s_merge + qrow * kMergeStride + c * 16 + qcol * 2;
+            float *row1 = row0 + 8 * kMergeStride;
+            switch (c) {
+                case 0: merge_slice(o[0], o[1], f0, f1, row0, row1, r > 0); break;
+                case 1: merge_slice(o[2], o[3], f0, f1, row0, row1, r > 0); break;
+                case 2: merge_slice(o[4], o[5], f0, f1, row0, row1, r > 0); break;
+                case 3: merge_slice(o[6], o[7], f0, f1, row0, row1, r > 0); break;
+                case 4: merge_slice(o[8], o[9], f0, f1, row0, row1, r > 0); break;
+                case 5: merge_slice(o[10], o[11], f0, f1, row0, row1, r > 0); break;
+                case 6: merge_slice(o[12], o[13], f0, f1, row0, row1, r > 0); break;
+                default: merge_slice(o[14], o[15], f0, f1, row0, row1, r > 0); break;
             }
             consumer_bar();
         }
         {
             // thread -> (row, 8 dims): 16 rows x 16 chunks = 256 consumer threads
             const int row = threadIdx.x >> 4, c8 = (threadIdx.x & 15) * 8;
+            const bool whole = pc.tile0 == 0 && pc.tile1 == pc.ntiles;
+            const int bh = pc.item * hkv + pc.head;
+            const long long oi = (static_cast<long long>(pc.item) * prm.num_q_heads + pc.head * g + row) * kHeadDim + c8;
+            const long long li = static_cast<long long>(pc.item) * prm.num_q_heads + pc.head * g + row;
             if (row < g) {
                 float M = -INFINITY;
 #pragma unroll
@@ -458,18 +490,13 @@ decode_splitkv_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
                 }
                 const float *src = s_merge + row * kMergeStride + c8;
                 const float4 x = *reinterpret_cast<const float4 *>(src), y = *reinterpret_cast<const float4 *>(src + 4);
-                const bool whole = pc.tile0 == 0 && pc.tile1 == pc.ntiles;
-                const int bh = pc.item * hkv + pc.head;
                 if (whole) {
                     const float inv = lsum > 0.f ? 1.f / lsum : 0.f;
                     uint4 packed;
                     packed.x = pack_bf16(x.x * inv, x.y * inv); packed.y = pack_bf16(x.z * inv, x.w * inv);
                     packed.z = pack_bf16(y.x * inv, y.y * inv); packed.w = pack_bf16(y.z * inv, y.w * inv);
-                    const long long oi = (static_cast<long long>(pc.item) * prm.num_q_heads + pc.head * g + row) * kHeadDim + c8;
                     *reinterpret_cast<uint4 *>(prm.out + oi) = packed;
-                    if (prm.lse != nullptr && c8 == 0)
-                        prm.lse[static_cast<long long>(pc.item) * prm.num_q_heads + pc.head * g + row] =
-                            lsum > 0.f ? (M + log2f(lsum)) * kLn2 : -INFINITY;
+                    if (prm.lse != nullptr && c8 == 0) prm.lse[li] = lsum > 0.f ? (M + log2f(lsum)) * kLn2 : -INFINITY;
                 } else {
                     float *slot = prm.slots + static_cast<size_t>(bh + blockIdx.x) * kSlotFloats;
                     *reinterpret_cast<float4 *>(slot + row * kHeadDim + c8) = x;
@@ -477,56 +504,51 @@ decode_splitkv_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
                     if (c8 == 0) { slot[kMaxGroup * kHeadDim + row] = M; slot[kMaxGroup * kHeadDim + kMaxGroup + row] = lsum; }
                 }
             }
-            if (threadIdx.x == 0 && pc.tile0 == 0) {
-                // the block that starts an (item, head) records which blocks hold its pieces
-                const int first = p / span, last = (p + pc.ntiles - 1) / span;
-                prm.info[pc.item * hkv + pc.head] = make_int2(first, last);
+            if (!whole) {
+                // cross-split combine by the last block to arrive: slots are published with a fence
+                // before the ticket is taken, and read back through L2 after it
+                const int line0 = p - pc.tile0;                         // start of this (item, head) on the tile line
+                const int first = line0 / span, last = (line0 + pc.ntiles - 1) / span;
+                __threadfence();
+                consumer_bar();
+                if (threadIdx.x == 0) {
+                    const int prev = atomicAdd(prm.tickets + bh, 1);
+                    const int is_last = prev == last - first;
+                    if (is_last) prm.tickets[bh] = 0;                   // every piece has arrived: ready for the next call
+                    *s_last = is_last;
+                }
+                consumer_bar();
+                if (*s_last) {
+                    __threadfence();
+                    if (row < g) {
+                        float M = -INFINITY;
+                        for (int i = first; i <= last; ++i)
+                            M = fmaxf(M, __ldcg(prm.slots + static_cast<size_t>(bh + i) * kSlotFloats + kMaxGroup * kHeadDim + row));
+                        float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+                        float lsum = 0.f;
+                        for (int i = first; i <= last; ++i) {
+                            const float *slot = prm.slots + static_cast<size_t>(bh + i) * kSlotFloats;
+                            const float mi = __ldcg(slot + kMaxGroup * kHeadDim + row);
+                            if (mi == -INFINITY) continue;
+                            const float a = exp2f(mi - M);
+                            const float4 x = __ldcg(reinterpret_cast<const float4 *>(slot + row * kHeadDim + c8));
+                            const float4 y = __ldcg(reinterpret_cast<const float4 *>(slot + row * kHeadDim + c8 + 4));
+                            acc[0] += x.x * a; acc[1] += x.y * a; acc[2] += x.z * a; acc[3] += x.w * a;
+                            acc[4] += y.x * a; acc[5] += y.y * a; acc[6] += y.z * a; acc[7] += y.w * a;
+                            lsum += __ldcg(slot + kMaxGroup * kHeadDim + kMaxGroup + row) * a;
+                        }
+                        const float inv = lsum > 0.f ? 1.f / lsum : 0.f;
+                        uint4 packed;
+                        packed.x = pack_bf16(acc[0] * inv, acc[1] * inv); packed.y = pack_bf16(acc[2] * inv, acc[3] * inv);
+                        packed.z = pack_bf16(acc[4] * inv, acc[5] * inv); packed.w = pack_bf16(acc[6] * inv, acc[7] * inv);
+                        *reinterpret_cast<uint4 *>(prm.out + oi) = packed;
+                        if (prm.lse != nullptr && c8 == 0) prm.lse[li] = lsum > 0.f ? (M + log2f(lsum)) * kLn2 : -INFINITY;
+                    }
+                }
             }
         }
-        consumer_bar();     // merge buffers are reused by the next piece
+        consumer_bar();     // merge buffers and the flag are reused by the next piece
         p += pc.tile1 - pc.tile0;
-    }
-}
-
-// Cross-split log-sum-exp combine.  One block per (item, kv head); thread d owns dim d.
-__global__ void __launch_bounds__(kHeadDim)
-combine_pieces_kernel(const DecodeParams prm) {
-    const int bh = blockIdx.x, item = bh / prm.num_kv_heads, head = bh % prm.num_kv_heads, d = threadIdx.x;
-    const int g = prm.group;
-    const int t = prm.traj_ids ? __ldg(prm.traj_ids + item) : item + prm.item_offset;
-    int L = 0;
-    if (t >= 0 && t < prm.num_traj) {
-        L = __ldg(prm.seq_lens + t);
-        if (L < 0 || L > prm.max_seq_len) L = 0;
-    }
-    const long long obase = (static_cast<long long>(item) * prm.num_q_heads + head * g) * kHeadDim + d;
-    if (L == 0) {
-        for (int r = 0; r < g; ++r) {
-            prm.out[obase + r * kHeadDim] = __float2bfloat16_rn(0.f);
-            if (prm.lse != nullptr && d == 0) prm.lse[static_cast<long long>(item) * prm.num_q_heads + head * g + r] = -INFINITY;
-        }
-        return;
-    }
-    const int2 fl = prm.info[bh];
-    if (fl.x == fl.y) return;          // a single piece: the decode kernel wrote the final result
-    for (int r = 0; r < g; ++r) {
-        float M = -INFINITY;
-        for (int i = fl.x; i <= fl.y; ++i)
-            M = fmaxf(M, __ldg(prm.slots + static_cast<size_t>(bh + i) * kSlotFloats + kMaxGroup * kHeadDim + r));
-        float acc = 0.f, lsum = 0.f;
-        if (M != -INFINITY) {
-            for (int i = fl.x; i <= fl.y; ++i) {
-                const float *slot = prm.slots + static_cast<size_t>(bh + i) * kSlotFloats;
-                const float mi = __ldg(slot + kMaxGroup * kHeadDim + r);
-                if (mi == -INFINITY) continue;
-                const float a = exp2f(mi - M);
-                acc += __ldg(slot + r * kHeadDim + d) * a;
-                lsum += __ldg(slot + kMaxGroup * kHeadDim + kMaxGroup + r) * a;
-            }
-        }
-        prm.out[obase + r * kHeadDim] = __float2bfloat16_rn(lsum > 0.f ? acc / lsum : 0.f);
-        if (prm.lse != nullptr && d == 0)
-            prm.lse[static_cast<long long>(item) * prm.num_q_heads + head * g + r] = lsum > 0.f ? (M + log2f(lsum)) * kLn2 : -INFINITY;
     }
 }
 
@@ -581,11 +603,17 @@ size_t info_bytes(int items, int hkv) { return (static_cast<size_t>(items) * hkv
 
 size_t decode_workspace_bytes(int max_items, int num_q_heads, int num_kv_heads, int max_seq_len, int sm_count) {
     (void)num_q_heads; (void)max_seq_len; (void)sm_count;
-    // per launch (at most kMaxItems items): one (first,last) record and one partial slot per
+    // per launch (at most kMaxItems items): one ticket counter and one partial slot per
     // (item, kv head), plus one slot per thread block (at most 1024 blocks)
     const int items = max_items < kMaxItems ? max_items : kMaxItems;
     const size_t slots = static_cast<size_t>(items) * num_kv_heads + 1024;
     return info_bytes(items, num_kv_heads) + slots * kSlotFloats * sizeof(float);
+}
+
+cudaError_t decode_reset_workspace(void *workspace, size_t bytes, cudaStream_t stream) {
+    // the ticket counters sit at the start of the workspace; a kernel that gave up may have left some behind
+    const size_t n = bytes < (size_t(1) << 20) ? bytes : (size_t(1) << 20);
+    return (workspace != nullptr && n != 0) ? cudaMemsetAsync(workspace, 0, n, stream) : cudaSuccess;
 }
 
 cudaError_t launch_decode_attn(const AttnCall &c, cudaStream_t stream, int64_t *launches, bool *too_small) {
@@ -631,15 +659,11 @@ cudaError_t launch_decode_attn(const AttnCall &c, cudaStream_t stream, int64_t *
         prm.out = c.out + static_cast<long long>(base) * c.num_q_heads * kHeadDim;
         prm.lse = c.lse ? c.lse + static_cast<long long>(base) * c.num_q_heads : nullptr;
         prm.scale_log2 = c.sm_scale * kLog2e;
-        prm.info = static_cast<int2 *>(c.workspace);
+        prm.tickets = static_cast<int *>(c.workspace);
         prm.slots = reinterpret_cast<float *>(static_cast<char *>(c.workspace) + info_bytes(chunk_items, hkv));
         prm.status = c.status;
         decode_splitkv_kernel<<<grid, kThreads, kSmemBytes, stream>>>(*reinterpret_cast<CUtensorMap *>(tc.kmap),
                                                                       *reinterpret_cast<CUtensorMap *>(tc.vmap), prm);
-        ++*launches;
-        e = cudaGetLastError();
-        if (e != cudaSuccess) return e;
-        combine_pieces_kernel<<<n * hkv, kHeadDim, 0, stream>>>(prm);
         ++*launches;
         e = cudaGetLastError();
         if (e != cudaSuccess) return e;
@@ -652,10 +676,10 @@ cudaError_t launch_decode_attn(const AttnCall &c, cudaStream_t stream, int64_t *
 // ==========================================================================================
 // Decode attention without any allocation (rollart_decode_attn_noalloc).
 //
-// The regular entry point keeps its partial slots, piece records and status word in memory that
+// The regular entry point keeps its partial slots, ticket counters and status word in memory that
 // rollart_create obtained with cudaMalloc.  This variant keeps them in the fixed device array
 // below instead, so a caller that must not (or cannot) allocate device memory can still run the
-// same two kernels.  The array is part of the loaded module: every GPU that loads the library
+// same kernel.  The array is part of the loaded module: every GPU that loads the library
 // holds these bytes until the process exits.
 // ==========================================================================================
 namespace rollart {
@@ -791,10 +815,12 @@ extern "C" rollart_status rollart_decode_attn_noalloc(int device, const rollart_
         cudaStream_t s = static_cast<cudaStream_t>(stream);
         DeviceStatus *status = device_status ? reinterpret_cast<DeviceStatus *>(device_status)
                                              : reinterpret_cast<DeviceStatus *>(su.scratch);
-        // the status word must start at zero; slots and piece records are written before they are read
-        e = cudaMemsetAsync(status, 0, sizeof(DeviceStatus), s);
+        // the status word and the ticket counters must start at zero (a call that gave up part-way may have
+        // left tickets behind); slots are written before they are read
+        e = cudaMemsetAsync(su.scratch, 0, kStaticStatusBytes + kStaticInfoBytes, s);
+        if (e == cudaSuccess && device_status) e = cudaMemsetAsync(status, 0, sizeof(DeviceStatus), s);
         if (e != cudaSuccess) {
-            write_err(err_buf, err_len, "clearing the status word failed: %s", cudaGetErrorString(e));
+            write_err(err_buf, err_len, "clearing the status word and tickets failed: %s", cudaGetErrorString(e));
             result = ROLLART_ERR_CUDA;
             break;
         }
@@ -808,16 +834,12 @@ extern "C" rollart_status rollart_decode_attn_noalloc(int device, const rollart_
         prm.out = static_cast<__nv_bfloat16 *>(out);
         prm.lse = lse;
         prm.scale_log2 = sm_scale * kLog2e;
-        prm.info = reinterpret_cast<int2 *>(su.scratch + kStaticStatusBytes);
+        prm.tickets = reinterpret_cast<int *>(su.scratch + kStaticStatusBytes);
         prm.slots = reinterpret_cast<float *>(su.scratch + kStaticStatusBytes + kStaticInfoBytes);
         prm.status = status;
         const int grid = su.sm_count < kStaticMaxGrid ? su.sm_count : kStaticMaxGrid;
         decode_splitkv_kernel<<<grid, kThreads, kSmemBytes, s>>>(kmap, vmap, prm);
         e = cudaGetLastError();
-        if (e == cudaSuccess) {
-            combine_pieces_kernel<<<n_items * hkv, kHeadDim, 0, s>>>(prm);
-            e = cudaGetLastError();
-        }
         if (e != cudaSuccess) {
             write_err(err_buf, err_len, "kernel launch failed: %s", cudaGetErrorString(e));
             result = ROLLART_ERR_CUDA;

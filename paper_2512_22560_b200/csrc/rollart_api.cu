@@ -264,6 +264,8 @@ rollart_status rollart_check(rollart_ctx *ctx, void *stream) {
     if (e != cudaSuccess) return cuda_fail(ctx, e, "rollart_check");
     const DeviceStatus hs = *ctx->h_status;
     if (hs.code == 0) return ROLLART_OK;
+    decode_reset_workspace(ctx->workspace, ctx->workspace_bytes, s);
+    cudaStreamSynchronize(s);
     static const char *const where[] = {"?", "kv_append", "decode_attn", "obs_chunk_attn", "combine"};
     const char *w = (hs.where >= 0 && hs.where < 5) ? where[hs.where] : "?";
     if (hs.code == ROLLART_ERR_TIMEOUT)

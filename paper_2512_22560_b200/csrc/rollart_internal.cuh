@@ -80,6 +80,8 @@ struct AttnCall {
 size_t decode_workspace_bytes(int max_items, int num_q_heads, int num_kv_heads, int max_seq_len, int sm_count);
 // returns cudaSuccess, or cudaErrorInvalidValue with *too_small = true if the workspace cannot hold the call
 cudaError_t launch_decode_attn(const AttnCall &c, cudaStream_t stream, int64_t *launches, bool *too_small);
+// zeroes the bookkeeping at the head of the workspace after a device-side error
+cudaError_t decode_reset_workspace(void *workspace, size_t bytes, cudaStream_t stream);
 cudaError_t launch_chunk_attn(const AttnCall &c, cudaStream_t stream, int64_t *launches, bool *too_small);
 
 }  // namespace rollart
