@@ -180,7 +180,7 @@ rollart_status rollart_obs_chunk_attn(rollart_ctx *ctx, const rollart_kv_pool *p
  *   err_buf/err_len [host] optional buffer that receives a NUL-terminated description whenever
  *                   the return value is not ROLLART_OK.
  *
- * Limits: n_items * num_kv_heads <= 2048 and n_items <= 1024 per call.  A larger call returns
+ * Limits: n_items * num_kv_heads <= 2048 and n_items <= 512 per call.  A larger call returns
  * ROLLART_ERR_WORKSPACE with a message that states the limit, and launches nothing; split the
  * batch and call again.
  *

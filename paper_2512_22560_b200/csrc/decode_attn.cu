@@ -17,8 +17,10 @@
 // ids come from the page table just ahead of the copy.  Eight consumer warps in two groups take
 // alternate tiles; each warp owns 16 keys of a tile and computes, for all (up to 16) query heads
 // of the GQA group at once, S = Q K^T and O += P V with bf16 mma.sync (fp32 accumulate) and an
-// online softmax in registers.  One K/V read serves the whole group.  HBM traffic is the KV
-// bytes once, plus Q, O and the few partial slots.
+// online softmax in registers.  One K/V read serves the whole group.  At the end of a piece the
+// eight warps merge into a double-buffered shared tile and go straight on to the next piece; a
+// tenth warp writes the tile out (output or slot), takes the ticket and does the combine, off
+// the consumers' critical path.  HBM traffic is the KV bytes once, plus Q, O and the few slots.
 #include <cuda.h>
 
 #include <cstdarg>
@@ -34,8 +36,10 @@ namespace {
 constexpr int kTile = 64;                 // keys per stage
 constexpr int kStages = 6;
 constexpr int kConsumerWarps = 8;         // two groups of four
-constexpr int kThreads = (kConsumerWarps + 1) * 32;
-constexpr int kMaxItems = 1024;           // items per launch (prefix table lives in shared memory)
+constexpr int kProducerWarp = kConsumerWarps;        // warp 8 issues the copies
+constexpr int kEpilogueWarp = kConsumerWarps + 1;    // warp 9 writes pieces out and combines splits
+constexpr int kThreads = (kConsumerWarps + 2) * 32;
+constexpr int kMaxItems = 512;            // items per launch (prefix table lives in shared memory)
 constexpr int kTensorBytes = kTile * kRowBytes;      // 16 KB of K (or V) per stage
 constexpr int kStageBytes = 2 * kTensorBytes;
 constexpr int kQBytes = kMaxGroup * kRowBytes;       // 4 KB
@@ -49,12 +53,14 @@ constexpr size_t kSlotFloats = kMaxGroup * kHeadDim + 2 * kMaxGroup;
 constexpr int kOffStages = 0;
 constexpr int kOffQ = kOffStages + kStages * kStageBytes;
 constexpr int kOffMerge = kOffQ + 2 * kQBytes;
-constexpr int kOffMl = kOffMerge + kMaxGroup * kMergeStride * 4;
-constexpr int kOffLens = kOffMl + kConsumerWarps * kMaxGroup * 2 * 4;
+constexpr int kMergeFloats = kMaxGroup * kMergeStride;              // one merge buffer; there are two
+constexpr int kMlFloats = kConsumerWarps * kMaxGroup * 2;           // (m, l) of every warp and row; two copies
+constexpr int kOffMl = kOffMerge + 2 * kMergeFloats * 4;
+constexpr int kOffLens = kOffMl + 2 * kMlFloats * 4;
 constexpr int kOffPrefix = kOffLens + kMaxItems * 4;
 constexpr int kOffBars = kOffPrefix + (kMaxItems + 32) * 4;
-constexpr int kNumBars = 2 * kStages + 4;
-constexpr int kOffAbort = kOffBars + kNumBars * 8;   // abort flag, then the last-arriver flag
+constexpr int kNumBars = 2 * kStages + 8;
+constexpr int kOffAbort = kOffBars + kNumBars * 8;
 constexpr int kSmemBytes = kOffAbort + 16 + 1024;    // + slack for the 1024-byte alignment
 
 struct DecodeParams {
@@ -199,12 +205,13 @@ decode_splitkv_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
     float *s_merge = reinterpret_cast<float *>(smem + kOffMerge);
     float *s_ml = reinterpret_cast<float *>(smem + kOffMl);
     volatile int *s_abort = reinterpret_cast<volatile int *>(smem + kOffAbort);
-    volatile int *s_last = s_abort + 1;
     const uint32_t bars = smem_u32(smem + kOffBars);
     auto bar_full = [&](int s) { return bars + 8u * s; };
     auto bar_empty = [&](int s) { return bars + 8u * (kStages + s); };
     auto bar_qfull = [&](int s) { return bars + 8u * (2 * kStages + s); };
     auto bar_qempty = [&](int s) { return bars + 8u * (2 * kStages + 2 + s); };
+    auto bar_epfull = [&](int s) { return bars + 8u * (2 * kStages + 4 + s); };
+    auto bar_epempty = [&](int s) { return bars + 8u * (2 * kStages + 6 + s); };
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int hkv = prm.num_kv_heads, P = prm.page_size, g = prm.group;
@@ -227,6 +234,7 @@ decode_splitkv_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) { mbar_init(bar_full(s), 1); mbar_init(bar_empty(s), kConsumerWarps / 2); }
         for (int s = 0; s < 2; ++s) { mbar_init(bar_qfull(s), 1); mbar_init(bar_qempty(s), kConsumerWarps); }
+        for (int s = 0; s < 2; ++s) { mbar_init(bar_epfull(s), 1); mbar_init(bar_epempty(s), 1); }
         *s_abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -266,7 +274,7 @@ decode_splitkv_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
     const int p_end = min(total, p_begin + span);
     if (p_begin >= p_end) return;
 
-    if (warp == kConsumerWarps) {
+    if (warp == kProducerWarp) {
         // =============================== producer warp ===============================
         const int pages_per_tile = kTile / P;
         const uint32_t page_bytes = static_cast<uint32_t>(P) * kRowBytes;
@@ -324,6 +332,121 @@ decode_splitkv_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
                 for (uint32_t it = 0; it < kSpinLimit; ++it)
                     if (mbar_try_wait(bar_full(m % kStages), (m / kStages) & 1)) break;
             }
+        }
+        return;
+    }
+
+    if (warp == kEpilogueWarp) {
+        // =============================== epilogue warp ===============================
+        // lane -> 4 dims of a row; rows are handled one after the other
+        int pcount = 0;
+        for (int p = p_begin; p < p_end; ++pcount) {
+            const Piece pc = piece_at(s_prefix, s_lens, prm.n_items, hkv, p, p_end);
+            const int eb = pcount & 1;
+            mbar_wait(bar_epfull(eb), (pcount >> 1) & 1, s_abort, prm.status, 5);
+            const float *mg = s_merge + eb * kMergeFloats;
+            const float *ml = s_ml + eb * kMlFloats;
+            const bool whole = pc.tile0 == 0 && pc.tile1 == pc.ntiles;
+            const int bh = pc.item * hkv + pc.head;
+            const long long obase = (static_cast<long long>(pc.item) * prm.num_q_heads + pc.head * g) * kHeadDim + lane * 4;
+            const long long lbase = static_cast<long long>(pc.item) * prm.num_q_heads + pc.head * g;
+            float *slot = prm.slots + static_cast<size_t>(bh + blockIdx.x) * kSlotFloats;
+            // block-level (M, l) of every row: lane r (< 16) owns row r
+            float Mrow = -INFINITY, lrow = 0.f;
+            if (lane < kMaxGroup) {
+#pragma unroll
+                for (int w = 0; w < kConsumerWarps; ++w) Mrow = fmaxf(Mrow, ml[(w * kMaxGroup + lane) * 2]);
+#pragma unroll
+                for (int w = 0; w < kConsumerWarps; ++w) {
+                    const float mw = ml[(w * kMaxGroup + lane) * 2];
+                    if (mw != -INFINITY) lrow += ml[(w * kMaxGroup + lane) * 2 + 1] * exp2f(mw - Mrow);
+                }
+            }
+            if (whole) {
+                for (int row = 0; row < g; ++row) {
+                    const float lsum = __shfl_sync(0xffffffffu, lrow, row);
+                    const float inv = lsum > 0.f ? 1.f / lsum : 0.f;
+                    const float4 x = *reinterpret_cast<const float4 *>(mg + row * kMergeStride + lane * 4);
+                    uint2 packed;
+                    packed.x = pack_bf16(x.x * inv, x.y * inv); packed.y = pack_bf16(x.z * inv, x.w * inv);
+                    *reinterpret_cast<uint2 *>(prm.out + obase + row * kHeadDim) = packed;
+                }
+                if (prm.lse != nullptr && lane < g) prm.lse[lbase + lane] = lrow > 0.f ? (Mrow + log2f(lrow)) * kLn2 : -INFINITY;
+            } else {
+                // Cross-split combine by the last block to arrive.  A block that finds every other piece
+                // already published is the last by construction and combines straight from its shared
+                // tile; otherwise it publishes its slot (fence, then ticket) and combines only if its
+                // ticket turns out to be the last one.  Slots are merged in block order either way.
+                const int line0 = p - pc.tile0;                         // start of this (item, head) on the tile line
+                const int first = line0 / span, last = (line0 + pc.ntiles - 1) / span;
+                int arrived = 0;
+                if (lane == 0) asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(arrived) : "l"(prm.tickets + bh) : "memory");
+                arrived = __shfl_sync(0xffffffffu, arrived, 0);
+                int is_last = arrived == last - first;
+                if (!is_last) {
+                    for (int row = 0; row < g; ++row)
+                        *reinterpret_cast<float4 *>(slot + row * kHeadDim + lane * 4) =
+                            *reinterpret_cast<const float4 *>(mg + row * kMergeStride + lane * 4);
+                    if (lane < g) { slot[kMaxGroup * kHeadDim + lane] = Mrow; slot[kMaxGroup * kHeadDim + kMaxGroup + lane] = lrow; }
+                    __threadfence();
+                    __syncwarp();
+                    if (lane == 0) is_last = atomicAdd(prm.tickets + bh, 1) == last - first;
+                    is_last = __shfl_sync(0xffffffffu, is_last, 0);
+                }
+                if (is_last) {
+                    __threadfence();
+                    const int row_l = lane < g ? lane : g - 1;          // lanes >= g shadow the last row
+                    float Mall = -INFINITY, lall = 0.f;
+                    float acc[kMaxGroup][4];
+#pragma unroll
+                    for (int r = 0; r < kMaxGroup; ++r) acc[r][0] = acc[r][1] = acc[r][2] = acc[r][3] = 0.f;
+                    for (int i = first; i <= last; ++i) {
+                        const bool mine = i == static_cast<int>(blockIdx.x);
+                        const float *sl = prm.slots + static_cast<size_t>(bh + i) * kSlotFloats;
+                        float4 x[kMaxGroup];
+                        float mi, li;
+                        if (mine) {
+                            mi = __shfl_sync(0xffffffffu, Mrow, row_l);
+                            li = __shfl_sync(0xffffffffu, lrow, row_l);
+#pragma unroll
+                            for (int r = 0; r < kMaxGroup; ++r)
+                                x[r] = *reinterpret_cast<const float4 *>(mg + min(r, g - 1) * kMergeStride + lane * 4);
+                        } else {
+                            mi = __ldcg(sl + kMaxGroup * kHeadDim + row_l);
+                            li = __ldcg(sl + kMaxGroup * kHeadDim + kMaxGroup + row_l);
+#pragma unroll
+                            for (int r = 0; r < kMaxGroup; ++r)   // all loads issued back to back (rows >= g repeat row g-1)
+                                x[r] = __ldcg(reinterpret_cast<const float4 *>(sl + min(r, g - 1) * kHeadDim + lane * 4));
+                        }
+                        const float Mnew = fmaxf(Mall, mi);
+                        const float keep = Mall == -INFINITY ? 0.f : exp2f(Mall - Mnew);
+                        const float a_l = mi == -INFINITY ? 0.f : exp2f(mi - Mnew);
+                        lall = lall * keep + li * a_l;
+                        Mall = Mnew;
+#pragma unroll
+                        for (int r = 0; r < kMaxGroup; ++r) {
+                            const float k = __shfl_sync(0xffffffffu, keep, r), a = __shfl_sync(0xffffffffu, a_l, r);
+                            acc[r][0] = acc[r][0] * k + x[r].x * a; acc[r][1] = acc[r][1] * k + x[r].y * a;
+                            acc[r][2] = acc[r][2] * k + x[r].z * a; acc[r][3] = acc[r][3] * k + x[r].w * a;
+                        }
+                    }
+#pragma unroll
+                    for (int r = 0; r < kMaxGroup; ++r) {
+                        const float lsum = __shfl_sync(0xffffffffu, lall, r);
+                        if (r < g) {
+                            const float inv = lsum > 0.f ? 1.f / lsum : 0.f;
+                            uint2 packed;
+                            packed.x = pack_bf16(acc[r][0] * inv, acc[r][1] * inv); packed.y = pack_bf16(acc[r][2] * inv, acc[r][3] * inv);
+                            *reinterpret_cast<uint2 *>(prm.out + obase + r * kHeadDim) = packed;
+                        }
+                    }
+                    if (prm.lse != nullptr && lane < g) prm.lse[lbase + lane] = lall > 0.f ? (Mall + log2f(lall)) * kLn2 : -INFINITY;
+                    if (lane == 0) prm.tickets[bh] = 0;                 // every piece has arrived: ready for the next call
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_epempty(eb));      // the shared tile may be refilled
+            p += pc.tile1 - pc.tile0;
         }
         return;
     }
@@ -436,19 +559,23 @@ decode_splitkv_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
             if (lane == 0) mbar_arrive(bar_empty(stage));
         }
 
-        // ---- merge the eight warps of the block (fixed order), then write the piece ----
+        // ---- merge the eight warps into the shared tile of this piece, hand it to the epilogue warp ----
+        const int eb = pcount & 1;
+        float *mrg = s_merge + eb * kMergeFloats;
+        float *ml = s_ml + eb * kMlFloats;
+        mbar_wait(bar_epempty(eb), ((pcount >> 1) & 1) ^ 1, s_abort, prm.status, 6);
         l0 += __shfl_xor_sync(0xffffffffu, l0, 1); l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
         l1 += __shfl_xor_sync(0xffffffffu, l1, 1); l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
         if (qcol == 0) {
-            s_ml[(warp * kMaxGroup + qrow) * 2] = m0;       s_ml[(warp * kMaxGroup + qrow) * 2 + 1] = l0;
-            s_ml[(warp * kMaxGroup + qrow + 8) * 2] = m1;   s_ml[(warp * kMaxGroup + qrow + 8) * 2 + 1] = l1;
+            ml[(warp * kMaxGroup + qrow) * 2] = m0;       ml[(warp * kMaxGroup + qrow) * 2 + 1] = l0;
+            ml[(warp * kMaxGroup + qrow + 8) * 2] = m1;   ml[(warp * kMaxGroup + qrow + 8) * 2 + 1] = l1;
         }
         consumer_bar();
         float M0 = -INFINITY, M1 = -INFINITY;
 #pragma unroll
         for (int w = 0; w < kConsumerWarps; ++w) {
-            M0 = fmaxf(M0, s_ml[(w * kMaxGroup + qrow) * 2]);
-            M1 = fmaxf(M1, s_ml[(w * kMaxGroup + qrow + 8) * 2]);
+            M0 = fmaxf(M0, ml[(w * kMaxGroup + qrow) * 2]);
+            M1 = fmaxf(M1, ml[(w * kMaxGroup + qrow + 8) * 2]);
         }
         const float f0 = m0 == -INFINITY ? 0.f : exp2f(m0 - M0);
         const float f1 = m1 == -INFINITY ? 0.f : exp2f(m1 - M1);
@@ -457,7 +584,7 @@ decode_splitkv_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
             // in round r this warp handles the 16-dim column slice (warp + r) mod 8, so all warps work in
             // every round and each slice receives the warps in a fixed order
             const int c = (warp + r) & 7;
-            float *row0 = s_merge + qrow * kMergeStride + c * 16 + qcol * 2;
+            float *row0 = mrg + qrow * kMergeStride + c * 16 + qcol * 2;
             float *row1 = row0 + 8 * kMergeStride;
             switch (c) {
                 case 0: merge_slice(o[0], o[1], f0, f1, row0, row1, r > 0); break;
@@ -471,83 +598,7 @@ decode_splitkv_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
             }
             consumer_bar();
         }
-        {
-            // thread -> (row, 8 dims): 16 rows x 16 chunks = 256 consumer threads
-            const int row = threadIdx.x >> 4, c8 = (threadIdx.x & 15) * 8;
-            const bool whole = pc.tile0 == 0 && pc.tile1 == pc.ntiles;
-            const int bh = pc.item * hkv + pc.head;
-            const long long oi = (static_cast<long long>(pc.item) * prm.num_q_heads + pc.head * g + row) * kHeadDim + c8;
-            const long long li = static_cast<long long>(pc.item) * prm.num_q_heads + pc.head * g + row;
-            if (row < g) {
-                float M = -INFINITY;
-#pragma unroll
-                for (int w = 0; w < kConsumerWarps; ++w) M = fmaxf(M, s_ml[(w * kMaxGroup + row) * 2]);
-                float lsum = 0.f;
-#pragma unroll
-                for (int w = 0; w < kConsumerWarps; ++w) {
-                    const float mw = s_ml[(w * kMaxGroup + row) * 2];
-                    if (mw != -INFINITY) lsum += s_ml[(w * kMaxGroup + row) * 2 + 1] * exp2f(mw - M);
-                }
-                const float *src = s_merge + row * kMergeStride + c8;
-                const float4 x = *reinterpret_cast<const float4 *>(src), y = *reinterpret_cast<const float4 *>(src + 4);
-                if (whole) {
-                    const float inv = lsum > 0.f ? 1.f / lsum : 0.f;
-                    uint4 packed;
-                    packed.x = pack_bf16(x.x * inv, x.y * inv); packed.y = pack_bf16(x.z * inv, x.w * inv);
-                    packed.z = pack_bf16(y.x * inv, y.y * inv); packed.w = pack_bf16(y.z * inv, y.w * inv);
-                    *reinterpret_cast<uint4 *>(prm.out + oi) = packed;
-                    if (prm.lse != nullptr && c8 == 0) prm.lse[li] = lsum > 0.f ? (M + log2f(lsum)) * kLn2 : -INFINITY;
-                } else {
-                    float *slot = prm.slots + static_cast<size_t>(bh + blockIdx.x) * kSlotFloats;
-                    *reinterpret_cast<float4 *>(slot + row * kHeadDim + c8) = x;
-                    *reinterpret_cast<float4 *>(slot + row * kHeadDim + c8 + 4) = y;
-                    if (c8 == 0) { slot[kMaxGroup * kHeadDim + row] = M; slot[kMaxGroup * kHeadDim + kMaxGroup + row] = lsum; }
-                }
-            }
-            if (!whole) {
-                // cross-split combine by the last block to arrive: slots are published with a fence
-                // before the ticket is taken, and read back through L2 after it
-                const int line0 = p - pc.tile0;                         // start of this (item, head) on the tile line
-                const int first = line0 / span, last = (line0 + pc.ntiles - 1) / span;
-                __threadfence();
-                consumer_bar();
-                if (threadIdx.x == 0) {
-                    const int prev = atomicAdd(prm.tickets + bh, 1);
-                    const int is_last = prev == last - first;
-                    if (is_last) prm.tickets[bh] = 0;                   // every piece has arrived: ready for the next call
-                    *s_last = is_last;
-                }
-                consumer_bar();
-                if (*s_last) {
-                    __threadfence();
-                    if (row < g) {
-                        float M = -INFINITY;
-                        for (int i = first; i <= last; ++i)
-                            M = fmaxf(M, __ldcg(prm.slots + static_cast<size_t>(bh + i) * kSlotFloats + kMaxGroup * kHeadDim + row));
-                        float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-                        float lsum = 0.f;
-                        for (int i = first; i <= last; ++i) {
-                            const float *slot = prm.slots + static_cast<size_t>(bh + i) * kSlotFloats;
-                            const float mi = __ldcg(slot + kMaxGroup * kHeadDim + row);
-                            if (mi == -INFINITY) continue;
-                            const float a = exp2f(mi - M);
-                            const float4 x = __ldcg(reinterpret_cast<const float4 *>(slot + row * kHeadDim + c8));
-                            const float4 y = __ldcg(reinterpret_cast<const float4 *>(slot + row * kHeadDim + c8 + 4));
-                            acc[0] += x.x * a; acc[1] += x.y * a; acc[2] += x.z * a; acc[3] += x.w * a;
-                            acc[4] += y.x * a; acc[5] += y.y * a; acc[6] += y.z * a; acc[7] += y.w * a;
-                            lsum += __ldcg(slot + kMaxGroup * kHeadDim + kMaxGroup + row) * a;
-                        }
-                        const float inv = lsum > 0.f ? 1.f / lsum : 0.f;
-                        uint4 packed;
-                        packed.x = pack_bf16(acc[0] * inv, acc[1] * inv); packed.y = pack_bf16(acc[2] * inv, acc[3] * inv);
-                        packed.z = pack_bf16(acc[4] * inv, acc[5] * inv); packed.w = pack_bf16(acc[6] * inv, acc[7] * inv);
-                        *reinterpret_cast<uint4 *>(prm.out + oi) = packed;
-                        if (prm.lse != nullptr && c8 == 0) prm.lse[li] = lsum > 0.f ? (M + log2f(lsum)) * kLn2 : -INFINITY;
-                    }
-                }
-            }
-        }
-        consumer_bar();     // merge buffers and the flag are reused by the next piece
+        if (threadIdx.x == 0) mbar_arrive(bar_epfull(eb));
         p += pc.tile1 - pc.tile0;
     }
 }

@@ -101,7 +101,7 @@ def decode_attn_noalloc(k_pool, v_pool, page_table, seq_lens, q, sm_scale, max_s
                         device_status=None, stream=None) -> None:
     """rollart_decode_attn_noalloc: decode attention for callers that must not allocate device
     memory.  No Context is involved; the scratch is a fixed array inside the library (limits:
-    n_items * num_kv_heads <= 2048, n_items <= 1024).  `device_status` is an optional int32[4]
+    n_items * num_kv_heads <= 2048, n_items <= 512).  `device_status` is an optional int32[4]
     CUDA tensor that receives the device-side status.  Calls that overlap on the GPU race on the
     shared array: keep them on one stream."""
     lib = load_library()
