@@ -245,6 +245,21 @@ def _sample_tensors(layout: W.Batch, ids) -> W.Batch:
     return W.fill_tensors(b, "cpu")
 
 
+def rank_seed(seed: int, rank: int) -> int:
+    """Replicas own disjoint, independently drawn trajectories: one seed per rank."""
+    return seed + rank
+
+
+def reduce_over_ranks(dist, device, maxima, sums):
+    """Max over ranks of the timings and sum over ranks of the unit counts (identity when dist is None)."""
+    t = torch.tensor(list(maxima), dtype=torch.float64, device=device)
+    u = torch.tensor(list(sums), dtype=torch.float64, device=device)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        dist.all_reduce(u, op=dist.ReduceOp.SUM)
+    return t.tolist(), u.tolist()
+
+
 def run_reference(args):
     """`--impl reference`: the CPU oracle on a bounded sample per step (rank 0 only)."""
     rank = int(os.environ.get("RANK", "0"))
@@ -302,7 +317,7 @@ def main():
         dist.init_process_group("nccl", device_id=device)
 
     spec = W.CONFIGS[args.config]
-    wl = DecodeWorkload(spec, args.seed + rank, device)      # replicas: each rank owns its own trajectories
+    wl = DecodeWorkload(spec, rank_seed(args.seed, rank), device)      # replicas: each rank owns its own trajectories
 
     def barrier():
         if dist is not None:
@@ -318,13 +333,8 @@ def main():
     e2e_ms, h2d, d2h = wl.time_e2e(max(10, args.steps // 4), 3)
     e2e_steps = max(10, args.steps // 4)
 
-    t = torch.tensor([total_ms, dec_ms, e2e_ms / e2e_steps], dtype=torch.float64, device=device)
-    items = torch.tensor([wl.n_items], dtype=torch.float64, device=device)
-    if dist is not None:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        dist.all_reduce(items, op=dist.ReduceOp.SUM)
-    total_ms, dec_ms, e2e_ms_step = (float(x) for x in t.tolist())
-    n_items_all = float(items.item())
+    (total_ms, dec_ms, e2e_ms_step), (n_items_all,) = reduce_over_ranks(
+        dist, device, [total_ms, dec_ms, e2e_ms / e2e_steps], [wl.n_items])
     ms_per_step = total_ms / args.steps
 
     if rank == 0:

@@ -1,0 +1,125 @@
+"""Full-size workloads in the launch configuration bench.py times, checked on sampled trajectories.
+
+The whole batch runs on the GPU (append + decode, and for the mixed batch the chunk call too);
+the oracle then recomputes a sample of trajectories one by one from a host copy of just their
+pages (page renumbering does not change the oracle's result: see the permutation pin)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from harness import DeviceBatch, assert_attn_close, assert_lse_close, dev_i32, make_ctx
+from paper_2512_22560_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+
+def sample_ids(lens, ids, k, rng):
+    """shortest, longest, median and a few random members of `ids`"""
+    order = ids[np.argsort(lens[ids], kind="stable")]
+    pick = {int(order[0]), int(order[-1]), int(order[len(order) // 2])}
+    while len(pick) < min(k, len(ids)):
+        pick.add(int(rng.choice(ids)))
+    return np.array(sorted(pick), dtype=np.int64)
+
+
+@pytest.mark.parametrize("cfg", [1, 2, 3, 4])
+def test_full_size_decode_sampled(cuda_device, cfg):
+    spec = W.CONFIGS[cfg]
+    batch = W.make_batch(spec, device=cuda_device)          # the seed and shapes bench.py uses
+    ids = batch.decode_ids
+    rows = batch.decode_rows()
+    msl = int(batch.seq_lens_after[ids].max())
+    ctx = make_ctx(spec, len(ids), msl)
+    db = DeviceBatch(batch, cuda_device)
+    # append only the decode trajectories' token, exactly as the bench step does
+    ridx = torch.from_numpy(rows).to(cuda_device)
+    q = db.q_new[ridx].contiguous()
+    ctx.kv_append(db.k_pool, db.v_pool, db.page_table, db.lens_before, dev_i32(np.arange(len(ids) + 1), cuda_device),
+                  db.k_new[ridx].contiguous(), db.v_new[ridx].contiguous(), traj_ids=dev_i32(ids, cuda_device),
+                  seq_lens_out=db.lens_after)
+    lens_after = db.lens_before.clone()
+    lens_after[torch.from_numpy(ids.astype(np.int64)).to(cuda_device)] += 1
+    out = torch.full_like(q, float("nan"))
+    lse = torch.full((len(ids), spec.num_q_heads), float("nan"), device=cuda_device)
+    ctx.decode_attn(db.k_pool, db.v_pool, db.page_table, lens_after, q, spec.sm_scale, msl, out, lse=lse,
+                    traj_ids=dev_i32(ids, cuda_device))
+    ctx.check()
+    assert torch.all(torch.isfinite(out.float())) and torch.all(torch.isfinite(lse))
+    # run twice: bit-identical (fixed schedule and merge order)
+    out2 = torch.empty_like(out)
+    ctx.decode_attn(db.k_pool, db.v_pool, db.page_table, lens_after, q, spec.sm_scale, msl, out2,
+                    traj_ids=dev_i32(ids, cuda_device))
+    ctx.check()
+    assert torch.equal(out.view(torch.int16), out2.view(torch.int16))
+
+    rng = np.random.default_rng(cfg)
+    pick = sample_ids(batch.seq_lens_before, ids, 5, rng)
+    # host copy of the sampled trajectories' pages AFTER the GPU append; the oracle's append must
+    # reproduce those bytes from the pre-append pages
+    post = W.extract_trajs(db_as_batch(batch, db), pick)
+    kp, vp = W.bf16_to_u16(post.k_pool), W.bf16_to_u16(post.v_pool)
+    after = post.seq_lens_before + 1
+    pos = {int(t): i for i, t in enumerate(ids)}
+    sel = np.array([pos[int(t)] for t in pick])
+    ref_o, ref_l = oracle.decode_attn(kp, vp, post.page_table, after, W.bf16_to_u16(q[torch.from_numpy(sel).to(cuda_device)]),
+                                      spec.sm_scale)
+    assert_attn_close(out[torch.from_numpy(sel).to(cuda_device)], ref_o, spec.name)
+    assert_lse_close(lse[torch.from_numpy(sel).to(cuda_device)], ref_l, spec.name)
+    # the appended token sits where the oracle's indexing says: last logical position of each sample
+    P = spec.page_size
+    for i, t in enumerate(pick):
+        L = int(batch.seq_lens_before[t])
+        pg = int(post.page_table[i, L // P])
+        r = int(batch.new_indptr[t])
+        assert np.array_equal(kp[pg, :, L % P, :], W.bf16_to_u16(batch.k_new[r]))
+        assert np.array_equal(vp[pg, :, L % P, :], W.bf16_to_u16(batch.v_new[r]))
+    ctx.close()
+
+
+def db_as_batch(batch, db):
+    """the batch with its pools replaced by the device pools after the GPU append"""
+    import dataclasses
+    b = dataclasses.replace(batch)
+    b.k_pool, b.v_pool = db.k_pool, db.v_pool
+    return b
+
+
+
+def test_full_size_mixed_batch_chunk_sampled_rows(cuda_device):
+    spec = W.CONFIGS[4]
+    batch = W.make_batch(spec, device=cuda_device)
+    ids = batch.chunk_ids
+    rows, q_indptr = batch.chunk_rows()
+    msl = int(batch.seq_lens_after.max())
+    ctx = make_ctx(spec, len(ids), msl)
+    db = DeviceBatch(batch, cuda_device)
+    db.append(ctx)                                            # all 128 trajectories: chunks and single tokens
+    q = db.q_new[torch.from_numpy(rows).to(cuda_device)].contiguous()
+    out = torch.full_like(q, float("nan"))
+    ctx.obs_chunk_attn(db.k_pool, db.v_pool, db.page_table, db.lens_after, dev_i32(q_indptr, cuda_device), q, spec.sm_scale,
+                       msl, out, traj_ids=dev_i32(ids, cuda_device))
+    ctx.check()
+    assert torch.all(torch.isfinite(out.float()))
+    # stratified rows of three chunk trajectories: first/last row, tile edges, page edges, random
+    rng = np.random.default_rng(44)
+    order = np.argsort(batch.n_new[ids], kind="stable")
+    pick_local = sorted({int(order[0]), int(order[-1]), int(order[len(order) // 2])})
+    pick = ids[pick_local]
+    post = W.extract_trajs(db_as_batch(batch, db), pick)
+    kp, vp = W.bf16_to_u16(post.k_pool), W.bf16_to_u16(post.v_pool)
+    after = post.seq_lens_before + post.n_new
+    row_traj, row_count, q_rows = [], [], []
+    for i, li in enumerate(pick_local):
+        n = int(batch.n_new[ids[li]])
+        cand = {0, 1, n - 1, n - 2, n // 2} | {r for e in range(32, n, 128) for r in (e - 1, e, e + 1)}
+        cand |= {int(x) for x in rng.integers(0, n, size=24)}
+        for j in sorted(c for c in cand if 0 <= c < n):
+            row_traj.append(i)
+            row_count.append(int(after[i]) - n + j + 1)
+            q_rows.append(int(q_indptr[li]) + j)
+    q_rows = np.array(q_rows)
+    qsel = q[torch.from_numpy(q_rows).to(cuda_device)]
+    ref_o, _ = oracle.attend_rows(kp, vp, post.page_table, row_traj, row_count, W.bf16_to_u16(qsel), spec.sm_scale)
+    assert_attn_close(out[torch.from_numpy(q_rows).to(cuda_device)], ref_o, "cfg4 chunk rows")
+    ctx.close()
