@@ -179,6 +179,59 @@ class DecodeWorkload:
         return dt * 1e3, h2d, d2h
 
 
+def chunk_flops(spec: W.WorkloadSpec, lens_after: np.ndarray, n_new: np.ndarray) -> float:
+    """Causal-exact flops of the chunk call: every (row, visible key) pair costs 4*D per q head (QK^T and PV)."""
+    pairs = 0
+    for L, n in zip(lens_after.astype(np.int64), n_new.astype(np.int64)):
+        prior = L - n
+        pairs += n * prior + n * (n + 1) // 2
+    return float(pairs) * spec.num_q_heads * 4 * spec.head_dim
+
+
+class ChunkWorkload:
+    """The observation-chunk half of a mixed batch: bulk append of the chunks, then chunk attention."""
+
+    def __init__(self, spec: W.WorkloadSpec, seed: int, device: torch.device):
+        from paper_2512_22560_b200 import rollart
+        self.spec, self.device = spec, device
+        b = W.make_batch(spec, seed=seed, device=device)
+        self.batch = b
+        ids = b.chunk_ids
+        rows, q_indptr = b.chunk_rows()
+        i32 = lambda a: torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).to(device)
+        ridx = torch.from_numpy(rows).to(device)
+        self.table, self.lens0, self.lens1 = i32(b.page_table), i32(b.seq_lens_before), i32(b.seq_lens_after)
+        self.traj_ids, self.q_indptr = i32(ids), i32(q_indptr)
+        self.q = b.q_new[ridx].contiguous()
+        self.k_new, self.v_new = b.k_new[ridx].contiguous(), b.v_new[ridx].contiguous()
+        self.out = torch.empty_like(self.q)
+        self.max_seq_len = int(b.seq_lens_after.max())
+        self.ctx = rollart.Context(device.index or 0, rollart.workspace_size(len(ids), spec.num_q_heads, spec.num_kv_heads,
+                                                                            self.max_seq_len))
+        self.flops = chunk_flops(spec, b.seq_lens_after[ids], b.n_new[ids])
+        self.append_bytes = 2 * 2 * self.k_new.numel() * 2      # K and V rows, read + write
+        self.rows = int(self.q.shape[0])
+
+    def append(self):
+        self.ctx.kv_append(self.batch.k_pool, self.batch.v_pool, self.table, self.lens0, self.q_indptr, self.k_new, self.v_new,
+                           traj_ids=self.traj_ids, seq_lens_out=self.lens1)
+
+    def attend(self):
+        self.ctx.obs_chunk_attn(self.batch.k_pool, self.batch.v_pool, self.table, self.lens1, self.q_indptr, self.q,
+                                self.spec.sm_scale, self.max_seq_len, self.out, traj_ids=self.traj_ids)
+
+    def time(self, steps: int, warmup: int):
+        for _ in range(warmup):
+            self.append(); self.attend()
+        torch.cuda.synchronize(self.device)
+        ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(steps)]
+        for s in range(steps):
+            ev[s][0].record(); self.append(); ev[s][1].record(); self.attend(); ev[s][2].record()
+        torch.cuda.synchronize(self.device)
+        self.ctx.check()
+        return (float(np.mean([e[0].elapsed_time(e[1]) for e in ev])), float(np.mean([e[1].elapsed_time(e[2]) for e in ev])))
+
+
 class CpuBaseline:
     """The oracle, as it stands, timed on a bounded sample of the workload's trajectories."""
 
@@ -379,6 +432,25 @@ def main():
                     torch.cuda.empty_cache()
                 except Exception as e:  # report, never hide
                     extra[W.CONFIGS[ci].name] = {"error": repr(e)}
+            try:
+                cw = ChunkWorkload(W.CONFIGS[4], args.seed, device)
+                app_ms, att_ms = cw.time(5, 2)
+                tf_peak = 1399.5
+                try:
+                    with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+                        tf_peak = float(json.load(f)["bf16_tflops_sustained"])
+                except Exception:
+                    pass
+                tfs = cw.flops / (att_ms * 1e-3) / 1e12
+                extra["cfg4_mixed_multiturn_chunk_half"] = {
+                    "chunk_rows": cw.rows, "chunk_attn_ms": att_ms, "tflops": tfs, "frac_of_measured_bf16_sustained": tfs / tf_peak,
+                    "append_ms": app_ms, "append_gbs": cw.append_bytes / (app_ms * 1e-3) / 1e9,
+                    "append_frac_of_measured_hbm": cw.append_bytes / (app_ms * 1e-3) / 1e9 / peak}
+                cw.ctx.close()
+                del cw
+                torch.cuda.empty_cache()
+            except Exception as e:
+                extra["cfg4_mixed_multiturn_chunk_half"] = {"error": repr(e)}
             line["other_workloads"] = extra
             info, _, _ = CpuBaseline(spec, args.seed).measure()
             line["cpu_baseline"] = info

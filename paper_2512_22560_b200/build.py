@@ -62,6 +62,8 @@ def build(force: bool = False, verbose: bool = False, ptxas_info: bool = False) 
                     sys.stderr.write(" ".join(cmd) + "\n" + r.stdout + r.stderr)
                 if r.returncode != 0:
                     raise RuntimeError("nvcc failed for " + cmd[-3])
+    for stale in set(glob.glob(os.path.join(OBJDIR, "*.o"))) - set(objs):
+        os.remove(stale)          # object of a source file that no longer exists
     if jobs or _stale(LIB, objs):
         tmp = LIB + f".tmp{os.getpid()}"
         cmd = [nvcc, "-shared", "-o", tmp] + objs
