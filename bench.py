@@ -349,6 +349,8 @@ def main():
     ap.add_argument("--seed", type=int, default=W.MASTER_SEED)
     ap.add_argument("--ref-budget", type=float, default=12.0, help="seconds of oracle work per reference step")
     ap.add_argument("--no-extra", action="store_true", help="skip the other decode workloads and the CPU baseline")
+    ap.add_argument("--chunk", action="store_true", help="time only the observation-chunk half of --config (for profiling)")
+    ap.add_argument("--shrink", type=int, default=1, help="with --chunk: divide context lengths by this (small profiling case)")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
@@ -370,6 +372,15 @@ def main():
         dist.init_process_group("nccl", device_id=device)
 
     spec = W.CONFIGS[args.config]
+    if args.chunk:
+        if args.shrink > 1:
+            spec = W.shrink(spec, max(2, spec.num_traj // args.shrink), args.shrink)
+        cw = ChunkWorkload(spec, args.seed, device)
+        app_ms, att_ms = cw.time(args.steps, args.warmup)
+        print(json.dumps({"workload": spec.name + " (chunk half)", "chunk_rows": cw.rows, "chunk_attn_ms": att_ms,
+                          "tflops": cw.flops / (att_ms * 1e-3) / 1e12, "append_ms": app_ms,
+                          "append_gbs": cw.append_bytes / (app_ms * 1e-3) / 1e9}))
+        return 0
     wl = DecodeWorkload(spec, rank_seed(args.seed, rank), device)      # replicas: each rank owns its own trajectories
 
     def barrier():

@@ -8,14 +8,15 @@
 //   S = Q K^T      tcgen05.mma, M 128 x N 64 x K 128, operands in 128B-swizzled shared memory
 //                  (Q and K tiles brought by TMA), fp32 accumulator in TMEM, double buffered
 //   softmax        one thread per query row (4 warps = 128 TMEM lanes): tcgen05.ld its 64 scores,
-//                  scale, causal/length mask, running max m and sum l, P = exp2(s - m) as bf16
-//                  written to shared memory as the next A operand; the O accumulator in TMEM is
-//                  rescaled only when a row's max has grown by more than 2^8
-//   O += P V       tcgen05.mma, M 128 x N 128 x K 64, V is the MN-major B operand straight from
-//                  its [key][dim] page layout
+//                  scale, causal/length mask, running max m and sum l, P = exp2(s - m) as packed
+//                  bf16 stored back with tcgen05.st over the first 32 columns of the same S
+//                  buffer; the O accumulator in TMEM is rescaled only when a row's max has grown
+//                  by more than 2^8, so the softmax warps normally never wait for an MMA
+//   O += P V       tcgen05.mma with the A operand (P) in TMEM, M 128 x N 128 x K 64; V is the
+//                  MN-major B operand straight from its [key][dim] page layout
 //
 // One warp issues the copies, one warp issues the MMAs, four warps do softmax and the epilogue.
-// A block uses 113 KB of shared memory and 256 TMEM columns, so two blocks share an SM and one
+// A block uses 97 KB of shared memory and 256 TMEM columns, so two blocks share an SM and one
 // block's softmax overlaps the other's MMAs.  Blocks are ordered (item, kv head, M-tile), so the
 // M-tiles that re-read one (item, head)'s keys run together and find them in L2.
 // Every wait is a bounded mbarrier poll; no block waits for another block.
@@ -42,17 +43,16 @@ constexpr int kHalfKV = kKeys * 128;       // 8 KB: 64 keys x 64 dims
 constexpr int kOffQ = 0;                                   // [half][row][128 B]
 constexpr int kOffK = kOffQ + 2 * kHalfQ;                  // stages x [half][key][128 B]
 constexpr int kOffV = kOffK + kStages * 2 * kHalfKV;
-constexpr int kOffP = kOffV + kStages * 2 * kHalfKV;       // [row][128 B] (64 keys)
-constexpr int kOffBars = kOffP + kRows * 128;
-constexpr int kNumBars = 1 + 4 * kStages + 2 * 2 + 2;      // q | k,v full/empty | s full/empty | p_full, o_done
+constexpr int kOffBars = kOffV + kStages * 2 * kHalfKV;
+constexpr int kNumBars = 1 + 4 * kStages + 2 + 1 + 2;      // q | k,v full/empty | s_full x2 | p_full | o_done x2
 constexpr int kOffTmemSlot = kOffBars + kNumBars * 8;
 constexpr int kOffAbort = kOffTmemSlot + 8;
 constexpr int kSmemUsed = kOffAbort + 8;
-constexpr int kSmemBytes = 115712;                         // two blocks per SM: 2 x (113 KB + 1 KB reserved) = 228 KB
-static_assert(kSmemUsed + 512 <= kSmemBytes, "shared memory budget");
-static_assert((kMaxItems + 1) * 4 <= kRows * 128, "the tile prefix is staged in the P buffer");
+constexpr int kSmemBytes = kSmemUsed + 1024;               // + slack for the 1024-byte alignment; two blocks fit an SM
+static_assert(2 * (kSmemBytes + 1024) <= 228 * 1024, "two blocks per SM");
+static_assert((kMaxItems + 1) * 4 <= kStages * 2 * kHalfKV, "the tile prefix is staged in the K stages");
 
-constexpr int kTmemCols = 256;             // S0 [0,64) S1 [64,128) O [128,256)
+constexpr int kTmemCols = 256;             // S0 [0,64) S1 [64,128) O [128,256); P overwrites the first 32 columns of its S
 
 struct ChunkParams {
     const int32_t *page_table;
@@ -131,6 +131,14 @@ __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint6
         "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
         ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
 }
+// same with the A operand in TMEM (lane = row, packed 16-bit pairs along the columns)
+__device__ __forceinline__ void umma_bf16_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
 // the mbarrier gets one arrival when every MMA issued so far by this thread has completed
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
@@ -193,9 +201,9 @@ chunk_attn_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constan
     const int tpt = kRows / g;                       // chunk tokens per M-tile
     volatile int *s_abort = reinterpret_cast<volatile int *>(smem + kOffAbort);
     volatile uint32_t *s_tmem = reinterpret_cast<volatile uint32_t *>(smem + kOffTmemSlot);
-    int *s_prefix = reinterpret_cast<int *>(smem + kOffP);     // staged in the P buffer during the prologue
+    int *s_prefix = reinterpret_cast<int *>(smem + kOffK);     // staged in the K stages during the prologue
 
-    if (static_cast<int>(smem - smem_raw) + kSmemUsed > kSmemBytes) {   // cannot happen with a 512-byte aligned window
+    if (static_cast<int>(smem - smem_raw) + kSmemUsed > kSmemBytes) {   // cannot happen: the slack covers any alignment
         if (threadIdx.x == 0) report(prm.status, ROLLART_ERR_CUDA, static_cast<int>(smem - smem_raw), 3);
         return;
     }
@@ -206,9 +214,8 @@ chunk_attn_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constan
     auto bar_vfull = [&](int s) { return bars + 8u * (1 + 2 * kStages + s); };
     auto bar_vempty = [&](int s) { return bars + 8u * (1 + 3 * kStages + s); };
     auto bar_sfull = [&](int s) { return bars + 8u * (1 + 4 * kStages + s); };
-    auto bar_sempty = [&](int s) { return bars + 8u * (1 + 4 * kStages + 2 + s); };
-    const uint32_t bar_pfull = bars + 8u * (1 + 4 * kStages + 4);
-    const uint32_t bar_odone = bars + 8u * (1 + 4 * kStages + 5);
+    const uint32_t bar_pfull = bars + 8u * (1 + 4 * kStages + 2);
+    auto bar_odone = [&](int s) { return bars + 8u * (1 + 4 * kStages + 3 + s); };   // PV of tile i commits to o_done(i & 1)
 
     // ---- which (item, kv head, M-tile) is this block?  tiles per item -> prefix -> search ----
     for (int i = threadIdx.x; i < prm.n_items; i += kThreads) {
@@ -222,9 +229,8 @@ chunk_attn_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constan
             mbar_init(bar_kfull(s), 1); mbar_init(bar_kempty(s), 1);
             mbar_init(bar_vfull(s), 1); mbar_init(bar_vempty(s), 1);
         }
-        for (int s = 0; s < 2; ++s) { mbar_init(bar_sfull(s), 1); mbar_init(bar_sempty(s), 4); }
+        for (int s = 0; s < 2; ++s) { mbar_init(bar_sfull(s), 1); mbar_init(bar_odone(s), 1); }
         mbar_init(bar_pfull, 4);
-        mbar_init(bar_odone, 1);
         *s_abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -259,7 +265,7 @@ chunk_attn_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constan
         head = rem / nt;
         mtile = rem - head * nt;
     }
-    __syncthreads();                 // everyone has read the prefix: the P buffer is free again
+    __syncthreads();                 // everyone has read the prefix: the K stages are free again
     if (unit >= total_units) return;
 
     // ---- geometry of this unit ----
@@ -343,7 +349,7 @@ chunk_attn_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constan
         // =============================== MMA warp ===============================
         constexpr uint32_t kIdescQK = idesc(kKeys, false);
         constexpr uint32_t kIdescPV = idesc(kHeadDim, true);
-        const uint32_t q_addr = smem_u32(smem + kOffQ), p_addr = smem_u32(smem + kOffP);
+        const uint32_t q_addr = smem_u32(smem + kOffQ);
         auto issue_pv = [&](int i) {
             const int stage = i % kStages;
             mbar_wait(bar_vfull(stage), (i / kStages) & 1, s_abort, prm.status, 3);
@@ -352,11 +358,11 @@ chunk_attn_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constan
             if (lane == 0 && !*s_abort) {
                 const uint32_t v_addr = smem_u32(smem + kOffV + stage * 2 * kHalfKV);
 #pragma unroll
-                for (int ks = 0; ks < kKeys / 16; ++ks)   // 16 keys per step: 32 B along P's row, 2048 B down V
-                    umma_bf16(tmem + 128, smem_desc(p_addr + ks * 32, 16), smem_desc(v_addr + ks * 2048, kHalfKV), kIdescPV,
-                              (i > 0 || ks > 0) ? 1u : 0u);
+                for (int ks = 0; ks < kKeys / 16; ++ks)   // 16 keys per step: 8 packed columns along P's row, 2048 B down V
+                    umma_bf16_ts(tmem + 128, tmem + (i & 1) * kKeys + ks * 8, smem_desc(v_addr + ks * 2048, kHalfKV), kIdescPV,
+                                 (i > 0 || ks > 0) ? 1u : 0u);
                 umma_commit(bar_vempty(stage));
-                umma_commit(bar_odone);
+                umma_commit(bar_odone(i & 1));
             }
             __syncwarp();
         };
@@ -364,7 +370,7 @@ chunk_attn_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constan
         for (int j = 0; j < n_tiles; ++j) {
             const int stage = j % kStages, sb = j & 1;
             mbar_wait(bar_kfull(stage), (j / kStages) & 1, s_abort, prm.status, 6);
-            mbar_wait(bar_sempty(sb), ((j >> 1) & 1) ^ 1, s_abort, prm.status, 7);
+            // S buffer sb last held P of tile j-2; PV(j-2) was issued before this QK and MMAs run in issue order
             tc_fence_after();
             if (lane == 0 && !*s_abort) {
                 const uint32_t k_addr = smem_u32(smem + kOffK + stage * 2 * kHalfKV);
@@ -389,7 +395,6 @@ chunk_attn_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constan
         const int tok_local = row / g, head_local = row - tok_local * g;
         const bool live = tok_local < toks;
         const int count = min(L, prior + tok0 + min(tok_local, toks - 1) + 1);   // keys this row sees (>= 1)
-        const uint32_t p_row = smem_u32(smem + kOffP) + row * 128;
         float m_ref = -INFINITY, l_sum = 0.f;
 
         for (int j = 0; j < n_tiles; ++j) {
@@ -400,9 +405,6 @@ chunk_attn_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constan
             tmem_ld32(lane_addr + sb * kKeys, sraw[0]);
             tmem_ld32(lane_addr + sb * kKeys + 32, sraw[1]);
             tmem_wait_ld();
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar_sempty(sb));         // the S buffer may be overwritten by QK of tile j + 2
 
             const int key0 = j * kKeys;
             const bool need_mask = key0 + kKeys > min_count;    // uniform over the block
@@ -434,30 +436,24 @@ chunk_attn_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constan
             l_sum = l_sum * corr + rsum;
             m_ref = m_new;
 
-            if (j >= 1) {
-                // PV of the previous tile has to be finished: P is free and O holds tiles 0 .. j-1
-                mbar_wait(bar_odone, (j - 1) & 1, s_abort, prm.status, 9);
+            if (j >= 1 && __any_sync(0xffffffffu, grow)) {
+                // rare: some row of this warp moved its reference max, so O (tiles 0 .. j-1) must be rescaled
+                // before PV of this tile; PV of tile j-1 has to be finished first
+                mbar_wait(bar_odone((j - 1) & 1), ((j - 1) >> 1) & 1, s_abort, prm.status, 9);
                 tc_fence_after();
-                if (__any_sync(0xffffffffu, grow)) {
 #pragma unroll 1
-                    for (int c0 = 0; c0 < kHeadDim; c0 += 32) {
-                        uint32_t oraw[32];
-                        tmem_ld32(lane_addr + 128 + c0, oraw);
-                        tmem_wait_ld();
+                for (int c0 = 0; c0 < kHeadDim; c0 += 32) {
+                    uint32_t oraw[32];
+                    tmem_ld32(lane_addr + 128 + c0, oraw);
+                    tmem_wait_ld();
 #pragma unroll
-                        for (int c = 0; c < 32; ++c) oraw[c] = __float_as_uint(__uint_as_float(oraw[c]) * corr);
-                        tmem_st32(lane_addr + 128 + c0, oraw);
-                    }
-                    tmem_wait_st();
+                    for (int c = 0; c < 32; ++c) oraw[c] = __float_as_uint(__uint_as_float(oraw[c]) * corr);
+                    tmem_st32(lane_addr + 128 + c0, oraw);
                 }
             }
-            // P as the next A operand: row `row`, 8 chunks of 8 keys, 128B swizzle
-#pragma unroll
-            for (int c = 0; c < 8; ++c) {
-                const uint32_t a = p_row + ((c ^ (row & 7)) << 4);
-                asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(a), "r"(packed[4 * c]), "r"(packed[4 * c + 1]),
-                             "r"(packed[4 * c + 2]), "r"(packed[4 * c + 3]) : "memory");
-            }
+            // P as the next A operand: 64 bf16 of this row as 32 packed columns over the start of its S buffer
+            tmem_st32(lane_addr + sb * kKeys, packed);
+            tmem_wait_st();
             if (key0 + kKeys > L) {
                 // keys at or beyond L are dead slots (or were never copied): their V rows must be 0, not garbage
                 mbar_wait(bar_vfull(j % kStages), (j / kStages) & 1, s_abort, prm.status, 10);
@@ -468,15 +464,15 @@ chunk_attn_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constan
                     asm volatile("st.shared.v4.b32 [%0], {%1,%1,%1,%1};" ::"r"(v_addr + (c >> 3) * kHalfKV + r * 128 + (c & 7) * 16),
                                  "r"(0) : "memory");
                 }
+                fence_proxy_async();      // the zeroed V rows become visible to the tensor core's reads
             }
-            fence_proxy_async();          // P (and the zeroed V rows) become visible to the tensor core's reads
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_pfull);
         }
 
         // ---- epilogue: O / l -> bf16 rows of out ----
-        mbar_wait(bar_odone, (n_tiles - 1) & 1, s_abort, prm.status, 11);
+        mbar_wait(bar_odone((n_tiles - 1) & 1), ((n_tiles - 1) >> 1) & 1, s_abort, prm.status, 11);
         tc_fence_after();
         const float inv = l_sum > 0.f ? 1.f / l_sum : 0.f;
         const long long orow = (static_cast<long long>(q_row0 + tok0 + tok_local) * prm.num_q_heads + head * g + head_local);
