@@ -33,7 +33,7 @@ constexpr int kKeys = 64;                  // keys per KV tile
 constexpr int kStages = 2;
 constexpr int kThreads = 192;              // warp 0 copies, warp 1 MMA, warps 2-5 softmax
 constexpr int kMaxItems = 1024;            // items per launch (tile prefix lives in shared memory)
-constexpr uint32_t kSpinLimit = 1u << 22;
+constexpr uint32_t kSpinLimit = 1u << 20;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 constexpr float kRescaleThreshold = 8.f;   // log2 units
@@ -44,7 +44,7 @@ constexpr int kOffQ = 0;                                   // [half][row][128 B]
 constexpr int kOffK = kOffQ + 2 * kHalfQ;                  // stages x [half][key][128 B]
 constexpr int kOffV = kOffK + kStages * 2 * kHalfKV;
 constexpr int kOffBars = kOffV + kStages * 2 * kHalfKV;
-constexpr int kNumBars = 1 + 4 * kStages + 2 + 1 + 2;      // q | k,v full/empty | s_full x2 | p_full | o_done x2
+constexpr int kNumBars = 1 + 4 * kStages + 2 + 2 + 2;      // q | k,v full/empty | s_full x2 | p_full x2 | o_done x2
 constexpr int kOffTmemSlot = kOffBars + kNumBars * 8;
 constexpr int kOffAbort = kOffTmemSlot + 8;
 constexpr int kSmemUsed = kOffAbort + 8;
@@ -100,6 +100,7 @@ __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatil
     if (*abort_flag == 0) {
         *abort_flag = 1;
         report(status, ROLLART_ERR_TIMEOUT, where, 3);
+        status->fatal = 1;         // later blocks of this launch do not start
     }
 }
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int x, int y) {
@@ -214,8 +215,9 @@ chunk_attn_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constan
     auto bar_vfull = [&](int s) { return bars + 8u * (1 + 2 * kStages + s); };
     auto bar_vempty = [&](int s) { return bars + 8u * (1 + 3 * kStages + s); };
     auto bar_sfull = [&](int s) { return bars + 8u * (1 + 4 * kStages + s); };
-    const uint32_t bar_pfull = bars + 8u * (1 + 4 * kStages + 2);
-    auto bar_odone = [&](int s) { return bars + 8u * (1 + 4 * kStages + 3 + s); };   // PV of tile i commits to o_done(i & 1)
+    // tile i uses p_full(i & 1) and o_done(i & 1): a warp that is a tile ahead of the others arrives on the other barrier
+    auto bar_pfull = [&](int s) { return bars + 8u * (1 + 4 * kStages + 2 + s); };
+    auto bar_odone = [&](int s) { return bars + 8u * (1 + 4 * kStages + 4 + s); };
 
     // ---- which (item, kv head, M-tile) is this block?  tiles per item -> prefix -> search ----
     for (int i = threadIdx.x; i < prm.n_items; i += kThreads) {
@@ -229,8 +231,7 @@ chunk_attn_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constan
             mbar_init(bar_kfull(s), 1); mbar_init(bar_kempty(s), 1);
             mbar_init(bar_vfull(s), 1); mbar_init(bar_vempty(s), 1);
         }
-        for (int s = 0; s < 2; ++s) { mbar_init(bar_sfull(s), 1); mbar_init(bar_odone(s), 1); }
-        mbar_init(bar_pfull, 4);
+        for (int s = 0; s < 2; ++s) { mbar_init(bar_sfull(s), 1); mbar_init(bar_odone(s), 1); mbar_init(bar_pfull(s), 4); }
         *s_abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -267,6 +268,7 @@ chunk_attn_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constan
     }
     __syncthreads();                 // everyone has read the prefix: the K stages are free again
     if (unit >= total_units) return;
+    if (*reinterpret_cast<volatile int *>(&prm.status->fatal) != 0) return;   // an earlier block ran out of patience: give up quickly
 
     // ---- geometry of this unit ----
     const int q_row0 = __ldg(prm.q_indptr + item);
@@ -353,7 +355,7 @@ chunk_attn_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constan
         auto issue_pv = [&](int i) {
             const int stage = i % kStages;
             mbar_wait(bar_vfull(stage), (i / kStages) & 1, s_abort, prm.status, 3);
-            mbar_wait(bar_pfull, i & 1, s_abort, prm.status, 4);
+            mbar_wait(bar_pfull(i & 1), (i >> 1) & 1, s_abort, prm.status, 4);
             tc_fence_after();
             if (lane == 0 && !*s_abort) {
                 const uint32_t v_addr = smem_u32(smem + kOffV + stage * 2 * kHalfKV);
@@ -468,7 +470,7 @@ chunk_attn_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constan
             }
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(bar_pfull);
+            if (lane == 0) mbar_arrive(bar_pfull(sb));
         }
 
         // ---- epilogue: O / l -> bf16 rows of out ----

@@ -18,7 +18,7 @@ struct DeviceStatus {
     int code;
     int detail;
     int where;
-    int pad;
+    int fatal;   // set with a timeout: blocks that have not started yet return at once
 };
 
 __device__ __forceinline__ void report(DeviceStatus *st, int code, int detail, int where) {
