@@ -171,6 +171,29 @@ __device__ __forceinline__ float ex2(float x) {
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
+// three-input max and two-wide fp32 FMA / ADD: half the instructions of the scalar forms
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+__device__ __forceinline__ float min3(float a, float b, float c) {
+    float d;
+    asm("min.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+__device__ __forceinline__ void fma2(float &d0, float &d1, float a0, float a1, float b, float c) {   // d = a * b + c, two lanes
+    asm("{\n\t.reg .b64 ra, rb, rc, rd;\n\t"
+        "mov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %4};\n\tmov.b64 rc, {%5, %5};\n\t"
+        "fma.rn.f32x2 rd, ra, rb, rc;\n\tmov.b64 {%0, %1}, rd;\n\t}"
+        : "=f"(d0), "=f"(d1) : "f"(a0), "f"(a1), "f"(b), "f"(c));
+}
+__device__ __forceinline__ void add2(float &d0, float &d1, float a0, float a1) {                      // d += a, two lanes
+    asm("{\n\t.reg .b64 ra, rd;\n\t"
+        "mov.b64 ra, {%2, %3};\n\tmov.b64 rd, {%0, %1};\n\t"
+        "add.rn.f32x2 rd, rd, ra;\n\tmov.b64 {%0, %1}, rd;\n\t}"
+        : "+f"(d0), "+f"(d1) : "f"(a0), "f"(a1));
+}
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t *>(&v);
@@ -410,31 +433,62 @@ chunk_attn_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constan
 
             const int key0 = j * kKeys;
             const bool need_mask = key0 + kKeys > min_count;    // uniform over the block
-            float s[2][32];
-            float rmax = -INFINITY;
+            const float scale = prm.scale_log2;
+            float rmax;
+            if (!need_mask) {
+                // the max of scale * s is scale * (max or min of s): take the extreme of the raw scores, 8 chains of 3-input ops
+                float e[8];
+                if (scale >= 0.f) {
 #pragma unroll
-            for (int h = 0; h < 2; ++h)
+                    for (int k = 0; k < 8; ++k) e[k] = max3(__uint_as_float(sraw[0][k]), __uint_as_float(sraw[0][8 + k]), __uint_as_float(sraw[0][16 + k]));
 #pragma unroll
-                for (int c = 0; c < 32; ++c) {
-                    float x = __uint_as_float(sraw[h][c]) * prm.scale_log2;
-                    if (need_mask && key0 + h * 32 + c >= count) x = -INFINITY;
-                    s[h][c] = x;
-                    rmax = fmaxf(rmax, x);
+                    for (int k = 0; k < 8; ++k) e[k] = max3(e[k], __uint_as_float(sraw[0][24 + k]), __uint_as_float(sraw[1][k]));
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) e[k] = max3(e[k], __uint_as_float(sraw[1][8 + k]), __uint_as_float(sraw[1][16 + k]));
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) e[k] = fmaxf(e[k], __uint_as_float(sraw[1][24 + k]));
+                    rmax = max3(max3(e[0], e[1], e[2]), max3(e[3], e[4], e[5]), fmaxf(e[6], e[7])) * scale;
+                } else {
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) e[k] = min3(__uint_as_float(sraw[0][k]), __uint_as_float(sraw[0][8 + k]), __uint_as_float(sraw[0][16 + k]));
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) e[k] = min3(e[k], __uint_as_float(sraw[0][24 + k]), __uint_as_float(sraw[1][k]));
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) e[k] = min3(e[k], __uint_as_float(sraw[1][8 + k]), __uint_as_float(sraw[1][16 + k]));
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) e[k] = fminf(e[k], __uint_as_float(sraw[1][24 + k]));
+                    rmax = min3(min3(e[0], e[1], e[2]), min3(e[3], e[4], e[5]), fminf(e[6], e[7])) * scale;
                 }
+            } else {
+                rmax = -INFINITY;
+#pragma unroll
+                for (int h = 0; h < 2; ++h)
+#pragma unroll
+                    for (int c = 0; c < 32; ++c)
+                        if (key0 + h * 32 + c < count) rmax = fmaxf(rmax, __uint_as_float(sraw[h][c]) * scale);
+            }
             // the reference max moves only when it has to (first tile) or when a row outgrew it by 2^8
             const bool grow = rmax > m_ref + kRescaleThreshold;
             const float m_new = grow ? rmax : m_ref;
             const float corr = grow ? ex2(m_ref - m_new) : 1.f;   // ex2(-inf) = 0 on the first tile
-            float rsum = 0.f;
+            const float neg_m = -m_new;
+            float rs[4] = {0.f, 0.f, 0.f, 0.f};
             uint32_t packed[32];
 #pragma unroll
             for (int h = 0; h < 2; ++h)
 #pragma unroll
                 for (int c = 0; c < 32; c += 2) {
-                    const float p0 = ex2(s[h][c] - m_new), p1 = ex2(s[h][c + 1] - m_new);
-                    rsum += p0 + p1;
+                    float x0, x1;
+                    fma2(x0, x1, __uint_as_float(sraw[h][c]), __uint_as_float(sraw[h][c + 1]), scale, neg_m);
+                    float p0 = ex2(x0), p1 = ex2(x1);
+                    if (need_mask) {
+                        p0 = key0 + h * 32 + c < count ? p0 : 0.f;
+                        p1 = key0 + h * 32 + c + 1 < count ? p1 : 0.f;
+                    }
+                    add2(rs[c & 2], rs[(c & 2) + 1], p0, p1);
                     packed[h * 16 + (c >> 1)] = pack_bf16(p0, p1);
                 }
+            const float rsum = (rs[0] + rs[1]) + (rs[2] + rs[3]);
             l_sum = l_sum * corr + rsum;
             m_ref = m_new;
 
