@@ -33,7 +33,8 @@ constexpr int kKeys = 64;                  // keys per KV tile
 constexpr int kStages = 2;
 constexpr int kThreads = 192;              // warp 0 copies, warp 1 MMA, warps 2-5 softmax
 constexpr int kMaxItems = 1024;            // items per launch (tile prefix lives in shared memory)
-constexpr uint32_t kSpinLimit = 1u << 20;
+constexpr uint32_t kSpinLimit = 1u << 17;   // polls per wait; each poll sleeps in hardware for up to kSuspendNs
+constexpr uint32_t kSuspendNs = 10000;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 constexpr float kRescaleThreshold = 8.f;   // log2 units
@@ -84,9 +85,9 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+        : "=r"(ok) : "r"(bar), "r"(parity), "r"(kSuspendNs) : "memory");
     return ok != 0;
 }
 // Bounded wait; once any thread of the block has given up, nobody waits any more, so every role
@@ -95,7 +96,7 @@ __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatil
                                           int where) {
     for (uint32_t it = 0; it < kSpinLimit; ++it) {
         if (mbar_try_wait(bar, parity)) return;
-        if ((it & 1023u) == 1023u && *abort_flag) return;
+        if (*abort_flag) return;
     }
     if (*abort_flag == 0) {
         *abort_flag = 1;

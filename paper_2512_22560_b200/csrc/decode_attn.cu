@@ -44,7 +44,8 @@ constexpr int kTensorBytes = kTile * kRowBytes;      // 16 KB of K (or V) per st
 constexpr int kStageBytes = 2 * kTensorBytes;
 constexpr int kQBytes = kMaxGroup * kRowBytes;       // 4 KB
 constexpr int kMergeStride = kHeadDim + 8;           // floats per merge-buffer row (padded)
-constexpr uint32_t kSpinLimit = 1u << 22;
+constexpr uint32_t kSpinLimit = 1u << 17;   // polls per wait; each poll sleeps in hardware for up to kSuspendNs
+constexpr uint32_t kSuspendNs = 10000;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 constexpr size_t kSlotFloats = kMaxGroup * kHeadDim + 2 * kMaxGroup;
@@ -97,9 +98,9 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+        : "=r"(ok) : "r"(bar), "r"(parity), "r"(kSuspendNs) : "memory");
     return ok != 0;
 }
 // Bounded wait.  Gives up when the limit runs out or another warp has already given up; the
@@ -108,7 +109,7 @@ __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatil
                                           int where) {
     for (uint32_t it = 0; it < kSpinLimit; ++it) {
         if (mbar_try_wait(bar, parity)) return;
-        if ((it & 1023u) == 1023u && *abort_flag) return;
+        if (*abort_flag) return;
     }
     if (*abort_flag == 0) {
         *abort_flag = 1;
