@@ -462,6 +462,16 @@ def main():
                 torch.cuda.empty_cache()
             except Exception as e:
                 extra["cfg4_mixed_multiturn_chunk_half"] = {"error": repr(e)}
+            try:
+                rw = ChunkWorkload(W.RECOMPUTE, args.seed, device)
+                app_ms, att_ms = rw.time(3, 2)
+                extra[W.RECOMPUTE.name] = {"rows": rw.rows, "chunk_attn_ms": att_ms, "tflops": rw.flops / (att_ms * 1e-3) / 1e12,
+                                           "append_ms": app_ms, "append_gbs": rw.append_bytes / (app_ms * 1e-3) / 1e9}
+                rw.ctx.close()
+                del rw
+                torch.cuda.empty_cache()
+            except Exception as e:
+                extra[W.RECOMPUTE.name] = {"error": repr(e)}
             line["other_workloads"] = extra
             info, _, _ = CpuBaseline(spec, args.seed).measure()
             line["cpu_baseline"] = info

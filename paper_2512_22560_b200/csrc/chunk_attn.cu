@@ -288,7 +288,7 @@ chunk_attn_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constan
         const int nt = max(1, s_prefix[lo + 1] - s_prefix[lo]);
         const int rem = unit - s_prefix[lo] * hkv;
         head = rem / nt;
-        mtile = rem - head * nt;
+        mtile = nt - 1 - (rem - head * nt);     // later M-tiles see more keys: start the longest ones first
     }
     __syncthreads();                 // everyone has read the prefix: the K stages are free again
     if (unit >= total_units) return;

@@ -50,6 +50,7 @@ class WorkloadSpec:
     chunk_fraction: float = 0.0   # fraction of trajectories that receive an observation chunk
     chunk_lo: int = 64
     chunk_hi: int = 2048
+    recompute: bool = False       # every trajectory re-enters with its whole context as one chunk (empty cache before)
     k_scale: float = 1.0          # multiplier on K data
     sm_scale: float = 1.0 / math.sqrt(HEAD_DIM)
     spare_pages: float = 0.125
@@ -66,6 +67,12 @@ CONFIGS = (
     WorkloadSpec("cfg4_mixed_multiturn", 128, 32, 8, 16, "uniform", len_lo=1024, len_hi=24576,
                  chunk_fraction=0.5, chunk_lo=64, chunk_hi=2048),
 )
+
+
+# KV-cache recomputation after a weight update (Sec. 6.2, step "recomp" of the asynchronous training
+# protocol): every in-flight trajectory rebuilds its cache, i.e. a causal prefill of its whole context
+# onto empty pages.  Same calls as the observation chunk, with no prior context.
+RECOMPUTE = WorkloadSpec("recompute_inflight", 16, 32, 8, 16, "uniform", len_lo=4096, len_hi=32768, recompute=True)
 
 
 def shrink(spec: WorkloadSpec, num_traj: int, len_div: int, chunk_div: int = 1) -> WorkloadSpec:
@@ -194,6 +201,10 @@ def make_layout(spec: WorkloadSpec, seed: int = MASTER_SEED) -> Batch:
         ids = rng.permutation(T)[:n_chunk]
         is_chunk[ids] = True
         n_new[ids] = rng.integers(spec.chunk_lo, spec.chunk_hi + 1, size=n_chunk)
+    if spec.recompute:
+        n_new = lens.copy()
+        lens = np.zeros(T, dtype=np.int32)
+        is_chunk[:] = True
     new_indptr = np.zeros(T + 1, dtype=np.int32)
     new_indptr[1:] = np.cumsum(n_new)
     pages = (lens.astype(np.int64) + n_new + spec.page_size - 1) // spec.page_size

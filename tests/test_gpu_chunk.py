@@ -41,6 +41,13 @@ def test_shrunk_mixed_batch_chunk_half(cuda_device):
     run_chunk_case(W.make_batch(W.shrink(W.CONFIGS[4], 8, 16, 8), seed=41), cuda_device)
 
 
+def test_recompute_from_empty_cache(cuda_device):
+    # KV recomputation: whole contexts as one causal chunk onto empty pages (prior = 0)
+    batch = W.make_batch(W.shrink(W.RECOMPUTE, 5, 16), seed=46)
+    assert batch.seq_lens_before.max() == 0 and batch.is_chunk.all()
+    run_chunk_case(batch, cuda_device)
+
+
 @pytest.mark.parametrize("P,hq,hkv", [(16, 8, 2), (32, 7, 1), (64, 16, 1), (16, 3, 3)])
 def test_chunk_edges(cuda_device, P, hq, hkv):
     prior = [0, 0, 1, P - 1, P, 5, 130, 64]
