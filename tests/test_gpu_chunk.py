@@ -102,3 +102,10 @@ def test_chunk_longer_than_trajectory_is_a_device_error(cuda_device):
     lens = dev_i32([10, 50], cuda_device)
     ctx.obs_chunk_attn(db.k_pool, db.v_pool, db.page_table, lens, dev_i32([0, 20, 40], cuda_device), q, 0.1, 100, out)
     assert ctx.status() == rollart.ERR_BOUNDS and "obs_chunk_attn" in ctx.last_error()
+
+
+def test_many_small_chunks_span_several_launches(cuda_device):
+    # 1100 chunk items of 1..5 tokens: more items than one launch's tile table holds, ragged single-tile units
+    spec = dataclasses.replace(W.CONFIGS[0], num_traj=1100, len_lo=1, len_hi=40, chunk_fraction=1.0, chunk_lo=1, chunk_hi=5,
+                               name="many_chunks")
+    run_chunk_case(W.make_batch(spec, seed=72), cuda_device)

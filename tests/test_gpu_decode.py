@@ -151,3 +151,9 @@ def test_host_side_validation(cuda_device):
         ctx.decode_attn(db.k_pool[:, :3].contiguous(), db.v_pool[:, :3].contiguous(), db.page_table, db.lens_before, q,
                         0.1, 8000, out)
     assert e.value.status == rollart.ERR_INVALID_ARG
+
+
+def test_more_items_than_one_launch_holds(cuda_device):
+    # 1300 short trajectories: the decode call splits into several launches (the per-launch length table is bounded)
+    spec = dataclasses.replace(W.CONFIGS[0], num_traj=1300, len_lo=1, len_hi=90, name="many_items")
+    run_decode_case(W.make_batch(spec, seed=71), cuda_device)
