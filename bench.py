@@ -42,6 +42,11 @@ def measured_peaks():
     return FALLBACK_HBM_GBS, "fallback"
 
 
+# dram__bytes_read.sum + dram__bytes_write.sum of one decode_splitkv_kernel launch, from the ncu capture summarised in
+# profiles/decode_splitkv_cfg1.md (default seed).  Valid only for the kernel as captured: set to None when it changes.
+MEASURED_TRAFFIC_BYTES = {"cfg1_7b_gqa_decode": 724.6e6}
+
+
 def decode_algorithmic_bytes(spec: W.WorkloadSpec, lens_after: np.ndarray) -> int:
     """K and V of every context token read once per kv head (shared by the group's q heads),
     Q in and O out, and the page-table entries that are needed."""
@@ -416,7 +421,8 @@ def main():
                        "parallelism": f"replicas x{world} (independent trajectories, no collective)"},
             "hbm_gbs": achieved, "hbm_frac_of_nominal_8tbs": achieved / NOMINAL_HBM_GBS,
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                         "peak_kind": f"of {peak_kind}", "traffic": None,
+                         "peak_kind": f"of {peak_kind}",
+                         "traffic": MEASURED_TRAFFIC_BYTES.get(spec.name) if args.seed == W.MASTER_SEED else None,
                          "kernel": "decode_splitkv_kernel (the decode_attn call: partial attention with the split combine fused in)",
                          "algorithmic_bytes_per_launch": wl.bytes, "ms_per_launch": dec_ms},
             "e2e": {"value": n_items_all / (e2e_ms_step * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
