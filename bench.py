@@ -163,6 +163,27 @@ class DecodeWorkload:
         self.ctx.check()
         return total, dec
 
+    def time_gather(self, steps: int = 5, warmup: int = 2):
+        """KV hand-off: all trajectories' caches gathered into contiguous rows.  (mean ms, bytes read + written)"""
+        b = self.batch
+        lens = b.seq_lens_before[self.ids]
+        indptr = np.concatenate([[0], np.cumsum(lens.astype(np.int64))])
+        if indptr[-1] >= 2 ** 31:
+            raise ValueError("too many rows for one gather call")
+        d_indptr = torch.from_numpy(indptr.astype(np.int32)).to(self.device)
+        k_out = torch.empty(int(indptr[-1]), self.spec.num_kv_heads, self.spec.head_dim, dtype=torch.bfloat16, device=self.device)
+        v_out = torch.empty_like(k_out)
+        ev = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(steps)]
+        for s in range(warmup + steps):
+            if s >= warmup:
+                ev[s - warmup][0].record()
+            self.ctx.kv_gather(b.k_pool, b.v_pool, self.table, self.lens0, d_indptr, k_out, v_out, traj_ids=self.traj_ids)
+            if s >= warmup:
+                ev[s - warmup][1].record()
+        torch.cuda.synchronize(self.device)
+        self.ctx.check()
+        return float(np.mean([e[0].elapsed_time(e[1]) for e in ev])), 2 * 2 * k_out.numel() * 2
+
     def time_e2e(self, steps: int, warmup: int):
         """Steps driven from HOST buffers: per step the new token's q/k/v go host->device from
         pinned memory and the attention output comes back device->host, inside the timed region."""
@@ -448,6 +469,10 @@ def main():
                                                  "frac_of_measured": gbs / peak, "frac_of_nominal_8tbs": gbs / NOMINAL_HBM_GBS,
                                                  "decode_tokens_per_s": w2.n_items / (tot / 20 * 1e-3),
                                                  "trajectories": w2.n_items}
+                    if ci == 3:
+                        g_ms, g_bytes = w2.time_gather()
+                        extra[W.CONFIGS[ci].name].update({"kv_gather_ms": g_ms, "kv_gather_gbs": g_bytes / (g_ms * 1e-3) / 1e9,
+                                                          "kv_gather_frac_of_measured_hbm": g_bytes / (g_ms * 1e-3) / 1e9 / peak})
                     w2.ctx.close()
                     del w2
                     torch.cuda.empty_cache()

@@ -118,6 +118,20 @@ rollart_status rollart_kv_append(rollart_ctx *ctx, const rollart_kv_pool *pool, 
                                  void *stream);
 
 /*
+ * KV gather: the inverse of rollart_kv_append, for handing a trajectory's cache to another worker
+ * (Sec. 6.3: with prefill/decode disaggregation the prefill worker's KV moves to a decode worker;
+ * Sec. 6.1: a trajectory resumes on another inference worker).  Item i copies the first
+ * n_i = out_indptr[i+1] - out_indptr[i] tokens of trajectory traj_ids[i] (NULL = identity) from its
+ * pages into rows out_indptr[i] .. of k_out / v_out ([device] bf16 [total_rows][num_kv_heads][head_dim],
+ * 16-byte aligned); the receiving side stores them with rollart_kv_append onto its own pages.
+ * Bit copy.  n_i > seq_lens[t], a trajectory id or a page id out of range are device-side
+ * ROLLART_ERR_BOUNDS errors; the offending rows are left unwritten.
+ */
+rollart_status rollart_kv_gather(rollart_ctx *ctx, const rollart_kv_pool *pool, const rollart_trajs *trajs,
+                                 const int32_t *traj_ids, const int32_t *out_indptr, int32_t n_items, int32_t total_rows,
+                                 void *k_out, void *v_out, void *stream);
+
+/*
  * Decode attention (Sec. 3.1: the decoding phase is bound by reading the whole context once per
  * generated token).  For item i with trajectory t = traj_ids[i], L = seq_lens[t] (lengths AFTER
  * the append: the query attends to its own K/V), query head hq, kv head h = hq / g:

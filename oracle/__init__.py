@@ -27,7 +27,7 @@ def lib():
     if _lib is None:
         L = ctypes.CDLL(_build())
         L.oracle_num_threads.restype = ctypes.c_int
-        for name in ("oracle_kv_append", "oracle_attend", "oracle_lse_combine"):
+        for name in ("oracle_kv_append", "oracle_kv_gather", "oracle_attend", "oracle_lse_combine"):
             getattr(L, name).restype = ctypes.c_int
         _lib = L
     return _lib
@@ -79,6 +79,27 @@ def kv_append(k_pool: np.ndarray, v_pool: np.ndarray, page_table: np.ndarray, se
         _p(tid), _p(new_indptr), ctypes.c_int32(n_items), _p(k_new), _p(v_new), _p(out))
     _check(rc)
     return out
+
+
+def kv_gather(k_pool: np.ndarray, v_pool: np.ndarray, page_table: np.ndarray, seq_lens: np.ndarray,
+              out_indptr: np.ndarray, traj_ids: Optional[np.ndarray] = None):
+    """Contiguous copies (k_out, v_out: uint16 [total][Hkv][D]) of the first n_i tokens of each listed
+    trajectory (Sec. 6.3, prefill/decode disaggregation hands a trajectory's cache to another worker)."""
+    num_pages, Hkv, P, D = _pool_dims(k_pool)
+    page_table = _c(page_table, np.int32)
+    seq_lens = _c(seq_lens, np.int32)
+    out_indptr = _c(out_indptr, np.int32)
+    n_items = len(out_indptr) - 1
+    tid = None if traj_ids is None else _c(traj_ids, np.int32)
+    total = int(out_indptr[-1])
+    k_out = np.zeros((total, Hkv, D), dtype=np.uint16)
+    v_out = np.zeros((total, Hkv, D), dtype=np.uint16)
+    rc = lib().oracle_kv_gather(
+        _p(k_pool), _p(v_pool), ctypes.c_int32(num_pages), ctypes.c_int32(P), ctypes.c_int32(Hkv), ctypes.c_int32(D),
+        _p(page_table), ctypes.c_int32(page_table.shape[1]), _p(seq_lens), ctypes.c_int32(len(seq_lens)),
+        _p(tid), _p(out_indptr), ctypes.c_int32(n_items), _p(k_out), _p(v_out))
+    _check(rc)
+    return k_out, v_out
 
 
 def attend_rows(k_pool: np.ndarray, v_pool: np.ndarray, page_table: np.ndarray,

@@ -18,6 +18,9 @@
  *            s_j = scale * <q, k_j>, j in [j0, c);  m = max_j s_j;
  *            w_j = exp(s_j - m);  Z = sum_j w_j;
  *            out = sum_j w_j v_j / Z;   lse = m + ln Z.
+ *   gather : the inverse of append, for handing a trajectory's cache to another worker
+ *            (prefill/decode disaggregation, Sec. 6.3): row r of item i is the token at logical
+ *            position r of trajectory t, copied bit for bit from its page slot.
  *   combine: parts (out_s, lse_s) over disjoint key ranges merge as
  *            M = max_s lse_s; a_s = exp(lse_s - M); out = sum a_s out_s / sum a_s;
  *            lse = M + ln sum a_s.
@@ -83,6 +86,35 @@ int oracle_kv_append(uint16_t *k_pool, uint16_t *v_pool, int32_t num_pages, int3
             }
         }
         if (seq_lens_out) seq_lens_out[t] = len + n;
+    }
+    return ORACLE_OK;
+}
+
+/* Gather.  Item i copies the first n_i = out_indptr[i+1] - out_indptr[i] tokens of trajectory
+ * traj_ids[i] (identity when NULL) into rows out_indptr[i].. of k_out/v_out ([total][Hkv][D]).
+ * n_i must not exceed the trajectory's length. */
+int oracle_kv_gather(const uint16_t *k_pool, const uint16_t *v_pool, int32_t num_pages, int32_t P, int32_t Hkv, int32_t D,
+                     const int32_t *page_table, int32_t max_pages, const int32_t *seq_lens, int32_t num_traj,
+                     const int32_t *traj_ids, const int32_t *out_indptr, int32_t n_items, uint16_t *k_out, uint16_t *v_out) {
+    if (P <= 0 || Hkv <= 0 || D <= 0 || n_items < 0) return ORACLE_BAD_ARG;
+    for (int32_t i = 0; i < n_items; ++i) {
+        int32_t t = traj_ids ? traj_ids[i] : i;
+        if (t < 0 || t >= num_traj) return ORACLE_BAD_ARG;
+        int32_t n = out_indptr[i + 1] - out_indptr[i];
+        if (n < 0 || n > seq_lens[t]) return ORACLE_BAD_LENGTH;
+        for (int32_t r = 0; r < n; ++r) {
+            int64_t lp = r / P;
+            if (lp >= max_pages) return ORACLE_BAD_LENGTH;
+            int32_t pg = page_table[(int64_t)t * max_pages + lp];
+            if (pg < 0 || pg >= num_pages) return ORACLE_BAD_PAGE;
+            int64_t row = (int64_t)out_indptr[i] + r;
+            for (int32_t h = 0; h < Hkv; ++h) {
+                int64_t src = (((int64_t)pg * Hkv + h) * P + r % P) * D;
+                int64_t dst = (row * Hkv + h) * D;
+                memcpy(k_out + dst, k_pool + src, (size_t)D * sizeof(uint16_t));
+                memcpy(v_out + dst, v_pool + src, (size_t)D * sizeof(uint16_t));
+            }
+        }
     }
     return ORACLE_OK;
 }

@@ -1,4 +1,5 @@
-// KV append: scatter the new tokens' K/V rows into the trajectories' pages (bit copy).
+// KV append: scatter the new tokens' K/V rows into the trajectories' pages (bit copy), and its
+// inverse, KV gather: copy a trajectory's tokens from its pages into contiguous rows.
 //
 // One thread moves 16 bytes of a K row and the matching 16 bytes of the V row.  A (token, kv head)
 // row is 256 B, so 16 consecutive threads cover it and a warp covers two heads of one token;
@@ -71,7 +72,50 @@ kv_append_kernel(__nv_bfloat16 *__restrict__ k_pool, __nv_bfloat16 *__restrict__
     reinterpret_cast<uint4 *>(v_pool)[dst] = vv;
 }
 
+// Gather: thread -> (output row, kv head, 16-byte piece); row r of item i is the token at logical position r.
+__global__ void __launch_bounds__(kThreads)
+kv_gather_kernel(const __nv_bfloat16 *__restrict__ k_pool, const __nv_bfloat16 *__restrict__ v_pool, int num_pages,
+                 int page_size, int num_kv_heads, const int32_t *__restrict__ page_table, int max_pages,
+                 const int32_t *__restrict__ seq_lens, int num_traj, const int32_t *__restrict__ traj_ids,
+                 const int32_t *__restrict__ out_indptr, int n_items, int total_rows, uint4 *__restrict__ k_out,
+                 uint4 *__restrict__ v_out, DeviceStatus *status) {
+    const long long gid = static_cast<long long>(blockIdx.x) * kThreads + threadIdx.x;
+    const long long n_vec = static_cast<long long>(total_rows) * num_kv_heads * kVecPerRow;
+    if (gid >= n_vec) return;
+    const int c = static_cast<int>(gid % kVecPerRow);
+    const long long rh = gid / kVecPerRow;
+    const int h = static_cast<int>(rh % num_kv_heads);
+    const int row = static_cast<int>(rh / num_kv_heads);
+    const int i = find_item(out_indptr, n_items, row);
+    const int t = traj_ids ? __ldg(traj_ids + i) : i;
+    if (t < 0 || t >= num_traj) { report(status, ROLLART_ERR_BOUNDS, t, 5); return; }
+    const int pos = row - __ldg(out_indptr + i);
+    if (pos >= __ldg(seq_lens + t)) { report(status, ROLLART_ERR_BOUNDS, pos, 5); return; }
+    const int lp = pos / page_size;
+    if (lp >= max_pages) { report(status, ROLLART_ERR_BOUNDS, lp, 5); return; }
+    const int pg = __ldg(page_table + static_cast<long long>(t) * max_pages + lp);
+    if (pg < 0 || pg >= num_pages) { report(status, ROLLART_ERR_BOUNDS, pg, 5); return; }
+    const long long src = ((static_cast<long long>(pg) * num_kv_heads + h) * page_size + (pos - lp * page_size)) * kVecPerRow + c;
+    k_out[gid] = __ldg(reinterpret_cast<const uint4 *>(k_pool) + src);
+    v_out[gid] = __ldg(reinterpret_cast<const uint4 *>(v_pool) + src);
+}
+
 }  // namespace
+
+cudaError_t launch_kv_gather(const rollart_kv_pool &pool, const rollart_trajs &trajs, const int32_t *traj_ids,
+                             const int32_t *out_indptr, int n_items, int total_rows, void *k_out, void *v_out,
+                             DeviceStatus *status, cudaStream_t stream, int64_t *launches) {
+    const long long n_vec = static_cast<long long>(total_rows) * pool.num_kv_heads * kVecPerRow;
+    if (n_vec == 0) return cudaSuccess;
+    const long long blocks = (n_vec + kThreads - 1) / kThreads;
+    if (blocks > 0x7FFFFFFFLL) return cudaErrorInvalidValue;
+    kv_gather_kernel<<<static_cast<unsigned>(blocks), kThreads, 0, stream>>>(
+        static_cast<const __nv_bfloat16 *>(pool.k_pool), static_cast<const __nv_bfloat16 *>(pool.v_pool), pool.num_pages,
+        pool.page_size, pool.num_kv_heads, trajs.page_table, trajs.max_pages_per_traj, trajs.seq_lens, trajs.num_traj,
+        traj_ids, out_indptr, n_items, total_rows, static_cast<uint4 *>(k_out), static_cast<uint4 *>(v_out), status);
+    ++*launches;
+    return cudaGetLastError();
+}
 
 cudaError_t launch_kv_append(const rollart_kv_pool &pool, const rollart_trajs &trajs, const int32_t *traj_ids,
                              const int32_t *new_indptr, int n_items, int total_new, const void *k_new,

@@ -191,6 +191,25 @@ rollart_status rollart_kv_append(rollart_ctx *ctx, const rollart_kv_pool *pool, 
     return ROLLART_OK;
 }
 
+rollart_status rollart_kv_gather(rollart_ctx *ctx, const rollart_kv_pool *pool, const rollart_trajs *trajs,
+                                 const int32_t *traj_ids, const int32_t *out_indptr, int32_t n_items, int32_t total_rows,
+                                 void *k_out, void *v_out, void *stream) {
+    if (!ctx) return ROLLART_ERR_INVALID_ARG;
+    rollart_status st;
+    if ((st = check_pool(ctx, pool)) != ROLLART_OK) return st;
+    if ((st = check_trajs(ctx, trajs)) != ROLLART_OK) return st;
+    if (n_items < 0 || total_rows < 0) return fail(ctx, ROLLART_ERR_INVALID_ARG, "negative n_items or total_rows");
+    if (n_items == 0 || total_rows == 0) return ROLLART_OK;
+    if (!out_indptr || !k_out || !v_out) return fail(ctx, ROLLART_ERR_INVALID_ARG, "out_indptr, k_out or v_out NULL");
+    if (!aligned16(k_out) || !aligned16(v_out)) return fail(ctx, ROLLART_ERR_INVALID_ARG, "k_out/v_out must be 16-byte aligned");
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return fail(ctx, ROLLART_ERR_CUDA, "cannot select device %d", ctx->device);
+    cudaError_t e = launch_kv_gather(*pool, *trajs, traj_ids, out_indptr, n_items, total_rows, k_out, v_out, ctx->d_status,
+                                     static_cast<cudaStream_t>(stream), &ctx->launches);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "kv_gather launch");
+    return ROLLART_OK;
+}
+
 // max_seq_len is only an upper bound: a page-table row cannot hold more than this anyway
 static int32_t clamp_bound(const rollart_kv_pool *pool, const rollart_trajs *trajs, int32_t max_seq_len) {
     const int64_t cap = static_cast<int64_t>(trajs->max_pages_per_traj) * pool->page_size;
@@ -266,8 +285,8 @@ rollart_status rollart_check(rollart_ctx *ctx, void *stream) {
     if (hs.code == 0) return ROLLART_OK;
     decode_reset_workspace(ctx->workspace, ctx->workspace_bytes, s);
     cudaStreamSynchronize(s);
-    static const char *const where[] = {"?", "kv_append", "decode_attn", "obs_chunk_attn", "combine"};
-    const char *w = (hs.where >= 0 && hs.where < 5) ? where[hs.where] : "?";
+    static const char *const where[] = {"?", "kv_append", "decode_attn", "obs_chunk_attn", "combine", "kv_gather"};
+    const char *w = (hs.where >= 0 && hs.where < 6) ? where[hs.where] : "?";
     if (hs.code == ROLLART_ERR_TIMEOUT)
         return fail(ctx, ROLLART_ERR_TIMEOUT, "%s: a bounded wait ran out (detail %d)", w, hs.detail);
     return fail(ctx, static_cast<rollart_status>(hs.code), "%s: index out of range on the device (detail %d)", w, hs.detail);

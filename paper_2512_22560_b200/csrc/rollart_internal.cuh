@@ -47,6 +47,10 @@ cudaError_t launch_kv_append(const rollart_kv_pool &pool, const rollart_trajs &t
                              const void *v_new, int32_t *seq_lens_out, DeviceStatus *status, cudaStream_t stream,
                              int64_t *launches);
 
+cudaError_t launch_kv_gather(const rollart_kv_pool &pool, const rollart_trajs &trajs, const int32_t *traj_ids,
+                             const int32_t *out_indptr, int n_items, int total_rows, void *k_out, void *v_out,
+                             DeviceStatus *status, cudaStream_t stream, int64_t *launches);
+
 // Host-side cache of the TMA tensor maps describing the K and V pools (re-encoded when the pools change).
 struct TmaCache {
     bool valid;

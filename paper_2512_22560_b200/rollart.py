@@ -21,7 +21,7 @@ _NAMES = ["OK", "ERR_INVALID_ARG", "ERR_UNSUPPORTED", "ERR_WORKSPACE", "ERR_CUDA
 EXPORTS = (
     "rollart_workspace_size", "rollart_create", "rollart_destroy", "rollart_kv_append", "rollart_decode_attn",
     "rollart_obs_chunk_attn", "rollart_check", "rollart_last_error", "rollart_launch_count",
-    "rollart_decode_attn_noalloc",
+    "rollart_decode_attn_noalloc", "rollart_kv_gather",
 )
 
 
@@ -62,6 +62,8 @@ def load_library() -> ctypes.CDLL:
     L.rollart_destroy.argtypes = [vp]
     L.rollart_kv_append.restype = ctypes.c_int
     L.rollart_kv_append.argtypes = [vp, ctypes.POINTER(_KVPool), ctypes.POINTER(_Trajs), vp, vp, i32, i32, vp, vp, vp, vp]
+    L.rollart_kv_gather.restype = ctypes.c_int
+    L.rollart_kv_gather.argtypes = [vp, ctypes.POINTER(_KVPool), ctypes.POINTER(_Trajs), vp, vp, i32, i32, vp, vp, vp]
     L.rollart_decode_attn.restype = ctypes.c_int
     L.rollart_decode_attn.argtypes = [vp, ctypes.POINTER(_KVPool), ctypes.POINTER(_Trajs), vp, i32, i32, vp, i32, f32,
                                       vp, vp, vp]
@@ -197,6 +199,21 @@ class Context:
             self._h, ctypes.byref(pool), ctypes.byref(trajs), _ptr(traj_ids, torch.int32, self.device),
             _ptr(new_indptr, torch.int32, self.device), n_items, total_new, _ptr(k_new, torch.bfloat16, self.device),
             _ptr(v_new, torch.bfloat16, self.device), _ptr(seq_lens_out, torch.int32, self.device), self._stream(stream))
+        if st != OK:
+            self._raise(st)
+
+    def kv_gather(self, k_pool, v_pool, page_table, seq_lens, out_indptr, k_out, v_out, traj_ids=None, stream=None) -> None:
+        pool = self._pool(k_pool, v_pool)
+        trajs = self._trajs(page_table, seq_lens)
+        n_items = out_indptr.shape[0] - 1
+        if k_out.shape != v_out.shape or tuple(k_out.shape[1:]) != (pool.num_kv_heads, pool.head_dim):
+            raise ValueError("k_out/v_out must be [total_rows][num_kv_heads][head_dim]")
+        if traj_ids is not None and traj_ids.shape[0] != n_items:
+            raise ValueError("traj_ids must have one entry per item")
+        st = self._lib.rollart_kv_gather(
+            self._h, ctypes.byref(pool), ctypes.byref(trajs), _ptr(traj_ids, torch.int32, self.device),
+            _ptr(out_indptr, torch.int32, self.device), n_items, k_out.shape[0], _ptr(k_out, torch.bfloat16, self.device),
+            _ptr(v_out, torch.bfloat16, self.device), self._stream(stream))
         if st != OK:
             self._raise(st)
 

@@ -100,3 +100,45 @@ def test_append_host_side_validation(cuda_device):
     with pytest.raises(rollart.RollartError) as e:
         ctx.kv_append(bad, bad, db.page_table, db.lens_before, db.new_indptr, db.k_new, db.v_new)
     assert e.value.status == rollart.ERR_UNSUPPORTED
+
+
+@pytest.mark.parametrize("i,T,div", [(0, 4, 1), (3, 3, 32), (4, 9, 16)])
+def test_gather_matches_oracle_and_round_trips_through_append(cuda_device, i, T, div):
+    """Hand-off of whole trajectories: gather from one pool, append into another (different page table)."""
+    batch = W.make_batch(W.shrink(W.CONFIGS[i], T, div, 8), seed=300 + i)
+    spec = batch.spec
+    db = DeviceBatch(batch, cuda_device)
+    ctx = rollart.Context(0, 0)
+    ids = np.array(sorted(range(T), key=lambda t: -t)[: max(2, T - 1)], np.int32)      # a subset in reverse order
+    lens = batch.seq_lens_before[ids]
+    indptr = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    total = int(indptr[-1])
+    k_out = torch.full((total, spec.num_kv_heads, 128), float("nan"), dtype=torch.bfloat16, device=cuda_device)
+    v_out = torch.full_like(k_out, float("nan"))
+    ctx.kv_gather(db.k_pool, db.v_pool, db.page_table, db.lens_before, dev_i32(indptr, cuda_device), k_out, v_out,
+                  traj_ids=dev_i32(ids, cuda_device))
+    ctx.check()
+    ko, vo = oracle.kv_gather(W.bf16_to_u16(batch.k_pool), W.bf16_to_u16(batch.v_pool), batch.page_table,
+                              batch.seq_lens_before, indptr, traj_ids=ids)
+    assert np.array_equal(W.bf16_to_u16(k_out), ko) and np.array_equal(W.bf16_to_u16(v_out), vo)
+    # receiving side: empty trajectories with their own pages
+    pages = (lens.astype(np.int64) + spec.page_size - 1) // spec.page_size
+    table2, num_pages2 = W.build_page_table(pages, 0.25, np.random.default_rng(9))
+    k2 = torch.zeros(num_pages2, spec.num_kv_heads, spec.page_size, 128, dtype=torch.bfloat16, device=cuda_device)
+    v2 = torch.zeros_like(k2)
+    zero = dev_i32(np.zeros(len(ids)), cuda_device)
+    after = torch.empty_like(zero)
+    ctx.kv_append(k2, v2, dev_i32(table2, cuda_device), zero, dev_i32(indptr, cuda_device), k_out, v_out, seq_lens_out=after)
+    k_back = torch.empty_like(k_out)
+    v_back = torch.empty_like(v_out)
+    ctx.kv_gather(k2, v2, dev_i32(table2, cuda_device), after, dev_i32(indptr, cuda_device), k_back, v_back)
+    ctx.check()
+    assert np.array_equal(after.cpu().numpy(), lens)
+    assert torch.equal(k_back.view(torch.int16), k_out.view(torch.int16)) and torch.equal(v_back.view(torch.int16), v_out.view(torch.int16))
+    # asking for more rows than a trajectory holds is reported, not read
+    bad = indptr.copy()
+    bad[-1] += 1
+    big = torch.zeros(total + 1, spec.num_kv_heads, 128, dtype=torch.bfloat16, device=cuda_device)
+    ctx.kv_gather(db.k_pool, db.v_pool, db.page_table, db.lens_before, dev_i32(bad, cuda_device), big, big.clone(),
+                  traj_ids=dev_i32(ids, cuda_device))
+    assert ctx.status() == rollart.ERR_BOUNDS and "kv_gather" in ctx.last_error()

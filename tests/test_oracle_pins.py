@@ -450,3 +450,29 @@ def test_out_of_range_page_is_an_error_not_a_read():
         oracle.decode_attn(kp, vp, bad, lens, q, 1.0)
     with pytest.raises(oracle.OracleError):
         oracle.decode_attn(kp, vp, table, np.array([33], np.int32), q, 1.0)   # longer than the table row
+
+
+# ---- gather: the inverse of append ---------------------------------------------------------------
+@pytest.mark.parametrize("P", [16, 64])
+def test_gather_returns_what_was_packed_and_inverts_append(P):
+    rng = np.random.default_rng(30)
+    lens = [1, P - 1, P, P + 1, 3 * P + 5]
+    K = [rng.integers(0, 65536, size=(L, 2, D), dtype=np.uint16) for L in lens]
+    V = [rng.integers(0, 65536, size=(L, 2, D), dtype=np.uint16) for L in lens]
+    kp, vp, table, sl = pack_pages(K, V, P, 2, D, rng=rng, fill_bits=0xFFFF)
+    indptr = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    ko, vo = oracle.kv_gather(kp, vp, table, sl, indptr)
+    assert np.array_equal(ko, np.concatenate(K)) and np.array_equal(vo, np.concatenate(V))
+    # a subset, in another order, and only a prefix of one trajectory
+    ids = np.array([4, 1], np.int32)
+    ko2, vo2 = oracle.kv_gather(kp, vp, table, sl, np.array([0, 2 * P + 1, 2 * P + 1 + lens[1]], np.int32), traj_ids=ids)
+    assert np.array_equal(ko2, np.concatenate([K[4][:2 * P + 1], K[1]]))
+    # gather then append into an empty pool with a different page table reproduces the logical contents
+    kp2 = np.zeros_like(kp); vp2 = np.zeros_like(vp)
+    table2 = table[:, ::-1].copy() if False else np.where(table >= 0, kp.shape[0] - 1 - table, -1).astype(np.int32)
+    after = oracle.kv_append(kp2, vp2, table2, np.zeros(len(lens), np.int32), indptr, ko, vo)
+    assert list(after) == lens
+    ko3, vo3 = oracle.kv_gather(kp2, vp2, table2, after, indptr)
+    assert np.array_equal(ko3, ko) and np.array_equal(vo3, vo)
+    with pytest.raises(oracle.OracleError):      # asking for more rows than the trajectory holds
+        oracle.kv_gather(kp, vp, table, sl, np.array([0, lens[0] + 1], np.int32))
