@@ -109,3 +109,28 @@ def test_many_small_chunks_span_several_launches(cuda_device):
     spec = dataclasses.replace(W.CONFIGS[0], num_traj=1100, len_lo=1, len_hi=40, chunk_fraction=1.0, chunk_lo=1, chunk_hi=5,
                                name="many_chunks")
     run_chunk_case(W.make_batch(spec, seed=72), cuda_device)
+
+
+def test_empty_items_and_empty_calls(cuda_device):
+    # an item with no chunk rows among live ones, and calls with nothing to do at all
+    spec = dataclasses.replace(W.CONFIGS[4], num_traj=4, name="empties")
+    batch = W.make_layout(W.shrink(spec, 4, 64, 16), seed=47)
+    batch.is_chunk[:] = True
+    batch.n_new = np.array([5, 0, 40, 1], np.int32)
+    batch.new_indptr = np.concatenate([[0], np.cumsum(batch.n_new)]).astype(np.int32)
+    P = batch.spec.page_size
+    pages = (batch.seq_lens_before.astype(np.int64) + batch.n_new + P - 1) // P
+    batch.page_table, batch.num_pages = W.build_page_table(pages, 0.3, np.random.default_rng(1))
+    W.fill_tensors(batch)
+    db, ctx, out, _ = run_chunk_case(batch, cuda_device)
+    empty_q = torch.zeros(0, batch.spec.num_q_heads, 128, dtype=torch.bfloat16, device=cuda_device)
+    n0 = ctx.launch_count
+    ctx.obs_chunk_attn(db.k_pool, db.v_pool, db.page_table, db.lens_after, dev_i32([0], cuda_device), empty_q, 0.1, 100,
+                       empty_q.clone())
+    ctx.decode_attn(db.k_pool, db.v_pool, db.page_table, db.lens_after, empty_q, 0.1, 100, empty_q.clone(),
+                    traj_ids=dev_i32([], cuda_device))
+    ctx.kv_append(db.k_pool, db.v_pool, db.page_table, db.lens_after, dev_i32([0], cuda_device),
+                  torch.zeros(0, batch.spec.num_kv_heads, 128, dtype=torch.bfloat16, device=cuda_device),
+                  torch.zeros(0, batch.spec.num_kv_heads, 128, dtype=torch.bfloat16, device=cuda_device))
+    ctx.check()
+    assert ctx.launch_count == n0          # nothing was enqueued
