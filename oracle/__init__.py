@@ -27,7 +27,8 @@ def lib():
     if _lib is None:
         L = ctypes.CDLL(_build())
         L.oracle_num_threads.restype = ctypes.c_int
-        for name in ("oracle_kv_append", "oracle_kv_gather", "oracle_attend", "oracle_lse_combine"):
+        for name in ("oracle_kv_append", "oracle_kv_gather", "oracle_attend", "oracle_lse_combine", "oracle_pages_reserve",
+                     "oracle_pages_release"):
             getattr(L, name).restype = ctypes.c_int
         _lib = L
     return _lib
@@ -100,6 +101,36 @@ def kv_gather(k_pool: np.ndarray, v_pool: np.ndarray, page_table: np.ndarray, se
         _p(tid), _p(out_indptr), ctypes.c_int32(n_items), _p(k_out), _p(v_out))
     _check(rc)
     return k_out, v_out
+
+
+def pages_reserve(free_pages: np.ndarray, free_count: int, page_size: int, page_table: np.ndarray, seq_lens: np.ndarray,
+                  new_tokens, traj_ids: Optional[np.ndarray] = None) -> int:
+    """Pops, in item order, the pages each trajectory needs to grow by new_tokens[i] (Sec. 6.1: ADD between
+    engine steps) and writes them into page_table IN PLACE.  Returns the new free count."""
+    assert free_pages.dtype == np.int32 and page_table.dtype == np.int32 and page_table.flags.c_contiguous
+    seq_lens = _c(seq_lens, np.int32)
+    new_tokens = _c(new_tokens, np.int32)
+    tid = None if traj_ids is None else _c(traj_ids, np.int32)
+    cnt = ctypes.c_int32(free_count)
+    rc = lib().oracle_pages_reserve(_p(free_pages), ctypes.byref(cnt), ctypes.c_int32(page_size), _p(page_table),
+                                    ctypes.c_int32(page_table.shape[1]), _p(seq_lens), ctypes.c_int32(len(seq_lens)), _p(tid),
+                                    _p(new_tokens), ctypes.c_int32(len(new_tokens)))
+    _check(rc)
+    return int(cnt.value)
+
+
+def pages_release(free_pages: np.ndarray, free_count: int, page_size: int, page_table: np.ndarray, seq_lens: np.ndarray,
+                  traj_ids: np.ndarray) -> int:
+    """Pushes, in item order, every page of the listed trajectories (Sec. 6.1 ABORT, Sec. 6.2 stale eviction); sets
+    their table entries to -1 and their lengths to 0, IN PLACE.  Returns the new free count."""
+    assert free_pages.dtype == np.int32 and page_table.dtype == np.int32 and seq_lens.dtype == np.int32
+    tid = _c(traj_ids, np.int32)
+    cnt = ctypes.c_int32(free_count)
+    rc = lib().oracle_pages_release(_p(free_pages), ctypes.byref(cnt), ctypes.c_int32(len(free_pages)), ctypes.c_int32(page_size),
+                                    _p(page_table), ctypes.c_int32(page_table.shape[1]), _p(seq_lens),
+                                    ctypes.c_int32(len(seq_lens)), _p(tid), ctypes.c_int32(len(tid)))
+    _check(rc)
+    return int(cnt.value)
 
 
 def attend_rows(k_pool: np.ndarray, v_pool: np.ndarray, page_table: np.ndarray,

@@ -21,6 +21,12 @@
  *   gather : the inverse of append, for handing a trajectory's cache to another worker
  *            (prefill/decode disaggregation, Sec. 6.3): row r of item i is the token at logical
  *            position r of trajectory t, copied bit for bit from its page slot.
+ *   reserve: page bookkeeping between engine steps (Sec. 6.1: ADD / ABORT commands are processed
+ *            between steps; Sec. 6.2: stale trajectories are evicted).  The free pages form a
+ *            stack; item i, in item order, pops the pages that its trajectory needs to grow by
+ *            new_tokens[i] and stores them in the next page-table entries.
+ *   release: item i, in item order, pushes the pages its trajectory owns (logical order), marks
+ *            the entries -1 and sets the length to 0.
  *   combine: parts (out_s, lse_s) over disjoint key ranges merge as
  *            M = max_s lse_s; a_s = exp(lse_s - M); out = sum a_s out_s / sum a_s;
  *            lse = M + ln sum a_s.
@@ -116,6 +122,60 @@ int oracle_kv_gather(const uint16_t *k_pool, const uint16_t *v_pool, int32_t num
             }
         }
     }
+    return ORACLE_OK;
+}
+
+/* Reserve.  free_pages[0 .. *free_count) is the stack (top at the end).  Returns ORACLE_BAD_LENGTH and
+ * changes nothing when the stack is too small or a trajectory would outgrow its page-table row. */
+int oracle_pages_reserve(int32_t *free_pages, int32_t *free_count, int32_t P, int32_t *page_table, int32_t max_pages,
+                         const int32_t *seq_lens, int32_t num_traj, const int32_t *traj_ids, const int32_t *new_tokens,
+                         int32_t n_items) {
+    if (P <= 0 || n_items < 0) return ORACLE_BAD_ARG;
+    int64_t need_total = 0;
+    for (int32_t i = 0; i < n_items; ++i) {
+        int32_t t = traj_ids ? traj_ids[i] : i;
+        if (t < 0 || t >= num_traj || new_tokens[i] < 0 || seq_lens[t] < 0) return ORACLE_BAD_ARG;
+        int64_t have = ((int64_t)seq_lens[t] + P - 1) / P;
+        int64_t want = ((int64_t)seq_lens[t] + new_tokens[i] + P - 1) / P;
+        if (want > max_pages) return ORACLE_BAD_LENGTH;
+        need_total += want - have;
+    }
+    if (need_total > *free_count) return ORACLE_BAD_LENGTH;
+    int32_t top = *free_count;
+    for (int32_t i = 0; i < n_items; ++i) {
+        int32_t t = traj_ids ? traj_ids[i] : i;
+        int64_t have = ((int64_t)seq_lens[t] + P - 1) / P;
+        int64_t want = ((int64_t)seq_lens[t] + new_tokens[i] + P - 1) / P;
+        for (int64_t lp = have; lp < want; ++lp) page_table[(int64_t)t * max_pages + lp] = free_pages[--top];
+    }
+    *free_count = top;
+    return ORACLE_OK;
+}
+
+/* Release.  seq_lens is updated in place (0 for the trajectories named). */
+int oracle_pages_release(int32_t *free_pages, int32_t *free_count, int32_t capacity, int32_t P, int32_t *page_table,
+                         int32_t max_pages, int32_t *seq_lens, int32_t num_traj, const int32_t *traj_ids, int32_t n_items) {
+    if (P <= 0 || n_items < 0) return ORACLE_BAD_ARG;
+    int64_t total = *free_count;
+    for (int32_t i = 0; i < n_items; ++i) {
+        int32_t t = traj_ids ? traj_ids[i] : i;
+        if (t < 0 || t >= num_traj || seq_lens[t] < 0) return ORACLE_BAD_ARG;
+        int64_t have = ((int64_t)seq_lens[t] + P - 1) / P;
+        if (have > max_pages) return ORACLE_BAD_LENGTH;
+        total += have;
+    }
+    if (total > capacity) return ORACLE_BAD_LENGTH;
+    int32_t top = *free_count;
+    for (int32_t i = 0; i < n_items; ++i) {
+        int32_t t = traj_ids ? traj_ids[i] : i;
+        int64_t have = ((int64_t)seq_lens[t] + P - 1) / P;
+        for (int64_t lp = 0; lp < have; ++lp) {
+            free_pages[top++] = page_table[(int64_t)t * max_pages + lp];
+            page_table[(int64_t)t * max_pages + lp] = -1;
+        }
+        seq_lens[t] = 0;
+    }
+    *free_count = top;
     return ORACLE_OK;
 }
 
