@@ -132,6 +132,31 @@ rollart_status rollart_kv_gather(rollart_ctx *ctx, const rollart_kv_pool *pool, 
                                  void *k_out, void *v_out, void *stream);
 
 /*
+ * Page bookkeeping between engine steps (Sec. 6.1: the inference worker processes ADD and ABORT commands
+ * between steps; Sec. 6.2: trajectories that have become too stale are evicted).  The free pages are a
+ * stack: free_pages [device] int32 [capacity] with *free_count [device] live entries, top at the end.
+ *
+ * rollart_pages_reserve: item i (trajectory traj_ids[i], NULL = identity) is about to grow by new_tokens[i]
+ *   [device] tokens; it pops ceil((len + n) / page_size) - ceil(len / page_size) pages, items in order, and
+ *   stores them in the next entries of its page-table row.  seq_lens is only read (rollart_kv_append moves
+ *   the lengths).  A new trajectory is one with len = 0.
+ * rollart_pages_release: item i pushes all pages of trajectory traj_ids[i] (logical order, items in order),
+ *   sets those table entries to -1 and seq_lens[t] to 0.
+ *
+ * page_table is the same [num_traj][max_pages_per_traj] table the other calls read.  Both calls are
+ * deterministic and all-or-nothing: if the stack is too small (or too full), a trajectory id or length is
+ * out of range, or a row would overflow, nothing changes and ROLLART_ERR_BOUNDS is recorded for
+ * rollart_check.  A trajectory may appear at most once per call.
+ */
+rollart_status rollart_pages_reserve(rollart_ctx *ctx, int32_t *free_pages, int32_t *free_count, int32_t page_size,
+                                     int32_t *page_table, int32_t max_pages_per_traj, const int32_t *seq_lens,
+                                     int32_t num_traj, const int32_t *traj_ids, const int32_t *new_tokens, int32_t n_items,
+                                     void *stream);
+rollart_status rollart_pages_release(rollart_ctx *ctx, int32_t *free_pages, int32_t *free_count, int32_t capacity,
+                                     int32_t page_size, int32_t *page_table, int32_t max_pages_per_traj, int32_t *seq_lens,
+                                     int32_t num_traj, const int32_t *traj_ids, int32_t n_items, void *stream);
+
+/*
  * Decode attention (Sec. 3.1: the decoding phase is bound by reading the whole context once per
  * generated token).  For item i with trajectory t = traj_ids[i], L = seq_lens[t] (lengths AFTER
  * the append: the query attends to its own K/V), query head hq, kv head h = hq / g:

@@ -210,6 +210,40 @@ rollart_status rollart_kv_gather(rollart_ctx *ctx, const rollart_kv_pool *pool, 
     return ROLLART_OK;
 }
 
+static rollart_status pages_common(rollart_ctx *ctx, bool reserve, int32_t *free_pages, int32_t *free_count, int32_t capacity,
+                                   int32_t page_size, int32_t *page_table, int32_t max_pages, int32_t *seq_lens,
+                                   int32_t num_traj, const int32_t *traj_ids, const int32_t *new_tokens, int32_t n_items,
+                                   void *stream) {
+    if (!ctx) return ROLLART_ERR_INVALID_ARG;
+    if (!free_pages || !free_count || !page_table || !seq_lens) return fail(ctx, ROLLART_ERR_INVALID_ARG, "NULL pointer");
+    if (page_size <= 0 || max_pages <= 0 || num_traj <= 0 || n_items < 0 || capacity < 0)
+        return fail(ctx, ROLLART_ERR_INVALID_ARG, "sizes must be positive");
+    if (n_items == 0) return ROLLART_OK;
+    if (reserve && !new_tokens) return fail(ctx, ROLLART_ERR_INVALID_ARG, "new_tokens NULL");
+    if (!reserve && !traj_ids) return fail(ctx, ROLLART_ERR_INVALID_ARG, "traj_ids NULL");
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return fail(ctx, ROLLART_ERR_CUDA, "cannot select device %d", ctx->device);
+    cudaError_t e = launch_pages(reserve, free_pages, free_count, capacity, page_size, page_table, max_pages, seq_lens, num_traj,
+                                 traj_ids, new_tokens, n_items, ctx->d_status, static_cast<cudaStream_t>(stream), &ctx->launches);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, reserve ? "pages_reserve launch" : "pages_release launch");
+    return ROLLART_OK;
+}
+
+rollart_status rollart_pages_reserve(rollart_ctx *ctx, int32_t *free_pages, int32_t *free_count, int32_t page_size,
+                                     int32_t *page_table, int32_t max_pages_per_traj, const int32_t *seq_lens,
+                                     int32_t num_traj, const int32_t *traj_ids, const int32_t *new_tokens, int32_t n_items,
+                                     void *stream) {
+    return pages_common(ctx, true, free_pages, free_count, 0, page_size, page_table, max_pages_per_traj,
+                        const_cast<int32_t *>(seq_lens), num_traj, traj_ids, new_tokens, n_items, stream);
+}
+
+rollart_status rollart_pages_release(rollart_ctx *ctx, int32_t *free_pages, int32_t *free_count, int32_t capacity,
+                                     int32_t page_size, int32_t *page_table, int32_t max_pages_per_traj, int32_t *seq_lens,
+                                     int32_t num_traj, const int32_t *traj_ids, int32_t n_items, void *stream) {
+    return pages_common(ctx, false, free_pages, free_count, capacity, page_size, page_table, max_pages_per_traj, seq_lens,
+                        num_traj, traj_ids, nullptr, n_items, stream);
+}
+
 // max_seq_len is only an upper bound: a page-table row cannot hold more than this anyway
 static int32_t clamp_bound(const rollart_kv_pool *pool, const rollart_trajs *trajs, int32_t max_seq_len) {
     const int64_t cap = static_cast<int64_t>(trajs->max_pages_per_traj) * pool->page_size;
@@ -285,8 +319,8 @@ rollart_status rollart_check(rollart_ctx *ctx, void *stream) {
     if (hs.code == 0) return ROLLART_OK;
     decode_reset_workspace(ctx->workspace, ctx->workspace_bytes, s);
     cudaStreamSynchronize(s);
-    static const char *const where[] = {"?", "kv_append", "decode_attn", "obs_chunk_attn", "combine", "kv_gather"};
-    const char *w = (hs.where >= 0 && hs.where < 6) ? where[hs.where] : "?";
+    static const char *const where[] = {"?", "kv_append", "decode_attn", "obs_chunk_attn", "combine", "kv_gather", "pages"};
+    const char *w = (hs.where >= 0 && hs.where < 7) ? where[hs.where] : "?";
     if (hs.code == ROLLART_ERR_TIMEOUT)
         return fail(ctx, ROLLART_ERR_TIMEOUT, "%s: a bounded wait ran out (detail %d)", w, hs.detail);
     return fail(ctx, static_cast<rollart_status>(hs.code), "%s: index out of range on the device (detail %d)", w, hs.detail);

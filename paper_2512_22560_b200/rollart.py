@@ -21,7 +21,7 @@ _NAMES = ["OK", "ERR_INVALID_ARG", "ERR_UNSUPPORTED", "ERR_WORKSPACE", "ERR_CUDA
 EXPORTS = (
     "rollart_workspace_size", "rollart_create", "rollart_destroy", "rollart_kv_append", "rollart_decode_attn",
     "rollart_obs_chunk_attn", "rollart_check", "rollart_last_error", "rollart_launch_count",
-    "rollart_decode_attn_noalloc", "rollart_kv_gather",
+    "rollart_decode_attn_noalloc", "rollart_kv_gather", "rollart_pages_reserve", "rollart_pages_release",
 )
 
 
@@ -64,6 +64,10 @@ def load_library() -> ctypes.CDLL:
     L.rollart_kv_append.argtypes = [vp, ctypes.POINTER(_KVPool), ctypes.POINTER(_Trajs), vp, vp, i32, i32, vp, vp, vp, vp]
     L.rollart_kv_gather.restype = ctypes.c_int
     L.rollart_kv_gather.argtypes = [vp, ctypes.POINTER(_KVPool), ctypes.POINTER(_Trajs), vp, vp, i32, i32, vp, vp, vp]
+    L.rollart_pages_reserve.restype = ctypes.c_int
+    L.rollart_pages_reserve.argtypes = [vp, vp, vp, i32, vp, i32, vp, i32, vp, vp, i32, vp]
+    L.rollart_pages_release.restype = ctypes.c_int
+    L.rollart_pages_release.argtypes = [vp, vp, vp, i32, i32, vp, i32, vp, i32, vp, i32, vp]
     L.rollart_decode_attn.restype = ctypes.c_int
     L.rollart_decode_attn.argtypes = [vp, ctypes.POINTER(_KVPool), ctypes.POINTER(_Trajs), vp, i32, i32, vp, i32, f32,
                                       vp, vp, vp]
@@ -199,6 +203,25 @@ class Context:
             self._h, ctypes.byref(pool), ctypes.byref(trajs), _ptr(traj_ids, torch.int32, self.device),
             _ptr(new_indptr, torch.int32, self.device), n_items, total_new, _ptr(k_new, torch.bfloat16, self.device),
             _ptr(v_new, torch.bfloat16, self.device), _ptr(seq_lens_out, torch.int32, self.device), self._stream(stream))
+        if st != OK:
+            self._raise(st)
+
+    def pages_reserve(self, free_pages, free_count, page_size, page_table, seq_lens, new_tokens, traj_ids=None, stream=None) -> None:
+        n_items = new_tokens.shape[0]
+        st = self._lib.rollart_pages_reserve(
+            self._h, _ptr(free_pages, torch.int32, self.device), _ptr(free_count, torch.int32, self.device), int(page_size),
+            _ptr(page_table, torch.int32, self.device), page_table.shape[1], _ptr(seq_lens, torch.int32, self.device),
+            page_table.shape[0], _ptr(traj_ids, torch.int32, self.device), _ptr(new_tokens, torch.int32, self.device), n_items,
+            self._stream(stream))
+        if st != OK:
+            self._raise(st)
+
+    def pages_release(self, free_pages, free_count, page_size, page_table, seq_lens, traj_ids, stream=None) -> None:
+        st = self._lib.rollart_pages_release(
+            self._h, _ptr(free_pages, torch.int32, self.device), _ptr(free_count, torch.int32, self.device),
+            free_pages.shape[0], int(page_size), _ptr(page_table, torch.int32, self.device), page_table.shape[1],
+            _ptr(seq_lens, torch.int32, self.device), page_table.shape[0], _ptr(traj_ids, torch.int32, self.device),
+            traj_ids.shape[0], self._stream(stream))
         if st != OK:
             self._raise(st)
 
