@@ -7,6 +7,7 @@ as uint16 bit patterns.  Every function here is pinned by tests/test_oracle_pins
 from __future__ import annotations
 
 import ctypes
+import os
 from typing import Optional, Sequence
 
 import numpy as np
@@ -25,7 +26,8 @@ class OracleError(ValueError):
 def lib():
     global _lib
     if _lib is None:
-        L = ctypes.CDLL(_build())
+        # the mutation test points this at a deliberately broken build to show that the pins notice
+        L = ctypes.CDLL(os.environ.get("ROLLART_ORACLE_LIB") or _build())
         L.oracle_num_threads.restype = ctypes.c_int
         for name in ("oracle_kv_append", "oracle_kv_gather", "oracle_attend", "oracle_lse_combine", "oracle_pages_reserve",
                      "oracle_pages_release"):
