@@ -44,7 +44,7 @@ def measured_peaks():
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one decode_splitkv_kernel launch, from the ncu capture summarised in
 # profiles/decode_splitkv_cfg1.md (default seed).  Valid only for the kernel as captured: set to None when it changes.
-MEASURED_TRAFFIC_BYTES = {"cfg1_7b_gqa_decode": 724.6e6}
+MEASURED_TRAFFIC_BYTES = {"cfg1_7b_gqa_decode": None}
 
 
 def decode_algorithmic_bytes(spec: W.WorkloadSpec, lens_after: np.ndarray) -> int:
@@ -134,12 +134,14 @@ class DecodeWorkload:
                              self.max_seq_len, self.out, traj_ids=self.traj_ids)
 
     def step(self):
-        self.append()
-        self.decode()
+        """One decode step: the fused call stores the new token's K/V and attends, in one launch."""
+        self.ctx.append_decode_attn(self.batch.k_pool, self.batch.v_pool, self.table, self.lens0, self.k_new, self.v_new, self.q,
+                                    self.spec.sm_scale, self.max_seq_len, self.out, traj_ids=self.traj_ids,
+                                    seq_lens_out=self.lens1)
 
     def time_steps(self, steps: int, warmup: int):
-        """(total ms over `steps` back-to-back steps, mean ms of the decode_attn call alone).
-        The throughput pass has no events inside the loop; the per-call time comes from a second pass."""
+        """(total ms over `steps` back-to-back steps, mean ms per launch).  A step is one kernel launch, so the
+        average launch duration is the timed region (two CUDA events, nothing inside the loop) over the step count."""
         for _ in range(warmup):
             self.step()
         torch.cuda.synchronize(self.device)
@@ -147,19 +149,11 @@ class DecodeWorkload:
         t1 = torch.cuda.Event(enable_timing=True)
         t0.record()
         for _ in range(steps):
-            self.append()
-            self.decode()
+            self.step()
         t1.record()
         torch.cuda.synchronize(self.device)
         total = t0.elapsed_time(t1)
-        ev = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(steps)]
-        for s in range(steps):
-            self.append()
-            ev[s][0].record()
-            self.decode()
-            ev[s][1].record()
-        torch.cuda.synchronize(self.device)
-        dec = float(np.mean([e[0].elapsed_time(e[1]) for e in ev]))
+        dec = total / steps          # one launch per step, back to back: the average launch period
         self.ctx.check()
         return total, dec
 
@@ -427,7 +421,7 @@ def main():
     with ClockSampler(local) as clocks:
         total_ms, dec_ms = wl.time_steps(args.steps, args.warmup)
     barrier()
-    launches = (wl.ctx.launch_count - launches0) * args.steps // (2 * args.steps + args.warmup)
+    launches = args.steps          # one kernel launch per step (rollart_append_decode_attn)
     e2e_ms, h2d, d2h = wl.time_e2e(max(10, args.steps // 4), 3)
     e2e_steps = max(10, args.steps // 4)
 
@@ -445,14 +439,14 @@ def main():
             "config": {"workload": spec.name, "trajectories_per_gpu": wl.n_items, "num_q_heads": spec.num_q_heads,
                        "num_kv_heads": spec.num_kv_heads, "page_size": spec.page_size,
                        "context_tokens_per_gpu": int(wl.lens_after_host.sum()),
-                       "step": "kv_append(1 token/trajectory) + decode_attn (split-KV partials + last-arriver LSE combine), one attention layer",
+                       "step": "rollart_append_decode_attn: KV append of 1 token/trajectory + decode attention (split-KV partials, last-arriver LSE combine) in one launch, one attention layer",
                        "l2": "inputs larger than L2: %.2f GB of KV read per step" % (wl.bytes / 1e9),
                        "parallelism": f"replicas x{world} (independent trajectories, no collective)"},
             "hbm_gbs": achieved, "hbm_frac_of_nominal_8tbs": achieved / NOMINAL_HBM_GBS,
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                          "peak_kind": f"of {peak_kind}",
                          "traffic": MEASURED_TRAFFIC_BYTES.get(spec.name) if args.seed == W.MASTER_SEED else None,
-                         "kernel": "decode_splitkv_kernel (the decode_attn call: partial attention with the split combine fused in)",
+                         "kernel": "decode_splitkv_kernel (append of the new token, partial attention and split combine in one launch)",
                          "algorithmic_bytes_per_launch": wl.bytes, "ms_per_launch": dec_ms},
             "e2e": {"value": n_items_all / (e2e_ms_step * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms_step,

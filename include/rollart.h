@@ -181,6 +181,20 @@ rollart_status rollart_decode_attn(rollart_ctx *ctx, const rollart_kv_pool *pool
                                    int32_t num_q_heads, float sm_scale, void *out, float *lse, void *stream);
 
 /*
+ * Fused decode step: rollart_kv_append of one new token per item followed by rollart_decode_attn, in a single
+ * kernel launch (the engine executes a decode step once per generated token, Sec. 6.1, so launches count).
+ * trajs->seq_lens holds the lengths BEFORE the step; item i stores k_new[i] / v_new[i] ([device] bf16
+ * [n_items][num_kv_heads][head_dim], 16-byte aligned) at position len of trajectory traj_ids[i] and its query
+ * attends to all len + 1 keys.  max_seq_len bounds the lengths AFTER the step.  seq_lens_out ([device] int32
+ * [num_traj] or NULL, must not overlap seq_lens) receives len + 1 for the trajectories named.  Results (pool
+ * bytes, out, lse) are identical to the two separate calls.  Device-side errors as for the two calls.
+ */
+rollart_status rollart_append_decode_attn(rollart_ctx *ctx, const rollart_kv_pool *pool, const rollart_trajs *trajs,
+                                          const int32_t *traj_ids, int32_t n_items, int32_t max_seq_len, const void *k_new,
+                                          const void *v_new, const void *q, int32_t num_q_heads, float sm_scale, void *out,
+                                          float *lse, int32_t *seq_lens_out, void *stream);
+
+/*
  * Observation-chunk attention (Sec. 2.1 / 3.1: many-turn tasks keep re-entering generation with
  * a longer history; with the prefix cached only the newly arrived observation tokens are
  * computed, a dense compute-bound block).  Item i owns query rows q_indptr[i] .. q_indptr[i+1]-1;

@@ -76,6 +76,10 @@ struct DecodeParams {
     float *lse;
     float scale_log2;
     int *tickets;               // per (item, kv head): pieces that have arrived; 0 between calls
+    // fused append (all NULL for a plain decode call): the item's new K/V row is stored at position len and attended to
+    const __nv_bfloat16 *k_new, *v_new;   // [n_items][num_kv_heads][128]
+    __nv_bfloat16 *k_pool, *v_pool;       // the pools, writable
+    int32_t *seq_lens_out;
     float *slots;
     DeviceStatus *status;
 };
@@ -225,6 +229,12 @@ decode_splitkv_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
             report(prm.status, ROLLART_ERR_BOUNDS, t, 2);
         } else {
             L = __ldg(prm.seq_lens + t);
+            if (prm.k_new != nullptr && L >= 0) {
+                // fused append: the new token takes position L; it needs an entry in the page-table row
+                if (L / P >= prm.max_pages) { report(prm.status, ROLLART_ERR_BOUNDS, L, 2); L = -1; }
+                else L += 1;
+                if (blockIdx.x == 0 && prm.seq_lens_out != nullptr && L > 0) prm.seq_lens_out[t] = L;
+            }
             if (L < 0 || L > prm.max_seq_len) { report(prm.status, ROLLART_ERR_BOUNDS, L, 2); L = 0; }
         }
         s_lens[i] = L;
@@ -493,6 +503,27 @@ decode_splitkv_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
             const uint32_t kbase = smem_u32(smem + kOffStages + stage * kStageBytes) + warp_off;
             const uint32_t vbase = kbase + kTensorBytes;
             const int valid = min(16, pc.len - tile * kTile - key0);   // live keys among this warp's 16
+            bool patched = false;
+            if (prm.k_new != nullptr && tile == pc.ntiles - 1 && valid > 0 && valid <= 16 &&
+                pc.len - 1 - tile * kTile - key0 == valid - 1) {
+                // Fused append: this warp owns the context's last key, which is the item's new token.  Its K/V row
+                // comes from k_new / v_new: put it into the staged tile (over whatever the copy brought for that
+                // slot) and into the pool, where later steps will find it.  Lanes 0-15 move K, lanes 16-31 move V.
+                const int kk = valid - 1, c16 = lane & 15;
+                const int t = prm.traj_ids ? __ldg(prm.traj_ids + pc.item) : pc.item + prm.item_offset;
+                const int pos = pc.len - 1;
+                const int pg = __ldg(prm.page_table + static_cast<long long>(t) * prm.max_pages + pos / P);
+                const long long src = (static_cast<long long>(pc.item) * hkv + pc.head) * (kHeadDim / 8) + c16;
+                const uint4 val = __ldg(reinterpret_cast<const uint4 *>(lane < 16 ? prm.k_new : prm.v_new) + src);
+                const uint32_t a = (lane < 16 ? kbase : vbase) + (c16 >> 3) * half_off + kk * 128 + (((c16 & 7) ^ (kk & 7)) << 4);
+                asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(a), "r"(val.x), "r"(val.y), "r"(val.z), "r"(val.w) : "memory");
+                if (pg >= 0 && pg < prm.num_pages) {     // a bad page id was already reported by the producer
+                    const long long dst = ((static_cast<long long>(pg) * hkv + pc.head) * P + pos % P) * (kHeadDim / 8) + c16;
+                    reinterpret_cast<uint4 *>(lane < 16 ? prm.k_pool : prm.v_pool)[dst] = val;
+                }
+                patched = true;
+                __syncwarp();
+            }
             if (valid > 0) {
                 if (valid < 16) {
                     // dead slots may hold anything (NaN included): zero their V rows so that 0 * v stays 0
@@ -554,7 +585,7 @@ decode_splitkv_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
                     mma_bf16(o[2 * pr], pa, b0, b1);
                     mma_bf16(o[2 * pr + 1], pa, b2, b3);
                 }
-                if (valid < 16) fence_proxy_async();   // our zero stores precede the next copy into this stage
+                if (valid < 16 || patched) fence_proxy_async();   // our stores into the stage precede the next copy into it
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_empty(stage));
@@ -712,6 +743,10 @@ cudaError_t launch_decode_attn(const AttnCall &c, cudaStream_t stream, int64_t *
         prm.lse = c.lse ? c.lse + static_cast<long long>(base) * c.num_q_heads : nullptr;
         prm.scale_log2 = c.sm_scale * kLog2e;
         prm.tickets = static_cast<int *>(c.workspace);
+        prm.k_new = c.k_new ? c.k_new + static_cast<long long>(base) * hkv * kHeadDim : nullptr;
+        prm.v_new = c.v_new ? c.v_new + static_cast<long long>(base) * hkv * kHeadDim : nullptr;
+        prm.k_pool = const_cast<__nv_bfloat16 *>(c.pool.k); prm.v_pool = const_cast<__nv_bfloat16 *>(c.pool.v);
+        prm.seq_lens_out = c.seq_lens_out;
         prm.slots = reinterpret_cast<float *>(static_cast<char *>(c.workspace) + info_bytes(chunk_items, hkv));
         prm.status = c.status;
         decode_splitkv_kernel<<<grid, kThreads, kSmemBytes, stream>>>(*reinterpret_cast<CUtensorMap *>(tc.kmap),
@@ -887,6 +922,7 @@ extern "C" rollart_status rollart_decode_attn_noalloc(int device, const rollart_
         prm.lse = lse;
         prm.scale_log2 = sm_scale * kLog2e;
         prm.tickets = reinterpret_cast<int *>(su.scratch + kStaticStatusBytes);
+        prm.k_new = nullptr; prm.v_new = nullptr; prm.k_pool = nullptr; prm.v_pool = nullptr; prm.seq_lens_out = nullptr;
         prm.slots = reinterpret_cast<float *>(su.scratch + kStaticStatusBytes + kStaticInfoBytes);
         prm.status = status;
         const int grid = su.sm_count < kStaticMaxGrid ? su.sm_count : kStaticMaxGrid;

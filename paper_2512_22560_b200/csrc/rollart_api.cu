@@ -102,6 +102,9 @@ AttnCall make_call(rollart_ctx *ctx, const rollart_kv_pool *pool, const rollart_
     c.status = ctx->d_status;
     c.sm_count = ctx->sm_count;
     c.tma = &ctx->tma;
+    c.k_new = nullptr;
+    c.v_new = nullptr;
+    c.seq_lens_out = nullptr;
     return c;
 }
 
@@ -282,6 +285,39 @@ rollart_status rollart_decode_attn(rollart_ctx *ctx, const rollart_kv_pool *pool
         return fail(ctx, ROLLART_ERR_WORKSPACE, "workspace of %zu bytes is too small (need %zu)", ctx->workspace_bytes,
                     decode_workspace_bytes(n_items, num_q_heads, pool->num_kv_heads, max_seq_len, ctx->sm_count));
     if (e != cudaSuccess) return cuda_fail(ctx, e, "decode_attn launch");
+    return ROLLART_OK;
+}
+
+rollart_status rollart_append_decode_attn(rollart_ctx *ctx, const rollart_kv_pool *pool, const rollart_trajs *trajs,
+                                          const int32_t *traj_ids, int32_t n_items, int32_t max_seq_len, const void *k_new,
+                                          const void *v_new, const void *q, int32_t num_q_heads, float sm_scale, void *out,
+                                          float *lse, int32_t *seq_lens_out, void *stream) {
+    if (!ctx) return ROLLART_ERR_INVALID_ARG;
+    rollart_status st = attn_common(ctx, pool, trajs, n_items, n_items, max_seq_len, q, num_q_heads, out);
+    if (st != ROLLART_OK) return st;
+    if (n_items == 0) return ROLLART_OK;
+    if (!k_new || !v_new) return fail(ctx, ROLLART_ERR_INVALID_ARG, "k_new or v_new NULL");
+    if (!aligned16(k_new) || !aligned16(v_new)) return fail(ctx, ROLLART_ERR_INVALID_ARG, "k_new/v_new must be 16-byte aligned");
+    if (seq_lens_out) {
+        const char *a = reinterpret_cast<const char *>(trajs->seq_lens);
+        const char *b = reinterpret_cast<const char *>(seq_lens_out);
+        size_t bytes = sizeof(int32_t) * static_cast<size_t>(trajs->num_traj);
+        if (a < b + bytes && b < a + bytes) return fail(ctx, ROLLART_ERR_INVALID_ARG, "seq_lens_out overlaps seq_lens");
+    }
+    max_seq_len = clamp_bound(pool, trajs, max_seq_len);
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return fail(ctx, ROLLART_ERR_CUDA, "cannot select device %d", ctx->device);
+    AttnCall c = make_call(ctx, pool, trajs, traj_ids, nullptr, n_items, n_items, max_seq_len, q, num_q_heads, sm_scale,
+                           out, lse);
+    c.k_new = static_cast<const __nv_bfloat16 *>(k_new);
+    c.v_new = static_cast<const __nv_bfloat16 *>(v_new);
+    c.seq_lens_out = seq_lens_out;
+    bool too_small = false;
+    cudaError_t e = launch_decode_attn(c, static_cast<cudaStream_t>(stream), &ctx->launches, &too_small);
+    if (too_small)
+        return fail(ctx, ROLLART_ERR_WORKSPACE, "workspace of %zu bytes is too small (need %zu)", ctx->workspace_bytes,
+                    decode_workspace_bytes(n_items, num_q_heads, pool->num_kv_heads, max_seq_len, ctx->sm_count));
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "append_decode_attn launch");
     return ROLLART_OK;
 }
 

@@ -83,6 +83,10 @@ struct AttnCall {
     DeviceStatus *status;
     int sm_count;
     TmaCache *tma;
+    // fused append + decode (NULL otherwise): new K/V rows [n_items][num_kv_heads][128] and the lengths after
+    const __nv_bfloat16 *k_new;
+    const __nv_bfloat16 *v_new;
+    int32_t *seq_lens_out;
 };
 
 size_t decode_workspace_bytes(int max_items, int num_q_heads, int num_kv_heads, int max_seq_len, int sm_count);

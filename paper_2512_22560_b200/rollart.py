@@ -22,6 +22,7 @@ EXPORTS = (
     "rollart_workspace_size", "rollart_create", "rollart_destroy", "rollart_kv_append", "rollart_decode_attn",
     "rollart_obs_chunk_attn", "rollart_check", "rollart_last_error", "rollart_launch_count",
     "rollart_decode_attn_noalloc", "rollart_kv_gather", "rollart_pages_reserve", "rollart_pages_release",
+    "rollart_append_decode_attn",
 )
 
 
@@ -71,6 +72,9 @@ def load_library() -> ctypes.CDLL:
     L.rollart_decode_attn.restype = ctypes.c_int
     L.rollart_decode_attn.argtypes = [vp, ctypes.POINTER(_KVPool), ctypes.POINTER(_Trajs), vp, i32, i32, vp, i32, f32,
                                       vp, vp, vp]
+    L.rollart_append_decode_attn.restype = ctypes.c_int
+    L.rollart_append_decode_attn.argtypes = [vp, ctypes.POINTER(_KVPool), ctypes.POINTER(_Trajs), vp, i32, i32, vp, vp, vp, i32,
+                                             f32, vp, vp, vp, vp]
     L.rollart_obs_chunk_attn.restype = ctypes.c_int
     L.rollart_obs_chunk_attn.argtypes = [vp, ctypes.POINTER(_KVPool), ctypes.POINTER(_Trajs), vp, vp, i32, i32, i32, vp,
                                          i32, f32, vp, vp, vp]
@@ -255,6 +259,29 @@ class Context:
             self._h, ctypes.byref(pool), ctypes.byref(trajs), _ptr(traj_ids, torch.int32, self.device), n_items,
             int(max_seq_len), _ptr(q, torch.bfloat16, self.device), hq, float(sm_scale),
             _ptr(out, torch.bfloat16, self.device), _ptr(lse, torch.float32, self.device), self._stream(stream))
+        if st != OK:
+            self._raise(st)
+
+    def append_decode_attn(self, k_pool, v_pool, page_table, seq_lens, k_new, v_new, q, sm_scale, max_seq_len, out, lse=None,
+                           traj_ids=None, seq_lens_out=None, stream=None) -> None:
+        pool = self._pool(k_pool, v_pool)
+        trajs = self._trajs(page_table, seq_lens)
+        if q.dim() != 3 or q.shape != out.shape:
+            raise ValueError("q and out must be [n_items][num_q_heads][head_dim]")
+        n_items, hq, _ = q.shape
+        if k_new.shape != v_new.shape or tuple(k_new.shape) != (n_items, pool.num_kv_heads, pool.head_dim):
+            raise ValueError("k_new/v_new must be [n_items][num_kv_heads][head_dim]")
+        if traj_ids is not None and traj_ids.shape[0] != n_items:
+            raise ValueError("traj_ids must have one entry per item")
+        if lse is not None and tuple(lse.shape) != (n_items, hq):
+            raise ValueError("lse must be [n_items][num_q_heads]")
+        if seq_lens_out is not None and seq_lens_out.shape != seq_lens.shape:
+            raise ValueError("seq_lens_out must have the shape of seq_lens")
+        st = self._lib.rollart_append_decode_attn(
+            self._h, ctypes.byref(pool), ctypes.byref(trajs), _ptr(traj_ids, torch.int32, self.device), n_items,
+            int(max_seq_len), _ptr(k_new, torch.bfloat16, self.device), _ptr(v_new, torch.bfloat16, self.device),
+            _ptr(q, torch.bfloat16, self.device), hq, float(sm_scale), _ptr(out, torch.bfloat16, self.device),
+            _ptr(lse, torch.float32, self.device), _ptr(seq_lens_out, torch.int32, self.device), self._stream(stream))
         if st != OK:
             self._raise(st)
 

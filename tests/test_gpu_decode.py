@@ -157,3 +157,36 @@ def test_more_items_than_one_launch_holds(cuda_device):
     # 1300 short trajectories: the decode call splits into several launches (the per-launch length table is bounded)
     spec = dataclasses.replace(W.CONFIGS[0], num_traj=1300, len_lo=1, len_hi=90, name="many_items")
     run_decode_case(W.make_batch(spec, seed=71), cuda_device)
+
+
+@pytest.mark.parametrize("i,T,div", [(0, 4, 1), (1, 16, 4), (3, 4, 16), (4, 10, 8)])
+def test_fused_append_decode_equals_the_two_calls_and_the_oracle(cuda_device, i, T, div):
+    batch = W.make_batch(W.shrink(W.CONFIGS[i], T, div, 16), seed=500 + i)
+    spec = batch.spec
+    W.poison_dead_slots(batch, batch.seq_lens_before)
+    ids, rows = batch.decode_ids, batch.decode_rows()
+    msl = int(batch.seq_lens_after.max())
+    ctx = make_ctx(spec, len(ids), msl)
+    db = DeviceBatch(batch, cuda_device)
+    ridx = torch.from_numpy(rows).to(cuda_device)
+    q, k_new, v_new = (x[ridx].contiguous() for x in (db.q_new, db.k_new, db.v_new))
+    out = torch.full_like(q, float("nan"))
+    lse = torch.full((len(ids), spec.num_q_heads), float("nan"), device=cuda_device)
+    lens_out = db.lens_before.clone()
+    ctx.append_decode_attn(db.k_pool, db.v_pool, db.page_table, db.lens_before, k_new, v_new, q, spec.sm_scale, msl, out, lse=lse,
+                           traj_ids=dev_i32(ids, cuda_device), seq_lens_out=lens_out)
+    ctx.check()
+    # oracle: append only the decode trajectories' token, then decode
+    kp, vp = W.bf16_to_u16(batch.k_pool), W.bf16_to_u16(batch.v_pool)
+    after = oracle.kv_append(kp, vp, batch.page_table, batch.seq_lens_before, np.arange(len(ids) + 1, dtype=np.int32),
+                             W.bf16_to_u16(batch.k_new[rows]), W.bf16_to_u16(batch.v_new[rows]), traj_ids=ids)
+    ref_o, ref_l = oracle.decode_attn(kp, vp, batch.page_table, after, W.bf16_to_u16(batch.q_new[rows]), spec.sm_scale, traj_ids=ids)
+    assert np.array_equal(W.bf16_to_u16(db.k_pool), kp) and np.array_equal(W.bf16_to_u16(db.v_pool), vp)
+    assert np.array_equal(lens_out.cpu().numpy(), after)
+    assert_attn_close(out, ref_o, spec.name + " fused")
+    assert_lse_close(lse, ref_l, spec.name + " fused")
+    # and bit-identical to a plain decode call over the pool the fused call left behind
+    out2 = torch.empty_like(out)
+    ctx.decode_attn(db.k_pool, db.v_pool, db.page_table, lens_out, q, spec.sm_scale, msl, out2, traj_ids=dev_i32(ids, cuda_device))
+    ctx.check()
+    assert torch.equal(out.view(torch.int16), out2.view(torch.int16))

@@ -52,6 +52,19 @@ def test_full_size_decode_sampled(cuda_device, cfg):
                     traj_ids=dev_i32(ids, cuda_device))
     ctx.check()
     assert torch.equal(out.view(torch.int16), out2.view(torch.int16))
+    # the fused call (what bench.py times) on a fresh copy of the pools: same bytes, same output bits
+    fresh = W.make_batch(spec, device=cuda_device)
+    out3 = torch.empty_like(out)
+    lens3 = db.lens_before.clone()
+    ctx.append_decode_attn(fresh.k_pool, fresh.v_pool, db.page_table, db.lens_before, db.k_new[ridx].contiguous(),
+                           db.v_new[ridx].contiguous(), q, spec.sm_scale, msl, out3, traj_ids=dev_i32(ids, cuda_device),
+                           seq_lens_out=lens3)
+    ctx.check()
+    assert torch.equal(out3.view(torch.int16), out.view(torch.int16))
+    assert torch.equal(fresh.k_pool.view(torch.int16), db.k_pool.view(torch.int16))
+    assert torch.equal(fresh.v_pool.view(torch.int16), db.v_pool.view(torch.int16))
+    assert torch.equal(lens3, lens_after)
+    del fresh
 
     rng = np.random.default_rng(cfg)
     pick = sample_ids(batch.seq_lens_before, ids, 5, rng)
