@@ -207,6 +207,58 @@ class DecodeWorkload:
         return dt * 1e3, stage_host.numel() * 2, hout.numel() * 2
 
 
+class GroupDecodeWorkload:
+    """GRPO groups whose members alias a shared prompt prefix: one decode step is the KV append of the new
+    tokens followed by the group decode call (prefix read once per group)."""
+
+    def __init__(self, spec: W.WorkloadSpec, seed: int, device: torch.device, group_size: int, fraction: float):
+        from paper_2512_22560_b200 import rollart
+        self.spec = spec
+        self.device = device
+        layout = W.make_layout(spec, seed)
+        indptr, shared = W.share_group_prefix(layout, group_size, fraction)
+        b = W.fill_tensors(layout, device)
+        self.batch = b
+        i32 = lambda a: torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).to(device)
+        self.table, self.lens0, self.lens1 = i32(b.page_table), i32(b.seq_lens_before), i32(b.seq_lens_after)
+        self.group_indptr, self.shared = i32(indptr), i32(shared)
+        self.new_indptr = i32(b.new_indptr)
+        self.q = b.q_new.contiguous()
+        self.out = torch.empty_like(self.q)
+        self.max_seq_len = int(b.seq_lens_after.max())
+        self.n_items = spec.num_traj
+        self.ctx = rollart.Context(device.index or 0, rollart.group_decode_workspace_size(
+            self.n_items, spec.num_q_heads, spec.num_kv_heads, self.max_seq_len))
+        per_token = 2 * spec.num_kv_heads * spec.head_dim * 2
+        self.bytes_per_trajectory_definition = decode_algorithmic_bytes(spec, b.seq_lens_after)
+        members = np.diff(indptr).astype(np.int64)
+        self.bytes_unique = self.bytes_per_trajectory_definition - int(((members - 1).clip(min=0) * shared).sum()) * per_token
+
+    def step_group(self):
+        b = self.batch
+        self.ctx.kv_append(b.k_pool, b.v_pool, self.table, self.lens0, self.new_indptr, b.k_new, b.v_new, seq_lens_out=self.lens1)
+        self.ctx.group_decode_attn(b.k_pool, b.v_pool, self.table, self.lens1, self.group_indptr, self.shared, self.q,
+                                   self.spec.sm_scale, self.max_seq_len, self.out)
+
+    def step_plain(self):
+        b = self.batch
+        self.ctx.append_decode_attn(b.k_pool, b.v_pool, self.table, self.lens0, b.k_new, b.v_new, self.q, self.spec.sm_scale,
+                                    self.max_seq_len, self.out, seq_lens_out=self.lens1)
+
+    def time(self, fn, steps: int, warmup: int) -> float:
+        for _ in range(warmup):
+            fn()
+        torch.cuda.synchronize(self.device)
+        t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t0.record()
+        for _ in range(steps):
+            fn()
+        t1.record()
+        torch.cuda.synchronize(self.device)
+        self.ctx.check()
+        return t0.elapsed_time(t1) / steps
+
+
 def chunk_flops(spec: W.WorkloadSpec, lens_after: np.ndarray, n_new: np.ndarray) -> float:
     """Causal-exact flops of the chunk call: every (row, visible key) pair costs 4*D per q head (QK^T and PV)."""
     pairs = 0
@@ -505,6 +557,24 @@ def main():
                 torch.cuda.empty_cache()
             except Exception as e:
                 extra[W.RECOMPUTE.name] = {"error": repr(e)}
+            for frac in (W.GROUP_SHARED_FRACTION, 1.0):
+                name = "%s_shared%.2f" % (W.GROUP_DECODE.name, frac)
+                try:
+                    gw = GroupDecodeWorkload(W.GROUP_DECODE, args.seed, device, W.GROUP_SIZE, frac)
+                    g_ms = gw.time(gw.step_group, 20, 3)
+                    p_ms = gw.time(gw.step_plain, 20, 3)
+                    extra[name] = {
+                        "trajectories": gw.n_items, "group_size": W.GROUP_SIZE, "shared_fraction_of_shortest_member": frac,
+                        "group_step_ms": g_ms, "plain_step_ms": p_ms, "speedup_over_plain_step": p_ms / g_ms,
+                        "decode_tokens_per_s": gw.n_items / (g_ms * 1e-3),
+                        "bytes_per_trajectory_definition": gw.bytes_per_trajectory_definition,
+                        "bytes_unique_pages": gw.bytes_unique, "unique_gbs": gw.bytes_unique / (g_ms * 1e-3) / 1e9,
+                        "plain_gbs": gw.bytes_per_trajectory_definition / (p_ms * 1e-3) / 1e9}
+                    gw.ctx.close()
+                    del gw
+                    torch.cuda.empty_cache()
+                except Exception as e:
+                    extra[name] = {"error": repr(e)}
             line["other_workloads"] = extra
             info, _, _ = CpuBaseline(spec, args.seed).measure()
             line["cpu_baseline"] = info

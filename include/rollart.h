@@ -195,6 +195,35 @@ rollart_status rollart_append_decode_attn(rollart_ctx *ctx, const rollart_kv_poo
                                           float *lse, int32_t *seq_lens_out, void *stream);
 
 /*
+ * Group decode step: rollart_decode_attn for a batch whose items form groups that share a prompt prefix.
+ * The paper trains with GRPO at a group size of 8 and runs the rollout engine with prefix caching (Sec. 7.1),
+ * so the members of a group hold the same first tokens and, with prefix sharing, their page-table rows list
+ * the same physical pages there.  Results are those of rollart_decode_attn (same definition of out and lse);
+ * the shared pages are read once per group instead of once per member: the prefix part runs on the tensor
+ * cores with the members' query rows stacked into one tile, the private remainder through the split-KV decode
+ * kernel, and the two parts are merged from their log-sum-exps (fp32 partial results, one rounding to bf16).
+ *
+ *   group_indptr   [device] int32 [n_groups + 1]: group j holds items group_indptr[j] .. group_indptr[j+1]-1
+ *                  (consecutive items of the batch; starts at 0, ends at n_items, non-decreasing).
+ *   shared_lens    [device] int32 [n_groups]: tokens of the shared prefix; a whole number of pages (0 allowed),
+ *                  not longer than any member's seq_lens entry.  For pages below shared_lens[j] / page_size the
+ *                  members' page-table rows must hold identical entries.
+ *   other arguments as for rollart_decode_attn.
+ * Workspace: rollart_group_decode_workspace_size(...) bytes (more than rollart_workspace_size: it adds two
+ * fp32 partial results per item); a smaller workspace returns ROLLART_ERR_WORKSPACE and launches nothing.
+ * Device-side checks: a group_indptr that is not such a partition, a shared length that is not page aligned
+ * or exceeds a member's length, and members whose rows differ on the shared pages are each reported as
+ * ROLLART_ERR_BOUNDS (the results of that call are then undefined, memory outside out/lse is not touched).
+ * Launches four kernels.  Groups of one member and shared_lens of 0 are valid (no saving).
+ */
+size_t rollart_group_decode_workspace_size(int32_t max_items, int32_t num_q_heads, int32_t num_kv_heads,
+                                           int32_t max_seq_len);
+rollart_status rollart_group_decode_attn(rollart_ctx *ctx, const rollart_kv_pool *pool, const rollart_trajs *trajs,
+                                         const int32_t *traj_ids, int32_t n_items, const int32_t *group_indptr,
+                                         const int32_t *shared_lens, int32_t n_groups, int32_t max_seq_len, const void *q,
+                                         int32_t num_q_heads, float sm_scale, void *out, float *lse, void *stream);
+
+/*
  * Observation-chunk attention (Sec. 2.1 / 3.1: many-turn tasks keep re-entering generation with
  * a longer history; with the prefix cached only the newly arrived observation tokens are
  * computed, a dense compute-bound block).  Item i owns query rows q_indptr[i] .. q_indptr[i+1]-1;

@@ -65,6 +65,9 @@ struct ChunkParams {
     __nv_bfloat16 *out;
     float *lse;
     float scale_log2;
+    // shared-prefix mode (NULL otherwise): every row of item i sees exactly the first shared_lens[i] keys, no causal mask
+    const int32_t *shared_lens;
+    float *out_f32;             // when set, result rows go here in fp32 instead of bf16 to `out`
     DeviceStatus *status;
 };
 
@@ -295,17 +298,29 @@ chunk_attn_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constan
     if (*reinterpret_cast<volatile int *>(&prm.status->fatal) != 0) return;   // an earlier block ran out of patience: give up quickly
 
     // ---- geometry of this unit ----
+    const bool shared_mode = prm.shared_lens != nullptr;
     const int q_row0 = __ldg(prm.q_indptr + item);
     const int n_chunk = __ldg(prm.q_indptr + item + 1) - q_row0;
     const int t = prm.traj_ids ? __ldg(prm.traj_ids + item) : item + prm.item_offset;
     int L = 0;
     bool bad = false;
-    if (t < 0 || t >= prm.num_traj) {
+    if (q_row0 < 0 || n_chunk < 0 || static_cast<long long>(q_row0) + n_chunk > prm.total_q) {
+        bad = true;                  // q_indptr does not describe rows of q
+        if (threadIdx.x == 0) report(prm.status, ROLLART_ERR_BOUNDS, q_row0, 3);
+    } else if (t < 0 || t >= prm.num_traj) {
         bad = true;
         if (threadIdx.x == 0) report(prm.status, ROLLART_ERR_BOUNDS, t, 3);
     } else {
         L = __ldg(prm.seq_lens + t);
-        if (L < 0 || L > prm.max_seq_len || n_chunk > L) {
+        if (shared_mode) {
+            const int s_len = __ldg(prm.shared_lens + item);
+            if (s_len < 0 || s_len > L) {
+                bad = true;
+                if (threadIdx.x == 0) report(prm.status, ROLLART_ERR_BOUNDS, s_len, 3);
+            }
+            L = s_len;               // keys beyond the shared prefix do not exist for this call
+        }
+        if (!bad && (L < 0 || L > prm.max_seq_len || (!shared_mode && n_chunk > L))) {
             bad = true;
             if (threadIdx.x == 0) report(prm.status, ROLLART_ERR_BOUNDS, L, 3);
         }
@@ -314,10 +329,22 @@ chunk_attn_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constan
     const int prior = L - n_chunk;
     const int tok0 = mtile * tpt;                              // first chunk token of this M-tile
     const int toks = min(tpt, n_chunk - tok0);                 // live tokens
-    const int max_count = prior + tok0 + toks;                 // keys visible to the last live row
-    const int min_count = prior + tok0 + 1;                    // keys visible to the first row
+    const int max_count = shared_mode ? L : prior + tok0 + toks;   // keys visible to the last live row
+    const int min_count = shared_mode ? L : prior + tok0 + 1;      // keys visible to the first row
     const int n_tiles = (max_count + kKeys - 1) / kKeys;
     const int32_t *table_row = prm.page_table + static_cast<long long>(t) * prm.max_pages;
+    if (n_tiles == 0) {
+        // only in shared-prefix mode with an empty prefix: the result is out = 0, lse = -inf
+        for (int idx = threadIdx.x; idx < toks * g * (kHeadDim / 4); idx += kThreads) {
+            const int r = idx / (kHeadDim / 4), c = idx - r * (kHeadDim / 4);
+            const int tk = r / g, hd = r - tk * g;
+            const long long orow = static_cast<long long>(q_row0 + tok0 + tk) * prm.num_q_heads + head * g + hd;
+            if (prm.out_f32 != nullptr) reinterpret_cast<float4 *>(prm.out_f32 + orow * kHeadDim)[c] = make_float4(0.f, 0.f, 0.f, 0.f);
+            else reinterpret_cast<uint2 *>(prm.out + orow * kHeadDim)[c] = make_uint2(0u, 0u);
+            if (c == 0 && prm.lse != nullptr) prm.lse[orow] = -INFINITY;
+        }
+        return;                      // uniform over the block, before any barrier or TMEM use
+    }
 
     // zero the Q tile (rows beyond tpt * g are never written by the copy) and allocate TMEM
     for (int i = threadIdx.x; i < 2 * kHalfQ / 16; i += kThreads) reinterpret_cast<uint4 *>(smem + kOffQ)[i] = make_uint4(0, 0, 0, 0);
@@ -420,7 +447,7 @@ chunk_attn_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constan
         const uint32_t lane_addr = tmem + (static_cast<uint32_t>(quarter * 32) << 16);
         const int tok_local = row / g, head_local = row - tok_local * g;
         const bool live = tok_local < toks;
-        const int count = min(L, prior + tok0 + min(tok_local, toks - 1) + 1);   // keys this row sees (>= 1)
+        const int count = shared_mode ? L : min(L, prior + tok0 + min(tok_local, toks - 1) + 1);   // keys this row sees (>= 1)
         float m_ref = -INFINITY, l_sum = 0.f;
 
         for (int j = 0; j < n_tiles; ++j) {
@@ -538,7 +565,13 @@ chunk_attn_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constan
             uint32_t oraw[32];
             tmem_ld32(lane_addr + 128 + c0, oraw);
             tmem_wait_ld();
-            if (live) {
+            if (live && prm.out_f32 != nullptr) {
+                float4 *dst = reinterpret_cast<float4 *>(prm.out_f32 + orow * kHeadDim + c0);
+#pragma unroll
+                for (int k = 0; k < 8; ++k)
+                    dst[k] = make_float4(__uint_as_float(oraw[4 * k]) * inv, __uint_as_float(oraw[4 * k + 1]) * inv,
+                                         __uint_as_float(oraw[4 * k + 2]) * inv, __uint_as_float(oraw[4 * k + 3]) * inv);
+            } else if (live) {
                 uint4 *dst = reinterpret_cast<uint4 *>(prm.out + orow * kHeadDim + c0);
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {
@@ -628,6 +661,8 @@ cudaError_t launch_chunk_attn(const AttnCall &c, cudaStream_t stream, int64_t *l
         prm.page_size = c.pool.page_size; prm.num_kv_heads = hkv; prm.num_q_heads = c.num_q_heads; prm.group = g;
         prm.n_items = n; prm.item_offset = base; prm.max_seq_len = c.max_seq_len; prm.total_q = c.total_q;
         prm.out = c.out; prm.lse = c.lse; prm.scale_log2 = c.sm_scale * kLog2e; prm.status = c.status;
+        prm.shared_lens = c.shared_lens ? c.shared_lens + base : nullptr;
+        prm.out_f32 = c.out_f32;
         // an upper bound on the M-tiles of these items: every item has at most one ragged tile
         const long long tiles = (static_cast<long long>(c.total_q) + tpt - 1) / tpt + n;
         const long long blocks = tiles * hkv;

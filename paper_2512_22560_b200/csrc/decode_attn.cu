@@ -80,6 +80,9 @@ struct DecodeParams {
     const __nv_bfloat16 *k_new, *v_new;   // [n_items][num_kv_heads][128]
     __nv_bfloat16 *k_pool, *v_pool;       // the pools, writable
     int32_t *seq_lens_out;
+    // group decode (NULL otherwise): per item, the first page_offset[i] pages of the table row are skipped
+    const int32_t *page_offset;
+    float *out_f32;             // when set, result rows go here in fp32 instead of bf16 to `out`
     float *slots;
     DeviceStatus *status;
 };
@@ -154,6 +157,16 @@ __device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], 
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t *>(&v);
+}
+// four consecutive result values of one row, at element index idx of the output
+__device__ __forceinline__ void store_out4(const DecodeParams &prm, long long idx, float a, float b, float c, float d) {
+    if (prm.out_f32 != nullptr) {
+        *reinterpret_cast<float4 *>(prm.out_f32 + idx) = make_float4(a, b, c, d);
+    } else {
+        uint2 packed;
+        packed.x = pack_bf16(a, b); packed.y = pack_bf16(c, d);
+        *reinterpret_cast<uint2 *>(prm.out + idx) = packed;
+    }
 }
 
 // One round of the end-of-piece merge: this warp adds (or, in the first round, stores) its two
@@ -236,6 +249,11 @@ decode_splitkv_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
                 if (blockIdx.x == 0 && prm.seq_lens_out != nullptr && L > 0) prm.seq_lens_out[t] = L;
             }
             if (L < 0 || L > prm.max_seq_len) { report(prm.status, ROLLART_ERR_BOUNDS, L, 2); L = 0; }
+            if (prm.page_offset != nullptr) {
+                const int off = __ldg(prm.page_offset + i);
+                if (off < 0 || static_cast<long long>(off) * P > L) { report(prm.status, ROLLART_ERR_BOUNDS, off, 2); L = 0; }
+                else L -= off * P;
+            }
         }
         s_lens[i] = L;
     }
@@ -272,8 +290,13 @@ decode_splitkv_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
         // trajectories without keys have no tile and no piece: their result is out = 0, lse = -inf
         for (int i = 0; i < prm.n_items; ++i) {
             if (s_lens[i] != 0) continue;
-            uint4 *o = reinterpret_cast<uint4 *>(prm.out + static_cast<long long>(i) * prm.num_q_heads * kHeadDim);
-            for (int k = threadIdx.x; k < prm.num_q_heads * kHeadDim / 8; k += kThreads) o[k] = make_uint4(0, 0, 0, 0);
+            if (prm.out_f32 != nullptr) {
+                float4 *o = reinterpret_cast<float4 *>(prm.out_f32 + static_cast<long long>(i) * prm.num_q_heads * kHeadDim);
+                for (int k = threadIdx.x; k < prm.num_q_heads * kHeadDim / 4; k += kThreads) o[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+            } else {
+                uint4 *o = reinterpret_cast<uint4 *>(prm.out + static_cast<long long>(i) * prm.num_q_heads * kHeadDim);
+                for (int k = threadIdx.x; k < prm.num_q_heads * kHeadDim / 8; k += kThreads) o[k] = make_uint4(0, 0, 0, 0);
+            }
             if (prm.lse != nullptr)
                 for (int k = threadIdx.x; k < prm.num_q_heads; k += kThreads)
                     prm.lse[static_cast<long long>(i) * prm.num_q_heads + k] = -INFINITY;
@@ -293,7 +316,8 @@ decode_splitkv_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
         for (int p = p_begin; p < p_end; ++pcount) {
             const Piece pc = piece_at(s_prefix, s_lens, prm.n_items, hkv, p, p_end);
             const int t = prm.traj_ids ? __ldg(prm.traj_ids + pc.item) : pc.item + prm.item_offset;
-            const int32_t *table_row = prm.page_table + static_cast<long long>(t) * prm.max_pages;
+            const int32_t *table_row = prm.page_table + static_cast<long long>(t) * prm.max_pages +
+                                       (prm.page_offset ? __ldg(prm.page_offset + pc.item) : 0);
             // Q rows of this (item, kv head): g contiguous rows of 256 B
             const int qs = pcount & 1;
             mbar_wait(bar_qempty(qs), ((pcount >> 1) & 1) ^ 1, s_abort, prm.status, 1);
@@ -378,9 +402,7 @@ decode_splitkv_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
                     const float lsum = __shfl_sync(0xffffffffu, lrow, row);
                     const float inv = lsum > 0.f ? 1.f / lsum : 0.f;
                     const float4 x = *reinterpret_cast<const float4 *>(mg + row * kMergeStride + lane * 4);
-                    uint2 packed;
-                    packed.x = pack_bf16(x.x * inv, x.y * inv); packed.y = pack_bf16(x.z * inv, x.w * inv);
-                    *reinterpret_cast<uint2 *>(prm.out + obase + row * kHeadDim) = packed;
+                    store_out4(prm, obase + row * kHeadDim, x.x * inv, x.y * inv, x.z * inv, x.w * inv);
                 }
                 if (prm.lse != nullptr && lane < g) prm.lse[lbase + lane] = lrow > 0.f ? (Mrow + log2f(lrow)) * kLn2 : -INFINITY;
             } else {
@@ -446,9 +468,7 @@ decode_splitkv_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
                         const float lsum = __shfl_sync(0xffffffffu, lall, r);
                         if (r < g) {
                             const float inv = lsum > 0.f ? 1.f / lsum : 0.f;
-                            uint2 packed;
-                            packed.x = pack_bf16(acc[r][0] * inv, acc[r][1] * inv); packed.y = pack_bf16(acc[r][2] * inv, acc[r][3] * inv);
-                            *reinterpret_cast<uint2 *>(prm.out + obase + r * kHeadDim) = packed;
+                            store_out4(prm, obase + r * kHeadDim, acc[r][0] * inv, acc[r][1] * inv, acc[r][2] * inv, acc[r][3] * inv);
                         }
                     }
                     if (prm.lse != nullptr && lane < g) prm.lse[lbase + lane] = lall > 0.f ? (Mall + log2f(lall)) * kLn2 : -INFINITY;
@@ -747,6 +767,8 @@ cudaError_t launch_decode_attn(const AttnCall &c, cudaStream_t stream, int64_t *
         prm.v_new = c.v_new ? c.v_new + static_cast<long long>(base) * hkv * kHeadDim : nullptr;
         prm.k_pool = const_cast<__nv_bfloat16 *>(c.pool.k); prm.v_pool = const_cast<__nv_bfloat16 *>(c.pool.v);
         prm.seq_lens_out = c.seq_lens_out;
+        prm.page_offset = c.page_offset ? c.page_offset + base : nullptr;
+        prm.out_f32 = c.out_f32 ? c.out_f32 + static_cast<long long>(base) * c.num_q_heads * kHeadDim : nullptr;
         prm.slots = reinterpret_cast<float *>(static_cast<char *>(c.workspace) + info_bytes(chunk_items, hkv));
         prm.status = c.status;
         decode_splitkv_kernel<<<grid, kThreads, kSmemBytes, stream>>>(*reinterpret_cast<CUtensorMap *>(tc.kmap),
@@ -923,6 +945,7 @@ extern "C" rollart_status rollart_decode_attn_noalloc(int device, const rollart_
         prm.scale_log2 = sm_scale * kLog2e;
         prm.tickets = reinterpret_cast<int *>(su.scratch + kStaticStatusBytes);
         prm.k_new = nullptr; prm.v_new = nullptr; prm.k_pool = nullptr; prm.v_pool = nullptr; prm.seq_lens_out = nullptr;
+        prm.page_offset = nullptr; prm.out_f32 = nullptr;
         prm.slots = reinterpret_cast<float *>(su.scratch + kStaticStatusBytes + kStaticInfoBytes);
         prm.status = status;
         const int grid = su.sm_count < kStaticMaxGrid ? su.sm_count : kStaticMaxGrid;

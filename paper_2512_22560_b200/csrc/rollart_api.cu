@@ -105,6 +105,9 @@ AttnCall make_call(rollart_ctx *ctx, const rollart_kv_pool *pool, const rollart_
     c.k_new = nullptr;
     c.v_new = nullptr;
     c.seq_lens_out = nullptr;
+    c.page_offset = nullptr;
+    c.shared_lens = nullptr;
+    c.out_f32 = nullptr;
     return c;
 }
 
@@ -321,6 +324,90 @@ rollart_status rollart_append_decode_attn(rollart_ctx *ctx, const rollart_kv_poo
     return ROLLART_OK;
 }
 
+namespace {
+// Workspace of a group decode call: the decode kernel's own workspace first, then these arrays.
+struct GroupLayout {
+    size_t group_traj, item_off, lse_a, lse_b, part_a, part_b, total;
+};
+GroupLayout group_layout(int n_items, int num_q_heads, int num_kv_heads, int max_seq_len, int sm_count) {
+    auto up = [](size_t x) { return (x + 255) & ~size_t(255); };
+    const size_t rows = static_cast<size_t>(n_items) * num_q_heads;
+    GroupLayout g;
+    size_t at = up(decode_workspace_bytes(n_items, num_q_heads, num_kv_heads, max_seq_len, sm_count));
+    g.group_traj = at; at += up(sizeof(int32_t) * static_cast<size_t>(n_items));
+    g.item_off = at;   at += up(sizeof(int32_t) * static_cast<size_t>(n_items));
+    g.lse_a = at;      at += up(sizeof(float) * rows);
+    g.lse_b = at;      at += up(sizeof(float) * rows);
+    g.part_a = at;     at += up(sizeof(float) * rows * kHeadDim);
+    g.part_b = at;     at += up(sizeof(float) * rows * kHeadDim);
+    g.total = at;
+    return g;
+}
+}  // namespace
+
+size_t rollart_group_decode_workspace_size(int32_t max_items, int32_t num_q_heads, int32_t num_kv_heads, int32_t max_seq_len) {
+    if (max_items <= 0 || num_q_heads <= 0 || num_kv_heads <= 0 || max_seq_len < 0) return 0;
+    return group_layout(max_items, num_q_heads, num_kv_heads, max_seq_len, /*sm_count=*/0).total;
+}
+
+rollart_status rollart_group_decode_attn(rollart_ctx *ctx, const rollart_kv_pool *pool, const rollart_trajs *trajs,
+                                         const int32_t *traj_ids, int32_t n_items, const int32_t *group_indptr,
+                                         const int32_t *shared_lens, int32_t n_groups, int32_t max_seq_len, const void *q,
+                                         int32_t num_q_heads, float sm_scale, void *out, float *lse, void *stream_) {
+    if (!ctx) return ROLLART_ERR_INVALID_ARG;
+    rollart_status st = attn_common(ctx, pool, trajs, n_items, n_items, max_seq_len, q, num_q_heads, out);
+    if (st != ROLLART_OK) return st;
+    if (n_groups < 0 || n_groups > n_items) return fail(ctx, ROLLART_ERR_INVALID_ARG, "n_groups must lie in [0, n_items]");
+    if (n_items == 0) return ROLLART_OK;
+    if (n_groups == 0) return fail(ctx, ROLLART_ERR_INVALID_ARG, "items without groups");
+    if (!group_indptr || !shared_lens) return fail(ctx, ROLLART_ERR_INVALID_ARG, "group_indptr or shared_lens NULL");
+    max_seq_len = clamp_bound(pool, trajs, max_seq_len);
+    const GroupLayout lay = group_layout(n_items, num_q_heads, pool->num_kv_heads, max_seq_len, ctx->sm_count);
+    if (!ctx->workspace || lay.total > ctx->workspace_bytes)
+        return fail(ctx, ROLLART_ERR_WORKSPACE, "workspace of %zu bytes is too small (need %zu)", ctx->workspace_bytes, lay.total);
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return fail(ctx, ROLLART_ERR_CUDA, "cannot select device %d", ctx->device);
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    char *ws = static_cast<char *>(ctx->workspace);
+    int32_t *group_traj = reinterpret_cast<int32_t *>(ws + lay.group_traj);
+    int32_t *item_off = reinterpret_cast<int32_t *>(ws + lay.item_off);
+    float *lse_a = reinterpret_cast<float *>(ws + lay.lse_a), *lse_b = reinterpret_cast<float *>(ws + lay.lse_b);
+    float *part_a = reinterpret_cast<float *>(ws + lay.part_a), *part_b = reinterpret_cast<float *>(ws + lay.part_b);
+
+    // items that a broken indptr leaves out of every group still get a defined offset
+    cudaError_t e = cudaMemsetAsync(ws + lay.group_traj, 0, lay.lse_a - lay.group_traj, stream);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "group_decode_attn memset");
+    AttnCall base = make_call(ctx, pool, trajs, traj_ids, nullptr, n_items, n_items, max_seq_len, q, num_q_heads, sm_scale,
+                              out, lse);
+    e = launch_group_prepare(base.trajs, traj_ids, n_items, group_indptr, shared_lens, n_groups, pool->page_size, group_traj,
+                             item_off, ctx->d_status, stream, &ctx->launches);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "group_decode_attn prepare launch");
+
+    bool too_small = false;
+    // shared prefix: the members' query rows of one group form the rows of an M-tile; every row sees the whole prefix
+    AttnCall sc = base;
+    sc.traj_ids = group_traj;
+    sc.q_indptr = group_indptr;
+    sc.n_items = n_groups;
+    sc.shared_lens = shared_lens;
+    sc.out_f32 = part_a;
+    sc.lse = lse_a;
+    e = launch_chunk_attn(sc, stream, &ctx->launches, &too_small);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "group_decode_attn shared-prefix launch");
+    // private remainder: the decode kernel over each member's pages after the prefix
+    AttnCall pc = base;
+    pc.page_offset = item_off;
+    pc.out_f32 = part_b;
+    pc.lse = lse_b;
+    e = launch_decode_attn(pc, stream, &ctx->launches, &too_small);
+    if (too_small) return fail(ctx, ROLLART_ERR_WORKSPACE, "workspace of %zu bytes is too small", ctx->workspace_bytes);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "group_decode_attn decode launch");
+    e = launch_group_merge(part_a, lse_a, part_b, lse_b, static_cast<long long>(n_items) * num_q_heads,
+                           static_cast<__nv_bfloat16 *>(out), lse, stream, &ctx->launches);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "group_decode_attn merge launch");
+    return ROLLART_OK;
+}
+
 rollart_status rollart_obs_chunk_attn(rollart_ctx *ctx, const rollart_kv_pool *pool, const rollart_trajs *trajs,
                                       const int32_t *traj_ids, const int32_t *q_indptr, int32_t n_items,
                                       int32_t total_q, int32_t max_seq_len, const void *q, int32_t num_q_heads,
@@ -355,8 +442,9 @@ rollart_status rollart_check(rollart_ctx *ctx, void *stream) {
     if (hs.code == 0) return ROLLART_OK;
     decode_reset_workspace(ctx->workspace, ctx->workspace_bytes, s);
     cudaStreamSynchronize(s);
-    static const char *const where[] = {"?", "kv_append", "decode_attn", "obs_chunk_attn", "combine", "kv_gather", "pages"};
-    const char *w = (hs.where >= 0 && hs.where < 7) ? where[hs.where] : "?";
+    static const char *const where[] = {"?", "kv_append", "decode_attn", "obs_chunk_attn", "combine", "kv_gather", "pages",
+                                        "group_decode"};
+    const char *w = (hs.where >= 0 && hs.where < 8) ? where[hs.where] : "?";
     if (hs.code == ROLLART_ERR_TIMEOUT)
         return fail(ctx, ROLLART_ERR_TIMEOUT, "%s: a bounded wait ran out (detail %d)", w, hs.detail);
     return fail(ctx, static_cast<rollart_status>(hs.code), "%s: index out of range on the device (detail %d)", w, hs.detail);

@@ -87,6 +87,10 @@ struct AttnCall {
     const __nv_bfloat16 *k_new;
     const __nv_bfloat16 *v_new;
     int32_t *seq_lens_out;
+    // group decode (all NULL otherwise)
+    const int32_t *page_offset;   // decode: per item, pages of the table row to skip (the keys before them are not attended to)
+    const int32_t *shared_lens;   // chunk: per item, every query row of the item sees exactly the first shared_lens[i] keys
+    float *out_f32;               // when set the result rows are written here in fp32 instead of bf16 to `out`
 };
 
 size_t decode_workspace_bytes(int max_items, int num_q_heads, int num_kv_heads, int max_seq_len, int sm_count);
@@ -95,5 +99,14 @@ cudaError_t launch_decode_attn(const AttnCall &c, cudaStream_t stream, int64_t *
 // zeroes the bookkeeping at the head of the workspace after a device-side error
 cudaError_t decode_reset_workspace(void *workspace, size_t bytes, cudaStream_t stream);
 cudaError_t launch_chunk_attn(const AttnCall &c, cudaStream_t stream, int64_t *launches, bool *too_small);
+
+// Group decode helpers.  `prepare` derives, per group, the trajectory whose table row stands for the shared
+// prefix and, per item, the pages to skip; it also checks that the members alias the same pages there.
+cudaError_t launch_group_prepare(const TrajView &trajs, const int32_t *traj_ids, int n_items, const int32_t *group_indptr,
+                                 const int32_t *shared_lens, int n_groups, int page_size, int32_t *group_traj,
+                                 int32_t *item_page_offset, DeviceStatus *status, cudaStream_t stream, int64_t *launches);
+// out = softmax-weighted sum of the two partial results (weights from their log-sum-exps); lse optional
+cudaError_t launch_group_merge(const float *part_a, const float *lse_a, const float *part_b, const float *lse_b,
+                               long long rows, __nv_bfloat16 *out, float *lse, cudaStream_t stream, int64_t *launches);
 
 }  // namespace rollart

@@ -22,7 +22,7 @@ EXPORTS = (
     "rollart_workspace_size", "rollart_create", "rollart_destroy", "rollart_kv_append", "rollart_decode_attn",
     "rollart_obs_chunk_attn", "rollart_check", "rollart_last_error", "rollart_launch_count",
     "rollart_decode_attn_noalloc", "rollart_kv_gather", "rollart_pages_reserve", "rollart_pages_release",
-    "rollart_append_decode_attn",
+    "rollart_append_decode_attn", "rollart_group_decode_attn", "rollart_group_decode_workspace_size",
 )
 
 
@@ -75,6 +75,11 @@ def load_library() -> ctypes.CDLL:
     L.rollart_append_decode_attn.restype = ctypes.c_int
     L.rollart_append_decode_attn.argtypes = [vp, ctypes.POINTER(_KVPool), ctypes.POINTER(_Trajs), vp, i32, i32, vp, vp, vp, i32,
                                              f32, vp, vp, vp, vp]
+    L.rollart_group_decode_workspace_size.restype = ctypes.c_size_t
+    L.rollart_group_decode_workspace_size.argtypes = [i32, i32, i32, i32]
+    L.rollart_group_decode_attn.restype = ctypes.c_int
+    L.rollart_group_decode_attn.argtypes = [vp, ctypes.POINTER(_KVPool), ctypes.POINTER(_Trajs), vp, i32, vp, vp, i32, i32,
+                                            vp, i32, f32, vp, vp, vp]
     L.rollart_obs_chunk_attn.restype = ctypes.c_int
     L.rollart_obs_chunk_attn.argtypes = [vp, ctypes.POINTER(_KVPool), ctypes.POINTER(_Trajs), vp, vp, i32, i32, i32, vp,
                                          i32, f32, vp, vp, vp]
@@ -93,6 +98,10 @@ def load_library() -> ctypes.CDLL:
 
 def workspace_size(max_items: int, num_q_heads: int, num_kv_heads: int, max_seq_len: int) -> int:
     return int(load_library().rollart_workspace_size(max_items, num_q_heads, num_kv_heads, max_seq_len))
+
+
+def group_decode_workspace_size(max_items: int, num_q_heads: int, num_kv_heads: int, max_seq_len: int) -> int:
+    return int(load_library().rollart_group_decode_workspace_size(max_items, num_q_heads, num_kv_heads, max_seq_len))
 
 
 def _ptr(t: Optional[torch.Tensor], dtype=None, device=None) -> Optional[int]:
@@ -282,6 +291,28 @@ class Context:
             int(max_seq_len), _ptr(k_new, torch.bfloat16, self.device), _ptr(v_new, torch.bfloat16, self.device),
             _ptr(q, torch.bfloat16, self.device), hq, float(sm_scale), _ptr(out, torch.bfloat16, self.device),
             _ptr(lse, torch.float32, self.device), _ptr(seq_lens_out, torch.int32, self.device), self._stream(stream))
+        if st != OK:
+            self._raise(st)
+
+    def group_decode_attn(self, k_pool, v_pool, page_table, seq_lens, group_indptr, shared_lens, q, sm_scale, max_seq_len,
+                          out, lse=None, traj_ids=None, stream=None) -> None:
+        pool = self._pool(k_pool, v_pool)
+        trajs = self._trajs(page_table, seq_lens)
+        if q.dim() != 3 or q.shape != out.shape:
+            raise ValueError("q and out must be [n_items][num_q_heads][head_dim]")
+        n_items, hq, _ = q.shape
+        n_groups = group_indptr.shape[0] - 1
+        if shared_lens.shape[0] != n_groups:
+            raise ValueError("shared_lens must have one entry per group")
+        if traj_ids is not None and traj_ids.shape[0] != n_items:
+            raise ValueError("traj_ids must have one entry per item")
+        if lse is not None and tuple(lse.shape) != (n_items, hq):
+            raise ValueError("lse must be [n_items][num_q_heads]")
+        st = self._lib.rollart_group_decode_attn(
+            self._h, ctypes.byref(pool), ctypes.byref(trajs), _ptr(traj_ids, torch.int32, self.device), n_items,
+            _ptr(group_indptr, torch.int32, self.device), _ptr(shared_lens, torch.int32, self.device), n_groups,
+            int(max_seq_len), _ptr(q, torch.bfloat16, self.device), hq, float(sm_scale),
+            _ptr(out, torch.bfloat16, self.device), _ptr(lse, torch.float32, self.device), self._stream(stream))
         if st != OK:
             self._raise(st)
 

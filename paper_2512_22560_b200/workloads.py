@@ -75,6 +75,15 @@ CONFIGS = (
 RECOMPUTE = WorkloadSpec("recompute_inflight", 16, 32, 8, 16, "uniform", len_lo=4096, len_hi=32768, recompute=True)
 
 
+# Decode step of GRPO groups under prefix caching (Sec. 7.1: group size 8, prefix caching on the rollout
+# engine): 64 groups of 8 trajectories with the 7B-like head shape; share_group_prefix() makes the
+# members of a group alias the pages of a common prompt prefix.
+GROUP_DECODE = WorkloadSpec("grpo_group8_decode", 512, 28, 4, 16, "turns", len_cap=16384,
+                            k_scale=1.0 / math.sqrt(HEAD_DIM), sm_scale=1.0)
+GROUP_SIZE = 8
+GROUP_SHARED_FRACTION = 0.5       # of the shortest member's context
+
+
 def shrink(spec: WorkloadSpec, num_traj: int, len_div: int, chunk_div: int = 1) -> WorkloadSpec:
     """A smaller workload of the same shape (same heads, page size, distribution family)."""
     return dataclasses.replace(
@@ -303,6 +312,25 @@ def plant_needles(batch: Batch, positions_per_traj: dict, beta: float = 3.0) -> 
                 row = int(batch.new_indptr[t]) + (pos - int(batch.seq_lens_before[t]))
                 batch.k_new[row] = kvec
             batch.needles.append((t, pos))
+
+
+def share_group_prefix(batch: Batch, group_size: int, fraction: float):
+    """Turns consecutive runs of `group_size` trajectories into groups that share a prompt prefix, the
+    way prefix caching leaves the members of a GRPO group (paper Sec. 7.1: group size 8, prefix caching
+    on): the members' page-table rows are made to list the first member's pages for the first
+    floor(fraction * shortest member length / page_size) pages.  Returns (group_indptr, shared_lens),
+    both int32; shared_lens is in tokens.  Only indices are rewritten: pool contents stay as they are,
+    the pages the other members owned there are simply no longer referenced."""
+    T, P = batch.spec.num_traj, batch.spec.page_size
+    starts = list(range(0, T, group_size)) + [T]
+    indptr = np.asarray(starts, dtype=np.int32)
+    shared = np.zeros(len(starts) - 1, dtype=np.int32)
+    for gi in range(len(starts) - 1):
+        a, b = starts[gi], starts[gi + 1]
+        pages = int(int(batch.seq_lens_before[a:b].min()) * fraction) // P
+        batch.page_table[a + 1:b, :pages] = batch.page_table[a, :pages]
+        shared[gi] = pages * P
+    return indptr, shared
 
 
 def extract_trajs(batch: Batch, ids: Sequence[int]) -> Batch:

@@ -79,3 +79,25 @@ def test_poison_and_needles_change_only_what_they_say():
     out, _ = oracle.decode_attn(kp, vp, b.page_table, after, W.bf16_to_u16(b.q_new), spec.sm_scale)
     assert np.all(np.isfinite(out))
     assert np.abs(out[0]).max() > 0.5
+
+
+def test_share_group_prefix_aliases_whole_pages_only():
+    spec = dataclasses.replace(W.shrink(W.CONFIGS[1], 19, 16), name="groups")
+    b = W.make_layout(spec, seed=3)
+    before = b.page_table.copy()
+    indptr, shared = W.share_group_prefix(b, 8, 0.7)
+    assert indptr.tolist() == [0, 8, 16, 19] and shared.dtype == np.int32
+    P = spec.page_size
+    for gi in range(3):
+        a, e = int(indptr[gi]), int(indptr[gi + 1])
+        s = int(shared[gi])
+        assert s % P == 0 and s <= int(b.seq_lens_before[a:e].min())
+        assert s == int(int(b.seq_lens_before[a:e].min()) * 0.7) // P * P
+        assert (b.page_table[a:e, :s // P] == before[a, :s // P]).all()          # the first member's pages
+        assert (b.page_table[a:e, s // P:] == before[a:e, s // P:]).all()        # the rest untouched
+    # distinct pages are still distinct outside the shared region: no page is listed by two different groups
+    owned = [set(b.page_table[t, :(int(b.seq_lens_before[t]) + 1 + P - 1) // P].tolist()) for t in range(19)]
+    for t in range(19):
+        for u in range(t + 1, 19):
+            if np.searchsorted(indptr, t, side="right") != np.searchsorted(indptr, u, side="right"):
+                assert not (owned[t] & owned[u])
