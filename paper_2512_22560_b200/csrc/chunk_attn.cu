@@ -1,26 +1,34 @@
 // Observation-chunk attention on the 5th-generation tensor cores (tcgen05 + TMEM).
 //
-// Work unit: (item, kv head, M-tile).  An M-tile is 128 query rows = floor(128 / g) consecutive
-// chunk tokens x the g query heads that share the kv head, so one K/V read serves all of them.
-// The unit walks the visible keys (the whole cached prefix, then the chunk itself up to the
-// diagonal) in tiles of 64 keys:
+// Work unit: (item, kv head, pair of M-tiles).  An M-tile is 128 query rows = floor(128 / g)
+// consecutive chunk tokens x the g query heads that share the kv head, so one K/V read serves all
+// of them; a block owns two consecutive M-tiles (256 rows share every K/V tile it brings in) and
+// walks the visible keys (the whole cached prefix, then the chunk itself up to the diagonal) in
+// tiles of 64 keys.  Per M-tile t and key tile j:
 //
-//   S = Q K^T      tcgen05.mma, M 128 x N 64 x K 128, operands in 128B-swizzled shared memory
-//                  (Q and K tiles brought by TMA), fp32 accumulator in TMEM, double buffered
-//   softmax        one thread per query row (4 warps = 128 TMEM lanes): tcgen05.ld its 64 scores,
-//                  scale, causal/length mask, running max m and sum l, P = exp2(s - m) as packed
-//                  bf16 stored back with tcgen05.st over the first 32 columns of the same S
-//                  buffer; the O accumulator in TMEM is rescaled only when a row's max has grown
-//                  by more than 2^8, so the softmax warps normally never wait for an MMA
-//   O += P V       tcgen05.mma with the A operand (P) in TMEM, M 128 x N 128 x K 64; V is the
-//                  MN-major B operand straight from its [key][dim] page layout
+//   S_t = Q_t K^T    tcgen05.mma, M 128 x N 64 x K 128, operands in 128B-swizzled shared memory
+//                    (Q and K tiles brought by TMA), fp32 accumulator in TMEM, two S buffers per
+//                    M-tile so that S(j+1) is computed while the softmax of tile j runs
+//   softmax          one warpgroup per M-tile, one thread per query row: tcgen05.ld its 64 scores,
+//                    P = exp2(scale * s - m) as packed bf16 stored back with tcgen05.st over the
+//                    first 32 columns of the same S buffer, row sum l.  After the first tile m is
+//                    not recomputed per tile: the exponentials are taken against the row's current
+//                    reference max, and only a row sum that explodes (or a masked tile) sends the
+//                    tile down the careful path (row max, new reference, O rescaled in TMEM).  One
+//                    pair of exponentials in four is evaluated on the FMA pipe (range reduction +
+//                    cubic) to take load off the special-function unit.
+//   O_t += P_t V     tcgen05.mma with the A operand (P) in TMEM, M 128 x N 128 x K 64; V is the
+//                    MN-major B operand straight from its [key][dim] page layout
 //
-// One warp issues the copies, one warp issues the MMAs, four warps do softmax and the epilogue.
-// A block uses 97 KB of shared memory and 256 TMEM columns, so two blocks share an SM and one
-// block's softmax overlaps the other's MMAs.  Blocks are ordered (item, kv head, M-tile), so the
-// M-tiles that re-read one (item, head)'s keys run together and find them in L2.
-// Every wait is a bounded mbarrier poll; no block waits for another block.
+// Warp roles: warp 0 issues the copies (page ids fetched 32 at a time, a batch ahead), warps 1 and
+// 2 each issue the MMAs of one M-tile, warps 4-7 and 8-11 are the two softmax warpgroups, which also
+// write the result.  A block uses ~194 KB of shared memory (Q 64 KB, 8 K/V stages of 16 KB) and all
+// 512 TMEM columns (2 x 2 S buffers of 64, 2 O accumulators of 128): one block per SM.
+// Blocks are ordered (item, kv head, pair), so the blocks that re-read one (item, head)'s keys run
+// together and find them in L2.  Every wait is a bounded mbarrier poll; no block waits for another.
 #include <cuda.h>
+
+#include <type_traits>
 
 #include "rollart_internal.cuh"
 
@@ -28,32 +36,36 @@ namespace rollart {
 
 namespace {
 
+
 constexpr int kRows = 128;                 // query rows of an M-tile (UMMA M)
 constexpr int kKeys = 64;                  // keys per KV tile
-constexpr int kStages = 2;
-constexpr int kThreads = 192;              // warp 0 copies, warp 1 MMA, warps 2-5 softmax
+constexpr int kStages = 8;                 // ring of KV tiles; K(j) and V(j) take alternate slots
+constexpr int kThreads = 384;              // warp 0 copies, warps 1-2 MMA of M-tile 0 / 1, warps 4-7 / 8-11 softmax of M-tile 0 / 1
 constexpr int kMaxItems = 1024;            // items per launch (tile prefix lives in shared memory)
-constexpr uint32_t kSpinLimit = 1u << 17;   // polls per wait; each poll sleeps in hardware for up to kSuspendNs
-constexpr uint32_t kSuspendNs = 10000;
+constexpr long long kWaitCycles = 2000000000LL;   // a wait gives up after about a second
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 constexpr float kRescaleThreshold = 8.f;   // log2 units
+constexpr float kRowSumLimit = 16777216.f; // 2^24: a tile's row sum above this sends the tile down the careful path
+constexpr int kPolyOneIn = 4;              // one pair of exponentials in this many goes to the FMA pipe
 
 constexpr int kHalfQ = kRows * 128;        // 16 KB: 128 rows x 64 dims
+constexpr int kTileQ = 2 * kHalfQ;
 constexpr int kHalfKV = kKeys * 128;       // 8 KB: 64 keys x 64 dims
-constexpr int kOffQ = 0;                                   // [half][row][128 B]
-constexpr int kOffK = kOffQ + 2 * kHalfQ;                  // stages x [half][key][128 B]
-constexpr int kOffV = kOffK + kStages * 2 * kHalfKV;
-constexpr int kOffBars = kOffV + kStages * 2 * kHalfKV;
-constexpr int kNumBars = 1 + 4 * kStages + 2 + 2 + 2;      // q | k,v full/empty | s_full x2 | p_full x2 | o_done x2
+constexpr int kTileKV = 2 * kHalfKV;
+constexpr int kOffQ = 0;                                   // [M-tile][half][row][128 B]
+constexpr int kOffKV = kOffQ + 2 * kTileQ;                 // stages x [half][key][128 B]
+constexpr int kOffBars = kOffKV + kStages * kTileKV;
+constexpr int kNumBars = 1 + 2 * kStages + 4 + 4 + 4;      // q | kv full/empty | per M-tile and S buffer: s_full, p_full, o_done
 constexpr int kOffTmemSlot = kOffBars + kNumBars * 8;
 constexpr int kOffAbort = kOffTmemSlot + 8;
 constexpr int kSmemUsed = kOffAbort + 8;
-constexpr int kSmemBytes = kSmemUsed + 1024;               // + slack for the 1024-byte alignment; two blocks fit an SM
-static_assert(2 * (kSmemBytes + 1024) <= 228 * 1024, "two blocks per SM");
-static_assert((kMaxItems + 1) * 4 <= kStages * 2 * kHalfKV, "the tile prefix is staged in the K stages");
+constexpr int kSmemBytes = kSmemUsed + 1024;               // + slack for the 1024-byte alignment
+static_assert(kSmemBytes <= 227 * 1024, "one block must fit an SM");
+static_assert((kMaxItems + 1) * 4 <= kStages * kTileKV, "the tile prefix is staged in the KV stages");
 
-constexpr int kTmemCols = 256;             // S0 [0,64) S1 [64,128) O [128,256); P overwrites the first 32 columns of its S
+constexpr int kTmemCols = 512;             // S buffer b of M-tile t at (2t + b) * 64; O_t at 256 + 128 t; P overwrites the first 32 columns of its S buffer
+constexpr int kTmemO = 256;
 
 struct ChunkParams {
     const int32_t *page_table;
@@ -88,18 +100,24 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity), "r"(kSuspendNs) : "memory");
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
-// Bounded wait; once any thread of the block has given up, nobody waits any more, so every role
-// runs its (bounded) loops to the end and the block exits with the error recorded.
+// Bounded wait.  The poll has no sleep in it: a sleeping poll wakes up to a microsecond late, and every hand-over
+// between the tensor core and the softmax warps would pay that.  Once any thread of the block has given up, nobody
+// waits any more, so every role runs its (bounded) loops to the end and the block exits with the error recorded.
 __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, DeviceStatus *status,
                                           int where) {
-    for (uint32_t it = 0; it < kSpinLimit; ++it) {
+    if (mbar_try_wait(bar, parity)) return;
+    const long long t0 = clock64();
+    for (uint32_t it = 1;; ++it) {
         if (mbar_try_wait(bar, parity)) return;
-        if (*abort_flag) return;
+        if ((it & 255u) == 0u) {
+            if (*abort_flag) return;
+            if (clock64() - t0 > kWaitCycles) break;
+        }
     }
     if (*abort_flag == 0) {
         *abort_flag = 1;
@@ -158,14 +176,18 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
           "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
         : "r"(taddr) : "memory");
 }
-__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
     asm volatile(
-        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
-        "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]),
+          "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
         ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
-          "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]),
-          "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]),
-          "r"(r[30]), "r"(r[31])
+          "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
         : "memory");
 }
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
@@ -198,6 +220,29 @@ __device__ __forceinline__ void add2(float &d0, float &d1, float a0, float a1) {
         "add.rn.f32x2 rd, rd, ra;\n\tmov.b64 {%0, %1}, rd;\n\t}"
         : "+f"(d0), "+f"(d1) : "f"(a0), "f"(a1));
 }
+__device__ __forceinline__ void fma2v(float &d0, float &d1, float a0, float a1, float b0, float b1, float c0, float c1) {   // d = a * b + c
+    asm("{\n\t.reg .b64 ra, rb, rc, rd;\n\t"
+        "mov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\tmov.b64 rc, {%6, %7};\n\t"
+        "fma.rn.f32x2 rd, ra, rb, rc;\n\tmov.b64 {%0, %1}, rd;\n\t}"
+        : "=f"(d0), "=f"(d1) : "f"(a0), "f"(a1), "f"(b0), "f"(b1), "f"(c0), "f"(c1));
+}
+// 2^x for a pair of arguments x <= 8 on the FMA pipe.  x = n + f with n = round(x), read from the low mantissa bits
+// of x + 1.5 * 2^23; 2^f on [-0.5, 0.5] by a cubic (relative error 7.5e-5, far below the bf16 rounding of P); n is
+// then added to the exponent field.  Arguments below -126 give 2^-126.
+__device__ __forceinline__ void ex2_poly2(float &p0, float &p1, float x0, float x1) {
+    constexpr float kMagic = 12582912.f;
+    x0 = fmaxf(x0, -126.f);
+    x1 = fmaxf(x1, -126.f);
+    float t0, t1, n0, n1, f0, f1, q0, q1;
+    fma2v(t0, t1, x0, x1, 1.f, 1.f, kMagic, kMagic);
+    fma2v(n0, n1, t0, t1, 1.f, 1.f, -kMagic, -kMagic);
+    fma2v(f0, f1, n0, n1, -1.f, -1.f, x0, x1);
+    fma2v(q0, q1, f0, f1, 0.0551716685f, 0.0551716685f, 0.2426111251f, 0.2426111251f);
+    fma2v(q0, q1, q0, q1, f0, f1, 0.6932609677f, 0.6932609677f);
+    fma2v(q0, q1, q0, q1, f0, f1, 0.9999280572f, 0.9999280572f);
+    p0 = __uint_as_float(__float_as_uint(q0) + (__float_as_uint(t0) << 23));
+    p1 = __uint_as_float(__float_as_uint(q1) + (__float_as_uint(t1) << 23));
+}
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t *>(&v);
@@ -219,7 +264,7 @@ constexpr uint32_t idesc(int n, bool b_mn_major) {
 // ------------------------------------------------------------------------------------------
 // Kernel
 // ------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(kThreads, 2)
+__global__ void __launch_bounds__(kThreads, 1)
 chunk_attn_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant__ CUtensorMap kmap,
                   const __grid_constant__ CUtensorMap vmap, const ChunkParams prm) {
     extern __shared__ uint8_t smem_raw[];
@@ -229,7 +274,7 @@ chunk_attn_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constan
     const int tpt = kRows / g;                       // chunk tokens per M-tile
     volatile int *s_abort = reinterpret_cast<volatile int *>(smem + kOffAbort);
     volatile uint32_t *s_tmem = reinterpret_cast<volatile uint32_t *>(smem + kOffTmemSlot);
-    int *s_prefix = reinterpret_cast<int *>(smem + kOffK);     // staged in the K stages during the prologue
+    int *s_prefix = reinterpret_cast<int *>(smem + kOffKV);    // staged in the KV stages during the prologue
 
     if (static_cast<int>(smem - smem_raw) + kSmemUsed > kSmemBytes) {   // cannot happen: the slack covers any alignment
         if (threadIdx.x == 0) report(prm.status, ROLLART_ERR_CUDA, static_cast<int>(smem - smem_raw), 3);
@@ -237,33 +282,31 @@ chunk_attn_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constan
     }
     const uint32_t bars = smem_u32(smem + kOffBars);
     const uint32_t bar_q = bars;
-    auto bar_kfull = [&](int s) { return bars + 8u * (1 + s); };
-    auto bar_kempty = [&](int s) { return bars + 8u * (1 + kStages + s); };
-    auto bar_vfull = [&](int s) { return bars + 8u * (1 + 2 * kStages + s); };
-    auto bar_vempty = [&](int s) { return bars + 8u * (1 + 3 * kStages + s); };
-    auto bar_sfull = [&](int s) { return bars + 8u * (1 + 4 * kStages + s); };
-    // tile i uses p_full(i & 1) and o_done(i & 1): a warp that is a tile ahead of the others arrives on the other barrier
-    auto bar_pfull = [&](int s) { return bars + 8u * (1 + 4 * kStages + 2 + s); };
-    auto bar_odone = [&](int s) { return bars + 8u * (1 + 4 * kStages + 4 + s); };
+    // ring slot r (K(j) is r = 2j, V(j) is r = 2j + 1) lives in stage r % kStages
+    auto bar_full = [&](int s) { return bars + 8u * (1 + s); };
+    auto bar_empty = [&](int s) { return bars + 8u * (1 + kStages + s); };
+    // key tile j of M-tile t uses S buffer b = j & 1 and the barriers of (t, b): a warp that is a tile ahead of the
+    // others of its warpgroup arrives on the other barrier
+    auto bar_sfull = [&](int t, int b) { return bars + 8u * (1 + 2 * kStages + 2 * t + b); };
+    auto bar_pfull = [&](int t, int b) { return bars + 8u * (1 + 2 * kStages + 4 + 2 * t + b); };
+    auto bar_odone = [&](int t, int b) { return bars + 8u * (1 + 2 * kStages + 8 + 2 * t + b); };
 
-    // ---- which (item, kv head, M-tile) is this block?  tiles per item -> prefix -> search ----
+    // ---- which (item, kv head, pair of M-tiles) is this block?  pairs per item -> prefix -> search ----
     for (int i = threadIdx.x; i < prm.n_items; i += kThreads) {
         const int n = __ldg(prm.q_indptr + i + 1) - __ldg(prm.q_indptr + i);
-        s_prefix[i + 1] = n > 0 ? (n + tpt - 1) / tpt : 0;
+        s_prefix[i + 1] = n > 0 ? (n + 2 * tpt - 1) / (2 * tpt) : 0;
     }
     if (threadIdx.x == 0) {
         s_prefix[0] = 0;
         mbar_init(bar_q, 1);
-        for (int s = 0; s < kStages; ++s) {
-            mbar_init(bar_kfull(s), 1); mbar_init(bar_kempty(s), 1);
-            mbar_init(bar_vfull(s), 1); mbar_init(bar_vempty(s), 1);
-        }
-        for (int s = 0; s < 2; ++s) { mbar_init(bar_sfull(s), 1); mbar_init(bar_odone(s), 1); mbar_init(bar_pfull(s), 4); }
+        for (int s = 0; s < kStages; ++s) mbar_init(bar_full(s), 1);      // the empty barriers count the live M-tiles: set up below
+        for (int t = 0; t < 2; ++t)
+            for (int b = 0; b < 2; ++b) { mbar_init(bar_sfull(t, b), 1); mbar_init(bar_odone(t, b), 1); mbar_init(bar_pfull(t, b), 4); }
         *s_abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
-    if (warp == 0) {        // inclusive scan of the tile counts, in place
+    if (warp == 0) {        // inclusive scan of the pair counts, in place
         const int per = (prm.n_items + 31) / 32;
         const int a = min(prm.n_items, lane * per), b = min(prm.n_items, a + per);
         int sum = 0;
@@ -280,7 +323,7 @@ chunk_attn_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constan
     __syncthreads();
     const int unit = blockIdx.x;
     const int total_units = s_prefix[prm.n_items] * hkv;
-    int item = 0, head = 0, mtile = 0;
+    int item = 0, head = 0, pair = 0;
     if (unit < total_units) {
         int lo = 0, hi = prm.n_items;
         while (hi - lo > 1) {
@@ -288,12 +331,12 @@ chunk_attn_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constan
             if (s_prefix[mid] * hkv <= unit) lo = mid; else hi = mid;
         }
         item = lo;
-        const int nt = max(1, s_prefix[lo + 1] - s_prefix[lo]);
+        const int np = max(1, s_prefix[lo + 1] - s_prefix[lo]);
         const int rem = unit - s_prefix[lo] * hkv;
-        head = rem / nt;
-        mtile = nt - 1 - (rem - head * nt);     // later M-tiles see more keys: start the longest ones first
+        head = rem / np;
+        pair = np - 1 - (rem - head * np);      // later M-tiles see more keys: start the longest ones first
     }
-    __syncthreads();                 // everyone has read the prefix: the K stages are free again
+    __syncthreads();                 // everyone has read the prefix: the KV stages are free again
     if (unit >= total_units) return;
     if (*reinterpret_cast<volatile int *>(&prm.status->fatal) != 0) return;   // an earlier block ran out of patience: give up quickly
 
@@ -327,14 +370,22 @@ chunk_attn_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constan
     }
     if (bad) return;                 // uniform over the block, before any barrier or TMEM use
     const int prior = L - n_chunk;
-    const int tok0 = mtile * tpt;                              // first chunk token of this M-tile
-    const int toks = min(tpt, n_chunk - tok0);                 // live tokens
-    const int max_count = shared_mode ? L : prior + tok0 + toks;   // keys visible to the last live row
-    const int min_count = shared_mode ? L : prior + tok0 + 1;      // keys visible to the first row
-    const int n_tiles = (max_count + kKeys - 1) / kKeys;
+    const int tok0 = pair * 2 * tpt;                            // first chunk token of M-tile 0
+    // per M-tile: live tokens, keys visible to its last live row / first row, key tiles (M-tile 1 may be absent)
+    int toks_[2], maxc_[2], minc_[2], nt_[2];
+#pragma unroll
+    for (int mt = 0; mt < 2; ++mt) {
+        const int first = tok0 + mt * tpt;
+        toks_[mt] = max(0, min(tpt, n_chunk - first));
+        maxc_[mt] = toks_[mt] == 0 ? 0 : (shared_mode ? L : prior + first + toks_[mt]);
+        minc_[mt] = shared_mode ? L : prior + first + 1;
+        nt_[mt] = (maxc_[mt] + kKeys - 1) / kKeys;
+    }
+    const int n0 = nt_[0], n1 = nt_[1], nmax = max(n0, n1);
     const int32_t *table_row = prm.page_table + static_cast<long long>(t) * prm.max_pages;
-    if (n_tiles == 0) {
+    if (nmax == 0) {
         // only in shared-prefix mode with an empty prefix: the result is out = 0, lse = -inf
+        const int toks = toks_[0] + toks_[1];
         for (int idx = threadIdx.x; idx < toks * g * (kHeadDim / 4); idx += kThreads) {
             const int r = idx / (kHeadDim / 4), c = idx - r * (kHeadDim / 4);
             const int tk = r / g, hd = r - tk * g;
@@ -346,9 +397,13 @@ chunk_attn_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constan
         return;                      // uniform over the block, before any barrier or TMEM use
     }
 
-    // zero the Q tile (rows beyond tpt * g are never written by the copy) and allocate TMEM
-    for (int i = threadIdx.x; i < 2 * kHalfQ / 16; i += kThreads) reinterpret_cast<uint4 *>(smem + kOffQ)[i] = make_uint4(0, 0, 0, 0);
+    // zero the Q tiles (rows beyond tpt * g are never written by the copy) and allocate TMEM
+    for (int i = threadIdx.x; i < 2 * kTileQ / 16; i += kThreads) reinterpret_cast<uint4 *>(smem + kOffQ)[i] = make_uint4(0, 0, 0, 0);
     fence_proxy_async();
+    if (threadIdx.x == 32) {
+        for (int s = 0; s < kStages; ++s) mbar_init(bar_empty(s), n1 > 0 ? 2 : 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
     if (warp == 0) tmem_alloc(smem_u32(smem + kOffTmemSlot), kTmemCols);
     tc_fence_before();
     __syncthreads();
@@ -358,233 +413,298 @@ chunk_attn_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constan
     if (warp == 0) {
         // =============================== copy warp ===============================
         if (lane == 0) {
-            mbar_arrive_expect_tx(bar_q, static_cast<uint32_t>(tpt * g) * kRowBytes);
-            tma_load_3d(smem_u32(smem + kOffQ), &qmap, bar_q, 0, head * g, q_row0 + tok0);
-            tma_load_3d(smem_u32(smem + kOffQ + kHalfQ), &qmap, bar_q, 64, head * g, q_row0 + tok0);
+            const int live_tiles = n1 > 0 ? 2 : 1;
+            mbar_arrive_expect_tx(bar_q, static_cast<uint32_t>(live_tiles * tpt * g) * kRowBytes);
+            for (int mt = 0; mt < live_tiles; ++mt) {
+                const uint32_t dst = smem_u32(smem + kOffQ + mt * kTileQ);
+                tma_load_3d(dst, &qmap, bar_q, 0, head * g, q_row0 + tok0 + mt * tpt);
+                tma_load_3d(dst + kHalfQ, &qmap, bar_q, 64, head * g, q_row0 + tok0 + mt * tpt);
+            }
         }
         const int pages_per_tile = kKeys / P;
+        const int tiles_per_batch = 32 / pages_per_tile;
         const uint32_t half_page = static_cast<uint32_t>(P) * 128;
-        for (int j = 0; j < n_tiles; ++j) {
-            const int stage = j % kStages;
-            const uint32_t par = ((j / kStages) & 1) ^ 1;
-            const int lp = j * pages_per_tile + lane;
+        // Page ids are fetched 32 at a time, one per lane (enough for 8 to 32 key tiles), and the next 32 are
+        // requested a whole batch ahead, so the table lookup (a dependent load) is off the copy loop's path.
+        auto load_ids = [&](int batch) {
+            const int lp = batch * 32 + lane;
             int pg = -1;
-            if (lane < pages_per_tile && lp * P < L) {
+            if (lp * P < L && lp < prm.max_pages) {
                 pg = __ldg(table_row + lp);
                 if (pg < 0 || pg >= prm.num_pages) { report(prm.status, ROLLART_ERR_BOUNDS, pg, 3); pg = -1; }
             }
+            return pg;
+        };
+        int ids_cur = load_ids(0), ids_next = load_ids(1);
+        for (int j = 0; j < nmax; ++j) {
+            if (*s_abort) break;
+            const int within = j % tiles_per_batch;
+            if (j > 0 && within == 0) { ids_cur = ids_next; ids_next = load_ids(j / tiles_per_batch + 1); }
+            int pg = __shfl_sync(0xffffffffu, ids_cur, (within * pages_per_tile + lane) & 31);
+            if (lane >= pages_per_tile) pg = -1;
             const uint32_t nvalid = __popc(__ballot_sync(0xffffffffu, pg >= 0));
             const int row = (pg * hkv + head) * P;
-            // K
-            mbar_wait(bar_kempty(stage), par, s_abort, prm.status, 1);
-            if (!*s_abort) {
-                if (lane == 0) mbar_arrive_expect_tx(bar_kfull(stage), nvalid * 2u * half_page);
+#pragma unroll
+            for (int kv = 0; kv < 2; ++kv) {           // K(j) then V(j)
+                const int r = 2 * j + kv, stage = r % kStages;
+                const uint32_t par = ((r / kStages) & 1) ^ 1;
+                mbar_wait(bar_empty(stage), par, s_abort, prm.status, 1 + kv);
+                if (lane == 0) mbar_arrive_expect_tx(bar_full(stage), nvalid * 2u * half_page);
                 __syncwarp();
                 if (pg >= 0) {
-                    const uint32_t dst = smem_u32(smem + kOffK + stage * 2 * kHalfKV) + lane * half_page;
-                    tma_load_2d(dst, &kmap, bar_kfull(stage), 0, row);
-                    tma_load_2d(dst + kHalfKV, &kmap, bar_kfull(stage), 64, row);
-                }
-            }
-            // V
-            mbar_wait(bar_vempty(stage), par, s_abort, prm.status, 2);
-            if (!*s_abort) {
-                if (lane == 0) mbar_arrive_expect_tx(bar_vfull(stage), nvalid * 2u * half_page);
-                __syncwarp();
-                if (pg >= 0) {
-                    const uint32_t dst = smem_u32(smem + kOffV + stage * 2 * kHalfKV) + lane * half_page;
-                    tma_load_2d(dst, &vmap, bar_vfull(stage), 0, row);
-                    tma_load_2d(dst + kHalfKV, &vmap, bar_vfull(stage), 64, row);
+                    const uint32_t dst = smem_u32(smem + kOffKV + stage * kTileKV) + lane * half_page;
+                    const CUtensorMap *map = kv == 0 ? &kmap : &vmap;
+                    tma_load_2d(dst, map, bar_full(stage), 0, row);
+                    tma_load_2d(dst + kHalfKV, map, bar_full(stage), 64, row);
                 }
             }
         }
-    } else if (warp == 1) {
-        // =============================== MMA warp ===============================
-        constexpr uint32_t kIdescQK = idesc(kKeys, false);
-        constexpr uint32_t kIdescPV = idesc(kHeadDim, true);
-        const uint32_t q_addr = smem_u32(smem + kOffQ);
-        auto issue_pv = [&](int i) {
-            const int stage = i % kStages;
-            mbar_wait(bar_vfull(stage), (i / kStages) & 1, s_abort, prm.status, 3);
-            mbar_wait(bar_pfull(i & 1), (i >> 1) & 1, s_abort, prm.status, 4);
-            tc_fence_after();
-            if (lane == 0 && !*s_abort) {
-                const uint32_t v_addr = smem_u32(smem + kOffV + stage * 2 * kHalfKV);
-#pragma unroll
-                for (int ks = 0; ks < kKeys / 16; ++ks)   // 16 keys per step: 8 packed columns along P's row, 2048 B down V
-                    umma_bf16_ts(tmem + 128, tmem + (i & 1) * kKeys + ks * 8, smem_desc(v_addr + ks * 2048, kHalfKV), kIdescPV,
-                                 (i > 0 || ks > 0) ? 1u : 0u);
-                umma_commit(bar_vempty(stage));
-                umma_commit(bar_odone(i & 1));
-            }
-            __syncwarp();
-        };
-        mbar_wait(bar_q, 0, s_abort, prm.status, 5);
-        for (int j = 0; j < n_tiles; ++j) {
-            const int stage = j % kStages, sb = j & 1;
-            mbar_wait(bar_kfull(stage), (j / kStages) & 1, s_abort, prm.status, 6);
-            // S buffer sb last held P of tile j-2; PV(j-2) was issued before this QK and MMAs run in issue order
-            tc_fence_after();
-            if (lane == 0 && !*s_abort) {
-                const uint32_t k_addr = smem_u32(smem + kOffK + stage * 2 * kHalfKV);
+    } else if (warp == 1 || warp == 2) {
+        // =============================== MMA warps ===============================
+        // One issuing thread per M-tile: warp 1 runs QK_0 / PV_0, warp 2 runs QK_1 / PV_1.  A thread that issues an
+        // MMA is held until the tensor core accepts it, so everything else that thread does between two MMAs is time
+        // the tensor core may idle; with one thread per M-tile each has half the MMAs and the waits of one M-tile do
+        // not delay the other's products.  Per thread the order is QK(0) | QK(j+1) PV(j) | ...: S of the next key
+        // tile is ready before the softmax of this one ends.  MMAs of one thread run in issue order, which is what
+        // protects the reuse of an S buffer (it holds P(j-1) until PV(j-1), issued before QK(j+1), has read it).
+        // Both threads release every KV stage (its barrier counts the live M-tiles), also for key tiles their own
+        // M-tile does not use.
+        const int mt = warp - 1;
+        const int my_tiles = mt == 0 ? n0 : n1;
+        if (lane == 0 && my_tiles > 0) {
+            constexpr uint32_t kIdescQK = idesc(kKeys, false);
+            constexpr uint32_t kIdescPV = idesc(kHeadDim, true);
+            const uint32_t kv_addr = smem_u32(smem + kOffKV);
+            const uint64_t q_desc = smem_desc(smem_u32(smem + kOffQ) + mt * kTileQ, 16);
+            const uint32_t s_tmem = tmem + mt * 2 * kKeys, o_tmem = tmem + kTmemO + mt * kHeadDim;
+            auto full_wait = [&](int r, int where) {
+                mbar_wait(bar_full(r % kStages), (r / kStages) & 1, s_abort, prm.status, where);
+            };
+            auto issue_qk = [&](int j) {
+                const uint64_t k_desc = smem_desc(kv_addr + ((2 * j) % kStages) * kTileKV, 16);
 #pragma unroll
                 for (int ks = 0; ks < kHeadDim / 16; ++ks) {   // 16 dims per step; the second 64 dims live in the other half
-                    const uint32_t qa = q_addr + (ks >> 2) * kHalfQ + (ks & 3) * 32;
-                    const uint32_t ka = k_addr + (ks >> 2) * kHalfKV + (ks & 3) * 32;
-                    umma_bf16(tmem + sb * kKeys, smem_desc(qa, 16), smem_desc(ka, 16), kIdescQK, ks > 0 ? 1u : 0u);
+                    const uint64_t qoff = static_cast<uint64_t>(((ks >> 2) * kHalfQ + (ks & 3) * 32) >> 4);
+                    const uint64_t koff = static_cast<uint64_t>(((ks >> 2) * kHalfKV + (ks & 3) * 32) >> 4);
+                    umma_bf16(s_tmem + (j & 1) * kKeys, q_desc + qoff, k_desc + koff, kIdescQK, ks > 0 ? 1u : 0u);
                 }
-                umma_commit(bar_kempty(stage));
-                umma_commit(bar_sfull(sb));
+                umma_commit(bar_sfull(mt, j & 1));
+                umma_commit(bar_empty((2 * j) % kStages));
+            };
+            mbar_wait(bar_q, 0, s_abort, prm.status, 5);
+            full_wait(0, 6);
+            tc_fence_after();
+            issue_qk(0);
+            for (int j = 0; j < nmax; ++j) {
+                if (j + 1 < nmax) {
+                    full_wait(2 * j + 2, 6);                // K(j+1)
+                    if (j + 1 < my_tiles) {
+                        tc_fence_after();
+                        issue_qk(j + 1);
+                    } else {
+                        umma_commit(bar_empty((2 * j + 2) % kStages));
+                    }
+                }
+                full_wait(2 * j + 1, 3);                    // V(j)
+                if (j < my_tiles) {
+                    mbar_wait(bar_pfull(mt, j & 1), (j >> 1) & 1, s_abort, prm.status, 4);
+                    tc_fence_after();
+                    const uint64_t v_desc = smem_desc(kv_addr + ((2 * j + 1) % kStages) * kTileKV, kHalfKV);
+                    const uint32_t acc0 = j > 0 ? 1u : 0u;
+#pragma unroll
+                    for (int ks = 0; ks < kKeys / 16; ++ks)     // 16 keys per step: 8 packed columns along P's row, 2048 B down V
+                        umma_bf16_ts(o_tmem, s_tmem + (j & 1) * kKeys + ks * 8, v_desc + static_cast<uint64_t>((ks * 2048) >> 4),
+                                     kIdescPV, ks > 0 ? 1u : acc0);
+                    umma_commit(bar_odone(mt, j & 1));
+                }
+                umma_commit(bar_empty((2 * j + 1) % kStages));   // V(j): this thread's PV(j), if any, has read it
             }
-            __syncwarp();
-            if (j >= 1) issue_pv(j - 1);
         }
-        issue_pv(n_tiles - 1);
-    } else {
-        // =============================== softmax warps ===============================
+        __syncwarp();
+    } else if (warp >= 4) {
+        // =============================== softmax warpgroups ===============================
+        const int mt = (warp - 4) >> 2;                       // M-tile of this warpgroup
+        const int wg_thread = ((warp - 4) & 3) * 32 + lane;
         const int quarter = warp & 3;                         // TMEM lanes 32 * quarter .. + 31 belong to this warp
         const int row = quarter * 32 + lane;
         const uint32_t lane_addr = tmem + (static_cast<uint32_t>(quarter * 32) << 16);
+        const uint32_t s_addr = lane_addr + mt * 2 * kKeys, o_addr = lane_addr + kTmemO + mt * kHeadDim;
+        const int my_tiles = mt == 0 ? n0 : n1;
+        const int toks = mt == 0 ? toks_[0] : toks_[1];
+        const int min_count = mt == 0 ? minc_[0] : minc_[1];
+        const int first_tok = tok0 + mt * tpt;
         const int tok_local = row / g, head_local = row - tok_local * g;
         const bool live = tok_local < toks;
-        const int count = shared_mode ? L : min(L, prior + tok0 + min(tok_local, toks - 1) + 1);   // keys this row sees (>= 1)
+        const int count = shared_mode ? L : min(L, prior + first_tok + min(tok_local, max(toks, 1) - 1) + 1);   // keys this row sees (>= 1)
+        const float scale = prm.scale_log2;
         float m_ref = -INFINITY, l_sum = 0.f;
 
-        for (int j = 0; j < n_tiles; ++j) {
+        for (int j = 0; j < my_tiles; ++j) {
             const int sb = j & 1;
-            mbar_wait(bar_sfull(sb), (j >> 1) & 1, s_abort, prm.status, 8);
+            const uint32_t sbuf = s_addr + sb * kKeys;
+            mbar_wait(bar_sfull(mt, sb), (j >> 1) & 1, s_abort, prm.status, 8);
             tc_fence_after();
             uint32_t sraw[2][32];
-            tmem_ld32(lane_addr + sb * kKeys, sraw[0]);
-            tmem_ld32(lane_addr + sb * kKeys + 32, sraw[1]);
+            tmem_ld32(sbuf, sraw[0]);
+            tmem_ld32(sbuf + 32, sraw[1]);
             tmem_wait_ld();
 
             const int key0 = j * kKeys;
-            const bool need_mask = key0 + kKeys > min_count;    // uniform over the block
-            const float scale = prm.scale_log2;
-            float rmax;
-            if (!need_mask) {
-                // the max of scale * s is scale * (max or min of s): take the extreme of the raw scores, 8 chains of 3-input ops
-                float e[8];
-                if (scale >= 0.f) {
+            const bool need_mask = key0 + kKeys > min_count;    // uniform over the warpgroup
+            const int live_keys = count - key0;                 // keys of this tile the row sees (masked tiles only)
+            float rs[4];
+            // two copies of the pass, chosen once per tile: the unmasked one (every tile but the last few of an
+            // M-tile) carries no compare / select per element
+            auto exp_pass = [&](auto masked_tag, float neg_m) {
+                constexpr bool kMasked = decltype(masked_tag)::value;
+                rs[0] = rs[1] = rs[2] = rs[3] = 0.f;
 #pragma unroll
-                    for (int k = 0; k < 8; ++k) e[k] = max3(__uint_as_float(sraw[0][k]), __uint_as_float(sraw[0][8 + k]), __uint_as_float(sraw[0][16 + k]));
+                for (int h = 0; h < 2; ++h) {
+                    uint32_t packed[16];
 #pragma unroll
-                    for (int k = 0; k < 8; ++k) e[k] = max3(e[k], __uint_as_float(sraw[0][24 + k]), __uint_as_float(sraw[1][k]));
-#pragma unroll
-                    for (int k = 0; k < 8; ++k) e[k] = max3(e[k], __uint_as_float(sraw[1][8 + k]), __uint_as_float(sraw[1][16 + k]));
-#pragma unroll
-                    for (int k = 0; k < 8; ++k) e[k] = fmaxf(e[k], __uint_as_float(sraw[1][24 + k]));
-                    rmax = max3(max3(e[0], e[1], e[2]), max3(e[3], e[4], e[5]), fmaxf(e[6], e[7])) * scale;
-                } else {
-#pragma unroll
-                    for (int k = 0; k < 8; ++k) e[k] = min3(__uint_as_float(sraw[0][k]), __uint_as_float(sraw[0][8 + k]), __uint_as_float(sraw[0][16 + k]));
-#pragma unroll
-                    for (int k = 0; k < 8; ++k) e[k] = min3(e[k], __uint_as_float(sraw[0][24 + k]), __uint_as_float(sraw[1][k]));
-#pragma unroll
-                    for (int k = 0; k < 8; ++k) e[k] = min3(e[k], __uint_as_float(sraw[1][8 + k]), __uint_as_float(sraw[1][16 + k]));
-#pragma unroll
-                    for (int k = 0; k < 8; ++k) e[k] = fminf(e[k], __uint_as_float(sraw[1][24 + k]));
-                    rmax = min3(min3(e[0], e[1], e[2]), min3(e[3], e[4], e[5]), fminf(e[6], e[7])) * scale;
-                }
-            } else {
-                rmax = -INFINITY;
-#pragma unroll
-                for (int h = 0; h < 2; ++h)
-#pragma unroll
-                    for (int c = 0; c < 32; ++c)
-                        if (key0 + h * 32 + c < count) rmax = fmaxf(rmax, __uint_as_float(sraw[h][c]) * scale);
-            }
-            // the reference max moves only when it has to (first tile) or when a row outgrew it by 2^8
-            const bool grow = rmax > m_ref + kRescaleThreshold;
-            const float m_new = grow ? rmax : m_ref;
-            const float corr = grow ? ex2(m_ref - m_new) : 1.f;   // ex2(-inf) = 0 on the first tile
-            const float neg_m = -m_new;
-            float rs[4] = {0.f, 0.f, 0.f, 0.f};
-            uint32_t packed[32];
-#pragma unroll
-            for (int h = 0; h < 2; ++h)
-#pragma unroll
-                for (int c = 0; c < 32; c += 2) {
-                    float x0, x1;
-                    fma2(x0, x1, __uint_as_float(sraw[h][c]), __uint_as_float(sraw[h][c + 1]), scale, neg_m);
-                    float p0 = ex2(x0), p1 = ex2(x1);
-                    if (need_mask) {
-                        p0 = key0 + h * 32 + c < count ? p0 : 0.f;
-                        p1 = key0 + h * 32 + c + 1 < count ? p1 : 0.f;
+                    for (int c = 0; c < 32; c += 2) {
+                        float x0, x1, p0, p1;
+                        fma2(x0, x1, __uint_as_float(sraw[h][c]), __uint_as_float(sraw[h][c + 1]), scale, neg_m);
+                        if (((c >> 1) % kPolyOneIn) == kPolyOneIn - 1) {
+                            ex2_poly2(p0, p1, x0, x1);
+                        } else {
+                            p0 = ex2(x0);
+                            p1 = ex2(x1);
+                        }
+                        if constexpr (kMasked) {
+                            p0 = h * 32 + c < live_keys ? p0 : 0.f;
+                            p1 = h * 32 + c + 1 < live_keys ? p1 : 0.f;
+                        }
+                        add2(rs[c & 2], rs[(c & 2) + 1], p0, p1);
+                        packed[c >> 1] = pack_bf16(p0, p1);
                     }
-                    add2(rs[c & 2], rs[(c & 2) + 1], p0, p1);
-                    packed[h * 16 + (c >> 1)] = pack_bf16(p0, p1);
+                    // P as the next A operand: 64 bf16 of this row as 32 packed columns over the start of its S buffer
+                    tmem_st16(sbuf + h * 16, packed);
                 }
-            const float rsum = (rs[0] + rs[1]) + (rs[2] + rs[3]);
-            l_sum = l_sum * corr + rsum;
-            m_ref = m_new;
-
-            if (j >= 1 && __any_sync(0xffffffffu, grow)) {
-                // rare: some row of this warp moved its reference max, so O (tiles 0 .. j-1) must be rescaled
-                // before PV of this tile; PV of tile j-1 has to be finished first
-                mbar_wait(bar_odone((j - 1) & 1), ((j - 1) >> 1) & 1, s_abort, prm.status, 9);
-                tc_fence_after();
-#pragma unroll 1
-                for (int c0 = 0; c0 < kHeadDim; c0 += 32) {
-                    uint32_t oraw[32];
-                    tmem_ld32(lane_addr + 128 + c0, oraw);
-                    tmem_wait_ld();
-#pragma unroll
-                    for (int c = 0; c < 32; ++c) oraw[c] = __float_as_uint(__uint_as_float(oraw[c]) * corr);
-                    tmem_st32(lane_addr + 128 + c0, oraw);
-                }
+                return (rs[0] + rs[1]) + (rs[2] + rs[3]);
+            };
+            // Fast path (every unmasked tile after the first): no max pass.  The exponentials are taken against the
+            // row's current reference max m_ref, which is the max of some earlier score, so later keys far below it
+            // rightly vanish; keys far above it make the row sum explode, and then (rarely) the tile is redone the
+            // careful way below.  Up to that bound P and the sums just carry a larger exponent: fp32 accumulation
+            // and the 8-bit mantissa of bf16 P lose nothing by it.
+            float rsum = 0.f, corr = 1.f;
+            bool careful = j == 0 || need_mask;
+            if (!careful) {
+                rsum = exp_pass(std::false_type{}, -m_ref);
+                careful = __any_sync(0xffffffffu, !(rsum <= kRowSumLimit));   // also true for inf / NaN
+                if (careful) tmem_wait_st();      // the stores of the abandoned pass land before the new ones
             }
-            // P as the next A operand: 64 bf16 of this row as 32 packed columns over the start of its S buffer
-            tmem_st32(lane_addr + sb * kKeys, packed);
+            if (careful) {
+                float rmax;
+                if (!need_mask) {
+                    // the max of scale * s is scale * (max or min of s): take the extreme of the raw scores, 8 chains of 3-input ops
+                    float e[8];
+                    if (scale >= 0.f) {
+#pragma unroll
+                        for (int k = 0; k < 8; ++k) e[k] = max3(__uint_as_float(sraw[0][k]), __uint_as_float(sraw[0][8 + k]), __uint_as_float(sraw[0][16 + k]));
+#pragma unroll
+                        for (int k = 0; k < 8; ++k) e[k] = max3(e[k], __uint_as_float(sraw[0][24 + k]), __uint_as_float(sraw[1][k]));
+#pragma unroll
+                        for (int k = 0; k < 8; ++k) e[k] = max3(e[k], __uint_as_float(sraw[1][8 + k]), __uint_as_float(sraw[1][16 + k]));
+#pragma unroll
+                        for (int k = 0; k < 8; ++k) e[k] = fmaxf(e[k], __uint_as_float(sraw[1][24 + k]));
+                        rmax = max3(max3(e[0], e[1], e[2]), max3(e[3], e[4], e[5]), fmaxf(e[6], e[7])) * scale;
+                    } else {
+#pragma unroll
+                        for (int k = 0; k < 8; ++k) e[k] = min3(__uint_as_float(sraw[0][k]), __uint_as_float(sraw[0][8 + k]), __uint_as_float(sraw[0][16 + k]));
+#pragma unroll
+                        for (int k = 0; k < 8; ++k) e[k] = min3(e[k], __uint_as_float(sraw[0][24 + k]), __uint_as_float(sraw[1][k]));
+#pragma unroll
+                        for (int k = 0; k < 8; ++k) e[k] = min3(e[k], __uint_as_float(sraw[1][8 + k]), __uint_as_float(sraw[1][16 + k]));
+#pragma unroll
+                        for (int k = 0; k < 8; ++k) e[k] = fminf(e[k], __uint_as_float(sraw[1][24 + k]));
+                        rmax = min3(min3(e[0], e[1], e[2]), min3(e[3], e[4], e[5]), fminf(e[6], e[7])) * scale;
+                    }
+                } else {
+                    // masked tile: keys the row does not see are left out (their scores may be anything)
+                    rmax = -INFINITY;
+#pragma unroll
+                    for (int h = 0; h < 2; ++h)
+#pragma unroll
+                        for (int c = 0; c < 32; ++c)
+                            if (h * 32 + c < live_keys) rmax = fmaxf(rmax, __uint_as_float(sraw[h][c]) * scale);
+                }
+                // the reference max moves only when it has to (first tile) or when a row outgrew it by 2^8
+                const bool grow = rmax > m_ref + kRescaleThreshold;
+                const float m_new = grow ? rmax : m_ref;
+                corr = grow ? ex2(m_ref - m_new) : 1.f;   // ex2(-inf) = 0 on the first tile
+                if (j >= 1 && __any_sync(0xffffffffu, grow)) {
+                    // rare: some row of this warp moved its reference max, so O (tiles 0 .. j-1) must be rescaled
+                    // before PV of this tile; PV of tile j-1 has to be finished first
+                    mbar_wait(bar_odone(mt, (j - 1) & 1), ((j - 1) >> 1) & 1, s_abort, prm.status, 9);
+                    tc_fence_after();
+#pragma unroll 1
+                    for (int c0 = 0; c0 < kHeadDim; c0 += 16) {
+                        uint32_t oraw[16];
+                        tmem_ld16(o_addr + c0, oraw);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int c = 0; c < 16; ++c) oraw[c] = __float_as_uint(__uint_as_float(oraw[c]) * corr);
+                        tmem_st16(o_addr + c0, oraw);
+                    }
+                }
+                m_ref = m_new;
+                rsum = need_mask ? exp_pass(std::true_type{}, -m_ref) : exp_pass(std::false_type{}, -m_ref);
+            }
+            l_sum = l_sum * corr + rsum;
             tmem_wait_st();
             if (key0 + kKeys > L) {
-                // keys at or beyond L are dead slots (or were never copied): their V rows must be 0, not garbage
-                mbar_wait(bar_vfull(j % kStages), (j / kStages) & 1, s_abort, prm.status, 10);
-                const uint32_t v_addr = smem_u32(smem + kOffV + (j % kStages) * 2 * kHalfKV);
+                // keys at or beyond L are dead slots (or were never copied): their V rows must be 0, not garbage.
+                // Each warpgroup does it before releasing its own PV (the two may both write the same zeros).
+                const int r = 2 * j + 1;
+                mbar_wait(bar_full(r % kStages), (r / kStages) & 1, s_abort, prm.status, 10);
+                const uint32_t v_addr = smem_u32(smem + kOffKV + (r % kStages) * kTileKV);
                 const int first_dead = L - key0;
-                for (int idx = threadIdx.x - 64; idx < (kKeys - first_dead) * 16; idx += 128) {
-                    const int r = first_dead + (idx >> 4), c = idx & 15;
-                    asm volatile("st.shared.v4.b32 [%0], {%1,%1,%1,%1};" ::"r"(v_addr + (c >> 3) * kHalfKV + r * 128 + (c & 7) * 16),
+                for (int idx = wg_thread; idx < (kKeys - first_dead) * 16; idx += 128) {
+                    const int rr = first_dead + (idx >> 4), c = idx & 15;
+                    asm volatile("st.shared.v4.b32 [%0], {%1,%1,%1,%1};" ::"r"(v_addr + (c >> 3) * kHalfKV + rr * 128 + (c & 7) * 16),
                                  "r"(0) : "memory");
                 }
                 fence_proxy_async();      // the zeroed V rows become visible to the tensor core's reads
             }
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(bar_pfull(sb));
+            if (lane == 0) mbar_arrive(bar_pfull(mt, sb));
         }
 
         // ---- epilogue: O / l -> bf16 rows of out ----
-        mbar_wait(bar_odone((n_tiles - 1) & 1), ((n_tiles - 1) >> 1) & 1, s_abort, prm.status, 11);
-        tc_fence_after();
-        const float inv = l_sum > 0.f ? 1.f / l_sum : 0.f;
-        const long long orow = (static_cast<long long>(q_row0 + tok0 + tok_local) * prm.num_q_heads + head * g + head_local);
+        if (my_tiles > 0) {
+            mbar_wait(bar_odone(mt, (my_tiles - 1) & 1), ((my_tiles - 1) >> 1) & 1, s_abort, prm.status, 11);
+            tc_fence_after();
+            const float inv = l_sum > 0.f ? 1.f / l_sum : 0.f;
+            const long long orow = (static_cast<long long>(q_row0 + first_tok + tok_local) * prm.num_q_heads + head * g + head_local);
 #pragma unroll 1
-        for (int c0 = 0; c0 < kHeadDim; c0 += 32) {
-            uint32_t oraw[32];
-            tmem_ld32(lane_addr + 128 + c0, oraw);
-            tmem_wait_ld();
-            if (live && prm.out_f32 != nullptr) {
-                float4 *dst = reinterpret_cast<float4 *>(prm.out_f32 + orow * kHeadDim + c0);
+            for (int c0 = 0; c0 < kHeadDim; c0 += 32) {
+                uint32_t oraw[32];
+                tmem_ld32(o_addr + c0, oraw);
+                tmem_wait_ld();
+                if (live && prm.out_f32 != nullptr) {
+                    float4 *dst = reinterpret_cast<float4 *>(prm.out_f32 + orow * kHeadDim + c0);
 #pragma unroll
-                for (int k = 0; k < 8; ++k)
-                    dst[k] = make_float4(__uint_as_float(oraw[4 * k]) * inv, __uint_as_float(oraw[4 * k + 1]) * inv,
-                                         __uint_as_float(oraw[4 * k + 2]) * inv, __uint_as_float(oraw[4 * k + 3]) * inv);
-            } else if (live) {
-                uint4 *dst = reinterpret_cast<uint4 *>(prm.out + orow * kHeadDim + c0);
+                    for (int k = 0; k < 8; ++k)
+                        dst[k] = make_float4(__uint_as_float(oraw[4 * k]) * inv, __uint_as_float(oraw[4 * k + 1]) * inv,
+                                             __uint_as_float(oraw[4 * k + 2]) * inv, __uint_as_float(oraw[4 * k + 3]) * inv);
+                } else if (live) {
+                    uint4 *dst = reinterpret_cast<uint4 *>(prm.out + orow * kHeadDim + c0);
 #pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    uint4 v;
-                    v.x = pack_bf16(__uint_as_float(oraw[8 * k]) * inv, __uint_as_float(oraw[8 * k + 1]) * inv);
-                    v.y = pack_bf16(__uint_as_float(oraw[8 * k + 2]) * inv, __uint_as_float(oraw[8 * k + 3]) * inv);
-                    v.z = pack_bf16(__uint_as_float(oraw[8 * k + 4]) * inv, __uint_as_float(oraw[8 * k + 5]) * inv);
-                    v.w = pack_bf16(__uint_as_float(oraw[8 * k + 6]) * inv, __uint_as_float(oraw[8 * k + 7]) * inv);
-                    dst[k] = v;
+                    for (int k = 0; k < 4; ++k) {
+                        uint4 v;
+                        v.x = pack_bf16(__uint_as_float(oraw[8 * k]) * inv, __uint_as_float(oraw[8 * k + 1]) * inv);
+                        v.y = pack_bf16(__uint_as_float(oraw[8 * k + 2]) * inv, __uint_as_float(oraw[8 * k + 3]) * inv);
+                        v.z = pack_bf16(__uint_as_float(oraw[8 * k + 4]) * inv, __uint_as_float(oraw[8 * k + 5]) * inv);
+                        v.w = pack_bf16(__uint_as_float(oraw[8 * k + 6]) * inv, __uint_as_float(oraw[8 * k + 7]) * inv);
+                        dst[k] = v;
+                    }
                 }
             }
+            if (live && prm.lse != nullptr) prm.lse[orow] = l_sum > 0.f ? (m_ref + log2f(l_sum)) * kLn2 : -INFINITY;
         }
-        if (live && prm.lse != nullptr) prm.lse[orow] = l_sum > 0.f ? (m_ref + log2f(l_sum)) * kLn2 : -INFINITY;
         tc_fence_before();
     }
 
@@ -663,9 +783,9 @@ cudaError_t launch_chunk_attn(const AttnCall &c, cudaStream_t stream, int64_t *l
         prm.out = c.out; prm.lse = c.lse; prm.scale_log2 = c.sm_scale * kLog2e; prm.status = c.status;
         prm.shared_lens = c.shared_lens ? c.shared_lens + base : nullptr;
         prm.out_f32 = c.out_f32;
-        // an upper bound on the M-tiles of these items: every item has at most one ragged tile
-        const long long tiles = (static_cast<long long>(c.total_q) + tpt - 1) / tpt + n;
-        const long long blocks = tiles * hkv;
+        // an upper bound on the M-tile pairs of these items: every item has at most one ragged pair
+        const long long pairs = (static_cast<long long>(c.total_q) + 2 * tpt - 1) / (2 * tpt) + n;
+        const long long blocks = pairs * hkv;
         if (blocks > 0x7FFFFFFFLL) return cudaErrorInvalidValue;
         chunk_attn_kernel<<<static_cast<unsigned>(blocks), kThreads, kSmemBytes, stream>>>(qmap, kmap, vmap, prm);
         ++*launches;
