@@ -44,8 +44,8 @@ constexpr int kTensorBytes = kTile * kRowBytes;      // 16 KB of K (or V) per st
 constexpr int kStageBytes = 2 * kTensorBytes;
 constexpr int kQBytes = kMaxGroup * kRowBytes;       // 4 KB
 constexpr int kMergeStride = kHeadDim + 8;           // floats per merge-buffer row (padded)
-constexpr uint32_t kSpinLimit = 1u << 17;   // polls per wait; each poll sleeps in hardware for up to kSuspendNs
-constexpr uint32_t kSuspendNs = 10000;
+constexpr uint32_t kSpinLimit = 1u << 17;   // polls of the drain loop that runs once a block has given up
+constexpr long long kWaitCycles = 2000000000LL;   // a wait gives up after about a second
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 constexpr size_t kSlotFloats = kMaxGroup * kHeadDim + 2 * kMaxGroup;
@@ -105,18 +105,24 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity), "r"(kSuspendNs) : "memory");
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
-// Bounded wait.  Gives up when the limit runs out or another warp has already given up; the
+// Bounded wait.  The poll has no sleep in it (a sleeping poll wakes up to a microsecond late, which the short
+// calls feel).  Gives up when the limit runs out or another warp has already given up; the
 // caller carries on (with garbage data) so that every barrier sequence still completes.
 __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, DeviceStatus *status,
                                           int where) {
-    for (uint32_t it = 0; it < kSpinLimit; ++it) {
+    if (mbar_try_wait(bar, parity)) return;
+    const long long t0 = clock64();
+    for (uint32_t it = 1;; ++it) {
         if (mbar_try_wait(bar, parity)) return;
-        if (*abort_flag) return;
+        if ((it & 255u) == 0u) {
+            if (*abort_flag) return;
+            if (clock64() - t0 > kWaitCycles) break;
+        }
     }
     if (*abort_flag == 0) {
         *abort_flag = 1;
