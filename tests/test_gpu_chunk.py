@@ -65,6 +65,39 @@ def test_chunk_edges(cuda_device, P, hq, hkv):
     run_chunk_case(batch, cuda_device)
 
 
+@pytest.mark.parametrize("shape", ["rising", "falling", "spike"])
+def test_chunk_scores_that_jump_between_key_tiles(cuda_device, shape):
+    # Keys whose magnitude changes by steps of 64 positions: scores of later key tiles tower over (or vanish
+    # under) those of the first tile, so the running reference max has to move, the accumulator has to be
+    # rescaled, and the result is close to one-hot (O(1) outputs: a wrong key would show).
+    P = 16
+    prior = [700, 333, 64, 129]
+    n_new = [100, 40, 70, 3]
+    spec = dataclasses.replace(W.CONFIGS[4], page_size=P, num_traj=len(prior), num_q_heads=8, num_kv_heads=2,
+                               name=f"chunk_jump_{shape}")
+    batch = W.make_layout(spec, seed=11)
+    batch.seq_lens_before = np.array(prior, np.int32)
+    batch.n_new = np.array(n_new, np.int32)
+    batch.is_chunk[:] = True
+    batch.new_indptr = np.concatenate([[0], np.cumsum(batch.n_new)]).astype(np.int32)
+    pages = (batch.seq_lens_before + batch.n_new + P - 1) // P
+    batch.page_table, batch.num_pages = W.build_page_table(pages.astype(np.int64), 0.3, np.random.default_rng(5))
+    W.fill_tensors(batch)
+    for t, L in enumerate(prior):
+        steps = (L + 63) // 64
+        for pos in range(L):
+            s = pos // 64
+            if shape == "rising":
+                gain = 1.0 + 6.0 * s
+            elif shape == "falling":
+                gain = 1.0 + 6.0 * (steps - 1 - s)
+            else:
+                gain = 60.0 if s == steps // 2 else 1.0
+            pg = int(batch.page_table[t, pos // P])
+            batch.k_pool[pg, :, pos % P, :] = (batch.k_pool[pg, :, pos % P, :].float() * gain).to(torch.bfloat16)
+    run_chunk_case(batch, cuda_device)
+
+
 def test_chunk_equals_sequential_append_and_decode_on_gpu(cuda_device):
     spec = dataclasses.replace(W.shrink(W.CONFIGS[4], 3, 64, 32), name="seq")
     batch = W.make_batch(spec, seed=43)
