@@ -317,6 +317,7 @@ decode_splitkv_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
     if (warp == kProducerWarp) {
         // =============================== producer warp ===============================
         const int pages_per_tile = kTile / P;
+        const int tiles_per_batch = 32 / pages_per_tile;
         const uint32_t page_bytes = static_cast<uint32_t>(P) * kRowBytes;
         int n = 0, pcount = 0;
         for (int p = p_begin; p < p_end; ++pcount) {
@@ -333,15 +334,24 @@ decode_splitkv_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
                           prm.q + (static_cast<long long>(pc.item) * prm.num_q_heads + pc.head * g) * kHeadDim,
                           static_cast<uint32_t>(g) * kRowBytes, bar_qfull(qs));
             }
-            for (int tile = pc.tile0; tile < pc.tile1; ++tile, ++n) {
-                const int stage = n % kStages;
-                // page ids of this tile, one lane per page
-                const int lp = tile * pages_per_tile + lane;
+            // Page ids are fetched 32 at a time, one per lane (8 to 32 tiles' worth), and the next 32 are requested a
+            // whole batch ahead, so the table lookup (a dependent load) is off the copy loop's path.
+            auto load_ids = [&](int first_tile) {
+                const int lp = first_tile * pages_per_tile + lane;
                 int pg = -1;
-                if (lane < pages_per_tile && lp * P < pc.len) {
+                if (first_tile + lane / pages_per_tile < pc.tile1 && lp * P < pc.len) {
                     pg = __ldg(table_row + lp);
                     if (pg < 0 || pg >= prm.num_pages) { report(prm.status, ROLLART_ERR_BOUNDS, pg, 2); pg = -1; }
                 }
+                return pg;
+            };
+            int ids_cur = load_ids(pc.tile0), ids_next = load_ids(pc.tile0 + tiles_per_batch);
+            for (int tile = pc.tile0; tile < pc.tile1; ++tile, ++n) {
+                const int stage = n % kStages;
+                const int within = (tile - pc.tile0) % tiles_per_batch;
+                if (tile > pc.tile0 && within == 0) { ids_cur = ids_next; ids_next = load_ids(tile + tiles_per_batch); }
+                int pg = __shfl_sync(0xffffffffu, ids_cur, (within * pages_per_tile + lane) & 31);
+                if (lane >= pages_per_tile) pg = -1;
                 const uint32_t nvalid = __popc(__ballot_sync(0xffffffffu, pg >= 0));
                 mbar_wait(bar_empty(stage), ((n / kStages) & 1) ^ 1, s_abort, prm.status, 2);
                 if (*s_abort) continue;
