@@ -59,10 +59,12 @@ constexpr int kMlFloats = kConsumerWarps * kMaxGroup * 2;           // (m, l) of
 constexpr int kOffMl = kOffMerge + 2 * kMergeFloats * 4;
 constexpr int kOffLens = kOffMl + 2 * kMlFloats * 4;
 constexpr int kOffPrefix = kOffLens + kMaxItems * 4;
-constexpr int kOffBars = kOffPrefix + (kMaxItems + 32) * 4;
+constexpr int kOffTraj = kOffPrefix + (kMaxItems + 32) * 4;   // trajectory of every item (read once from global memory)
+constexpr int kOffBars = kOffTraj + kMaxItems * 4;
 constexpr int kNumBars = 2 * kStages + 8;
 constexpr int kOffAbort = kOffBars + kNumBars * 8;
 constexpr int kSmemBytes = kOffAbort + 16 + 1024;    // + slack for the 1024-byte alignment
+static_assert(kSmemBytes <= 227 * 1024, "the block must fit the shared memory of an SM");
 
 struct DecodeParams {
     const int32_t *page_table;
@@ -226,6 +228,7 @@ decode_splitkv_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     int *s_lens = reinterpret_cast<int *>(smem + kOffLens);
     int *s_prefix = reinterpret_cast<int *>(smem + kOffPrefix);
+    int *s_traj = reinterpret_cast<int *>(smem + kOffTraj);
     float *s_merge = reinterpret_cast<float *>(smem + kOffMerge);
     float *s_ml = reinterpret_cast<float *>(smem + kOffMl);
     volatile int *s_abort = reinterpret_cast<volatile int *>(smem + kOffAbort);
@@ -240,9 +243,26 @@ decode_splitkv_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int hkv = prm.num_kv_heads, P = prm.page_size, g = prm.group;
 
+    // Launched with programmatic stream serialisation, this grid may start while the kernel before it in the stream
+    // is still draining: let the next launch do the same, set up what needs no global memory, and only then wait
+    // for the earlier kernel's results (lengths, pages, tickets) to be complete and visible.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    // zero both Q buffers once: rows >= g are never written by the copies and must read as 0
+    for (int i = threadIdx.x; i < 2 * kQBytes / 16; i += kThreads)
+        reinterpret_cast<uint4 *>(smem + kOffQ)[i] = make_uint4(0, 0, 0, 0);
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) { mbar_init(bar_full(s), 1); mbar_init(bar_empty(s), kConsumerWarps / 2); }
+        for (int s = 0; s < 2; ++s) { mbar_init(bar_qfull(s), 1); mbar_init(bar_qempty(s), kConsumerWarps); }
+        for (int s = 0; s < 2; ++s) { mbar_init(bar_epfull(s), 1); mbar_init(bar_epempty(s), 1); }
+        *s_abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+
     // ---- lengths -> tiles per item -> exclusive prefix (shared memory) ----
     for (int i = threadIdx.x; i < prm.n_items; i += kThreads) {
         const int t = prm.traj_ids ? __ldg(prm.traj_ids + i) : i + prm.item_offset;
+        s_traj[i] = t;
         int L = 0;
         if (t < 0 || t >= prm.num_traj) {
             report(prm.status, ROLLART_ERR_BOUNDS, t, 2);
@@ -262,16 +282,6 @@ decode_splitkv_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
             }
         }
         s_lens[i] = L;
-    }
-    // zero both Q buffers once: rows >= g are never written by the copies and must read as 0
-    for (int i = threadIdx.x; i < 2 * kQBytes / 16; i += kThreads)
-        reinterpret_cast<uint4 *>(smem + kOffQ)[i] = make_uint4(0, 0, 0, 0);
-    if (threadIdx.x == 0) {
-        for (int s = 0; s < kStages; ++s) { mbar_init(bar_full(s), 1); mbar_init(bar_empty(s), kConsumerWarps / 2); }
-        for (int s = 0; s < 2; ++s) { mbar_init(bar_qfull(s), 1); mbar_init(bar_qempty(s), kConsumerWarps); }
-        for (int s = 0; s < 2; ++s) { mbar_init(bar_epfull(s), 1); mbar_init(bar_epempty(s), 1); }
-        *s_abort = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
     if (warp == 0) {
@@ -322,7 +332,7 @@ decode_splitkv_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
         int n = 0, pcount = 0;
         for (int p = p_begin; p < p_end; ++pcount) {
             const Piece pc = piece_at(s_prefix, s_lens, prm.n_items, hkv, p, p_end);
-            const int t = prm.traj_ids ? __ldg(prm.traj_ids + pc.item) : pc.item + prm.item_offset;
+            const int t = s_traj[pc.item];
             const int32_t *table_row = prm.page_table + static_cast<long long>(t) * prm.max_pages +
                                        (prm.page_offset ? __ldg(prm.page_offset + pc.item) : 0);
             // Q rows of this (item, kv head): g contiguous rows of 256 B
@@ -546,7 +556,7 @@ decode_splitkv_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
                 // comes from k_new / v_new: put it into the staged tile (over whatever the copy brought for that
                 // slot) and into the pool, where later steps will find it.  Lanes 0-15 move K, lanes 16-31 move V.
                 const int kk = valid - 1, c16 = lane & 15;
-                const int t = prm.traj_ids ? __ldg(prm.traj_ids + pc.item) : pc.item + prm.item_offset;
+                const int t = s_traj[pc.item];
                 const int pos = pc.len - 1;
                 const int pg = __ldg(prm.page_table + static_cast<long long>(t) * prm.max_pages + pos / P);
                 const long long src = (static_cast<long long>(pc.item) * hkv + pc.head) * (kHeadDim / 8) + c16;
@@ -787,10 +797,17 @@ cudaError_t launch_decode_attn(const AttnCall &c, cudaStream_t stream, int64_t *
         prm.out_f32 = c.out_f32 ? c.out_f32 + static_cast<long long>(base) * c.num_q_heads * kHeadDim : nullptr;
         prm.slots = reinterpret_cast<float *>(static_cast<char *>(c.workspace) + info_bytes(chunk_items, hkv));
         prm.status = c.status;
-        decode_splitkv_kernel<<<grid, kThreads, kSmemBytes, stream>>>(*reinterpret_cast<CUtensorMap *>(tc.kmap),
-                                                                      *reinterpret_cast<CUtensorMap *>(tc.vmap), prm);
+        // programmatic stream serialisation: back-to-back decode launches overlap this grid's set-up with the
+        // previous grid's tail (the kernel waits for that grid before it reads anything)
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(grid); cfg.blockDim = dim3(kThreads); cfg.dynamicSmemBytes = kSmemBytes; cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr; cfg.numAttrs = 1;
+        e = cudaLaunchKernelEx(&cfg, decode_splitkv_kernel, *reinterpret_cast<CUtensorMap *>(tc.kmap),
+                               *reinterpret_cast<CUtensorMap *>(tc.vmap), prm);
         ++*launches;
-        e = cudaGetLastError();
         if (e != cudaSuccess) return e;
     }
     return cudaSuccess;
