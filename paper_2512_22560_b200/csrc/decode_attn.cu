@@ -2,8 +2,10 @@
 // block per SM.
 //
 // Schedule.  Every (item, kv head) owns ceil(L / 64) key tiles.  All tiles of the call are laid
-// on one line, ordered (item, kv head, tile), and the line is cut into gridDim.x equal spans, one
-// per thread block.  A block therefore reads the same number of bytes as every other block
+// on one line, ordered (item, kv head, tile), each (item, head) followed by a few units of padding
+// that stand for the fixed cost of working on one more (item, head) (query fetch, the merge of
+// the warps, the write-out: 2.7 us measured, four tile times), and the line is cut into gridDim.x
+// equal spans, one per thread block.  A block therefore has the same work as every other block
 // whatever the length mix, and a span that crosses an (item, head) boundary simply starts a new
 // "piece".  A piece that covers its (item, head) entirely writes the final bf16 output; otherwise
 // it writes an un-normalised fp32 partial (O, m, l) into a workspace slot and takes a ticket; the
@@ -34,6 +36,7 @@ namespace rollart {
 namespace {
 
 constexpr int kTile = 64;                 // keys per stage
+constexpr int kPieceCost = 4;             // what starting another (item, head) costs a block, in tile times (measured: 2.7 us)
 constexpr int kStages = 6;
 constexpr int kConsumerWarps = 8;         // two groups of four
 constexpr int kProducerWarp = kConsumerWarps;        // warp 8 issues the copies
@@ -199,7 +202,12 @@ __device__ __forceinline__ void merge_slice(const float (&a)[4], const float (&b
 // ------------------------------------------------------------------------------------------
 struct Piece {
     int item, head, tile0, tile1, ntiles, len;
+    int line0;      // where this (item, head) starts on the line
+    int advance;    // how far this piece moves the walk along the line
 };
+
+// Length of an (item, head) on the line: its tiles plus the fixed cost of a piece.
+__device__ __forceinline__ int line_len(int len) { return len > 0 ? (len + kTile - 1) / kTile + kPieceCost : 0; }
 
 __device__ __forceinline__ Piece piece_at(const int *prefix, const int *lens, int n_items, int hkv, int p, int p_end) {
     int lo = 0, hi = n_items;                     // largest item with prefix[item] * hkv <= p
@@ -209,11 +217,15 @@ __device__ __forceinline__ Piece piece_at(const int *prefix, const int *lens, in
     }
     Piece pc;
     pc.item = lo;
-    pc.ntiles = max(1, prefix[lo + 1] - prefix[lo]);
+    const int padded = max(1 + kPieceCost, prefix[lo + 1] - prefix[lo]);
+    pc.ntiles = padded - kPieceCost;
     const int rem = p - prefix[lo] * hkv;
-    pc.head = rem / pc.ntiles;
-    pc.tile0 = rem - pc.head * pc.ntiles;
-    pc.tile1 = min(pc.ntiles, pc.tile0 + (p_end - p));
+    pc.head = rem / padded;
+    const int off = rem - pc.head * padded;       // position inside the (item, head): tiles first, then the padding
+    pc.tile0 = min(off, pc.ntiles);
+    pc.tile1 = min(pc.ntiles, off + (p_end - p));
+    pc.line0 = p - off;
+    pc.advance = min(padded - off, p_end - p);
     pc.len = lens[lo];
     return pc;
 }
@@ -288,7 +300,7 @@ decode_splitkv_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
         const int per = (prm.n_items + 31) / 32;
         const int a = min(prm.n_items, lane * per), b = min(prm.n_items, a + per);
         int sum = 0;
-        for (int i = a; i < b; ++i) sum += (s_lens[i] + kTile - 1) / kTile;
+        for (int i = a; i < b; ++i) sum += line_len(s_lens[i]);
         int incl = sum;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
@@ -296,7 +308,7 @@ decode_splitkv_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
             if (lane >= o) incl += v;
         }
         int run = incl - sum;
-        for (int i = a; i < b; ++i) { s_prefix[i] = run; run += (s_lens[i] + kTile - 1) / kTile; }
+        for (int i = a; i < b; ++i) { s_prefix[i] = run; run += line_len(s_lens[i]); }
         if (lane == 31) s_prefix[prm.n_items] = incl;
     }
     fence_proxy_async();      // the zeroed Q rows are ordered before the bulk copies that land beside them
@@ -330,8 +342,10 @@ decode_splitkv_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
         const int tiles_per_batch = 32 / pages_per_tile;
         const uint32_t page_bytes = static_cast<uint32_t>(P) * kRowBytes;
         int n = 0, pcount = 0;
-        for (int p = p_begin; p < p_end; ++pcount) {
+        for (int p = p_begin; p < p_end;) {
             const Piece pc = piece_at(s_prefix, s_lens, prm.n_items, hkv, p, p_end);
+            p += pc.advance;
+            if (pc.tile0 >= pc.tile1) continue;       // the span touches only the padding of this (item, head)
             const int t = s_traj[pc.item];
             const int32_t *table_row = prm.page_table + static_cast<long long>(t) * prm.max_pages +
                                        (prm.page_offset ? __ldg(prm.page_offset + pc.item) : 0);
@@ -383,7 +397,7 @@ decode_splitkv_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
                     }
                 }
             }
-            p += pc.tile1 - pc.tile0;
+            ++pcount;
         }
         // every copy this warp issued has been waited for by the consumers unless the block gave up;
         // in that case wait (bounded) for the copies still in flight before the block exits
@@ -401,8 +415,10 @@ decode_splitkv_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
         // =============================== epilogue warp ===============================
         // lane -> 4 dims of a row; rows are handled one after the other
         int pcount = 0;
-        for (int p = p_begin; p < p_end; ++pcount) {
+        for (int p = p_begin; p < p_end;) {
             const Piece pc = piece_at(s_prefix, s_lens, prm.n_items, hkv, p, p_end);
+            p += pc.advance;
+            if (pc.tile0 >= pc.tile1) continue;
             const int eb = pcount & 1;
             mbar_wait(bar_epfull(eb), (pcount >> 1) & 1, s_abort, prm.status, 5);
             const float *mg = s_merge + eb * kMergeFloats;
@@ -436,8 +452,8 @@ decode_splitkv_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
                 // already published is the last by construction and combines straight from its shared
                 // tile; otherwise it publishes its slot (fence, then ticket) and combines only if its
                 // ticket turns out to be the last one.  Slots are merged in block order either way.
-                const int line0 = p - pc.tile0;                         // start of this (item, head) on the tile line
-                const int first = line0 / span, last = (line0 + pc.ntiles - 1) / span;
+                // blocks whose spans hold tiles of this (item, head): the padding at its end belongs to no piece
+                const int first = pc.line0 / span, last = (pc.line0 + pc.ntiles - 1) / span;
                 int arrived = 0;
                 if (lane == 0) asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(arrived) : "l"(prm.tickets + bh) : "memory");
                 arrived = __shfl_sync(0xffffffffu, arrived, 0);
@@ -503,7 +519,7 @@ decode_splitkv_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_epempty(eb));      // the shared tile may be refilled
-            p += pc.tile1 - pc.tile0;
+            ++pcount;
         }
         return;
     }
@@ -524,8 +540,10 @@ decode_splitkv_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
     const int v_chunk_lo = lm >> 1;
 
     int n = 0, pcount = 0;
-    for (int p = p_begin; p < p_end; ++pcount) {
+    for (int p = p_begin; p < p_end;) {
         const Piece pc = piece_at(s_prefix, s_lens, prm.n_items, hkv, p, p_end);
+        p += pc.advance;
+        if (pc.tile0 >= pc.tile1) continue;
         const int qs = pcount & 1;
         mbar_wait(bar_qfull(qs), (pcount >> 1) & 1, s_abort, prm.status, 3);
         uint32_t qa[8][4];
@@ -677,7 +695,7 @@ decode_splitkv_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
             consumer_bar();
         }
         if (threadIdx.x == 0) mbar_arrive(bar_epfull(eb));
-        p += pc.tile1 - pc.tile0;
+        ++pcount;
     }
 }
 
@@ -751,7 +769,7 @@ cudaError_t launch_decode_attn(const AttnCall &c, cudaStream_t stream, int64_t *
     const size_t need = decode_workspace_bytes(chunk_items, c.num_q_heads, hkv, c.max_seq_len, c.sm_count);
     if (c.workspace == nullptr || need > c.workspace_bytes) { *too_small = true; return cudaErrorInvalidValue; }
     // the tile line of one launch must fit an int
-    const long long tiles_bound = (static_cast<long long>(c.max_seq_len) + kTile - 1) / kTile * hkv;
+    const long long tiles_bound = ((static_cast<long long>(c.max_seq_len) + kTile - 1) / kTile + kPieceCost) * hkv;
     int per_launch = chunk_items;
     while (per_launch > 1 && tiles_bound * per_launch > 0x3FFFFFFFLL) per_launch /= 2;
 
@@ -901,7 +919,7 @@ extern "C" rollart_status rollart_decode_attn_noalloc(int device, const rollart_
     }
     const long long cap = static_cast<long long>(trajs->max_pages_per_traj) * pool->page_size;
     if (max_seq_len > cap) max_seq_len = static_cast<int32_t>(cap > 0x7FFFFFFF ? 0x7FFFFFFF : cap);
-    if ((static_cast<long long>(max_seq_len) + kTile - 1) / kTile * hkv * n_items > 0x3FFFFFFFLL) {
+    if (((static_cast<long long>(max_seq_len) + kTile - 1) / kTile + kPieceCost) * hkv * n_items > 0x3FFFFFFFLL) {
         write_err(err_buf, err_len, "n_items x num_kv_heads x max_seq_len too large for one launch");
         return ROLLART_ERR_WORKSPACE;
     }
