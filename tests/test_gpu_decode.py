@@ -159,6 +159,19 @@ def test_more_items_than_one_launch_holds(cuda_device):
     run_decode_case(W.make_batch(spec, seed=71), cuda_device)
 
 
+@pytest.mark.parametrize("lens", [[5, 5, 5], [1], [70, 3, 130, 2, 64]])
+def test_fewer_tiles_than_blocks(cuda_device, lens):
+    # a call far smaller than the machine: most blocks get nothing, and some spans of the tile line hold only the
+    # fixed-cost padding that follows an (item, head), i.e. no piece at all
+    spec = dataclasses.replace(W.CONFIGS[0], num_traj=len(lens), num_q_heads=4, num_kv_heads=1, name="tiny_line")
+    batch = W.make_layout(spec, seed=5)
+    batch.seq_lens_before = np.array(lens, np.int32)
+    pages = (batch.seq_lens_before + 1 + spec.page_size - 1) // spec.page_size
+    batch.page_table, batch.num_pages = W.build_page_table(pages.astype(np.int64), 0.3, np.random.default_rng(9))
+    W.fill_tensors(batch)
+    run_decode_case(batch, cuda_device)
+
+
 @pytest.mark.parametrize("i,T,div", [(0, 4, 1), (1, 16, 4), (3, 4, 16), (4, 10, 8)])
 def test_fused_append_decode_equals_the_two_calls_and_the_oracle(cuda_device, i, T, div):
     batch = W.make_batch(W.shrink(W.CONFIGS[i], T, div, 16), seed=500 + i)
