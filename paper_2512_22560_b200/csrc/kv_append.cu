@@ -48,6 +48,10 @@ kv_append_kernel(__nv_bfloat16 *__restrict__ k_pool, __nv_bfloat16 *__restrict__
 
     const long long n_vec = static_cast<long long>(total_new) * num_kv_heads * kVecPerRow;
     if (gid >= n_vec) return;
+    // the rows to move do not depend on where they go: start their loads before the chain of dependent
+    // look-ups (item search, length, page id), so that the two latencies overlap
+    const uint4 kv = __ldg(k_new + gid);
+    const uint4 vv = __ldg(v_new + gid);
     const int c = static_cast<int>(gid % kVecPerRow);
     const long long rh = gid / kVecPerRow;
     const int h = static_cast<int>(rh % num_kv_heads);
@@ -66,8 +70,6 @@ kv_append_kernel(__nv_bfloat16 *__restrict__ k_pool, __nv_bfloat16 *__restrict__
     const int slot = static_cast<int>(pos - lp * page_size);
 
     const long long dst = ((static_cast<long long>(pg) * num_kv_heads + h) * page_size + slot) * kVecPerRow + c;
-    const uint4 kv = __ldg(k_new + gid);
-    const uint4 vv = __ldg(v_new + gid);
     reinterpret_cast<uint4 *>(k_pool)[dst] = kv;
     reinterpret_cast<uint4 *>(v_pool)[dst] = vv;
 }
