@@ -20,7 +20,8 @@
 //   O_t += P_t V     tcgen05.mma with the A operand (P) in TMEM, M 128 x N 128 x K 64; V is the
 //                    MN-major B operand straight from its [key][dim] page layout
 //
-// Warp roles: warp 0 issues the copies (page ids fetched 32 at a time, a batch ahead), warps 1 and
+// Warp roles: warp 0 issues the copies (page ids fetched 32 at a time, a batch ahead; two boxes per
+// page for K, whose MMAs span the keys of several pages, one box per page for V), warps 1 and
 // 2 each issue the MMAs of one M-tile, warps 4-7 and 8-11 are the two softmax warpgroups, which also
 // write the result.  A block uses ~194 KB of shared memory (Q 64 KB, 8 K/V stages of 16 KB) and all
 // 512 TMEM columns (2 x 2 S buffers of 64, 2 O accumulators of 128): one block per SM.
@@ -54,7 +55,7 @@ constexpr int kTileQ = 2 * kHalfQ;
 constexpr int kHalfKV = kKeys * 128;       // 8 KB: 64 keys x 64 dims
 constexpr int kTileKV = 2 * kHalfKV;
 constexpr int kOffQ = 0;                                   // [M-tile][half][row][128 B]
-constexpr int kOffKV = kOffQ + 2 * kTileQ;                 // stages x [half][key][128 B]
+constexpr int kOffKV = kOffQ + 2 * kTileQ;                 // stages: a K tile is [half][key][128 B], a V tile [page][half][slot][128 B]
 constexpr int kOffBars = kOffKV + kStages * kTileKV;
 constexpr int kNumBars = 1 + 2 * kStages + 4 + 4 + 4;      // q | kv full/empty | per M-tile and S buffer: s_full, p_full, o_done
 constexpr int kOffTmemSlot = kOffBars + kNumBars * 8;
@@ -134,6 +135,11 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map
     asm volatile(
         "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
         ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(x), "r"(y), "r"(z) : "memory");
+}
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1, int c2, int c3) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
 }
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -452,10 +458,15 @@ chunk_attn_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constan
                 if (lane == 0) mbar_arrive_expect_tx(bar_full(stage), nvalid * 2u * half_page);
                 __syncwarp();
                 if (pg >= 0) {
-                    const uint32_t dst = smem_u32(smem + kOffKV + stage * kTileKV) + lane * half_page;
-                    const CUtensorMap *map = kv == 0 ? &kmap : &vmap;
-                    tma_load_2d(dst, map, bar_full(stage), 0, row);
-                    tma_load_2d(dst + kHalfKV, map, bar_full(stage), 64, row);
+                    const uint32_t stage_addr = smem_u32(smem + kOffKV + stage * kTileKV);
+                    if (kv == 0) {
+                        // K tile as [half][key][128 B]: two boxes per page (a QK^T MMA spans the keys of all pages)
+                        tma_load_2d(stage_addr + lane * half_page, &kmap, bar_full(stage), 0, row);
+                        tma_load_2d(stage_addr + lane * half_page + kHalfKV, &kmap, bar_full(stage), 64, row);
+                    } else {
+                        // V tile as [page][half][slot][128 B]: one box per page (a PV MMA step stays inside a page)
+                        tma_load_4d(stage_addr + lane * 2u * half_page, &vmap, bar_full(stage), 0, 0, 0, pg * hkv + head);
+                    }
                 }
             }
         }
@@ -477,6 +488,13 @@ chunk_attn_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constan
             const uint32_t kv_addr = smem_u32(smem + kOffKV);
             const uint64_t q_desc = smem_desc(smem_u32(smem + kOffQ) + mt * kTileQ, 16);
             const uint32_t s_tmem = tmem + mt * 2 * kKeys, o_tmem = tmem + kTmemO + mt * kHeadDim;
+            // V stage image is [page][half][slot][128 B]: the 16 keys of PV step ks sit in page (16 ks) / P at slot
+            // (16 ks) % P; the two 64-dim halves of a page are P * 128 B apart
+            const uint32_t v_half = static_cast<uint32_t>(P) * 128u;
+            uint64_t v_off[kKeys / 16];
+#pragma unroll
+            for (int ks = 0; ks < kKeys / 16; ++ks)
+                v_off[ks] = static_cast<uint64_t>((((ks * 16) / P) * P * kRowBytes + ((ks * 16) % P) * 128) >> 4);
             auto full_wait = [&](int r, int where) {
                 mbar_wait(bar_full(r % kStages), (r / kStages) & 1, s_abort, prm.status, where);
             };
@@ -509,12 +527,11 @@ chunk_attn_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constan
                 if (j < my_tiles) {
                     mbar_wait(bar_pfull(mt, j & 1), (j >> 1) & 1, s_abort, prm.status, 4);
                     tc_fence_after();
-                    const uint64_t v_desc = smem_desc(kv_addr + ((2 * j + 1) % kStages) * kTileKV, kHalfKV);
+                    const uint64_t v_desc = smem_desc(kv_addr + ((2 * j + 1) % kStages) * kTileKV, v_half);
                     const uint32_t acc0 = j > 0 ? 1u : 0u;
 #pragma unroll
                     for (int ks = 0; ks < kKeys / 16; ++ks)     // 16 keys per step: 8 packed columns along P's row, 2048 B down V
-                        umma_bf16_ts(o_tmem, s_tmem + (j & 1) * kKeys + ks * 8, v_desc + static_cast<uint64_t>((ks * 2048) >> 4),
-                                     kIdescPV, ks > 0 ? 1u : acc0);
+                        umma_bf16_ts(o_tmem, s_tmem + (j & 1) * kKeys + ks * 8, v_desc + v_off[ks], kIdescPV, ks > 0 ? 1u : acc0);
                     umma_commit(bar_odone(mt, j & 1));
                 }
                 umma_commit(bar_empty((2 * j + 1) % kStages));   // V(j): this thread's PV(j), if any, has read it
@@ -663,8 +680,8 @@ chunk_attn_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constan
                 const int first_dead = L - key0;
                 for (int idx = wg_thread; idx < (kKeys - first_dead) * 16; idx += 128) {
                     const int rr = first_dead + (idx >> 4), c = idx & 15;
-                    asm volatile("st.shared.v4.b32 [%0], {%1,%1,%1,%1};" ::"r"(v_addr + (c >> 3) * kHalfKV + rr * 128 + (c & 7) * 16),
-                                 "r"(0) : "memory");
+                    const uint32_t a = v_addr + (rr / P) * (P * kRowBytes) + (c >> 3) * (P * 128) + (rr % P) * 128 + (c & 7) * 16;
+                    asm volatile("st.shared.v4.b32 [%0], {%1,%1,%1,%1};" ::"r"(a), "r"(0) : "memory");
                 }
                 fence_proxy_async();      // the zeroed V rows become visible to the tensor core's reads
             }
@@ -745,6 +762,19 @@ bool encode_pool_rows(CUtensorMap *map, const void *pool, int num_pages, int hkv
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// pool as [unit = (page, head)][slot][half][64 dims]; one box = one (page, head) tile, landing as [half][slot][128 B]
+bool encode_pool_pages(CUtensorMap *map, const void *pool, int num_pages, int hkv, int P) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[4] = {64, static_cast<cuuint64_t>(P), 2, static_cast<cuuint64_t>(num_pages) * hkv};
+    const cuuint64_t strides[3] = {kRowBytes, 128, static_cast<cuuint64_t>(P) * kRowBytes};
+    const cuuint32_t box[4] = {64, static_cast<cuuint32_t>(P), 2, 1};
+    const cuuint32_t ones[4] = {1, 1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(pool), dims, strides, box, ones,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 // q as [token][q head][128 dims]; one box = 64 dims x g heads x (128 / g) tokens, landing as
 // [token][head][128 B]: exactly the rows of an M-tile.  Tokens past the end read as zero.
 bool encode_q_map(CUtensorMap *map, const void *q, int total_q, int hq, int g) {
@@ -769,7 +799,7 @@ cudaError_t launch_chunk_attn(const AttnCall &c, cudaStream_t stream, int64_t *l
     CUtensorMap qmap, kmap, vmap;
     if (!encode_q_map(&qmap, c.q, c.total_q, c.num_q_heads, g) ||
         !encode_pool_rows(&kmap, c.pool.k, c.pool.num_pages, hkv, c.pool.page_size) ||
-        !encode_pool_rows(&vmap, c.pool.v, c.pool.num_pages, hkv, c.pool.page_size))
+        !encode_pool_pages(&vmap, c.pool.v, c.pool.num_pages, hkv, c.pool.page_size))
         return cudaErrorInvalidValue;
     for (int base = 0; base < c.n_items; base += kMaxItems) {
         const int n = c.n_items - base < kMaxItems ? c.n_items - base : kMaxItems;
