@@ -20,8 +20,8 @@
 //   O_t += P_t V     tcgen05.mma with the A operand (P) in TMEM, M 128 x N 128 x K 64; V is the
 //                    MN-major B operand straight from its [key][dim] page layout
 //
-// Warp roles: warp 0 issues the copies (page ids fetched 32 at a time, a batch ahead; two boxes per
-// page for K, whose MMAs span the keys of several pages, one box per page for V), warps 1 and
+// Warp roles: warps 0 and 3 issue the copies (0: Q and K, two boxes per page since a QK^T MMA spans the
+// keys of several pages; 3: V, one box per page; page ids fetched 32 at a time, a batch ahead), warps 1 and
 // 2 each issue the MMAs of one M-tile, warps 4-7 and 8-11 are the two softmax warpgroups, which also
 // write the result.  A block uses ~194 KB of shared memory (Q 64 KB, 8 K/V stages of 16 KB) and all
 // 512 TMEM columns (2 x 2 S buffers of 64, 2 O accumulators of 128): one block per SM.
@@ -41,7 +41,7 @@ namespace {
 constexpr int kRows = 128;                 // query rows of an M-tile (UMMA M)
 constexpr int kKeys = 64;                  // keys per KV tile
 constexpr int kStages = 8;                 // ring of KV tiles; K(j) and V(j) take alternate slots
-constexpr int kThreads = 384;              // warp 0 copies, warps 1-2 MMA of M-tile 0 / 1, warps 4-7 / 8-11 softmax of M-tile 0 / 1
+constexpr int kThreads = 384;              // warps 0 / 3 copy K / V, warps 1-2 MMA of M-tile 0 / 1, warps 4-7 / 8-11 softmax of M-tile 0 / 1
 constexpr int kMaxItems = 1024;            // items per launch (tile prefix lives in shared memory)
 constexpr long long kWaitCycles = 2000000000LL;   // a wait gives up after about a second
 constexpr float kLog2e = 1.4426950408889634f;
@@ -60,7 +60,8 @@ constexpr int kOffBars = kOffKV + kStages * kTileKV;
 constexpr int kNumBars = 1 + 2 * kStages + 4 + 4 + 4;      // q | kv full/empty | per M-tile and S buffer: s_full, p_full, o_done
 constexpr int kOffTmemSlot = kOffBars + kNumBars * 8;
 constexpr int kOffAbort = kOffTmemSlot + 8;
-constexpr int kSmemUsed = kOffAbort + 8;
+constexpr int kOffMl = kOffAbort + 8;                         // (m, l) of the second key stream of a lone M-tile, per row
+constexpr int kSmemUsed = kOffMl + kRows * 8;
 constexpr int kSmemBytes = kSmemUsed + 1024;               // + slack for the 1024-byte alignment
 static_assert(kSmemBytes <= 227 * 1024, "one block must fit an SM");
 static_assert((kMaxItems + 1) * 4 <= kStages * kTileKV, "the tile prefix is staged in the KV stages");
@@ -388,6 +389,11 @@ chunk_attn_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constan
         nt_[mt] = (maxc_[mt] + kKeys - 1) / kKeys;
     }
     const int n0 = nt_[0], n1 = nt_[1], nmax = max(n0, n1);
+    // A lone M-tile (the ragged end of a chunk, or a small shared-prefix group) would leave half of the block idle:
+    // its key tiles are then dealt alternately to the two halves (even tiles to MMA thread / warpgroup 0, odd tiles
+    // to 1), each with its own S buffers, running max, sum and O accumulator, and the two are merged at the end.
+    const bool split = n1 == 0 && n0 >= 2;
+    const int step = split ? 2 : 1;
     const int32_t *table_row = prm.page_table + static_cast<long long>(t) * prm.max_pages;
     if (nmax == 0) {
         // only in shared-prefix mode with an empty prefix: the result is out = 0, lse = -inf
@@ -407,7 +413,7 @@ chunk_attn_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constan
     for (int i = threadIdx.x; i < 2 * kTileQ / 16; i += kThreads) reinterpret_cast<uint4 *>(smem + kOffQ)[i] = make_uint4(0, 0, 0, 0);
     fence_proxy_async();
     if (threadIdx.x == 32) {
-        for (int s = 0; s < kStages; ++s) mbar_init(bar_empty(s), n1 > 0 ? 2 : 1);
+        for (int s = 0; s < kStages; ++s) mbar_init(bar_empty(s), n1 > 0 ? 2 : 1);     // readers of a K/V tile
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 0) tmem_alloc(smem_u32(smem + kOffTmemSlot), kTmemCols);
@@ -416,9 +422,12 @@ chunk_attn_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constan
     tc_fence_after();
     const uint32_t tmem = *s_tmem;
 
-    if (warp == 0) {
-        // =============================== copy warp ===============================
-        if (lane == 0) {
+    if (warp == 0 || warp == 3) {
+        // =============================== copy warps ===============================
+        // Warp 0 brings the Q tiles and every K tile, warp 3 every V tile: a thread is held for some 80 cycles by each
+        // tensor copy it issues, and twelve of them per key tile from one warp were close to the tile period.
+        const int kv = warp == 3 ? 1 : 0;
+        if (kv == 0 && lane == 0) {
             const int live_tiles = n1 > 0 ? 2 : 1;
             mbar_arrive_expect_tx(bar_q, static_cast<uint32_t>(live_tiles * tpt * g) * kRowBytes);
             for (int mt = 0; mt < live_tiles; ++mt) {
@@ -437,36 +446,38 @@ chunk_attn_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constan
             int pg = -1;
             if (lp * P < L && lp < prm.max_pages) {
                 pg = __ldg(table_row + lp);
-                if (pg < 0 || pg >= prm.num_pages) { report(prm.status, ROLLART_ERR_BOUNDS, pg, 3); pg = -1; }
+                if (pg < 0 || pg >= prm.num_pages) {
+                    if (kv == 0) report(prm.status, ROLLART_ERR_BOUNDS, pg, 3);
+                    pg = -1;
+                }
             }
             return pg;
         };
         int ids_cur = load_ids(0), ids_next = load_ids(1);
         for (int j = 0; j < nmax; ++j) {
-            if (*s_abort) break;
             const int within = j % tiles_per_batch;
-            if (j > 0 && within == 0) { ids_cur = ids_next; ids_next = load_ids(j / tiles_per_batch + 1); }
+            if (j > 0 && within == 0) {
+                if (*s_abort) break;
+                ids_cur = ids_next;
+                ids_next = load_ids(j / tiles_per_batch + 1);
+            }
             int pg = __shfl_sync(0xffffffffu, ids_cur, (within * pages_per_tile + lane) & 31);
             if (lane >= pages_per_tile) pg = -1;
             const uint32_t nvalid = __popc(__ballot_sync(0xffffffffu, pg >= 0));
-            const int row = (pg * hkv + head) * P;
-#pragma unroll
-            for (int kv = 0; kv < 2; ++kv) {           // K(j) then V(j)
-                const int r = 2 * j + kv, stage = r % kStages;
-                const uint32_t par = ((r / kStages) & 1) ^ 1;
-                mbar_wait(bar_empty(stage), par, s_abort, prm.status, 1 + kv);
-                if (lane == 0) mbar_arrive_expect_tx(bar_full(stage), nvalid * 2u * half_page);
-                __syncwarp();
-                if (pg >= 0) {
-                    const uint32_t stage_addr = smem_u32(smem + kOffKV + stage * kTileKV);
-                    if (kv == 0) {
-                        // K tile as [half][key][128 B]: two boxes per page (a QK^T MMA spans the keys of all pages)
-                        tma_load_2d(stage_addr + lane * half_page, &kmap, bar_full(stage), 0, row);
-                        tma_load_2d(stage_addr + lane * half_page + kHalfKV, &kmap, bar_full(stage), 64, row);
-                    } else {
-                        // V tile as [page][half][slot][128 B]: one box per page (a PV MMA step stays inside a page)
-                        tma_load_4d(stage_addr + lane * 2u * half_page, &vmap, bar_full(stage), 0, 0, 0, pg * hkv + head);
-                    }
+            const int r = 2 * j + kv, stage = r % kStages;       // K(j) and V(j) take alternate slots of the ring
+            mbar_wait(bar_empty(stage), ((r / kStages) & 1) ^ 1, s_abort, prm.status, 1 + kv);
+            if (lane == 0) mbar_arrive_expect_tx(bar_full(stage), nvalid * 2u * half_page);
+            __syncwarp();
+            if (pg >= 0) {
+                const uint32_t stage_addr = smem_u32(smem + kOffKV + stage * kTileKV);
+                if (kv == 0) {
+                    // K tile as [half][key][128 B]: two boxes per page (a QK^T MMA spans the keys of all pages)
+                    const int row = (pg * hkv + head) * P;
+                    tma_load_2d(stage_addr + lane * half_page, &kmap, bar_full(stage), 0, row);
+                    tma_load_2d(stage_addr + lane * half_page + kHalfKV, &kmap, bar_full(stage), 64, row);
+                } else {
+                    // V tile as [page][half][slot][128 B]: one box per page (a PV MMA step stays inside a page)
+                    tma_load_4d(stage_addr + lane * 2u * half_page, &vmap, bar_full(stage), 0, 0, 0, pg * hkv + head);
                 }
             }
         }
@@ -481,12 +492,14 @@ chunk_attn_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constan
         // Both threads release every KV stage (its barrier counts the live M-tiles), also for key tiles their own
         // M-tile does not use.
         const int mt = warp - 1;
-        const int my_tiles = mt == 0 ? n0 : n1;
-        if (lane == 0 && my_tiles > 0) {
+        // key tiles of this thread: j = first + i * step for i < cnt
+        const int first = split ? mt : 0;
+        const int cnt = split ? (n0 - mt + 1) / 2 : (mt == 0 ? n0 : n1);
+        if (lane == 0 && cnt > 0) {
             constexpr uint32_t kIdescQK = idesc(kKeys, false);
             constexpr uint32_t kIdescPV = idesc(kHeadDim, true);
             const uint32_t kv_addr = smem_u32(smem + kOffKV);
-            const uint64_t q_desc = smem_desc(smem_u32(smem + kOffQ) + mt * kTileQ, 16);
+            const uint64_t q_desc = smem_desc(smem_u32(smem + kOffQ) + (split ? 0 : mt) * kTileQ, 16);
             const uint32_t s_tmem = tmem + mt * 2 * kKeys, o_tmem = tmem + kTmemO + mt * kHeadDim;
             // V stage image is [page][half][slot][128 B]: the 16 keys of PV step ks sit in page (16 ks) / P at slot
             // (16 ks) % P; the two 64-dim halves of a page are P * 128 B apart
@@ -498,44 +511,44 @@ chunk_attn_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constan
             auto full_wait = [&](int r, int where) {
                 mbar_wait(bar_full(r % kStages), (r / kStages) & 1, s_abort, prm.status, where);
             };
-            auto issue_qk = [&](int j) {
+            auto issue_qk = [&](int i) {
+                const int j = first + i * step;
+                full_wait(2 * j, 6);                        // K(j)
+                tc_fence_after();
                 const uint64_t k_desc = smem_desc(kv_addr + ((2 * j) % kStages) * kTileKV, 16);
 #pragma unroll
                 for (int ks = 0; ks < kHeadDim / 16; ++ks) {   // 16 dims per step; the second 64 dims live in the other half
                     const uint64_t qoff = static_cast<uint64_t>(((ks >> 2) * kHalfQ + (ks & 3) * 32) >> 4);
                     const uint64_t koff = static_cast<uint64_t>(((ks >> 2) * kHalfKV + (ks & 3) * 32) >> 4);
-                    umma_bf16(s_tmem + (j & 1) * kKeys, q_desc + qoff, k_desc + koff, kIdescQK, ks > 0 ? 1u : 0u);
+                    umma_bf16(s_tmem + (i & 1) * kKeys, q_desc + qoff, k_desc + koff, kIdescQK, ks > 0 ? 1u : 0u);
                 }
-                umma_commit(bar_sfull(mt, j & 1));
+                umma_commit(bar_sfull(mt, i & 1));
                 umma_commit(bar_empty((2 * j) % kStages));
             };
             mbar_wait(bar_q, 0, s_abort, prm.status, 5);
-            full_wait(0, 6);
-            tc_fence_after();
             issue_qk(0);
-            for (int j = 0; j < nmax; ++j) {
-                if (j + 1 < nmax) {
-                    full_wait(2 * j + 2, 6);                // K(j+1)
-                    if (j + 1 < my_tiles) {
-                        tc_fence_after();
-                        issue_qk(j + 1);
-                    } else {
-                        umma_commit(bar_empty((2 * j + 2) % kStages));
-                    }
-                }
+            for (int i = 0; i < cnt; ++i) {
+                const int j = first + i * step;
+                if (i + 1 < cnt) issue_qk(i + 1);
                 full_wait(2 * j + 1, 3);                    // V(j)
-                if (j < my_tiles) {
-                    mbar_wait(bar_pfull(mt, j & 1), (j >> 1) & 1, s_abort, prm.status, 4);
-                    tc_fence_after();
-                    const uint64_t v_desc = smem_desc(kv_addr + ((2 * j + 1) % kStages) * kTileKV, v_half);
-                    const uint32_t acc0 = j > 0 ? 1u : 0u;
+                mbar_wait(bar_pfull(mt, i & 1), (i >> 1) & 1, s_abort, prm.status, 4);
+                tc_fence_after();
+                const uint64_t v_desc = smem_desc(kv_addr + ((2 * j + 1) % kStages) * kTileKV, v_half);
+                const uint32_t acc0 = i > 0 ? 1u : 0u;
 #pragma unroll
-                    for (int ks = 0; ks < kKeys / 16; ++ks)     // 16 keys per step: 8 packed columns along P's row, 2048 B down V
-                        umma_bf16_ts(o_tmem, s_tmem + (j & 1) * kKeys + ks * 8, v_desc + v_off[ks], kIdescPV, ks > 0 ? 1u : acc0);
-                    umma_commit(bar_odone(mt, j & 1));
-                }
-                umma_commit(bar_empty((2 * j + 1) % kStages));   // V(j): this thread's PV(j), if any, has read it
+                for (int ks = 0; ks < kKeys / 16; ++ks)     // 16 keys per step: 8 packed columns along P's row
+                    umma_bf16_ts(o_tmem, s_tmem + (i & 1) * kKeys + ks * 8, v_desc + v_off[ks], kIdescPV, ks > 0 ? 1u : acc0);
+                umma_commit(bar_odone(mt, i & 1));
+                umma_commit(bar_empty((2 * j + 1) % kStages));   // V(j)
             }
+            // key tiles that only the other M-tile uses (it sees more keys): this thread releases them unread
+            if (!split)
+                for (int j = cnt; j < nmax; ++j) {
+                    full_wait(2 * j, 6);
+                    umma_commit(bar_empty((2 * j) % kStages));
+                    full_wait(2 * j + 1, 3);
+                    umma_commit(bar_empty((2 * j + 1) % kStages));
+                }
         }
         __syncwarp();
     } else if (warp >= 4) {
@@ -546,20 +559,24 @@ chunk_attn_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constan
         const int row = quarter * 32 + lane;
         const uint32_t lane_addr = tmem + (static_cast<uint32_t>(quarter * 32) << 16);
         const uint32_t s_addr = lane_addr + mt * 2 * kKeys, o_addr = lane_addr + kTmemO + mt * kHeadDim;
-        const int my_tiles = mt == 0 ? n0 : n1;
-        const int toks = mt == 0 ? toks_[0] : toks_[1];
-        const int min_count = mt == 0 ? minc_[0] : minc_[1];
-        const int first_tok = tok0 + mt * tpt;
+        // key tiles of this warpgroup: j = first + i * step for i < cnt; a lone M-tile (split) is M-tile 0 for both
+        const int first = split ? mt : 0;
+        const int cnt = split ? (n0 - mt + 1) / 2 : (mt == 0 ? n0 : n1);
+        const int gt = split ? 0 : mt;                         // whose rows these are
+        const int toks = gt == 0 ? toks_[0] : toks_[1];
+        const int min_count = gt == 0 ? minc_[0] : minc_[1];
+        const int first_tok = tok0 + gt * tpt;
         const int tok_local = row / g, head_local = row - tok_local * g;
         const bool live = tok_local < toks;
         const int count = shared_mode ? L : min(L, prior + first_tok + min(tok_local, max(toks, 1) - 1) + 1);   // keys this row sees (>= 1)
         const float scale = prm.scale_log2;
         float m_ref = -INFINITY, l_sum = 0.f;
 
-        for (int j = 0; j < my_tiles; ++j) {
-            const int sb = j & 1;
+        for (int i = 0; i < cnt; ++i) {
+            const int j = first + i * step;
+            const int sb = i & 1;
             const uint32_t sbuf = s_addr + sb * kKeys;
-            mbar_wait(bar_sfull(mt, sb), (j >> 1) & 1, s_abort, prm.status, 8);
+            mbar_wait(bar_sfull(mt, sb), (i >> 1) & 1, s_abort, prm.status, 8);
             tc_fence_after();
             uint32_t sraw[2][32];
             tmem_ld32(sbuf, sraw[0]);
@@ -606,7 +623,7 @@ chunk_attn_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constan
             // careful way below.  Up to that bound P and the sums just carry a larger exponent: fp32 accumulation
             // and the 8-bit mantissa of bf16 P lose nothing by it.
             float rsum = 0.f, corr = 1.f;
-            bool careful = j == 0 || need_mask;
+            bool careful = i == 0 || need_mask;
             if (!careful) {
                 rsum = exp_pass(std::false_type{}, -m_ref);
                 careful = __any_sync(0xffffffffu, !(rsum <= kRowSumLimit));   // also true for inf / NaN
@@ -651,10 +668,10 @@ chunk_attn_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constan
                 const bool grow = rmax > m_ref + kRescaleThreshold;
                 const float m_new = grow ? rmax : m_ref;
                 corr = grow ? ex2(m_ref - m_new) : 1.f;   // ex2(-inf) = 0 on the first tile
-                if (j >= 1 && __any_sync(0xffffffffu, grow)) {
-                    // rare: some row of this warp moved its reference max, so O (tiles 0 .. j-1) must be rescaled
-                    // before PV of this tile; PV of tile j-1 has to be finished first
-                    mbar_wait(bar_odone(mt, (j - 1) & 1), ((j - 1) >> 1) & 1, s_abort, prm.status, 9);
+                if (i >= 1 && __any_sync(0xffffffffu, grow)) {
+                    // rare: some row of this warp moved its reference max, so O (the tiles before this one) must be
+                    // rescaled before PV of this tile; PV of the previous tile has to be finished first
+                    mbar_wait(bar_odone(mt, (i - 1) & 1), ((i - 1) >> 1) & 1, s_abort, prm.status, 9);
                     tc_fence_after();
 #pragma unroll 1
                     for (int c0 = 0; c0 < kHeadDim; c0 += 16) {
@@ -691,31 +708,58 @@ chunk_attn_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constan
         }
 
         // ---- epilogue: O / l -> bf16 rows of out ----
-        if (my_tiles > 0) {
-            mbar_wait(bar_odone(mt, (my_tiles - 1) & 1), ((my_tiles - 1) >> 1) & 1, s_abort, prm.status, 11);
+        if (cnt > 0) {
+            mbar_wait(bar_odone(mt, (cnt - 1) & 1), ((cnt - 1) >> 1) & 1, s_abort, prm.status, 11);
             tc_fence_after();
+        }
+        float w0 = 1.f, w1 = 0.f;                // weights of the two key streams of a lone M-tile
+        if (split) {
+            // warpgroup 1 hands its (m, l) to warpgroup 0, which owns the same TMEM lanes and reads both accumulators
+            float *ml = reinterpret_cast<float *>(smem + kOffMl);
+            if (mt == 1) { ml[2 * row] = m_ref; ml[2 * row + 1] = l_sum; }
+            tc_fence_before();
+            asm volatile("bar.sync 1, 256;" ::: "memory");
+            tc_fence_after();
+            if (mt == 0) {
+                const float m1 = ml[2 * row], l1 = ml[2 * row + 1];
+                const float m_all = fmaxf(m_ref, m1);
+                w0 = m_ref == -INFINITY ? 0.f : ex2(m_ref - m_all);
+                w1 = m1 == -INFINITY ? 0.f : ex2(m1 - m_all);
+                l_sum = l_sum * w0 + l1 * w1;
+                m_ref = m_all;
+            }
+        }
+        if (cnt > 0 && !(split && mt == 1)) {
             const float inv = l_sum > 0.f ? 1.f / l_sum : 0.f;
+            const float f0 = w0 * inv, f1 = w1 * inv;
             const long long orow = (static_cast<long long>(q_row0 + first_tok + tok_local) * prm.num_q_heads + head * g + head_local);
 #pragma unroll 1
             for (int c0 = 0; c0 < kHeadDim; c0 += 32) {
                 uint32_t oraw[32];
                 tmem_ld32(o_addr + c0, oraw);
                 tmem_wait_ld();
+                float ov[32];
+#pragma unroll
+                for (int k = 0; k < 32; ++k) ov[k] = __uint_as_float(oraw[k]) * f0;
+                if (split) {                     // uniform over the block
+                    tmem_ld32(o_addr + kHeadDim + c0, oraw);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int k = 0; k < 32; ++k) ov[k] = fmaf(__uint_as_float(oraw[k]), f1, ov[k]);
+                }
                 if (live && prm.out_f32 != nullptr) {
                     float4 *dst = reinterpret_cast<float4 *>(prm.out_f32 + orow * kHeadDim + c0);
 #pragma unroll
-                    for (int k = 0; k < 8; ++k)
-                        dst[k] = make_float4(__uint_as_float(oraw[4 * k]) * inv, __uint_as_float(oraw[4 * k + 1]) * inv,
-                                             __uint_as_float(oraw[4 * k + 2]) * inv, __uint_as_float(oraw[4 * k + 3]) * inv);
+                    for (int k = 0; k < 8; ++k) dst[k] = make_float4(ov[4 * k], ov[4 * k + 1], ov[4 * k + 2], ov[4 * k + 3]);
                 } else if (live) {
                     uint4 *dst = reinterpret_cast<uint4 *>(prm.out + orow * kHeadDim + c0);
 #pragma unroll
                     for (int k = 0; k < 4; ++k) {
                         uint4 v;
-                        v.x = pack_bf16(__uint_as_float(oraw[8 * k]) * inv, __uint_as_float(oraw[8 * k + 1]) * inv);
-                        v.y = pack_bf16(__uint_as_float(oraw[8 * k + 2]) * inv, __uint_as_float(oraw[8 * k + 3]) * inv);
-                        v.z = pack_bf16(__uint_as_float(oraw[8 * k + 4]) * inv, __uint_as_float(oraw[8 * k + 5]) * inv);
-                        v.w = pack_bf16(__uint_as_float(oraw[8 * k + 6]) * inv, __uint_as_float(oraw[8 * k + 7]) * inv);
+                        v.x = pack_bf16(ov[8 * k], ov[8 * k + 1]);
+                        v.y = pack_bf16(ov[8 * k + 2], ov[8 * k + 3]);
+                        v.z = pack_bf16(ov[8 * k + 4], ov[8 * k + 5]);
+                        v.w = pack_bf16(ov[8 * k + 6], ov[8 * k + 7]);
                         dst[k] = v;
                     }
                 }
