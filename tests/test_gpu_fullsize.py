@@ -90,6 +90,46 @@ def test_full_size_decode_sampled(cuda_device, cfg):
     ctx.close()
 
 
+@pytest.mark.parametrize("cfg", [1, 2, 3])
+def test_full_size_decode_with_needles(cuda_device, cfg):
+    # The same full-size step with keys planted that dominate the softmax (outputs of order one instead of
+    # ~1/sqrt(L): a wrong key, page or split would show): first and last token, page edges, the appended token,
+    # and one every 2048 positions so that every block's span of the sampled trajectories holds some.
+    spec = W.CONFIGS[cfg]
+    batch = W.make_batch(spec, device=cuda_device)
+    ids = batch.decode_ids
+    rng = np.random.default_rng(100 + cfg)
+    pick = sample_ids(batch.seq_lens_before, ids, 4, rng)
+    P = spec.page_size
+    pos = {}
+    for t in pick:
+        L = int(batch.seq_lens_before[t])
+        special = {0, L - 1, min(L - 1, P - 1), min(L - 1, P), (L // P) * P if L % P else L - P, L}
+        pos[int(t)] = sorted(special | set(range(1027, L, 2048)))
+    W.plant_needles(batch, pos)
+    rows = batch.decode_rows()
+    msl = int(batch.seq_lens_after[ids].max())
+    ctx = make_ctx(spec, len(ids), msl)
+    db = DeviceBatch(batch, cuda_device)
+    ridx = torch.from_numpy(rows).to(cuda_device)
+    q = db.q_new[ridx].contiguous()
+    out = torch.full_like(q, float("nan"))
+    lse = torch.full((len(ids), spec.num_q_heads), float("nan"), device=cuda_device)
+    ctx.append_decode_attn(db.k_pool, db.v_pool, db.page_table, db.lens_before, db.k_new[ridx].contiguous(),
+                           db.v_new[ridx].contiguous(), q, spec.sm_scale, msl, out, lse=lse, traj_ids=dev_i32(ids, cuda_device),
+                           seq_lens_out=db.lens_after)
+    ctx.check()
+    post = W.extract_trajs(db_as_batch(batch, db), pick)
+    kp, vp = W.bf16_to_u16(post.k_pool), W.bf16_to_u16(post.v_pool)
+    where = {int(t): i for i, t in enumerate(ids)}
+    sel = torch.from_numpy(np.array([where[int(t)] for t in pick])).to(cuda_device)
+    ref_o, ref_l = oracle.decode_attn(kp, vp, post.page_table, post.seq_lens_before + 1, W.bf16_to_u16(q[sel]), spec.sm_scale)
+    st = assert_attn_close(out[sel], ref_o, spec.name + " (needles)")
+    assert st["rms_ref"] > 0.1, st
+    assert_lse_close(lse[sel], ref_l, spec.name + " (needles)")
+    ctx.close()
+
+
 def db_as_batch(batch, db):
     """the batch with its pools replaced by the device pools after the GPU append"""
     import dataclasses
