@@ -195,6 +195,33 @@ rollart_status rollart_append_decode_attn(rollart_ctx *ctx, const rollart_kv_poo
                                           float *lse, int32_t *seq_lens_out, void *stream);
 
 /*
+ * fp8 KV pools.  Decoding is bound by reading the whole context once per generated token (Sec. 3.1), so a cache held
+ * in 8 bits halves the bytes of a decode step.  The two calls below are rollart_kv_append and rollart_decode_attn for
+ * pools whose elements are E4M3 codes (OCP 8-bit floating point: 1 sign, 4 exponent bits with bias 7, 3 mantissa
+ * bits, no infinities, largest finite value 448): pool->k_pool / v_pool are [device] uint8
+ * [num_pages][num_kv_heads][page_size][head_dim], 16-byte aligned, with one scale per pool and call: a key is
+ * k_scale * value(code), a value is v_scale * value(code).  Both scales must be positive and finite.
+ *
+ * rollart_kv_append_fp8: arguments as rollart_kv_append; k_new / v_new are bf16.  Every element is stored as
+ *   code = nearest E4M3 code (ties to even, magnitudes above 448 saturate to +-448) of x * (1 / scale), the
+ *   reciprocal and the product each rounded to fp32.  No other byte of the pools changes.
+ * rollart_decode_attn_fp8: arguments and result as rollart_decode_attn (q, out bf16; lse fp32) with
+ *   s_j = sm_scale * k_scale * <q, value(K code)>, out = v_scale * sum_j softmax(s)_j * value(V code).
+ *   Arithmetic: the codes and the query are converted to f16 (exact for the codes; a query element beyond the f16
+ *   range, |q| > 65504, is not supported), fp32 scores, softmax and accumulation; softmax weights are rounded to f16
+ *   before they multiply V.  Same schedule, same workspace, same errors as rollart_decode_attn.
+ * The paper does not describe a cache format; the fp8 pool is this library's option.
+ */
+rollart_status rollart_kv_append_fp8(rollart_ctx *ctx, const rollart_kv_pool *pool, const rollart_trajs *trajs,
+                                     const int32_t *traj_ids, const int32_t *new_indptr, int32_t n_items,
+                                     int32_t total_new, const void *k_new, const void *v_new, float k_scale, float v_scale,
+                                     int32_t *seq_lens_out, void *stream);
+rollart_status rollart_decode_attn_fp8(rollart_ctx *ctx, const rollart_kv_pool *pool, const rollart_trajs *trajs,
+                                       const int32_t *traj_ids, int32_t n_items, int32_t max_seq_len, const void *q,
+                                       int32_t num_q_heads, float sm_scale, float k_scale, float v_scale, void *out,
+                                       float *lse, void *stream);
+
+/*
  * Group decode step: rollart_decode_attn for a batch whose items form groups that share a prompt prefix.
  * The paper trains with GRPO at a group size of 8 and runs the rollout engine with prefix caching (Sec. 7.1),
  * so the members of a group hold the same first tokens and, with prefix sharing, their page-table rows list

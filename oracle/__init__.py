@@ -30,7 +30,7 @@ def lib():
         L = ctypes.CDLL(os.environ.get("ROLLART_ORACLE_LIB") or _build())
         L.oracle_num_threads.restype = ctypes.c_int
         for name in ("oracle_kv_append", "oracle_kv_gather", "oracle_attend", "oracle_lse_combine", "oracle_pages_reserve",
-                     "oracle_pages_release"):
+                     "oracle_pages_release", "oracle_e4m3_decode", "oracle_e4m3_encode"):
             getattr(L, name).restype = ctypes.c_int
         _lib = L
     return _lib
@@ -221,3 +221,58 @@ def lse_combine(parts_out: np.ndarray, parts_lse: np.ndarray):
         _check(rc)
         lse[i] = one.value
     return out.reshape(*inner, D), lse.reshape(inner)
+
+
+# ---- fp8 (E4M3) KV pools -------------------------------------------------------------------------
+
+def e4m3_decode(codes: np.ndarray) -> np.ndarray:
+    """Values (float64) of E4M3 codes (uint8)."""
+    codes = _c(codes, np.uint8)
+    out = np.empty(codes.shape, dtype=np.float64)
+    _check(lib().oracle_e4m3_decode(_p(codes), ctypes.c_int64(codes.size), _p(out)))
+    return out
+
+
+def e4m3_encode(x: np.ndarray) -> np.ndarray:
+    """Nearest E4M3 code (uint8) of each float32, ties to even, saturating at +-448."""
+    x = _c(x, np.float32)
+    out = np.empty(x.shape, dtype=np.uint8)
+    _check(lib().oracle_e4m3_encode(_p(x), ctypes.c_int64(x.size), _p(out)))
+    return out
+
+
+def bf16_bits_to_f32(bits: np.ndarray) -> np.ndarray:
+    return (np.ascontiguousarray(bits, dtype=np.uint16).astype(np.uint32) << 16).view(np.float32)
+
+
+def fp8_quantize_rows(rows_bf16: np.ndarray, scale: float) -> np.ndarray:
+    """E4M3 codes of bf16 rows (uint16 bit patterns) for a pool with the given scale: encode(x * (1 / scale)),
+    the reciprocal and the product both rounded to fp32 (the precision the quantised append works in)."""
+    inv = np.float32(1.0) / np.float32(scale)
+    return e4m3_encode(bf16_bits_to_f32(rows_bf16) * inv)
+
+
+def kv_append_fp8(k_pool: np.ndarray, v_pool: np.ndarray, page_table, seq_lens, new_indptr, k_new_bf16, v_new_bf16,
+                  k_scale: float, v_scale: float, traj_ids=None) -> np.ndarray:
+    """Quantised append into uint8 pools [pages][Hkv][P][D]: the rows are quantised, then appended by the same
+    bit copy as the bf16 pools (a row of D bytes is moved as D / 2 16-bit units)."""
+    assert k_pool.dtype == np.uint8 and v_pool.dtype == np.uint8 and k_pool.shape[-1] % 2 == 0
+    kq = fp8_quantize_rows(k_new_bf16, k_scale)
+    vq = fp8_quantize_rows(v_new_bf16, v_scale)
+    return kv_append(k_pool.view(np.uint16), v_pool.view(np.uint16), page_table, seq_lens, new_indptr,
+                     kq.view(np.uint16), vq.view(np.uint16), traj_ids=traj_ids)
+
+
+def fp8_pool_as_bf16_bits(pool: np.ndarray) -> np.ndarray:
+    """The pool's values (unit scale) as bf16 bit patterns: every finite E4M3 value is a bf16 value, so this is exact.
+    NaN codes become bf16 NaN."""
+    v = e4m3_decode(pool).astype(np.float32)
+    return (v.view(np.uint32) >> 16).astype(np.uint16)
+
+
+def decode_attn_fp8(k_pool, v_pool, page_table, seq_lens, q, sm_scale, k_scale, v_scale, traj_ids=None):
+    """Decode attention over fp8 pools: keys are k_scale * code value, values v_scale * code value, so the result is
+    v_scale * attention(sm_scale * k_scale; code values)."""
+    out, lse = decode_attn(fp8_pool_as_bf16_bits(k_pool), fp8_pool_as_bf16_bits(v_pool), page_table, seq_lens, q,
+                           float(np.float32(sm_scale) * np.float32(k_scale)), traj_ids=traj_ids)
+    return out * float(np.float32(v_scale)), lse

@@ -31,6 +31,13 @@
  *            M = max_s lse_s; a_s = exp(lse_s - M); out = sum a_s out_s / sum a_s;
  *            lse = M + ln sum a_s.
  *
+ *   e4m3   : the 8-bit floating-point code of an fp8 KV pool (OCP 8-bit floating point specification, E4M3:
+ *            1 sign, 4 exponent bits with bias 7, 3 mantissa bits; exponent field 0 holds the subnormals
+ *            m/8 * 2^-6; there are no infinities and S.1111.111 is NaN, so the largest finite value is
+ *            1.75 * 2^8 = 448).  encode rounds a float to the nearest code, ties to the even code, and
+ *            saturates to +-448; decode returns the code's value.  A quantised append is encode applied
+ *            to (row element * 1/scale), the product taken in fp32, followed by the plain bit-copy append.
+ *
  * Everything floating point is fp64; bf16 inputs convert exactly.  No blocking,
  * no online softmax, no reordering: two passes over the keys, in index order.
  * Parity status: every function here is pinned by tests/test_oracle_pins.py
@@ -268,5 +275,46 @@ int oracle_lse_combine(int32_t n_parts, int32_t D, const double *parts_out, cons
     }
     for (int32_t d = 0; d < D; ++d) out[d] /= A;
     *lse = M + log(A);
+    return ORACLE_OK;
+}
+
+/* E4M3 decode: value of each code as a double (NaN for 0x7f / 0xff). */
+int oracle_e4m3_decode(const uint8_t *codes, int64_t n, double *out) {
+    for (int64_t i = 0; i < n; ++i) {
+        const int c = codes[i];
+        const int e = (c >> 3) & 15, m = c & 7;
+        double v;
+        if (e == 15 && m == 7) v = NAN;
+        else if (e == 0) v = ldexp((double)m / 8.0, -6);
+        else v = ldexp(1.0 + (double)m / 8.0, e - 7);
+        out[i] = (c & 0x80) ? -v : v;
+    }
+    return ORACLE_OK;
+}
+
+/* E4M3 encode: nearest code, ties to even, magnitudes of 448 and above (and infinities) give +-448, NaN gives 0x7f. */
+int oracle_e4m3_encode(const float *x, int64_t n, uint8_t *codes) {
+    for (int64_t i = 0; i < n; ++i) {
+        const float f = x[i];
+        if (isnan(f)) { codes[i] = 0x7f; continue; }
+        const uint8_t sign = signbit(f) ? 0x80 : 0x00;
+        const double a = fabs((double)f);
+        uint8_t mag;
+        if (a >= 448.0) {
+            mag = 0x7e;
+        } else if (a < ldexp(1.0, -6)) {
+            /* subnormal range: multiples of 2^-9; 8 of them is the smallest normal, code 0x08 */
+            mag = (uint8_t)nearbyint(ldexp(a, 9));
+        } else {
+            int e;
+            const double fr = frexp(a, &e);          /* a = fr * 2^e, fr in [0.5, 1) */
+            int ex = e - 1;                           /* a = (2 fr) * 2^ex, 2 fr in [1, 2) */
+            int m = (int)nearbyint((2.0 * fr - 1.0) * 8.0);
+            if (m == 8) { m = 0; ex += 1; }
+            const int code = ((ex + 7) << 3) | m;
+            mag = code > 0x7e ? 0x7e : (uint8_t)code;
+        }
+        codes[i] = sign | mag;
+    }
     return ORACLE_OK;
 }

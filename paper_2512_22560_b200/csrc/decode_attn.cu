@@ -42,6 +42,8 @@ constexpr int kConsumerWarps = 8;         // two groups of four
 constexpr int kProducerWarp = kConsumerWarps;        // warp 8 issues the copies
 constexpr int kEpilogueWarp = kConsumerWarps + 1;    // warp 9 writes pieces out and combines splits
 constexpr int kThreads = (kConsumerWarps + 2) * 32;
+constexpr int kProducerWarpV = kConsumerWarps + 2;   // fp8 only: warp 10 issues the V copies (warp 8 the K copies)
+constexpr int kThreadsFp8 = kThreads + 32;
 constexpr int kMaxItems = 512;            // items per launch (prefix table lives in shared memory)
 constexpr int kTensorBytes = kTile * kRowBytes;      // 16 KB of K (or V) per stage
 constexpr int kStageBytes = 2 * kTensorBytes;
@@ -64,7 +66,8 @@ constexpr int kOffLens = kOffMl + 2 * kMlFloats * 4;
 constexpr int kOffPrefix = kOffLens + kMaxItems * 4;
 constexpr int kOffTraj = kOffPrefix + (kMaxItems + 32) * 4;   // trajectory of every item (read once from global memory)
 constexpr int kOffBars = kOffTraj + kMaxItems * 4;
-constexpr int kNumBars = 2 * kStages + 8;
+constexpr int kStagesFp8 = 2 * kStages;           // an fp8 tile is half the bytes: twice the stages in the same memory
+constexpr int kNumBars = 2 * kStagesFp8 + 8;
 constexpr int kOffAbort = kOffBars + kNumBars * 8;
 constexpr int kSmemBytes = kOffAbort + 16 + 1024;    // + slack for the 1024-byte alignment
 static_assert(kSmemBytes <= 227 * 1024, "the block must fit the shared memory of an SM");
@@ -79,7 +82,8 @@ struct DecodeParams {
     const __nv_bfloat16 *q;
     __nv_bfloat16 *out;
     float *lse;
-    float scale_log2;
+    float scale_log2;           // sm_scale * log2(e) (times the K scale of an fp8 pool)
+    float out_scale;            // 1, or the V scale of an fp8 pool: applied where a result is normalised
     int *tickets;               // per (item, kv head): pieces that have arrived; 0 between calls
     // fused append (all NULL for a plain decode call): the item's new K/V row is stored at position len and attended to
     const __nv_bfloat16 *k_new, *v_new;   // [n_items][num_kv_heads][128]
@@ -169,6 +173,32 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t *>(&v);
 }
+__device__ __forceinline__ void mma_f16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_f16(float lo, float hi) {
+    uint32_t d;
+    asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+    return d;
+}
+// two bf16 (one 32-bit word) -> two f16
+__device__ __forceinline__ uint32_t bf16x2_to_f16x2(uint32_t w) {
+    return pack_f16(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
+}
+// the two E4M3 bytes in the low (high) half of w -> two f16, low byte first
+__device__ __forceinline__ uint32_t e4m3x2_to_f16x2_lo(uint32_t w) {
+    uint32_t d;
+    asm("{\n\t.reg .b16 lo, hi;\n\tmov.b32 {lo, hi}, %1;\n\tcvt.rn.f16x2.e4m3x2 %0, lo;\n\t}" : "=r"(d) : "r"(w));
+    return d;
+}
+__device__ __forceinline__ uint32_t e4m3x2_to_f16x2_hi(uint32_t w) {
+    uint32_t d;
+    asm("{\n\t.reg .b16 lo, hi;\n\tmov.b32 {lo, hi}, %1;\n\tcvt.rn.f16x2.e4m3x2 %0, hi;\n\t}" : "=r"(d) : "r"(w));
+    return d;
+}
 // four consecutive result values of one row, at element index idx of the output
 __device__ __forceinline__ void store_out4(const DecodeParams &prm, long long idx, float a, float b, float c, float d) {
     if (prm.out_f32 != nullptr) {
@@ -194,6 +224,21 @@ __device__ __forceinline__ void merge_slice(const float (&a)[4], const float (&b
     }
     *reinterpret_cast<float2 *>(row0) = a0; *reinterpret_cast<float2 *>(row1) = a1;
     *reinterpret_cast<float2 *>(row0 + 8) = b0; *reinterpret_cast<float2 *>(row1 + 8) = b1;
+}
+
+// The same for the fp8 path, whose two accumulator tiles of a 16-dim slice hold, per row, dims 4t, 4t+2 (a) and
+// 4t+1, 4t+3 (b) of the slice (t = lane & 3): four consecutive values per row.
+__device__ __forceinline__ void merge_slice_fp8(const float (&a)[4], const float (&b)[4], float f0, float f1, float *row0,
+                                                float *row1, bool add) {
+    float4 x0 = make_float4(a[0] * f0, b[0] * f0, a[1] * f0, b[1] * f0);
+    float4 x1 = make_float4(a[2] * f1, b[2] * f1, a[3] * f1, b[3] * f1);
+    if (add) {
+        const float4 y0 = *reinterpret_cast<float4 *>(row0), y1 = *reinterpret_cast<float4 *>(row1);
+        x0.x += y0.x; x0.y += y0.y; x0.z += y0.z; x0.w += y0.w;
+        x1.x += y1.x; x1.y += y1.y; x1.z += y1.z; x1.w += y1.w;
+    }
+    *reinterpret_cast<float4 *>(row0) = x0;
+    *reinterpret_cast<float4 *>(row1) = x1;
 }
 
 // ------------------------------------------------------------------------------------------
@@ -233,9 +278,17 @@ __device__ __forceinline__ Piece piece_at(const int *prefix, const int *lens, in
 // ------------------------------------------------------------------------------------------
 // Kernel
 // ------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(kThreads, 1)
+// kFp8: the pools hold E4M3 bytes (rows of 128 B) instead of bf16 (rows of 256 B).  The schedule, the pieces, the merge
+// and the combine are the same; the tiles are half the bytes (twice the stages), K and V are converted to f16 as the
+// fragments are loaded and the products run as f16 MMAs (the query is converted once per piece).
+template <bool kFp8>
+__global__ void __launch_bounds__(kFp8 ? kThreadsFp8 : kThreads, 1)
 decode_splitkv_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__ CUtensorMap vmap,
                       const DecodeParams prm) {
+    constexpr int kS = kFp8 ? kStagesFp8 : kStages;                 // stages of the ring
+    constexpr int kSB = kFp8 ? kStageBytes / 2 : kStageBytes;       // bytes of a stage: K image then V image
+    constexpr int kTB = kSB / 2;
+    constexpr int kT = kFp8 ? kThreadsFp8 : kThreads;               // threads of the block
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     int *s_lens = reinterpret_cast<int *>(smem + kOffLens);
@@ -246,11 +299,11 @@ decode_splitkv_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
     volatile int *s_abort = reinterpret_cast<volatile int *>(smem + kOffAbort);
     const uint32_t bars = smem_u32(smem + kOffBars);
     auto bar_full = [&](int s) { return bars + 8u * s; };
-    auto bar_empty = [&](int s) { return bars + 8u * (kStages + s); };
-    auto bar_qfull = [&](int s) { return bars + 8u * (2 * kStages + s); };
-    auto bar_qempty = [&](int s) { return bars + 8u * (2 * kStages + 2 + s); };
-    auto bar_epfull = [&](int s) { return bars + 8u * (2 * kStages + 4 + s); };
-    auto bar_epempty = [&](int s) { return bars + 8u * (2 * kStages + 6 + s); };
+    auto bar_empty = [&](int s) { return bars + 8u * (kS + s); };
+    auto bar_qfull = [&](int s) { return bars + 8u * (2 * kS + s); };
+    auto bar_qempty = [&](int s) { return bars + 8u * (2 * kS + 2 + s); };
+    auto bar_epfull = [&](int s) { return bars + 8u * (2 * kS + 4 + s); };
+    auto bar_epempty = [&](int s) { return bars + 8u * (2 * kS + 6 + s); };
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int hkv = prm.num_kv_heads, P = prm.page_size, g = prm.group;
@@ -260,10 +313,10 @@ decode_splitkv_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
     // for the earlier kernel's results (lengths, pages, tickets) to be complete and visible.
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     // zero both Q buffers once: rows >= g are never written by the copies and must read as 0
-    for (int i = threadIdx.x; i < 2 * kQBytes / 16; i += kThreads)
+    for (int i = threadIdx.x; i < 2 * kQBytes / 16; i += kT)
         reinterpret_cast<uint4 *>(smem + kOffQ)[i] = make_uint4(0, 0, 0, 0);
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kStages; ++s) { mbar_init(bar_full(s), 1); mbar_init(bar_empty(s), kConsumerWarps / 2); }
+        for (int s = 0; s < kS; ++s) { mbar_init(bar_full(s), kFp8 ? 2 : 1); mbar_init(bar_empty(s), kConsumerWarps / 2); }
         for (int s = 0; s < 2; ++s) { mbar_init(bar_qfull(s), 1); mbar_init(bar_qempty(s), kConsumerWarps); }
         for (int s = 0; s < 2; ++s) { mbar_init(bar_epfull(s), 1); mbar_init(bar_epempty(s), 1); }
         *s_abort = 0;
@@ -272,7 +325,7 @@ decode_splitkv_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
     asm volatile("griddepcontrol.wait;" ::: "memory");
 
     // ---- lengths -> tiles per item -> exclusive prefix (shared memory) ----
-    for (int i = threadIdx.x; i < prm.n_items; i += kThreads) {
+    for (int i = threadIdx.x; i < prm.n_items; i += kT) {
         const int t = prm.traj_ids ? __ldg(prm.traj_ids + i) : i + prm.item_offset;
         s_traj[i] = t;
         int L = 0;
@@ -320,13 +373,13 @@ decode_splitkv_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
             if (s_lens[i] != 0) continue;
             if (prm.out_f32 != nullptr) {
                 float4 *o = reinterpret_cast<float4 *>(prm.out_f32 + static_cast<long long>(i) * prm.num_q_heads * kHeadDim);
-                for (int k = threadIdx.x; k < prm.num_q_heads * kHeadDim / 4; k += kThreads) o[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+                for (int k = threadIdx.x; k < prm.num_q_heads * kHeadDim / 4; k += kT) o[k] = make_float4(0.f, 0.f, 0.f, 0.f);
             } else {
                 uint4 *o = reinterpret_cast<uint4 *>(prm.out + static_cast<long long>(i) * prm.num_q_heads * kHeadDim);
-                for (int k = threadIdx.x; k < prm.num_q_heads * kHeadDim / 8; k += kThreads) o[k] = make_uint4(0, 0, 0, 0);
+                for (int k = threadIdx.x; k < prm.num_q_heads * kHeadDim / 8; k += kT) o[k] = make_uint4(0, 0, 0, 0);
             }
             if (prm.lse != nullptr)
-                for (int k = threadIdx.x; k < prm.num_q_heads; k += kThreads)
+                for (int k = threadIdx.x; k < prm.num_q_heads; k += kT)
                     prm.lse[static_cast<long long>(i) * prm.num_q_heads + k] = -INFINITY;
         }
     }
@@ -336,11 +389,15 @@ decode_splitkv_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
     const int p_end = min(total, p_begin + span);
     if (p_begin >= p_end) return;
 
-    if (warp == kProducerWarp) {
-        // =============================== producer warp ===============================
+    if (warp == kProducerWarp || (kFp8 && warp == kProducerWarpV)) {
+        // =============================== producer warp(s) ===============================
+        // bf16: one warp brings K and V.  fp8: a tile is half the bytes, so twice as many copies per second are due and
+        // one warp cannot issue them (a thread is held some 80 cycles by each): warp 8 brings K (and Q), warp 10 brings
+        // V, each with its own arrival on the stage's barrier.
+        const bool do_k = !kFp8 || warp == kProducerWarp, do_v = !kFp8 || warp == kProducerWarpV;
         const int pages_per_tile = kTile / P;
         const int tiles_per_batch = 32 / pages_per_tile;
-        const uint32_t page_bytes = static_cast<uint32_t>(P) * kRowBytes;
+        const uint32_t page_bytes = static_cast<uint32_t>(P) * (kFp8 ? kHeadDim : kRowBytes);   // one (page, head) image of K or V
         int n = 0, pcount = 0;
         for (int p = p_begin; p < p_end;) {
             const Piece pc = piece_at(s_prefix, s_lens, prm.n_items, hkv, p, p_end);
@@ -351,8 +408,8 @@ decode_splitkv_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
                                        (prm.page_offset ? __ldg(prm.page_offset + pc.item) : 0);
             // Q rows of this (item, kv head): g contiguous rows of 256 B
             const int qs = pcount & 1;
-            mbar_wait(bar_qempty(qs), ((pcount >> 1) & 1) ^ 1, s_abort, prm.status, 1);
-            if (lane == 0 && !*s_abort) {
+            if (do_k) mbar_wait(bar_qempty(qs), ((pcount >> 1) & 1) ^ 1, s_abort, prm.status, 1);
+            if (do_k && lane == 0 && !*s_abort) {
                 mbar_arrive_expect_tx(bar_qfull(qs), static_cast<uint32_t>(g) * kRowBytes);
                 bulk_load(smem_u32(smem + kOffQ + qs * kQBytes),
                           prm.q + (static_cast<long long>(pc.item) * prm.num_q_heads + pc.head * g) * kHeadDim,
@@ -371,21 +428,25 @@ decode_splitkv_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
             };
             int ids_cur = load_ids(pc.tile0), ids_next = load_ids(pc.tile0 + tiles_per_batch);
             for (int tile = pc.tile0; tile < pc.tile1; ++tile, ++n) {
-                const int stage = n % kStages;
+                const int stage = n % kS;
                 const int within = (tile - pc.tile0) % tiles_per_batch;
                 if (tile > pc.tile0 && within == 0) { ids_cur = ids_next; ids_next = load_ids(tile + tiles_per_batch); }
                 int pg = __shfl_sync(0xffffffffu, ids_cur, (within * pages_per_tile + lane) & 31);
                 if (lane >= pages_per_tile) pg = -1;
                 const uint32_t nvalid = __popc(__ballot_sync(0xffffffffu, pg >= 0));
-                mbar_wait(bar_empty(stage), ((n / kStages) & 1) ^ 1, s_abort, prm.status, 2);
+                mbar_wait(bar_empty(stage), ((n / kS) & 1) ^ 1, s_abort, prm.status, 2);
                 if (*s_abort) continue;
-                if (lane == 0) mbar_arrive_expect_tx(bar_full(stage), nvalid * 2u * page_bytes);
+                if (lane == 0) mbar_arrive_expect_tx(bar_full(stage), nvalid * (kFp8 ? 1u : 2u) * page_bytes);
                 __syncwarp();
                 if (pg >= 0) {
-                    const uint32_t kdst = smem_u32(smem + kOffStages + stage * kStageBytes) + lane * page_bytes;
-                    const uint32_t vdst = kdst + kTensorBytes;
+                    const uint32_t kdst = smem_u32(smem + kOffStages + stage * kSB) + lane * page_bytes;
+                    const uint32_t vdst = kdst + kTB;
                     const int unit = pg * hkv + pc.head;          // (page, head) tile index
-                    if (prm.four_d) {
+                    if constexpr (kFp8) {
+                        // rows of 128 B: one box per (page, head), landing as [slot][128 B]
+                        if (do_k) tma_load_2d(kdst, &kmap, bar_full(stage), 0, unit * P);
+                        else tma_load_2d(vdst, &vmap, bar_full(stage), 0, unit * P);
+                    } else if (prm.four_d) {
                         tma_load_4d(kdst, &kmap, bar_full(stage), 0, 0, 0, unit);
                         tma_load_4d(vdst, &vmap, bar_full(stage), 0, 0, 0, unit);
                     } else {
@@ -402,10 +463,10 @@ decode_splitkv_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
         // every copy this warp issued has been waited for by the consumers unless the block gave up;
         // in that case wait (bounded) for the copies still in flight before the block exits
         if (*s_abort && lane == 0) {
-            for (int k = 0; k < kStages && k < n; ++k) {
+            for (int k = 0; k < kS && k < n; ++k) {
                 const int m = n - 1 - k;
                 for (uint32_t it = 0; it < kSpinLimit; ++it)
-                    if (mbar_try_wait(bar_full(m % kStages), (m / kStages) & 1)) break;
+                    if (mbar_try_wait(bar_full(m % kS), (m / kS) & 1)) break;
             }
         }
         return;
@@ -442,7 +503,7 @@ decode_splitkv_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
             if (whole) {
                 for (int row = 0; row < g; ++row) {
                     const float lsum = __shfl_sync(0xffffffffu, lrow, row);
-                    const float inv = lsum > 0.f ? 1.f / lsum : 0.f;
+                    const float inv = lsum > 0.f ? prm.out_scale / lsum : 0.f;
                     const float4 x = *reinterpret_cast<const float4 *>(mg + row * kMergeStride + lane * 4);
                     store_out4(prm, obase + row * kHeadDim, x.x * inv, x.y * inv, x.z * inv, x.w * inv);
                 }
@@ -509,7 +570,7 @@ decode_splitkv_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
                     for (int r = 0; r < kMaxGroup; ++r) {
                         const float lsum = __shfl_sync(0xffffffffu, lall, r);
                         if (r < g) {
-                            const float inv = lsum > 0.f ? 1.f / lsum : 0.f;
+                            const float inv = lsum > 0.f ? prm.out_scale / lsum : 0.f;
                             store_out4(prm, obase + r * kHeadDim, acc[r][0] * inv, acc[r][1] * inv, acc[r][2] * inv, acc[r][3] * inv);
                         }
                     }
@@ -529,7 +590,9 @@ decode_splitkv_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
     const int qrow = lane >> 2, qcol = lane & 3;          // fragment row / column-pair of this lane
     // byte offset of this warp's 16 keys inside a K (or V) stage image, and ldmatrix lane offsets
     const int key0 = wq * 16;
-    const uint32_t warp_off = static_cast<uint32_t>((key0 / P) * P * kRowBytes + (key0 % P) * 128);
+    // (fp8: the rows of a tile are 128 B and lie one after the other)
+    const uint32_t warp_off = kFp8 ? static_cast<uint32_t>(key0 * 128)
+                                   : static_cast<uint32_t>((key0 / P) * P * kRowBytes + (key0 % P) * 128);
     const uint32_t half_off = static_cast<uint32_t>(P) * 128;      // second 64 dims of a page image
     const int lm = lane >> 3, lr = lane & 7;
     // K: matrices (keys 0-7 | 8-15) x (dim chunk even | odd)
@@ -547,7 +610,18 @@ decode_splitkv_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
         const int qs = pcount & 1;
         mbar_wait(bar_qfull(qs), (pcount >> 1) & 1, s_abort, prm.status, 3);
         uint32_t qa[8][4];
-        {
+        if constexpr (kFp8) {
+            // The 16 dims of a step reach the K fragments four bytes per lane (dims 4t .. 4t+3 for t = lane & 3): the
+            // step's contraction slots 2t, 2t+1, 2t+8, 2t+9 are those four dims, in the query fragments as well.
+            const uint8_t *qrow0 = smem + kOffQ + qs * kQBytes + qrow * kRowBytes + qcol * 8;
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks) {
+                const uint2 lo = *reinterpret_cast<const uint2 *>(qrow0 + ks * 32);
+                const uint2 hi = *reinterpret_cast<const uint2 *>(qrow0 + 8 * kRowBytes + ks * 32);
+                qa[ks][0] = bf16x2_to_f16x2(lo.x); qa[ks][1] = bf16x2_to_f16x2(hi.x);
+                qa[ks][2] = bf16x2_to_f16x2(lo.y); qa[ks][3] = bf16x2_to_f16x2(hi.y);
+            }
+        } else {
             const uint32_t qbase = smem_u32(smem + kOffQ + qs * kQBytes) + ((lm & 1) * 8 + lr) * kRowBytes + (lm >> 1) * 16;
 #pragma unroll
             for (int ks = 0; ks < 8; ++ks) ldmatrix_x4(qa[ks][0], qa[ks][1], qa[ks][2], qa[ks][3], qbase + ks * 32);
@@ -562,13 +636,13 @@ decode_splitkv_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
 
         for (int tile = pc.tile0; tile < pc.tile1; ++tile, ++n) {
             if ((n & 1) != grp) continue;
-            const int stage = n % kStages;
-            mbar_wait(bar_full(stage), (n / kStages) & 1, s_abort, prm.status, 4);
-            const uint32_t kbase = smem_u32(smem + kOffStages + stage * kStageBytes) + warp_off;
-            const uint32_t vbase = kbase + kTensorBytes;
+            const int stage = n % kS;
+            mbar_wait(bar_full(stage), (n / kS) & 1, s_abort, prm.status, 4);
+            const uint32_t kbase = smem_u32(smem + kOffStages + stage * kSB) + warp_off;
+            const uint32_t vbase = kbase + kTB;
             const int valid = min(16, pc.len - tile * kTile - key0);   // live keys among this warp's 16
             bool patched = false;
-            if (prm.k_new != nullptr && tile == pc.ntiles - 1 && valid > 0 && valid <= 16 &&
+            if (!kFp8 && prm.k_new != nullptr && tile == pc.ntiles - 1 && valid > 0 && valid <= 16 &&
                 pc.len - 1 - tile * kTile - key0 == valid - 1) {
                 // Fused append: this warp owns the context's last key, which is the item's new token.  Its K/V row
                 // comes from k_new / v_new: put it into the staged tile (over whatever the copy brought for that
@@ -591,9 +665,10 @@ decode_splitkv_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
             if (valid > 0) {
                 if (valid < 16) {
                     // dead slots may hold anything (NaN included): zero their V rows so that 0 * v stays 0
-                    for (int idx = lane; idx < (16 - valid) * 16; idx += 32) {
-                        const int r = valid + (idx >> 4), c = idx & 15;
-                        const uint32_t a = vbase + (c >> 3) * half_off + r * 128 + (c & 7) * 16;
+                    constexpr int kVecPerKey = kFp8 ? 8 : 16;       // 16-byte pieces of a V row
+                    for (int idx = lane; idx < (16 - valid) * kVecPerKey; idx += 32) {
+                        const int r = valid + idx / kVecPerKey, c = idx % kVecPerKey;
+                        const uint32_t a = kFp8 ? vbase + r * 128 + c * 16 : vbase + (c >> 3) * half_off + r * 128 + (c & 7) * 16;
                         asm volatile("st.shared.v4.b32 [%0], {%1,%1,%1,%1};" ::"r"(a), "r"(0) : "memory");
                     }
                     __syncwarp();
@@ -601,13 +676,28 @@ decode_splitkv_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
                 float s[2][4];
 #pragma unroll
                 for (int nt = 0; nt < 2; ++nt) s[nt][0] = s[nt][1] = s[nt][2] = s[nt][3] = 0.f;
+                if constexpr (kFp8) {
+                    // one load brings keys 0-7 and 8-15 for two 16-dim chunks (a row of 128 B holds 8 chunks of 16 B);
+                    // each 32-bit register is the lane's four dims of a key: its halves are the two B registers
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks) {
-                    const int chunk = ks * 2 + k_chunk_lo;
-                    uint32_t b0, b1, b2, b3;
-                    ldmatrix_x4(b0, b1, b2, b3, kbase + (chunk >> 3) * half_off + k_lane_off + (((chunk & 7) ^ lr) << 4));
-                    mma_bf16(s[0], qa[ks], b0, b1);
-                    mma_bf16(s[1], qa[ks], b2, b3);
+                    for (int cp = 0; cp < 4; ++cp) {
+                        const int chunk = cp * 2 + (lm >> 1);
+                        uint32_t r0, r1, r2, r3;
+                        ldmatrix_x4(r0, r1, r2, r3, kbase + ((lm & 1) * 8 + lr) * 128 + ((chunk ^ lr) << 4));
+                        mma_f16(s[0], qa[2 * cp], e4m3x2_to_f16x2_lo(r0), e4m3x2_to_f16x2_hi(r0));
+                        mma_f16(s[1], qa[2 * cp], e4m3x2_to_f16x2_lo(r1), e4m3x2_to_f16x2_hi(r1));
+                        mma_f16(s[0], qa[2 * cp + 1], e4m3x2_to_f16x2_lo(r2), e4m3x2_to_f16x2_hi(r2));
+                        mma_f16(s[1], qa[2 * cp + 1], e4m3x2_to_f16x2_lo(r3), e4m3x2_to_f16x2_hi(r3));
+                    }
+                } else {
+#pragma unroll
+                    for (int ks = 0; ks < 8; ++ks) {
+                        const int chunk = ks * 2 + k_chunk_lo;
+                        uint32_t b0, b1, b2, b3;
+                        ldmatrix_x4(b0, b1, b2, b3, kbase + (chunk >> 3) * half_off + k_lane_off + (((chunk & 7) ^ lr) << 4));
+                        mma_bf16(s[0], qa[ks], b0, b1);
+                        mma_bf16(s[1], qa[ks], b2, b3);
+                    }
                 }
 #pragma unroll
                 for (int nt = 0; nt < 2; ++nt)
@@ -638,16 +728,40 @@ decode_splitkv_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
                     const float p12 = exp2f(s[1][2] - m1), p13 = exp2f(s[1][3] - m1);
                     l0 += (p00 + p01) + (p10 + p11);
                     l1 += (p02 + p03) + (p12 + p13);
-                    pa[0] = pack_bf16(p00, p01); pa[1] = pack_bf16(p02, p03);
-                    pa[2] = pack_bf16(p10, p11); pa[3] = pack_bf16(p12, p13);
+                    if constexpr (kFp8) {
+                        pa[0] = pack_f16(p00, p01); pa[1] = pack_f16(p02, p03);
+                        pa[2] = pack_f16(p10, p11); pa[3] = pack_f16(p12, p13);
+                    } else {
+                        pa[0] = pack_bf16(p00, p01); pa[1] = pack_bf16(p02, p03);
+                        pa[2] = pack_bf16(p10, p11); pa[3] = pack_bf16(p12, p13);
+                    }
                 }
+                if constexpr (kFp8) {
+                    // the transposed load hands a lane, for keys 2t and 2t+1, the two dims 2g, 2g+1 of a chunk
+                    // (g = lane >> 2): bytes are regrouped into (key 2t, key 2t+1) pairs for the even and the odd
+                    // dim, which feed two MMAs; their accumulator columns 2t, 2t+1 are then dims 4t, 4t+2 and
+                    // 4t+1, 4t+3 of the chunk
 #pragma unroll
-                for (int pr = 0; pr < 8; ++pr) {
-                    const int chunk = pr * 2 + v_chunk_lo;
-                    uint32_t b0, b1, b2, b3;
-                    ldmatrix_x4_trans(b0, b1, b2, b3, vbase + (chunk >> 3) * half_off + v_lane_off + (((chunk & 7) ^ lr) << 4));
-                    mma_bf16(o[2 * pr], pa, b0, b1);
-                    mma_bf16(o[2 * pr + 1], pa, b2, b3);
+                    for (int cp = 0; cp < 4; ++cp) {
+                        const int chunk = cp * 2 + (lm >> 1);
+                        uint32_t r0, r1, r2, r3;
+                        ldmatrix_x4_trans(r0, r1, r2, r3, vbase + ((lm & 1) * 8 + lr) * 128 + ((chunk ^ lr) << 4));
+                        const uint32_t x0 = __byte_perm(r0, 0, 0x3120), x1 = __byte_perm(r1, 0, 0x3120);
+                        const uint32_t x2 = __byte_perm(r2, 0, 0x3120), x3 = __byte_perm(r3, 0, 0x3120);
+                        mma_f16(o[4 * cp], pa, e4m3x2_to_f16x2_lo(x0), e4m3x2_to_f16x2_lo(x1));
+                        mma_f16(o[4 * cp + 1], pa, e4m3x2_to_f16x2_hi(x0), e4m3x2_to_f16x2_hi(x1));
+                        mma_f16(o[4 * cp + 2], pa, e4m3x2_to_f16x2_lo(x2), e4m3x2_to_f16x2_lo(x3));
+                        mma_f16(o[4 * cp + 3], pa, e4m3x2_to_f16x2_hi(x2), e4m3x2_to_f16x2_hi(x3));
+                    }
+                } else {
+#pragma unroll
+                    for (int pr = 0; pr < 8; ++pr) {
+                        const int chunk = pr * 2 + v_chunk_lo;
+                        uint32_t b0, b1, b2, b3;
+                        ldmatrix_x4_trans(b0, b1, b2, b3, vbase + (chunk >> 3) * half_off + v_lane_off + (((chunk & 7) ^ lr) << 4));
+                        mma_bf16(o[2 * pr], pa, b0, b1);
+                        mma_bf16(o[2 * pr + 1], pa, b2, b3);
+                    }
                 }
                 if (valid < 16 || patched) fence_proxy_async();   // our stores into the stage precede the next copy into it
             }
@@ -680,8 +794,20 @@ decode_splitkv_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
             // in round r this warp handles the 16-dim column slice (warp + r) mod 8, so all warps work in
             // every round and each slice receives the warps in a fixed order
             const int c = (warp + r) & 7;
-            float *row0 = mrg + qrow * kMergeStride + c * 16 + qcol * 2;
+            float *row0 = mrg + qrow * kMergeStride + c * 16 + qcol * (kFp8 ? 4 : 2);
             float *row1 = row0 + 8 * kMergeStride;
+            if constexpr (kFp8) {
+                switch (c) {
+                    case 0: merge_slice_fp8(o[0], o[1], f0, f1, row0, row1, r > 0); break;
+                    case 1: merge_slice_fp8(o[2], o[3], f0, f1, row0, row1, r > 0); break;
+                    case 2: merge_slice_fp8(o[4], o[5], f0, f1, row0, row1, r > 0); break;
+                    case 3: merge_slice_fp8(o[6], o[7], f0, f1, row0, row1, r > 0); break;
+                    case 4: merge_slice_fp8(o[8], o[9], f0, f1, row0, row1, r > 0); break;
+                    case 5: merge_slice_fp8(o[10], o[11], f0, f1, row0, row1, r > 0); break;
+                    case 6: merge_slice_fp8(o[12], o[13], f0, f1, row0, row1, r > 0); break;
+                    default: merge_slice_fp8(o[14], o[15], f0, f1, row0, row1, r > 0); break;
+                }
+            } else
             switch (c) {
                 case 0: merge_slice(o[0], o[1], f0, f1, row0, row1, r > 0); break;
                 case 1: merge_slice(o[2], o[3], f0, f1, row0, row1, r > 0); break;
@@ -744,6 +870,19 @@ bool encode_pool_map(CUtensorMap *map, const void *pool, int num_pages, int hkv,
     return r == CUDA_SUCCESS;
 }
 
+// fp8 pool as [rows = pages * heads * slots][128 B]; one box = one (page, head) image of P rows
+bool encode_pool_map_fp8(CUtensorMap *map, const void *pool, int num_pages, int hkv, int P) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {kHeadDim, static_cast<cuuint64_t>(num_pages) * hkv * P};
+    const cuuint64_t strides[1] = {kHeadDim};
+    const cuuint32_t box[2] = {kHeadDim, static_cast<cuuint32_t>(P)};
+    const cuuint32_t ones[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void *>(pool), dims, strides, box, ones,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 size_t info_bytes(int items, int hkv) { return (static_cast<size_t>(items) * hkv * sizeof(int2) + 255) & ~size_t(255); }
 
 }  // namespace
@@ -773,21 +912,30 @@ cudaError_t launch_decode_attn(const AttnCall &c, cudaStream_t stream, int64_t *
     int per_launch = chunk_items;
     while (per_launch > 1 && tiles_bound * per_launch > 0x3FFFFFFFLL) per_launch /= 2;
 
-    cudaError_t e = cudaFuncSetAttribute(decode_splitkv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    cudaError_t e = cudaFuncSetAttribute(c.fp8 ? decode_splitkv_kernel<true> : decode_splitkv_kernel<false>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (e != cudaSuccess) return e;
     if (c.tma == nullptr) return cudaErrorInvalidValue;
     TmaCache &tc = *c.tma;
     if (!tc.valid || tc.k != c.pool.k || tc.v != c.pool.v || tc.num_pages != c.pool.num_pages || tc.hkv != hkv ||
-        tc.page_size != c.pool.page_size) {
+        tc.page_size != c.pool.page_size || tc.fp8 != (c.fp8 ? 1 : 0)) {
         CUtensorMap *km = reinterpret_cast<CUtensorMap *>(tc.kmap), *vm = reinterpret_cast<CUtensorMap *>(tc.vmap);
-        bool four = encode_pool_map(km, c.pool.k, c.pool.num_pages, hkv, c.pool.page_size, true) &&
-                    encode_pool_map(vm, c.pool.v, c.pool.num_pages, hkv, c.pool.page_size, true);
-        if (!four) {
+        bool four = false;
+        if (c.fp8) {
+            if (!encode_pool_map_fp8(km, c.pool.k, c.pool.num_pages, hkv, c.pool.page_size) ||
+                !encode_pool_map_fp8(vm, c.pool.v, c.pool.num_pages, hkv, c.pool.page_size))
+                return cudaErrorInvalidValue;
+        } else {
+            four = encode_pool_map(km, c.pool.k, c.pool.num_pages, hkv, c.pool.page_size, true) &&
+                   encode_pool_map(vm, c.pool.v, c.pool.num_pages, hkv, c.pool.page_size, true);
+        }
+        if (!four && !c.fp8) {
             if (!encode_pool_map(km, c.pool.k, c.pool.num_pages, hkv, c.pool.page_size, false) ||
                 !encode_pool_map(vm, c.pool.v, c.pool.num_pages, hkv, c.pool.page_size, false))
                 return cudaErrorInvalidValue;
         }
         tc.four_d = four ? 1 : 0;
+        tc.fp8 = c.fp8 ? 1 : 0;
         tc.k = c.pool.k; tc.v = c.pool.v; tc.num_pages = c.pool.num_pages; tc.hkv = hkv; tc.page_size = c.pool.page_size;
         tc.valid = true;
     }
@@ -805,7 +953,8 @@ cudaError_t launch_decode_attn(const AttnCall &c, cudaStream_t stream, int64_t *
         prm.q = c.q + static_cast<long long>(base) * c.num_q_heads * kHeadDim;
         prm.out = c.out + static_cast<long long>(base) * c.num_q_heads * kHeadDim;
         prm.lse = c.lse ? c.lse + static_cast<long long>(base) * c.num_q_heads : nullptr;
-        prm.scale_log2 = c.sm_scale * kLog2e;
+        prm.scale_log2 = c.sm_scale * kLog2e * (c.fp8 ? c.k_scale : 1.f);
+        prm.out_scale = c.fp8 ? c.v_scale : 1.f;
         prm.tickets = static_cast<int *>(c.workspace);
         prm.k_new = c.k_new ? c.k_new + static_cast<long long>(base) * hkv * kHeadDim : nullptr;
         prm.v_new = c.v_new ? c.v_new + static_cast<long long>(base) * hkv * kHeadDim : nullptr;
@@ -818,13 +967,13 @@ cudaError_t launch_decode_attn(const AttnCall &c, cudaStream_t stream, int64_t *
         // programmatic stream serialisation: back-to-back decode launches overlap this grid's set-up with the
         // previous grid's tail (the kernel waits for that grid before it reads anything)
         cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3(grid); cfg.blockDim = dim3(kThreads); cfg.dynamicSmemBytes = kSmemBytes; cfg.stream = stream;
+        cfg.gridDim = dim3(grid); cfg.blockDim = dim3(c.fp8 ? kThreadsFp8 : kThreads); cfg.dynamicSmemBytes = kSmemBytes; cfg.stream = stream;
         cudaLaunchAttribute attr[1];
         attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
         attr[0].val.programmaticStreamSerializationAllowed = 1;
         cfg.attrs = attr; cfg.numAttrs = 1;
-        e = cudaLaunchKernelEx(&cfg, decode_splitkv_kernel, *reinterpret_cast<CUtensorMap *>(tc.kmap),
-                               *reinterpret_cast<CUtensorMap *>(tc.vmap), prm);
+        e = cudaLaunchKernelEx(&cfg, c.fp8 ? decode_splitkv_kernel<true> : decode_splitkv_kernel<false>,
+                               *reinterpret_cast<CUtensorMap *>(tc.kmap), *reinterpret_cast<CUtensorMap *>(tc.vmap), prm);
         ++*launches;
         if (e != cudaSuccess) return e;
     }
@@ -948,7 +1097,7 @@ extern "C" rollart_status rollart_decode_attn_noalloc(int device, const rollart_
             if (e == cudaSuccess) e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, device);
             if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device);
             if (e == cudaSuccess)
-                e = cudaFuncSetAttribute(decode_splitkv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+                e = cudaFuncSetAttribute(decode_splitkv_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
             if (e != cudaSuccess || ptr == nullptr) {
                 write_err(err_buf, err_len, "set-up on device %d failed: %s", device, cudaGetErrorString(e));
                 result = ROLLART_ERR_CUDA;
@@ -994,13 +1143,14 @@ extern "C" rollart_status rollart_decode_attn_noalloc(int device, const rollart_
         prm.out = static_cast<__nv_bfloat16 *>(out);
         prm.lse = lse;
         prm.scale_log2 = sm_scale * kLog2e;
+        prm.out_scale = 1.f;
         prm.tickets = reinterpret_cast<int *>(su.scratch + kStaticStatusBytes);
         prm.k_new = nullptr; prm.v_new = nullptr; prm.k_pool = nullptr; prm.v_pool = nullptr; prm.seq_lens_out = nullptr;
         prm.page_offset = nullptr; prm.out_f32 = nullptr;
         prm.slots = reinterpret_cast<float *>(su.scratch + kStaticStatusBytes + kStaticInfoBytes);
         prm.status = status;
         const int grid = su.sm_count < kStaticMaxGrid ? su.sm_count : kStaticMaxGrid;
-        decode_splitkv_kernel<<<grid, kThreads, kSmemBytes, s>>>(kmap, vmap, prm);
+        decode_splitkv_kernel<false><<<grid, kThreads, kSmemBytes, s>>>(kmap, vmap, prm);
         e = cudaGetLastError();
         if (e != cudaSuccess) {
             write_err(err_buf, err_len, "kernel launch failed: %s", cudaGetErrorString(e));

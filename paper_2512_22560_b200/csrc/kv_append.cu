@@ -25,8 +25,25 @@ __device__ __forceinline__ int find_item(const int32_t *__restrict__ indptr, int
     return lo;
 }
 
+// eight bf16 (one 16-byte piece of a row) -> eight E4M3 codes: code = nearest (ties to even, saturating at +-448) of
+// x * inv_scale, the product rounded to fp32 first
+__device__ __forceinline__ uint2 quantize8(const uint4 &v, float inv_scale) {
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    uint32_t h[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const float lo = __uint_as_float(w[i] << 16) * inv_scale, hi = __uint_as_float(w[i] & 0xffff0000u) * inv_scale;
+        uint16_t p;
+        asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(p) : "f"(hi), "f"(lo));    // first operand -> upper byte
+        h[i] = p;
+    }
+    return make_uint2(h[0] | (h[1] << 16), h[2] | (h[3] << 16));
+}
+
+// kFp8: the pools hold E4M3 codes (rows of 128 B); the new rows arrive as bf16 and are quantised on the way.
+template <bool kFp8>
 __global__ void __launch_bounds__(kThreads)
-kv_append_kernel(__nv_bfloat16 *__restrict__ k_pool, __nv_bfloat16 *__restrict__ v_pool, int num_pages, int page_size,
+kv_append_kernel(void *__restrict__ k_pool, void *__restrict__ v_pool, float k_inv_scale, float v_inv_scale, int num_pages, int page_size,
                  int num_kv_heads, const int32_t *__restrict__ page_table, int max_pages,
                  const int32_t *__restrict__ seq_lens, int num_traj, const int32_t *__restrict__ traj_ids,
                  const int32_t *__restrict__ new_indptr, int n_items, int total_new,
@@ -70,8 +87,13 @@ kv_append_kernel(__nv_bfloat16 *__restrict__ k_pool, __nv_bfloat16 *__restrict__
     const int slot = static_cast<int>(pos - lp * page_size);
 
     const long long dst = ((static_cast<long long>(pg) * num_kv_heads + h) * page_size + slot) * kVecPerRow + c;
-    reinterpret_cast<uint4 *>(k_pool)[dst] = kv;
-    reinterpret_cast<uint4 *>(v_pool)[dst] = vv;
+    if constexpr (kFp8) {
+        reinterpret_cast<uint2 *>(k_pool)[dst] = quantize8(kv, k_inv_scale);
+        reinterpret_cast<uint2 *>(v_pool)[dst] = quantize8(vv, v_inv_scale);
+    } else {
+        reinterpret_cast<uint4 *>(k_pool)[dst] = kv;
+        reinterpret_cast<uint4 *>(v_pool)[dst] = vv;
+    }
 }
 
 // Gather: thread -> (output row, kv head, 16-byte piece); row r of item i is the token at logical position r.
@@ -122,14 +144,15 @@ cudaError_t launch_kv_gather(const rollart_kv_pool &pool, const rollart_trajs &t
 cudaError_t launch_kv_append(const rollart_kv_pool &pool, const rollart_trajs &trajs, const int32_t *traj_ids,
                              const int32_t *new_indptr, int n_items, int total_new, const void *k_new,
                              const void *v_new, int32_t *seq_lens_out, DeviceStatus *status, cudaStream_t stream,
-                             int64_t *launches) {
+                             int64_t *launches, bool fp8, float k_scale, float v_scale) {
     const long long n_vec = static_cast<long long>(total_new) * pool.num_kv_heads * kVecPerRow;
     const long long n_thr = n_vec > n_items ? n_vec : n_items;
     if (n_thr == 0) return cudaSuccess;
     const long long blocks = (n_thr + kThreads - 1) / kThreads;
     if (blocks > 0x7FFFFFFFLL) return cudaErrorInvalidValue;
-    kv_append_kernel<<<static_cast<unsigned>(blocks), kThreads, 0, stream>>>(
-        static_cast<__nv_bfloat16 *>(pool.k_pool), static_cast<__nv_bfloat16 *>(pool.v_pool), pool.num_pages,
+    auto kernel = fp8 ? kv_append_kernel<true> : kv_append_kernel<false>;
+    kernel<<<static_cast<unsigned>(blocks), kThreads, 0, stream>>>(
+        pool.k_pool, pool.v_pool, fp8 ? 1.f / k_scale : 1.f, fp8 ? 1.f / v_scale : 1.f, pool.num_pages,
         pool.page_size, pool.num_kv_heads, trajs.page_table, trajs.max_pages_per_traj, trajs.seq_lens, trajs.num_traj,
         traj_ids, new_indptr, n_items, total_new, static_cast<const uint4 *>(k_new), static_cast<const uint4 *>(v_new),
         seq_lens_out, status);

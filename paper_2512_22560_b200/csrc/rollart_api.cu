@@ -108,6 +108,9 @@ AttnCall make_call(rollart_ctx *ctx, const rollart_kv_pool *pool, const rollart_
     c.page_offset = nullptr;
     c.shared_lens = nullptr;
     c.out_f32 = nullptr;
+    c.fp8 = false;
+    c.k_scale = 1.f;
+    c.v_scale = 1.f;
     return c;
 }
 
@@ -170,10 +173,11 @@ rollart_status rollart_destroy(rollart_ctx *ctx) {
     return ROLLART_OK;
 }
 
-rollart_status rollart_kv_append(rollart_ctx *ctx, const rollart_kv_pool *pool, const rollart_trajs *trajs,
-                                 const int32_t *traj_ids, const int32_t *new_indptr, int32_t n_items,
-                                 int32_t total_new, const void *k_new, const void *v_new, int32_t *seq_lens_out,
-                                 void *stream) {
+namespace {
+rollart_status append_impl(rollart_ctx *ctx, const rollart_kv_pool *pool, const rollart_trajs *trajs,
+                           const int32_t *traj_ids, const int32_t *new_indptr, int32_t n_items, int32_t total_new,
+                           const void *k_new, const void *v_new, int32_t *seq_lens_out, void *stream, bool fp8,
+                           float k_scale, float v_scale) {
     if (!ctx) return ROLLART_ERR_INVALID_ARG;
     rollart_status st;
     if ((st = check_pool(ctx, pool)) != ROLLART_OK) return st;
@@ -192,9 +196,29 @@ rollart_status rollart_kv_append(rollart_ctx *ctx, const rollart_kv_pool *pool, 
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return fail(ctx, ROLLART_ERR_CUDA, "cannot select device %d", ctx->device);
     cudaError_t e = launch_kv_append(*pool, *trajs, traj_ids, new_indptr, n_items, total_new, k_new, v_new, seq_lens_out,
-                                     ctx->d_status, static_cast<cudaStream_t>(stream), &ctx->launches);
+                                     ctx->d_status, static_cast<cudaStream_t>(stream), &ctx->launches, fp8, k_scale, v_scale);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "kv_append launch");
     return ROLLART_OK;
+}
+}  // namespace
+
+rollart_status rollart_kv_append(rollart_ctx *ctx, const rollart_kv_pool *pool, const rollart_trajs *trajs,
+                                 const int32_t *traj_ids, const int32_t *new_indptr, int32_t n_items,
+                                 int32_t total_new, const void *k_new, const void *v_new, int32_t *seq_lens_out,
+                                 void *stream) {
+    return append_impl(ctx, pool, trajs, traj_ids, new_indptr, n_items, total_new, k_new, v_new, seq_lens_out, stream, false,
+                       1.f, 1.f);
+}
+
+rollart_status rollart_kv_append_fp8(rollart_ctx *ctx, const rollart_kv_pool *pool, const rollart_trajs *trajs,
+                                     const int32_t *traj_ids, const int32_t *new_indptr, int32_t n_items,
+                                     int32_t total_new, const void *k_new, const void *v_new, float k_scale, float v_scale,
+                                     int32_t *seq_lens_out, void *stream) {
+    if (!ctx) return ROLLART_ERR_INVALID_ARG;
+    if (!(k_scale > 0.f) || !(v_scale > 0.f) || !isfinite(k_scale) || !isfinite(v_scale))
+        return fail(ctx, ROLLART_ERR_INVALID_ARG, "k_scale and v_scale must be positive and finite");
+    return append_impl(ctx, pool, trajs, traj_ids, new_indptr, n_items, total_new, k_new, v_new, seq_lens_out, stream, true,
+                       k_scale, v_scale);
 }
 
 rollart_status rollart_kv_gather(rollart_ctx *ctx, const rollart_kv_pool *pool, const rollart_trajs *trajs,
@@ -288,6 +312,33 @@ rollart_status rollart_decode_attn(rollart_ctx *ctx, const rollart_kv_pool *pool
         return fail(ctx, ROLLART_ERR_WORKSPACE, "workspace of %zu bytes is too small (need %zu)", ctx->workspace_bytes,
                     decode_workspace_bytes(n_items, num_q_heads, pool->num_kv_heads, max_seq_len, ctx->sm_count));
     if (e != cudaSuccess) return cuda_fail(ctx, e, "decode_attn launch");
+    return ROLLART_OK;
+}
+
+rollart_status rollart_decode_attn_fp8(rollart_ctx *ctx, const rollart_kv_pool *pool, const rollart_trajs *trajs,
+                                       const int32_t *traj_ids, int32_t n_items, int32_t max_seq_len, const void *q,
+                                       int32_t num_q_heads, float sm_scale, float k_scale, float v_scale, void *out,
+                                       float *lse, void *stream) {
+    if (!ctx) return ROLLART_ERR_INVALID_ARG;
+    rollart_status st = attn_common(ctx, pool, trajs, n_items, n_items, max_seq_len, q, num_q_heads, out);
+    if (st != ROLLART_OK) return st;
+    if (!(k_scale > 0.f) || !(v_scale > 0.f) || !isfinite(k_scale) || !isfinite(v_scale))
+        return fail(ctx, ROLLART_ERR_INVALID_ARG, "k_scale and v_scale must be positive and finite");
+    if (n_items == 0) return ROLLART_OK;
+    max_seq_len = clamp_bound(pool, trajs, max_seq_len);
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return fail(ctx, ROLLART_ERR_CUDA, "cannot select device %d", ctx->device);
+    AttnCall c = make_call(ctx, pool, trajs, traj_ids, nullptr, n_items, n_items, max_seq_len, q, num_q_heads, sm_scale,
+                           out, lse);
+    c.fp8 = true;
+    c.k_scale = k_scale;
+    c.v_scale = v_scale;
+    bool too_small = false;
+    cudaError_t e = launch_decode_attn(c, static_cast<cudaStream_t>(stream), &ctx->launches, &too_small);
+    if (too_small)
+        return fail(ctx, ROLLART_ERR_WORKSPACE, "workspace of %zu bytes is too small (need %zu)", ctx->workspace_bytes,
+                    decode_workspace_bytes(n_items, num_q_heads, pool->num_kv_heads, max_seq_len, ctx->sm_count));
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "decode_attn_fp8 launch");
     return ROLLART_OK;
 }
 

@@ -45,7 +45,7 @@ struct TrajView {
 cudaError_t launch_kv_append(const rollart_kv_pool &pool, const rollart_trajs &trajs, const int32_t *traj_ids,
                              const int32_t *new_indptr, int n_items, int total_new, const void *k_new,
                              const void *v_new, int32_t *seq_lens_out, DeviceStatus *status, cudaStream_t stream,
-                             int64_t *launches);
+                             int64_t *launches, bool fp8 = false, float k_scale = 1.f, float v_scale = 1.f);
 
 cudaError_t launch_kv_gather(const rollart_kv_pool &pool, const rollart_trajs &trajs, const int32_t *traj_ids,
                              const int32_t *out_indptr, int n_items, int total_rows, void *k_out, void *v_out,
@@ -60,7 +60,7 @@ struct TmaCache {
     bool valid;
     const void *k;
     const void *v;
-    int num_pages, hkv, page_size, four_d;
+    int num_pages, hkv, page_size, four_d, fp8;
     alignas(64) unsigned char kmap[128];
     alignas(64) unsigned char vmap[128];
 };
@@ -91,6 +91,9 @@ struct AttnCall {
     const int32_t *page_offset;   // decode: per item, pages of the table row to skip (the keys before them are not attended to)
     const int32_t *shared_lens;   // chunk: per item, every query row of the item sees exactly the first shared_lens[i] keys
     float *out_f32;               // when set the result rows are written here in fp32 instead of bf16 to `out`
+    // fp8 (E4M3) pools, decode only: keys are k_scale * code value, values v_scale * code value
+    bool fp8;
+    float k_scale, v_scale;
 };
 
 size_t decode_workspace_bytes(int max_items, int num_q_heads, int num_kv_heads, int max_seq_len, int sm_count);

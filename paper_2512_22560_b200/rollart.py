@@ -23,6 +23,7 @@ EXPORTS = (
     "rollart_obs_chunk_attn", "rollart_check", "rollart_last_error", "rollart_launch_count",
     "rollart_decode_attn_noalloc", "rollart_kv_gather", "rollart_pages_reserve", "rollart_pages_release",
     "rollart_append_decode_attn", "rollart_group_decode_attn", "rollart_group_decode_workspace_size",
+    "rollart_decode_attn_fp8", "rollart_kv_append_fp8",
 )
 
 
@@ -72,6 +73,12 @@ def load_library() -> ctypes.CDLL:
     L.rollart_decode_attn.restype = ctypes.c_int
     L.rollart_decode_attn.argtypes = [vp, ctypes.POINTER(_KVPool), ctypes.POINTER(_Trajs), vp, i32, i32, vp, i32, f32,
                                       vp, vp, vp]
+    L.rollart_kv_append_fp8.restype = ctypes.c_int
+    L.rollart_kv_append_fp8.argtypes = [vp, ctypes.POINTER(_KVPool), ctypes.POINTER(_Trajs), vp, vp, i32, i32, vp, vp, f32, f32,
+                                        vp, vp]
+    L.rollart_decode_attn_fp8.restype = ctypes.c_int
+    L.rollart_decode_attn_fp8.argtypes = [vp, ctypes.POINTER(_KVPool), ctypes.POINTER(_Trajs), vp, i32, i32, vp, i32, f32,
+                                          f32, f32, vp, vp, vp]
     L.rollart_append_decode_attn.restype = ctypes.c_int
     L.rollart_append_decode_attn.argtypes = [vp, ctypes.POINTER(_KVPool), ctypes.POINTER(_Trajs), vp, i32, i32, vp, vp, vp, i32,
                                              f32, vp, vp, vp, vp]
@@ -193,6 +200,13 @@ class Context:
         n, h, p, d = k_pool.shape
         return _KVPool(_ptr(k_pool, torch.bfloat16, self.device), _ptr(v_pool, torch.bfloat16, self.device), n, p, h, d)
 
+    def _pool_fp8(self, k_pool: torch.Tensor, v_pool: torch.Tensor) -> _KVPool:
+        """fp8 pools travel as uint8 tensors [num_pages][num_kv_heads][page_size][head_dim] of E4M3 codes"""
+        if k_pool.dim() != 4 or k_pool.shape != v_pool.shape:
+            raise ValueError("pools must be [num_pages][num_kv_heads][page_size][head_dim] with equal shapes")
+        n, h, p, d = k_pool.shape
+        return _KVPool(_ptr(k_pool, torch.uint8, self.device), _ptr(v_pool, torch.uint8, self.device), n, p, h, d)
+
     def _trajs(self, page_table: torch.Tensor, seq_lens: torch.Tensor) -> _Trajs:
         if page_table.dim() != 2 or seq_lens.dim() != 1 or page_table.shape[0] != seq_lens.shape[0]:
             raise ValueError("page_table must be [num_traj][max_pages], seq_lens [num_traj]")
@@ -216,6 +230,26 @@ class Context:
             self._h, ctypes.byref(pool), ctypes.byref(trajs), _ptr(traj_ids, torch.int32, self.device),
             _ptr(new_indptr, torch.int32, self.device), n_items, total_new, _ptr(k_new, torch.bfloat16, self.device),
             _ptr(v_new, torch.bfloat16, self.device), _ptr(seq_lens_out, torch.int32, self.device), self._stream(stream))
+        if st != OK:
+            self._raise(st)
+
+    def kv_append_fp8(self, k_pool, v_pool, page_table, seq_lens, new_indptr, k_new, v_new, k_scale, v_scale,
+                      traj_ids=None, seq_lens_out=None, stream=None) -> None:
+        pool = self._pool_fp8(k_pool, v_pool)
+        trajs = self._trajs(page_table, seq_lens)
+        n_items = new_indptr.shape[0] - 1
+        total_new = k_new.shape[0]
+        if k_new.shape != v_new.shape or tuple(k_new.shape[1:]) != (pool.num_kv_heads, pool.head_dim):
+            raise ValueError("k_new/v_new must be [total_new][num_kv_heads][head_dim]")
+        if traj_ids is not None and traj_ids.shape[0] != n_items:
+            raise ValueError("traj_ids must have one entry per item")
+        if seq_lens_out is not None and seq_lens_out.shape != seq_lens.shape:
+            raise ValueError("seq_lens_out must have the shape of seq_lens")
+        st = self._lib.rollart_kv_append_fp8(
+            self._h, ctypes.byref(pool), ctypes.byref(trajs), _ptr(traj_ids, torch.int32, self.device),
+            _ptr(new_indptr, torch.int32, self.device), n_items, total_new, _ptr(k_new, torch.bfloat16, self.device),
+            _ptr(v_new, torch.bfloat16, self.device), float(k_scale), float(v_scale),
+            _ptr(seq_lens_out, torch.int32, self.device), self._stream(stream))
         if st != OK:
             self._raise(st)
 
@@ -267,6 +301,24 @@ class Context:
         st = self._lib.rollart_decode_attn(
             self._h, ctypes.byref(pool), ctypes.byref(trajs), _ptr(traj_ids, torch.int32, self.device), n_items,
             int(max_seq_len), _ptr(q, torch.bfloat16, self.device), hq, float(sm_scale),
+            _ptr(out, torch.bfloat16, self.device), _ptr(lse, torch.float32, self.device), self._stream(stream))
+        if st != OK:
+            self._raise(st)
+
+    def decode_attn_fp8(self, k_pool, v_pool, page_table, seq_lens, q, sm_scale, k_scale, v_scale, max_seq_len, out,
+                        lse=None, traj_ids=None, stream=None) -> None:
+        pool = self._pool_fp8(k_pool, v_pool)
+        trajs = self._trajs(page_table, seq_lens)
+        if q.dim() != 3 or q.shape != out.shape:
+            raise ValueError("q and out must be [n_items][num_q_heads][head_dim]")
+        n_items, hq, _ = q.shape
+        if traj_ids is not None and traj_ids.shape[0] != n_items:
+            raise ValueError("traj_ids must have one entry per item")
+        if lse is not None and tuple(lse.shape) != (n_items, hq):
+            raise ValueError("lse must be [n_items][num_q_heads]")
+        st = self._lib.rollart_decode_attn_fp8(
+            self._h, ctypes.byref(pool), ctypes.byref(trajs), _ptr(traj_ids, torch.int32, self.device), n_items,
+            int(max_seq_len), _ptr(q, torch.bfloat16, self.device), hq, float(sm_scale), float(k_scale), float(v_scale),
             _ptr(out, torch.bfloat16, self.device), _ptr(lse, torch.float32, self.device), self._stream(stream))
         if st != OK:
             self._raise(st)
