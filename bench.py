@@ -157,6 +157,32 @@ class DecodeWorkload:
         self.ctx.check()
         return total, dec
 
+    def time_fp8_steps(self, steps: int, warmup: int, k_scale: float = 0.03, v_scale: float = 0.03):
+        """The same step over fp8 (E4M3) pools: quantised append of the new token + fp8 decode attention (two launches).
+        The pools are the bf16 pools quantised with the given scales.  Returns (ms per step, KV bytes read per step)."""
+        b = self.batch
+        k8 = (b.k_pool.float() * (1.0 / k_scale)).to(torch.float8_e4m3fn).view(torch.uint8)
+        v8 = (b.v_pool.float() * (1.0 / v_scale)).to(torch.float8_e4m3fn).view(torch.uint8)
+
+        def step():
+            self.ctx.kv_append_fp8(k8, v8, self.table, self.lens0, self.indptr, self.k_new, self.v_new, k_scale, v_scale,
+                                   traj_ids=self.traj_ids, seq_lens_out=self.lens1)
+            self.ctx.decode_attn_fp8(k8, v8, self.table, self.lens1, self.q, self.spec.sm_scale, k_scale, v_scale,
+                                     self.max_seq_len, self.out, traj_ids=self.traj_ids)
+
+        for _ in range(warmup):
+            step()
+        torch.cuda.synchronize(self.device)
+        t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t0.record()
+        for _ in range(steps):
+            step()
+        t1.record()
+        torch.cuda.synchronize(self.device)
+        self.ctx.check()
+        kv_bytes = int(self.lens_after_host.astype(np.int64).sum()) * 2 * self.spec.num_kv_heads * self.spec.head_dim
+        return t0.elapsed_time(t1) / steps, kv_bytes + 2 * self.q.numel() * 2
+
     def time_gather(self, steps: int = 5, warmup: int = 2):
         """KV hand-off: all trajectories' caches gathered into contiguous rows.  (mean ms, bytes read + written)"""
         b = self.batch
@@ -510,6 +536,23 @@ def main():
             extra = {}
             del wl
             torch.cuda.empty_cache()
+            for ci in (1, 2, 3):
+                # the decode step over fp8 pools (half the KV bytes), beside the bf16 step of the same workload
+                name = W.CONFIGS[ci].name + "_fp8_pool"
+                try:
+                    w8 = DecodeWorkload(W.CONFIGS[ci], args.seed, device)
+                    _, bf_ms = w8.time_steps(200 if ci == 1 else 20, 3)
+                    f8_ms, f8_bytes = w8.time_fp8_steps(200 if ci == 1 else 20, 3)
+                    extra[name] = {"step_ms": f8_ms, "bf16_step_ms": bf_ms, "speedup_over_bf16_step": bf_ms / f8_ms,
+                                   "decode_tokens_per_s": w8.n_items / (f8_ms * 1e-3),
+                                   "hbm_gbs_of_fp8_bytes": f8_bytes / (f8_ms * 1e-3) / 1e9,
+                                   "frac_of_measured": f8_bytes / (f8_ms * 1e-3) / 1e9 / peak,
+                                   "launches_per_step": 2}
+                    w8.ctx.close()
+                    del w8
+                    torch.cuda.empty_cache()
+                except Exception as e:
+                    extra[name] = {"error": repr(e)}
             for ci in (2, 3, 4):
                 try:
                     w2 = DecodeWorkload(W.CONFIGS[ci], args.seed, device)
