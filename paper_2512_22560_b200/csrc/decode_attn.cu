@@ -41,9 +41,9 @@ constexpr int kStages = 6;
 constexpr int kConsumerWarps = 8;         // two groups of four
 constexpr int kProducerWarp = kConsumerWarps;        // warp 8 issues the copies
 constexpr int kEpilogueWarp = kConsumerWarps + 1;    // warp 9 writes pieces out and combines splits
-constexpr int kThreads = (kConsumerWarps + 2) * 32;
-constexpr int kProducerWarpV = kConsumerWarps + 2;   // fp8 only: warp 10 issues the V copies (warp 8 the K copies)
-constexpr int kThreadsFp8 = kThreads + 32;
+constexpr int kProducerWarpV = kConsumerWarps + 2;   // warp 10 issues the V copies (warp 8 the K copies and Q)
+constexpr int kThreads = (kConsumerWarps + 3) * 32;
+constexpr int kThreadsFp8 = kThreads;
 constexpr int kMaxItems = 512;            // items per launch (prefix table lives in shared memory)
 constexpr int kTensorBytes = kTile * kRowBytes;      // 16 KB of K (or V) per stage
 constexpr int kStageBytes = 2 * kTensorBytes;
@@ -316,7 +316,7 @@ decode_splitkv_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
     for (int i = threadIdx.x; i < 2 * kQBytes / 16; i += kT)
         reinterpret_cast<uint4 *>(smem + kOffQ)[i] = make_uint4(0, 0, 0, 0);
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kS; ++s) { mbar_init(bar_full(s), kFp8 ? 2 : 1); mbar_init(bar_empty(s), kConsumerWarps / 2); }
+        for (int s = 0; s < kS; ++s) { mbar_init(bar_full(s), 2); mbar_init(bar_empty(s), kConsumerWarps / 2); }
         for (int s = 0; s < 2; ++s) { mbar_init(bar_qfull(s), 1); mbar_init(bar_qempty(s), kConsumerWarps); }
         for (int s = 0; s < 2; ++s) { mbar_init(bar_epfull(s), 1); mbar_init(bar_epempty(s), 1); }
         *s_abort = 0;
@@ -389,12 +389,12 @@ decode_splitkv_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
     const int p_end = min(total, p_begin + span);
     if (p_begin >= p_end) return;
 
-    if (warp == kProducerWarp || (kFp8 && warp == kProducerWarpV)) {
-        // =============================== producer warp(s) ===============================
-        // bf16: one warp brings K and V.  fp8: a tile is half the bytes, so twice as many copies per second are due and
-        // one warp cannot issue them (a thread is held some 80 cycles by each): warp 8 brings K (and Q), warp 10 brings
-        // V, each with its own arrival on the stage's barrier.
-        const bool do_k = !kFp8 || warp == kProducerWarp, do_v = !kFp8 || warp == kProducerWarpV;
+    if (warp == kProducerWarp || warp == kProducerWarpV) {
+        // =============================== producer warps ===============================
+        // Warp 8 brings K (and Q), warp 10 brings V, each with its own arrival on the stage's barrier: a thread is held
+        // some 80 cycles by each tensor copy, and with 16-token pages one warp issuing all of them was as slow as the
+        // memory (the fp8 pools, with half the bytes per copy, made it the limit).
+        const bool do_k = warp == kProducerWarp;
         const int pages_per_tile = kTile / P;
         const int tiles_per_batch = 32 / pages_per_tile;
         const uint32_t page_bytes = static_cast<uint32_t>(P) * (kFp8 ? kHeadDim : kRowBytes);   // one (page, head) image of K or V
@@ -436,7 +436,7 @@ decode_splitkv_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
                 const uint32_t nvalid = __popc(__ballot_sync(0xffffffffu, pg >= 0));
                 mbar_wait(bar_empty(stage), ((n / kS) & 1) ^ 1, s_abort, prm.status, 2);
                 if (*s_abort) continue;
-                if (lane == 0) mbar_arrive_expect_tx(bar_full(stage), nvalid * (kFp8 ? 1u : 2u) * page_bytes);
+                if (lane == 0) mbar_arrive_expect_tx(bar_full(stage), nvalid * page_bytes);
                 __syncwarp();
                 if (pg >= 0) {
                     const uint32_t kdst = smem_u32(smem + kOffStages + stage * kSB) + lane * page_bytes;
@@ -447,14 +447,14 @@ decode_splitkv_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
                         if (do_k) tma_load_2d(kdst, &kmap, bar_full(stage), 0, unit * P);
                         else tma_load_2d(vdst, &vmap, bar_full(stage), 0, unit * P);
                     } else if (prm.four_d) {
-                        tma_load_4d(kdst, &kmap, bar_full(stage), 0, 0, 0, unit);
-                        tma_load_4d(vdst, &vmap, bar_full(stage), 0, 0, 0, unit);
+                        if (do_k) tma_load_4d(kdst, &kmap, bar_full(stage), 0, 0, 0, unit);
+                        else tma_load_4d(vdst, &vmap, bar_full(stage), 0, 0, 0, unit);
                     } else {
                         const int row = unit * P;
-                        tma_load_2d(kdst, &kmap, bar_full(stage), 0, row);
-                        tma_load_2d(kdst + page_bytes / 2, &kmap, bar_full(stage), 64, row);
-                        tma_load_2d(vdst, &vmap, bar_full(stage), 0, row);
-                        tma_load_2d(vdst + page_bytes / 2, &vmap, bar_full(stage), 64, row);
+                        const uint32_t dst = do_k ? kdst : vdst;
+                        const CUtensorMap *map = do_k ? &kmap : &vmap;
+                        tma_load_2d(dst, map, bar_full(stage), 0, row);
+                        tma_load_2d(dst + page_bytes / 2, map, bar_full(stage), 64, row);
                     }
                 }
             }
