@@ -398,7 +398,9 @@ decode_splitkv_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
         const int pages_per_tile = kTile / P;
         const int tiles_per_batch = 32 / pages_per_tile;
         const uint32_t page_bytes = static_cast<uint32_t>(P) * (kFp8 ? kHeadDim : kRowBytes);   // one (page, head) image of K or V
-        int n = 0, pcount = 0;
+        int n = 0, pcount = 0, stage = 0;          // stage = n % kS, phase = (n / kS) & 1, kept as running values
+        uint32_t phase = 0;
+        bool gave_up = false;
         for (int p = p_begin; p < p_end;) {
             const Piece pc = piece_at(s_prefix, s_lens, prm.n_items, hkv, p, p_end);
             p += pc.advance;
@@ -428,33 +430,35 @@ decode_splitkv_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
             };
             int ids_cur = load_ids(pc.tile0), ids_next = load_ids(pc.tile0 + tiles_per_batch);
             for (int tile = pc.tile0; tile < pc.tile1; ++tile, ++n) {
-                const int stage = n % kS;
-                const int within = (tile - pc.tile0) % tiles_per_batch;
+                const int within = (tile - pc.tile0) & (tiles_per_batch - 1);      // a power of two
                 if (tile > pc.tile0 && within == 0) { ids_cur = ids_next; ids_next = load_ids(tile + tiles_per_batch); }
                 int pg = __shfl_sync(0xffffffffu, ids_cur, (within * pages_per_tile + lane) & 31);
                 if (lane >= pages_per_tile) pg = -1;
                 const uint32_t nvalid = __popc(__ballot_sync(0xffffffffu, pg >= 0));
-                mbar_wait(bar_empty(stage), ((n / kS) & 1) ^ 1, s_abort, prm.status, 2);
-                if (*s_abort) continue;
-                if (lane == 0) mbar_arrive_expect_tx(bar_full(stage), nvalid * page_bytes);
+                mbar_wait(bar_empty(stage), phase ^ 1u, s_abort, prm.status, 2);
+                if ((n & 15) == 0 && *s_abort) gave_up = true;       // looked at now and then: the copy loop is on the clock
+                const int this_stage = stage;
+                if (++stage == kS) { stage = 0; phase ^= 1u; }
+                if (gave_up) continue;
+                if (lane == 0) mbar_arrive_expect_tx(bar_full(this_stage), nvalid * page_bytes);
                 __syncwarp();
                 if (pg >= 0) {
-                    const uint32_t kdst = smem_u32(smem + kOffStages + stage * kSB) + lane * page_bytes;
+                    const uint32_t kdst = smem_u32(smem + kOffStages + this_stage * kSB) + lane * page_bytes;
                     const uint32_t vdst = kdst + kTB;
                     const int unit = pg * hkv + pc.head;          // (page, head) tile index
                     if constexpr (kFp8) {
                         // rows of 128 B: one box per (page, head), landing as [slot][128 B]
-                        if (do_k) tma_load_2d(kdst, &kmap, bar_full(stage), 0, unit * P);
-                        else tma_load_2d(vdst, &vmap, bar_full(stage), 0, unit * P);
+                        if (do_k) tma_load_2d(kdst, &kmap, bar_full(this_stage), 0, unit * P);
+                        else tma_load_2d(vdst, &vmap, bar_full(this_stage), 0, unit * P);
                     } else if (prm.four_d) {
-                        if (do_k) tma_load_4d(kdst, &kmap, bar_full(stage), 0, 0, 0, unit);
-                        else tma_load_4d(vdst, &vmap, bar_full(stage), 0, 0, 0, unit);
+                        if (do_k) tma_load_4d(kdst, &kmap, bar_full(this_stage), 0, 0, 0, unit);
+                        else tma_load_4d(vdst, &vmap, bar_full(this_stage), 0, 0, 0, unit);
                     } else {
                         const int row = unit * P;
                         const uint32_t dst = do_k ? kdst : vdst;
                         const CUtensorMap *map = do_k ? &kmap : &vmap;
-                        tma_load_2d(dst, map, bar_full(stage), 0, row);
-                        tma_load_2d(dst + page_bytes / 2, map, bar_full(stage), 64, row);
+                        tma_load_2d(dst, map, bar_full(this_stage), 0, row);
+                        tma_load_2d(dst + page_bytes / 2, map, bar_full(this_stage), 64, row);
                     }
                 }
             }
