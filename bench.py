@@ -44,7 +44,7 @@ def measured_peaks():
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one decode_splitkv_kernel launch, from the ncu capture summarised in
 # profiles/decode_splitkv_cfg1.md (default seed).  Valid only for the kernel as captured: set to None when it changes.
-MEASURED_TRAFFIC_BYTES = {"cfg1_7b_gqa_decode": 724.9e6}
+MEASURED_TRAFFIC_BYTES = {"cfg1_7b_gqa_decode": 725.6e6}
 
 
 def decode_algorithmic_bytes(spec: W.WorkloadSpec, lens_after: np.ndarray) -> int:
@@ -457,6 +457,7 @@ def main():
     ap.add_argument("--no-extra", action="store_true", help="skip the other decode workloads and the CPU baseline")
     ap.add_argument("--chunk", action="store_true", help="time only the observation-chunk half of --config (for profiling)")
     ap.add_argument("--shrink", type=int, default=1, help="with --chunk: divide context lengths by this (small profiling case)")
+    ap.add_argument("--fp8", action="store_true", help="time only the fp8-pool decode step of --config (for profiling)")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
@@ -486,6 +487,12 @@ def main():
         print(json.dumps({"workload": spec.name + " (chunk half)", "chunk_rows": cw.rows, "chunk_attn_ms": att_ms,
                           "tflops": cw.flops / (att_ms * 1e-3) / 1e12, "append_ms": app_ms,
                           "append_gbs": cw.append_bytes / (app_ms * 1e-3) / 1e9}))
+        return 0
+    if args.fp8:
+        w8 = DecodeWorkload(spec, args.seed, device)
+        f8_ms, f8_bytes = w8.time_fp8_steps(args.steps, args.warmup)
+        print(json.dumps({"workload": spec.name + " (fp8 pools: quantised append + decode)", "step_ms": f8_ms,
+                          "decode_tokens_per_s": w8.n_items / (f8_ms * 1e-3), "hbm_gbs_of_fp8_bytes": f8_bytes / (f8_ms * 1e-3) / 1e9}))
         return 0
     wl = DecodeWorkload(spec, rank_seed(args.seed, rank), device)      # replicas: each rank owns its own trajectories
 
