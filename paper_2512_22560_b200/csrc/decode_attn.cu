@@ -13,10 +13,10 @@
 // the log-sum-exp rule (cross-split combine) and writes the output.  The cut and the merge order
 // are fixed functions of the lengths, so reruns are bit identical.
 //
-// Data path.  A producer warp walks the block's span and brings each 64-key tile of K and V
-// (32 KB) into a ring of shared-memory stages with TMA tensor copies, one box per (page, head)
+// Data path.  Two producer warps (one for K and the queries, one for V) walk the block's span and
+// bring each 64-key tile of K and V (32 KB) into a ring of shared-memory stages with TMA tensor copies, one box per (page, head)
 // (or per half row), 128-byte swizzled so that ldmatrix reads are bank-conflict free; the page
-// ids come from the page table just ahead of the copy.  Eight consumer warps in two groups take
+// ids come from the page table a batch ahead of the copies.  Eight consumer warps in two groups take
 // alternate tiles; each warp owns 16 keys of a tile and computes, for all (up to 16) query heads
 // of the GQA group at once, S = Q K^T and O += P V with bf16 mma.sync (fp32 accumulate) and an
 // online softmax in registers.  One K/V read serves the whole group.  At the end of a piece the
