@@ -29,6 +29,12 @@ MUTANTS = {
     "reserve_rounds_down": ("int64_t want = ((int64_t)seq_lens[t] + new_tokens[i] + P - 1) / P;\n        for (int64_t lp = have;",
                             "int64_t want = ((int64_t)seq_lens[t] + new_tokens[i]) / P;\n        for (int64_t lp = have;"),
     "release_keeps_length": ("        seq_lens[t] = 0;\n", "        seq_lens[t] = seq_lens[t];\n"),
+    "e4m3_wrong_bias": ("else v = ldexp(1.0 + (double)m / 8.0, e - 7);", "else v = ldexp(1.0 + (double)m / 8.0, e - 8);"),
+    "e4m3_subnormals_as_normals": ("else if (e == 0) v = ldexp((double)m / 8.0, -6);",
+                                   "else if (e == 0) v = ldexp(1.0 + (double)m / 8.0, -7);"),
+    "e4m3_truncates": ("int m = (int)nearbyint((2.0 * fr - 1.0) * 8.0);", "int m = (int)floor((2.0 * fr - 1.0) * 8.0);"),
+    "e4m3_ties_away": ("int m = (int)nearbyint((2.0 * fr - 1.0) * 8.0);", "int m = (int)round((2.0 * fr - 1.0) * 8.0);"),
+    "e4m3_subnormal_step": ("mag = (uint8_t)nearbyint(ldexp(a, 9));", "mag = (uint8_t)nearbyint(ldexp(a, 8));"),
 }
 
 
@@ -42,7 +48,8 @@ def test_pins_catch_planted_mistake(name, tmp_path):
     subprocess.run(["gcc", "-O2", "-std=c11", "-fPIC", "-shared", "-fopenmp", "-o", str(so_file), str(c_file), "-lm"], check=True)
     env = dict(os.environ, ROLLART_ORACLE_LIB=str(so_file))
     r = subprocess.run([sys.executable, "-m", "pytest", "-x", "-q", "-p", "no:cacheprovider",
-                        os.path.join(ROOT, "tests", "test_oracle_pins.py"), os.path.join(ROOT, "tests", "test_oracle_pages.py")],
+                        os.path.join(ROOT, "tests", "test_oracle_pins.py"), os.path.join(ROOT, "tests", "test_oracle_pages.py"),
+                        os.path.join(ROOT, "tests", "test_oracle_fp8.py")],
                        cwd=ROOT, env=env, capture_output=True, text=True, timeout=300)
     assert r.returncode != 0, f"the pins did not notice the planted mistake '{name}'"
     assert "failed" in r.stdout or "error" in r.stdout.lower(), r.stdout[-400:]
