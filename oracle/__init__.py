@@ -2,7 +2,8 @@
 
 TEST INFRASTRUCTURE ONLY.  Nothing in the product package imports this; only the tests,
 the smoke check and the bench's CPU-baseline leg do.  Arrays are numpy; bf16 data travels
-as uint16 bit patterns.  Every function here is pinned by tests/test_oracle_pins.py.
+as uint16 bit patterns.  Every function here is pinned by tests/test_oracle_pins.py, tests/test_oracle_pages.py
+or tests/test_oracle_fp8.py.
 """
 from __future__ import annotations
 

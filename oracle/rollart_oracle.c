@@ -40,7 +40,8 @@
  *
  * Everything floating point is fp64; bf16 inputs convert exactly.  No blocking,
  * no online softmax, no reordering: two passes over the keys, in index order.
- * Parity status: every function here is pinned by tests/test_oracle_pins.py
+ * Parity status: every function here is pinned by tests/test_oracle_pins.py, tests/test_oracle_pages.py or
+ * tests/test_oracle_fp8.py
  * (closed forms, invariants, an independent dense routine, brute force).
  */
 #include <math.h>
