@@ -66,8 +66,7 @@ constexpr int kOffLens = kOffMl + 2 * kMlFloats * 4;
 constexpr int kOffPrefix = kOffLens + kMaxItems * 4;
 constexpr int kOffTraj = kOffPrefix + (kMaxItems + 32) * 4;   // trajectory of every item (read once from global memory)
 constexpr int kOffBars = kOffTraj + kMaxItems * 4;
-constexpr int kStagesFp8 = 2 * kStages;           // an fp8 tile is half the bytes: twice the stages in the same memory
-constexpr int kNumBars = 2 * kStagesFp8 + 8;
+constexpr int kNumBars = 2 * kStages + 8;
 constexpr int kOffAbort = kOffBars + kNumBars * 8;
 constexpr int kSmemBytes = kOffAbort + 16 + 1024;    // + slack for the 1024-byte alignment
 static_assert(kSmemBytes <= 227 * 1024, "the block must fit the shared memory of an SM");
@@ -252,7 +251,7 @@ struct Piece {
 };
 
 // Length of an (item, head) on the line: its tiles plus the fixed cost of a piece.
-__device__ __forceinline__ int line_len(int len) { return len > 0 ? (len + kTile - 1) / kTile + kPieceCost : 0; }
+__device__ __forceinline__ int line_len(int len, int tile_keys) { return len > 0 ? (len + tile_keys - 1) / tile_keys + kPieceCost : 0; }
 
 __device__ __forceinline__ Piece piece_at(const int *prefix, const int *lens, int n_items, int hkv, int p, int p_end) {
     int lo = 0, hi = n_items;                     // largest item with prefix[item] * hkv <= p
@@ -279,15 +278,17 @@ __device__ __forceinline__ Piece piece_at(const int *prefix, const int *lens, in
 // Kernel
 // ------------------------------------------------------------------------------------------
 // kFp8: the pools hold E4M3 bytes (rows of 128 B) instead of bf16 (rows of 256 B).  The schedule, the pieces, the merge
-// and the combine are the same; the tiles are half the bytes (twice the stages), K and V are converted to f16 as the
-// fragments are loaded and the products run as f16 MMAs (the query is converted once per piece).
+// and the combine are the same; a tile is 128 keys (the same bytes per stage, and half as many hand-overs per byte: a
+// warp owns 32 keys of a tile), K and V are converted to f16 as the fragments are loaded and the products run as f16
+// MMAs (the query is converted once per piece).
 template <bool kFp8>
 __global__ void __launch_bounds__(kFp8 ? kThreadsFp8 : kThreads, 1)
 decode_splitkv_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_constant__ CUtensorMap vmap,
                       const DecodeParams prm) {
-    constexpr int kS = kFp8 ? kStagesFp8 : kStages;                 // stages of the ring
-    constexpr int kSB = kFp8 ? kStageBytes / 2 : kStageBytes;       // bytes of a stage: K image then V image
+    constexpr int kS = kStages;                                     // stages of the ring
+    constexpr int kSB = kStageBytes;                                // bytes of a stage: K image then V image
     constexpr int kTB = kSB / 2;
+    constexpr int kTK = kFp8 ? 2 * kTile : kTile;                   // keys of a tile
     constexpr int kT = kFp8 ? kThreadsFp8 : kThreads;               // threads of the block
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -353,7 +354,7 @@ decode_splitkv_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
         const int per = (prm.n_items + 31) / 32;
         const int a = min(prm.n_items, lane * per), b = min(prm.n_items, a + per);
         int sum = 0;
-        for (int i = a; i < b; ++i) sum += line_len(s_lens[i]);
+        for (int i = a; i < b; ++i) sum += line_len(s_lens[i], kTK);
         int incl = sum;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
@@ -361,7 +362,7 @@ decode_splitkv_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
             if (lane >= o) incl += v;
         }
         int run = incl - sum;
-        for (int i = a; i < b; ++i) { s_prefix[i] = run; run += line_len(s_lens[i]); }
+        for (int i = a; i < b; ++i) { s_prefix[i] = run; run += line_len(s_lens[i], kTK); }
         if (lane == 31) s_prefix[prm.n_items] = incl;
     }
     fence_proxy_async();      // the zeroed Q rows are ordered before the bulk copies that land beside them
@@ -395,7 +396,7 @@ decode_splitkv_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
         // some 80 cycles by each tensor copy, and with 16-token pages one warp issuing all of them was as slow as the
         // memory (the fp8 pools, with half the bytes per copy, made it the limit).
         const bool do_k = warp == kProducerWarp;
-        const int pages_per_tile = kTile / P;
+        const int pages_per_tile = kTK / P;
         const int tiles_per_batch = 32 / pages_per_tile;
         const uint32_t page_bytes = static_cast<uint32_t>(P) * (kFp8 ? kHeadDim : kRowBytes);   // one (page, head) image of K or V
         int n = 0, pcount = 0, stage = 0;          // stage = n % kS, phase = (n / kS) & 1, kept as running values
@@ -593,7 +594,7 @@ decode_splitkv_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
     const int grp = warp >> 2, wq = warp & 3;
     const int qrow = lane >> 2, qcol = lane & 3;          // fragment row / column-pair of this lane
     // byte offset of this warp's 16 keys inside a K (or V) stage image, and ldmatrix lane offsets
-    const int key0 = wq * 16;
+    const int key0 = wq * (kFp8 ? 32 : 16);
     // (fp8: the rows of a tile are 128 B and lie one after the other)
     const uint32_t warp_off = kFp8 ? static_cast<uint32_t>(key0 * 128)
                                    : static_cast<uint32_t>((key0 / P) * P * kRowBytes + (key0 % P) * 128);
@@ -644,103 +645,69 @@ decode_splitkv_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
             mbar_wait(bar_full(stage), (n / kS) & 1, s_abort, prm.status, 4);
             const uint32_t kbase = smem_u32(smem + kOffStages + stage * kSB) + warp_off;
             const uint32_t vbase = kbase + kTB;
-            const int valid = min(16, pc.len - tile * kTile - key0);   // live keys among this warp's 16
-            bool patched = false;
-            if (!kFp8 && prm.k_new != nullptr && tile == pc.ntiles - 1 && valid > 0 && valid <= 16 &&
-                pc.len - 1 - tile * kTile - key0 == valid - 1) {
-                // Fused append: this warp owns the context's last key, which is the item's new token.  Its K/V row
-                // comes from k_new / v_new: put it into the staged tile (over whatever the copy brought for that
-                // slot) and into the pool, where later steps will find it.  Lanes 0-15 move K, lanes 16-31 move V.
-                const int kk = valid - 1, c16 = lane & 15;
-                const int t = s_traj[pc.item];
-                const int pos = pc.len - 1;
-                const int pg = __ldg(prm.page_table + static_cast<long long>(t) * prm.max_pages + pos / P);
-                const long long src = (static_cast<long long>(pc.item) * hkv + pc.head) * (kHeadDim / 8) + c16;
-                const uint4 val = __ldg(reinterpret_cast<const uint4 *>(lane < 16 ? prm.k_new : prm.v_new) + src);
-                const uint32_t a = (lane < 16 ? kbase : vbase) + (c16 >> 3) * half_off + kk * 128 + (((c16 & 7) ^ (kk & 7)) << 4);
-                asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(a), "r"(val.x), "r"(val.y), "r"(val.z), "r"(val.w) : "memory");
-                if (pg >= 0 && pg < prm.num_pages) {     // a bad page id was already reported by the producer
-                    const long long dst = ((static_cast<long long>(pg) * hkv + pc.head) * P + pos % P) * (kHeadDim / 8) + c16;
-                    reinterpret_cast<uint4 *>(lane < 16 ? prm.k_pool : prm.v_pool)[dst] = val;
-                }
-                patched = true;
-                __syncwarp();
-            }
-            if (valid > 0) {
-                if (valid < 16) {
-                    // dead slots may hold anything (NaN included): zero their V rows so that 0 * v stays 0
-                    constexpr int kVecPerKey = kFp8 ? 8 : 16;       // 16-byte pieces of a V row
-                    for (int idx = lane; idx < (16 - valid) * kVecPerKey; idx += 32) {
-                        const int r = valid + idx / kVecPerKey, c = idx % kVecPerKey;
-                        const uint32_t a = kFp8 ? vbase + r * 128 + c * 16 : vbase + (c >> 3) * half_off + r * 128 + (c & 7) * 16;
-                        asm volatile("st.shared.v4.b32 [%0], {%1,%1,%1,%1};" ::"r"(a), "r"(0) : "memory");
+            if constexpr (kFp8) {
+                // ---- fp8: this warp owns 32 keys of the 128-key tile, as two halves of 16 that share one softmax update ----
+                const int valid = min(32, pc.len - tile * kTK - key0);
+                if (valid > 0) {
+                    if (valid < 32) {
+                        // dead slots may hold anything (NaN codes included): zero their V rows so that 0 * v stays 0
+                        for (int idx = lane; idx < (32 - valid) * 8; idx += 32) {
+                            const uint32_t a = vbase + (valid + (idx >> 3)) * 128 + (idx & 7) * 16;
+                            asm volatile("st.shared.v4.b32 [%0], {%1,%1,%1,%1};" ::"r"(a), "r"(0) : "memory");
+                        }
+                        __syncwarp();
                     }
-                    __syncwarp();
-                }
-                float s[2][4];
+                    float s[4][4];      // [half * 2 + key octet]
 #pragma unroll
-                for (int nt = 0; nt < 2; ++nt) s[nt][0] = s[nt][1] = s[nt][2] = s[nt][3] = 0.f;
-                if constexpr (kFp8) {
-                    // one load brings keys 0-7 and 8-15 for two 16-dim chunks (a row of 128 B holds 8 chunks of 16 B);
-                    // each 32-bit register is the lane's four dims of a key: its halves are the two B registers
+                    for (int i = 0; i < 4; ++i) s[i][0] = s[i][1] = s[i][2] = s[i][3] = 0.f;
+                    // one load brings keys 0-7 and 8-15 of a half for two 16-dim chunks (a row of 128 B holds 8 chunks of
+                    // 16 B); each 32-bit register is the lane's four dims of a key: its halves are the two B registers
 #pragma unroll
                     for (int cp = 0; cp < 4; ++cp) {
                         const int chunk = cp * 2 + (lm >> 1);
-                        uint32_t r0, r1, r2, r3;
-                        ldmatrix_x4(r0, r1, r2, r3, kbase + ((lm & 1) * 8 + lr) * 128 + ((chunk ^ lr) << 4));
-                        mma_f16(s[0], qa[2 * cp], e4m3x2_to_f16x2_lo(r0), e4m3x2_to_f16x2_hi(r0));
-                        mma_f16(s[1], qa[2 * cp], e4m3x2_to_f16x2_lo(r1), e4m3x2_to_f16x2_hi(r1));
-                        mma_f16(s[0], qa[2 * cp + 1], e4m3x2_to_f16x2_lo(r2), e4m3x2_to_f16x2_hi(r2));
-                        mma_f16(s[1], qa[2 * cp + 1], e4m3x2_to_f16x2_lo(r3), e4m3x2_to_f16x2_hi(r3));
-                    }
-                } else {
 #pragma unroll
-                    for (int ks = 0; ks < 8; ++ks) {
-                        const int chunk = ks * 2 + k_chunk_lo;
-                        uint32_t b0, b1, b2, b3;
-                        ldmatrix_x4(b0, b1, b2, b3, kbase + (chunk >> 3) * half_off + k_lane_off + (((chunk & 7) ^ lr) << 4));
-                        mma_bf16(s[0], qa[ks], b0, b1);
-                        mma_bf16(s[1], qa[ks], b2, b3);
+                        for (int hf = 0; hf < 2; ++hf) {
+                            uint32_t r0, r1, r2, r3;
+                            ldmatrix_x4(r0, r1, r2, r3, kbase + (hf * 16 + (lm & 1) * 8 + lr) * 128 + ((chunk ^ lr) << 4));
+                            mma_f16(s[2 * hf], qa[2 * cp], e4m3x2_to_f16x2_lo(r0), e4m3x2_to_f16x2_hi(r0));
+                            mma_f16(s[2 * hf + 1], qa[2 * cp], e4m3x2_to_f16x2_lo(r1), e4m3x2_to_f16x2_hi(r1));
+                            mma_f16(s[2 * hf], qa[2 * cp + 1], e4m3x2_to_f16x2_lo(r2), e4m3x2_to_f16x2_hi(r2));
+                            mma_f16(s[2 * hf + 1], qa[2 * cp + 1], e4m3x2_to_f16x2_lo(r3), e4m3x2_to_f16x2_hi(r3));
+                        }
                     }
-                }
 #pragma unroll
-                for (int nt = 0; nt < 2; ++nt)
+                    for (int i = 0; i < 4; ++i)
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const int col = nt * 8 + qcol * 2 + (e & 1);
-                        s[nt][e] = col < valid ? s[nt][e] * prm.scale_log2 : -INFINITY;
+                        for (int e = 0; e < 4; ++e) {
+                            const int col = i * 8 + qcol * 2 + (e & 1);
+                            s[i][e] = col < valid ? s[i][e] * prm.scale_log2 : -INFINITY;
+                        }
+                    float r0 = fmaxf(fmaxf(fmaxf(s[0][0], s[0][1]), fmaxf(s[1][0], s[1][1])), fmaxf(fmaxf(s[2][0], s[2][1]), fmaxf(s[3][0], s[3][1])));
+                    float r1 = fmaxf(fmaxf(fmaxf(s[0][2], s[0][3]), fmaxf(s[1][2], s[1][3])), fmaxf(fmaxf(s[2][2], s[2][3]), fmaxf(s[3][2], s[3][3])));
+                    r0 = fmaxf(r0, __shfl_xor_sync(0xffffffffu, r0, 1));
+                    r0 = fmaxf(r0, __shfl_xor_sync(0xffffffffu, r0, 2));
+                    r1 = fmaxf(r1, __shfl_xor_sync(0xffffffffu, r1, 1));
+                    r1 = fmaxf(r1, __shfl_xor_sync(0xffffffffu, r1, 2));
+                    const float n0 = fmaxf(m0, r0), n1 = fmaxf(m1, r1);
+                    if (__any_sync(0xffffffffu, n0 > m0 || n1 > m1)) {
+                        const float c0 = exp2f(m0 - n0), c1 = exp2f(m1 - n1);     // exp2(-inf) = 0 on the first tile
+                        l0 *= c0; l1 *= c1;
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) { o[j][0] *= c0; o[j][1] *= c0; o[j][2] *= c1; o[j][3] *= c1; }
+                        m0 = n0; m1 = n1;
                     }
-                float r0 = fmaxf(fmaxf(s[0][0], s[0][1]), fmaxf(s[1][0], s[1][1]));
-                float r1 = fmaxf(fmaxf(s[0][2], s[0][3]), fmaxf(s[1][2], s[1][3]));
-                r0 = fmaxf(r0, __shfl_xor_sync(0xffffffffu, r0, 1));
-                r0 = fmaxf(r0, __shfl_xor_sync(0xffffffffu, r0, 2));
-                r1 = fmaxf(r1, __shfl_xor_sync(0xffffffffu, r1, 1));
-                r1 = fmaxf(r1, __shfl_xor_sync(0xffffffffu, r1, 2));
-                const float n0 = fmaxf(m0, r0), n1 = fmaxf(m1, r1);
-                if (__any_sync(0xffffffffu, n0 > m0 || n1 > m1)) {
-                    const float c0 = exp2f(m0 - n0), c1 = exp2f(m1 - n1);     // exp2(-inf) = 0 on the first tile
-                    l0 *= c0; l1 *= c1;
+                    uint32_t pa[2][4];
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) { o[j][0] *= c0; o[j][1] *= c0; o[j][2] *= c1; o[j][3] *= c1; }
-                    m0 = n0; m1 = n1;
-                }
-                uint32_t pa[4];
-                {
-                    const float p00 = exp2f(s[0][0] - m0), p01 = exp2f(s[0][1] - m0);
-                    const float p02 = exp2f(s[0][2] - m1), p03 = exp2f(s[0][3] - m1);
-                    const float p10 = exp2f(s[1][0] - m0), p11 = exp2f(s[1][1] - m0);
-                    const float p12 = exp2f(s[1][2] - m1), p13 = exp2f(s[1][3] - m1);
-                    l0 += (p00 + p01) + (p10 + p11);
-                    l1 += (p02 + p03) + (p12 + p13);
-                    if constexpr (kFp8) {
-                        pa[0] = pack_f16(p00, p01); pa[1] = pack_f16(p02, p03);
-                        pa[2] = pack_f16(p10, p11); pa[3] = pack_f16(p12, p13);
-                    } else {
-                        pa[0] = pack_bf16(p00, p01); pa[1] = pack_bf16(p02, p03);
-                        pa[2] = pack_bf16(p10, p11); pa[3] = pack_bf16(p12, p13);
+                    for (int hf = 0; hf < 2; ++hf) {
+                        const float p00 = exp2f(s[2 * hf][0] - m0), p01 = exp2f(s[2 * hf][1] - m0);
+                        const float p02 = exp2f(s[2 * hf][2] - m1), p03 = exp2f(s[2 * hf][3] - m1);
+                        const float p10 = exp2f(s[2 * hf + 1][0] - m0), p11 = exp2f(s[2 * hf + 1][1] - m0);
+                        const float p12 = exp2f(s[2 * hf + 1][2] - m1), p13 = exp2f(s[2 * hf + 1][3] - m1);
+                        l0 += (p00 + p01) + (p10 + p11);
+                        l1 += (p02 + p03) + (p12 + p13);
+                        pa[hf][0] = pack_f16(p00, p01); pa[hf][1] = pack_f16(p02, p03);
+                        pa[hf][2] = pack_f16(p10, p11); pa[hf][3] = pack_f16(p12, p13);
                     }
-                }
-                if constexpr (kFp8) {
                     // the transposed load hands a lane, for keys 2t and 2t+1, the two dims 2g, 2g+1 of a chunk
                     // (g = lane >> 2): bytes are regrouped into (key 2t, key 2t+1) pairs for the even and the odd
                     // dim, which feed two MMAs; their accumulator columns 2t, 2t+1 are then dims 4t, 4t+2 and
@@ -748,17 +715,97 @@ decode_splitkv_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
 #pragma unroll
                     for (int cp = 0; cp < 4; ++cp) {
                         const int chunk = cp * 2 + (lm >> 1);
-                        uint32_t r0, r1, r2, r3;
-                        ldmatrix_x4_trans(r0, r1, r2, r3, vbase + ((lm & 1) * 8 + lr) * 128 + ((chunk ^ lr) << 4));
-                        const uint32_t x0 = __byte_perm(r0, 0, 0x3120), x1 = __byte_perm(r1, 0, 0x3120);
-                        const uint32_t x2 = __byte_perm(r2, 0, 0x3120), x3 = __byte_perm(r3, 0, 0x3120);
-                        mma_f16(o[4 * cp], pa, e4m3x2_to_f16x2_lo(x0), e4m3x2_to_f16x2_lo(x1));
-                        mma_f16(o[4 * cp + 1], pa, e4m3x2_to_f16x2_hi(x0), e4m3x2_to_f16x2_hi(x1));
-                        mma_f16(o[4 * cp + 2], pa, e4m3x2_to_f16x2_lo(x2), e4m3x2_to_f16x2_lo(x3));
-                        mma_f16(o[4 * cp + 3], pa, e4m3x2_to_f16x2_hi(x2), e4m3x2_to_f16x2_hi(x3));
-                    }
-                } else {
 #pragma unroll
+                        for (int hf = 0; hf < 2; ++hf) {
+                            uint32_t r0v, r1v, r2v, r3v;
+                            ldmatrix_x4_trans(r0v, r1v, r2v, r3v, vbase + (hf * 16 + (lm & 1) * 8 + lr) * 128 + ((chunk ^ lr) << 4));
+                            const uint32_t x0 = __byte_perm(r0v, 0, 0x3120), x1 = __byte_perm(r1v, 0, 0x3120);
+                            const uint32_t x2 = __byte_perm(r2v, 0, 0x3120), x3 = __byte_perm(r3v, 0, 0x3120);
+                            mma_f16(o[4 * cp], pa[hf], e4m3x2_to_f16x2_lo(x0), e4m3x2_to_f16x2_lo(x1));
+                            mma_f16(o[4 * cp + 1], pa[hf], e4m3x2_to_f16x2_hi(x0), e4m3x2_to_f16x2_hi(x1));
+                            mma_f16(o[4 * cp + 2], pa[hf], e4m3x2_to_f16x2_lo(x2), e4m3x2_to_f16x2_lo(x3));
+                            mma_f16(o[4 * cp + 3], pa[hf], e4m3x2_to_f16x2_hi(x2), e4m3x2_to_f16x2_hi(x3));
+                        }
+                    }
+                    if (valid < 32) fence_proxy_async();   // our stores into the stage precede the next copy into it
+                }
+            } else {
+                const int valid = min(16, pc.len - tile * kTile - key0);   // live keys among this warp's 16
+                bool patched = false;
+                if (prm.k_new != nullptr && tile == pc.ntiles - 1 && valid > 0 && valid <= 16 &&
+                    pc.len - 1 - tile * kTile - key0 == valid - 1) {
+                    // Fused append: this warp owns the context's last key, which is the item's new token.  Its K/V row
+                    // comes from k_new / v_new: put it into the staged tile (over whatever the copy brought for that
+                    // slot) and into the pool, where later steps will find it.  Lanes 0-15 move K, lanes 16-31 move V.
+                    const int kk = valid - 1, c16 = lane & 15;
+                    const int t = s_traj[pc.item];
+                    const int pos = pc.len - 1;
+                    const int pg = __ldg(prm.page_table + static_cast<long long>(t) * prm.max_pages + pos / P);
+                    const long long src = (static_cast<long long>(pc.item) * hkv + pc.head) * (kHeadDim / 8) + c16;
+                    const uint4 val = __ldg(reinterpret_cast<const uint4 *>(lane < 16 ? prm.k_new : prm.v_new) + src);
+                    const uint32_t a = (lane < 16 ? kbase : vbase) + (c16 >> 3) * half_off + kk * 128 + (((c16 & 7) ^ (kk & 7)) << 4);
+                    asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(a), "r"(val.x), "r"(val.y), "r"(val.z), "r"(val.w) : "memory");
+                    if (pg >= 0 && pg < prm.num_pages) {     // a bad page id was already reported by the producer
+                        const long long dst = ((static_cast<long long>(pg) * hkv + pc.head) * P + pos % P) * (kHeadDim / 8) + c16;
+                        reinterpret_cast<uint4 *>(lane < 16 ? prm.k_pool : prm.v_pool)[dst] = val;
+                    }
+                    patched = true;
+                    __syncwarp();
+                }
+                if (valid > 0) {
+                    if (valid < 16) {
+                        // dead slots may hold anything (NaN included): zero their V rows so that 0 * v stays 0
+                        for (int idx = lane; idx < (16 - valid) * 16; idx += 32) {
+                            const int r = valid + (idx >> 4), c = idx & 15;
+                            const uint32_t a = vbase + (c >> 3) * half_off + r * 128 + (c & 7) * 16;
+                            asm volatile("st.shared.v4.b32 [%0], {%1,%1,%1,%1};" ::"r"(a), "r"(0) : "memory");
+                        }
+                        __syncwarp();
+                    }
+                    float s[2][4];
+    #pragma unroll
+                    for (int nt = 0; nt < 2; ++nt) s[nt][0] = s[nt][1] = s[nt][2] = s[nt][3] = 0.f;
+    #pragma unroll
+                    for (int ks = 0; ks < 8; ++ks) {
+                        const int chunk = ks * 2 + k_chunk_lo;
+                        uint32_t b0, b1, b2, b3;
+                        ldmatrix_x4(b0, b1, b2, b3, kbase + (chunk >> 3) * half_off + k_lane_off + (((chunk & 7) ^ lr) << 4));
+                        mma_bf16(s[0], qa[ks], b0, b1);
+                        mma_bf16(s[1], qa[ks], b2, b3);
+                    }
+    #pragma unroll
+                    for (int nt = 0; nt < 2; ++nt)
+    #pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const int col = nt * 8 + qcol * 2 + (e & 1);
+                            s[nt][e] = col < valid ? s[nt][e] * prm.scale_log2 : -INFINITY;
+                        }
+                    float r0 = fmaxf(fmaxf(s[0][0], s[0][1]), fmaxf(s[1][0], s[1][1]));
+                    float r1 = fmaxf(fmaxf(s[0][2], s[0][3]), fmaxf(s[1][2], s[1][3]));
+                    r0 = fmaxf(r0, __shfl_xor_sync(0xffffffffu, r0, 1));
+                    r0 = fmaxf(r0, __shfl_xor_sync(0xffffffffu, r0, 2));
+                    r1 = fmaxf(r1, __shfl_xor_sync(0xffffffffu, r1, 1));
+                    r1 = fmaxf(r1, __shfl_xor_sync(0xffffffffu, r1, 2));
+                    const float n0 = fmaxf(m0, r0), n1 = fmaxf(m1, r1);
+                    if (__any_sync(0xffffffffu, n0 > m0 || n1 > m1)) {
+                        const float c0 = exp2f(m0 - n0), c1 = exp2f(m1 - n1);     // exp2(-inf) = 0 on the first tile
+                        l0 *= c0; l1 *= c1;
+    #pragma unroll
+                        for (int j = 0; j < 16; ++j) { o[j][0] *= c0; o[j][1] *= c0; o[j][2] *= c1; o[j][3] *= c1; }
+                        m0 = n0; m1 = n1;
+                    }
+                    uint32_t pa[4];
+                    {
+                        const float p00 = exp2f(s[0][0] - m0), p01 = exp2f(s[0][1] - m0);
+                        const float p02 = exp2f(s[0][2] - m1), p03 = exp2f(s[0][3] - m1);
+                        const float p10 = exp2f(s[1][0] - m0), p11 = exp2f(s[1][1] - m0);
+                        const float p12 = exp2f(s[1][2] - m1), p13 = exp2f(s[1][3] - m1);
+                        l0 += (p00 + p01) + (p10 + p11);
+                        l1 += (p02 + p03) + (p12 + p13);
+                        pa[0] = pack_bf16(p00, p01); pa[1] = pack_bf16(p02, p03);
+                        pa[2] = pack_bf16(p10, p11); pa[3] = pack_bf16(p12, p13);
+                    }
+    #pragma unroll
                     for (int pr = 0; pr < 8; ++pr) {
                         const int chunk = pr * 2 + v_chunk_lo;
                         uint32_t b0, b1, b2, b3;
@@ -766,8 +813,8 @@ decode_splitkv_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
                         mma_bf16(o[2 * pr], pa, b0, b1);
                         mma_bf16(o[2 * pr + 1], pa, b2, b3);
                     }
+                    if (valid < 16 || patched) fence_proxy_async();   // our stores into the stage precede the next copy into it
                 }
-                if (valid < 16 || patched) fence_proxy_async();   // our stores into the stage precede the next copy into it
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_empty(stage));
