@@ -210,6 +210,9 @@ rollart_status rollart_append_decode_attn(rollart_ctx *ctx, const rollart_kv_poo
  *   Arithmetic: the codes and the query are converted to f16 (exact for the codes; a query element beyond the f16
  *   range, |q| > 65504, is not supported), fp32 scores, softmax and accumulation; softmax weights are rounded to f16
  *   before they multiply V.  Same schedule, same workspace, same errors as rollart_decode_attn.
+ * rollart_append_decode_attn_fp8: rollart_kv_append_fp8 of one new token per item followed by
+ *   rollart_decode_attn_fp8, in a single kernel launch; arguments as rollart_append_decode_attn plus the two scales.
+ *   Pool bytes, out and lse are identical to the two separate calls.
  * The paper does not describe a cache format; the fp8 pool is this library's option.
  */
 rollart_status rollart_kv_append_fp8(rollart_ctx *ctx, const rollart_kv_pool *pool, const rollart_trajs *trajs,
@@ -220,6 +223,11 @@ rollart_status rollart_decode_attn_fp8(rollart_ctx *ctx, const rollart_kv_pool *
                                        const int32_t *traj_ids, int32_t n_items, int32_t max_seq_len, const void *q,
                                        int32_t num_q_heads, float sm_scale, float k_scale, float v_scale, void *out,
                                        float *lse, void *stream);
+rollart_status rollart_append_decode_attn_fp8(rollart_ctx *ctx, const rollart_kv_pool *pool, const rollart_trajs *trajs,
+                                              const int32_t *traj_ids, int32_t n_items, int32_t max_seq_len,
+                                              const void *k_new, const void *v_new, const void *q, int32_t num_q_heads,
+                                              float sm_scale, float k_scale, float v_scale, void *out, float *lse,
+                                              int32_t *seq_lens_out, void *stream);
 
 /*
  * Group decode step: rollart_decode_attn for a batch whose items form groups that share a prompt prefix.

@@ -83,10 +83,11 @@ struct DecodeParams {
     float *lse;
     float scale_log2;           // sm_scale * log2(e) (times the K scale of an fp8 pool)
     float out_scale;            // 1, or the V scale of an fp8 pool: applied where a result is normalised
+    float k_inv_scale, v_inv_scale;   // fp8 fused append: 1 / scale of the pools
     int *tickets;               // per (item, kv head): pieces that have arrived; 0 between calls
     // fused append (all NULL for a plain decode call): the item's new K/V row is stored at position len and attended to
     const __nv_bfloat16 *k_new, *v_new;   // [n_items][num_kv_heads][128]
-    __nv_bfloat16 *k_pool, *v_pool;       // the pools, writable
+    void *k_pool, *v_pool;                // the pools, writable (bf16 or E4M3 bytes)
     int32_t *seq_lens_out;
     // group decode (NULL otherwise): per item, the first page_offset[i] pages of the table row are skipped
     const int32_t *page_offset;
@@ -648,6 +649,27 @@ decode_splitkv_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
             if constexpr (kFp8) {
                 // ---- fp8: this warp owns 32 keys of the 128-key tile, as two halves of 16 that share one softmax update ----
                 const int valid = min(32, pc.len - tile * kTK - key0);
+                bool patched = false;
+                if (prm.k_new != nullptr && tile == pc.ntiles - 1 && valid > 0 && pc.len - 1 - tile * kTK - key0 == valid - 1) {
+                    // Fused append: this warp owns the context's last key, which is the item's new token.  Its K/V row
+                    // comes from k_new / v_new (bf16): it is quantised and put into the staged tile (over whatever the
+                    // copy brought for that slot) and into the pool.  Lanes 0-15 move K, lanes 16-31 move V, 8 codes each.
+                    const int kk = valid - 1, c8 = lane & 15;
+                    const int t = s_traj[pc.item];
+                    const int pos = pc.len - 1;
+                    const int pg = __ldg(prm.page_table + static_cast<long long>(t) * prm.max_pages + pos / P);
+                    const long long src = (static_cast<long long>(pc.item) * hkv + pc.head) * (kHeadDim / 8) + c8;
+                    const uint4 val = __ldg(reinterpret_cast<const uint4 *>(lane < 16 ? prm.k_new : prm.v_new) + src);
+                    const uint2 code = quantize8(val, lane < 16 ? prm.k_inv_scale : prm.v_inv_scale);
+                    const uint32_t a = (lane < 16 ? kbase : vbase) + kk * 128 + (((c8 >> 1) ^ (kk & 7)) << 4) + (c8 & 1) * 8;
+                    asm volatile("st.shared.v2.b32 [%0], {%1,%2};" ::"r"(a), "r"(code.x), "r"(code.y) : "memory");
+                    if (pg >= 0 && pg < prm.num_pages) {     // a bad page id was already reported by the producer
+                        const long long dst = ((static_cast<long long>(pg) * hkv + pc.head) * P + pos % P) * (kHeadDim / 8) + c8;
+                        static_cast<uint2 *>(lane < 16 ? prm.k_pool : prm.v_pool)[dst] = code;
+                    }
+                    patched = true;
+                    __syncwarp();
+                }
                 if (valid > 0) {
                     if (valid < 32) {
                         // dead slots may hold anything (NaN codes included): zero their V rows so that 0 * v stays 0
@@ -727,7 +749,7 @@ decode_splitkv_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
                             mma_f16(o[4 * cp + 3], pa[hf], e4m3x2_to_f16x2_hi(x2), e4m3x2_to_f16x2_hi(x3));
                         }
                     }
-                    if (valid < 32) fence_proxy_async();   // our stores into the stage precede the next copy into it
+                    if (valid < 32 || patched) fence_proxy_async();   // our stores into the stage precede the next copy into it
                 }
             } else {
                 const int valid = min(16, pc.len - tile * kTile - key0);   // live keys among this warp's 16
@@ -747,7 +769,7 @@ decode_splitkv_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
                     asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(a), "r"(val.x), "r"(val.y), "r"(val.z), "r"(val.w) : "memory");
                     if (pg >= 0 && pg < prm.num_pages) {     // a bad page id was already reported by the producer
                         const long long dst = ((static_cast<long long>(pg) * hkv + pc.head) * P + pos % P) * (kHeadDim / 8) + c16;
-                        reinterpret_cast<uint4 *>(lane < 16 ? prm.k_pool : prm.v_pool)[dst] = val;
+                        static_cast<uint4 *>(lane < 16 ? prm.k_pool : prm.v_pool)[dst] = val;
                     }
                     patched = true;
                     __syncwarp();
@@ -1006,10 +1028,12 @@ cudaError_t launch_decode_attn(const AttnCall &c, cudaStream_t stream, int64_t *
         prm.lse = c.lse ? c.lse + static_cast<long long>(base) * c.num_q_heads : nullptr;
         prm.scale_log2 = c.sm_scale * kLog2e * (c.fp8 ? c.k_scale : 1.f);
         prm.out_scale = c.fp8 ? c.v_scale : 1.f;
+        prm.k_inv_scale = c.fp8 ? 1.f / c.k_scale : 1.f;
+        prm.v_inv_scale = c.fp8 ? 1.f / c.v_scale : 1.f;
         prm.tickets = static_cast<int *>(c.workspace);
         prm.k_new = c.k_new ? c.k_new + static_cast<long long>(base) * hkv * kHeadDim : nullptr;
         prm.v_new = c.v_new ? c.v_new + static_cast<long long>(base) * hkv * kHeadDim : nullptr;
-        prm.k_pool = const_cast<__nv_bfloat16 *>(c.pool.k); prm.v_pool = const_cast<__nv_bfloat16 *>(c.pool.v);
+        prm.k_pool = const_cast<__nv_bfloat16 *>(c.pool.k); prm.v_pool = const_cast<__nv_bfloat16 *>(c.pool.v);   // (bytes, for fp8)
         prm.seq_lens_out = c.seq_lens_out;
         prm.page_offset = c.page_offset ? c.page_offset + base : nullptr;
         prm.out_f32 = c.out_f32 ? c.out_f32 + static_cast<long long>(base) * c.num_q_heads * kHeadDim : nullptr;

@@ -25,21 +25,6 @@ __device__ __forceinline__ int find_item(const int32_t *__restrict__ indptr, int
     return lo;
 }
 
-// eight bf16 (one 16-byte piece of a row) -> eight E4M3 codes: code = nearest (ties to even, saturating at +-448) of
-// x * inv_scale, the product rounded to fp32 first
-__device__ __forceinline__ uint2 quantize8(const uint4 &v, float inv_scale) {
-    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-    uint32_t h[4];
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        const float lo = __uint_as_float(w[i] << 16) * inv_scale, hi = __uint_as_float(w[i] & 0xffff0000u) * inv_scale;
-        uint16_t p;
-        asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(p) : "f"(hi), "f"(lo));    // first operand -> upper byte
-        h[i] = p;
-    }
-    return make_uint2(h[0] | (h[1] << 16), h[2] | (h[3] << 16));
-}
-
 // kFp8: the pools hold E4M3 codes (rows of 128 B); the new rows arrive as bf16 and are quantised on the way.
 template <bool kFp8>
 __global__ void __launch_bounds__(kThreads)

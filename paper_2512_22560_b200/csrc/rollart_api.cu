@@ -342,10 +342,11 @@ rollart_status rollart_decode_attn_fp8(rollart_ctx *ctx, const rollart_kv_pool *
     return ROLLART_OK;
 }
 
-rollart_status rollart_append_decode_attn(rollart_ctx *ctx, const rollart_kv_pool *pool, const rollart_trajs *trajs,
-                                          const int32_t *traj_ids, int32_t n_items, int32_t max_seq_len, const void *k_new,
-                                          const void *v_new, const void *q, int32_t num_q_heads, float sm_scale, void *out,
-                                          float *lse, int32_t *seq_lens_out, void *stream) {
+namespace {
+rollart_status append_decode_impl(rollart_ctx *ctx, const rollart_kv_pool *pool, const rollart_trajs *trajs,
+                                  const int32_t *traj_ids, int32_t n_items, int32_t max_seq_len, const void *k_new,
+                                  const void *v_new, const void *q, int32_t num_q_heads, float sm_scale, void *out,
+                                  float *lse, int32_t *seq_lens_out, void *stream, bool fp8, float k_scale, float v_scale) {
     if (!ctx) return ROLLART_ERR_INVALID_ARG;
     rollart_status st = attn_common(ctx, pool, trajs, n_items, n_items, max_seq_len, q, num_q_heads, out);
     if (st != ROLLART_OK) return st;
@@ -366,6 +367,9 @@ rollart_status rollart_append_decode_attn(rollart_ctx *ctx, const rollart_kv_poo
     c.k_new = static_cast<const __nv_bfloat16 *>(k_new);
     c.v_new = static_cast<const __nv_bfloat16 *>(v_new);
     c.seq_lens_out = seq_lens_out;
+    c.fp8 = fp8;
+    c.k_scale = k_scale;
+    c.v_scale = v_scale;
     bool too_small = false;
     cudaError_t e = launch_decode_attn(c, static_cast<cudaStream_t>(stream), &ctx->launches, &too_small);
     if (too_small)
@@ -373,6 +377,27 @@ rollart_status rollart_append_decode_attn(rollart_ctx *ctx, const rollart_kv_poo
                     decode_workspace_bytes(n_items, num_q_heads, pool->num_kv_heads, max_seq_len, ctx->sm_count));
     if (e != cudaSuccess) return cuda_fail(ctx, e, "append_decode_attn launch");
     return ROLLART_OK;
+}
+}  // namespace
+
+rollart_status rollart_append_decode_attn(rollart_ctx *ctx, const rollart_kv_pool *pool, const rollart_trajs *trajs,
+                                          const int32_t *traj_ids, int32_t n_items, int32_t max_seq_len, const void *k_new,
+                                          const void *v_new, const void *q, int32_t num_q_heads, float sm_scale, void *out,
+                                          float *lse, int32_t *seq_lens_out, void *stream) {
+    return append_decode_impl(ctx, pool, trajs, traj_ids, n_items, max_seq_len, k_new, v_new, q, num_q_heads, sm_scale, out,
+                              lse, seq_lens_out, stream, false, 1.f, 1.f);
+}
+
+rollart_status rollart_append_decode_attn_fp8(rollart_ctx *ctx, const rollart_kv_pool *pool, const rollart_trajs *trajs,
+                                              const int32_t *traj_ids, int32_t n_items, int32_t max_seq_len,
+                                              const void *k_new, const void *v_new, const void *q, int32_t num_q_heads,
+                                              float sm_scale, float k_scale, float v_scale, void *out, float *lse,
+                                              int32_t *seq_lens_out, void *stream) {
+    if (!ctx) return ROLLART_ERR_INVALID_ARG;
+    if (!(k_scale > 0.f) || !(v_scale > 0.f) || !isfinite(k_scale) || !isfinite(v_scale))
+        return fail(ctx, ROLLART_ERR_INVALID_ARG, "k_scale and v_scale must be positive and finite");
+    return append_decode_impl(ctx, pool, trajs, traj_ids, n_items, max_seq_len, k_new, v_new, q, num_q_heads, sm_scale, out,
+                              lse, seq_lens_out, stream, true, k_scale, v_scale);
 }
 
 namespace {

@@ -28,6 +28,21 @@ __device__ __forceinline__ void report(DeviceStatus *st, int code, int detail, i
     }
 }
 
+// eight bf16 (one 16-byte piece of a row) -> eight E4M3 codes: code = nearest (ties to even, saturating at +-448) of
+// x * inv_scale, the product rounded to fp32 first
+__device__ __forceinline__ uint2 quantize8(const uint4 &v, float inv_scale) {
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    uint32_t h[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const float lo = __uint_as_float(w[i] << 16) * inv_scale, hi = __uint_as_float(w[i] & 0xffff0000u) * inv_scale;
+        uint16_t p;
+        asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(p) : "f"(hi), "f"(lo));    // first operand -> upper byte
+        h[i] = p;
+    }
+    return make_uint2(h[0] | (h[1] << 16), h[2] | (h[3] << 16));
+}
+
 struct PoolView {
     const __nv_bfloat16 *k;
     const __nv_bfloat16 *v;
@@ -91,7 +106,7 @@ struct AttnCall {
     const int32_t *page_offset;   // decode: per item, pages of the table row to skip (the keys before them are not attended to)
     const int32_t *shared_lens;   // chunk: per item, every query row of the item sees exactly the first shared_lens[i] keys
     float *out_f32;               // when set the result rows are written here in fp32 instead of bf16 to `out`
-    // fp8 (E4M3) pools, decode only: keys are k_scale * code value, values v_scale * code value
+    // fp8 (E4M3) pools (decode and fused append + decode): keys are k_scale * code value, values v_scale * code value
     bool fp8;
     float k_scale, v_scale;
 };

@@ -23,7 +23,7 @@ EXPORTS = (
     "rollart_obs_chunk_attn", "rollart_check", "rollart_last_error", "rollart_launch_count",
     "rollart_decode_attn_noalloc", "rollart_kv_gather", "rollart_pages_reserve", "rollart_pages_release",
     "rollart_append_decode_attn", "rollart_group_decode_attn", "rollart_group_decode_workspace_size",
-    "rollart_decode_attn_fp8", "rollart_kv_append_fp8",
+    "rollart_decode_attn_fp8", "rollart_kv_append_fp8", "rollart_append_decode_attn_fp8",
 )
 
 
@@ -73,6 +73,9 @@ def load_library() -> ctypes.CDLL:
     L.rollart_decode_attn.restype = ctypes.c_int
     L.rollart_decode_attn.argtypes = [vp, ctypes.POINTER(_KVPool), ctypes.POINTER(_Trajs), vp, i32, i32, vp, i32, f32,
                                       vp, vp, vp]
+    L.rollart_append_decode_attn_fp8.restype = ctypes.c_int
+    L.rollart_append_decode_attn_fp8.argtypes = [vp, ctypes.POINTER(_KVPool), ctypes.POINTER(_Trajs), vp, i32, i32, vp, vp, vp, i32,
+                                                 f32, f32, f32, vp, vp, vp, vp]
     L.rollart_kv_append_fp8.restype = ctypes.c_int
     L.rollart_kv_append_fp8.argtypes = [vp, ctypes.POINTER(_KVPool), ctypes.POINTER(_Trajs), vp, vp, i32, i32, vp, vp, f32, f32,
                                         vp, vp]
@@ -320,6 +323,28 @@ class Context:
             self._h, ctypes.byref(pool), ctypes.byref(trajs), _ptr(traj_ids, torch.int32, self.device), n_items,
             int(max_seq_len), _ptr(q, torch.bfloat16, self.device), hq, float(sm_scale), float(k_scale), float(v_scale),
             _ptr(out, torch.bfloat16, self.device), _ptr(lse, torch.float32, self.device), self._stream(stream))
+        if st != OK:
+            self._raise(st)
+
+    def append_decode_attn_fp8(self, k_pool, v_pool, page_table, seq_lens, k_new, v_new, q, sm_scale, k_scale, v_scale,
+                               max_seq_len, out, lse=None, traj_ids=None, seq_lens_out=None, stream=None) -> None:
+        pool = self._pool_fp8(k_pool, v_pool)
+        trajs = self._trajs(page_table, seq_lens)
+        if q.dim() != 3 or q.shape != out.shape:
+            raise ValueError("q and out must be [n_items][num_q_heads][head_dim]")
+        n_items, hq, _ = q.shape
+        if k_new.shape != v_new.shape or tuple(k_new.shape) != (n_items, pool.num_kv_heads, pool.head_dim):
+            raise ValueError("k_new/v_new must be [n_items][num_kv_heads][head_dim]")
+        if traj_ids is not None and traj_ids.shape[0] != n_items:
+            raise ValueError("traj_ids must have one entry per item")
+        if lse is not None and tuple(lse.shape) != (n_items, hq):
+            raise ValueError("lse must be [n_items][num_q_heads]")
+        st = self._lib.rollart_append_decode_attn_fp8(
+            self._h, ctypes.byref(pool), ctypes.byref(trajs), _ptr(traj_ids, torch.int32, self.device), n_items,
+            int(max_seq_len), _ptr(k_new, torch.bfloat16, self.device), _ptr(v_new, torch.bfloat16, self.device),
+            _ptr(q, torch.bfloat16, self.device), hq, float(sm_scale), float(k_scale), float(v_scale),
+            _ptr(out, torch.bfloat16, self.device), _ptr(lse, torch.float32, self.device),
+            _ptr(seq_lens_out, torch.int32, self.device), self._stream(stream))
         if st != OK:
             self._raise(st)
 

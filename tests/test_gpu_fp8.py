@@ -102,6 +102,44 @@ def test_append_of_chunks_saturation_and_scales(cuda_device):
     ctx.close()
 
 
+@pytest.mark.parametrize("i,T,div", [(0, 4, 1), (1, 16, 4), (3, 4, 16), (4, 10, 8)])
+def test_fused_fp8_step_equals_the_two_calls(cuda_device, i, T, div):
+    spec = W.CONFIGS[i] if i == 0 else W.shrink(W.CONFIGS[i], T, div, 16)
+    batch = W.make_batch(spec, seed=500 + i)
+    ids = batch.decode_ids
+    rows = torch.from_numpy(batch.decode_rows())
+    k8 = oracle.fp8_quantize_rows(W.bf16_to_u16(batch.k_pool), KS)
+    v8 = oracle.fp8_quantize_rows(W.bf16_to_u16(batch.v_pool), VS)
+    table, lens0 = dev_i32(batch.page_table, cuda_device), dev_i32(batch.seq_lens_before, cuda_device)
+    tid = dev_i32(ids, cuda_device)
+    q = batch.q_new[rows].contiguous().to(cuda_device)
+    kn, vn = batch.k_new[rows].contiguous().to(cuda_device), batch.v_new[rows].contiguous().to(cuda_device)
+    msl = int(batch.seq_lens_after.max())
+    ctx = make_ctx(spec, len(ids), msl)
+    res = []
+    for fused in (False, True):
+        dk, dv = torch.from_numpy(k8.copy()).to(cuda_device), torch.from_numpy(v8.copy()).to(cuda_device)
+        lens1 = lens0.clone()
+        out = torch.full_like(q, float("nan"))
+        lse = torch.full((len(ids), spec.num_q_heads), float("nan"), device=cuda_device)
+        if fused:
+            lens_out = torch.full_like(lens0, -7)
+            ctx.append_decode_attn_fp8(dk, dv, table, lens0, kn, vn, q, spec.sm_scale, KS, VS, msl, out, lse=lse, traj_ids=tid,
+                                       seq_lens_out=lens_out)
+            lens1[tid.long()] = lens_out[tid.long()]
+        else:
+            ctx.kv_append_fp8(dk, dv, table, lens0, dev_i32(np.arange(len(ids) + 1), cuda_device), kn, vn, KS, VS, traj_ids=tid,
+                              seq_lens_out=lens1)
+            ctx.decode_attn_fp8(dk, dv, table, lens1, q, spec.sm_scale, KS, VS, msl, out, lse=lse, traj_ids=tid)
+        ctx.check()
+        res.append((dk, dv, lens1, out, lse))
+    a, b = res
+    assert torch.equal(a[0], b[0]) and torch.equal(a[1], b[1]), "pool bytes differ"
+    assert torch.equal(a[2][tid.long()], b[2][tid.long()])
+    assert torch.equal(a[3].view(torch.int16), b[3].view(torch.int16)) and torch.equal(a[4], b[4])
+    ctx.close()
+
+
 def test_host_side_validation(cuda_device):
     spec = W.CONFIGS[0]
     b = W.make_batch(spec)
