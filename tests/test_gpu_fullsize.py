@@ -130,6 +130,56 @@ def test_full_size_decode_with_needles(cuda_device, cfg):
     ctx.close()
 
 
+@pytest.mark.parametrize("cfg", [1, 2, 3])
+def test_full_size_fp8_step_sampled(cuda_device, cfg):
+    # The fused fp8 step (quantised append + decode in one launch) at full size, as bench.py times it; the oracle
+    # recomputes sampled trajectories from a host copy of their pages' codes after the step.
+    spec = W.CONFIGS[cfg]
+    ks, vs = 0.03, 0.03
+    batch = W.make_batch(spec, device=cuda_device)
+    ids = batch.decode_ids
+    rows = batch.decode_rows()
+    msl = int(batch.seq_lens_after[ids].max())
+    ctx = make_ctx(spec, len(ids), msl)
+    # any codes will do for the existing cache (the oracle reads the same bytes): a clamped cast of the bf16 pools
+    k8 = (batch.k_pool.float() / ks).clamp_(-448, 448).to(torch.float8_e4m3fn).view(torch.uint8)
+    v8 = (batch.v_pool.float() / vs).clamp_(-448, 448).to(torch.float8_e4m3fn).view(torch.uint8)
+    table, lens0 = dev_i32(batch.page_table, cuda_device), dev_i32(batch.seq_lens_before, cuda_device)
+    lens1 = torch.full_like(lens0, -7)
+    ridx = torch.from_numpy(rows).to(cuda_device)
+    q, kn, vn = batch.q_new[ridx].contiguous(), batch.k_new[ridx].contiguous(), batch.v_new[ridx].contiguous()
+    out = torch.full_like(q, float("nan"))
+    lse = torch.full((len(ids), spec.num_q_heads), float("nan"), device=cuda_device)
+    tid = dev_i32(ids, cuda_device)
+    ctx.append_decode_attn_fp8(k8, v8, table, lens0, kn, vn, q, spec.sm_scale, ks, vs, msl, out, lse=lse, traj_ids=tid,
+                               seq_lens_out=lens1)
+    ctx.check()
+    assert torch.all(torch.isfinite(out.float())) and torch.all(torch.isfinite(lse))
+    rng = np.random.default_rng(40 + cfg)
+    pick = sample_ids(batch.seq_lens_before, ids, 4, rng)
+    import dataclasses
+    b8 = dataclasses.replace(batch)
+    b8.k_pool, b8.v_pool = k8, v8
+    post = W.extract_trajs(b8, pick)
+    kp, vp = post.k_pool.numpy(), post.v_pool.numpy()
+    where = {int(t): i for i, t in enumerate(ids)}
+    sel = torch.from_numpy(np.array([where[int(t)] for t in pick])).to(cuda_device)
+    ref_o, ref_l = oracle.decode_attn_fp8(kp, vp, post.page_table, post.seq_lens_before + 1, W.bf16_to_u16(q[sel]),
+                                          spec.sm_scale, ks, vs)
+    assert_attn_close(out[sel], ref_o, spec.name + " fp8")
+    assert_lse_close(lse[sel], ref_l, spec.name + " fp8")
+    # the appended token's codes are the oracle's quantisation of its row, at the slot the oracle's indexing names
+    P = spec.page_size
+    kq = oracle.fp8_quantize_rows(W.bf16_to_u16(kn[sel]), ks)
+    vq = oracle.fp8_quantize_rows(W.bf16_to_u16(vn[sel]), vs)
+    for i, t in enumerate(pick):
+        L = int(batch.seq_lens_before[t])
+        pg = int(post.page_table[i, L // P])
+        assert np.array_equal(kp[pg, :, L % P, :], kq[i]) and np.array_equal(vp[pg, :, L % P, :], vq[i])
+    assert torch.equal(lens1[tid.long()].cpu(), torch.from_numpy(batch.seq_lens_before[ids] + 1).to(torch.int32))
+    ctx.close()
+
+
 def db_as_batch(batch, db):
     """the batch with its pools replaced by the device pools after the GPU append"""
     import dataclasses
