@@ -380,9 +380,15 @@ class CpuBaseline:
 
     def measure(self):
         t, toks = self.run(self.take)
+        # a sample that finishes in a fraction of a second is repeated (fresh copies of the pools each pass) until
+        # about 1.5 s of wall time on all cores has gone by; the mean pass is reported
+        passes = [t]
+        while sum(passes) < 1.5 and len(passes) < 30:
+            passes.append(self.run(self.take)[0])
+        t = float(np.mean(passes))
         info = {"value": len(self.take) / t, "unit": UNIT, "cores": self.oracle.num_threads(), "kind": "oracle",
                 "sample": f"{len(self.take)} of {self.n_dec} trajectories of {self.spec.name} ({toks} context tokens), "
-                          f"append + decode, {t:.2f} s wall"}
+                          f"append + decode, mean of {len(passes)} passes of {t:.2f} s wall"}
         return info, t, len(self.take)
 
 
