@@ -565,6 +565,27 @@ def main():
                     torch.cuda.empty_cache()
                 except Exception as e:
                     extra[name] = {"error": repr(e)}
+            try:
+                # the tiny case lives in L2: a latency figure, back to back and after a write larger than L2
+                w0 = DecodeWorkload(W.CONFIGS[0], args.seed, device)
+                _, hot_ms = w0.time_steps(200, 10)
+                flush = torch.empty(256 << 20, dtype=torch.uint8, device=device)
+                ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(20)]
+                for a, b in ev:
+                    flush.fill_(1)
+                    a.record(); w0.step(); b.record()
+                torch.cuda.synchronize(device)
+                w0.ctx.check()
+                extra[W.CONFIGS[0].name] = {"step_us_back_to_back": hot_ms * 1e3,
+                                            "step_us_after_l2_flush": float(np.median([a.elapsed_time(b) for a, b in ev])) * 1e3,
+                                            "trajectories": w0.n_items, "kv_bytes": w0.bytes,
+                                            "note": "back to back = launch period (bounded below by the host's issue rate); "
+                                                    "after flush = events around one launch"}
+                w0.ctx.close()
+                del w0, flush
+                torch.cuda.empty_cache()
+            except Exception as e:
+                extra[W.CONFIGS[0].name] = {"error": repr(e)}
             for ci in (2, 3, 4):
                 try:
                     w2 = DecodeWorkload(W.CONFIGS[ci], args.seed, device)
