@@ -205,8 +205,8 @@ class DecodeWorkload:
 
     def time_e2e(self, steps: int, warmup: int):
         """Steps driven from HOST buffers: per step the new token's q/k/v go host->device from pinned
-        memory (one staging buffer, one copy) and the attention output comes back device->host, inside
-        the timed region."""
+        memory (one staging buffer, one copy) and the attention output goes device->host (the kernel stores it
+        into a pinned host buffer, no separate copy), inside the timed region."""
         nq, nk = self.q.numel(), self.k_new.numel()
         stage_dev = torch.empty(nq + 2 * nk, dtype=torch.bfloat16, device=self.device)
         stage_host = torch.cat([self.q.flatten(), self.k_new.flatten(), self.v_new.flatten()]).cpu().pin_memory()
@@ -215,11 +215,11 @@ class DecodeWorkload:
         self.k_new = stage_dev[nq:nq + nk].view_as(k_new)
         self.v_new = stage_dev[nq + nk:].view_as(v_new)
         hout = torch.empty_like(self.out, device="cpu").pin_memory()
+        dout, self.out = self.out, hout             # the kernel writes the result straight into the pinned host buffer
 
         def one():
             stage_dev.copy_(stage_host, non_blocking=True)
             self.step()
-            hout.copy_(self.out, non_blocking=True)
             torch.cuda.synchronize(self.device)     # the host consumes each step's result
 
         for _ in range(warmup):
@@ -228,7 +228,7 @@ class DecodeWorkload:
         for _ in range(steps):
             one()
         dt = time.perf_counter() - t0
-        self.q, self.k_new, self.v_new = q, k_new, v_new
+        self.q, self.k_new, self.v_new, self.out = q, k_new, v_new, dout
         return dt * 1e3, stage_host.numel() * 2, hout.numel() * 2
 
 
@@ -540,7 +540,7 @@ def main():
                          "algorithmic_bytes_per_launch": wl.bytes, "ms_per_launch": dec_ms},
             "e2e": {"value": n_items_all / (e2e_ms_step * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms_step,
-                    "note": "per step: q, k_new, v_new host->device from one pinned staging buffer, out device->host, host sync; the KV pool is resident engine state"},
+                    "note": "per step: q, k_new, v_new host->device from one pinned staging buffer, out written by the kernel into a pinned host buffer, host sync; the KV pool is resident engine state"},
             "gpu_launches": int(launches),
             "clocks": clocks.summary(),
         }

@@ -167,6 +167,10 @@ rollart_status rollart_pages_release(rollart_ctx *ctx, int32_t *free_pages, int3
  *
  *   q, out            [device] bf16 [n_items][num_q_heads][head_dim], 16-byte aligned.
  *   lse               [device] fp32 [n_items][num_q_heads] or NULL.
+ *                     out and lse are only stored to, so either may also be page-locked host memory that the
+ *                     device can address (cudaHostAlloc under unified addressing): the result then reaches the
+ *                     host with the kernel's own stores and is readable once the stream has been synchronised.
+ *                     The same holds for the fused and the fp8 decode calls below.
  *   max_seq_len       [host value] an upper bound on every L of this call; sizes the schedule and
  *                     the workspace check (values above max_pages_per_traj * page_size are
  *                     clamped to it).  A longer trajectory is reported as ROLLART_ERR_BOUNDS.

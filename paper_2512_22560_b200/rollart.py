@@ -114,9 +114,17 @@ def group_decode_workspace_size(max_items: int, num_q_heads: int, num_kv_heads: 
     return int(load_library().rollart_group_decode_workspace_size(max_items, num_q_heads, num_kv_heads, max_seq_len))
 
 
-def _ptr(t: Optional[torch.Tensor], dtype=None, device=None) -> Optional[int]:
+def _ptr(t: Optional[torch.Tensor], dtype=None, device=None, host_ok: bool = False) -> Optional[int]:
     if t is None:
         return None
+    if host_ok and not t.is_cuda:
+        # a result buffer may be page-locked host memory (mapped into the device's address space under unified
+        # addressing): the kernel then writes the result straight to the host
+        if not t.is_pinned() or not t.is_contiguous():
+            raise ValueError("a host result buffer must be a contiguous pinned tensor")
+        if dtype is not None and t.dtype != dtype:
+            raise ValueError(f"expected dtype {dtype}, got {t.dtype}")
+        return t.data_ptr()
     if not t.is_cuda or not t.is_contiguous():
         raise ValueError("expected a contiguous CUDA tensor")
     if dtype is not None and t.dtype != dtype:
@@ -304,7 +312,7 @@ class Context:
         st = self._lib.rollart_decode_attn(
             self._h, ctypes.byref(pool), ctypes.byref(trajs), _ptr(traj_ids, torch.int32, self.device), n_items,
             int(max_seq_len), _ptr(q, torch.bfloat16, self.device), hq, float(sm_scale),
-            _ptr(out, torch.bfloat16, self.device), _ptr(lse, torch.float32, self.device), self._stream(stream))
+            _ptr(out, torch.bfloat16, self.device, True), _ptr(lse, torch.float32, self.device, True), self._stream(stream))
         if st != OK:
             self._raise(st)
 
@@ -322,7 +330,7 @@ class Context:
         st = self._lib.rollart_decode_attn_fp8(
             self._h, ctypes.byref(pool), ctypes.byref(trajs), _ptr(traj_ids, torch.int32, self.device), n_items,
             int(max_seq_len), _ptr(q, torch.bfloat16, self.device), hq, float(sm_scale), float(k_scale), float(v_scale),
-            _ptr(out, torch.bfloat16, self.device), _ptr(lse, torch.float32, self.device), self._stream(stream))
+            _ptr(out, torch.bfloat16, self.device, True), _ptr(lse, torch.float32, self.device, True), self._stream(stream))
         if st != OK:
             self._raise(st)
 
@@ -343,7 +351,7 @@ class Context:
             self._h, ctypes.byref(pool), ctypes.byref(trajs), _ptr(traj_ids, torch.int32, self.device), n_items,
             int(max_seq_len), _ptr(k_new, torch.bfloat16, self.device), _ptr(v_new, torch.bfloat16, self.device),
             _ptr(q, torch.bfloat16, self.device), hq, float(sm_scale), float(k_scale), float(v_scale),
-            _ptr(out, torch.bfloat16, self.device), _ptr(lse, torch.float32, self.device),
+            _ptr(out, torch.bfloat16, self.device, True), _ptr(lse, torch.float32, self.device, True),
             _ptr(seq_lens_out, torch.int32, self.device), self._stream(stream))
         if st != OK:
             self._raise(st)
@@ -366,8 +374,8 @@ class Context:
         st = self._lib.rollart_append_decode_attn(
             self._h, ctypes.byref(pool), ctypes.byref(trajs), _ptr(traj_ids, torch.int32, self.device), n_items,
             int(max_seq_len), _ptr(k_new, torch.bfloat16, self.device), _ptr(v_new, torch.bfloat16, self.device),
-            _ptr(q, torch.bfloat16, self.device), hq, float(sm_scale), _ptr(out, torch.bfloat16, self.device),
-            _ptr(lse, torch.float32, self.device), _ptr(seq_lens_out, torch.int32, self.device), self._stream(stream))
+            _ptr(q, torch.bfloat16, self.device), hq, float(sm_scale), _ptr(out, torch.bfloat16, self.device, True),
+            _ptr(lse, torch.float32, self.device, True), _ptr(seq_lens_out, torch.int32, self.device), self._stream(stream))
         if st != OK:
             self._raise(st)
 

@@ -203,3 +203,32 @@ def test_fused_append_decode_equals_the_two_calls_and_the_oracle(cuda_device, i,
     ctx.decode_attn(db.k_pool, db.v_pool, db.page_table, lens_out, q, spec.sm_scale, msl, out2, traj_ids=dev_i32(ids, cuda_device))
     ctx.check()
     assert torch.equal(out.view(torch.int16), out2.view(torch.int16))
+
+
+@pytest.mark.parametrize("i,T,div", [(0, 4, 1), (1, 16, 4), (3, 4, 16)])
+def test_results_written_straight_to_pinned_host_memory(cuda_device, i, T, div):
+    """out / lse may be page-locked host tensors: the kernel's stores then cross to the host; same bits as device buffers."""
+    batch = W.make_batch(W.shrink(W.CONFIGS[i], T, div, 16), seed=700 + i)
+    spec = batch.spec
+    ids, rows = batch.decode_ids, batch.decode_rows()
+    msl = int(batch.seq_lens_after.max())
+    ctx = make_ctx(spec, len(ids), msl)
+    db = DeviceBatch(batch, cuda_device)
+    db.append(ctx)
+    q = db.q_new[torch.from_numpy(rows).to(cuda_device)].contiguous()
+    tid = dev_i32(ids, cuda_device)
+    out_d = torch.full_like(q, float("nan"))
+    lse_d = torch.full((len(ids), spec.num_q_heads), float("nan"), device=cuda_device)
+    ctx.decode_attn(db.k_pool, db.v_pool, db.page_table, db.lens_after, q, spec.sm_scale, msl, out_d, lse=lse_d, traj_ids=tid)
+    out_h = torch.full(tuple(q.shape), float("nan"), dtype=torch.bfloat16).pin_memory()
+    lse_h = torch.full(tuple(lse_d.shape), float("nan")).pin_memory()
+    ctx.decode_attn(db.k_pool, db.v_pool, db.page_table, db.lens_after, q, spec.sm_scale, msl, out_h, lse=lse_h, traj_ids=tid)
+    ctx.check()                                                       # synchronises the stream: the host may read now
+    assert torch.equal(out_h.view(torch.int16), out_d.cpu().view(torch.int16)) and torch.equal(lse_h, lse_d.cpu())
+    kp, vp, after = oracle_append(batch)
+    ref_o, _ = oracle.decode_attn(kp, vp, batch.page_table, after, W.bf16_to_u16(batch.q_new[rows]), spec.sm_scale, traj_ids=ids)
+    assert_attn_close(out_h, ref_o, spec.name + " host out")
+    with pytest.raises(ValueError):
+        ctx.decode_attn(db.k_pool, db.v_pool, db.page_table, db.lens_after, q, spec.sm_scale, msl,
+                        torch.empty(tuple(q.shape), dtype=torch.bfloat16), traj_ids=tid)          # pageable host memory
+    ctx.close()
