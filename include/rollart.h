@@ -217,6 +217,11 @@ rollart_status rollart_append_decode_attn(rollart_ctx *ctx, const rollart_kv_poo
  * rollart_append_decode_attn_fp8: rollart_kv_append_fp8 of one new token per item followed by
  *   rollart_decode_attn_fp8, in a single kernel launch; arguments as rollart_append_decode_attn plus the two scales.
  *   Pool bytes, out and lse are identical to the two separate calls.
+ * rollart_kv_gather_fp8 / rollart_kv_append_fp8_codes: the hand-over of an fp8 cache to another worker (Sec. 6.3), as
+ *   rollart_kv_gather / rollart_kv_append do it for bf16 pools.  The gather copies the codes of the first n_i tokens of
+ *   each listed trajectory into k_out / v_out ([device] uint8 [total_rows][num_kv_heads][head_dim], 16-byte aligned);
+ *   the append stores rows of codes (k_codes / v_codes, same layout) onto the receiving pool's pages.  Both are bit
+ *   copies: the scales travel with the caller and must be the same on both sides.  Errors as for the bf16 calls.
  * The paper does not describe a cache format; the fp8 pool is this library's option.
  */
 rollart_status rollart_kv_append_fp8(rollart_ctx *ctx, const rollart_kv_pool *pool, const rollart_trajs *trajs,
@@ -232,6 +237,15 @@ rollart_status rollart_append_decode_attn_fp8(rollart_ctx *ctx, const rollart_kv
                                               const void *k_new, const void *v_new, const void *q, int32_t num_q_heads,
                                               float sm_scale, float k_scale, float v_scale, void *out, float *lse,
                                               int32_t *seq_lens_out, void *stream);
+
+rollart_status rollart_kv_gather_fp8(rollart_ctx *ctx, const rollart_kv_pool *pool, const rollart_trajs *trajs,
+                                     const int32_t *traj_ids, const int32_t *out_indptr, int32_t n_items, int32_t total_rows,
+                                     void *k_out, void *v_out, void *stream);
+
+rollart_status rollart_kv_append_fp8_codes(rollart_ctx *ctx, const rollart_kv_pool *pool, const rollart_trajs *trajs,
+                                           const int32_t *traj_ids, const int32_t *new_indptr, int32_t n_items,
+                                           int32_t total_new, const void *k_codes, const void *v_codes,
+                                           int32_t *seq_lens_out, void *stream);
 
 /*
  * Group decode step: rollart_decode_attn for a batch whose items form groups that share a prompt prefix.

@@ -264,6 +264,22 @@ def kv_append_fp8(k_pool: np.ndarray, v_pool: np.ndarray, page_table, seq_lens, 
                      kq.view(np.uint16), vq.view(np.uint16), traj_ids=traj_ids)
 
 
+def kv_append_fp8_codes(k_pool: np.ndarray, v_pool: np.ndarray, page_table, seq_lens, new_indptr, k_codes, v_codes,
+                        traj_ids=None) -> np.ndarray:
+    """Append of rows that already hold codes (uint8 [total][Hkv][D]) into uint8 pools: the bit copy of kv_append,
+    a row of D bytes moved as D / 2 16-bit units (Sec. 6.3: the receiving side of a cache hand-over)."""
+    assert k_pool.dtype == np.uint8 and v_pool.dtype == np.uint8 and k_pool.shape[-1] % 2 == 0
+    return kv_append(k_pool.view(np.uint16), v_pool.view(np.uint16), page_table, seq_lens, new_indptr,
+                     _c(k_codes, np.uint8).view(np.uint16), _c(v_codes, np.uint8).view(np.uint16), traj_ids=traj_ids)
+
+
+def kv_gather_fp8(k_pool: np.ndarray, v_pool: np.ndarray, page_table, seq_lens, out_indptr, traj_ids=None):
+    """kv_gather over uint8 pools of codes: (k_out, v_out) uint8 [total][Hkv][D] (Sec. 6.3: the sending side)."""
+    assert k_pool.dtype == np.uint8 and v_pool.dtype == np.uint8 and k_pool.shape[-1] % 2 == 0
+    k16, v16 = kv_gather(k_pool.view(np.uint16), v_pool.view(np.uint16), page_table, seq_lens, out_indptr, traj_ids=traj_ids)
+    return k16.view(np.uint8), v16.view(np.uint8)
+
+
 def fp8_pool_as_bf16_bits(pool: np.ndarray) -> np.ndarray:
     """The pool's values (unit scale) as bf16 bit patterns: every finite E4M3 value is a bf16 value, so this is exact.
     NaN codes become bf16 NaN."""

@@ -177,7 +177,7 @@ namespace {
 rollart_status append_impl(rollart_ctx *ctx, const rollart_kv_pool *pool, const rollart_trajs *trajs,
                            const int32_t *traj_ids, const int32_t *new_indptr, int32_t n_items, int32_t total_new,
                            const void *k_new, const void *v_new, int32_t *seq_lens_out, void *stream, bool fp8,
-                           float k_scale, float v_scale) {
+                           float k_scale, float v_scale, bool rows_are_codes = false) {
     if (!ctx) return ROLLART_ERR_INVALID_ARG;
     rollart_status st;
     if ((st = check_pool(ctx, pool)) != ROLLART_OK) return st;
@@ -196,7 +196,8 @@ rollart_status append_impl(rollart_ctx *ctx, const rollart_kv_pool *pool, const 
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return fail(ctx, ROLLART_ERR_CUDA, "cannot select device %d", ctx->device);
     cudaError_t e = launch_kv_append(*pool, *trajs, traj_ids, new_indptr, n_items, total_new, k_new, v_new, seq_lens_out,
-                                     ctx->d_status, static_cast<cudaStream_t>(stream), &ctx->launches, fp8, k_scale, v_scale);
+                                     ctx->d_status, static_cast<cudaStream_t>(stream), &ctx->launches, fp8, k_scale, v_scale,
+                                     rows_are_codes);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "kv_append launch");
     return ROLLART_OK;
 }
@@ -221,9 +222,18 @@ rollart_status rollart_kv_append_fp8(rollart_ctx *ctx, const rollart_kv_pool *po
                        k_scale, v_scale);
 }
 
-rollart_status rollart_kv_gather(rollart_ctx *ctx, const rollart_kv_pool *pool, const rollart_trajs *trajs,
-                                 const int32_t *traj_ids, const int32_t *out_indptr, int32_t n_items, int32_t total_rows,
-                                 void *k_out, void *v_out, void *stream) {
+rollart_status rollart_kv_append_fp8_codes(rollart_ctx *ctx, const rollart_kv_pool *pool, const rollart_trajs *trajs,
+                                           const int32_t *traj_ids, const int32_t *new_indptr, int32_t n_items,
+                                           int32_t total_new, const void *k_codes, const void *v_codes,
+                                           int32_t *seq_lens_out, void *stream) {
+    return append_impl(ctx, pool, trajs, traj_ids, new_indptr, n_items, total_new, k_codes, v_codes, seq_lens_out, stream, true,
+                       1.f, 1.f, true);
+}
+
+namespace {
+rollart_status gather_impl(rollart_ctx *ctx, const rollart_kv_pool *pool, const rollart_trajs *trajs,
+                           const int32_t *traj_ids, const int32_t *out_indptr, int32_t n_items, int32_t total_rows,
+                           void *k_out, void *v_out, void *stream, bool fp8) {
     if (!ctx) return ROLLART_ERR_INVALID_ARG;
     rollart_status st;
     if ((st = check_pool(ctx, pool)) != ROLLART_OK) return st;
@@ -235,9 +245,22 @@ rollart_status rollart_kv_gather(rollart_ctx *ctx, const rollart_kv_pool *pool, 
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return fail(ctx, ROLLART_ERR_CUDA, "cannot select device %d", ctx->device);
     cudaError_t e = launch_kv_gather(*pool, *trajs, traj_ids, out_indptr, n_items, total_rows, k_out, v_out, ctx->d_status,
-                                     static_cast<cudaStream_t>(stream), &ctx->launches);
+                                     static_cast<cudaStream_t>(stream), &ctx->launches, fp8);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "kv_gather launch");
     return ROLLART_OK;
+}
+}  // namespace
+
+rollart_status rollart_kv_gather(rollart_ctx *ctx, const rollart_kv_pool *pool, const rollart_trajs *trajs,
+                                 const int32_t *traj_ids, const int32_t *out_indptr, int32_t n_items, int32_t total_rows,
+                                 void *k_out, void *v_out, void *stream) {
+    return gather_impl(ctx, pool, trajs, traj_ids, out_indptr, n_items, total_rows, k_out, v_out, stream, false);
+}
+
+rollart_status rollart_kv_gather_fp8(rollart_ctx *ctx, const rollart_kv_pool *pool, const rollart_trajs *trajs,
+                                     const int32_t *traj_ids, const int32_t *out_indptr, int32_t n_items, int32_t total_rows,
+                                     void *k_out, void *v_out, void *stream) {
+    return gather_impl(ctx, pool, trajs, traj_ids, out_indptr, n_items, total_rows, k_out, v_out, stream, true);
 }
 
 static rollart_status pages_common(rollart_ctx *ctx, bool reserve, int32_t *free_pages, int32_t *free_count, int32_t capacity,

@@ -60,11 +60,12 @@ struct TrajView {
 cudaError_t launch_kv_append(const rollart_kv_pool &pool, const rollart_trajs &trajs, const int32_t *traj_ids,
                              const int32_t *new_indptr, int n_items, int total_new, const void *k_new,
                              const void *v_new, int32_t *seq_lens_out, DeviceStatus *status, cudaStream_t stream,
-                             int64_t *launches, bool fp8 = false, float k_scale = 1.f, float v_scale = 1.f);
+                             int64_t *launches, bool fp8 = false, float k_scale = 1.f, float v_scale = 1.f,
+                             bool rows_are_codes = false);
 
 cudaError_t launch_kv_gather(const rollart_kv_pool &pool, const rollart_trajs &trajs, const int32_t *traj_ids,
                              const int32_t *out_indptr, int n_items, int total_rows, void *k_out, void *v_out,
-                             DeviceStatus *status, cudaStream_t stream, int64_t *launches);
+                             DeviceStatus *status, cudaStream_t stream, int64_t *launches, bool fp8 = false);
 
 cudaError_t launch_pages(bool reserve, int32_t *free_pages, int32_t *free_count, int capacity, int page_size,
                          int32_t *page_table, int max_pages, int32_t *seq_lens, int num_traj, const int32_t *traj_ids,

@@ -24,6 +24,7 @@ EXPORTS = (
     "rollart_decode_attn_noalloc", "rollart_kv_gather", "rollart_pages_reserve", "rollart_pages_release",
     "rollart_append_decode_attn", "rollart_group_decode_attn", "rollart_group_decode_workspace_size",
     "rollart_decode_attn_fp8", "rollart_kv_append_fp8", "rollart_append_decode_attn_fp8",
+    "rollart_kv_gather_fp8", "rollart_kv_append_fp8_codes",
 )
 
 
@@ -66,6 +67,10 @@ def load_library() -> ctypes.CDLL:
     L.rollart_kv_append.argtypes = [vp, ctypes.POINTER(_KVPool), ctypes.POINTER(_Trajs), vp, vp, i32, i32, vp, vp, vp, vp]
     L.rollart_kv_gather.restype = ctypes.c_int
     L.rollart_kv_gather.argtypes = [vp, ctypes.POINTER(_KVPool), ctypes.POINTER(_Trajs), vp, vp, i32, i32, vp, vp, vp]
+    L.rollart_kv_gather_fp8.restype = ctypes.c_int
+    L.rollart_kv_gather_fp8.argtypes = L.rollart_kv_gather.argtypes
+    L.rollart_kv_append_fp8_codes.restype = ctypes.c_int
+    L.rollart_kv_append_fp8_codes.argtypes = L.rollart_kv_append.argtypes
     L.rollart_pages_reserve.restype = ctypes.c_int
     L.rollart_pages_reserve.argtypes = [vp, vp, vp, i32, vp, i32, vp, i32, vp, vp, i32, vp]
     L.rollart_pages_release.restype = ctypes.c_int
@@ -295,6 +300,42 @@ class Context:
             self._h, ctypes.byref(pool), ctypes.byref(trajs), _ptr(traj_ids, torch.int32, self.device),
             _ptr(out_indptr, torch.int32, self.device), n_items, k_out.shape[0], _ptr(k_out, torch.bfloat16, self.device),
             _ptr(v_out, torch.bfloat16, self.device), self._stream(stream))
+        if st != OK:
+            self._raise(st)
+
+    def kv_gather_fp8(self, k_pool, v_pool, page_table, seq_lens, out_indptr, k_out, v_out, traj_ids=None, stream=None) -> None:
+        """kv_gather for pools of E4M3 codes: k_out / v_out are uint8 [total_rows][num_kv_heads][head_dim]"""
+        pool = self._pool_fp8(k_pool, v_pool)
+        trajs = self._trajs(page_table, seq_lens)
+        n_items = out_indptr.shape[0] - 1
+        if k_out.shape != v_out.shape or tuple(k_out.shape[1:]) != (pool.num_kv_heads, pool.head_dim):
+            raise ValueError("k_out/v_out must be [total_rows][num_kv_heads][head_dim]")
+        if traj_ids is not None and traj_ids.shape[0] != n_items:
+            raise ValueError("traj_ids must have one entry per item")
+        st = self._lib.rollart_kv_gather_fp8(
+            self._h, ctypes.byref(pool), ctypes.byref(trajs), _ptr(traj_ids, torch.int32, self.device),
+            _ptr(out_indptr, torch.int32, self.device), n_items, k_out.shape[0], _ptr(k_out, torch.uint8, self.device),
+            _ptr(v_out, torch.uint8, self.device), self._stream(stream))
+        if st != OK:
+            self._raise(st)
+
+    def kv_append_fp8_codes(self, k_pool, v_pool, page_table, seq_lens, new_indptr, k_codes, v_codes, traj_ids=None,
+                            seq_lens_out=None, stream=None) -> None:
+        """kv_append of rows that already hold E4M3 codes (uint8 [total_new][num_kv_heads][head_dim]): a bit copy"""
+        pool = self._pool_fp8(k_pool, v_pool)
+        trajs = self._trajs(page_table, seq_lens)
+        n_items = new_indptr.shape[0] - 1
+        total_new = k_codes.shape[0]
+        if k_codes.shape != v_codes.shape or tuple(k_codes.shape[1:]) != (pool.num_kv_heads, pool.head_dim):
+            raise ValueError("k_codes/v_codes must be [total_new][num_kv_heads][head_dim]")
+        if traj_ids is not None and traj_ids.shape[0] != n_items:
+            raise ValueError("traj_ids must have one entry per item")
+        if seq_lens_out is not None and seq_lens_out.shape != seq_lens.shape:
+            raise ValueError("seq_lens_out must have the shape of seq_lens")
+        st = self._lib.rollart_kv_append_fp8_codes(
+            self._h, ctypes.byref(pool), ctypes.byref(trajs), _ptr(traj_ids, torch.int32, self.device),
+            _ptr(new_indptr, torch.int32, self.device), n_items, total_new, _ptr(k_codes, torch.uint8, self.device),
+            _ptr(v_codes, torch.uint8, self.device), _ptr(seq_lens_out, torch.int32, self.device), self._stream(stream))
         if st != OK:
             self._raise(st)
 

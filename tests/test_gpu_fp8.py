@@ -157,3 +157,61 @@ def test_host_side_validation(cuda_device):
     with pytest.raises(ValueError):
         ctx.decode_attn_fp8(b.k_pool.to(cuda_device), b.v_pool.to(cuda_device), table, lens, q, spec.sm_scale, 1.0, 1.0, 600, out)
     ctx.close()
+
+
+@pytest.mark.parametrize("i,T,div", [(0, 4, 1), (3, 3, 32), (4, 9, 16)])
+def test_hand_over_of_an_fp8_cache(cuda_device, i, T, div):
+    """gather the codes of whole trajectories, append them onto another worker's pool: every byte against the oracle,
+    and decode attention over the received cache equals decode attention over the sender's."""
+    batch = W.make_batch(W.shrink(W.CONFIGS[i], T, div, 8), seed=600 + i)
+    spec = batch.spec
+    P, H = spec.page_size, spec.num_kv_heads
+    k8 = oracle.fp8_quantize_rows(W.bf16_to_u16(batch.k_pool), KS)
+    v8 = oracle.fp8_quantize_rows(W.bf16_to_u16(batch.v_pool), VS)
+    dk, dv = torch.from_numpy(k8.copy()).to(cuda_device), torch.from_numpy(v8.copy()).to(cuda_device)
+    table, lens0 = dev_i32(batch.page_table, cuda_device), dev_i32(batch.seq_lens_before, cuda_device)
+    ctx = make_ctx(spec, T, int(batch.seq_lens_before.max()) + 1)
+    ids = np.array(sorted(range(T), key=lambda t: -t)[: max(2, T - 1)], np.int32)      # a subset in reverse order
+    lens = batch.seq_lens_before[ids]
+    indptr = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    total = int(indptr[-1])
+    k_out = torch.full((total, H, 128), 0xEE, dtype=torch.uint8, device=cuda_device)
+    v_out = torch.full_like(k_out, 0xEE)
+    ctx.kv_gather_fp8(dk, dv, table, lens0, dev_i32(indptr, cuda_device), k_out, v_out, traj_ids=dev_i32(ids, cuda_device))
+    ctx.check()
+    ko, vo = oracle.kv_gather_fp8(k8, v8, batch.page_table, batch.seq_lens_before, indptr, traj_ids=ids)
+    assert np.array_equal(k_out.cpu().numpy(), ko) and np.array_equal(v_out.cpu().numpy(), vo)
+    # the receiving worker: empty trajectories on their own pages, pool bytes poisoned
+    pages = (lens.astype(np.int64) + P - 1) // P
+    table2, num_pages2 = W.build_page_table(pages, 0.25, np.random.default_rng(9))
+    k2 = np.full((num_pages2, H, P, 128), 0x7F, np.uint8)
+    v2 = np.full((num_pages2, H, P, 128), 0xFF, np.uint8)
+    dk2, dv2 = torch.from_numpy(k2.copy()).to(cuda_device), torch.from_numpy(v2.copy()).to(cuda_device)
+    zero = dev_i32(np.zeros(len(ids)), cuda_device)
+    after = torch.empty_like(zero)
+    ctx.kv_append_fp8_codes(dk2, dv2, dev_i32(table2, cuda_device), zero, dev_i32(indptr, cuda_device), k_out, v_out,
+                            seq_lens_out=after)
+    ctx.check()
+    ref_after = oracle.kv_append_fp8_codes(k2, v2, table2, np.zeros(len(ids), np.int32), indptr, ko, vo)
+    assert np.array_equal(after.cpu().numpy(), ref_after) and np.array_equal(ref_after, lens)
+    assert np.array_equal(dk2.cpu().numpy(), k2) and np.array_equal(dv2.cpu().numpy(), v2)
+    # decode over the received cache == decode over the sender's, bit for bit; and both within tolerance of the oracle
+    live = np.flatnonzero(lens > 0)
+    q = batch.q_new[: len(live)].contiguous().to(cuda_device)
+    o1, o2 = torch.full_like(q, float("nan")), torch.full_like(q, float("nan"))
+    msl = int(lens.max())
+    ctx.decode_attn_fp8(dk, dv, table, lens0, q, spec.sm_scale, KS, VS, msl, o1, traj_ids=dev_i32(ids[live], cuda_device))
+    ctx.decode_attn_fp8(dk2, dv2, dev_i32(table2, cuda_device), after, q, spec.sm_scale, KS, VS, msl, o2,
+                        traj_ids=dev_i32(live, cuda_device))
+    ctx.check()
+    assert torch.equal(o1.view(torch.int16), o2.view(torch.int16))
+    ref_o, _ = oracle.decode_attn_fp8(k2, v2, table2, ref_after, W.bf16_to_u16(batch.q_new[: len(live)]), spec.sm_scale, KS, VS,
+                                      traj_ids=live.astype(np.int32))
+    assert_attn_close(o2, ref_o, spec.name + " fp8 hand-over")
+    # asking for more rows than a trajectory holds is reported, not read
+    bad = indptr.copy()
+    bad[-1] += 1
+    big = torch.zeros(total + 1, H, 128, dtype=torch.uint8, device=cuda_device)
+    ctx.kv_gather_fp8(dk, dv, table, lens0, dev_i32(bad, cuda_device), big, big.clone(), traj_ids=dev_i32(ids, cuda_device))
+    assert ctx.status() == rollart.ERR_BOUNDS and "kv_gather" in ctx.last_error()
+    ctx.close()

@@ -104,3 +104,37 @@ def test_fp8_attention_equals_bf16_attention_on_the_dequantised_pool():
         w = np.exp(s - s.max())
         np.testing.assert_allclose(out[0, hq], 2.0 * (w @ vv[h]) / w.sum(), rtol=1e-12, atol=1e-12)
         np.testing.assert_allclose(lse[0, hq], s.max() + math.log(w.sum()), rtol=1e-12)
+
+
+def test_hand_over_of_codes_is_a_bit_copy_token_by_token():
+    # gather then append onto another pool with another page table: every live token's codes arrive unchanged, in
+    # order; checked with plain loops over (trajectory, position)
+    rng = np.random.default_rng(2)
+    P, H, D = 16, 3, 128
+    src_k = rng.integers(0, 256, (7, H, P, D)).astype(np.uint8)
+    src_v = rng.integers(0, 256, (7, H, P, D)).astype(np.uint8)
+    table = np.array([[5, 0, 3], [6, 2, -1], [1, 4, -1]], np.int32)
+    lens = np.array([40, 17, 0], np.int32)
+    ids = np.array([1, 0], np.int32)                                          # hand over trajectory 1, then 0
+    n = np.array([17, 33], np.int32)                                          # all of 1, the first 33 tokens of 0
+    indptr = np.array([0, 17, 50], np.int32)
+    gk, gv = oracle.kv_gather_fp8(src_k, src_v, table, lens, indptr, traj_ids=ids)
+    assert gk.shape == (50, H, D) and gk.dtype == np.uint8
+    for i, t in enumerate(ids):
+        for pos in range(n[i]):
+            assert np.array_equal(gk[indptr[i] + pos], src_k[table[t, pos // P], :, pos % P])
+            assert np.array_equal(gv[indptr[i] + pos], src_v[table[t, pos // P], :, pos % P])
+    dst_k = np.full((6, H, P, D), 0x55, np.uint8)
+    dst_v = np.full((6, H, P, D), 0xAA, np.uint8)
+    dtable = np.array([[2, 0, 4], [1, 5, 3]], np.int32)
+    dlens = np.array([3, 0], np.int32)                                        # receiver 0 already holds 3 tokens
+    after = oracle.kv_append_fp8_codes(dst_k, dst_v, dtable, dlens, indptr, gk, gv)
+    assert list(after) == [20, 33]
+    touched = np.zeros((6, P), bool)
+    for i in range(2):
+        for r in range(n[i]):
+            pos = dlens[i] + r
+            pg = dtable[i, pos // P]
+            assert np.array_equal(dst_k[pg, :, pos % P], gk[indptr[i] + r]) and np.array_equal(dst_v[pg, :, pos % P], gv[indptr[i] + r])
+            touched[pg, pos % P] = True
+    assert np.all(dst_k[~touched[:, None, :].repeat(H, 1)] == 0x55) and np.all(dst_v[~touched[:, None, :].repeat(H, 1)] == 0xAA)
