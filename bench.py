@@ -337,6 +337,36 @@ class ChunkWorkload:
         return (float(np.mean([e[0].elapsed_time(e[1]) for e in ev])), float(np.mean([e[1].elapsed_time(e[2]) for e in ev])))
 
 
+    def time_fp8(self, steps: int, warmup: int, k_scale: float = 0.03, v_scale: float = 0.03):
+        """The same half over fp8 (E4M3) pools: quantising append of the chunks, then chunk attention over the fp8 cache
+        (expansion of the listed contexts to bf16 into a scratch pool + the bf16 kernel).  (append ms, attention ms)"""
+        from paper_2512_22560_b200 import rollart
+        b, spec = self.batch, self.spec
+        k8 = (b.k_pool.float() * (1.0 / k_scale)).to(torch.float8_e4m3fn).view(torch.uint8)
+        v8 = (b.v_pool.float() * (1.0 / v_scale)).to(torch.float8_e4m3fn).view(torch.uint8)
+        need = rollart.obs_chunk_fp8_scratch_size(len(b.chunk_ids), spec.num_kv_heads, spec.page_size, self.max_seq_len)
+        scratch = torch.empty(need, dtype=torch.uint8, device=self.device)
+
+        def append():
+            self.ctx.kv_append_fp8(k8, v8, self.table, self.lens0, self.q_indptr, self.k_new, self.v_new, k_scale, v_scale,
+                                   traj_ids=self.traj_ids, seq_lens_out=self.lens1)
+
+        def attend():
+            self.ctx.obs_chunk_attn_fp8(k8, v8, self.table, self.lens1, self.q_indptr, self.q, spec.sm_scale, k_scale, v_scale,
+                                        self.max_seq_len, self.out, scratch, traj_ids=self.traj_ids)
+
+        for _ in range(warmup):
+            append(); attend()
+        torch.cuda.synchronize(self.device)
+        ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(steps)]
+        for i in range(steps):
+            ev[i][0].record(); append(); ev[i][1].record(); attend(); ev[i][2].record()
+        torch.cuda.synchronize(self.device)
+        self.ctx.check()
+        return (float(np.mean([e[0].elapsed_time(e[1]) for e in ev])), float(np.mean([e[1].elapsed_time(e[2]) for e in ev])),
+                need)
+
+
 class CpuBaseline:
     """The oracle, as it stands, timed on a bounded sample of the workload's trajectories."""
 
@@ -618,6 +648,14 @@ def main():
                     "chunk_rows": cw.rows, "chunk_attn_ms": att_ms, "tflops": tfs, "frac_of_measured_bf16_sustained": tfs / tf_peak,
                     "append_ms": app_ms, "append_gbs": cw.append_bytes / (app_ms * 1e-3) / 1e9,
                     "append_frac_of_measured_hbm": cw.append_bytes / (app_ms * 1e-3) / 1e9 / peak}
+                try:
+                    a8, t8, need = cw.time_fp8(5, 2)
+                    extra["cfg4_mixed_multiturn_chunk_half_fp8_pool"] = {
+                        "chunk_attn_ms": t8, "bf16_chunk_attn_ms": att_ms, "ratio_to_bf16": t8 / att_ms,
+                        "tflops": cw.flops / (t8 * 1e-3) / 1e12, "append_ms": a8, "scratch_bytes": need,
+                        "launches": 2, "note": "contexts expanded to bf16 into the scratch pool, then the bf16 kernel"}
+                except Exception as e:
+                    extra["cfg4_mixed_multiturn_chunk_half_fp8_pool"] = {"error": repr(e)}
                 cw.ctx.close()
                 del cw
                 torch.cuda.empty_cache()

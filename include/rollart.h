@@ -292,6 +292,28 @@ rollart_status rollart_obs_chunk_attn(rollart_ctx *ctx, const rollart_kv_pool *p
                                       float sm_scale, void *out, float *lse, void *stream);
 
 /*
+ * Observation-chunk attention over fp8 pools (pool->k_pool / v_pool hold E4M3 codes as for rollart_decode_attn_fp8;
+ * the chunk's own tokens have been appended with rollart_kv_append_fp8).  Same rows, mask and formula as
+ * rollart_obs_chunk_attn with keys k_scale * value(code) and values v_scale * value(code):
+ *   s_j = sm_scale * k_scale * <q, value(K code)>,  out = v_scale * sum_j softmax(s)_j * value(V code).
+ * This phase is bound by the tensor cores, not by reading the cache (Sec. 3.1), so the call first expands the listed
+ * trajectories' contexts to bf16 (exact: every finite E4M3 value is a bf16 value) into `scratch` and then runs the
+ * bf16 kernel over that copy; the expansion is one pass at the HBM rate, a few per cent of the attention.
+ *   scratch        [device] 256-byte aligned, at least rollart_obs_chunk_fp8_scratch_size(n_items, num_kv_heads,
+ *                  page_size, max_seq_len) bytes (two bf16 pools of n_items * ceil(max_seq_len / page_size) pages plus
+ *                  a page table and lengths for them); owned by the caller, contents undefined afterwards.  A smaller
+ *                  buffer returns ROLLART_ERR_WORKSPACE and launches nothing.
+ *   other arguments, errors and arithmetic as for rollart_obs_chunk_attn (bf16 operands: here the exact code values).
+ * Launches two kernels.  A code of NaN in a live slot gives NaN results for the rows that see it, as a bf16 NaN would.
+ */
+size_t rollart_obs_chunk_fp8_scratch_size(int32_t n_items, int32_t num_kv_heads, int32_t page_size, int32_t max_seq_len);
+rollart_status rollart_obs_chunk_attn_fp8(rollart_ctx *ctx, const rollart_kv_pool *pool, const rollart_trajs *trajs,
+                                          const int32_t *traj_ids, const int32_t *q_indptr, int32_t n_items,
+                                          int32_t total_q, int32_t max_seq_len, const void *q, int32_t num_q_heads,
+                                          float sm_scale, float k_scale, float v_scale, void *out, float *lse,
+                                          void *scratch, size_t scratch_bytes, void *stream);
+
+/*
  * Decode attention for callers that cannot allocate device memory.  The paper has no counterpart
  * to this call; it exists for the way the library gets embedded.
  *

@@ -293,3 +293,12 @@ def decode_attn_fp8(k_pool, v_pool, page_table, seq_lens, q, sm_scale, k_scale, 
     out, lse = decode_attn(fp8_pool_as_bf16_bits(k_pool), fp8_pool_as_bf16_bits(v_pool), page_table, seq_lens, q,
                            float(np.float32(sm_scale) * np.float32(k_scale)), traj_ids=traj_ids)
     return out * float(np.float32(v_scale)), lse
+
+
+def obs_chunk_attn_fp8(k_pool, v_pool, page_table, seq_lens, q_indptr, q, sm_scale, k_scale, v_scale, traj_ids=None,
+                       rows: Optional[Sequence[int]] = None):
+    """Observation-chunk attention over fp8 pools: the rows and the mask of obs_chunk_attn with keys
+    k_scale * code value and values v_scale * code value."""
+    out, lse = obs_chunk_attn(fp8_pool_as_bf16_bits(k_pool), fp8_pool_as_bf16_bits(v_pool), page_table, seq_lens, q_indptr, q,
+                              float(np.float32(sm_scale) * np.float32(k_scale)), traj_ids=traj_ids, rows=rows)
+    return out * float(np.float32(v_scale)), lse

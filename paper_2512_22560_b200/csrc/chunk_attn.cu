@@ -79,6 +79,7 @@ struct ChunkParams {
     __nv_bfloat16 *out;
     float *lse;
     float scale_log2;
+    float out_scale;            // the result is multiplied by this (the value scale of an fp8 cache expanded to bf16; else 1)
     // shared-prefix mode (NULL otherwise): every row of item i sees exactly the first shared_lens[i] keys, no causal mask
     const int32_t *shared_lens;
     float *out_f32;             // when set, result rows go here in fp32 instead of bf16 to `out`
@@ -730,7 +731,7 @@ chunk_attn_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constan
             }
         }
         if (cnt > 0 && !(split && mt == 1)) {
-            const float inv = l_sum > 0.f ? 1.f / l_sum : 0.f;
+            const float inv = l_sum > 0.f ? prm.out_scale / l_sum : 0.f;
             const float f0 = w0 * inv, f1 = w1 * inv;
             const long long orow = (static_cast<long long>(q_row0 + first_tok + tok_local) * prm.num_q_heads + head * g + head_local);
 #pragma unroll 1
@@ -854,7 +855,7 @@ cudaError_t launch_chunk_attn(const AttnCall &c, cudaStream_t stream, int64_t *l
         prm.max_pages = c.trajs.max_pages; prm.num_traj = c.trajs.num_traj; prm.num_pages = c.pool.num_pages;
         prm.page_size = c.pool.page_size; prm.num_kv_heads = hkv; prm.num_q_heads = c.num_q_heads; prm.group = g;
         prm.n_items = n; prm.item_offset = base; prm.max_seq_len = c.max_seq_len; prm.total_q = c.total_q;
-        prm.out = c.out; prm.lse = c.lse; prm.scale_log2 = c.sm_scale * kLog2e; prm.status = c.status;
+        prm.out = c.out; prm.lse = c.lse; prm.scale_log2 = c.sm_scale * kLog2e; prm.out_scale = c.v_scale; prm.status = c.status;
         prm.shared_lens = c.shared_lens ? c.shared_lens + base : nullptr;
         prm.out_f32 = c.out_f32;
         // an upper bound on the M-tile pairs of these items: every item has at most one ragged pair

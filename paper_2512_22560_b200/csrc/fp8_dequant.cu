@@ -1,0 +1,148 @@
+// Observation-chunk attention over fp8 pools, first half: the contexts of the listed trajectories are expanded from
+// E4M3 codes to bf16 into a scratch pool of the same page geometry, and the chunk kernel then runs over the scratch
+// pool.  Every finite E4M3 value is a bf16 value, so the expansion is exact; the pool scales are applied by the
+// attention kernel (k_scale folded into the score scale, v_scale into the final normalisation).
+//
+// The chunk path is bound by the tensor cores (Sec. 3.1: prefill is the compute-bound phase), so one extra pass over
+// the context at the HBM rate (1 byte read, 2 written per element) costs a few per cent of the attention itself.
+//
+// Scratch layout: item i of the call owns scratch pages i * pages_per_item .. (i + 1) * pages_per_item - 1 in logical
+// order, pages_per_item = ceil(max_seq_len / page_size); the scratch page table row of item i lists exactly those
+// ids, and its length is the trajectory's.  One thread block expands one (item, logical page): all kv heads of a page
+// are one contiguous run in both pools.
+#include "rollart_internal.cuh"
+
+namespace rollart {
+
+namespace {
+
+constexpr int kThreads = 256;
+
+// two E4M3 codes (low 16 bits of `pair`) -> two bf16: e4m3 -> f16 -> f32 -> bf16, every step exact
+__device__ __forceinline__ uint32_t e4m3x2_to_bf16x2(uint32_t pair) {
+    uint32_t h2;
+    asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h2) : "h"(static_cast<uint16_t>(pair)));
+    const float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&h2));
+    const __nv_bfloat162 b = __floats2bfloat162_rn(f.x, f.y);
+    return *reinterpret_cast<const uint32_t *>(&b);
+}
+
+// four E4M3 codes -> four bf16.  A code's seven low bits, placed at bit 20 of an fp32 word, are its exponent and mantissa
+// fields with the fp32 bias in place of the E4M3 one (a subnormal code becomes an fp32 subnormal), so one multiplication
+// by 2^(127-7) gives the code's value exactly; its upper half is the bf16.  NaN codes (S.1111.111) are not covered by
+// that and take the conversion instructions.
+__device__ __forceinline__ void expand4(uint32_t w, uint32_t &lo, uint32_t &hi) {
+    if ((((w & 0x7F7F7F7Fu) + 0x01010101u) & 0x80808080u) != 0u) {
+        lo = e4m3x2_to_bf16x2(w);
+        hi = e4m3x2_to_bf16x2(w >> 16);
+        return;
+    }
+    const float up = 0x1p120f;
+    const uint32_t f0 = __float_as_uint(__uint_as_float((w & 0x0000007Fu) << 20) * up);
+    const uint32_t f1 = __float_as_uint(__uint_as_float((w & 0x00007F00u) << 12) * up);
+    const uint32_t f2 = __float_as_uint(__uint_as_float((w & 0x007F0000u) << 4) * up);
+    const uint32_t f3 = __float_as_uint(__uint_as_float((w & 0x7F000000u) >> 4) * up);
+    const uint32_t sgn = w & 0x80808080u;
+    lo = __byte_perm(f0, f1, 0x7632) | __byte_perm(sgn, 0u, 0x1404);      // upper halves of f0, f1; signs to bits 15 and 31
+    hi = __byte_perm(f2, f3, 0x7632) | __byte_perm(sgn, 0u, 0x3424);
+}
+
+__device__ __forceinline__ void expand16(const uint4 &codes, uint4 &lo, uint4 &hi) {
+    expand4(codes.x, lo.x, lo.y);
+    expand4(codes.y, lo.z, lo.w);
+    expand4(codes.z, hi.x, hi.y);
+    expand4(codes.w, hi.z, hi.w);
+}
+
+__global__ void __launch_bounds__(kThreads)
+fp8_pages_to_bf16_kernel(const uint4 *__restrict__ k_pool, const uint4 *__restrict__ v_pool, int num_pages, int page_size,
+                         int num_kv_heads, const int32_t *__restrict__ page_table, int max_pages,
+                         const int32_t *__restrict__ seq_lens, int num_traj, const int32_t *__restrict__ traj_ids,
+                         int n_items, int pages_per_item, int max_seq_len, uint4 *__restrict__ k_scratch,
+                         uint4 *__restrict__ v_scratch, int32_t *__restrict__ scratch_table,
+                         int32_t *__restrict__ scratch_lens, DeviceStatus *status) {
+    const int item = blockIdx.x / pages_per_item;
+    const int lp = blockIdx.x - item * pages_per_item;
+    if (item >= n_items) return;
+    const int t = traj_ids ? __ldg(traj_ids + item) : item;
+    const bool t_ok = t >= 0 && t < num_traj;
+    int len = t_ok ? __ldg(seq_lens + t) : 0;
+    const bool len_ok = len >= 0 && len <= max_seq_len && static_cast<long long>(len) <= static_cast<long long>(max_pages) * page_size;
+    const long long s = static_cast<long long>(item) * pages_per_item + lp;      // this block's scratch page
+    if (threadIdx.x == 0) {
+        scratch_table[s] = static_cast<int32_t>(s);
+        if (lp == 0) {
+            if (!t_ok) report(status, ROLLART_ERR_BOUNDS, t, 3);
+            else if (!len_ok) report(status, ROLLART_ERR_BOUNDS, len, 3);
+            scratch_lens[item] = t_ok && len_ok ? len : 0;    // a bad item is reported and then attends to nothing
+        }
+    }
+    if (!t_ok || !len_ok || static_cast<long long>(lp) * page_size >= len) return;
+    const int pg = __ldg(page_table + static_cast<long long>(t) * max_pages + lp);
+    if (pg < 0 || pg >= num_pages) {
+        if (threadIdx.x == 0) report(status, ROLLART_ERR_BOUNDS, pg, 3);
+        return;
+    }
+    const int vec_per_page = num_kv_heads * page_size * (kHeadDim / 16);         // 16 codes per uint4
+    const uint4 *ks = k_pool + static_cast<long long>(pg) * vec_per_page;
+    const uint4 *vs = v_pool + static_cast<long long>(pg) * vec_per_page;
+    uint4 *kd = k_scratch + s * vec_per_page * 2;
+    uint4 *vd = v_scratch + s * vec_per_page * 2;
+    // two pieces of K and of V per thread and round: four independent loads in flight
+    for (int j = threadIdx.x; j < vec_per_page; j += 2 * kThreads) {
+        const int j2 = j + kThreads;
+        const bool two = j2 < vec_per_page;
+        const uint4 kc = __ldg(ks + j), vc = __ldg(vs + j);
+        uint4 kc2 = make_uint4(0u, 0u, 0u, 0u), vc2 = kc2;
+        if (two) { kc2 = __ldg(ks + j2); vc2 = __ldg(vs + j2); }
+        uint4 a, b;
+        expand16(kc, a, b);
+        kd[2 * j] = a;
+        kd[2 * j + 1] = b;
+        expand16(vc, a, b);
+        vd[2 * j] = a;
+        vd[2 * j + 1] = b;
+        if (two) {
+            expand16(kc2, a, b);
+            kd[2 * j2] = a;
+            kd[2 * j2 + 1] = b;
+            expand16(vc2, a, b);
+            vd[2 * j2] = a;
+            vd[2 * j2 + 1] = b;
+        }
+    }
+}
+
+size_t align_up(size_t x) { return (x + 255) & ~static_cast<size_t>(255); }
+
+}  // namespace
+
+Fp8ChunkScratch fp8_chunk_scratch_layout(int n_items, int num_kv_heads, int page_size, int max_seq_len) {
+    Fp8ChunkScratch L;
+    L.pages_per_item = (max_seq_len + page_size - 1) / page_size;
+    if (L.pages_per_item < 1) L.pages_per_item = 1;
+    L.num_pages = static_cast<long long>(n_items) * L.pages_per_item;
+    const size_t pool_bytes = static_cast<size_t>(L.num_pages) * num_kv_heads * page_size * kRowBytes;
+    L.off_k = 0;
+    L.off_v = align_up(pool_bytes);
+    L.off_table = L.off_v + align_up(pool_bytes);
+    L.off_lens = L.off_table + align_up(static_cast<size_t>(L.num_pages) * sizeof(int32_t));
+    L.bytes = L.off_lens + align_up(static_cast<size_t>(n_items) * sizeof(int32_t));
+    return L;
+}
+
+cudaError_t launch_fp8_pages_to_bf16(const rollart_kv_pool &pool, const rollart_trajs &trajs, const int32_t *traj_ids,
+                                     int n_items, int max_seq_len, const Fp8ChunkScratch &L, void *scratch,
+                                     DeviceStatus *status, cudaStream_t stream, int64_t *launches) {
+    if (L.num_pages > 0x7FFFFFFFLL) return cudaErrorInvalidValue;
+    char *base = static_cast<char *>(scratch);
+    fp8_pages_to_bf16_kernel<<<static_cast<unsigned>(L.num_pages), kThreads, 0, stream>>>(
+        static_cast<const uint4 *>(pool.k_pool), static_cast<const uint4 *>(pool.v_pool), pool.num_pages, pool.page_size,
+        pool.num_kv_heads, trajs.page_table, trajs.max_pages_per_traj, trajs.seq_lens, trajs.num_traj, traj_ids, n_items,
+        L.pages_per_item, max_seq_len, reinterpret_cast<uint4 *>(base + L.off_k), reinterpret_cast<uint4 *>(base + L.off_v),
+        reinterpret_cast<int32_t *>(base + L.off_table), reinterpret_cast<int32_t *>(base + L.off_lens), status);
+    ++*launches;
+    return cudaGetLastError();
+}
+
+}  // namespace rollart

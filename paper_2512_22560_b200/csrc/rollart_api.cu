@@ -528,6 +528,56 @@ rollart_status rollart_obs_chunk_attn(rollart_ctx *ctx, const rollart_kv_pool *p
     return ROLLART_OK;
 }
 
+size_t rollart_obs_chunk_fp8_scratch_size(int32_t n_items, int32_t num_kv_heads, int32_t page_size, int32_t max_seq_len) {
+    if (n_items <= 0 || num_kv_heads <= 0 || page_size <= 0 || max_seq_len < 0) return 0;
+    return fp8_chunk_scratch_layout(n_items, num_kv_heads, page_size, max_seq_len).bytes;
+}
+
+rollart_status rollart_obs_chunk_attn_fp8(rollart_ctx *ctx, const rollart_kv_pool *pool, const rollart_trajs *trajs,
+                                          const int32_t *traj_ids, const int32_t *q_indptr, int32_t n_items,
+                                          int32_t total_q, int32_t max_seq_len, const void *q, int32_t num_q_heads,
+                                          float sm_scale, float k_scale, float v_scale, void *out, float *lse,
+                                          void *scratch, size_t scratch_bytes, void *stream) {
+    if (!ctx) return ROLLART_ERR_INVALID_ARG;
+    rollart_status st = attn_common(ctx, pool, trajs, n_items, total_q, max_seq_len, q, num_q_heads, out);
+    if (st != ROLLART_OK) return st;
+    if (!(k_scale > 0.f) || !(v_scale > 0.f) || !isfinite(k_scale) || !isfinite(v_scale))
+        return fail(ctx, ROLLART_ERR_INVALID_ARG, "k_scale and v_scale must be positive and finite");
+    if (n_items == 0 || total_q == 0) return ROLLART_OK;
+    if (!q_indptr) return fail(ctx, ROLLART_ERR_INVALID_ARG, "q_indptr NULL");
+    max_seq_len = clamp_bound(pool, trajs, max_seq_len);
+    const Fp8ChunkScratch L = fp8_chunk_scratch_layout(n_items, pool->num_kv_heads, pool->page_size, max_seq_len);
+    if (!scratch || (reinterpret_cast<uintptr_t>(scratch) & 255u) != 0)
+        return fail(ctx, ROLLART_ERR_INVALID_ARG, "scratch must be a 256-byte aligned device buffer");
+    if (scratch_bytes < L.bytes)
+        return fail(ctx, ROLLART_ERR_WORKSPACE, "scratch of %zu bytes is too small (need %zu)", scratch_bytes, L.bytes);
+    if (L.num_pages > 0x7FFFFFFFLL) return fail(ctx, ROLLART_ERR_UNSUPPORTED, "too many scratch pages");
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return fail(ctx, ROLLART_ERR_CUDA, "cannot select device %d", ctx->device);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    cudaError_t e = launch_fp8_pages_to_bf16(*pool, *trajs, traj_ids, n_items, max_seq_len, L, scratch, ctx->d_status, s,
+                                             &ctx->launches);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "fp8 expansion launch");
+    // the attention itself runs over the expanded copy: item i is row i of the scratch table
+    char *base = static_cast<char *>(scratch);
+    rollart_kv_pool spool = *pool;
+    spool.k_pool = base + L.off_k;
+    spool.v_pool = base + L.off_v;
+    spool.num_pages = static_cast<int32_t>(L.num_pages);
+    rollart_trajs strajs;
+    strajs.page_table = reinterpret_cast<const int32_t *>(base + L.off_table);
+    strajs.max_pages_per_traj = L.pages_per_item;
+    strajs.seq_lens = reinterpret_cast<const int32_t *>(base + L.off_lens);
+    strajs.num_traj = n_items;
+    AttnCall c = make_call(ctx, &spool, &strajs, nullptr, q_indptr, n_items, total_q, max_seq_len, q, num_q_heads,
+                           sm_scale * k_scale, out, lse);
+    c.v_scale = v_scale;
+    bool too_small = false;
+    e = launch_chunk_attn(c, s, &ctx->launches, &too_small);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "obs_chunk_attn launch");
+    return ROLLART_OK;
+}
+
 rollart_status rollart_check(rollart_ctx *ctx, void *stream) {
     if (!ctx) return ROLLART_ERR_INVALID_ARG;
     DeviceGuard guard(ctx->device);

@@ -107,7 +107,8 @@ struct AttnCall {
     const int32_t *page_offset;   // decode: per item, pages of the table row to skip (the keys before them are not attended to)
     const int32_t *shared_lens;   // chunk: per item, every query row of the item sees exactly the first shared_lens[i] keys
     float *out_f32;               // when set the result rows are written here in fp32 instead of bf16 to `out`
-    // fp8 (E4M3) pools (decode and fused append + decode): keys are k_scale * code value, values v_scale * code value
+    // fp8 (E4M3) pools (decode and fused append + decode): keys are k_scale * code value, values v_scale * code value.
+    // The chunk kernel reads bf16 only; it multiplies its result by v_scale (1 for bf16 pools).
     bool fp8;
     float k_scale, v_scale;
 };
@@ -118,6 +119,18 @@ cudaError_t launch_decode_attn(const AttnCall &c, cudaStream_t stream, int64_t *
 // zeroes the bookkeeping at the head of the workspace after a device-side error
 cudaError_t decode_reset_workspace(void *workspace, size_t bytes, cudaStream_t stream);
 cudaError_t launch_chunk_attn(const AttnCall &c, cudaStream_t stream, int64_t *launches, bool *too_small);
+
+// Observation-chunk attention over fp8 pools: the listed trajectories' contexts are expanded to bf16 into a scratch
+// pool (item i owns pages i * pages_per_item ..), with a scratch page table and scratch lengths behind the two pools.
+struct Fp8ChunkScratch {
+    int pages_per_item;
+    long long num_pages;
+    size_t off_k, off_v, off_table, off_lens, bytes;
+};
+Fp8ChunkScratch fp8_chunk_scratch_layout(int n_items, int num_kv_heads, int page_size, int max_seq_len);
+cudaError_t launch_fp8_pages_to_bf16(const rollart_kv_pool &pool, const rollart_trajs &trajs, const int32_t *traj_ids,
+                                     int n_items, int max_seq_len, const Fp8ChunkScratch &layout, void *scratch,
+                                     DeviceStatus *status, cudaStream_t stream, int64_t *launches);
 
 // Group decode helpers.  `prepare` derives, per group, the trajectory whose table row stands for the shared
 // prefix and, per item, the pages to skip; it also checks that the members alias the same pages there.

@@ -24,7 +24,8 @@ EXPORTS = (
     "rollart_decode_attn_noalloc", "rollart_kv_gather", "rollart_pages_reserve", "rollart_pages_release",
     "rollart_append_decode_attn", "rollart_group_decode_attn", "rollart_group_decode_workspace_size",
     "rollart_decode_attn_fp8", "rollart_kv_append_fp8", "rollart_append_decode_attn_fp8",
-    "rollart_kv_gather_fp8", "rollart_kv_append_fp8_codes",
+    "rollart_kv_gather_fp8", "rollart_kv_append_fp8_codes", "rollart_obs_chunk_attn_fp8",
+    "rollart_obs_chunk_fp8_scratch_size",
 )
 
 
@@ -98,6 +99,11 @@ def load_library() -> ctypes.CDLL:
     L.rollart_obs_chunk_attn.restype = ctypes.c_int
     L.rollart_obs_chunk_attn.argtypes = [vp, ctypes.POINTER(_KVPool), ctypes.POINTER(_Trajs), vp, vp, i32, i32, i32, vp,
                                          i32, f32, vp, vp, vp]
+    L.rollart_obs_chunk_fp8_scratch_size.restype = ctypes.c_size_t
+    L.rollart_obs_chunk_fp8_scratch_size.argtypes = [i32, i32, i32, i32]
+    L.rollart_obs_chunk_attn_fp8.restype = ctypes.c_int
+    L.rollart_obs_chunk_attn_fp8.argtypes = [vp, ctypes.POINTER(_KVPool), ctypes.POINTER(_Trajs), vp, vp, i32, i32, i32, vp,
+                                             i32, f32, f32, f32, vp, vp, vp, ctypes.c_size_t, vp]
     L.rollart_decode_attn_noalloc.restype = ctypes.c_int
     L.rollart_decode_attn_noalloc.argtypes = [ctypes.c_int, ctypes.POINTER(_KVPool), ctypes.POINTER(_Trajs), vp, i32, i32,
                                               vp, i32, f32, vp, vp, vp, vp, ctypes.c_char_p, ctypes.c_size_t]
@@ -117,6 +123,10 @@ def workspace_size(max_items: int, num_q_heads: int, num_kv_heads: int, max_seq_
 
 def group_decode_workspace_size(max_items: int, num_q_heads: int, num_kv_heads: int, max_seq_len: int) -> int:
     return int(load_library().rollart_group_decode_workspace_size(max_items, num_q_heads, num_kv_heads, max_seq_len))
+
+
+def obs_chunk_fp8_scratch_size(n_items: int, num_kv_heads: int, page_size: int, max_seq_len: int) -> int:
+    return int(load_library().rollart_obs_chunk_fp8_scratch_size(n_items, num_kv_heads, page_size, max_seq_len))
 
 
 def _ptr(t: Optional[torch.Tensor], dtype=None, device=None, host_ok: bool = False) -> Optional[int]:
@@ -459,6 +469,29 @@ class Context:
             _ptr(q_indptr, torch.int32, self.device), n_items, total_q, int(max_seq_len),
             _ptr(q, torch.bfloat16, self.device), hq, float(sm_scale), _ptr(out, torch.bfloat16, self.device),
             _ptr(lse, torch.float32, self.device), self._stream(stream))
+        if st != OK:
+            self._raise(st)
+
+    def obs_chunk_attn_fp8(self, k_pool, v_pool, page_table, seq_lens, q_indptr, q, sm_scale, k_scale, v_scale, max_seq_len,
+                           out, scratch, lse=None, traj_ids=None, stream=None) -> None:
+        """obs_chunk_attn over pools of E4M3 codes; `scratch` is a uint8 CUDA tensor of at least
+        obs_chunk_fp8_scratch_size(n_items, num_kv_heads, page_size, max_seq_len) bytes"""
+        pool = self._pool_fp8(k_pool, v_pool)
+        trajs = self._trajs(page_table, seq_lens)
+        if q.dim() != 3 or q.shape != out.shape:
+            raise ValueError("q and out must be [total_q][num_q_heads][head_dim]")
+        total_q, hq, _ = q.shape
+        n_items = q_indptr.shape[0] - 1
+        if traj_ids is not None and traj_ids.shape[0] != n_items:
+            raise ValueError("traj_ids must have one entry per item")
+        if lse is not None and tuple(lse.shape) != (total_q, hq):
+            raise ValueError("lse must be [total_q][num_q_heads]")
+        st = self._lib.rollart_obs_chunk_attn_fp8(
+            self._h, ctypes.byref(pool), ctypes.byref(trajs), _ptr(traj_ids, torch.int32, self.device),
+            _ptr(q_indptr, torch.int32, self.device), n_items, total_q, int(max_seq_len),
+            _ptr(q, torch.bfloat16, self.device), hq, float(sm_scale), float(k_scale), float(v_scale),
+            _ptr(out, torch.bfloat16, self.device), _ptr(lse, torch.float32, self.device),
+            _ptr(scratch, torch.uint8, self.device), scratch.numel(), self._stream(stream))
         if st != OK:
             self._raise(st)
 

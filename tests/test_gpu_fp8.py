@@ -215,3 +215,143 @@ def test_hand_over_of_an_fp8_cache(cuda_device, i, T, div):
     ctx.kv_gather_fp8(dk, dv, table, lens0, dev_i32(bad, cuda_device), big, big.clone(), traj_ids=dev_i32(ids, cuda_device))
     assert ctx.status() == rollart.ERR_BOUNDS and "kv_gather" in ctx.last_error()
     ctx.close()
+
+
+def run_fp8_chunk_case(batch, device, ks=KS, vs=VS, scratch_slack=0):
+    """Quantise the existing cache with the oracle, append the chunks through the quantising append, then run
+    observation-chunk attention over the fp8 pools on the GPU and in the oracle."""
+    spec = batch.spec
+    P = spec.page_size
+    ids = batch.chunk_ids
+    rows, q_indptr = batch.chunk_rows()
+    k8 = oracle.fp8_quantize_rows(W.bf16_to_u16(batch.k_pool), ks)
+    v8 = oracle.fp8_quantize_rows(W.bf16_to_u16(batch.v_pool), vs)
+    live = np.zeros(k8.shape[:1] + k8.shape[2:3], bool)
+    for t in range(spec.num_traj):
+        L = int(batch.seq_lens_before[t])
+        for lp in range((L + P - 1) // P):
+            live[batch.page_table[t, lp], : min(P, L - lp * P)] = True
+    dead = ~live                                                             # NaN codes wherever no token lives
+    k8[np.broadcast_to(dead[:, None, :, None], k8.shape)] = 0x7F
+    v8[np.broadcast_to(dead[:, None, :, None], v8.shape)] = 0xFF
+    dk, dv = torch.from_numpy(k8.copy()).to(device), torch.from_numpy(v8.copy()).to(device)
+    table, lens0 = dev_i32(batch.page_table, device), dev_i32(batch.seq_lens_before, device)
+    lens1 = torch.empty_like(lens0)
+    msl = int(batch.seq_lens_after.max())
+    ctx = make_ctx(spec, max(1, len(ids)), msl)
+    ctx.kv_append_fp8(dk, dv, table, lens0, dev_i32(batch.new_indptr, device), batch.k_new.to(device), batch.v_new.to(device),
+                      ks, vs, seq_lens_out=lens1)
+    after = oracle.kv_append_fp8(k8, v8, batch.page_table, batch.seq_lens_before, batch.new_indptr,
+                                 W.bf16_to_u16(batch.k_new), W.bf16_to_u16(batch.v_new), ks, vs)
+    q = batch.q_new[torch.from_numpy(rows)].contiguous()
+    out = torch.full_like(q, float("nan"), device=device)
+    lse = torch.full((q.shape[0], spec.num_q_heads), float("nan"), device=device)
+    need = rollart.obs_chunk_fp8_scratch_size(len(ids), spec.num_kv_heads, P, msl)
+    scratch = torch.full((need + scratch_slack,), 0xFF, dtype=torch.uint8, device=device)      # bf16 NaN everywhere
+    ctx.obs_chunk_attn_fp8(dk, dv, table, lens1, dev_i32(q_indptr, device), q.to(device), spec.sm_scale, ks, vs, msl, out,
+                           scratch, lse=lse, traj_ids=dev_i32(ids, device))
+    ctx.check()
+    assert np.array_equal(dk.cpu().numpy(), k8) and np.array_equal(dv.cpu().numpy(), v8), "the call must not touch the pools"
+    ref_o, ref_l = oracle.obs_chunk_attn_fp8(k8, v8, batch.page_table, after, q_indptr, W.bf16_to_u16(q), spec.sm_scale, ks, vs,
+                                             traj_ids=ids)
+    assert_attn_close(out, ref_o, spec.name + " fp8 chunk")
+    assert_lse_close(lse, ref_l, spec.name + " fp8 chunk")
+    return ctx, (dk, dv, table, lens1), (q, q_indptr, ids, msl), out
+
+
+def test_fp8_chunk_shrunk_mixed_batch(cuda_device):
+    run_fp8_chunk_case(W.make_batch(W.shrink(W.CONFIGS[4], 8, 16, 8), seed=41), cuda_device)[0].close()
+
+
+def test_fp8_chunk_recompute_from_empty_cache(cuda_device):
+    batch = W.make_batch(W.shrink(W.RECOMPUTE, 5, 16), seed=46)
+    run_fp8_chunk_case(batch, cuda_device)[0].close()
+
+
+@pytest.mark.parametrize("P,hq,hkv", [(16, 8, 2), (32, 7, 1), (64, 16, 1), (16, 3, 3)])
+def test_fp8_chunk_edges(cuda_device, P, hq, hkv):
+    prior = [0, 0, 1, P - 1, P, 5, 130, 64]
+    n_new = [1, P + 3, P, 2, 1, 130, 31, 128]
+    spec = dataclasses.replace(W.CONFIGS[4], page_size=P, num_traj=len(prior), num_q_heads=hq, num_kv_heads=hkv,
+                               name=f"fp8_chunk_edge_{P}_{hq}_{hkv}")
+    batch = W.make_layout(spec, seed=3)
+    batch.seq_lens_before = np.array(prior, np.int32)
+    batch.n_new = np.array(n_new, np.int32)
+    batch.is_chunk[:] = True
+    batch.new_indptr = np.concatenate([[0], np.cumsum(batch.n_new)]).astype(np.int32)
+    pages = (batch.seq_lens_before + batch.n_new + P - 1) // P
+    batch.page_table, batch.num_pages = W.build_page_table(pages.astype(np.int64), 0.3, np.random.default_rng(2))
+    W.fill_tensors(batch)
+    run_fp8_chunk_case(batch, cuda_device, scratch_slack=4096)[0].close()
+
+
+def test_fp8_chunk_last_row_agrees_with_fp8_decode_and_errors_are_reported(cuda_device):
+    batch = W.make_batch(W.shrink(W.CONFIGS[4], 6, 32, 16), seed=77)
+    spec = batch.spec
+    ctx, (dk, dv, table, lens1), (q, q_indptr, ids, msl), out = run_fp8_chunk_case(batch, cuda_device)
+    # the last row of a chunk sees the whole context: the decode kernel must agree within a few bf16 ulps
+    last = torch.from_numpy(q_indptr[1:].astype(np.int64) - 1)
+    qd = q[last].contiguous().to(cuda_device)
+    od = torch.empty_like(qd)
+    ctx.decode_attn_fp8(dk, dv, table, lens1, qd, spec.sm_scale, KS, VS, msl, od, traj_ids=dev_i32(ids, cuda_device))
+    ctx.check()
+    a, b = out[last.to(cuda_device)].float(), od.float()
+    assert torch.all((a - b).abs() <= 2e-2 * b.abs() + 2e-3)
+    qi = dev_i32(q_indptr, cuda_device)
+    tid = dev_i32(ids, cuda_device)
+    need = rollart.obs_chunk_fp8_scratch_size(len(ids), spec.num_kv_heads, spec.page_size, msl)
+    scratch = torch.empty(need, dtype=torch.uint8, device=cuda_device)
+    qg = q.to(cuda_device)
+    with pytest.raises(rollart.RollartError) as e:
+        ctx.obs_chunk_attn_fp8(dk, dv, table, lens1, qi, qg, spec.sm_scale, KS, VS, msl, out, scratch[: need - 256], traj_ids=tid)
+    assert e.value.status == rollart.ERR_WORKSPACE
+    for ks, vs in [(0.0, 1.0), (1.0, float("inf")), (float("nan"), 1.0)]:
+        with pytest.raises(rollart.RollartError):
+            ctx.obs_chunk_attn_fp8(dk, dv, table, lens1, qi, qg, spec.sm_scale, ks, vs, msl, out, scratch, traj_ids=tid)
+    # a page id out of range and a length above the bound are device-side errors, nothing is read through them
+    bad_table = table.clone()
+    bad_table[int(ids[0]), 0] = dk.shape[0] + 5
+    ctx.obs_chunk_attn_fp8(dk, dv, bad_table, lens1, qi, qg, spec.sm_scale, KS, VS, msl, out, scratch, traj_ids=tid)
+    assert ctx.status() == rollart.ERR_BOUNDS and "obs_chunk_attn" in ctx.last_error()
+    ctx.obs_chunk_attn_fp8(dk, dv, table, lens1, qi, qg, spec.sm_scale, KS, VS, 64, out, scratch, traj_ids=tid)
+    assert ctx.status() == rollart.ERR_BOUNDS
+    ctx.close()
+
+
+def test_fp8_expansion_is_exact_for_every_code(cuda_device):
+    """The bf16 copy the chunk call makes of the cache, read back from the scratch buffer: every one of the 256 codes
+    (NaN codes included, in live slots here) against the oracle's decoder, bit for bit."""
+    P, H, D = 16, 3, 128
+    rng = np.random.default_rng(5)
+    lens = np.array([37, 16, 1, 80], np.int32)
+    pages = (lens.astype(np.int64) + P - 1) // P
+    table, num_pages = W.build_page_table(pages, 0.25, np.random.default_rng(4))
+    k8 = rng.integers(0, 256, (num_pages, H, P, D)).astype(np.uint8)
+    v8 = rng.integers(0, 256, (num_pages, H, P, D)).astype(np.uint8)
+    k8[table[0, 0], 0, 0, :] = np.arange(128, dtype=np.uint8)                  # every code at least once
+    k8[table[0, 0], 0, 1, :] = np.arange(128, 256, dtype=np.uint8)
+    spec = dataclasses.replace(W.CONFIGS[0], page_size=P, num_traj=4, num_q_heads=6, num_kv_heads=H, name="fp8_expand")
+    msl = int(lens.max())
+    ctx = make_ctx(spec, 4, msl)
+    need = rollart.obs_chunk_fp8_scratch_size(4, H, P, msl)
+    scratch = torch.zeros(need, dtype=torch.uint8, device=cuda_device)
+    q = torch.zeros(4, 6, D, dtype=torch.bfloat16, device=cuda_device)
+    out = torch.empty_like(q)
+    ctx.obs_chunk_attn_fp8(torch.from_numpy(k8).to(cuda_device), torch.from_numpy(v8).to(cuda_device), dev_i32(table, cuda_device),
+                           dev_i32(lens, cuda_device), dev_i32(np.arange(5), cuda_device), q, 1.0, 1.0, 1.0, msl, out, scratch)
+    ctx.check()
+    ppi = (msl + P - 1) // P
+    pool_bytes = 4 * ppi * H * P * D * 2
+    sc = scratch.cpu().numpy()
+    off_v = (pool_bytes + 255) // 256 * 256
+    for name, codes, off in (("k", k8, 0), ("v", v8, off_v)):
+        got = sc[off: off + pool_bytes].view(np.uint16).reshape(4 * ppi, H, P, D)
+        for i in range(4):
+            for lp in range(int(pages[i])):
+                want = oracle.fp8_pool_as_bf16_bits(codes[table[i, lp]])
+                g = got[i * ppi + lp]
+                nan_w = (want & 0x7FFF) > 0x7F80
+                nan_g = (g & 0x7FFF) > 0x7F80
+                assert np.array_equal(nan_w, nan_g), (name, i, lp)
+                assert np.array_equal(g[~nan_w], want[~nan_w]), (name, i, lp)
+    ctx.close()

@@ -138,3 +138,39 @@ def test_hand_over_of_codes_is_a_bit_copy_token_by_token():
             assert np.array_equal(dst_k[pg, :, pos % P], gk[indptr[i] + r]) and np.array_equal(dst_v[pg, :, pos % P], gv[indptr[i] + r])
             touched[pg, pos % P] = True
     assert np.all(dst_k[~touched[:, None, :].repeat(H, 1)] == 0x55) and np.all(dst_v[~touched[:, None, :].repeat(H, 1)] == 0xAA)
+
+
+def test_fp8_chunk_rows_against_a_dense_evaluation_and_against_decode():
+    # chunk row j of n sees the first L - n + j + 1 keys: each row checked against numpy over the dequantised
+    # context, and the last row against the fp8 decode call (which sees all L keys)
+    rng = np.random.default_rng(3)
+    P, H, D = 16, 2, 128
+    codes_k = rng.integers(0, 256, (6, H, P, D)).astype(np.uint8)
+    codes_v = rng.integers(0, 256, (6, H, P, D)).astype(np.uint8)
+    codes_k = (codes_k & 0x80) | np.minimum(codes_k & 0x7F, 0x3F)            # |value| < 2: moderate scores, no NaN
+    codes_v[(codes_v & 0x7F) == 0x7F] = 0x10
+    table = np.array([[4, 2, 0, 5], [1, 3, -1, -1]], np.int32)
+    lens = np.array([55, 20], np.int32)
+    n = [9, 20]                                                               # trajectory 1: the whole context is the chunk
+    q_indptr = np.array([0, 9, 29], np.int32)
+    q = ((rng.standard_normal((29, 4, D)) * 0.5).astype(np.float32).view(np.uint32) >> 16).astype(np.uint16)
+    ks, vs, sm = 0.5, 2.0, 0.25
+    out, lse = oracle.obs_chunk_attn_fp8(codes_k, codes_v, table, lens, q_indptr, q, sm, ks, vs)
+    assert out.shape == (29, 4, D) and lse.shape == (29, 4)
+    qf = (q.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+    for t in range(2):
+        npg = (lens[t] + P - 1) // P
+        kv = oracle.e4m3_decode(codes_k)[table[t, :npg]].transpose(1, 0, 2, 3).reshape(H, -1, D)
+        vv = oracle.e4m3_decode(codes_v)[table[t, :npg]].transpose(1, 0, 2, 3).reshape(H, -1, D)
+        for j in range(n[t]):
+            c = lens[t] - n[t] + j + 1
+            r = q_indptr[t] + j
+            for hq in range(4):
+                s = sm * ks * (kv[hq // 2, :c] @ qf[r, hq])
+                w = np.exp(s - s.max())
+                np.testing.assert_allclose(out[r, hq], vs * (w @ vv[hq // 2, :c]) / w.sum(), rtol=1e-12, atol=1e-12)
+                np.testing.assert_allclose(lse[r, hq], s.max() + math.log(w.sum()), rtol=1e-12)
+    last = q_indptr[1:] - 1
+    d_out, d_lse = oracle.decode_attn_fp8(codes_k, codes_v, table, lens, q[last], sm, ks, vs)
+    np.testing.assert_allclose(out[last], d_out, rtol=1e-13, atol=1e-13)
+    np.testing.assert_allclose(lse[last], d_lse, rtol=1e-13)
