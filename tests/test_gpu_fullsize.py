@@ -9,6 +9,7 @@ import torch
 
 import oracle
 from harness import DeviceBatch, assert_attn_close, assert_lse_close, dev_i32, make_ctx
+from paper_2512_22560_b200 import rollart
 from paper_2512_22560_b200 import workloads as W
 
 pytestmark = pytest.mark.gpu
@@ -225,4 +226,57 @@ def test_full_size_mixed_batch_chunk_sampled_rows(cuda_device):
     qsel = q[torch.from_numpy(q_rows).to(cuda_device)]
     ref_o, _ = oracle.attend_rows(kp, vp, post.page_table, row_traj, row_count, W.bf16_to_u16(qsel), spec.sm_scale)
     assert_attn_close(out[torch.from_numpy(q_rows).to(cuda_device)], ref_o, "cfg4 chunk rows")
+    ctx.close()
+
+
+def test_full_size_mixed_batch_fp8_chunk_sampled_rows(cuda_device):
+    # the chunk half of the mixed batch over fp8 pools, as bench.py times it: quantising append of everything, chunk
+    # attention over the codes (expansion into the scratch pool + the bf16 kernel); sampled rows against the oracle,
+    # which reads a host copy of the sampled trajectories' codes after the append
+    import dataclasses
+    spec = W.CONFIGS[4]
+    ks, vs = 0.03, 0.03
+    batch = W.make_batch(spec, device=cuda_device)
+    ids = batch.chunk_ids
+    rows, q_indptr = batch.chunk_rows()
+    msl = int(batch.seq_lens_after.max())
+    ctx = make_ctx(spec, len(ids), msl)
+    k8 = (batch.k_pool.float() / ks).clamp_(-448, 448).to(torch.float8_e4m3fn).view(torch.uint8)
+    v8 = (batch.v_pool.float() / vs).clamp_(-448, 448).to(torch.float8_e4m3fn).view(torch.uint8)
+    table, lens0 = dev_i32(batch.page_table, cuda_device), dev_i32(batch.seq_lens_before, cuda_device)
+    lens1 = torch.empty_like(lens0)
+    ctx.kv_append_fp8(k8, v8, table, lens0, dev_i32(batch.new_indptr, cuda_device), batch.k_new, batch.v_new, ks, vs,
+                      seq_lens_out=lens1)
+    q = batch.q_new[torch.from_numpy(rows).to(cuda_device)].contiguous()
+    out = torch.full_like(q, float("nan"))
+    need = rollart.obs_chunk_fp8_scratch_size(len(ids), spec.num_kv_heads, spec.page_size, msl)
+    scratch = torch.empty(need, dtype=torch.uint8, device=cuda_device)
+    ctx.obs_chunk_attn_fp8(k8, v8, table, lens1, dev_i32(q_indptr, cuda_device), q, spec.sm_scale, ks, vs, msl, out, scratch,
+                           traj_ids=dev_i32(ids, cuda_device))
+    ctx.check()
+    assert torch.all(torch.isfinite(out.float()))
+    del scratch
+    rng = np.random.default_rng(45)
+    order = np.argsort(batch.n_new[ids], kind="stable")
+    pick_local = sorted({int(order[0]), int(order[-1]), int(order[len(order) // 2])})
+    pick = ids[pick_local]
+    b8 = dataclasses.replace(batch)
+    b8.k_pool, b8.v_pool = k8, v8
+    post = W.extract_trajs(b8, pick)
+    kp, vp = post.k_pool.numpy(), post.v_pool.numpy()
+    after = post.seq_lens_before + post.n_new
+    row_traj, row_count, q_rows = [], [], []
+    for i, li in enumerate(pick_local):
+        n = int(batch.n_new[ids[li]])
+        cand = {0, 1, n - 1, n - 2, n // 2} | {r for e in range(32, n, 128) for r in (e - 1, e, e + 1)}
+        cand |= {int(x) for x in rng.integers(0, n, size=24)}
+        for j in sorted(c for c in cand if 0 <= c < n):
+            row_traj.append(i)
+            row_count.append(int(after[i]) - n + j + 1)
+            q_rows.append(int(q_indptr[li]) + j)
+    q_rows = torch.from_numpy(np.array(q_rows)).to(cuda_device)
+    sm = float(np.float32(spec.sm_scale) * np.float32(ks))
+    ref_o, _ = oracle.attend_rows(oracle.fp8_pool_as_bf16_bits(kp), oracle.fp8_pool_as_bf16_bits(vp), post.page_table, row_traj,
+                                  row_count, W.bf16_to_u16(q[q_rows]), sm)
+    assert_attn_close(out[q_rows], ref_o * float(np.float32(vs)), "cfg4 fp8 chunk rows")
     ctx.close()
