@@ -605,12 +605,27 @@ def main():
                     flush.fill_(1)
                     a.record(); w0.step(); b.record()
                 torch.cuda.synchronize(device)
+                # 16 steps captured into one CUDA graph (Sec. 7.1: rollout runs with CUDA graphs): the launch period
+                # without the host's issue rate in it
+                graph = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(graph, stream=torch.cuda.Stream(device=device)):
+                    for _ in range(16):
+                        w0.step()
+                for _ in range(3):
+                    graph.replay()
+                g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                g0.record()
+                for _ in range(20):
+                    graph.replay()
+                g1.record()
+                torch.cuda.synchronize(device)
                 w0.ctx.check()
                 extra[W.CONFIGS[0].name] = {"step_us_back_to_back": hot_ms * 1e3,
+                                            "step_us_graph_replay": g0.elapsed_time(g1) / (20 * 16) * 1e3,
                                             "step_us_after_l2_flush": float(np.median([a.elapsed_time(b) for a, b in ev])) * 1e3,
                                             "trajectories": w0.n_items, "kv_bytes": w0.bytes,
-                                            "note": "back to back = launch period (bounded below by the host's issue rate); "
-                                                    "after flush = events around one launch"}
+                                            "note": "back to back = launch period of eager calls; graph replay = the same from a CUDA graph of "
+                                                    "16 steps (no host issue cost); after flush = events around one launch"}
                 w0.ctx.close()
                 del w0, flush
                 torch.cuda.empty_cache()

@@ -167,3 +167,34 @@ def test_empty_items_and_empty_calls(cuda_device):
                   torch.zeros(0, batch.spec.num_kv_heads, 128, dtype=torch.bfloat16, device=cuda_device))
     ctx.check()
     assert ctx.launch_count == n0          # nothing was enqueued
+
+
+def test_append_and_chunk_attention_replayed_from_a_cuda_graph(cuda_device):
+    """kv_append + obs_chunk_attn captured once into a CUDA graph (Sec. 7.1: rollout runs with CUDA graphs) and replayed:
+    the same bits as the eager calls."""
+    batch = W.make_batch(W.shrink(W.CONFIGS[4], 6, 32, 16), seed=91)
+    db, ctx, out_eager, _ = run_chunk_case(batch, cuda_device)
+    spec = batch.spec
+    ids = batch.chunk_ids
+    rows, q_indptr = batch.chunk_rows()
+    msl = int(batch.seq_lens_after.max())
+    db2 = DeviceBatch(batch, cuda_device)                          # the pools as they were before the append
+    q = db2.q_new[torch.from_numpy(rows).to(cuda_device)].contiguous()
+    out = torch.full_like(q, float("nan"))
+    qi, tid = dev_i32(q_indptr, cuda_device), dev_i32(ids, cuda_device)
+    lens_after = torch.empty_like(db2.lens_before)
+    graph = torch.cuda.CUDAGraph()
+    torch.cuda.synchronize(cuda_device)
+    with torch.cuda.graph(graph, stream=torch.cuda.Stream(device=cuda_device)):
+        ctx.kv_append(db2.k_pool, db2.v_pool, db2.page_table, db2.lens_before, db2.new_indptr, db2.k_new, db2.v_new,
+                      seq_lens_out=lens_after)
+        ctx.obs_chunk_attn(db2.k_pool, db2.v_pool, db2.page_table, lens_after, qi, q, spec.sm_scale, msl, out, traj_ids=tid)
+    for _ in range(2):                                             # the append is idempotent: same rows to the same slots
+        out.fill_(float("nan"))
+        graph.replay()
+    torch.cuda.synchronize(cuda_device)
+    ctx.check()
+    assert torch.equal(out.view(torch.int16), out_eager.view(torch.int16))
+    assert torch.equal(db2.k_pool.view(torch.int16), db.k_pool.view(torch.int16))
+    assert torch.equal(lens_after, db.lens_after)
+    ctx.close()

@@ -232,3 +232,73 @@ def test_results_written_straight_to_pinned_host_memory(cuda_device, i, T, div):
         ctx.decode_attn(db.k_pool, db.v_pool, db.page_table, db.lens_after, q, spec.sm_scale, msl,
                         torch.empty(tuple(q.shape), dtype=torch.bfloat16), traj_ids=tid)          # pageable host memory
     ctx.close()
+
+
+def test_decode_steps_replayed_from_a_cuda_graph(cuda_device):
+    """The engine runs rollout with CUDA graphs (Sec. 7.1): the calls are asynchronous, allocate nothing and read their
+    lengths on the device, so one captured step replays for every following token.  Four replayed steps (lengths
+    advancing on the device) against four eager steps: pools, lengths and outputs bit for bit, and the last step
+    against the oracle."""
+    steps = 4
+    batch = W.make_batch(W.shrink(W.CONFIGS[1], 12, 4, 16), seed=800)
+    spec = batch.spec
+    ids = batch.decode_ids
+    n = len(ids)
+    msl = int(batch.seq_lens_before.max()) + steps
+    P = spec.page_size
+    # pages for the extra tokens: one more table column, and the rows that need a page take one of the spare pages
+    table = np.concatenate([batch.page_table, np.full((spec.num_traj, 1), -1, np.int32)], axis=1)
+    used = set(int(p) for t in range(spec.num_traj) for p in table[t, : (int(batch.seq_lens_after[t]) + P - 1) // P])
+    spare = [p for p in range(batch.num_pages) if p not in used]
+    for t in ids:
+        have = (int(batch.seq_lens_after[t]) + P - 1) // P
+        want = (int(batch.seq_lens_before[t]) + steps + P - 1) // P
+        for lp in range(have, want):
+            table[t, lp] = spare.pop()
+    g = torch.Generator(device="cpu").manual_seed(5)
+    qs = torch.randn(steps, n, spec.num_q_heads, 128, generator=g).to(torch.bfloat16).to(cuda_device)
+    kns = torch.randn(steps, n, spec.num_kv_heads, 128, generator=g).to(torch.bfloat16).to(cuda_device)
+    vns = torch.randn(steps, n, spec.num_kv_heads, 128, generator=g).to(torch.bfloat16).to(cuda_device)
+    tid = dev_i32(ids, cuda_device)
+    d_table = dev_i32(table, cuda_device)
+    ctx = make_ctx(spec, n, msl)
+
+    def fresh():
+        return (batch.k_pool.clone().to(cuda_device), batch.v_pool.clone().to(cuda_device),
+                dev_i32(batch.seq_lens_before, cuda_device), dev_i32(batch.seq_lens_before, cuda_device))
+
+    # eager
+    kp, vp, la, lb = fresh()
+    outs_e = torch.full_like(qs, float("nan"))
+    for s in range(steps):
+        ctx.append_decode_attn(kp, vp, d_table, la, kns[s], vns[s], qs[s], spec.sm_scale, msl, outs_e[s], traj_ids=tid,
+                               seq_lens_out=lb)
+        la.copy_(lb)
+    ctx.check()
+    # one captured step, replayed
+    kp2, vp2, la2, lb2 = fresh()
+    q_in, k_in, v_in = torch.empty_like(qs[0]), torch.empty_like(kns[0]), torch.empty_like(vns[0])
+    o_out = torch.full_like(qs[0], float("nan"))
+    side = torch.cuda.Stream(device=cuda_device)
+    graph = torch.cuda.CUDAGraph()
+    q_in.copy_(qs[0]); k_in.copy_(kns[0]); v_in.copy_(vns[0])
+    torch.cuda.synchronize(cuda_device)
+    with torch.cuda.graph(graph, stream=side):
+        ctx.append_decode_attn(kp2, vp2, d_table, la2, k_in, v_in, q_in, spec.sm_scale, msl, o_out, traj_ids=tid, seq_lens_out=lb2)
+        la2.copy_(lb2)
+    outs_g = torch.full_like(qs, float("nan"))
+    for s in range(steps):
+        q_in.copy_(qs[s]); k_in.copy_(kns[s]); v_in.copy_(vns[s])
+        graph.replay()
+        outs_g[s].copy_(o_out)
+    torch.cuda.synchronize(cuda_device)
+    ctx.check()
+    assert torch.equal(kp.view(torch.int16), kp2.view(torch.int16)) and torch.equal(vp.view(torch.int16), vp2.view(torch.int16))
+    assert torch.equal(la, la2) and torch.equal(la.cpu(), torch.from_numpy(np.where(
+        np.isin(np.arange(spec.num_traj), ids), batch.seq_lens_before + steps, batch.seq_lens_before)).to(torch.int32))
+    assert torch.equal(outs_e.view(torch.int16), outs_g.view(torch.int16))
+    # the last step against the oracle, over the pools the replays left behind
+    ref_o, _ = oracle.decode_attn(W.bf16_to_u16(kp2), W.bf16_to_u16(vp2), table, la2.cpu().numpy(), W.bf16_to_u16(qs[-1]),
+                                  spec.sm_scale, traj_ids=ids)
+    assert_attn_close(outs_g[-1], ref_o, "graph replay, last step")
+    ctx.close()
