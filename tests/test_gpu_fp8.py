@@ -355,3 +355,13 @@ def test_fp8_expansion_is_exact_for_every_code(cuda_device):
                 assert np.array_equal(nan_w, nan_g), (name, i, lp)
                 assert np.array_equal(g[~nan_w], want[~nan_w]), (name, i, lp)
     ctx.close()
+
+
+def test_fp8_more_items_than_one_launch_holds(cuda_device):
+    # 1300 short trajectories through the fp8 append + decode (several launches per call), and 1100 chunk items of
+    # 1..5 tokens through the fp8 chunk call (the second launch starts at a scratch row other than 0)
+    spec = dataclasses.replace(W.CONFIGS[0], num_traj=1300, len_lo=1, len_hi=90, name="fp8_many_items")
+    run_fp8_case(W.make_batch(spec, seed=71), cuda_device)
+    spec = dataclasses.replace(W.CONFIGS[0], num_traj=1100, len_lo=1, len_hi=40, chunk_fraction=1.0, chunk_lo=1, chunk_hi=5,
+                               name="fp8_many_chunks")
+    run_fp8_chunk_case(W.make_batch(spec, seed=72), cuda_device)[0].close()
