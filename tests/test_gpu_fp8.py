@@ -365,3 +365,33 @@ def test_fp8_more_items_than_one_launch_holds(cuda_device):
     spec = dataclasses.replace(W.CONFIGS[0], num_traj=1100, len_lo=1, len_hi=40, chunk_fraction=1.0, chunk_lo=1, chunk_hi=5,
                                name="fp8_many_chunks")
     run_fp8_chunk_case(W.make_batch(spec, seed=72), cuda_device)[0].close()
+
+
+def test_fp8_empty_items_and_empty_calls(cuda_device):
+    # an item with no chunk rows among live ones, and fp8 calls with nothing to do at all
+    spec = dataclasses.replace(W.CONFIGS[4], num_traj=4, name="fp8_empties")
+    batch = W.make_layout(W.shrink(spec, 4, 64, 16), seed=47)
+    batch.is_chunk[:] = True
+    batch.n_new = np.array([5, 0, 40, 1], np.int32)
+    batch.new_indptr = np.concatenate([[0], np.cumsum(batch.n_new)]).astype(np.int32)
+    P = batch.spec.page_size
+    pages = (batch.seq_lens_before.astype(np.int64) + batch.n_new + P - 1) // P
+    batch.page_table, batch.num_pages = W.build_page_table(pages, 0.3, np.random.default_rng(1))
+    W.fill_tensors(batch)
+    ctx, (dk, dv, table, lens1), _, _ = run_fp8_chunk_case(batch, cuda_device)
+    hq, hkv = batch.spec.num_q_heads, batch.spec.num_kv_heads
+    empty_q = torch.zeros(0, hq, 128, dtype=torch.bfloat16, device=cuda_device)
+    empty_kv = torch.zeros(0, hkv, 128, dtype=torch.bfloat16, device=cuda_device)
+    empty_codes = torch.zeros(0, hkv, 128, dtype=torch.uint8, device=cuda_device)
+    scratch = torch.empty(1 << 20, dtype=torch.uint8, device=cuda_device)
+    n0 = ctx.launch_count
+    ctx.obs_chunk_attn_fp8(dk, dv, table, lens1, dev_i32([0], cuda_device), empty_q, 0.1, KS, VS, 100, empty_q.clone(), scratch)
+    ctx.decode_attn_fp8(dk, dv, table, lens1, empty_q, 0.1, KS, VS, 100, empty_q.clone(), traj_ids=dev_i32([], cuda_device))
+    ctx.append_decode_attn_fp8(dk, dv, table, lens1, empty_kv, empty_kv.clone(), empty_q, 0.1, KS, VS, 100, empty_q.clone(),
+                               traj_ids=dev_i32([], cuda_device))
+    ctx.kv_append_fp8(dk, dv, table, lens1, dev_i32([0], cuda_device), empty_kv, empty_kv.clone(), KS, VS)
+    ctx.kv_append_fp8_codes(dk, dv, table, lens1, dev_i32([0], cuda_device), empty_codes, empty_codes.clone())
+    ctx.kv_gather_fp8(dk, dv, table, lens1, dev_i32([0], cuda_device), empty_codes, empty_codes.clone())
+    ctx.check()
+    assert ctx.launch_count == n0          # nothing was enqueued
+    ctx.close()
