@@ -270,6 +270,28 @@ class GroupDecodeWorkload:
         self.ctx.append_decode_attn(b.k_pool, b.v_pool, self.table, self.lens0, b.k_new, b.v_new, self.q, self.spec.sm_scale,
                                     self.max_seq_len, self.out, seq_lens_out=self.lens1)
 
+    def make_fp8(self, k_scale: float = 0.03, v_scale: float = 0.03):
+        """fp8 (E4M3) copies of the pools (aliased prefix pages hold the same codes) and the scratch of the group call"""
+        from paper_2512_22560_b200 import rollart
+        b, spec = self.batch, self.spec
+        self.k8 = (b.k_pool.float() * (1.0 / k_scale)).to(torch.float8_e4m3fn).view(torch.uint8)
+        self.v8 = (b.v_pool.float() * (1.0 / v_scale)).to(torch.float8_e4m3fn).view(torch.uint8)
+        self.ks, self.vs = k_scale, v_scale
+        need = rollart.obs_chunk_fp8_scratch_size(self.group_indptr.numel() - 1, spec.num_kv_heads, spec.page_size, self.max_seq_len)
+        self.scratch = torch.empty(need, dtype=torch.uint8, device=self.device)
+
+    def step_group_fp8(self):
+        b = self.batch
+        self.ctx.kv_append_fp8(self.k8, self.v8, self.table, self.lens0, self.new_indptr, b.k_new, b.v_new, self.ks, self.vs,
+                               seq_lens_out=self.lens1)
+        self.ctx.group_decode_attn_fp8(self.k8, self.v8, self.table, self.lens1, self.group_indptr, self.shared, self.q,
+                                       self.spec.sm_scale, self.ks, self.vs, self.max_seq_len, self.out, self.scratch)
+
+    def step_plain_fp8(self):
+        b = self.batch
+        self.ctx.append_decode_attn_fp8(self.k8, self.v8, self.table, self.lens0, b.k_new, b.v_new, self.q, self.spec.sm_scale,
+                                        self.ks, self.vs, self.max_seq_len, self.out, seq_lens_out=self.lens1)
+
     def time(self, fn, steps: int, warmup: int) -> float:
         for _ in range(warmup):
             fn()
@@ -699,6 +721,14 @@ def main():
                         "bytes_per_trajectory_definition": gw.bytes_per_trajectory_definition,
                         "bytes_unique_pages": gw.bytes_unique, "unique_gbs": gw.bytes_unique / (g_ms * 1e-3) / 1e9,
                         "plain_gbs": gw.bytes_per_trajectory_definition / (p_ms * 1e-3) / 1e9}
+                    try:
+                        gw.make_fp8()
+                        g8 = gw.time(gw.step_group_fp8, 20, 3)
+                        p8 = gw.time(gw.step_plain_fp8, 20, 3)
+                        extra[name]["fp8_pool"] = {"group_step_ms": g8, "plain_step_ms": p8, "speedup_over_plain_fp8_step": p8 / g8,
+                                                   "speedup_over_plain_bf16_step": p_ms / g8, "launches_per_group_step": 6}
+                    except Exception as e:
+                        extra[name]["fp8_pool"] = {"error": repr(e)}
                     gw.ctx.close()
                     del gw
                     torch.cuda.empty_cache()

@@ -277,6 +277,22 @@ rollart_status rollart_group_decode_attn(rollart_ctx *ctx, const rollart_kv_pool
                                          int32_t num_q_heads, float sm_scale, void *out, float *lse, void *stream);
 
 /*
+ * Group decode over fp8 pools: rollart_group_decode_attn with keys k_scale * value(code) and values
+ * v_scale * value(code) (pools of E4M3 codes as for rollart_decode_attn_fp8).  The shared prefixes, one per group,
+ * are expanded to bf16 into `scratch` for the tensor-core kernel (as rollart_obs_chunk_attn_fp8 does for whole
+ * contexts); the private remainders are read as codes by the fp8 decode kernel.
+ *   scratch   [device] 256-byte aligned, at least rollart_obs_chunk_fp8_scratch_size(n_groups, num_kv_heads, page_size,
+ *             max_seq_len) bytes; owned by the caller, contents undefined afterwards.
+ * Workspace, checks and errors as for rollart_group_decode_attn; a scratch buffer that is too small returns
+ * ROLLART_ERR_WORKSPACE and launches nothing.  Launches five kernels.
+ */
+rollart_status rollart_group_decode_attn_fp8(rollart_ctx *ctx, const rollart_kv_pool *pool, const rollart_trajs *trajs,
+                                             const int32_t *traj_ids, int32_t n_items, const int32_t *group_indptr,
+                                             const int32_t *shared_lens, int32_t n_groups, int32_t max_seq_len, const void *q,
+                                             int32_t num_q_heads, float sm_scale, float k_scale, float v_scale, void *out,
+                                             float *lse, void *scratch, size_t scratch_bytes, void *stream);
+
+/*
  * Observation-chunk attention (Sec. 2.1 / 3.1: many-turn tasks keep re-entering generation with
  * a longer history; with the prefix cached only the newly arrived observation tokens are
  * computed, a dense compute-bound block).  Item i owns query rows q_indptr[i] .. q_indptr[i+1]-1;

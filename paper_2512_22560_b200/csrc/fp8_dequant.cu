@@ -58,7 +58,8 @@ __global__ void __launch_bounds__(kThreads)
 fp8_pages_to_bf16_kernel(const uint4 *__restrict__ k_pool, const uint4 *__restrict__ v_pool, int num_pages, int page_size,
                          int num_kv_heads, const int32_t *__restrict__ page_table, int max_pages,
                          const int32_t *__restrict__ seq_lens, int num_traj, const int32_t *__restrict__ traj_ids,
-                         int n_items, int pages_per_item, int max_seq_len, uint4 *__restrict__ k_scratch,
+                         const int32_t *__restrict__ lens_override, int n_items, int pages_per_item, int max_seq_len,
+                         uint4 *__restrict__ k_scratch,
                          uint4 *__restrict__ v_scratch, int32_t *__restrict__ scratch_table,
                          int32_t *__restrict__ scratch_lens, DeviceStatus *status) {
     const int item = blockIdx.x / pages_per_item;
@@ -66,7 +67,8 @@ fp8_pages_to_bf16_kernel(const uint4 *__restrict__ k_pool, const uint4 *__restri
     if (item >= n_items) return;
     const int t = traj_ids ? __ldg(traj_ids + item) : item;
     const bool t_ok = t >= 0 && t < num_traj;
-    int len = t_ok ? __ldg(seq_lens + t) : 0;
+    // lens_override (group decode): only the first lens_override[item] tokens, the group's shared prefix, are wanted
+    const int len = !t_ok ? 0 : lens_override ? __ldg(lens_override + item) : __ldg(seq_lens + t);
     const bool len_ok = len >= 0 && len <= max_seq_len && static_cast<long long>(len) <= static_cast<long long>(max_pages) * page_size;
     const long long s = static_cast<long long>(item) * pages_per_item + lp;      // this block's scratch page
     if (threadIdx.x == 0) {
@@ -132,14 +134,14 @@ Fp8ChunkScratch fp8_chunk_scratch_layout(int n_items, int num_kv_heads, int page
 }
 
 cudaError_t launch_fp8_pages_to_bf16(const rollart_kv_pool &pool, const rollart_trajs &trajs, const int32_t *traj_ids,
-                                     int n_items, int max_seq_len, const Fp8ChunkScratch &L, void *scratch,
-                                     DeviceStatus *status, cudaStream_t stream, int64_t *launches) {
+                                     const int32_t *lens_override, int n_items, int max_seq_len, const Fp8ChunkScratch &L,
+                                     void *scratch, DeviceStatus *status, cudaStream_t stream, int64_t *launches) {
     if (L.num_pages > 0x7FFFFFFFLL) return cudaErrorInvalidValue;
     char *base = static_cast<char *>(scratch);
     fp8_pages_to_bf16_kernel<<<static_cast<unsigned>(L.num_pages), kThreads, 0, stream>>>(
         static_cast<const uint4 *>(pool.k_pool), static_cast<const uint4 *>(pool.v_pool), pool.num_pages, pool.page_size,
-        pool.num_kv_heads, trajs.page_table, trajs.max_pages_per_traj, trajs.seq_lens, trajs.num_traj, traj_ids, n_items,
-        L.pages_per_item, max_seq_len, reinterpret_cast<uint4 *>(base + L.off_k), reinterpret_cast<uint4 *>(base + L.off_v),
+        pool.num_kv_heads, trajs.page_table, trajs.max_pages_per_traj, trajs.seq_lens, trajs.num_traj, traj_ids, lens_override,
+        n_items, L.pages_per_item, max_seq_len, reinterpret_cast<uint4 *>(base + L.off_k), reinterpret_cast<uint4 *>(base + L.off_v),
         reinterpret_cast<int32_t *>(base + L.off_table), reinterpret_cast<int32_t *>(base + L.off_lens), status);
     ++*launches;
     return cudaGetLastError();

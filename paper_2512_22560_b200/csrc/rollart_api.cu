@@ -449,13 +449,16 @@ size_t rollart_group_decode_workspace_size(int32_t max_items, int32_t num_q_head
     return group_layout(max_items, num_q_heads, num_kv_heads, max_seq_len, /*sm_count=*/0).total;
 }
 
-rollart_status rollart_group_decode_attn(rollart_ctx *ctx, const rollart_kv_pool *pool, const rollart_trajs *trajs,
-                                         const int32_t *traj_ids, int32_t n_items, const int32_t *group_indptr,
-                                         const int32_t *shared_lens, int32_t n_groups, int32_t max_seq_len, const void *q,
-                                         int32_t num_q_heads, float sm_scale, void *out, float *lse, void *stream_) {
+static rollart_status group_decode_impl(rollart_ctx *ctx, const rollart_kv_pool *pool, const rollart_trajs *trajs,
+                                        const int32_t *traj_ids, int32_t n_items, const int32_t *group_indptr,
+                                        const int32_t *shared_lens, int32_t n_groups, int32_t max_seq_len, const void *q,
+                                        int32_t num_q_heads, float sm_scale, void *out, float *lse, void *stream_, bool fp8,
+                                        float k_scale, float v_scale, void *scratch, size_t scratch_bytes) {
     if (!ctx) return ROLLART_ERR_INVALID_ARG;
     rollart_status st = attn_common(ctx, pool, trajs, n_items, n_items, max_seq_len, q, num_q_heads, out);
     if (st != ROLLART_OK) return st;
+    if (fp8 && (!(k_scale > 0.f) || !(v_scale > 0.f) || !isfinite(k_scale) || !isfinite(v_scale)))
+        return fail(ctx, ROLLART_ERR_INVALID_ARG, "k_scale and v_scale must be positive and finite");
     if (n_groups < 0 || n_groups > n_items) return fail(ctx, ROLLART_ERR_INVALID_ARG, "n_groups must lie in [0, n_items]");
     if (n_items == 0) return ROLLART_OK;
     if (n_groups == 0) return fail(ctx, ROLLART_ERR_INVALID_ARG, "items without groups");
@@ -464,6 +467,16 @@ rollart_status rollart_group_decode_attn(rollart_ctx *ctx, const rollart_kv_pool
     const GroupLayout lay = group_layout(n_items, num_q_heads, pool->num_kv_heads, max_seq_len, ctx->sm_count);
     if (!ctx->workspace || lay.total > ctx->workspace_bytes)
         return fail(ctx, ROLLART_ERR_WORKSPACE, "workspace of %zu bytes is too small (need %zu)", ctx->workspace_bytes, lay.total);
+    Fp8ChunkScratch sl{};
+    if (fp8) {
+        // the prefixes (one per group) are expanded to bf16 for the tensor-core kernel; the private parts are read as codes
+        sl = fp8_chunk_scratch_layout(n_groups, pool->num_kv_heads, pool->page_size, max_seq_len);
+        if (!scratch || (reinterpret_cast<uintptr_t>(scratch) & 255u) != 0)
+            return fail(ctx, ROLLART_ERR_INVALID_ARG, "scratch must be a 256-byte aligned device buffer");
+        if (scratch_bytes < sl.bytes)
+            return fail(ctx, ROLLART_ERR_WORKSPACE, "scratch of %zu bytes is too small (need %zu)", scratch_bytes, sl.bytes);
+        if (sl.num_pages > 0x7FFFFFFFLL) return fail(ctx, ROLLART_ERR_UNSUPPORTED, "too many scratch pages");
+    }
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return fail(ctx, ROLLART_ERR_CUDA, "cannot select device %d", ctx->device);
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
@@ -491,6 +504,19 @@ rollart_status rollart_group_decode_attn(rollart_ctx *ctx, const rollart_kv_pool
     sc.shared_lens = shared_lens;
     sc.out_f32 = part_a;
     sc.lse = lse_a;
+    if (fp8) {
+        e = launch_fp8_pages_to_bf16(*pool, *trajs, group_traj, shared_lens, n_groups, max_seq_len, sl, scratch, ctx->d_status,
+                                     stream, &ctx->launches);
+        if (e != cudaSuccess) return cuda_fail(ctx, e, "group_decode_attn fp8 expansion launch");
+        char *sb = static_cast<char *>(scratch);
+        sc.pool = PoolView{reinterpret_cast<const __nv_bfloat16 *>(sb + sl.off_k), reinterpret_cast<const __nv_bfloat16 *>(sb + sl.off_v),
+                           static_cast<int>(sl.num_pages), pool->page_size, pool->num_kv_heads};
+        sc.trajs = TrajView{reinterpret_cast<const int32_t *>(sb + sl.off_table), reinterpret_cast<const int32_t *>(sb + sl.off_lens),
+                            sl.pages_per_item, n_groups};
+        sc.traj_ids = nullptr;              // group j is row j of the scratch table
+        sc.sm_scale = sm_scale * k_scale;
+        sc.v_scale = v_scale;
+    }
     e = launch_chunk_attn(sc, stream, &ctx->launches, &too_small);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "group_decode_attn shared-prefix launch");
     // private remainder: the decode kernel over each member's pages after the prefix
@@ -498,6 +524,9 @@ rollart_status rollart_group_decode_attn(rollart_ctx *ctx, const rollart_kv_pool
     pc.page_offset = item_off;
     pc.out_f32 = part_b;
     pc.lse = lse_b;
+    pc.fp8 = fp8;
+    pc.k_scale = k_scale;
+    pc.v_scale = v_scale;
     e = launch_decode_attn(pc, stream, &ctx->launches, &too_small);
     if (too_small) return fail(ctx, ROLLART_ERR_WORKSPACE, "workspace of %zu bytes is too small", ctx->workspace_bytes);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "group_decode_attn decode launch");
@@ -505,6 +534,23 @@ rollart_status rollart_group_decode_attn(rollart_ctx *ctx, const rollart_kv_pool
                            static_cast<__nv_bfloat16 *>(out), lse, stream, &ctx->launches);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "group_decode_attn merge launch");
     return ROLLART_OK;
+}
+
+rollart_status rollart_group_decode_attn(rollart_ctx *ctx, const rollart_kv_pool *pool, const rollart_trajs *trajs,
+                                         const int32_t *traj_ids, int32_t n_items, const int32_t *group_indptr,
+                                         const int32_t *shared_lens, int32_t n_groups, int32_t max_seq_len, const void *q,
+                                         int32_t num_q_heads, float sm_scale, void *out, float *lse, void *stream) {
+    return group_decode_impl(ctx, pool, trajs, traj_ids, n_items, group_indptr, shared_lens, n_groups, max_seq_len, q,
+                             num_q_heads, sm_scale, out, lse, stream, false, 1.f, 1.f, nullptr, 0);
+}
+
+rollart_status rollart_group_decode_attn_fp8(rollart_ctx *ctx, const rollart_kv_pool *pool, const rollart_trajs *trajs,
+                                             const int32_t *traj_ids, int32_t n_items, const int32_t *group_indptr,
+                                             const int32_t *shared_lens, int32_t n_groups, int32_t max_seq_len, const void *q,
+                                             int32_t num_q_heads, float sm_scale, float k_scale, float v_scale, void *out,
+                                             float *lse, void *scratch, size_t scratch_bytes, void *stream) {
+    return group_decode_impl(ctx, pool, trajs, traj_ids, n_items, group_indptr, shared_lens, n_groups, max_seq_len, q,
+                             num_q_heads, sm_scale, out, lse, stream, true, k_scale, v_scale, scratch, scratch_bytes);
 }
 
 rollart_status rollart_obs_chunk_attn(rollart_ctx *ctx, const rollart_kv_pool *pool, const rollart_trajs *trajs,
@@ -555,7 +601,7 @@ rollart_status rollart_obs_chunk_attn_fp8(rollart_ctx *ctx, const rollart_kv_poo
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return fail(ctx, ROLLART_ERR_CUDA, "cannot select device %d", ctx->device);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    cudaError_t e = launch_fp8_pages_to_bf16(*pool, *trajs, traj_ids, n_items, max_seq_len, L, scratch, ctx->d_status, s,
+    cudaError_t e = launch_fp8_pages_to_bf16(*pool, *trajs, traj_ids, nullptr, n_items, max_seq_len, L, scratch, ctx->d_status, s,
                                              &ctx->launches);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "fp8 expansion launch");
     // the attention itself runs over the expanded copy: item i is row i of the scratch table

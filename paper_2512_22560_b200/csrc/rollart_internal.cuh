@@ -128,9 +128,11 @@ struct Fp8ChunkScratch {
     size_t off_k, off_v, off_table, off_lens, bytes;
 };
 Fp8ChunkScratch fp8_chunk_scratch_layout(int n_items, int num_kv_heads, int page_size, int max_seq_len);
+// lens_override (nullable): per item, expand only that many tokens instead of the trajectory's length
 cudaError_t launch_fp8_pages_to_bf16(const rollart_kv_pool &pool, const rollart_trajs &trajs, const int32_t *traj_ids,
-                                     int n_items, int max_seq_len, const Fp8ChunkScratch &layout, void *scratch,
-                                     DeviceStatus *status, cudaStream_t stream, int64_t *launches);
+                                     const int32_t *lens_override, int n_items, int max_seq_len,
+                                     const Fp8ChunkScratch &layout, void *scratch, DeviceStatus *status, cudaStream_t stream,
+                                     int64_t *launches);
 
 // Group decode helpers.  `prepare` derives, per group, the trajectory whose table row stands for the shared
 // prefix and, per item, the pages to skip; it also checks that the members alias the same pages there.

@@ -25,7 +25,7 @@ EXPORTS = (
     "rollart_append_decode_attn", "rollart_group_decode_attn", "rollart_group_decode_workspace_size",
     "rollart_decode_attn_fp8", "rollart_kv_append_fp8", "rollart_append_decode_attn_fp8",
     "rollart_kv_gather_fp8", "rollart_kv_append_fp8_codes", "rollart_obs_chunk_attn_fp8",
-    "rollart_obs_chunk_fp8_scratch_size",
+    "rollart_obs_chunk_fp8_scratch_size", "rollart_group_decode_attn_fp8",
 )
 
 
@@ -99,6 +99,9 @@ def load_library() -> ctypes.CDLL:
     L.rollart_obs_chunk_attn.restype = ctypes.c_int
     L.rollart_obs_chunk_attn.argtypes = [vp, ctypes.POINTER(_KVPool), ctypes.POINTER(_Trajs), vp, vp, i32, i32, i32, vp,
                                          i32, f32, vp, vp, vp]
+    L.rollart_group_decode_attn_fp8.restype = ctypes.c_int
+    L.rollart_group_decode_attn_fp8.argtypes = [vp, ctypes.POINTER(_KVPool), ctypes.POINTER(_Trajs), vp, i32, vp, vp, i32, i32,
+                                                vp, i32, f32, f32, f32, vp, vp, vp, ctypes.c_size_t, vp]
     L.rollart_obs_chunk_fp8_scratch_size.restype = ctypes.c_size_t
     L.rollart_obs_chunk_fp8_scratch_size.argtypes = [i32, i32, i32, i32]
     L.rollart_obs_chunk_attn_fp8.restype = ctypes.c_int
@@ -449,6 +452,31 @@ class Context:
             _ptr(group_indptr, torch.int32, self.device), _ptr(shared_lens, torch.int32, self.device), n_groups,
             int(max_seq_len), _ptr(q, torch.bfloat16, self.device), hq, float(sm_scale),
             _ptr(out, torch.bfloat16, self.device), _ptr(lse, torch.float32, self.device), self._stream(stream))
+        if st != OK:
+            self._raise(st)
+
+    def group_decode_attn_fp8(self, k_pool, v_pool, page_table, seq_lens, group_indptr, shared_lens, q, sm_scale, k_scale,
+                              v_scale, max_seq_len, out, scratch, lse=None, traj_ids=None, stream=None) -> None:
+        """group_decode_attn over pools of E4M3 codes; `scratch` is a uint8 CUDA tensor of at least
+        obs_chunk_fp8_scratch_size(n_groups, num_kv_heads, page_size, max_seq_len) bytes"""
+        pool = self._pool_fp8(k_pool, v_pool)
+        trajs = self._trajs(page_table, seq_lens)
+        if q.dim() != 3 or q.shape != out.shape:
+            raise ValueError("q and out must be [n_items][num_q_heads][head_dim]")
+        n_items, hq, _ = q.shape
+        n_groups = group_indptr.shape[0] - 1
+        if shared_lens.shape[0] != n_groups:
+            raise ValueError("shared_lens must have one entry per group")
+        if traj_ids is not None and traj_ids.shape[0] != n_items:
+            raise ValueError("traj_ids must have one entry per item")
+        if lse is not None and tuple(lse.shape) != (n_items, hq):
+            raise ValueError("lse must be [n_items][num_q_heads]")
+        st = self._lib.rollart_group_decode_attn_fp8(
+            self._h, ctypes.byref(pool), ctypes.byref(trajs), _ptr(traj_ids, torch.int32, self.device), n_items,
+            _ptr(group_indptr, torch.int32, self.device), _ptr(shared_lens, torch.int32, self.device), n_groups,
+            int(max_seq_len), _ptr(q, torch.bfloat16, self.device), hq, float(sm_scale), float(k_scale), float(v_scale),
+            _ptr(out, torch.bfloat16, self.device), _ptr(lse, torch.float32, self.device),
+            _ptr(scratch, torch.uint8, self.device), scratch.numel(), self._stream(stream))
         if st != OK:
             self._raise(st)
 

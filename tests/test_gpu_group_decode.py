@@ -202,3 +202,65 @@ def test_full_size_group_decode_sampled(cuda_device):
     assert_attn_close(out[sel], ref_o, spec.name)
     assert_lse_close(lse[sel], ref_l, spec.name)
     ctx.close()
+
+
+def run_fp8_group_case(spec, seed, group_size, fraction, device, ks=0.03, vs=0.02):
+    """The group call over fp8 pools: the cache is the oracle's quantisation of the bf16 recipe (members alias the same
+    prefix pages, so they hold the same codes), the new token goes through the quantising append; expected values are
+    the oracle's plain fp8 decode over each member's own row."""
+    batch = W.make_batch(spec, seed=seed)
+    indptr, shared = W.share_group_prefix(batch, group_size, fraction)
+    T = spec.num_traj
+    msl = int(batch.seq_lens_after.max())
+    k8 = oracle.fp8_quantize_rows(W.bf16_to_u16(batch.k_pool), ks)
+    v8 = oracle.fp8_quantize_rows(W.bf16_to_u16(batch.v_pool), vs)
+    dk, dv = torch.from_numpy(k8.copy()).to(device), torch.from_numpy(v8.copy()).to(device)
+    table, lens0 = dev_i32(batch.page_table, device), dev_i32(batch.seq_lens_before, device)
+    lens1 = torch.empty_like(lens0)
+    ctx = group_ctx(spec, T, msl)
+    ctx.kv_append_fp8(dk, dv, table, lens0, dev_i32(batch.new_indptr, device), batch.k_new.to(device), batch.v_new.to(device),
+                      ks, vs, seq_lens_out=lens1)
+    after = oracle.kv_append_fp8(k8, v8, batch.page_table, batch.seq_lens_before, batch.new_indptr,
+                                 W.bf16_to_u16(batch.k_new), W.bf16_to_u16(batch.v_new), ks, vs)
+    q = batch.q_new.contiguous().to(device)
+    out = torch.full_like(q, float("nan"))
+    lse = torch.full((T, spec.num_q_heads), float("nan"), device=device)
+    n_groups = len(indptr) - 1
+    need = rollart.obs_chunk_fp8_scratch_size(n_groups, spec.num_kv_heads, spec.page_size, msl)
+    scratch = torch.full((need,), 0xFF, dtype=torch.uint8, device=device)
+    ctx.group_decode_attn_fp8(dk, dv, table, lens1, dev_i32(indptr, device), dev_i32(shared, device), q, spec.sm_scale, ks, vs,
+                              msl, out, scratch, lse=lse)
+    ctx.check()
+    assert np.array_equal(dk.cpu().numpy(), k8) and np.array_equal(dv.cpu().numpy(), v8)
+    ref_o, ref_l = oracle.decode_attn_fp8(k8, v8, batch.page_table, after, W.bf16_to_u16(batch.q_new), spec.sm_scale, ks, vs)
+    assert_attn_close(out, ref_o, f"{spec.name} fp8 group={group_size} frac={fraction}")
+    assert_lse_close(lse, ref_l, spec.name + " fp8")
+    out2 = torch.full_like(q, float("nan"))
+    ctx.decode_attn_fp8(dk, dv, table, lens1, q, spec.sm_scale, ks, vs, msl, out2)
+    ctx.check()
+    assert torch.allclose(out.float(), out2.float(), atol=4e-3, rtol=2e-2)
+    with pytest.raises(rollart.RollartError) as e:
+        ctx.group_decode_attn_fp8(dk, dv, table, lens1, dev_i32(indptr, device), dev_i32(shared, device), q, spec.sm_scale, ks,
+                                  vs, msl, out, scratch[: max(256, need - 256)], lse=lse)
+    assert e.value.status == rollart.ERR_WORKSPACE
+    ctx.close()
+    return shared
+
+
+@pytest.mark.parametrize("group_size,fraction", [(8, 0.6), (8, 1.0), (3, 0.5), (1, 0.7), (8, 0.0), (40, 0.8)])
+def test_fp8_group_decode_matches_oracle_gqa7(cuda_device, group_size, fraction):
+    spec = dataclasses.replace(W.shrink(W.CONFIGS[1], 40, 16), name="fp8_group_gqa7")
+    shared = run_fp8_group_case(spec, 31, group_size, fraction, cuda_device)
+    if fraction > 0 and group_size > 1:
+        assert shared.max() > 0
+
+
+@pytest.mark.parametrize("cfg,div", [(2, 32), (3, 64), (4, 16)])
+def test_fp8_group_decode_other_shapes(cuda_device, cfg, div):
+    spec = dataclasses.replace(W.shrink(W.CONFIGS[cfg], 24, div), chunk_fraction=0.0, name=f"fp8_group_cfg{cfg}")
+    run_fp8_group_case(spec, 32 + cfg, 8, 0.75, cuda_device)
+
+
+def test_fp8_group_decode_many_items(cuda_device):
+    spec = dataclasses.replace(W.CONFIGS[0], num_traj=600, len_lo=40, len_hi=200, name="fp8_group_many")
+    run_fp8_group_case(spec, 35, 1, 0.9, cuda_device)
