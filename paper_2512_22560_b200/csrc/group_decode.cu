@@ -54,13 +54,26 @@ group_prepare_kernel(const int32_t *__restrict__ page_table, const int32_t *__re
     }
     if (bad || b - a < 2 || pages == 0) return;
     const int32_t *row0 = page_table + static_cast<long long>(t0) * max_pages;
-    const long long checks = static_cast<long long>(b - a - 1) * pages;
-    for (long long idx = threadIdx.x; idx < checks; idx += kPrepThreads) {
-        const int m = a + 1 + static_cast<int>(idx / pages), lp = static_cast<int>(idx % pages);
-        const int t = traj_ids ? __ldg(traj_ids + m) : m;
-        if (t < 0 || t >= num_traj) continue;      // reported above
-        if (__ldg(page_table + static_cast<long long>(t) * max_pages + lp) != __ldg(row0 + lp))
-            report(status, ROLLART_ERR_BOUNDS, m, 7);   // this member does not alias the group's prefix pages
+    // every thread keeps its pages of the first member's row and compares the other members' rows against them
+    for (int lp0 = threadIdx.x; lp0 < pages; lp0 += kPrepThreads * 4) {
+        int ref[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const int lp = lp0 + k * kPrepThreads;
+            ref[k] = lp < pages ? __ldg(row0 + lp) : 0;
+        }
+        for (int m = a + 1; m < b; ++m) {
+            const int t = traj_ids ? __ldg(traj_ids + m) : m;
+            if (t < 0 || t >= num_traj) continue;      // reported above
+            const int32_t *row = page_table + static_cast<long long>(t) * max_pages;
+            bool differ = false;
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const int lp = lp0 + k * kPrepThreads;
+                if (lp < pages && __ldg(row + lp) != ref[k]) differ = true;
+            }
+            if (differ) report(status, ROLLART_ERR_BOUNDS, m, 7);   // this member does not alias the group's prefix pages
+        }
     }
 }
 
