@@ -42,7 +42,7 @@ constexpr int kRows = 128;                 // query rows of an M-tile (UMMA M)
 constexpr int kKeys = 64;                  // keys per KV tile
 constexpr int kStages = 8;                 // ring of KV tiles; K(j) and V(j) take alternate slots
 constexpr int kThreads = 384;              // warps 0 / 3 copy K / V, warps 1-2 MMA of M-tile 0 / 1, warps 4-7 / 8-11 softmax of M-tile 0 / 1
-constexpr int kMaxItems = 1024;            // items per launch (tile prefix lives in shared memory)
+constexpr int kMaxItems = kChunkItemsPerLaunch;   // items per launch (tile prefix lives in shared memory)
 constexpr long long kWaitCycles = 2000000000LL;   // a wait gives up after about a second
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
@@ -83,6 +83,7 @@ struct ChunkParams {
     // shared-prefix mode (NULL otherwise): every row of item i sees exactly the first shared_lens[i] keys, no causal mask
     const int32_t *shared_lens;
     float *out_f32;             // when set, result rows go here in fp32 instead of bf16 to `out`
+    const int32_t *item_order;  // NULL, or a permutation of the launch's items: blocks take the items in this order
     DeviceStatus *status;
 };
 
@@ -300,8 +301,13 @@ chunk_attn_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constan
     auto bar_odone = [&](int t, int b) { return bars + 8u * (1 + 2 * kStages + 8 + 2 * t + b); };
 
     // ---- which (item, kv head, pair of M-tiles) is this block?  pairs per item -> prefix -> search ----
+    auto ordered = [&](int k) {        // the k-th item to be taken (clamped: the order is only a schedule, never an index check)
+        if (prm.item_order == nullptr) return k;
+        return min(max(__ldg(prm.item_order + k), 0), prm.n_items - 1);
+    };
     for (int i = threadIdx.x; i < prm.n_items; i += kThreads) {
-        const int n = __ldg(prm.q_indptr + i + 1) - __ldg(prm.q_indptr + i);
+        const int it = ordered(i);
+        const int n = __ldg(prm.q_indptr + it + 1) - __ldg(prm.q_indptr + it);
         s_prefix[i + 1] = n > 0 ? (n + 2 * tpt - 1) / (2 * tpt) : 0;
     }
     if (threadIdx.x == 0) {
@@ -338,7 +344,7 @@ chunk_attn_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constan
             const int mid = (lo + hi) >> 1;
             if (s_prefix[mid] * hkv <= unit) lo = mid; else hi = mid;
         }
-        item = lo;
+        item = ordered(lo);
         const int np = max(1, s_prefix[lo + 1] - s_prefix[lo]);
         const int rem = unit - s_prefix[lo] * hkv;
         head = rem / np;
@@ -858,6 +864,7 @@ cudaError_t launch_chunk_attn(const AttnCall &c, cudaStream_t stream, int64_t *l
         prm.out = c.out; prm.lse = c.lse; prm.scale_log2 = c.sm_scale * kLog2e; prm.out_scale = c.v_scale; prm.status = c.status;
         prm.shared_lens = c.shared_lens ? c.shared_lens + base : nullptr;
         prm.out_f32 = c.out_f32;
+        prm.item_order = c.item_order ? c.item_order + base : nullptr;
         // an upper bound on the M-tile pairs of these items: every item has at most one ragged pair
         const long long pairs = (static_cast<long long>(c.total_q) + 2 * tpt - 1) / (2 * tpt) + n;
         const long long blocks = pairs * hkv;

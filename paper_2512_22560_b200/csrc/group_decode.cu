@@ -21,8 +21,32 @@ __global__ void __launch_bounds__(kPrepThreads)
 group_prepare_kernel(const int32_t *__restrict__ page_table, const int32_t *__restrict__ seq_lens,
                      const int32_t *__restrict__ traj_ids, int n_items, const int32_t *__restrict__ group_indptr,
                      const int32_t *__restrict__ shared_lens, int n_groups, int page_size, int max_pages, int num_traj,
-                     int32_t *__restrict__ group_traj, int32_t *__restrict__ item_page_offset, DeviceStatus *status) {
+                     int32_t *__restrict__ group_traj, int32_t *__restrict__ item_page_offset,
+                     int32_t *__restrict__ group_order, DeviceStatus *status) {
     const int gi = blockIdx.x;
+    {
+        // Rank of this group among the groups of its launch batch by shared length, longest first (ties by index): the
+        // prefix pass takes the groups in that order, so the long ones do not start last.  Whatever the lengths are,
+        // (length, index) is a total order, so the ranks of a batch are a permutation of it.
+        __shared__ int s_cnt[kPrepThreads / 32];
+        const int base = gi / kChunkItemsPerLaunch * kChunkItemsPerLaunch;
+        const int n = min(kChunkItemsPerLaunch, n_groups - base);
+        const int mine = __ldg(shared_lens + gi);
+        int cnt = 0;
+        for (int j = threadIdx.x; j < n; j += kPrepThreads) {
+            const int v = __ldg(shared_lens + base + j);
+            cnt += (v > mine || (v == mine && base + j < gi)) ? 1 : 0;
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
+        if ((threadIdx.x & 31) == 0) s_cnt[threadIdx.x >> 5] = cnt;
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            int rank = 0;
+            for (int w = 0; w < kPrepThreads / 32; ++w) rank += s_cnt[w];
+            group_order[base + rank] = gi - base;
+        }
+    }
     const int a = __ldg(group_indptr + gi), b = __ldg(group_indptr + gi + 1);
     const int s_len = __ldg(shared_lens + gi);
     bool bad = a < 0 || b < a || b > n_items || (gi == 0 && a != 0) || (gi == n_groups - 1 && b != n_items);
@@ -107,12 +131,13 @@ group_merge_kernel(const float *__restrict__ part_a, const float *__restrict__ l
 
 cudaError_t launch_group_prepare(const TrajView &trajs, const int32_t *traj_ids, int n_items, const int32_t *group_indptr,
                                  const int32_t *shared_lens, int n_groups, int page_size, int32_t *group_traj,
-                                 int32_t *item_page_offset, DeviceStatus *status, cudaStream_t stream, int64_t *launches) {
+                                 int32_t *item_page_offset, int32_t *group_order, DeviceStatus *status, cudaStream_t stream,
+                                 int64_t *launches) {
     if (n_groups <= 0) return cudaSuccess;
     group_prepare_kernel<<<n_groups, kPrepThreads, 0, stream>>>(trajs.page_table, trajs.seq_lens, traj_ids, n_items,
                                                                 group_indptr, shared_lens, n_groups, page_size,
                                                                 trajs.max_pages, trajs.num_traj, group_traj,
-                                                                item_page_offset, status);
+                                                                item_page_offset, group_order, status);
     ++*launches;
     return cudaGetLastError();
 }

@@ -108,6 +108,7 @@ AttnCall make_call(rollart_ctx *ctx, const rollart_kv_pool *pool, const rollart_
     c.page_offset = nullptr;
     c.shared_lens = nullptr;
     c.out_f32 = nullptr;
+    c.item_order = nullptr;
     c.fp8 = false;
     c.k_scale = 1.f;
     c.v_scale = 1.f;
@@ -426,7 +427,7 @@ rollart_status rollart_append_decode_attn_fp8(rollart_ctx *ctx, const rollart_kv
 namespace {
 // Workspace of a group decode call: the decode kernel's own workspace first, then these arrays.
 struct GroupLayout {
-    size_t group_traj, item_off, lse_a, lse_b, part_a, part_b, total;
+    size_t group_traj, item_off, group_order, lse_a, lse_b, part_a, part_b, total;
 };
 GroupLayout group_layout(int n_items, int num_q_heads, int num_kv_heads, int max_seq_len, int sm_count) {
     auto up = [](size_t x) { return (x + 255) & ~size_t(255); };
@@ -435,6 +436,7 @@ GroupLayout group_layout(int n_items, int num_q_heads, int num_kv_heads, int max
     size_t at = up(decode_workspace_bytes(n_items, num_q_heads, num_kv_heads, max_seq_len, sm_count));
     g.group_traj = at; at += up(sizeof(int32_t) * static_cast<size_t>(n_items));
     g.item_off = at;   at += up(sizeof(int32_t) * static_cast<size_t>(n_items));
+    g.group_order = at; at += up(sizeof(int32_t) * static_cast<size_t>(n_items));
     g.lse_a = at;      at += up(sizeof(float) * rows);
     g.lse_b = at;      at += up(sizeof(float) * rows);
     g.part_a = at;     at += up(sizeof(float) * rows * kHeadDim);
@@ -483,6 +485,7 @@ static rollart_status group_decode_impl(rollart_ctx *ctx, const rollart_kv_pool 
     char *ws = static_cast<char *>(ctx->workspace);
     int32_t *group_traj = reinterpret_cast<int32_t *>(ws + lay.group_traj);
     int32_t *item_off = reinterpret_cast<int32_t *>(ws + lay.item_off);
+    int32_t *group_order = reinterpret_cast<int32_t *>(ws + lay.group_order);
     float *lse_a = reinterpret_cast<float *>(ws + lay.lse_a), *lse_b = reinterpret_cast<float *>(ws + lay.lse_b);
     float *part_a = reinterpret_cast<float *>(ws + lay.part_a), *part_b = reinterpret_cast<float *>(ws + lay.part_b);
 
@@ -492,7 +495,7 @@ static rollart_status group_decode_impl(rollart_ctx *ctx, const rollart_kv_pool 
     AttnCall base = make_call(ctx, pool, trajs, traj_ids, nullptr, n_items, n_items, max_seq_len, q, num_q_heads, sm_scale,
                               out, lse);
     e = launch_group_prepare(base.trajs, traj_ids, n_items, group_indptr, shared_lens, n_groups, pool->page_size, group_traj,
-                             item_off, ctx->d_status, stream, &ctx->launches);
+                             item_off, group_order, ctx->d_status, stream, &ctx->launches);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "group_decode_attn prepare launch");
 
     bool too_small = false;
@@ -504,6 +507,7 @@ static rollart_status group_decode_impl(rollart_ctx *ctx, const rollart_kv_pool 
     sc.shared_lens = shared_lens;
     sc.out_f32 = part_a;
     sc.lse = lse_a;
+    sc.item_order = group_order;        // longest prefixes first: the blocks of this pass differ a lot in length
     if (fp8) {
         e = launch_fp8_pages_to_bf16(*pool, *trajs, group_traj, shared_lens, n_groups, max_seq_len, sl, scratch, ctx->d_status,
                                      stream, &ctx->launches);

@@ -107,6 +107,7 @@ struct AttnCall {
     const int32_t *page_offset;   // decode: per item, pages of the table row to skip (the keys before them are not attended to)
     const int32_t *shared_lens;   // chunk: per item, every query row of the item sees exactly the first shared_lens[i] keys
     float *out_f32;               // when set the result rows are written here in fp32 instead of bf16 to `out`
+    const int32_t *item_order;    // chunk: per batch of kChunkItemsPerLaunch items, the order in which blocks take them
     // fp8 (E4M3) pools (decode and fused append + decode): keys are k_scale * code value, values v_scale * code value.
     // The chunk kernel reads bf16 only; it multiplies its result by v_scale (1 for bf16 pools).
     bool fp8;
@@ -134,11 +135,15 @@ cudaError_t launch_fp8_pages_to_bf16(const rollart_kv_pool &pool, const rollart_
                                      const Fp8ChunkScratch &layout, void *scratch, DeviceStatus *status, cudaStream_t stream,
                                      int64_t *launches);
 
+// items per launch of the chunk kernel (its per-item table lives in shared memory)
+constexpr int kChunkItemsPerLaunch = 1024;
+
 // Group decode helpers.  `prepare` derives, per group, the trajectory whose table row stands for the shared
 // prefix and, per item, the pages to skip; it also checks that the members alias the same pages there.
 cudaError_t launch_group_prepare(const TrajView &trajs, const int32_t *traj_ids, int n_items, const int32_t *group_indptr,
                                  const int32_t *shared_lens, int n_groups, int page_size, int32_t *group_traj,
-                                 int32_t *item_page_offset, DeviceStatus *status, cudaStream_t stream, int64_t *launches);
+                                 int32_t *item_page_offset, int32_t *group_order, DeviceStatus *status, cudaStream_t stream,
+                                 int64_t *launches);
 // out = softmax-weighted sum of the two partial results (weights from their log-sum-exps); lse optional
 cudaError_t launch_group_merge(const float *part_a, const float *lse_a, const float *part_b, const float *lse_b,
                                long long rows, __nv_bfloat16 *out, float *lse, cudaStream_t stream, int64_t *launches);
