@@ -67,11 +67,12 @@ def test_group_decode_other_shapes(cuda_device, cfg, div):
     run_group_case(spec, 32 + cfg, 8, 0.75, cuda_device)
 
 
-@pytest.mark.parametrize("group_size", [8, 1])
-def test_group_decode_many_items(cuda_device, group_size):
-    # more items (and, with groups of one, more groups) than one launch of either kernel takes (512):
-    # the per-launch offsets of every array
-    spec = dataclasses.replace(W.CONFIGS[0], num_traj=600, len_lo=40, len_hi=200, name="group_many")
+@pytest.mark.parametrize("group_size,num_traj", [(8, 600), (1, 600), (1, 1100), (2, 2300)])
+def test_group_decode_many_items(cuda_device, group_size, num_traj):
+    # more items (and, with small groups, more groups) than one launch of either kernel takes (512 items for the
+    # decode kernel, 1024 groups for the prefix pass, whose longest-first order is per launch): the per-launch
+    # offsets of every array
+    spec = dataclasses.replace(W.CONFIGS[0], num_traj=num_traj, len_lo=40, len_hi=200, name="group_many")
     run_group_case(spec, 35, group_size, 0.9, cuda_device, poison=False)
 
 
@@ -261,6 +262,7 @@ def test_fp8_group_decode_other_shapes(cuda_device, cfg, div):
     run_fp8_group_case(spec, 32 + cfg, 8, 0.75, cuda_device)
 
 
-def test_fp8_group_decode_many_items(cuda_device):
-    spec = dataclasses.replace(W.CONFIGS[0], num_traj=600, len_lo=40, len_hi=200, name="fp8_group_many")
+@pytest.mark.parametrize("num_traj", [600, 1100])
+def test_fp8_group_decode_many_items(cuda_device, num_traj):
+    spec = dataclasses.replace(W.CONFIGS[0], num_traj=num_traj, len_lo=40, len_hi=200, name="fp8_group_many")
     run_fp8_group_case(spec, 35, 1, 0.9, cuda_device)
