@@ -395,3 +395,32 @@ def test_fp8_empty_items_and_empty_calls(cuda_device):
     ctx.check()
     assert ctx.launch_count == n0          # nothing was enqueued
     ctx.close()
+
+
+def test_fp8_reruns_are_bit_identical(cuda_device):
+    # fixed schedule, fixed merge and combine order, no float atomics: the fp8 decode and chunk calls repeat bit for bit
+    batch = W.make_batch(W.shrink(W.CONFIGS[4], 10, 8, 16), seed=88)
+    spec = batch.spec
+    ctx, (dk, dv, table, lens1), (q, q_indptr, ids, msl), out = run_fp8_chunk_case(batch, cuda_device)
+    need = rollart.obs_chunk_fp8_scratch_size(len(ids), spec.num_kv_heads, spec.page_size, msl)
+    scratch = torch.empty(need, dtype=torch.uint8, device=cuda_device)
+    qg, qi, tid = q.to(cuda_device), dev_i32(q_indptr, cuda_device), dev_i32(ids, cuda_device)
+    lse0 = torch.empty(q.shape[0], spec.num_q_heads, device=cuda_device)
+    for _ in range(3):
+        o = torch.full_like(out, float("nan"))
+        lse = torch.full_like(lse0, float("nan"))
+        ctx.obs_chunk_attn_fp8(dk, dv, table, lens1, qi, qg, spec.sm_scale, KS, VS, msl, o, scratch, lse=lse, traj_ids=tid)
+        ctx.check()
+        assert torch.equal(o.view(torch.int16), out.view(torch.int16))
+        lse0 = lse if _ == 0 else lse0
+        assert torch.equal(lse, lse0)
+    dids = dev_i32(batch.decode_ids, cuda_device)
+    qd = batch.q_new[torch.from_numpy(batch.decode_rows())].contiguous().to(cuda_device)
+    first = None
+    for _ in range(3):
+        o = torch.full_like(qd, float("nan"))
+        ctx.decode_attn_fp8(dk, dv, table, lens1, qd, spec.sm_scale, KS, VS, msl, o, traj_ids=dids)
+        ctx.check()
+        first = o if first is None else first
+        assert torch.equal(o.view(torch.int16), first.view(torch.int16))
+    ctx.close()
