@@ -281,10 +281,11 @@ rollart_status rollart_group_decode_attn(rollart_ctx *ctx, const rollart_kv_pool
  * v_scale * value(code) (pools of E4M3 codes as for rollart_decode_attn_fp8).  The shared prefixes, one per group,
  * are expanded to bf16 into `scratch` for the tensor-core kernel (as rollart_obs_chunk_attn_fp8 does for whole
  * contexts); the private remainders are read as codes by the fp8 decode kernel.
- *   scratch   [device] 256-byte aligned, at least rollart_obs_chunk_fp8_scratch_size(n_groups, num_kv_heads, page_size,
- *             max_seq_len) bytes; owned by the caller, contents undefined afterwards.
- * Workspace, checks and errors as for rollart_group_decode_attn; a scratch buffer that is too small returns
- * ROLLART_ERR_WORKSPACE and launches nothing.  Launches five kernels.
+ *   scratch   [device] 256-byte aligned, sized as for rollart_obs_chunk_attn_fp8 with the groups as items and the shared
+ *             prefixes as their contexts (rollart_obs_chunk_fp8_scratch_size(n_groups, ...) always suffices); owned by
+ *             the caller, contents undefined afterwards.
+ * Workspace, checks and errors as for rollart_group_decode_attn; scratch errors as for rollart_obs_chunk_attn_fp8.
+ * Launches six kernels.
  */
 rollart_status rollart_group_decode_attn_fp8(rollart_ctx *ctx, const rollart_kv_pool *pool, const rollart_trajs *trajs,
                                              const int32_t *traj_ids, int32_t n_items, const int32_t *group_indptr,
@@ -315,14 +316,21 @@ rollart_status rollart_obs_chunk_attn(rollart_ctx *ctx, const rollart_kv_pool *p
  * This phase is bound by the tensor cores, not by reading the cache (Sec. 3.1), so the call first expands the listed
  * trajectories' contexts to bf16 (exact: every finite E4M3 value is a bf16 value) into `scratch` and then runs the
  * bf16 kernel over that copy; the expansion is one pass at the HBM rate, a few per cent of the attention.
- *   scratch        [device] 256-byte aligned, at least rollart_obs_chunk_fp8_scratch_size(n_items, num_kv_heads,
- *                  page_size, max_seq_len) bytes (two bf16 pools of n_items * ceil(max_seq_len / page_size) pages plus
- *                  a page table and lengths for them); owned by the caller, contents undefined afterwards.  A smaller
- *                  buffer returns ROLLART_ERR_WORKSPACE and launches nothing.
+ *   scratch        [device] 256-byte aligned; owned by the caller, contents undefined afterwards.  It holds two bf16
+ *                  pools into which the items' pages are packed one after the other (a running sum of
+ *                  ceil(L / page_size) taken on the device), plus a page table, lengths and offsets for them.
+ *                  rollart_obs_chunk_fp8_scratch_size(n_items, num_kv_heads, page_size, max_seq_len) bytes always
+ *                  suffice (every item at the bound); rollart_obs_chunk_fp8_scratch_size_for_pages(..., total_pages)
+ *                  gives the size for a caller who knows a bound on the pages the listed contexts hold (its page
+ *                  allocator does).  A buffer that cannot hold one page returns ROLLART_ERR_WORKSPACE and launches
+ *                  nothing; one that turns out smaller than the contexts is a device-side ROLLART_ERR_WORKSPACE:
+ *                  the items that do not fit are skipped (their rows of out are not written).
  *   other arguments, errors and arithmetic as for rollart_obs_chunk_attn (bf16 operands: here the exact code values).
- * Launches two kernels.  A code of NaN in a live slot gives NaN results for the rows that see it, as a bf16 NaN would.
+ * Launches three kernels.  A code of NaN in a live slot gives NaN results for the rows that see it, as a bf16 NaN would.
  */
 size_t rollart_obs_chunk_fp8_scratch_size(int32_t n_items, int32_t num_kv_heads, int32_t page_size, int32_t max_seq_len);
+size_t rollart_obs_chunk_fp8_scratch_size_for_pages(int32_t n_items, int32_t num_kv_heads, int32_t page_size,
+                                                    int32_t max_seq_len, int64_t total_pages);
 rollart_status rollart_obs_chunk_attn_fp8(rollart_ctx *ctx, const rollart_kv_pool *pool, const rollart_trajs *trajs,
                                           const int32_t *traj_ids, const int32_t *q_indptr, int32_t n_items,
                                           int32_t total_q, int32_t max_seq_len, const void *q, int32_t num_q_heads,

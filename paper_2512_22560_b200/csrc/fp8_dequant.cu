@@ -6,10 +6,11 @@
 // The chunk path is bound by the tensor cores (Sec. 3.1: prefill is the compute-bound phase), so one extra pass over
 // the context at the HBM rate (1 byte read, 2 written per element) costs a few per cent of the attention itself.
 //
-// Scratch layout: item i of the call owns scratch pages i * pages_per_item .. (i + 1) * pages_per_item - 1 in logical
-// order, pages_per_item = ceil(max_seq_len / page_size); the scratch page table row of item i lists exactly those
-// ids, and its length is the trajectory's.  One thread block expands one (item, logical page): all kv heads of a page
-// are one contiguous run in both pools.
+// Scratch layout: two bf16 pools of `capacity_pages` pages, then a page table [n_items][pages_per_item]
+// (pages_per_item = ceil(max_seq_len / page_size)), the lengths, and the first scratch page of every item.  The items'
+// pages are packed one after the other in logical order (a plan kernel takes the running sum of ceil(len / page_size)
+// on the device), so the pools need as many pages as the listed contexts hold, not n_items times the longest bound.
+// One thread block expands one (item, logical page): all kv heads of a page are one contiguous run in both pools.
 #include "rollart_internal.cuh"
 
 namespace rollart {
@@ -54,32 +55,87 @@ __device__ __forceinline__ void expand16(const uint4 &codes, uint4 &lo, uint4 &h
     expand4(codes.w, hi.z, hi.w);
 }
 
+constexpr int kPlanThreads = 1024;
+
+// One block: validates every item, writes its length (0 for a bad item, which is reported and then attends to nothing)
+// and the index of its first scratch page (running sum of the page counts, items in call order).
+__global__ void __launch_bounds__(kPlanThreads)
+fp8_scratch_plan_kernel(const int32_t *__restrict__ seq_lens, int num_traj, const int32_t *__restrict__ traj_ids,
+                        const int32_t *__restrict__ lens_override, int n_items, int page_size, int max_pages, int max_seq_len,
+                        long long capacity_pages, int32_t *__restrict__ scratch_lens, int32_t *__restrict__ first_page,
+                        DeviceStatus *status) {
+    __shared__ int s_warp[kPlanThreads / 32];
+    __shared__ long long s_carry;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (threadIdx.x == 0) s_carry = 0;
+    __syncthreads();
+    for (int base = 0; base < n_items; base += kPlanThreads) {
+        const int item = base + threadIdx.x;
+        int len = 0, pages = 0;
+        if (item < n_items) {
+            const int t = traj_ids ? __ldg(traj_ids + item) : item;
+            if (t < 0 || t >= num_traj) {
+                report(status, ROLLART_ERR_BOUNDS, t, 3);
+            } else {
+                // lens_override (group decode): only the first lens_override[item] tokens, the group's shared prefix
+                len = lens_override ? __ldg(lens_override + item) : __ldg(seq_lens + t);
+                if (len < 0 || len > max_seq_len || static_cast<long long>(len) > static_cast<long long>(max_pages) * page_size) {
+                    report(status, ROLLART_ERR_BOUNDS, len, 3);
+                    len = 0;
+                }
+            }
+            pages = (len + page_size - 1) / page_size;
+        }
+        // exclusive prefix of `pages` over the block, on top of the carry of the earlier rounds
+        int incl = pages;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int v = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += v;
+        }
+        if (lane == 31) s_warp[warp] = incl;
+        __syncthreads();
+        if (warp == 0) {
+            int w = s_warp[lane];
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int v = __shfl_up_sync(0xffffffffu, w, o);
+                if (lane >= o) w += v;
+            }
+            s_warp[lane] = w;                      // inclusive over the warps
+        }
+        __syncthreads();
+        const long long before = s_carry + (warp > 0 ? s_warp[warp - 1] : 0) + (incl - pages);
+        if (item < n_items) {
+            if (before + pages > capacity_pages) {        // the scratch pools are smaller than the contexts listed
+                report(status, ROLLART_ERR_WORKSPACE, item, 3);
+                len = 0;
+            }
+            scratch_lens[item] = len;
+            first_page[item] = static_cast<int32_t>(before < 0x7FFFFFFFLL ? before : 0x7FFFFFFFLL);
+        }
+        __syncthreads();
+        if (threadIdx.x == kPlanThreads - 1) s_carry += s_warp[kPlanThreads / 32 - 1];
+        __syncthreads();
+    }
+}
+
 __global__ void __launch_bounds__(kThreads)
 fp8_pages_to_bf16_kernel(const uint4 *__restrict__ k_pool, const uint4 *__restrict__ v_pool, int num_pages, int page_size,
-                         int num_kv_heads, const int32_t *__restrict__ page_table, int max_pages,
-                         const int32_t *__restrict__ seq_lens, int num_traj, const int32_t *__restrict__ traj_ids,
-                         const int32_t *__restrict__ lens_override, int n_items, int pages_per_item, int max_seq_len,
-                         uint4 *__restrict__ k_scratch,
-                         uint4 *__restrict__ v_scratch, int32_t *__restrict__ scratch_table,
-                         int32_t *__restrict__ scratch_lens, DeviceStatus *status) {
+                         int num_kv_heads, const int32_t *__restrict__ page_table, int max_pages, int num_traj,
+                         const int32_t *__restrict__ traj_ids, int n_items, int pages_per_item,
+                         const int32_t *__restrict__ scratch_lens, const int32_t *__restrict__ first_page,
+                         uint4 *__restrict__ k_scratch, uint4 *__restrict__ v_scratch, int32_t *__restrict__ scratch_table,
+                         DeviceStatus *status) {
     const int item = blockIdx.x / pages_per_item;
     const int lp = blockIdx.x - item * pages_per_item;
     if (item >= n_items) return;
-    const int t = traj_ids ? __ldg(traj_ids + item) : item;
-    const bool t_ok = t >= 0 && t < num_traj;
-    // lens_override (group decode): only the first lens_override[item] tokens, the group's shared prefix, are wanted
-    const int len = !t_ok ? 0 : lens_override ? __ldg(lens_override + item) : __ldg(seq_lens + t);
-    const bool len_ok = len >= 0 && len <= max_seq_len && static_cast<long long>(len) <= static_cast<long long>(max_pages) * page_size;
-    const long long s = static_cast<long long>(item) * pages_per_item + lp;      // this block's scratch page
-    if (threadIdx.x == 0) {
-        scratch_table[s] = static_cast<int32_t>(s);
-        if (lp == 0) {
-            if (!t_ok) report(status, ROLLART_ERR_BOUNDS, t, 3);
-            else if (!len_ok) report(status, ROLLART_ERR_BOUNDS, len, 3);
-            scratch_lens[item] = t_ok && len_ok ? len : 0;    // a bad item is reported and then attends to nothing
-        }
-    }
-    if (!t_ok || !len_ok || static_cast<long long>(lp) * page_size >= len) return;
+    const int len = __ldg(scratch_lens + item);                      // validated by the plan kernel, 0 for a bad item
+    if (static_cast<long long>(lp) * page_size >= len) return;
+    const int t = traj_ids ? __ldg(traj_ids + item) : item;          // in range: len > 0
+    if (t < 0 || t >= num_traj) return;
+    const long long s = static_cast<long long>(__ldg(first_page + item)) + lp;      // this block's scratch page
+    if (threadIdx.x == 0) scratch_table[static_cast<long long>(item) * pages_per_item + lp] = static_cast<int32_t>(s);
     const int pg = __ldg(page_table + static_cast<long long>(t) * max_pages + lp);
     if (pg < 0 || pg >= num_pages) {
         if (threadIdx.x == 0) report(status, ROLLART_ERR_BOUNDS, pg, 3);
@@ -119,30 +175,65 @@ size_t align_up(size_t x) { return (x + 255) & ~static_cast<size_t>(255); }
 
 }  // namespace
 
-Fp8ChunkScratch fp8_chunk_scratch_layout(int n_items, int num_kv_heads, int page_size, int max_seq_len) {
-    Fp8ChunkScratch L;
+namespace {
+// the small arrays behind the pools: page table, lengths, first page of every item
+size_t tail_bytes(int n_items, int pages_per_item) {
+    return align_up(static_cast<size_t>(n_items) * pages_per_item * sizeof(int32_t)) +
+           2 * align_up(static_cast<size_t>(n_items) * sizeof(int32_t));
+}
+}  // namespace
+
+size_t fp8_chunk_scratch_bytes(int n_items, int num_kv_heads, int page_size, int max_seq_len, long long total_pages) {
+    int ppi = (max_seq_len + page_size - 1) / page_size;
+    if (ppi < 1) ppi = 1;
+    const long long worst = static_cast<long long>(n_items) * ppi;
+    if (total_pages < 0 || total_pages > worst) total_pages = worst;
+    if (total_pages < 1) total_pages = 1;
+    const size_t pool_bytes = align_up(static_cast<size_t>(total_pages) * num_kv_heads * page_size * kRowBytes);
+    return 2 * pool_bytes + tail_bytes(n_items, ppi);
+}
+
+Fp8ChunkScratch fp8_chunk_scratch_layout(int n_items, int num_kv_heads, int page_size, int max_seq_len, size_t scratch_bytes) {
+    Fp8ChunkScratch L{};
     L.pages_per_item = (max_seq_len + page_size - 1) / page_size;
     if (L.pages_per_item < 1) L.pages_per_item = 1;
-    L.num_pages = static_cast<long long>(n_items) * L.pages_per_item;
-    const size_t pool_bytes = static_cast<size_t>(L.num_pages) * num_kv_heads * page_size * kRowBytes;
+    const size_t tail = tail_bytes(n_items, L.pages_per_item);
+    const size_t page_bytes = static_cast<size_t>(num_kv_heads) * page_size * kRowBytes;
+    L.capacity_pages = 0;
+    if (scratch_bytes > tail + 512) {
+        const size_t each = ((scratch_bytes - tail) / 2) & ~static_cast<size_t>(255);     // one pool, 256-byte aligned
+        L.capacity_pages = static_cast<long long>(each / page_bytes);
+    }
+    const long long worst = static_cast<long long>(n_items) * L.pages_per_item;
+    if (L.capacity_pages > worst) L.capacity_pages = worst;
+    const size_t pool_bytes = align_up(static_cast<size_t>(L.capacity_pages) * page_bytes);
     L.off_k = 0;
-    L.off_v = align_up(pool_bytes);
-    L.off_table = L.off_v + align_up(pool_bytes);
-    L.off_lens = L.off_table + align_up(static_cast<size_t>(L.num_pages) * sizeof(int32_t));
-    L.bytes = L.off_lens + align_up(static_cast<size_t>(n_items) * sizeof(int32_t));
+    L.off_v = pool_bytes;
+    L.off_table = 2 * pool_bytes;
+    L.off_lens = L.off_table + align_up(static_cast<size_t>(n_items) * L.pages_per_item * sizeof(int32_t));
+    L.off_first = L.off_lens + align_up(static_cast<size_t>(n_items) * sizeof(int32_t));
+    L.bytes = L.off_first + align_up(static_cast<size_t>(n_items) * sizeof(int32_t));
     return L;
 }
 
 cudaError_t launch_fp8_pages_to_bf16(const rollart_kv_pool &pool, const rollart_trajs &trajs, const int32_t *traj_ids,
                                      const int32_t *lens_override, int n_items, int max_seq_len, const Fp8ChunkScratch &L,
                                      void *scratch, DeviceStatus *status, cudaStream_t stream, int64_t *launches) {
-    if (L.num_pages > 0x7FFFFFFFLL) return cudaErrorInvalidValue;
+    const long long blocks = static_cast<long long>(n_items) * L.pages_per_item;
+    if (blocks > 0x7FFFFFFFLL || L.capacity_pages > 0x7FFFFFFFLL) return cudaErrorInvalidValue;
     char *base = static_cast<char *>(scratch);
-    fp8_pages_to_bf16_kernel<<<static_cast<unsigned>(L.num_pages), kThreads, 0, stream>>>(
+    int32_t *lens = reinterpret_cast<int32_t *>(base + L.off_lens), *first = reinterpret_cast<int32_t *>(base + L.off_first);
+    fp8_scratch_plan_kernel<<<1, kPlanThreads, 0, stream>>>(trajs.seq_lens, trajs.num_traj, traj_ids, lens_override, n_items,
+                                                            pool.page_size, trajs.max_pages_per_traj, max_seq_len,
+                                                            L.capacity_pages, lens, first, status);
+    ++*launches;
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    fp8_pages_to_bf16_kernel<<<static_cast<unsigned>(blocks), kThreads, 0, stream>>>(
         static_cast<const uint4 *>(pool.k_pool), static_cast<const uint4 *>(pool.v_pool), pool.num_pages, pool.page_size,
-        pool.num_kv_heads, trajs.page_table, trajs.max_pages_per_traj, trajs.seq_lens, trajs.num_traj, traj_ids, lens_override,
-        n_items, L.pages_per_item, max_seq_len, reinterpret_cast<uint4 *>(base + L.off_k), reinterpret_cast<uint4 *>(base + L.off_v),
-        reinterpret_cast<int32_t *>(base + L.off_table), reinterpret_cast<int32_t *>(base + L.off_lens), status);
+        pool.num_kv_heads, trajs.page_table, trajs.max_pages_per_traj, trajs.num_traj, traj_ids, n_items, L.pages_per_item, lens,
+        first, reinterpret_cast<uint4 *>(base + L.off_k), reinterpret_cast<uint4 *>(base + L.off_v),
+        reinterpret_cast<int32_t *>(base + L.off_table), status);
     ++*launches;
     return cudaGetLastError();
 }

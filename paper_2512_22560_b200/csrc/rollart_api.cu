@@ -472,12 +472,13 @@ static rollart_status group_decode_impl(rollart_ctx *ctx, const rollart_kv_pool 
     Fp8ChunkScratch sl{};
     if (fp8) {
         // the prefixes (one per group) are expanded to bf16 for the tensor-core kernel; the private parts are read as codes
-        sl = fp8_chunk_scratch_layout(n_groups, pool->num_kv_heads, pool->page_size, max_seq_len);
+        sl = fp8_chunk_scratch_layout(n_groups, pool->num_kv_heads, pool->page_size, max_seq_len, scratch_bytes);
         if (!scratch || (reinterpret_cast<uintptr_t>(scratch) & 255u) != 0)
             return fail(ctx, ROLLART_ERR_INVALID_ARG, "scratch must be a 256-byte aligned device buffer");
-        if (scratch_bytes < sl.bytes)
-            return fail(ctx, ROLLART_ERR_WORKSPACE, "scratch of %zu bytes is too small (need %zu)", scratch_bytes, sl.bytes);
-        if (sl.num_pages > 0x7FFFFFFFLL) return fail(ctx, ROLLART_ERR_UNSUPPORTED, "too many scratch pages");
+        if (sl.capacity_pages < 1)
+            return fail(ctx, ROLLART_ERR_WORKSPACE, "scratch of %zu bytes cannot hold a single page", scratch_bytes);
+        if (static_cast<long long>(n_groups) * sl.pages_per_item > 0x7FFFFFFFLL)
+            return fail(ctx, ROLLART_ERR_UNSUPPORTED, "too many scratch pages");
     }
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return fail(ctx, ROLLART_ERR_CUDA, "cannot select device %d", ctx->device);
@@ -514,7 +515,7 @@ static rollart_status group_decode_impl(rollart_ctx *ctx, const rollart_kv_pool 
         if (e != cudaSuccess) return cuda_fail(ctx, e, "group_decode_attn fp8 expansion launch");
         char *sb = static_cast<char *>(scratch);
         sc.pool = PoolView{reinterpret_cast<const __nv_bfloat16 *>(sb + sl.off_k), reinterpret_cast<const __nv_bfloat16 *>(sb + sl.off_v),
-                           static_cast<int>(sl.num_pages), pool->page_size, pool->num_kv_heads};
+                           static_cast<int>(sl.capacity_pages), pool->page_size, pool->num_kv_heads};
         sc.trajs = TrajView{reinterpret_cast<const int32_t *>(sb + sl.off_table), reinterpret_cast<const int32_t *>(sb + sl.off_lens),
                             sl.pages_per_item, n_groups};
         sc.traj_ids = nullptr;              // group j is row j of the scratch table
@@ -580,7 +581,13 @@ rollart_status rollart_obs_chunk_attn(rollart_ctx *ctx, const rollart_kv_pool *p
 
 size_t rollart_obs_chunk_fp8_scratch_size(int32_t n_items, int32_t num_kv_heads, int32_t page_size, int32_t max_seq_len) {
     if (n_items <= 0 || num_kv_heads <= 0 || page_size <= 0 || max_seq_len < 0) return 0;
-    return fp8_chunk_scratch_layout(n_items, num_kv_heads, page_size, max_seq_len).bytes;
+    return fp8_chunk_scratch_bytes(n_items, num_kv_heads, page_size, max_seq_len, -1);
+}
+
+size_t rollart_obs_chunk_fp8_scratch_size_for_pages(int32_t n_items, int32_t num_kv_heads, int32_t page_size,
+                                                    int32_t max_seq_len, int64_t total_pages) {
+    if (n_items <= 0 || num_kv_heads <= 0 || page_size <= 0 || max_seq_len < 0 || total_pages < 0) return 0;
+    return fp8_chunk_scratch_bytes(n_items, num_kv_heads, page_size, max_seq_len, total_pages);
 }
 
 rollart_status rollart_obs_chunk_attn_fp8(rollart_ctx *ctx, const rollart_kv_pool *pool, const rollart_trajs *trajs,
@@ -596,12 +603,13 @@ rollart_status rollart_obs_chunk_attn_fp8(rollart_ctx *ctx, const rollart_kv_poo
     if (n_items == 0 || total_q == 0) return ROLLART_OK;
     if (!q_indptr) return fail(ctx, ROLLART_ERR_INVALID_ARG, "q_indptr NULL");
     max_seq_len = clamp_bound(pool, trajs, max_seq_len);
-    const Fp8ChunkScratch L = fp8_chunk_scratch_layout(n_items, pool->num_kv_heads, pool->page_size, max_seq_len);
+    const Fp8ChunkScratch L = fp8_chunk_scratch_layout(n_items, pool->num_kv_heads, pool->page_size, max_seq_len, scratch_bytes);
     if (!scratch || (reinterpret_cast<uintptr_t>(scratch) & 255u) != 0)
         return fail(ctx, ROLLART_ERR_INVALID_ARG, "scratch must be a 256-byte aligned device buffer");
-    if (scratch_bytes < L.bytes)
-        return fail(ctx, ROLLART_ERR_WORKSPACE, "scratch of %zu bytes is too small (need %zu)", scratch_bytes, L.bytes);
-    if (L.num_pages > 0x7FFFFFFFLL) return fail(ctx, ROLLART_ERR_UNSUPPORTED, "too many scratch pages");
+    if (L.capacity_pages < 1)
+        return fail(ctx, ROLLART_ERR_WORKSPACE, "scratch of %zu bytes cannot hold a single page", scratch_bytes);
+    if (static_cast<long long>(n_items) * L.pages_per_item > 0x7FFFFFFFLL)
+        return fail(ctx, ROLLART_ERR_UNSUPPORTED, "too many scratch pages");
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return fail(ctx, ROLLART_ERR_CUDA, "cannot select device %d", ctx->device);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
@@ -613,7 +621,7 @@ rollart_status rollart_obs_chunk_attn_fp8(rollart_ctx *ctx, const rollart_kv_poo
     rollart_kv_pool spool = *pool;
     spool.k_pool = base + L.off_k;
     spool.v_pool = base + L.off_v;
-    spool.num_pages = static_cast<int32_t>(L.num_pages);
+    spool.num_pages = static_cast<int32_t>(L.capacity_pages);
     rollart_trajs strajs;
     strajs.page_table = reinterpret_cast<const int32_t *>(base + L.off_table);
     strajs.max_pages_per_traj = L.pages_per_item;
@@ -646,6 +654,8 @@ rollart_status rollart_check(rollart_ctx *ctx, void *stream) {
     const char *w = (hs.where >= 0 && hs.where < 8) ? where[hs.where] : "?";
     if (hs.code == ROLLART_ERR_TIMEOUT)
         return fail(ctx, ROLLART_ERR_TIMEOUT, "%s: a bounded wait ran out (detail %d)", w, hs.detail);
+    if (hs.code == ROLLART_ERR_WORKSPACE)
+        return fail(ctx, ROLLART_ERR_WORKSPACE, "%s: the scratch buffer is smaller than the contexts listed (item %d)", w, hs.detail);
     return fail(ctx, static_cast<rollart_status>(hs.code), "%s: index out of range on the device (detail %d)", w, hs.detail);
 }
 

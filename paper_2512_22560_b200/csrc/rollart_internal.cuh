@@ -124,11 +124,14 @@ cudaError_t launch_chunk_attn(const AttnCall &c, cudaStream_t stream, int64_t *l
 // Observation-chunk attention over fp8 pools: the listed trajectories' contexts are expanded to bf16 into a scratch
 // pool (item i owns pages i * pages_per_item ..), with a scratch page table and scratch lengths behind the two pools.
 struct Fp8ChunkScratch {
-    int pages_per_item;
-    long long num_pages;
-    size_t off_k, off_v, off_table, off_lens, bytes;
+    int pages_per_item;            // row length of the scratch page table
+    long long capacity_pages;      // pages each of the two scratch pools can hold
+    size_t off_k, off_v, off_table, off_lens, off_first, bytes;
 };
-Fp8ChunkScratch fp8_chunk_scratch_layout(int n_items, int num_kv_heads, int page_size, int max_seq_len);
+// bytes for pools of `total_pages` pages (negative or above n_items * pages_per_item: that worst case) plus the small arrays
+size_t fp8_chunk_scratch_bytes(int n_items, int num_kv_heads, int page_size, int max_seq_len, long long total_pages);
+// how a buffer of scratch_bytes is divided; capacity_pages = 0 if it cannot hold even one page
+Fp8ChunkScratch fp8_chunk_scratch_layout(int n_items, int num_kv_heads, int page_size, int max_seq_len, size_t scratch_bytes);
 // lens_override (nullable): per item, expand only that many tokens instead of the trajectory's length
 cudaError_t launch_fp8_pages_to_bf16(const rollart_kv_pool &pool, const rollart_trajs &trajs, const int32_t *traj_ids,
                                      const int32_t *lens_override, int n_items, int max_seq_len,

@@ -26,6 +26,7 @@ EXPORTS = (
     "rollart_decode_attn_fp8", "rollart_kv_append_fp8", "rollart_append_decode_attn_fp8",
     "rollart_kv_gather_fp8", "rollart_kv_append_fp8_codes", "rollart_obs_chunk_attn_fp8",
     "rollart_obs_chunk_fp8_scratch_size", "rollart_group_decode_attn_fp8",
+    "rollart_obs_chunk_fp8_scratch_size_for_pages",
 )
 
 
@@ -104,6 +105,8 @@ def load_library() -> ctypes.CDLL:
                                                 vp, i32, f32, f32, f32, vp, vp, vp, ctypes.c_size_t, vp]
     L.rollart_obs_chunk_fp8_scratch_size.restype = ctypes.c_size_t
     L.rollart_obs_chunk_fp8_scratch_size.argtypes = [i32, i32, i32, i32]
+    L.rollart_obs_chunk_fp8_scratch_size_for_pages.restype = ctypes.c_size_t
+    L.rollart_obs_chunk_fp8_scratch_size_for_pages.argtypes = [i32, i32, i32, i32, i64]
     L.rollart_obs_chunk_attn_fp8.restype = ctypes.c_int
     L.rollart_obs_chunk_attn_fp8.argtypes = [vp, ctypes.POINTER(_KVPool), ctypes.POINTER(_Trajs), vp, vp, i32, i32, i32, vp,
                                              i32, f32, f32, f32, vp, vp, vp, ctypes.c_size_t, vp]
@@ -128,8 +131,14 @@ def group_decode_workspace_size(max_items: int, num_q_heads: int, num_kv_heads: 
     return int(load_library().rollart_group_decode_workspace_size(max_items, num_q_heads, num_kv_heads, max_seq_len))
 
 
-def obs_chunk_fp8_scratch_size(n_items: int, num_kv_heads: int, page_size: int, max_seq_len: int) -> int:
-    return int(load_library().rollart_obs_chunk_fp8_scratch_size(n_items, num_kv_heads, page_size, max_seq_len))
+def obs_chunk_fp8_scratch_size(n_items: int, num_kv_heads: int, page_size: int, max_seq_len: int,
+                               total_pages: Optional[int] = None) -> int:
+    """bytes of scratch for the fp8 chunk / group calls: the worst case (every item at max_seq_len), or, with
+    total_pages, enough for contexts that hold at most that many pages in all"""
+    lib = load_library()
+    if total_pages is None:
+        return int(lib.rollart_obs_chunk_fp8_scratch_size(n_items, num_kv_heads, page_size, max_seq_len))
+    return int(lib.rollart_obs_chunk_fp8_scratch_size_for_pages(n_items, num_kv_heads, page_size, max_seq_len, int(total_pages)))
 
 
 def _ptr(t: Optional[torch.Tensor], dtype=None, device=None, host_ok: bool = False) -> Optional[int]:

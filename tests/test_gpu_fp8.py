@@ -302,9 +302,21 @@ def test_fp8_chunk_last_row_agrees_with_fp8_decode_and_errors_are_reported(cuda_
     need = rollart.obs_chunk_fp8_scratch_size(len(ids), spec.num_kv_heads, spec.page_size, msl)
     scratch = torch.empty(need, dtype=torch.uint8, device=cuda_device)
     qg = q.to(cuda_device)
-    with pytest.raises(rollart.RollartError) as e:
-        ctx.obs_chunk_attn_fp8(dk, dv, table, lens1, qi, qg, spec.sm_scale, KS, VS, msl, out, scratch[: need - 256], traj_ids=tid)
+    with pytest.raises(rollart.RollartError) as e:          # cannot hold a single page: refused on the host
+        ctx.obs_chunk_attn_fp8(dk, dv, table, lens1, qi, qg, spec.sm_scale, KS, VS, msl, out, scratch[:4096], traj_ids=tid)
     assert e.value.status == rollart.ERR_WORKSPACE
+    # exactly the pages the listed contexts hold: enough; one page fewer: the device reports it and skips what does not fit
+    P = spec.page_size
+    pages = int(((batch.seq_lens_after[ids].astype(np.int64) + P - 1) // P).sum())
+    exact = rollart.obs_chunk_fp8_scratch_size(len(ids), spec.num_kv_heads, P, msl, total_pages=pages)
+    assert exact < need
+    out2 = torch.full_like(out, float("nan"))
+    ctx.obs_chunk_attn_fp8(dk, dv, table, lens1, qi, qg, spec.sm_scale, KS, VS, msl, out2, scratch[:exact], traj_ids=tid)
+    ctx.check()
+    assert torch.equal(out2.view(torch.int16), out.view(torch.int16))
+    short = rollart.obs_chunk_fp8_scratch_size(len(ids), spec.num_kv_heads, P, msl, total_pages=pages - 1)
+    ctx.obs_chunk_attn_fp8(dk, dv, table, lens1, qi, qg, spec.sm_scale, KS, VS, msl, out2, scratch[:short], traj_ids=tid)
+    assert ctx.status() == rollart.ERR_WORKSPACE and "scratch" in ctx.last_error()
     for ks, vs in [(0.0, 1.0), (1.0, float("inf")), (float("nan"), 1.0)]:
         with pytest.raises(rollart.RollartError):
             ctx.obs_chunk_attn_fp8(dk, dv, table, lens1, qi, qg, spec.sm_scale, ks, vs, msl, out, scratch, traj_ids=tid)
@@ -340,16 +352,18 @@ def test_fp8_expansion_is_exact_for_every_code(cuda_device):
     ctx.obs_chunk_attn_fp8(torch.from_numpy(k8).to(cuda_device), torch.from_numpy(v8).to(cuda_device), dev_i32(table, cuda_device),
                            dev_i32(lens, cuda_device), dev_i32(np.arange(5), cuda_device), q, 1.0, 1.0, 1.0, msl, out, scratch)
     ctx.check()
+    # worst-case sizing: each pool holds 4 * ppi pages; the items' pages are packed in call order
     ppi = (msl + P - 1) // P
     pool_bytes = 4 * ppi * H * P * D * 2
     sc = scratch.cpu().numpy()
     off_v = (pool_bytes + 255) // 256 * 256
+    first = np.concatenate([[0], np.cumsum(pages)])
     for name, codes, off in (("k", k8, 0), ("v", v8, off_v)):
         got = sc[off: off + pool_bytes].view(np.uint16).reshape(4 * ppi, H, P, D)
         for i in range(4):
             for lp in range(int(pages[i])):
                 want = oracle.fp8_pool_as_bf16_bits(codes[table[i, lp]])
-                g = got[i * ppi + lp]
+                g = got[first[i] + lp]
                 nan_w = (want & 0x7FFF) > 0x7F80
                 nan_g = (g & 0x7FFF) > 0x7F80
                 assert np.array_equal(nan_w, nan_g), (name, i, lp)

@@ -242,7 +242,7 @@ def run_fp8_group_case(spec, seed, group_size, fraction, device, ks=0.03, vs=0.0
     assert torch.allclose(out.float(), out2.float(), atol=4e-3, rtol=2e-2)
     with pytest.raises(rollart.RollartError) as e:
         ctx.group_decode_attn_fp8(dk, dv, table, lens1, dev_i32(indptr, device), dev_i32(shared, device), q, spec.sm_scale, ks,
-                                  vs, msl, out, scratch[: max(256, need - 256)], lse=lse)
+                                  vs, msl, out, scratch[:1024], lse=lse)
     assert e.value.status == rollart.ERR_WORKSPACE
     ctx.close()
     return shared
