@@ -199,6 +199,25 @@ rollart_status rollart_append_decode_attn(rollart_ctx *ctx, const rollart_kv_poo
                                           float *lse, int32_t *seq_lens_out, void *stream);
 
 /*
+ * The fused decode step driven from host buffers: q, k_new and v_new are [host] page-locked buffers (cudaHostAlloc /
+ * cudaHostRegister), layouts as for rollart_append_decode_attn.  The call enqueues their copy into `staging`
+ * (cudaMemcpyAsync on `stream`: one copy if the three buffers follow one another in host memory in the order q, k_new,
+ * v_new, else three) and then the fused step from there.  `out` and `lse` may be device buffers or page-locked host
+ * buffers (see rollart_decode_attn), so a whole step can go host -> device -> host inside this one call; the host may
+ * read the result once the stream has been synchronised and may rewrite its input buffers from then on.
+ *   staging   [device] 256-byte aligned, at least rollart_host_staging_size(n_items, num_q_heads, num_kv_heads)
+ *             bytes; owned by the caller.  Too small: ROLLART_ERR_WORKSPACE, nothing is enqueued.
+ * Pageable host buffers are not refused, but their copy is staged by the driver and the call may block until it is
+ * done.  Everything else as for rollart_append_decode_attn.  Launches one kernel.
+ */
+size_t rollart_host_staging_size(int32_t n_items, int32_t num_q_heads, int32_t num_kv_heads);
+rollart_status rollart_append_decode_attn_host(rollart_ctx *ctx, const rollart_kv_pool *pool, const rollart_trajs *trajs,
+                                               const int32_t *traj_ids, int32_t n_items, int32_t max_seq_len,
+                                               const void *k_new_host, const void *v_new_host, const void *q_host,
+                                               int32_t num_q_heads, float sm_scale, void *out, float *lse,
+                                               int32_t *seq_lens_out, void *staging, size_t staging_bytes, void *stream);
+
+/*
  * fp8 KV pools.  Decoding is bound by reading the whole context once per generated token (Sec. 3.1), so a cache held
  * in 8 bits halves the bytes of a decode step.  The two calls below are rollart_kv_append and rollart_decode_attn for
  * pools whose elements are E4M3 codes (OCP 8-bit floating point: 1 sign, 4 exponent bits with bias 7, 3 mantissa

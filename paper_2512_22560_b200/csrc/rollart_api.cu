@@ -412,6 +412,64 @@ rollart_status rollart_append_decode_attn(rollart_ctx *ctx, const rollart_kv_poo
                               lse, seq_lens_out, stream, false, 1.f, 1.f);
 }
 
+size_t rollart_host_staging_size(int32_t n_items, int32_t num_q_heads, int32_t num_kv_heads) {
+    if (n_items <= 0 || num_q_heads <= 0 || num_kv_heads <= 0) return 0;
+    return (static_cast<size_t>(n_items) * num_q_heads + 2 * static_cast<size_t>(n_items) * num_kv_heads) * kRowBytes;
+}
+
+rollart_status rollart_append_decode_attn_host(rollart_ctx *ctx, const rollart_kv_pool *pool, const rollart_trajs *trajs,
+                                               const int32_t *traj_ids, int32_t n_items, int32_t max_seq_len,
+                                               const void *k_new_host, const void *v_new_host, const void *q_host,
+                                               int32_t num_q_heads, float sm_scale, void *out, float *lse,
+                                               int32_t *seq_lens_out, void *staging, size_t staging_bytes, void *stream) {
+    if (!ctx) return ROLLART_ERR_INVALID_ARG;
+    rollart_status st = attn_common(ctx, pool, trajs, n_items, n_items, max_seq_len, q_host, num_q_heads, out);
+    if (st != ROLLART_OK) return st;
+    if (n_items == 0) return ROLLART_OK;
+    if (!k_new_host || !v_new_host) return fail(ctx, ROLLART_ERR_INVALID_ARG, "k_new or v_new NULL");
+    if (!aligned16(k_new_host) || !aligned16(v_new_host)) return fail(ctx, ROLLART_ERR_INVALID_ARG, "k_new/v_new must be 16-byte aligned");
+    const size_t need = rollart_host_staging_size(n_items, num_q_heads, pool->num_kv_heads);
+    if (!staging || (reinterpret_cast<uintptr_t>(staging) & 255u) != 0)
+        return fail(ctx, ROLLART_ERR_INVALID_ARG, "staging must be a 256-byte aligned device buffer");
+    if (staging_bytes < need) return fail(ctx, ROLLART_ERR_WORKSPACE, "staging of %zu bytes is too small (need %zu)", staging_bytes, need);
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return fail(ctx, ROLLART_ERR_CUDA, "cannot select device %d", ctx->device);
+    // what the step itself would refuse is refused before the copy is enqueued
+    if (seq_lens_out) {
+        const char *a = reinterpret_cast<const char *>(trajs->seq_lens);
+        const char *b = reinterpret_cast<const char *>(seq_lens_out);
+        size_t bytes = sizeof(int32_t) * static_cast<size_t>(trajs->num_traj);
+        if (a < b + bytes && b < a + bytes) return fail(ctx, ROLLART_ERR_INVALID_ARG, "seq_lens_out overlaps seq_lens");
+    }
+    {
+        const size_t ws = decode_workspace_bytes(n_items, num_q_heads, pool->num_kv_heads, clamp_bound(pool, trajs, max_seq_len),
+                                                 ctx->sm_count);
+        if (!ctx->workspace || ws > ctx->workspace_bytes)
+            return fail(ctx, ROLLART_ERR_WORKSPACE, "workspace of %zu bytes is too small (need %zu)", ctx->workspace_bytes, ws);
+    }
+    const size_t q_bytes = static_cast<size_t>(n_items) * num_q_heads * kRowBytes;        // multiples of 256
+    const size_t kv_bytes = static_cast<size_t>(n_items) * pool->num_kv_heads * kRowBytes;
+    char *sb = static_cast<char *>(staging);
+    void *sq = sb, *sk = sb + q_bytes, *sv = sb + q_bytes + kv_bytes;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const char *hq = static_cast<const char *>(q_host);
+    cudaError_t e = cudaErrorInvalidValue;
+    if (hq + q_bytes == k_new_host && hq + q_bytes + kv_bytes == v_new_host) {
+        // the three buffers follow one another in host memory (q, k_new, v_new): one copy moves them all, provided
+        // they are parts of one page-locked allocation (a copy across two allocations is refused up front)
+        e = cudaMemcpyAsync(sq, q_host, q_bytes + 2 * kv_bytes, cudaMemcpyHostToDevice, s);
+        if (e != cudaSuccess) cudaGetLastError();
+    }
+    if (e != cudaSuccess) {
+        e = cudaMemcpyAsync(sq, q_host, q_bytes, cudaMemcpyHostToDevice, s);
+        if (e == cudaSuccess) e = cudaMemcpyAsync(sk, k_new_host, kv_bytes, cudaMemcpyHostToDevice, s);
+        if (e == cudaSuccess) e = cudaMemcpyAsync(sv, v_new_host, kv_bytes, cudaMemcpyHostToDevice, s);
+    }
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "host -> device copy");
+    return append_decode_impl(ctx, pool, trajs, traj_ids, n_items, max_seq_len, sk, sv, sq, num_q_heads, sm_scale, out, lse,
+                              seq_lens_out, stream, false, 1.f, 1.f);
+}
+
 rollart_status rollart_append_decode_attn_fp8(rollart_ctx *ctx, const rollart_kv_pool *pool, const rollart_trajs *trajs,
                                               const int32_t *traj_ids, int32_t n_items, int32_t max_seq_len,
                                               const void *k_new, const void *v_new, const void *q, int32_t num_q_heads,

@@ -26,7 +26,7 @@ EXPORTS = (
     "rollart_decode_attn_fp8", "rollart_kv_append_fp8", "rollart_append_decode_attn_fp8",
     "rollart_kv_gather_fp8", "rollart_kv_append_fp8_codes", "rollart_obs_chunk_attn_fp8",
     "rollart_obs_chunk_fp8_scratch_size", "rollart_group_decode_attn_fp8",
-    "rollart_obs_chunk_fp8_scratch_size_for_pages",
+    "rollart_obs_chunk_fp8_scratch_size_for_pages", "rollart_append_decode_attn_host", "rollart_host_staging_size",
 )
 
 
@@ -92,6 +92,11 @@ def load_library() -> ctypes.CDLL:
     L.rollart_append_decode_attn.restype = ctypes.c_int
     L.rollart_append_decode_attn.argtypes = [vp, ctypes.POINTER(_KVPool), ctypes.POINTER(_Trajs), vp, i32, i32, vp, vp, vp, i32,
                                              f32, vp, vp, vp, vp]
+    L.rollart_host_staging_size.restype = ctypes.c_size_t
+    L.rollart_host_staging_size.argtypes = [i32, i32, i32]
+    L.rollart_append_decode_attn_host.restype = ctypes.c_int
+    L.rollart_append_decode_attn_host.argtypes = [vp, ctypes.POINTER(_KVPool), ctypes.POINTER(_Trajs), vp, i32, i32, vp, vp, vp, i32,
+                                                  f32, vp, vp, vp, vp, ctypes.c_size_t, vp]
     L.rollart_group_decode_workspace_size.restype = ctypes.c_size_t
     L.rollart_group_decode_workspace_size.argtypes = [i32, i32, i32, i32]
     L.rollart_group_decode_attn.restype = ctypes.c_int
@@ -131,6 +136,18 @@ def group_decode_workspace_size(max_items: int, num_q_heads: int, num_kv_heads: 
     return int(load_library().rollart_group_decode_workspace_size(max_items, num_q_heads, num_kv_heads, max_seq_len))
 
 
+def host_staging_size(n_items: int, num_q_heads: int, num_kv_heads: int) -> int:
+    return int(load_library().rollart_host_staging_size(n_items, num_q_heads, num_kv_heads))
+
+
+def _host_ptr(t: torch.Tensor, dtype) -> int:
+    # pinned-ness is the caller's business here (Tensor.is_pinned costs several microseconds a call, and a pageable
+    # buffer is not wrong, only slow: its copy is staged by the driver)
+    if t.is_cuda or not t.is_contiguous() or t.dtype != dtype:
+        raise ValueError(f"expected a contiguous host tensor of dtype {dtype}")
+    return t.data_ptr()
+
+
 def obs_chunk_fp8_scratch_size(n_items: int, num_kv_heads: int, page_size: int, max_seq_len: int,
                                total_pages: Optional[int] = None) -> int:
     """bytes of scratch for the fp8 chunk / group calls: the worst case (every item at max_seq_len), or, with
@@ -142,22 +159,23 @@ def obs_chunk_fp8_scratch_size(n_items: int, num_kv_heads: int, page_size: int, 
 
 
 def _ptr(t: Optional[torch.Tensor], dtype=None, device=None, host_ok: bool = False) -> Optional[int]:
+    """Address of a contiguous CUDA tensor (of the given dtype, on the given device).  With host_ok a host tensor is
+    accepted too, provided it is pinned: a result buffer may be page-locked host memory, mapped into the device's
+    address space under unified addressing, and the kernel then writes the result straight to the host (a pageable
+    buffer has no device address and is refused here)."""
     if t is None:
         return None
-    if host_ok and not t.is_cuda:
-        # a result buffer may be page-locked host memory (mapped into the device's address space under unified
-        # addressing): the kernel then writes the result straight to the host
-        if not t.is_pinned() or not t.is_contiguous():
-            raise ValueError("a host result buffer must be a contiguous pinned tensor")
-        if dtype is not None and t.dtype != dtype:
-            raise ValueError(f"expected dtype {dtype}, got {t.dtype}")
-        return t.data_ptr()
-    if not t.is_cuda or not t.is_contiguous():
-        raise ValueError("expected a contiguous CUDA tensor")
+    if not t.is_contiguous():
+        raise ValueError("expected a contiguous tensor")
     if dtype is not None and t.dtype != dtype:
         raise ValueError(f"expected dtype {dtype}, got {t.dtype}")
-    if device is not None and t.device.index != device:
-        raise ValueError(f"tensor on cuda:{t.device.index}, context on cuda:{device}")
+    if t.is_cuda:
+        if device is not None and t.get_device() != device:
+            raise ValueError(f"tensor on cuda:{t.get_device()}, context on cuda:{device}")
+    elif not host_ok:
+        raise ValueError("expected a contiguous CUDA tensor")
+    elif not t.is_pinned():
+        raise ValueError("a host result buffer must be a pinned tensor")
     return t.data_ptr()
 
 
@@ -197,6 +215,22 @@ def decode_attn_noalloc(k_pool, v_pool, page_table, seq_lens, q, sm_scale, max_s
         _ptr(device_status, torch.int32, dev), sptr, buf, len(buf))
     if st != OK:
         raise RollartError(st, buf.value.decode())
+
+
+class BoundCall:
+    """A library call with its arguments marshalled once, for a loop that repeats it on the same buffers (a decode
+    loop rewrites the contents of its buffers, not their addresses): calling the object issues the call again at the
+    cost of the foreign call alone.  Holds references to the tensors so that the addresses stay valid."""
+
+    __slots__ = ("_ctx", "_fn", "_args", "_keep")
+
+    def __init__(self, ctx, fn, args, keep):
+        self._ctx, self._fn, self._args, self._keep = ctx, fn, args, keep
+
+    def __call__(self) -> None:
+        st = self._fn(*self._args)
+        if st != OK:
+            self._ctx._raise(st)
 
 
 class Context:
@@ -441,6 +475,47 @@ class Context:
             _ptr(lse, torch.float32, self.device, True), _ptr(seq_lens_out, torch.int32, self.device), self._stream(stream))
         if st != OK:
             self._raise(st)
+
+    def _append_decode_attn_host_args(self, k_pool, v_pool, page_table, seq_lens, k_new, v_new, q, sm_scale, max_seq_len, out,
+                                      staging, lse, traj_ids, seq_lens_out, stream):
+        pool = self._pool(k_pool, v_pool)
+        trajs = self._trajs(page_table, seq_lens)
+        if q.dim() != 3 or q.shape != out.shape:
+            raise ValueError("q and out must be [n_items][num_q_heads][head_dim]")
+        n_items, hq, _ = q.shape
+        if k_new.shape != v_new.shape or tuple(k_new.shape) != (n_items, pool.num_kv_heads, pool.head_dim):
+            raise ValueError("k_new/v_new must be [n_items][num_kv_heads][head_dim]")
+        if traj_ids is not None and traj_ids.shape[0] != n_items:
+            raise ValueError("traj_ids must have one entry per item")
+        if lse is not None and tuple(lse.shape) != (n_items, hq):
+            raise ValueError("lse must be [n_items][num_q_heads]")
+        if seq_lens_out is not None and seq_lens_out.shape != seq_lens.shape:
+            raise ValueError("seq_lens_out must have the shape of seq_lens")
+        args = (self._h, ctypes.byref(pool), ctypes.byref(trajs), _ptr(traj_ids, torch.int32, self.device), n_items,
+                int(max_seq_len), _host_ptr(k_new, torch.bfloat16), _host_ptr(v_new, torch.bfloat16), _host_ptr(q, torch.bfloat16),
+                hq, float(sm_scale), _ptr(out, torch.bfloat16, self.device, True), _ptr(lse, torch.float32, self.device, True),
+                _ptr(seq_lens_out, torch.int32, self.device), _ptr(staging, torch.uint8, self.device), staging.numel(),
+                self._stream(stream))
+        keep = (pool, trajs, k_pool, v_pool, page_table, seq_lens, k_new, v_new, q, out, staging, lse, traj_ids, seq_lens_out)
+        return args, keep
+
+    def append_decode_attn_host(self, k_pool, v_pool, page_table, seq_lens, k_new, v_new, q, sm_scale, max_seq_len, out,
+                                staging, lse=None, traj_ids=None, seq_lens_out=None, stream=None) -> None:
+        """append_decode_attn with q / k_new / v_new in pinned host tensors (the call enqueues their copy);
+        `staging` is a uint8 CUDA tensor of at least host_staging_size(n_items, num_q_heads, num_kv_heads) bytes"""
+        args, _ = self._append_decode_attn_host_args(k_pool, v_pool, page_table, seq_lens, k_new, v_new, q, sm_scale, max_seq_len,
+                                                     out, staging, lse, traj_ids, seq_lens_out, stream)
+        st = self._lib.rollart_append_decode_attn_host(*args)
+        if st != OK:
+            self._raise(st)
+
+    def bind_append_decode_attn_host(self, k_pool, v_pool, page_table, seq_lens, k_new, v_new, q, sm_scale, max_seq_len, out,
+                                     staging, lse=None, traj_ids=None, seq_lens_out=None, stream=None) -> BoundCall:
+        """The same call with its arguments marshalled once: the returned object repeats it on the same buffers and the
+        same stream (the one current now, unless `stream` is given)."""
+        args, keep = self._append_decode_attn_host_args(k_pool, v_pool, page_table, seq_lens, k_new, v_new, q, sm_scale,
+                                                        max_seq_len, out, staging, lse, traj_ids, seq_lens_out, stream)
+        return BoundCall(self, self._lib.rollart_append_decode_attn_host, args, keep)
 
     def group_decode_attn(self, k_pool, v_pool, page_table, seq_lens, group_indptr, shared_lens, q, sm_scale, max_seq_len,
                           out, lse=None, traj_ids=None, stream=None) -> None:

@@ -302,3 +302,65 @@ def test_decode_steps_replayed_from_a_cuda_graph(cuda_device):
                                   spec.sm_scale, traj_ids=ids)
     assert_attn_close(outs_g[-1], ref_o, "graph replay, last step")
     ctx.close()
+
+
+@pytest.mark.parametrize("i,T,div", [(0, 4, 1), (1, 16, 4), (3, 4, 16)])
+def test_fused_step_driven_from_host_buffers(cuda_device, i, T, div):
+    """q / k_new / v_new in pinned host memory, copied in by the call itself, result written to pinned host
+    memory: pools, lengths and outputs bit for bit as with device buffers; a second step after the host has rewritten
+    its buffers sees the new values."""
+    batch = W.make_batch(W.shrink(W.CONFIGS[i], T, div, 16), seed=900 + i)
+    spec = batch.spec
+    ids, rows = batch.decode_ids, batch.decode_rows()
+    n = len(ids)
+    msl = int(batch.seq_lens_after.max()) + 1
+    table = np.concatenate([batch.page_table, np.full((spec.num_traj, 1), -1, np.int32)], axis=1)
+    P = spec.page_size
+    used = set(int(p) for t in range(spec.num_traj) for p in table[t, : (int(batch.seq_lens_after[t]) + P - 1) // P])
+    spare = [p for p in range(batch.num_pages) if p not in used]
+    for t in ids:                                                # room for a second token
+        have, want = (int(batch.seq_lens_after[t]) + P - 1) // P, (int(batch.seq_lens_before[t]) + 2 + P - 1) // P
+        for lp in range(have, want):
+            table[t, lp] = spare.pop()
+    ctx = make_ctx(spec, n, msl)
+    d_table, tid = dev_i32(table, cuda_device), dev_i32(ids, cuda_device)
+    ridx = torch.from_numpy(rows)
+    steps = [(batch.q_new[ridx].contiguous(), batch.k_new[ridx].contiguous(), batch.v_new[ridx].contiguous())]
+    steps.append(tuple((x.float() * -0.5 + 0.25).to(torch.bfloat16) for x in steps[0]))
+    staging = torch.empty(rollart.host_staging_size(n, spec.num_q_heads, spec.num_kv_heads), dtype=torch.uint8, device=cuda_device)
+    res = {}
+    for mode in ("device", "host"):
+        kp, vp = batch.k_pool.clone().to(cuda_device), batch.v_pool.clone().to(cuda_device)
+        la, lb = dev_i32(batch.seq_lens_before, cuda_device), dev_i32(batch.seq_lens_before, cuda_device)
+        hq_, hk_, hv_ = (torch.empty_like(x).pin_memory() for x in steps[0])
+        outs = []
+        for q, kn, vn in steps:
+            if mode == "device":
+                out = torch.full_like(q, float("nan"), device=cuda_device)
+                ctx.append_decode_attn(kp, vp, d_table, la, kn.to(cuda_device), vn.to(cuda_device), q.to(cuda_device),
+                                       spec.sm_scale, msl, out, traj_ids=tid, seq_lens_out=lb)
+            else:
+                hq_.copy_(q); hk_.copy_(kn); hv_.copy_(vn)       # the host rewrites its buffers between the steps
+                out = torch.full(tuple(q.shape), float("nan"), dtype=torch.bfloat16).pin_memory()
+                ctx.append_decode_attn_host(kp, vp, d_table, la, hk_, hv_, hq_, spec.sm_scale, msl, out, staging, traj_ids=tid,
+                                            seq_lens_out=lb)
+            la.copy_(lb)
+            ctx.check()
+            outs.append(out.cpu().clone())
+        res[mode] = (kp, vp, la.clone(), outs)
+    a, b = res["device"], res["host"]
+    assert torch.equal(a[0].view(torch.int16), b[0].view(torch.int16)) and torch.equal(a[1].view(torch.int16), b[1].view(torch.int16))
+    assert torch.equal(a[2], b[2])
+    for x, y in zip(a[3], b[3]):
+        assert torch.equal(x.view(torch.int16), y.view(torch.int16))
+    ref_o, _ = oracle.decode_attn(W.bf16_to_u16(b[0]), W.bf16_to_u16(b[1]), table, b[2].cpu().numpy(), W.bf16_to_u16(steps[1][0]),
+                                  spec.sm_scale, traj_ids=ids)
+    assert_attn_close(b[3][1], ref_o, spec.name + " host step")
+    with pytest.raises(ValueError):                              # device tensors are not host buffers
+        ctx.append_decode_attn_host(b[0], b[1], d_table, b[2], hk_.to(cuda_device), hv_, hq_, spec.sm_scale, msl,
+                                    torch.empty(tuple(hq_.shape), dtype=torch.bfloat16).pin_memory(), staging, traj_ids=tid)
+    with pytest.raises(rollart.RollartError) as e:
+        ctx.append_decode_attn_host(b[0], b[1], d_table, b[2], hk_, hv_, hq_, spec.sm_scale, msl,
+                                    torch.empty(tuple(hq_.shape), dtype=torch.bfloat16).pin_memory(), staging[:256], traj_ids=tid)
+    assert e.value.status == rollart.ERR_WORKSPACE
+    ctx.close()
