@@ -120,6 +120,8 @@ cudaError_t launch_decode_attn(const AttnCall &c, cudaStream_t stream, int64_t *
 // zeroes the bookkeeping at the head of the workspace after a device-side error
 cudaError_t decode_reset_workspace(void *workspace, size_t bytes, cudaStream_t stream);
 cudaError_t launch_chunk_attn(const AttnCall &c, cudaStream_t stream, int64_t *launches, bool *too_small);
+// the causal chunk call on CTA pairs (no shared-prefix mode, bf16 output): what launch_chunk_attn runs for such calls
+cudaError_t launch_chunk_attn_pair(const AttnCall &c, cudaStream_t stream, int64_t *launches);
 
 // Observation-chunk attention over fp8 pools: the listed trajectories' contexts are expanded to bf16 into a scratch
 // pool (item i owns pages i * pages_per_item ..), with a scratch page table and scratch lengths behind the two pools.
