@@ -607,11 +607,9 @@ chunk_attn_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constan
 
 cudaError_t launch_chunk_attn(const AttnCall &c, cudaStream_t stream, int64_t *launches, bool *too_small) {
     (void)too_small;
-    // plain causal chunks can run on CTA pairs (chunk_attn_pair.cu); this kernel keeps the shared-prefix mode of the group
-    // decode call.  The pair kernel passes every parity test but is the slower one so far, so it is not the default yet.
-    constexpr bool kCausalOnPairs = false;
-    if (kCausalOnPairs && c.shared_lens == nullptr && c.out_f32 == nullptr && c.item_order == nullptr)
-        return launch_chunk_attn_pair(c, stream, launches);
+    // plain causal chunks run on CTA pairs (chunk_attn_pair.cu); this kernel keeps the shared-prefix mode of the group
+    // decode call (one M-tile per group: a pair would idle its second CTA, and that pass is bound by memory)
+    if (c.shared_lens == nullptr && c.out_f32 == nullptr && c.item_order == nullptr) return launch_chunk_attn_pair(c, stream, launches);
     const int hkv = c.pool.num_kv_heads, g = c.num_q_heads / hkv, tpt = kRows / g;
     cudaError_t e = cudaFuncSetAttribute(chunk_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (e != cudaSuccess) return e;

@@ -9,23 +9,28 @@
 //                  memory: per MMA step an SM reads 4 KB of Q and 2 KB of K for 64 cycles of math, where one CTA
 //                  alone with 64-key tiles read 6 KB per 32 cycles and was held by its shared-memory port.  Two S
 //                  buffers, so S(j+1) is computed while the softmax of tile j runs.
-//   softmax        two warpgroups per CTA, one thread per (row, half of the 128 columns): tcgen05.ld its 64 scores,
-//                  P = exp2(scale * s - m) as packed bf16 stored back over the start of its half of the S buffer, row
-//                  sum.  After the first tile m is not recomputed per tile: the exponentials are taken against the
-//                  row's current reference max, and only a row sum that explodes (or a masked tile) sends the tile
-//                  down the careful path (row max over both halves, new reference, O rescaled in tensor memory).  The
-//                  two threads of a row agree on that through shared memory and a 64-thread named barrier per tile.
-//                  One pair of exponentials in kPolyOneIn is evaluated on the FMA pipe.
-//   O += P V       one MMA of M 256 x N 128 x K 128 with the A operand (P) in tensor memory; each CTA supplies HALF of
-//                  V's dims (64) for all 128 keys, straight from the [key][dim] page layout (MN-major B).
+//   softmax        two warpgroups per CTA, each with its own KEY STREAM: warpgroup w takes keys 64 w .. 64 w + 63 of
+//                  every tile, one thread per query row: tcgen05.ld its 64 scores, P = exp2(scale * s - m) as packed
+//                  bf16 stored back over the start of its half of the S buffer, row sum.  A stream has its own
+//                  reference max, row sum and O accumulator, so the two warps that share a row (they sit on the same
+//                  SM sub-partition: tensor-memory lanes are tied to warp % 4) never exchange anything while the keys
+//                  stream by; the two streams are merged once, at the end.  After a stream's first tile m is not
+//                  recomputed per tile: the exponentials are taken against the current reference max, and only a row
+//                  sum that explodes (or a masked tile) sends the tile down the careful path (row max, new reference,
+//                  the stream's O rescaled in tensor memory).  One pair of exponentials in kPolyOneIn is evaluated
+//                  on the FMA pipe.
+//   O_w += P_w V   per stream an MMA of M 256 x N 128 x K 64 with the A operand (P) in tensor memory; each CTA supplies
+//                  HALF of V's dims (64) for the keys, straight from the [key][dim] page layout (MN-major B).
 //
 // Roles per CTA (12 warps): warp 0 copies Q and the CTA's half of every K tile, warp 3 its half of every V tile (TMA,
 // one box per page; page ids fetched 32 at a time, a batch ahead); warp 2 waits for each landed tile, zeroes the V
 // rows of dead keys in the last tile and tells the leader that this CTA's half is ready; warp 1 of the leader (the
-// even CTA) issues every MMA; warps 4-7 and 8-11 are the softmax warpgroups, which also write the result.
+// even CTA) issues every MMA (the whole warp walks the loop so that descriptors are warp-uniform values; one elected
+// lane issues); warps 4-7 and 8-11 are the softmax warpgroups, which also write the result.
 // Completion of MMAs reaches both CTAs through tcgen05.commit to the barriers of both; all other cross-CTA signals are
 // mbarrier arrivals at the leader.  No load is multicast: each CTA copies what it needs itself.
-// A CTA uses ~194 KB of shared memory (Q 32 KB, 10 K/V stages of 16 KB) and 384 of its 512 tensor-memory columns.
+// A CTA uses ~194 KB of shared memory (Q 32 KB, 10 K/V stages of 16 KB) and all 512 tensor-memory columns (two S
+// buffers of 128, two O accumulators of 128).
 // Every wait is a bounded mbarrier poll; a pair in which any wait ran out tells both CTAs and runs to its end.
 #include <cuda.h>
 
@@ -46,6 +51,7 @@ constexpr int kOwnKeys = kKeys / 2;        // keys of a K tile held by one CTA
 constexpr int kOwnDims = kHeadDim / 2;     // dims of a V tile held by one CTA
 constexpr int kStages = 10;                // ring of stages; K(j) and V(j) take alternate slots
 constexpr int kThreads = 384;
+constexpr int kCols = kKeys / 2;           // S columns (keys) of a tile per softmax thread: one key stream per warpgroup
 constexpr int kMaxItems = kChunkItemsPerLaunch;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
@@ -61,21 +67,19 @@ static_assert(kStageBytes == kKeys * kOwnDims * 2, "a V half tile fills a stage 
 constexpr int kOffQ = 0;
 constexpr int kOffKV = kOffQ + kTileQ;
 constexpr int kOffBars = kOffKV + kStages * kStageBytes;
-constexpr int kNumBars = 2 + 3 * kStages + 6;   // q_full, q_ready | full, empty, ready per stage | s_full, p_full, o_done per S buffer
+constexpr int kNumBars = 2 + 3 * kStages + 10;  // q_full, q_ready | full, empty, ready per stage | s_full per S buffer | p_full, o_done per key stream and S buffer
 constexpr int kOffTmemSlot = kOffBars + kNumBars * 8;
 constexpr int kOffAbort = kOffTmemSlot + 8;
 constexpr int kOffFatal = kOffAbort + 8;                   // the leader's reading of the status word's fatal flag
-constexpr int kOffXFlag = kOffFatal + 8;                   // [tile parity][row quarter][warpgroup]
-constexpr int kOffXMax = kOffXFlag + 2 * 4 * 2 * 4;        // [tile parity][warpgroup][row]
-constexpr int kOffXSum = kOffXMax + 2 * 2 * kRows * 4;     // [warpgroup][row]
-constexpr int kSmemUsed = kOffXSum + 2 * kRows * 4;
+constexpr int kOffXMl = kOffFatal + 8;                     // [stream][row]: (m, l) of each key stream, for the final merge
+constexpr int kSmemUsed = kOffXMl + 2 * kRows * 8;
 constexpr int kSmemBytes = kSmemUsed + 1024;               // + slack for the 1024-byte alignment
 static_assert(kSmemBytes <= 227 * 1024, "one block must fit an SM");
 static_assert((kMaxItems + 1) * 4 <= kStages * kStageBytes, "the tile prefix is staged in the KV stages");
 static_assert(kStages % 2 == 0, "K tiles and V tiles alternate in the ring");
 
-constexpr int kTmemCols = 512;             // S buffer b at columns b * 128; O at 256; P(keys 64 w ..) over columns 64 w .. 64 w + 31 of its S buffer
-constexpr int kTmemO = 256;
+constexpr int kTmemCols = 512;             // S buffer b at columns b * 128; stream w's P over the first 32 columns of its half (64 w ..) of the S buffer
+constexpr int kTmemO = 256;                // O of stream w at 256 + 128 w
 
 struct PairParams {
     const int32_t *page_table;
@@ -96,10 +100,10 @@ struct PairParams {
 __device__ __forceinline__ void pair_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, uint32_t peer_abort,
                                           DeviceStatus *status, int where) {
     constexpr long long kWaitCycles = 2000000000LL;   // about a second
-    if (mbar_try_wait_cluster(bar, parity)) return;
+    if (mbar_try_wait(bar, parity)) return;
     const long long t0 = clock64();
     for (uint32_t it = 1;; ++it) {
-        if (mbar_try_wait_cluster(bar, parity)) return;
+        if (mbar_try_wait(bar, parity)) return;
         if ((it & 255u) == 0u) {
             if (*abort_flag) return;
             if (clock64() - t0 > kWaitCycles) break;
@@ -138,8 +142,8 @@ chunk_attn_pair_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_co
     auto bar_empty = [&](int s) { return bars + 8u * (2 + kStages + s); };       // the MMAs that read the stage are done
     auto bar_ready = [&](int s) { return bars + 8u * (2 + 2 * kStages + s); };   // leader: both CTAs' halves are in place
     auto bar_sfull = [&](int b) { return bars + 8u * (2 + 3 * kStages + b); };
-    auto bar_pfull = [&](int b) { return bars + 8u * (2 + 3 * kStages + 2 + b); };   // leader: P of both CTAs is stored
-    auto bar_odone = [&](int b) { return bars + 8u * (2 + 3 * kStages + 4 + b); };
+    auto bar_pfull = [&](int w, int b) { return bars + 8u * (2 + 3 * kStages + 2 + 2 * w + b); };   // leader: stream w's P of both CTAs is stored
+    auto bar_odone = [&](int w, int b) { return bars + 8u * (2 + 3 * kStages + 6 + 2 * w + b); };
     const uint32_t peer_abort = map_to_cta(smem_u32(smem + kOffAbort), rank ^ 1u);
 
     // ---- which (item, kv head, pair of M-tiles) is this cluster?  pairs per item -> prefix -> search ----
@@ -216,7 +220,10 @@ chunk_attn_pair_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_co
         mbar_init(bar_qfull, 1);
         mbar_init(bar_qready, 2);
         for (int s = 0; s < kStages; ++s) { mbar_init(bar_full(s), 1); mbar_init(bar_empty(s), 1); mbar_init(bar_ready(s), 2); }
-        for (int b = 0; b < 2; ++b) { mbar_init(bar_sfull(b), 1); mbar_init(bar_odone(b), 1); mbar_init(bar_pfull(b), 16); }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(bar_sfull(b), 1);
+            for (int w = 0; w < 2; ++w) { mbar_init(bar_odone(w, b), 1); mbar_init(bar_pfull(w, b), 8); }   // 4 warps x 2 CTAs
+        }
         *s_abort = 0;
         // an earlier block ran out of patience: the leader's reading of the flag decides for the pair
         s_fatal[0] = *reinterpret_cast<volatile int *>(&prm.status->fatal) != 0 ? 1 : 0;
@@ -326,9 +333,14 @@ chunk_attn_pair_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_co
         // One thread issues QK(0) | QK(j+1) PV(j) | ...: S of the next key tile is ready before the softmax of this one
         // ends.  MMAs run in issue order, which is what protects the reuse of an S buffer (it holds P(j-1) until
         // PV(j-1), issued before QK(j+1), has read it).
-        if (rank == 0 && lane == 0) {
+        // The whole warp walks the loop (waits, descriptor arithmetic: warp-uniform values, which the compiler can keep
+        // in uniform registers, where the MMA instruction takes its operands from); only the MMA and commit
+        // instructions themselves are predicated on one elected lane.
+        if (rank == 0) {
             constexpr uint32_t kIdescQK = idesc(2 * kRows, kKeys, false);
             constexpr uint32_t kIdescPV = idesc(2 * kRows, kHeadDim, true);
+            const bool elected = elect_one();
+            const uint32_t tm = __shfl_sync(0xffffffffu, tmem, 0);
             const uint32_t kv_addr = smem_u32(smem + kOffKV);
             const uint64_t q_desc = smem_desc(smem_u32(smem + kOffQ), 16);
             auto ready_wait = [&](int r, int where) {
@@ -338,51 +350,63 @@ chunk_attn_pair_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_co
                 ready_wait(2 * j, 8);                       // K(j), both halves
                 tc_fence_after();
                 const uint64_t k_desc = smem_desc(kv_addr + ((2 * j) % kStages) * kStageBytes, 16);
+                const uint32_t s_tm = tm + (j & 1) * kKeys;
 #pragma unroll
                 for (int ks = 0; ks < kHeadDim / 16; ++ks) {   // 16 dims per step; the second 64 dims live in the other half
                     const uint64_t qoff = static_cast<uint64_t>(((ks >> 2) * kHalfQ + (ks & 3) * 32) >> 4);
                     const uint64_t koff = static_cast<uint64_t>(((ks >> 2) * kHalfK + (ks & 3) * 32) >> 4);
-                    umma_pair_bf16(tmem + (j & 1) * kKeys, q_desc + qoff, k_desc + koff, kIdescQK, ks > 0 ? 1u : 0u);
+                    if (elected) umma_pair_bf16(s_tm, q_desc + qoff, k_desc + koff, kIdescQK, ks > 0 ? 1u : 0u);
                 }
-                umma_pair_commit(bar_sfull(j & 1));
-                umma_pair_commit(bar_empty((2 * j) % kStages));
+                if (elected) {
+                    umma_pair_commit(bar_sfull(j & 1));
+                    umma_pair_commit(bar_empty((2 * j) % kStages));
+                }
+                __syncwarp();
             };
             pair_wait(bar_qready, 0, s_abort, peer_abort, prm.status, 9);
             issue_qk(0);
             for (int j = 0; j < nmax; ++j) {
                 if (j + 1 < nmax) issue_qk(j + 1);
                 ready_wait(2 * j + 1, 10);                  // V(j), both halves
-                pair_wait(bar_pfull(j & 1), (j >> 1) & 1, s_abort, peer_abort, prm.status, 11);
-                tc_fence_after();
                 // V half tile is [key][128 B]: the 16 keys of step ks start 2 KB further on; 8-key groups are 1 KB apart
                 const uint64_t v_desc = smem_desc(kv_addr + ((2 * j + 1) % kStages) * kStageBytes, 1024);
-                const uint32_t p_tmem = tmem + (j & 1) * kKeys;
+                const uint32_t p_tm = tm + (j & 1) * kKeys;
+                const uint32_t acc0 = j > 0 ? 1u : 0u;
 #pragma unroll
-                for (int ks = 0; ks < kKeys / 16; ++ks)     // 16 keys per step: 8 packed columns of P's row
-                    umma_pair_bf16_ts(tmem + kTmemO, p_tmem + (ks >> 2) * 64 + (ks & 3) * 8,
-                                      v_desc + static_cast<uint64_t>((ks * 16 * 128) >> 4), kIdescPV, (ks > 0 || j > 0) ? 1u : 0u);
-                umma_pair_commit(bar_empty((2 * j + 1) % kStages));
-                umma_pair_commit(bar_odone(j & 1));
+                for (int w = 0; w < 2; ++w) {               // the two key streams: keys 64 w .. 64 w + 63 of the tile into O_w
+                    pair_wait(bar_pfull(w, j & 1), (j >> 1) & 1, s_abort, peer_abort, prm.status, 11);
+                    tc_fence_after();
+#pragma unroll
+                    for (int ks = 0; ks < kCols / 16; ++ks)     // 16 keys per step: 8 packed columns of P's row
+                        if (elected)
+                            umma_pair_bf16_ts(tm + kTmemO + w * kHeadDim, p_tm + w * kCols + ks * 8,
+                                              v_desc + static_cast<uint64_t>(((w * kCols + ks * 16) * 128) >> 4), kIdescPV,
+                                              ks > 0 ? 1u : acc0);
+                    if (elected) {
+                        if (w == 1) umma_pair_commit(bar_empty((2 * j + 1) % kStages));
+                        umma_pair_commit(bar_odone(w, j & 1));
+                    }
+                    __syncwarp();
+                }
             }
         }
         __syncwarp();
     } else {
         // =============================== softmax warpgroups ===============================
-        const int wg = (warp - 4) >> 2;                       // which 64 of the 128 columns of a tile
+        // Warpgroup w owns key stream w: keys 64 w .. 64 w + 63 of every tile, with its own reference max, row sum and
+        // O accumulator, so the two warps that share a row never have to agree on anything while the keys stream by;
+        // the two streams are merged once, at the end.
+        const int wg = (warp - 4) >> 2;
         const int quarter = warp & 3;                         // tensor-memory lanes 32 * quarter .. + 31 belong to this warp
         const int row = quarter * 32 + lane;
-        const int bar_id = 1 + quarter;                       // the two warps that share these rows meet here
         const uint32_t lane_addr = tmem + (static_cast<uint32_t>(quarter * 32) << 16);
-        const uint32_t s_addr = lane_addr + wg * 64, o_addr = lane_addr + kTmemO + wg * 64;
+        const uint32_t s_addr = lane_addr + wg * kCols, o_addr = lane_addr + kTmemO + wg * kHeadDim;
         const int tok_local = row / g, head_local = row - tok_local * g;
         const bool live = tok_local < toks;
         const int count = min(L, prior + first_tok + min(tok_local, max(toks, 1) - 1) + 1);   // keys this row sees (>= 1)
         const float scale = prm.scale_log2;
-        const uint32_t leader_pfull[2] = {map_to_cta(bar_pfull(0), 0), map_to_cta(bar_pfull(1), 0)};
-        volatile int *x_flag = reinterpret_cast<volatile int *>(smem + kOffXFlag);
-        volatile float *x_max = reinterpret_cast<volatile float *>(smem + kOffXMax);
-        volatile float *x_sum = reinterpret_cast<volatile float *>(smem + kOffXSum);
-        float m_ref = -INFINITY, l_sum = 0.f;     // l_sum: this thread's 64 columns of every tile
+        const uint32_t leader_pfull = map_to_cta(bar_pfull(wg, 0), 0);
+        float m_ref = -INFINITY, l_sum = 0.f;
 
         for (int j = 0; j < nmax; ++j) {
             const int sb = j & 1;
@@ -396,7 +420,7 @@ chunk_attn_pair_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_co
 
             const int key0 = j * kKeys;
             const bool need_mask = key0 + kKeys > min_count;    // the same for every thread of the CTA
-            const int live_keys = count - key0 - wg * 64;       // of this thread's 64 columns, those the row sees
+            const int live_keys = count - key0 - wg * kCols;    // of this thread's 64 columns, those the row sees
             float rs[4];
             // two copies of the pass, chosen once per tile: the unmasked one carries no compare / select per element
             auto exp_pass = [&](auto masked_tag, float neg_m) {
@@ -422,24 +446,21 @@ chunk_attn_pair_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_co
                         add2(rs[c & 2], rs[(c & 2) + 1], p0, p1);
                         packed[c >> 1] = pack_bf16(p0, p1);
                     }
-                    // P as the next A operand: 32 keys of this row as 16 packed columns at the start of this half of the S buffer
+                    // P as the next A operand: 32 keys of this row as 16 packed columns at the start of this stream's half of the S buffer
                     tmem_st16(sbuf + h * 16, packed);
                 }
                 return (rs[0] + rs[1]) + (rs[2] + rs[3]);
             };
             // Fast path (every unmasked tile after the first): no max pass.  The exponentials are taken against the
-            // row's reference max m_ref (the max of some earlier score, so later keys far below it rightly vanish);
-            // keys far above it make a row sum explode, and then the tile is redone the careful way.  Up to that
-            // bound P and the sums just carry a larger exponent.  Both threads of a row must take the same path (they
-            // share m_ref and O), so the two warps exchange what they saw.
+            // stream's reference max m_ref (the max of some earlier score, so later keys far below it rightly vanish);
+            // keys far above it make the row sum explode, and then (rarely) the tile is redone the careful way below.
+            // Up to that bound P and the sums just carry a larger exponent: fp32 accumulation and the 8-bit mantissa
+            // of bf16 P lose nothing by it.
             float rsum = 0.f, corr = 1.f;
             bool careful = j == 0 || need_mask;
             if (!careful) {
                 rsum = exp_pass(std::false_type{}, -m_ref);
-                const bool mine = __any_sync(0xffffffffu, !(rsum <= kRowSumLimit));   // also true for inf / NaN
-                if (lane == 0) x_flag[(sb * 4 + quarter) * 2 + wg] = mine ? 1 : 0;
-                named_bar_sync(bar_id, 64);
-                careful = mine || x_flag[(sb * 4 + quarter) * 2 + (wg ^ 1)] != 0;
+                careful = __any_sync(0xffffffffu, !(rsum <= kRowSumLimit));   // also true for inf / NaN
                 if (careful) tmem_wait_st();      // the stores of the abandoned pass land before the new ones
             }
             if (careful) {
@@ -469,7 +490,8 @@ chunk_attn_pair_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_co
                         rmax = min3(min3(e[0], e[1], e[2]), min3(e[3], e[4], e[5]), fminf(e[6], e[7])) * scale;
                     }
                 } else {
-                    // masked tile: keys the row does not see are left out (their scores may be anything)
+                    // masked tile: keys the row does not see are left out (their scores may be anything); a row that sees
+                    // none of this stream's keys keeps rmax = -inf and stores P = 0
                     rmax = -INFINITY;
 #pragma unroll
                     for (int h = 0; h < 2; ++h)
@@ -477,22 +499,17 @@ chunk_attn_pair_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_co
                         for (int c = 0; c < 32; ++c)
                             if (h * 32 + c < live_keys) rmax = fmaxf(rmax, __uint_as_float(sraw[h][c]) * scale);
                 }
-                // the row's max over all 128 columns: the other half comes from the partner thread
-                x_max[(sb * 2 + wg) * kRows + row] = rmax;
-                named_bar_sync(bar_id, 64);
-                rmax = fmaxf(rmax, x_max[(sb * 2 + (wg ^ 1)) * kRows + row]);
-                // the reference max moves only when it has to (first tile) or when a row outgrew it by 2^8
+                // the reference max moves only when it has to (first keys of the stream) or when a row outgrew it by 2^8
                 const bool grow = rmax > m_ref + kRescaleThreshold;
                 const float m_new = grow ? rmax : m_ref;
-                corr = grow ? ex2(m_ref - m_new) : 1.f;   // ex2(-inf) = 0 on the first tile
+                corr = grow ? ex2(m_ref - m_new) : 1.f;   // ex2(-inf) = 0 while the stream has seen nothing
                 if (j >= 1 && __any_sync(0xffffffffu, grow)) {
-                    // rare: some row of this warp moved its reference max, so O (the tiles before this one) must be
-                    // rescaled before PV of this tile; PV of the previous tile has to be finished first.  The partner
-                    // warp decides the same and rescales the other 64 columns.
-                    pair_wait(bar_odone((j - 1) & 1), ((j - 1) >> 1) & 1, s_abort, peer_abort, prm.status, 13);
+                    // rare: some row of this warp moved its reference max, so this stream's O (the tiles before this
+                    // one) must be rescaled before PV of this tile; PV of the previous tile has to be finished first
+                    pair_wait(bar_odone(wg, (j - 1) & 1), ((j - 1) >> 1) & 1, s_abort, peer_abort, prm.status, 13);
                     tc_fence_after();
 #pragma unroll 1
-                    for (int c0 = 0; c0 < 64; c0 += 16) {
+                    for (int c0 = 0; c0 < kHeadDim; c0 += 16) {
                         uint32_t oraw[16];
                         tmem_ld16(o_addr + c0, oraw);
                         tmem_wait_ld();
@@ -502,42 +519,55 @@ chunk_attn_pair_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_co
                     }
                 }
                 m_ref = m_new;
+                // a stream that has not seen a key yet (m_ref = -inf) stores zeros through the masked pass
                 rsum = need_mask ? exp_pass(std::true_type{}, -m_ref) : exp_pass(std::false_type{}, -m_ref);
             }
             l_sum = l_sum * corr + rsum;
             tmem_wait_st();
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive_cluster(leader_pfull[sb]);
+            if (lane == 0) mbar_arrive_cluster(leader_pfull + 8u * sb);
         }
 
-        // ---- epilogue: O / l -> bf16 rows of out; each warpgroup writes its 64 dims ----
-        pair_wait(bar_odone((nmax - 1) & 1), ((nmax - 1) >> 1) & 1, s_abort, peer_abort, prm.status, 14);
+        // ---- epilogue: merge the two streams, O / l -> bf16 rows of out; warpgroup w writes dims 64 w .. 64 w + 63 ----
+        pair_wait(bar_odone(0, (nmax - 1) & 1), ((nmax - 1) >> 1) & 1, s_abort, peer_abort, prm.status, 14);
+        pair_wait(bar_odone(1, (nmax - 1) & 1), ((nmax - 1) >> 1) & 1, s_abort, peer_abort, prm.status, 14);
         tc_fence_after();
-        x_sum[wg * kRows + row] = l_sum;
-        named_bar_sync(bar_id, 64);
-        const float l_all = l_sum + x_sum[(wg ^ 1) * kRows + row];
+        volatile float *x_ml = reinterpret_cast<volatile float *>(smem + kOffXMl);
+        x_ml[(wg * kRows + row) * 2] = m_ref;
+        x_ml[(wg * kRows + row) * 2 + 1] = l_sum;
+        named_bar_sync(1 + quarter, 64);                      // the two warps that share these rows
+        const float m0 = x_ml[row * 2], l0 = x_ml[row * 2 + 1], m1 = x_ml[(kRows + row) * 2], l1 = x_ml[(kRows + row) * 2 + 1];
+        const float m_all = fmaxf(m0, m1);
+        const float w0 = m0 == -INFINITY ? 0.f : ex2(m0 - m_all), w1 = m1 == -INFINITY ? 0.f : ex2(m1 - m_all);
+        const float l_all = l0 * w0 + l1 * w1;
         const float inv = l_all > 0.f ? prm.out_scale / l_all : 0.f;
+        const float f0 = w0 * inv, f1 = w1 * inv;
+        const uint32_t o_both = lane_addr + kTmemO + wg * kCols;      // this warpgroup's 64 dims, in O_0; O_1 is 128 columns on
         const long long orow = (static_cast<long long>(q_row0 + first_tok + tok_local) * prm.num_q_heads + head * g + head_local);
 #pragma unroll 1
-        for (int c0 = 0; c0 < 64; c0 += 32) {
-            uint32_t oraw[32];
-            tmem_ld32(o_addr + c0, oraw);
+        for (int c0 = 0; c0 < kCols; c0 += 32) {
+            uint32_t oa[32], ob[32];
+            tmem_ld32(o_both + c0, oa);
+            tmem_ld32(o_both + kHeadDim + c0, ob);
             tmem_wait_ld();
             if (live) {
-                uint4 *dst = reinterpret_cast<uint4 *>(prm.out + orow * kHeadDim + wg * 64 + c0);
+                float ov[32];
+#pragma unroll
+                for (int k = 0; k < 32; ++k) ov[k] = fmaf(__uint_as_float(ob[k]), f1, __uint_as_float(oa[k]) * f0);
+                uint4 *dst = reinterpret_cast<uint4 *>(prm.out + orow * kHeadDim + wg * kCols + c0);
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {
                     uint4 v;
-                    v.x = pack_bf16(__uint_as_float(oraw[8 * k]) * inv, __uint_as_float(oraw[8 * k + 1]) * inv);
-                    v.y = pack_bf16(__uint_as_float(oraw[8 * k + 2]) * inv, __uint_as_float(oraw[8 * k + 3]) * inv);
-                    v.z = pack_bf16(__uint_as_float(oraw[8 * k + 4]) * inv, __uint_as_float(oraw[8 * k + 5]) * inv);
-                    v.w = pack_bf16(__uint_as_float(oraw[8 * k + 6]) * inv, __uint_as_float(oraw[8 * k + 7]) * inv);
+                    v.x = pack_bf16(ov[8 * k], ov[8 * k + 1]);
+                    v.y = pack_bf16(ov[8 * k + 2], ov[8 * k + 3]);
+                    v.z = pack_bf16(ov[8 * k + 4], ov[8 * k + 5]);
+                    v.w = pack_bf16(ov[8 * k + 6], ov[8 * k + 7]);
                     dst[k] = v;
                 }
             }
         }
-        if (live && wg == 0 && prm.lse != nullptr) prm.lse[orow] = l_all > 0.f ? (m_ref + log2f(l_all)) * kLn2 : -INFINITY;
+        if (live && wg == 0 && prm.lse != nullptr) prm.lse[orow] = l_all > 0.f ? (m_all + log2f(l_all)) * kLn2 : -INFINITY;
     }
 
     // ---- all roles of both CTAs meet (nothing of the pair is in flight any more); the tensor memory goes back ----
