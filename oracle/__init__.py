@@ -31,7 +31,7 @@ def lib():
         L = ctypes.CDLL(os.environ.get("ROLLART_ORACLE_LIB") or _build())
         L.oracle_num_threads.restype = ctypes.c_int
         for name in ("oracle_kv_append", "oracle_kv_gather", "oracle_attend", "oracle_lse_combine", "oracle_pages_reserve",
-                     "oracle_pages_release", "oracle_e4m3_decode", "oracle_e4m3_encode"):
+                     "oracle_pages_release", "oracle_pages_evict_stale", "oracle_e4m3_decode", "oracle_e4m3_encode"):
             getattr(L, name).restype = ctypes.c_int
         _lib = L
     return _lib
@@ -134,6 +134,25 @@ def pages_release(free_pages: np.ndarray, free_count: int, page_size: int, page_
                                     ctypes.c_int32(len(seq_lens)), _p(tid), ctypes.c_int32(len(tid)))
     _check(rc)
     return int(cnt.value)
+
+
+def pages_evict_stale(free_pages: np.ndarray, free_count: int, page_size: int, page_table: np.ndarray, seq_lens: np.ndarray,
+                      start_version, current_version: int, alpha: int):
+    """Sec. 6.2 (asynchronous bound alpha): every live trajectory whose start version is older than
+    current_version - alpha gives its pages back (as pages_release would for those trajectories in ascending
+    order), IN PLACE.  Returns (new free count, ids of the evicted trajectories)."""
+    assert free_pages.dtype == np.int32 and page_table.dtype == np.int32 and seq_lens.dtype == np.int32
+    sv = _c(start_version, np.int32)
+    assert len(sv) == len(seq_lens)
+    cnt = ctypes.c_int32(free_count)
+    ids = np.full(len(seq_lens), -1, np.int32)
+    n = ctypes.c_int32(0)
+    rc = lib().oracle_pages_evict_stale(_p(free_pages), ctypes.byref(cnt), ctypes.c_int32(len(free_pages)), ctypes.c_int32(page_size),
+                                        _p(page_table), ctypes.c_int32(page_table.shape[1]), _p(seq_lens),
+                                        ctypes.c_int32(len(seq_lens)), _p(sv), ctypes.c_int32(current_version),
+                                        ctypes.c_int32(alpha), _p(ids), ctypes.byref(n))
+    _check(rc)
+    return int(cnt.value), ids[: n.value].copy()
 
 
 def attend_rows(k_pool: np.ndarray, v_pool: np.ndarray, page_table: np.ndarray,

@@ -4,8 +4,8 @@
  * only the tests, the smoke check and the bench's CPU-baseline leg do.
  *
  * What it computes.  The paper treats the rollout engine step as a black box
- * ("a decode or prefill step for a batch of requests", Sec. 6.1, inference
- * worker event loop) acting on trajectories whose context grows by one
+ * (the inference worker's event loop runs one decode or prefill step at a time
+ * over the requests it holds, Sec. 6.1) acting on trajectories whose context grows by one
  * (observation, action) pair per turn (Sec. 6.1, EnvManager) and whose decode
  * phase is bound by reading that whole context per generated token (Sec. 3.1).
  * The paper prints no formula for the step; the operation has a plain
@@ -184,6 +184,25 @@ int oracle_pages_release(int32_t *free_pages, int32_t *free_count, int32_t capac
         seq_lens[t] = 0;
     }
     *free_count = top;
+    return ORACLE_OK;
+}
+
+/* Stale eviction (Sec. 6.2, asynchronous bound alpha).  With the agent LLM at version n, a buffered trajectory must
+ * have been initiated by a version no older than n - alpha; the ones outside this window are aborted.  Here: every
+ * live trajectory (len > 0) with start_version[t] < n - alpha gives its pages back, exactly as oracle_pages_release
+ * does for the list of those trajectories in ascending order; evicted_ids receives that list, *n_evicted its length. */
+int oracle_pages_evict_stale(int32_t *free_pages, int32_t *free_count, int32_t capacity, int32_t P, int32_t *page_table,
+                             int32_t max_pages, int32_t *seq_lens, int32_t num_traj, const int32_t *start_version,
+                             int32_t current_version, int32_t alpha, int32_t *evicted_ids, int32_t *n_evicted) {
+    if (P <= 0 || num_traj < 0) return ORACLE_BAD_ARG;
+    int32_t n = 0;
+    for (int32_t t = 0; t < num_traj; ++t) {
+        if (seq_lens[t] < 0) return ORACLE_BAD_ARG;
+        if (seq_lens[t] > 0 && (int64_t)start_version[t] < (int64_t)current_version - (int64_t)alpha) evicted_ids[n++] = t;
+    }
+    int rc = oracle_pages_release(free_pages, free_count, capacity, P, page_table, max_pages, seq_lens, num_traj, evicted_ids, n);
+    if (rc != ORACLE_OK) return rc;
+    *n_evicted = n;
     return ORACLE_OK;
 }
 

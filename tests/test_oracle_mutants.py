@@ -29,6 +29,9 @@ MUTANTS = {
     "reserve_rounds_down": ("int64_t want = ((int64_t)seq_lens[t] + new_tokens[i] + P - 1) / P;\n        for (int64_t lp = have;",
                             "int64_t want = ((int64_t)seq_lens[t] + new_tokens[i]) / P;\n        for (int64_t lp = have;"),
     "release_keeps_length": ("        seq_lens[t] = 0;\n", "        seq_lens[t] = seq_lens[t];\n"),
+    "evict_includes_the_boundary_version": ("(int64_t)start_version[t] < (int64_t)current_version - (int64_t)alpha)",
+                                             "(int64_t)start_version[t] <= (int64_t)current_version - (int64_t)alpha)"),
+    "evict_takes_empty_rows": ("if (seq_lens[t] > 0 && (int64_t)start_version[t]", "if (seq_lens[t] >= 0 && (int64_t)start_version[t]"),
     "e4m3_wrong_bias": ("else v = ldexp(1.0 + (double)m / 8.0, e - 7);", "else v = ldexp(1.0 + (double)m / 8.0, e - 8);"),
     "e4m3_subnormals_as_normals": ("else if (e == 0) v = ldexp((double)m / 8.0, -6);",
                                    "else if (e == 0) v = ldexp(1.0 + (double)m / 8.0, -7);"),

@@ -90,3 +90,54 @@ def test_release_then_reserve_reuses_pages_in_stack_order():
     assert (table == -1).all() and lens.tolist() == [0, 0]
     cnt = oracle.pages_reserve(free, cnt, P, table, lens, np.array([17], np.int32), traj_ids=np.array([1], np.int32))
     assert cnt == 3 and table[1].tolist() == [2, 1, -1]
+
+
+def test_stale_eviction_against_list_model_and_closed_form():
+    # Sec. 6.2: with the model at version n, trajectories started before version n - alpha are evicted.  Independent
+    # model: python lists and the release model above; closed form: how many go and how many pages come back.
+    rng = np.random.default_rng(5)
+    P, T, max_pages, num_pages = 16, 40, 6, 300
+    for trial in range(20):
+        lens = rng.integers(0, max_pages * P + 1, size=T).astype(np.int32)
+        lens[rng.integers(0, T, size=6)] = 0                      # empty rows own nothing and are never evicted
+        pages = -(-lens // P)
+        perm = rng.permutation(num_pages).astype(np.int32)
+        table = np.full((T, max_pages), -1, np.int32)
+        o = 0
+        for t in range(T):
+            table[t, :pages[t]] = perm[o:o + pages[t]]
+            o += int(pages[t])
+        free = np.zeros(num_pages, np.int32)
+        cnt = num_pages - o
+        free[:cnt] = perm[o:]
+        n, alpha = int(rng.integers(3, 9)), int(rng.integers(0, 4))
+        sv = rng.integers(0, n + 1, size=T).astype(np.int32)
+        sv[rng.integers(0, T, size=5)] = n - alpha                # on the boundary: still inside the window
+        stale = [t for t in range(T) if lens[t] > 0 and sv[t] < n - alpha]
+        m_free, m_table, m_lens = simulate(free[:cnt], P, table, lens, [("release", t, 0) for t in stale])
+        table2, lens2 = table.copy(), lens.copy()
+        new_cnt, ids = oracle.pages_evict_stale(free, cnt, P, table2, lens2, sv, n, alpha)
+        assert ids.tolist() == stale
+        assert new_cnt == cnt + int(pages[stale].sum()) == len(m_free) and free[:new_cnt].tolist() == m_free
+        assert table2.tolist() == m_table and lens2.tolist() == m_lens
+        assert all(sv[t] >= n - alpha or lens[t] == 0 for t in range(T) if lens2[t] == lens[t])
+
+
+def test_stale_eviction_boundary_and_all_or_nothing():
+    P = 16
+    table = np.array([[4, 5, -1], [6, -1, -1], [7, -1, -1], [-1, -1, -1]], np.int32)
+    lens = np.array([20, 16, 3, 0], np.int32)
+    free = np.array([9, 0, 0, 0, 0, 0], np.int32)
+    # version 5, alpha 1: started at 4 stays, started at 3 goes; the empty row (version 0) is not a trajectory
+    cnt, ids = oracle.pages_evict_stale(free, 1, P, table, lens, np.array([3, 4, 3, 0], np.int32), 5, 1)
+    assert ids.tolist() == [0, 2] and cnt == 4 and free[:4].tolist() == [9, 4, 5, 7]
+    assert lens.tolist() == [0, 16, 0, 0] and table.tolist() == [[-1, -1, -1], [6, -1, -1], [-1, -1, -1], [-1, -1, -1]]
+    # alpha large enough: nothing goes
+    cnt2, ids2 = oracle.pages_evict_stale(free, cnt, P, table, lens, np.array([3, 4, 3, 0], np.int32), 5, 9)
+    assert cnt2 == cnt and len(ids2) == 0
+    # a stack that cannot take the pages: refused, nothing changes
+    small = np.array([1, 0], np.int32)
+    t0, l0 = table.copy(), lens.copy()
+    with pytest.raises(oracle.OracleError):
+        oracle.pages_evict_stale(small, 2, P, table, lens, np.array([0, 0, 0, 0], np.int32), 5, 1)
+    assert np.array_equal(table, t0) and np.array_equal(lens, l0) and small.tolist() == [1, 0]
