@@ -3,9 +3,10 @@
  *
  * Scope.  The rollout stage of agentic RL advances many independent trajectories; each one
  * appends tokens to its own growing context (an observation from the environment, then the
- * tokens of the next action) and the inference worker repeatedly "executes a decode or prefill
- * step for a batch of requests" (paper Sec. 6.1, trajectory-level rollout; Sec. 3.1: decoding is
- * memory-bandwidth bound, observation prefill compute bound).  This library is the attention
+ * tokens of the next action) while the inference worker runs one decode or prefill step after
+ * another over the batch of requests it currently holds (paper Sec. 6.1, trajectory-level rollout
+ * and step-wise command processing; Sec. 3.1: decoding is memory-bandwidth bound, observation
+ * prefill compute bound).  This library is the attention
  * part of that engine step over a paged bf16 KV cache:
  *
  *   rollart_kv_append       write the new tokens' K/V rows into the trajectories' pages
@@ -110,7 +111,8 @@ rollart_status rollart_destroy(rollart_ctx *ctx);
  * already be present in the page table (page allocation is the caller's).  The copy is bit exact;
  * no other byte of the pools changes.  Device-side errors (ROLLART_ERR_BOUNDS): trajectory id out
  * of range, negative length, position beyond max_pages_per_traj * page_size, page id outside
- * [0, num_pages): the offending row is skipped.
+ * [0, num_pages), a new_indptr that is not non-decreasing from 0 to total_new (a row that falls
+ * outside its item's range): the offending row is skipped.
  */
 rollart_status rollart_kv_append(rollart_ctx *ctx, const rollart_kv_pool *pool, const rollart_trajs *trajs,
                                  const int32_t *traj_ids, const int32_t *new_indptr, int32_t n_items,
@@ -124,8 +126,9 @@ rollart_status rollart_kv_append(rollart_ctx *ctx, const rollart_kv_pool *pool, 
  * n_i = out_indptr[i+1] - out_indptr[i] tokens of trajectory traj_ids[i] (NULL = identity) from its
  * pages into rows out_indptr[i] .. of k_out / v_out ([device] bf16 [total_rows][num_kv_heads][head_dim],
  * 16-byte aligned); the receiving side stores them with rollart_kv_append onto its own pages.
- * Bit copy.  n_i > seq_lens[t], a trajectory id or a page id out of range are device-side
- * ROLLART_ERR_BOUNDS errors; the offending rows are left unwritten.
+ * Bit copy.  n_i > seq_lens[t], a trajectory id or a page id out of range, and an out_indptr that is not
+ * non-decreasing from 0 to total_rows are device-side ROLLART_ERR_BOUNDS errors; the offending rows are
+ * left unwritten.
  */
 rollart_status rollart_kv_gather(rollart_ctx *ctx, const rollart_kv_pool *pool, const rollart_trajs *trajs,
                                  const int32_t *traj_ids, const int32_t *out_indptr, int32_t n_items, int32_t total_rows,
@@ -155,6 +158,27 @@ rollart_status rollart_pages_reserve(rollart_ctx *ctx, int32_t *free_pages, int3
 rollart_status rollart_pages_release(rollart_ctx *ctx, int32_t *free_pages, int32_t *free_count, int32_t capacity,
                                      int32_t page_size, int32_t *page_table, int32_t max_pages_per_traj, int32_t *seq_lens,
                                      int32_t num_traj, const int32_t *traj_ids, int32_t n_items, void *stream);
+
+/*
+ * Stale eviction (Sec. 6.2, asynchronous bound alpha: with the agent LLM at version n, a trajectory in flight must
+ * have been started by a version no older than n - alpha; trajectories outside this window are aborted before the
+ * next batch is formed).  The caller keeps the version each trajectory was started under in start_version; this call
+ * selects the stale ones on the device and returns their pages, so that the selection needs no round trip to the host:
+ *
+ *   stale(t)  =  seq_lens[t] > 0  and  start_version[t] < current_version - alpha          (alpha >= 0)
+ *
+ * The stale trajectories, in ascending order of t, are released exactly as rollart_pages_release would release that
+ * list (pages pushed in logical order, table entries set to -1, seq_lens[t] set to 0).
+ *   start_version   [device] int32 [num_traj]
+ *   evicted_ids     [device] int32 [num_traj]: receives the released trajectories, in ascending order
+ *   n_evicted       [device] int32: receives how many there are
+ * Deterministic and all-or-nothing: if the stack cannot take the pages (capacity), or a length is negative or longer
+ * than its table row, nothing changes, *n_evicted is set to 0 and ROLLART_ERR_BOUNDS is recorded for rollart_check.
+ */
+rollart_status rollart_pages_evict_stale(rollart_ctx *ctx, int32_t *free_pages, int32_t *free_count, int32_t capacity,
+                                         int32_t page_size, int32_t *page_table, int32_t max_pages_per_traj, int32_t *seq_lens,
+                                         int32_t num_traj, const int32_t *start_version, int32_t current_version, int32_t alpha,
+                                         int32_t *evicted_ids, int32_t *n_evicted, void *stream);
 
 /*
  * Decode attention (Sec. 3.1: the decoding phase is bound by reading the whole context once per
@@ -191,7 +215,11 @@ rollart_status rollart_decode_attn(rollart_ctx *ctx, const rollart_kv_pool *pool
  * [n_items][num_kv_heads][head_dim], 16-byte aligned) at position len of trajectory traj_ids[i] and its query
  * attends to all len + 1 keys.  max_seq_len bounds the lengths AFTER the step.  seq_lens_out ([device] int32
  * [num_traj] or NULL, must not overlap seq_lens) receives len + 1 for the trajectories named.  Results (pool
- * bytes, out, lse) are identical to the two separate calls.  Device-side errors as for the two calls.
+ * bytes, out, lse) are identical to the two separate calls.  Device-side errors as for the two calls, with one
+ * difference: an item that the device rejects (its new position has no page-table entry, or len + 1 exceeds
+ * max_seq_len) is skipped as a whole: its row is not stored, its seq_lens_out entry is left unwritten, its out row
+ * is 0, so a trajectory that outgrows the bound of a captured decode loop stops advancing instead of leaving
+ * unwritten rows behind.
  */
 rollart_status rollart_append_decode_attn(rollart_ctx *ctx, const rollart_kv_pool *pool, const rollart_trajs *trajs,
                                           const int32_t *traj_ids, int32_t n_items, int32_t max_seq_len, const void *k_new,
@@ -368,9 +396,11 @@ rollart_status rollart_obs_chunk_attn_fp8(rollart_ctx *ctx, const rollart_kv_poo
  *
  * What it does: exactly what rollart_decode_attn does (same kernels, same arithmetic, same
  * meaning of every shared argument), without a context.  The partial results, the ticket counters
- * and a status word live in a fixed array of about 19.2 MB that is part of the library image:
- * every GPU that loads the library holds that memory until the process exits, whether or not
- * this call is ever used.  The call performs no cudaMalloc / cudaFree and calls nothing that does.
+ * and a status word live in a fixed array of about 19.2 MB that is part of the library image.
+ * The call performs no cudaMalloc / cudaFree and calls nothing that does.  The array itself is
+ * not free, though: the CUDA runtime loads a library's kernels and fixed arrays when they are
+ * first used, so the first call on a device (see below) is the moment at which that GPU gives up
+ * the 19.2 MB, and it keeps them until the process exits.
  *
  *   device          CUDA device that owns every [device] pointer of the call.
  *   device_status   [device] int32[4] or NULL.  Cleared on `stream` at the start of the call;
@@ -391,8 +421,12 @@ rollart_status rollart_obs_chunk_attn_fp8(rollart_ctx *ctx, const rollart_kv_poo
  * results: keep these calls on one stream, or order the streams with events.
  *
  * First call on a device: it looks up the device address of the array (cudaGetSymbolAddress,
- * with that device current) and raises the kernel's shared-memory limit.  Make this first call
- * before starting any stream capture; later calls only enqueue work on `stream`.
+ * with that device current) and raises the kernel's shared-memory limit; this is also when the
+ * runtime places the array in device memory.  A call with n_items = 0 does exactly this set-up and
+ * nothing else: it is the warm-up.  Make it at start-up, before the embedding program takes the
+ * device's remaining memory for itself (afterwards the set-up can fail for lack of room: the call
+ * then returns ROLLART_ERR_CUDA and says so in err_buf) and before any stream capture; later
+ * calls only enqueue work on `stream`.
  */
 rollart_status rollart_decode_attn_noalloc(int device, const rollart_kv_pool *pool, const rollart_trajs *trajs,
                                            const int32_t *traj_ids, int32_t n_items, int32_t max_seq_len, const void *q,

@@ -339,9 +339,10 @@ decode_splitkv_kernel(const __grid_constant__ CUtensorMap kmap, const __grid_con
                 // fused append: the new token takes position L; it needs an entry in the page-table row
                 if (L / P >= prm.max_pages) { report(prm.status, ROLLART_ERR_BOUNDS, L, 2); L = -1; }
                 else L += 1;
-                if (blockIdx.x == 0 && prm.seq_lens_out != nullptr && L > 0) prm.seq_lens_out[t] = L;
             }
             if (L < 0 || L > prm.max_seq_len) { report(prm.status, ROLLART_ERR_BOUNDS, L, 2); L = 0; }
+            // the length advances only for an item whose new row is stored (no piece runs for a rejected item)
+            if (prm.k_new != nullptr && blockIdx.x == 0 && prm.seq_lens_out != nullptr && L > 0) prm.seq_lens_out[t] = L;
             if (prm.page_offset != nullptr) {
                 const int off = __ldg(prm.page_offset + i);
                 if (off < 0 || static_cast<long long>(off) * P > L) { report(prm.status, ROLLART_ERR_BOUNDS, off, 2); L = 0; }
@@ -1133,7 +1134,6 @@ extern "C" rollart_status rollart_decode_attn_noalloc(int device, const rollart_
         write_err(err_buf, err_len, "pools, q and out must be 16-byte aligned");
         return ROLLART_ERR_INVALID_ARG;
     }
-    if (n_items == 0) return ROLLART_OK;
     // the fixed scratch bounds the call
     if (n_items > kMaxItems || static_cast<long long>(n_items) * hkv > kStaticMaxUnits) {
         write_err(err_buf, err_len,
@@ -1173,6 +1173,14 @@ extern "C" rollart_status rollart_decode_attn_noalloc(int device, const rollart_
             if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device);
             if (e == cudaSuccess)
                 e = cudaFuncSetAttribute(decode_splitkv_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+            if (e == cudaErrorMemoryAllocation) {
+                cudaGetLastError();
+                write_err(err_buf, err_len, "set-up on device %d failed: the device has no room left for the library's fixed scratch "
+                          "array (%zu bytes, taken when the library's kernels are first loaded): make the first call, which may be "
+                          "an empty one, before the device's memory is given away", device, kStaticBytes);
+                result = ROLLART_ERR_CUDA;
+                break;
+            }
             if (e != cudaSuccess || ptr == nullptr) {
                 write_err(err_buf, err_len, "set-up on device %d failed: %s", device, cudaGetErrorString(e));
                 result = ROLLART_ERR_CUDA;
@@ -1187,6 +1195,7 @@ extern "C" rollart_status rollart_decode_attn_noalloc(int device, const rollart_
             su.sm_count = sms;
             su.done = true;
         }
+        if (n_items == 0) break;      // an empty call is the warm-up: the set-up above is all it does
         CUtensorMap kmap, vmap;
         bool four = encode_pool_map(&kmap, pool->k_pool, pool->num_pages, hkv, pool->page_size, true) &&
                     encode_pool_map(&vmap, pool->v_pool, pool->num_pages, hkv, pool->page_size, true);
@@ -1219,6 +1228,7 @@ extern "C" rollart_status rollart_decode_attn_noalloc(int device, const rollart_
         prm.lse = lse;
         prm.scale_log2 = sm_scale * kLog2e;
         prm.out_scale = 1.f;
+        prm.k_inv_scale = 1.f; prm.v_inv_scale = 1.f;
         prm.tickets = reinterpret_cast<int *>(su.scratch + kStaticStatusBytes);
         prm.k_new = nullptr; prm.v_new = nullptr; prm.k_pool = nullptr; prm.v_pool = nullptr; prm.seq_lens_out = nullptr;
         prm.page_offset = nullptr; prm.out_f32 = nullptr;

@@ -69,7 +69,10 @@ kv_append_kernel(void *__restrict__ k_pool, void *__restrict__ v_pool, float k_i
     if (t < 0 || t >= num_traj) { report(status, ROLLART_ERR_BOUNDS, t, 1); return; }
     const int len = __ldg(seq_lens + t);
     if (len < 0) { report(status, ROLLART_ERR_BOUNDS, len, 1); return; }
-    const long long pos = static_cast<long long>(len) + (row - __ldg(new_indptr + i));
+    // a row outside its item's range means new_indptr is not a non-decreasing array from 0 to total_new
+    const int first = __ldg(new_indptr + i);
+    if (row < first || row >= __ldg(new_indptr + i + 1)) { report(status, ROLLART_ERR_BOUNDS, row, 1); return; }
+    const long long pos = static_cast<long long>(len) + (row - first);
     const long long lp = pos / page_size;
     if (lp >= max_pages) { report(status, ROLLART_ERR_BOUNDS, static_cast<int>(lp), 1); return; }
     const int pg = __ldg(page_table + static_cast<long long>(t) * max_pages + lp);
@@ -105,7 +108,9 @@ kv_gather_kernel(const void *__restrict__ k_pool, const void *__restrict__ v_poo
     const int i = find_item(out_indptr, n_items, row);
     const int t = traj_ids ? __ldg(traj_ids + i) : i;
     if (t < 0 || t >= num_traj) { report(status, ROLLART_ERR_BOUNDS, t, 5); return; }
-    const int pos = row - __ldg(out_indptr + i);
+    const int first = __ldg(out_indptr + i);
+    if (row < first || row >= __ldg(out_indptr + i + 1)) { report(status, ROLLART_ERR_BOUNDS, row, 5); return; }   // malformed out_indptr
+    const int pos = row - first;
     if (pos >= __ldg(seq_lens + t)) { report(status, ROLLART_ERR_BOUNDS, pos, 5); return; }
     const int lp = pos / page_size;
     if (lp >= max_pages) { report(status, ROLLART_ERR_BOUNDS, lp, 5); return; }

@@ -129,6 +129,99 @@ __global__ void __launch_bounds__(kThreads) pages_kernel(const PageArgs a) {
     if (threadIdx.x == 0) *a.free_count = kReserve ? top - moved : top + moved;
 }
 
+struct EvictArgs {
+    int32_t *free_pages;
+    int32_t *free_count;
+    int capacity;
+    int page_size;
+    int32_t *page_table;
+    int max_pages;
+    int32_t *seq_lens;
+    int num_traj;
+    const int32_t *start_version;
+    long long threshold;       // current version - alpha: trajectories started before it are stale
+    int32_t *evicted_ids;
+    int32_t *n_evicted;
+    DeviceStatus *status;
+};
+
+// Stale eviction: the live trajectories whose start version lies before the window give their pages back, in
+// trajectory order, exactly as the release kernel does for that list; the list itself is written out.  Selection
+// and positions come from block-wide scans (a stable compaction), so the result does not depend on timing.
+__global__ void __launch_bounds__(kThreads) pages_evict_kernel(const EvictArgs a) {
+    __shared__ int s_warp[32];
+    __shared__ int s_total, s_bad;
+    __shared__ int s_count[kThreads], s_off[kThreads];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (threadIdx.x == 0) s_bad = 0;
+    __syncthreads();
+    auto stale_pages = [&](int t, bool &stale) {      // pages of trajectory t if it is stale (else 0); -1 if its length is invalid
+        stale = false;
+        const int len = a.seq_lens[t];
+        if (len < 0) return -1;
+        if (len == 0 || static_cast<long long>(__ldg(a.start_version + t)) >= a.threshold) return 0;
+        const long long have = (static_cast<long long>(len) + a.page_size - 1) / a.page_size;
+        if (have > a.max_pages) return -1;
+        stale = true;
+        return static_cast<int>(have);
+    };
+
+    // pass 1: validate and count; nothing is written yet
+    int my_pages = 0, my_items = 0;
+    for (int t = threadIdx.x; t < a.num_traj; t += kThreads) {
+        bool stale;
+        const int n = stale_pages(t, stale);
+        if (n < 0) { s_bad = 1; continue; }
+        my_pages += n;
+        my_items += stale ? 1 : 0;
+    }
+    block_exclusive_scan(my_pages, s_warp, &s_total);
+    const int moved = s_total;
+    block_exclusive_scan(my_items, s_warp, &s_total);
+    const int gone = s_total;
+    const int top = *a.free_count;
+    if (s_bad || top < 0 || static_cast<long long>(top) + moved > a.capacity) {
+        if (threadIdx.x == 0) {
+            report(a.status, ROLLART_ERR_BOUNDS, s_bad ? -1 : moved, 6);
+            *a.n_evicted = 0;
+        }
+        return;
+    }
+
+    // pass 2: chunks of kThreads trajectories in order; a warp moves the pages of one trajectory
+    int base_pages = 0, base_items = 0;
+    for (int c0 = 0; c0 < a.num_traj; c0 += kThreads) {
+        const int t = c0 + threadIdx.x;
+        bool stale = false;
+        const int cnt = t < a.num_traj ? max(0, stale_pages(t, stale)) : 0;
+        const int off_pages = block_exclusive_scan(cnt, s_warp, &s_total);
+        const int chunk_pages = s_total;
+        const int off_items = block_exclusive_scan(stale ? 1 : 0, s_warp, &s_total);
+        const int chunk_items = s_total;
+        s_count[threadIdx.x] = stale ? cnt : -1;
+        s_off[threadIdx.x] = base_pages + off_pages;
+        if (stale) a.evicted_ids[base_items + off_items] = t;
+        __syncthreads();
+        const int n_here = min(kThreads, a.num_traj - c0);
+        for (int it = warp; it < n_here; it += kWarps) {
+            if (s_count[it] < 0) continue;
+            int32_t *row = a.page_table + static_cast<long long>(c0 + it) * a.max_pages;
+            for (int k = lane; k < s_count[it]; k += 32) {
+                a.free_pages[top + s_off[it] + k] = row[k];                    // push in trajectory order
+                row[k] = -1;
+            }
+            if (lane == 0) a.seq_lens[c0 + it] = 0;
+        }
+        base_pages += chunk_pages;
+        base_items += chunk_items;
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        *a.free_count = top + moved;
+        *a.n_evicted = gone;
+    }
+}
+
 }  // namespace
 
 cudaError_t launch_pages(bool reserve, int32_t *free_pages, int32_t *free_count, int capacity, int page_size,
@@ -138,6 +231,17 @@ cudaError_t launch_pages(bool reserve, int32_t *free_pages, int32_t *free_count,
                n_items, status};
     if (reserve) pages_kernel<true><<<1, kThreads, 0, stream>>>(a);
     else pages_kernel<false><<<1, kThreads, 0, stream>>>(a);
+    ++*launches;
+    return cudaGetLastError();
+}
+
+cudaError_t launch_pages_evict(int32_t *free_pages, int32_t *free_count, int capacity, int page_size, int32_t *page_table,
+                               int max_pages, int32_t *seq_lens, int num_traj, const int32_t *start_version,
+                               int current_version, int alpha, int32_t *evicted_ids, int32_t *n_evicted, DeviceStatus *status,
+                               cudaStream_t stream, int64_t *launches) {
+    EvictArgs a{free_pages, free_count, capacity, page_size, page_table, max_pages, seq_lens, num_traj, start_version,
+                static_cast<long long>(current_version) - static_cast<long long>(alpha), evicted_ids, n_evicted, status};
+    pages_evict_kernel<<<1, kThreads, 0, stream>>>(a);
     ++*launches;
     return cudaGetLastError();
 }

@@ -298,6 +298,25 @@ rollart_status rollart_pages_release(rollart_ctx *ctx, int32_t *free_pages, int3
                         num_traj, traj_ids, nullptr, n_items, stream);
 }
 
+rollart_status rollart_pages_evict_stale(rollart_ctx *ctx, int32_t *free_pages, int32_t *free_count, int32_t capacity,
+                                         int32_t page_size, int32_t *page_table, int32_t max_pages_per_traj, int32_t *seq_lens,
+                                         int32_t num_traj, const int32_t *start_version, int32_t current_version, int32_t alpha,
+                                         int32_t *evicted_ids, int32_t *n_evicted, void *stream) {
+    if (!ctx) return ROLLART_ERR_INVALID_ARG;
+    if (!free_pages || !free_count || !page_table || !seq_lens || !start_version || !evicted_ids || !n_evicted)
+        return fail(ctx, ROLLART_ERR_INVALID_ARG, "NULL pointer");
+    if (page_size <= 0 || max_pages_per_traj <= 0 || num_traj <= 0 || capacity < 0)
+        return fail(ctx, ROLLART_ERR_INVALID_ARG, "sizes must be positive");
+    if (alpha < 0) return fail(ctx, ROLLART_ERR_INVALID_ARG, "alpha must not be negative");
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return fail(ctx, ROLLART_ERR_CUDA, "cannot select device %d", ctx->device);
+    cudaError_t e = launch_pages_evict(free_pages, free_count, capacity, page_size, page_table, max_pages_per_traj, seq_lens,
+                                       num_traj, start_version, current_version, alpha, evicted_ids, n_evicted, ctx->d_status,
+                                       static_cast<cudaStream_t>(stream), &ctx->launches);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "pages_evict_stale launch");
+    return ROLLART_OK;
+}
+
 // max_seq_len is only an upper bound: a page-table row cannot hold more than this anyway
 static int32_t clamp_bound(const rollart_kv_pool *pool, const rollart_trajs *trajs, int32_t max_seq_len) {
     const int64_t cap = static_cast<int64_t>(trajs->max_pages_per_traj) * pool->page_size;

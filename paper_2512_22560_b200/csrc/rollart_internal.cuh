@@ -71,6 +71,11 @@ cudaError_t launch_pages(bool reserve, int32_t *free_pages, int32_t *free_count,
                          int32_t *page_table, int max_pages, int32_t *seq_lens, int num_traj, const int32_t *traj_ids,
                          const int32_t *new_tokens, int n_items, DeviceStatus *status, cudaStream_t stream, int64_t *launches);
 
+cudaError_t launch_pages_evict(int32_t *free_pages, int32_t *free_count, int capacity, int page_size, int32_t *page_table,
+                               int max_pages, int32_t *seq_lens, int num_traj, const int32_t *start_version,
+                               int current_version, int alpha, int32_t *evicted_ids, int32_t *n_evicted, DeviceStatus *status,
+                               cudaStream_t stream, int64_t *launches);
+
 // Host-side cache of the TMA tensor maps describing the K and V pools (re-encoded when the pools change).
 struct TmaCache {
     bool valid;

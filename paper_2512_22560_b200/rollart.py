@@ -27,6 +27,7 @@ EXPORTS = (
     "rollart_kv_gather_fp8", "rollart_kv_append_fp8_codes", "rollart_obs_chunk_attn_fp8",
     "rollart_obs_chunk_fp8_scratch_size", "rollart_group_decode_attn_fp8",
     "rollart_obs_chunk_fp8_scratch_size_for_pages", "rollart_append_decode_attn_host", "rollart_host_staging_size",
+    "rollart_pages_evict_stale",
 )
 
 
@@ -77,6 +78,8 @@ def load_library() -> ctypes.CDLL:
     L.rollart_pages_reserve.argtypes = [vp, vp, vp, i32, vp, i32, vp, i32, vp, vp, i32, vp]
     L.rollart_pages_release.restype = ctypes.c_int
     L.rollart_pages_release.argtypes = [vp, vp, vp, i32, i32, vp, i32, vp, i32, vp, i32, vp]
+    L.rollart_pages_evict_stale.restype = ctypes.c_int
+    L.rollart_pages_evict_stale.argtypes = [vp, vp, vp, i32, i32, vp, i32, vp, i32, vp, i32, i32, vp, vp, vp]
     L.rollart_decode_attn.restype = ctypes.c_int
     L.rollart_decode_attn.argtypes = [vp, ctypes.POINTER(_KVPool), ctypes.POINTER(_Trajs), vp, i32, i32, vp, i32, f32,
                                       vp, vp, vp]
@@ -341,6 +344,20 @@ class Context:
             free_pages.shape[0], int(page_size), _ptr(page_table, torch.int32, self.device), page_table.shape[1],
             _ptr(seq_lens, torch.int32, self.device), page_table.shape[0], _ptr(traj_ids, torch.int32, self.device),
             traj_ids.shape[0], self._stream(stream))
+        if st != OK:
+            self._raise(st)
+
+    def pages_evict_stale(self, free_pages, free_count, page_size, page_table, seq_lens, start_version, current_version, alpha,
+                          evicted_ids, n_evicted, stream=None) -> None:
+        """rollart_pages_evict_stale: releases the live trajectories started before version current_version - alpha"""
+        if start_version.shape[0] != page_table.shape[0] or evicted_ids.shape[0] < page_table.shape[0]:
+            raise ValueError("start_version and evicted_ids need one entry per trajectory")
+        st = self._lib.rollart_pages_evict_stale(
+            self._h, _ptr(free_pages, torch.int32, self.device), _ptr(free_count, torch.int32, self.device),
+            free_pages.shape[0], int(page_size), _ptr(page_table, torch.int32, self.device), page_table.shape[1],
+            _ptr(seq_lens, torch.int32, self.device), page_table.shape[0], _ptr(start_version, torch.int32, self.device),
+            int(current_version), int(alpha), _ptr(evicted_ids, torch.int32, self.device),
+            _ptr(n_evicted, torch.int32, self.device), self._stream(stream))
         if st != OK:
             self._raise(st)
 

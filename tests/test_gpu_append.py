@@ -88,6 +88,33 @@ def test_append_device_side_errors_are_reported_not_fatal(cuda_device):
     assert np.array_equal(W.bf16_to_u16(db.k_pool), kp)
 
 
+def test_malformed_indptr_is_a_device_side_error_and_touches_nothing(cuda_device):
+    # new_indptr[0] = 3: the first rows belong to no item.  Before the check such a row computed a negative position
+    # and stored in front of its page; now it is reported and skipped.
+    batch = W.make_batch(W.shrink(W.CONFIGS[0], 4, 4), seed=13)
+    db = DeviceBatch(batch, cuda_device)
+    ctx = rollart.Context(0, 0)
+    k_before, v_before = db.k_pool.clone(), db.v_pool.clone()
+    indptr = db.new_indptr.clone()
+    indptr[:] = int(db.new_indptr[-1])        # every item empty, and rows 0 .. total-1 lie before indptr[0]
+    ctx.kv_append(db.k_pool, db.v_pool, db.page_table, db.lens_before, indptr, db.k_new, db.v_new)
+    assert ctx.status() == rollart.ERR_BOUNDS
+    assert torch.equal(db.k_pool.view(torch.int16), k_before.view(torch.int16))
+    assert torch.equal(db.v_pool.view(torch.int16), v_before.view(torch.int16))
+    # the gather has the same check: rows before out_indptr[0] are left unwritten
+    lens = batch.seq_lens_before
+    good = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    total = int(good[-1])
+    k_out = torch.full((total, batch.spec.num_kv_heads, 128), 7.0, dtype=torch.bfloat16, device=cuda_device)
+    v_out = k_out.clone()
+    bad = good.copy()
+    bad[0] = 3
+    ctx.kv_gather(db.k_pool, db.v_pool, db.page_table, db.lens_before, dev_i32(bad, cuda_device), k_out, v_out)
+    assert ctx.status() == rollart.ERR_BOUNDS
+    assert bool(torch.all(k_out[:3] == 7.0)) and bool(torch.all(v_out[:3] == 7.0))
+    ctx.close()
+
+
 def test_append_host_side_validation(cuda_device):
     batch = W.make_batch(W.shrink(W.CONFIGS[0], 2, 4), seed=12)
     db = DeviceBatch(batch, cuda_device)

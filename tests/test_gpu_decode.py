@@ -205,6 +205,36 @@ def test_fused_append_decode_equals_the_two_calls_and_the_oracle(cuda_device, i,
     assert torch.equal(out.view(torch.int16), out2.view(torch.int16))
 
 
+def test_fused_step_skips_an_item_that_outgrows_the_bound(cuda_device):
+    # max_seq_len one short for the longest trajectory: that item is rejected as a whole (error reported, row not
+    # stored, length not advanced, output row 0); every other item is as the oracle says.
+    batch = W.make_batch(W.shrink(W.CONFIGS[0], 4, 1), seed=77)
+    spec = batch.spec
+    ids, rows = batch.decode_ids, batch.decode_rows()
+    longest = int(np.argmax(batch.seq_lens_after[ids]))
+    msl = int(batch.seq_lens_after[ids].max()) - 1
+    ctx = make_ctx(spec, len(ids), msl + 1)
+    db = DeviceBatch(batch, cuda_device)
+    ridx = torch.from_numpy(rows).to(cuda_device)
+    q, k_new, v_new = (x[ridx].contiguous() for x in (db.q_new, db.k_new, db.v_new))
+    out = torch.full_like(q, float("nan"))
+    lens_out = torch.full_like(db.lens_before, -5)
+    ctx.append_decode_attn(db.k_pool, db.v_pool, db.page_table, db.lens_before, k_new, v_new, q, spec.sm_scale, msl, out,
+                           traj_ids=dev_i32(ids, cuda_device), seq_lens_out=lens_out)
+    assert ctx.status() == rollart.ERR_BOUNDS
+    keep = np.array([j for j in range(len(ids)) if j != longest])
+    kp, vp = W.bf16_to_u16(batch.k_pool), W.bf16_to_u16(batch.v_pool)
+    after = oracle.kv_append(kp, vp, batch.page_table, batch.seq_lens_before, np.arange(len(keep) + 1, dtype=np.int32),
+                             W.bf16_to_u16(batch.k_new[rows[keep]]), W.bf16_to_u16(batch.v_new[rows[keep]]), traj_ids=ids[keep])
+    assert np.array_equal(W.bf16_to_u16(db.k_pool), kp) and np.array_equal(W.bf16_to_u16(db.v_pool), vp)   # the rejected row was not stored
+    got = lens_out.cpu().numpy()
+    assert got[ids[longest]] == -5 and np.array_equal(got[ids[keep]], after[ids[keep]])
+    ref_o, _ = oracle.decode_attn(kp, vp, batch.page_table, after, W.bf16_to_u16(batch.q_new[rows[keep]]), spec.sm_scale, traj_ids=ids[keep])
+    assert_attn_close(out[torch.from_numpy(keep).to(cuda_device)], ref_o, "fused step, items within the bound")
+    assert bool(torch.all(out[longest] == 0))
+    ctx.close()
+
+
 @pytest.mark.parametrize("i,T,div", [(0, 4, 1), (1, 16, 4), (3, 4, 16)])
 def test_results_written_straight_to_pinned_host_memory(cuda_device, i, T, div):
     """out / lse may be page-locked host tensors: the kernel's stores then cross to the host; same bits as device buffers."""

@@ -102,3 +102,46 @@ def test_many_items_use_several_scan_chunks(cuda_device):
     ctx.check()
     assert int(d_cnt.item()) == cnt and np.array_equal(d_free.cpu().numpy()[:cnt], free[:cnt])
     assert np.array_equal(d_table.cpu().numpy(), table) and np.array_equal(d_lens.cpu().numpy(), lens)
+
+
+def test_stale_eviction_matches_oracle_over_several_versions(cuda_device):
+    # Sec. 6.2: the model version advances, trajectories started before the window are evicted, new ones start under
+    # the current version; every array is compared with the oracle after each step.  2500 trajectories: the kernel
+    # walks them in several chunks.
+    rng = np.random.default_rng(8)
+    P, T, max_pages, num_pages = 16, 2500, 6, 9000
+    free = rng.permutation(num_pages).astype(np.int32)
+    cnt = num_pages
+    table = np.full((T, max_pages), -1, np.int32)
+    lens = np.zeros(T, np.int32)
+    sv = np.zeros(T, np.int32)
+    d_free, d_cnt = dev_i32(free, cuda_device), dev_i32([cnt], cuda_device)
+    d_table, d_lens = dev_i32(table, cuda_device), dev_i32(lens, cuda_device)
+    d_ids, d_n = torch.full((T,), -9, dtype=torch.int32, device=cuda_device), dev_i32([-9], cuda_device)
+    ctx = rollart.Context(0, 0)
+    alpha = 1
+    for version in range(1, 7):
+        # trajectories without pages start under this version and take some
+        starters = np.flatnonzero(lens == 0)
+        starters = starters[rng.random(len(starters)) < 0.6].astype(np.int32)
+        new = rng.integers(1, max_pages * P + 1, size=len(starters)).astype(np.int32)
+        cnt = oracle.pages_reserve(free, cnt, P, table, lens, new, traj_ids=starters)
+        ctx.pages_reserve(d_free, d_cnt, P, d_table, d_lens, dev_i32(new, cuda_device), traj_ids=dev_i32(starters, cuda_device))
+        lens[starters] += new
+        sv[starters] = version
+        d_lens.copy_(dev_i32(lens, cuda_device))
+        cnt, ids = oracle.pages_evict_stale(free, cnt, P, table, lens, sv, version, alpha)
+        ctx.pages_evict_stale(d_free, d_cnt, P, d_table, d_lens, dev_i32(sv, cuda_device), version, alpha, d_ids, d_n)
+        ctx.check()
+        assert int(d_n.item()) == len(ids) and np.array_equal(d_ids.cpu().numpy()[: len(ids)], ids)
+        assert int(d_cnt.item()) == cnt and np.array_equal(d_free.cpu().numpy()[:cnt], free[:cnt])
+        assert np.array_equal(d_table.cpu().numpy(), table) and np.array_equal(d_lens.cpu().numpy(), lens)
+        if version >= 3:
+            assert len(ids) > 0
+    # a stack too small for the returned pages: refused, nothing changes, the count reads 0
+    small = d_free[: cnt + 1].clone()
+    t0, l0 = d_table.clone(), d_lens.clone()
+    ctx.pages_evict_stale(small, d_cnt, P, d_table, d_lens, dev_i32(sv, cuda_device), 50, 0, d_ids, d_n)
+    assert ctx.status() == rollart.ERR_BOUNDS
+    assert int(d_n.item()) == 0 and int(d_cnt.item()) == cnt and torch.equal(d_table, t0) and torch.equal(d_lens, l0)
+    ctx.close()

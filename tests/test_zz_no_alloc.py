@@ -6,10 +6,12 @@ engine that has already given the whole GPU to its KV-cache pool, or code that r
 They cannot create a Context (that is where the regular path allocates its workspace), so the
 library offers one call that keeps its scratch in a fixed array inside the library image.  This
 test drives that call through the C ABI twice in a row, with different inputs, and checks each
-result against what the regular rollart_decode_attn call gives for the same inputs, within the
-tolerance used by the other attention tests.  The second call shows that whatever the first one
-left in the shared array does not leak into later results.  This file is named so that pytest
-collects it last.
+result against what the regular rollart_decode_attn call gives for the same inputs (the two run
+the same kernel on the same grid, so the results must be the same bits, which is stricter than
+the tolerance of the other attention tests) and against the CPU oracle within that tolerance.  The
+second call shows that whatever the first one left in the shared array does not leak into later
+results.  A third test makes the documented warm-up call (n_items = 0: set-up only) and then a
+call that launches.  This file is named so that pytest collects it last.
 """
 import dataclasses
 
@@ -17,7 +19,8 @@ import numpy as np
 import pytest
 import torch
 
-from harness import ATOL, RTOL, DeviceBatch, dev_i32, make_ctx
+import oracle
+from harness import ATOL, RTOL, DeviceBatch, assert_attn_close, assert_lse_close, dev_i32, make_ctx, oracle_append
 from paper_2512_22560_b200 import rollart
 from paper_2512_22560_b200 import workloads as W
 
@@ -61,6 +64,13 @@ def test_noalloc_decode_matches_regular_entry_point_twice(cuda_device):
     assert status[0].item() == 0
     assert _close(out1, ref1)
     assert torch.allclose(lse1, ref_lse1, atol=1e-3, rtol=1e-3)
+    assert torch.equal(out1.view(torch.int16), ref1.view(torch.int16)) and torch.equal(lse1, ref_lse1)
+    # and against the oracle, so that this test does not lean on the regular entry point alone
+    kp, vp, after = oracle_append(batch)
+    qbits = W.bf16_to_u16(batch.q_new)
+    o_ref, l_ref = oracle.decode_attn(kp, vp, batch.page_table, after, qbits, spec.sm_scale)
+    assert_attn_close(out1, o_ref, "noalloc call 1")
+    assert_lse_close(lse1, l_ref, "noalloc call 1")
 
     # call 2, right after: a different subset in a different order with other queries and shorter lengths
     ids = dev_i32([3, 0, 4], cuda_device)
@@ -75,7 +85,34 @@ def test_noalloc_decode_matches_regular_entry_point_twice(cuda_device):
     assert status[0].item() == 0
     assert _close(out2, ref2)
     assert torch.allclose(lse2, ref_lse2, atol=1e-3, rtol=1e-3)
+    assert torch.equal(out2.view(torch.int16), ref2.view(torch.int16)) and torch.equal(lse2, ref_lse2)
+    o_ref2, l_ref2 = oracle.decode_attn(kp, vp, batch.page_table, after // 3, W.bf16_to_u16(q2.cpu()), spec.sm_scale,
+                                        traj_ids=np.array([3, 0, 4]))
+    assert_attn_close(out2, o_ref2, "noalloc call 2")
+    assert_lse_close(lse2, l_ref2, "noalloc call 2")
     ctx.close()
+
+
+def test_noalloc_empty_call_is_the_warm_up(cuda_device):
+    # An embedder makes this call at start-up, before it takes the rest of the device's memory: with n_items = 0 the
+    # entry point does its per-device set-up (symbol address, shared-memory limit) and launches nothing.
+    spec = dataclasses.replace(W.CONFIGS[0], num_traj=3, name="noalloc_warm_up")
+    batch = W.make_batch(spec, seed=93)
+    db = DeviceBatch(batch, cuda_device)
+    empty = torch.zeros(0, spec.num_q_heads, 128, dtype=torch.bfloat16, device=cuda_device)
+    rollart.decode_attn_noalloc(db.k_pool, db.v_pool, db.page_table, db.lens_before, empty, spec.sm_scale, 600,
+                                torch.zeros_like(empty))
+    # then a call that launches, checked against the oracle
+    q = db.q_new[:3].contiguous()
+    out = torch.full_like(q, float("nan"))
+    status = torch.full((4,), 5, dtype=torch.int32, device=cuda_device)
+    rollart.decode_attn_noalloc(db.k_pool, db.v_pool, db.page_table, db.lens_before, q, spec.sm_scale, 600, out,
+                                device_status=status)
+    torch.cuda.synchronize()
+    assert status[0].item() == 0
+    ref, _ = oracle.decode_attn(W.bf16_to_u16(batch.k_pool), W.bf16_to_u16(batch.v_pool), batch.page_table,
+                                batch.seq_lens_before, W.bf16_to_u16(batch.q_new[:3]), spec.sm_scale)
+    assert_attn_close(out, ref, "noalloc after warm-up")
 
 
 def test_noalloc_rejects_calls_beyond_its_fixed_scratch_and_reports_device_errors(cuda_device):
