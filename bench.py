@@ -42,9 +42,25 @@ def measured_peaks():
     return FALLBACK_HBM_GBS, "fallback"
 
 
-# dram__bytes_read.sum + dram__bytes_write.sum of one decode_splitkv_kernel launch, from the ncu capture summarised in
-# profiles/decode_splitkv_cfg1.md (default seed).  Valid only for the kernel as captured: set to None when it changes.
-MEASURED_TRAFFIC_BYTES = {"cfg1_7b_gqa_decode": 725.6e6}
+def measured_traffic(workload: str, seed: int):
+    """dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, from the tracked record of an
+    ncu capture.  The record names the workload, the seed and the SHA-256 of the kernel's source files at capture time:
+    any other workload or seed, or a source file that has changed since, gives None (the counters no longer describe
+    the kernel that runs)."""
+    import hashlib
+    path = os.path.join(ROOT, "profiles", "decode_splitkv_traffic.json")
+    try:
+        with open(path) as f:
+            rec = json.load(f)
+        if rec["workload"] != workload or int(rec["seed"]) != int(seed):
+            return None
+        for rel, digest in rec["source_sha256"].items():
+            with open(os.path.join(ROOT, rel), "rb") as f:
+                if hashlib.sha256(f.read()).hexdigest() != digest:
+                    return None
+        return float(rec["dram_bytes_per_launch"])
+    except Exception:
+        return None
 
 
 def decode_algorithmic_bytes(spec: W.WorkloadSpec, lens_after: np.ndarray) -> int:
@@ -167,23 +183,30 @@ class DecodeWorkload:
                                     self.spec.sm_scale, self.max_seq_len, self.out, traj_ids=self.traj_ids,
                                     seq_lens_out=self.lens1)
 
-    def time_steps(self, steps: int, warmup: int):
-        """(total ms over `steps` back-to-back steps, mean ms per launch).  A step is one kernel launch, so the
-        average launch duration is the timed region (two CUDA events, nothing inside the loop) over the step count."""
+    def time_steps(self, steps: int, warmup: int, min_total_ms: float = 0.0):
+        """Times loops of exactly `steps` back-to-back steps (two CUDA events per loop, nothing inside the loop).  A loop
+        that lasts less than min_total_ms is repeated until the loops together last about that long, so that a short
+        `steps` does not rest on one window of a few milliseconds.  Returns the list of loop times in ms.  A step is
+        one kernel launch, so loop time / steps is the average launch period."""
         for _ in range(warmup):
             self.step()
         torch.cuda.synchronize(self.device)
-        t0 = torch.cuda.Event(enable_timing=True)
-        t1 = torch.cuda.Event(enable_timing=True)
-        t0.record()
-        for _ in range(steps):
-            self.step()
-        t1.record()
-        torch.cuda.synchronize(self.device)
-        total = t0.elapsed_time(t1)
-        dec = total / steps          # one launch per step, back to back: the average launch period
+
+        def loops(n):
+            ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n)]
+            for a, b in ev:
+                a.record()
+                for _ in range(steps):
+                    self.step()
+                b.record()
+            torch.cuda.synchronize(self.device)
+            return [a.elapsed_time(b) for a, b in ev]
+
+        times = loops(1)
+        if times[0] < min_total_ms:
+            times += loops(min(2000, int(np.ceil(min_total_ms / max(times[0], 1e-3))) - 1))
         self.ctx.check()
-        return total, dec
+        return times
 
     def time_fp8_steps(self, steps: int, warmup: int, k_scale: float = 0.03, v_scale: float = 0.03):
         """The same step over fp8 (E4M3) pools: quantised append of the new token + fp8 decode attention in one launch.
@@ -588,46 +611,53 @@ def main():
             dist.barrier()
         torch.cuda.synchronize(device)
 
-    launches0 = wl.ctx.launch_count
     barrier()
     with ClockSampler(local) as clocks:
-        total_ms, dec_ms = wl.time_steps(args.steps, args.warmup)
+        # loops of exactly --steps steps; short loops are repeated until the timed region spans about a quarter of a
+        # second, so that the value does not rest on one window of a few milliseconds and the clock sampler sees it
+        loop_ms = wl.time_steps(args.steps, args.warmup, min_total_ms=250.0)
     barrier()
-    launches = args.steps          # one kernel launch per step (rollart_append_decode_attn)
+    per_step = np.array(loop_ms) / args.steps
+    launches = args.steps * len(loop_ms)          # one kernel launch per step (rollart_append_decode_attn)
     # the host-driven loop needs a longer warm-up than the device-timed one: its first few hundred steps run
     # up to 25 % slower (host-side caches and clocks), which 3 steps do not cover
-    e2e_ms, h2d, d2h = wl.time_e2e(max(10, args.steps // 4), max(args.warmup, 200))
-    e2e_steps = max(10, args.steps // 4)
+    e2e_steps = max(10, min(500, max(args.steps, 200) // 4))
+    e2e_ms, h2d, d2h = wl.time_e2e(e2e_steps, max(args.warmup, 200))
 
-    (total_ms, dec_ms, e2e_ms_step), (n_items_all,) = reduce_over_ranks(
-        dist, device, [total_ms, dec_ms, e2e_ms / e2e_steps], [wl.n_items])
-    ms_per_step = total_ms / args.steps
+    (ms_per_step, ms_min, ms_max, e2e_ms_step), (n_items_all,) = reduce_over_ranks(
+        dist, device, [float(np.median(per_step)), float(per_step.min()), float(per_step.max()), e2e_ms / e2e_steps], [wl.n_items])
+    dec_ms = ms_per_step
 
     if rank == 0:
         peak, peak_kind = measured_peaks()
         achieved = wl.bytes / (dec_ms * 1e-3) / 1e9
-        line = {
+        main = {
             "metric": METRIC, "value": n_items_all / (ms_per_step * 1e-3), "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "repeats": len(loop_ms), "ms_per_step_min": ms_min, "ms_per_step_median": ms_per_step, "ms_per_step_max": ms_max,
             "config": {"workload": spec.name, "trajectories_per_gpu": wl.n_items, "num_q_heads": spec.num_q_heads,
                        "num_kv_heads": spec.num_kv_heads, "page_size": spec.page_size,
                        "context_tokens_per_gpu": int(wl.lens_after_host.sum()),
                        "step": "rollart_append_decode_attn: KV append of 1 token/trajectory + decode attention (split-KV partials, last-arriver LSE combine) in one launch, one attention layer",
                        "l2": "inputs larger than L2: %.2f GB of KV read per step" % (wl.bytes / 1e9),
+                       "timing": "loops of exactly `steps` steps between two CUDA events, repeated `repeats` times back to back; ms_per_step = median loop / steps, max over ranks",
                        "parallelism": f"replicas x{world} (independent trajectories, no collective)"},
             "hbm_gbs": achieved, "hbm_frac_of_nominal_8tbs": achieved / NOMINAL_HBM_GBS,
-            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                         "peak_kind": f"of {peak_kind}",
-                         "traffic": MEASURED_TRAFFIC_BYTES.get(spec.name) if args.seed == W.MASTER_SEED else None,
-                         "kernel": "decode_splitkv_kernel (append of the new token, partial attention and split combine in one launch)",
-                         "algorithmic_bytes_per_launch": wl.bytes, "ms_per_launch": dec_ms},
             "e2e": {"value": n_items_all / (e2e_ms_step * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms_step,
                     "note": "per step one rollart_append_decode_attn_host call (arguments marshalled once): q, k_new, v_new host->device from one pinned buffer, out written by the kernel into a pinned host buffer, host sync; the KV pool is resident engine state"},
             "gpu_launches": int(launches),
             "clocks": clocks.summary(),
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                         "peak_kind": f"of {peak_kind}",
+                         "traffic": measured_traffic(spec.name, args.seed),
+                         "kernel": "decode_splitkv_kernel (append of the new token, partial attention and split combine in one launch)",
+                         "algorithmic_bytes_per_launch": wl.bytes, "ms_per_launch": dec_ms},
         }
+        targets = {spec.name: {"ms": dec_ms, "hbm_gbs": achieved, "frac_of_measured": achieved / peak,
+                               "frac_of_nominal_8tbs": achieved / NOMINAL_HBM_GBS}}
+        line = {}
         if not args.no_extra and world == 1:
             extra = {}
             del wl
@@ -637,7 +667,7 @@ def main():
                 name = W.CONFIGS[ci].name + "_fp8_pool"
                 try:
                     w8 = DecodeWorkload(W.CONFIGS[ci], args.seed, device)
-                    _, bf_ms = w8.time_steps(200 if ci == 1 else 20, 3)
+                    bf_ms = float(np.median(w8.time_steps(200 if ci == 1 else 20, 3))) / (200 if ci == 1 else 20)
                     f8_ms, f8_bytes = w8.time_fp8_steps(200 if ci == 1 else 20, 3)
                     extra[name] = {"step_ms": f8_ms, "bf16_step_ms": bf_ms, "speedup_over_bf16_step": bf_ms / f8_ms,
                                    "decode_tokens_per_s": w8.n_items / (f8_ms * 1e-3),
@@ -652,7 +682,7 @@ def main():
             try:
                 # the tiny case lives in L2: a latency figure, back to back and after a write larger than L2
                 w0 = DecodeWorkload(W.CONFIGS[0], args.seed, device)
-                _, hot_ms = w0.time_steps(200, 10)
+                hot_ms = float(np.median(w0.time_steps(200, 10, min_total_ms=50.0))) / 200
                 flush = torch.empty(256 << 20, dtype=torch.uint8, device=device)
                 ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(20)]
                 for a, b in ev:
@@ -688,12 +718,17 @@ def main():
             for ci in (2, 3, 4):
                 try:
                     w2 = DecodeWorkload(W.CONFIGS[ci], args.seed, device)
-                    tot, dms = w2.time_steps(20, 3)
+                    loops = np.array(w2.time_steps(20, 3, min_total_ms=150.0)) / 20
+                    dms = float(np.median(loops))
                     gbs = w2.bytes / (dms * 1e-3) / 1e9
-                    extra[W.CONFIGS[ci].name] = {"decode_ms": dms, "step_ms": tot / 20, "hbm_gbs": gbs,
+                    extra[W.CONFIGS[ci].name] = {"step_ms": dms, "step_ms_min": float(loops.min()), "step_ms_max": float(loops.max()),
+                                                 "repeats": len(loops), "hbm_gbs": gbs,
                                                  "frac_of_measured": gbs / peak, "frac_of_nominal_8tbs": gbs / NOMINAL_HBM_GBS,
-                                                 "decode_tokens_per_s": w2.n_items / (tot / 20 * 1e-3),
+                                                 "decode_tokens_per_s": w2.n_items / (dms * 1e-3),
                                                  "trajectories": w2.n_items}
+                    if ci in (2, 3):
+                        targets[W.CONFIGS[ci].name] = {"ms": dms, "hbm_gbs": gbs, "frac_of_measured": gbs / peak,
+                                                       "frac_of_nominal_8tbs": gbs / NOMINAL_HBM_GBS}
                     if ci == 3:
                         g_ms, g_bytes = w2.time_gather()
                         extra[W.CONFIGS[ci].name].update({"kv_gather_ms": g_ms, "kv_gather_gbs": g_bytes / (g_ms * 1e-3) / 1e9,
@@ -706,15 +741,18 @@ def main():
             try:
                 cw = ChunkWorkload(W.CONFIGS[4], args.seed, device)
                 app_ms, att_ms = cw.time(5, 2)
-                tf_peak = 1399.5
+                tf_peak, tf_burst = 1399.5, 1590.0           # the fallbacks (sustained, burst) if the measured peaks are absent
                 try:
                     with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
-                        tf_peak = float(json.load(f)["bf16_tflops_sustained"])
+                        mp = json.load(f)
+                    tf_peak, tf_burst = float(mp["bf16_tflops_sustained"]), float(mp["bf16_tflops"])
                 except Exception:
                     pass
                 tfs = cw.flops / (att_ms * 1e-3) / 1e12
                 extra["cfg4_mixed_multiturn_chunk_half"] = {
                     "chunk_rows": cw.rows, "chunk_attn_ms": att_ms, "tflops": tfs, "frac_of_measured_bf16_sustained": tfs / tf_peak,
+                    "frac_of_measured_bf16_burst": tfs / tf_burst,
+                    "kernel": "chunk_attn_pair_kernel (tcgen05 cta_group::2, one launch per call)",
                     "append_ms": app_ms, "append_gbs": cw.append_bytes / (app_ms * 1e-3) / 1e9,
                     "append_frac_of_measured_hbm": cw.append_bytes / (app_ms * 1e-3) / 1e9 / peak}
                 try:
@@ -733,7 +771,9 @@ def main():
             try:
                 rw = ChunkWorkload(W.RECOMPUTE, args.seed, device)
                 app_ms, att_ms = rw.time(3, 2)
-                extra[W.RECOMPUTE.name] = {"rows": rw.rows, "chunk_attn_ms": att_ms, "tflops": rw.flops / (att_ms * 1e-3) / 1e12,
+                rtf = rw.flops / (att_ms * 1e-3) / 1e12
+                extra[W.RECOMPUTE.name] = {"rows": rw.rows, "chunk_attn_ms": att_ms, "tflops": rtf,
+                                           "frac_of_measured_bf16_sustained": rtf / tf_peak, "frac_of_measured_bf16_burst": rtf / tf_burst,
                                            "append_ms": app_ms, "append_gbs": rw.append_bytes / (app_ms * 1e-3) / 1e9}
                 rw.ctx.close()
                 del rw
@@ -768,7 +808,10 @@ def main():
                     extra[name] = {"error": repr(e)}
             line["other_workloads"] = extra
             info, _, _ = CpuBaseline(spec, args.seed).measure()
-            line["cpu_baseline"] = info
+            main["cpu_baseline"] = info
+        # the long block of other workloads goes first, the headline keys and the three target workloads last
+        line.update(main)
+        line["targets"] = targets
         print(json.dumps(line))
     if dist is not None:
         dist.barrier()

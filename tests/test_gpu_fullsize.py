@@ -280,3 +280,179 @@ def test_full_size_mixed_batch_fp8_chunk_sampled_rows(cuda_device):
                                   row_count, W.bf16_to_u16(q[q_rows]), sm)
     assert_attn_close(out[q_rows], ref_o * float(np.float32(vs)), "cfg4 fp8 chunk rows")
     ctx.close()
+
+
+def _stratified_rows(n, tile, rng, n_random):
+    """first / last rows, rows around tile edges near the start, the middle and the end of an n-row chunk, random rows"""
+    edges = [e for e in range(tile, n, tile)]
+    near = edges[:3] + edges[len(edges) // 2: len(edges) // 2 + 3] + edges[-3:]
+    cand = {0, 1, n - 2, n - 1} | {r for e in near for r in (e - 1, e, e + 1)}
+    cand |= {int(x) for x in rng.integers(0, n, size=n_random)}
+    return sorted(c for c in cand if 0 <= c < n)
+
+
+def test_full_size_recompute_sampled_rows(cuda_device):
+    # KV recomputation at the size bench.py times: whole contexts of up to 32 K tokens as one causal chunk onto empty
+    # pages.  Thousands of M-tiles per (item, head), thousands of key tiles on the last ones.  Rows of the shortest,
+    # the median and the longest trajectory against the oracle, out and lse.
+    spec = W.RECOMPUTE
+    batch = W.make_batch(spec, device=cuda_device)
+    ids = batch.chunk_ids
+    rows, q_indptr = batch.chunk_rows()
+    msl = int(batch.seq_lens_after.max())
+    ctx = make_ctx(spec, len(ids), msl)
+    db = DeviceBatch(batch, cuda_device)
+    db.append(ctx)
+    q = db.q_new[torch.from_numpy(rows).to(cuda_device)].contiguous()
+    out = torch.full_like(q, float("nan"))
+    lse = torch.full((q.shape[0], spec.num_q_heads), float("nan"), device=cuda_device)
+    ctx.obs_chunk_attn(db.k_pool, db.v_pool, db.page_table, db.lens_after, dev_i32(q_indptr, cuda_device), q, spec.sm_scale,
+                       msl, out, lse=lse, traj_ids=dev_i32(ids, cuda_device))
+    ctx.check()
+    assert torch.all(torch.isfinite(out.float())) and torch.all(torch.isfinite(lse))
+    rng = np.random.default_rng(46)
+    order = np.argsort(batch.n_new[ids], kind="stable")
+    pick_local = sorted({int(order[0]), int(order[-1]), int(order[len(order) // 2])})
+    pick = ids[pick_local]
+    post = W.extract_trajs(db_as_batch(batch, db), pick)
+    kp, vp = W.bf16_to_u16(post.k_pool), W.bf16_to_u16(post.v_pool)
+    after = post.seq_lens_before + post.n_new
+    tile = 128 // (spec.num_q_heads // spec.num_kv_heads)           # chunk tokens per 128-row tile of the kernel
+    row_traj, row_count, q_rows = [], [], []
+    for i, li in enumerate(pick_local):
+        n = int(batch.n_new[ids[li]])
+        for j in _stratified_rows(n, tile, rng, 64):
+            row_traj.append(i)
+            row_count.append(int(after[i]) - n + j + 1)
+            q_rows.append(int(q_indptr[li]) + j)
+    q_rows = torch.from_numpy(np.array(q_rows)).to(cuda_device)
+    ref_o, ref_l = oracle.attend_rows(kp, vp, post.page_table, row_traj, row_count, W.bf16_to_u16(q[q_rows]), spec.sm_scale)
+    assert_attn_close(out[q_rows], ref_o, "recompute rows")
+    assert_lse_close(lse[q_rows], ref_l, "recompute rows")
+    ctx.close()
+
+
+def test_full_size_mixed_batch_chunk_lse_and_needles(cuda_device):
+    # The chunk half of the mixed batch with keys planted that dominate the softmax of sampled chunk rows (outputs of
+    # order one: a wrong key, page or tile would show): for each sampled row, keys aligned with that row's own
+    # queries in the prior cache (first token, page edges, one every 2048 positions), at the first chunk token and at
+    # the row's own position.  out and lse of those rows and of their neighbours against the oracle.
+    spec = W.CONFIGS[4]
+    batch = W.make_batch(spec, device=cuda_device)
+    ids = batch.chunk_ids
+    rows, q_indptr = batch.chunk_rows()
+    g, P = spec.num_q_heads // spec.num_kv_heads, spec.page_size
+    rng = np.random.default_rng(47)
+    order = np.argsort(batch.n_new[ids], kind="stable")
+    pick_local = sorted({int(order[0]), int(order[-1]), int(order[len(order) // 2])})
+    tile = 128 // g
+    sampled = {}                                                     # local index -> chunk rows with needles
+    for li in pick_local:
+        t = int(ids[li])
+        n, prior = int(batch.n_new[t]), int(batch.seq_lens_before[t])
+        edges = [e for e in range(tile, n, tile)]
+        js = sorted({0, n - 1, n // 2} | {r for e in edges[:2] + edges[-2:] for r in (e - 1, e)} | {int(x) for x in rng.integers(0, n, size=6)})
+        js = [j for j in js if 0 <= j < n]
+        sampled[li] = js
+        for k, j in enumerate(js):
+            qrow = int(batch.new_indptr[t]) + j
+            qv = batch.q_new[qrow].float().view(spec.num_kv_heads, g, spec.head_dim)
+            count = prior + j + 1
+            want = {0, P - 1, P, prior - 1, prior, count - 1} | set(range(1027, count, 2048))
+            for pos in sorted(p_ for p_ in want if 0 <= p_ < count):
+                pos = min(count - 1, pos + 3 * k) if pos not in (prior, count - 1) else pos     # rows do not share needles
+                kvec = (3.0 * qv[:, pos % g, :]).to(torch.bfloat16)
+                if pos < prior:
+                    batch.k_pool[int(batch.page_table[t, pos // P]), :, pos % P, :] = kvec
+                else:
+                    batch.k_new[int(batch.new_indptr[t]) + (pos - prior)] = kvec
+    msl = int(batch.seq_lens_after.max())
+    ctx = make_ctx(spec, len(ids), msl)
+    db = DeviceBatch(batch, cuda_device)
+    db.append(ctx)
+    q = db.q_new[torch.from_numpy(rows).to(cuda_device)].contiguous()
+    out = torch.full_like(q, float("nan"))
+    lse = torch.full((q.shape[0], spec.num_q_heads), float("nan"), device=cuda_device)
+    ctx.obs_chunk_attn(db.k_pool, db.v_pool, db.page_table, db.lens_after, dev_i32(q_indptr, cuda_device), q, spec.sm_scale,
+                       msl, out, lse=lse, traj_ids=dev_i32(ids, cuda_device))
+    ctx.check()
+    post = W.extract_trajs(db_as_batch(batch, db), ids[pick_local])
+    kp, vp = W.bf16_to_u16(post.k_pool), W.bf16_to_u16(post.v_pool)
+    after = post.seq_lens_before + post.n_new
+    row_traj, row_count, q_rows = [], [], []
+    for i, li in enumerate(pick_local):
+        n = int(batch.n_new[ids[li]])
+        for j in sorted({r for j in sampled[li] for r in (j - 1, j, j + 1) if 0 <= r < n}):
+            row_traj.append(i)
+            row_count.append(int(after[i]) - n + j + 1)
+            q_rows.append(int(q_indptr[li]) + j)
+    q_rows = torch.from_numpy(np.array(q_rows)).to(cuda_device)
+    ref_o, ref_l = oracle.attend_rows(kp, vp, post.page_table, row_traj, row_count, W.bf16_to_u16(q[q_rows]), spec.sm_scale)
+    st = assert_attn_close(out[q_rows], ref_o, "cfg4 chunk rows (needles)")
+    assert st["rms_ref"] > 0.1, st
+    assert_lse_close(lse[q_rows], ref_l, "cfg4 chunk rows (needles)")
+    ctx.close()
+
+
+def test_full_size_mixed_batch_decode_half_with_needles(cuda_device):
+    # the decode half of the mixed batch (64 single-token trajectories among 128) with planted keys, as the decode
+    # needle test above does for the three decode workloads
+    spec = W.CONFIGS[4]
+    batch = W.make_batch(spec, device=cuda_device)
+    ids = batch.decode_ids
+    rng = np.random.default_rng(104)
+    pick = sample_ids(batch.seq_lens_before, ids, 4, rng)
+    P = spec.page_size
+    pos = {}
+    for t in pick:
+        L = int(batch.seq_lens_before[t])
+        special = {0, L - 1, min(L - 1, P - 1), min(L - 1, P), (L // P) * P if L % P else L - P, L}
+        pos[int(t)] = sorted(special | set(range(1027, L, 2048)))
+    W.plant_needles(batch, pos)
+    rows = batch.decode_rows()
+    msl = int(batch.seq_lens_after[ids].max())
+    ctx = make_ctx(spec, len(ids), msl)
+    db = DeviceBatch(batch, cuda_device)
+    ridx = torch.from_numpy(rows).to(cuda_device)
+    q = db.q_new[ridx].contiguous()
+    out = torch.full_like(q, float("nan"))
+    lse = torch.full((len(ids), spec.num_q_heads), float("nan"), device=cuda_device)
+    ctx.append_decode_attn(db.k_pool, db.v_pool, db.page_table, db.lens_before, db.k_new[ridx].contiguous(),
+                           db.v_new[ridx].contiguous(), q, spec.sm_scale, msl, out, lse=lse, traj_ids=dev_i32(ids, cuda_device),
+                           seq_lens_out=db.lens_after)
+    ctx.check()
+    post = W.extract_trajs(db_as_batch(batch, db), pick)
+    where = {int(t): i for i, t in enumerate(ids)}
+    sel = torch.from_numpy(np.array([where[int(t)] for t in pick])).to(cuda_device)
+    ref_o, ref_l = oracle.decode_attn(W.bf16_to_u16(post.k_pool), W.bf16_to_u16(post.v_pool), post.page_table,
+                                      post.seq_lens_before + 1, W.bf16_to_u16(q[sel]), spec.sm_scale)
+    st = assert_attn_close(out[sel], ref_o, spec.name + " decode half (needles)")
+    assert st["rms_ref"] > 0.1, st
+    assert_lse_close(lse[sel], ref_l, spec.name + " decode half (needles)")
+    ctx.close()
+
+
+def test_full_size_kv_gather_sampled(cuda_device):
+    # the hand-off gather at the size bench.py times (the long-horizon workload: 32 trajectories, 2.6 M tokens): every
+    # byte of three sampled trajectories' rows against the oracle's gather over a host copy of their pages
+    spec = W.CONFIGS[3]
+    batch = W.make_batch(spec, device=cuda_device)
+    lens = batch.seq_lens_before
+    indptr = np.concatenate([[0], np.cumsum(lens.astype(np.int64))])
+    assert indptr[-1] < 2 ** 31
+    ctx = rollart.Context(0, 0)
+    table, d_lens = dev_i32(batch.page_table, cuda_device), dev_i32(lens, cuda_device)
+    k_out = torch.full((int(indptr[-1]), spec.num_kv_heads, spec.head_dim), float("nan"), dtype=torch.bfloat16, device=cuda_device)
+    v_out = torch.full_like(k_out, float("nan"))
+    ctx.kv_gather(batch.k_pool, batch.v_pool, table, d_lens, dev_i32(indptr, cuda_device), k_out, v_out)
+    ctx.check()
+    rng = np.random.default_rng(48)
+    pick = sample_ids(lens, np.arange(spec.num_traj), 3, rng)
+    post = W.extract_trajs(batch, pick)
+    sub_indptr = np.concatenate([[0], np.cumsum(post.seq_lens_before.astype(np.int64))]).astype(np.int32)
+    rk, rv = oracle.kv_gather(W.bf16_to_u16(post.k_pool), W.bf16_to_u16(post.v_pool), post.page_table, post.seq_lens_before, sub_indptr)
+    for i, t in enumerate(pick):
+        a, b = int(indptr[t]), int(indptr[t + 1])
+        assert np.array_equal(W.bf16_to_u16(k_out[a:b]), rk[sub_indptr[i]:sub_indptr[i + 1]])
+        assert np.array_equal(W.bf16_to_u16(v_out[a:b]), rv[sub_indptr[i]:sub_indptr[i + 1]])
+    ctx.close()

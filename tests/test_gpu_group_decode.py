@@ -205,6 +205,50 @@ def test_full_size_group_decode_sampled(cuda_device):
     ctx.close()
 
 
+def test_full_size_fp8_group_decode_sampled(cuda_device):
+    """The group call over fp8 pools on the GRPO workload at the size bench.py times: quantising append, group call,
+    sampled members recomputed by the oracle's plain fp8 decode from a host copy of their pages' codes."""
+    dev = cuda_device
+    spec = W.GROUP_DECODE
+    ks, vs = 0.03, 0.02
+    layout = W.make_layout(spec, W.MASTER_SEED)
+    indptr, shared = W.share_group_prefix(layout, W.GROUP_SIZE, W.GROUP_SHARED_FRACTION)
+    batch = W.fill_tensors(layout, dev)
+    # any codes will do for the existing cache (the oracle reads the same bytes); aliased prefix pages are the same
+    # physical pages, so the members of a group see the same codes there
+    k8 = (batch.k_pool.float() / ks).clamp_(-448, 448).to(torch.float8_e4m3fn).view(torch.uint8)
+    v8 = (batch.v_pool.float() / vs).clamp_(-448, 448).to(torch.float8_e4m3fn).view(torch.uint8)
+    T = spec.num_traj
+    msl = int(batch.seq_lens_after.max())
+    table, lens0 = dev_i32(batch.page_table, dev), dev_i32(batch.seq_lens_before, dev)
+    lens1 = torch.empty_like(lens0)
+    ctx = group_ctx(spec, T, msl)
+    ctx.kv_append_fp8(k8, v8, table, lens0, dev_i32(batch.new_indptr, dev), batch.k_new, batch.v_new, ks, vs, seq_lens_out=lens1)
+    q = batch.q_new.contiguous()
+    out = torch.full_like(q, float("nan"))
+    lse = torch.full((T, spec.num_q_heads), float("nan"), device=dev)
+    need = rollart.obs_chunk_fp8_scratch_size(len(indptr) - 1, spec.num_kv_heads, spec.page_size, msl)
+    scratch = torch.empty(need, dtype=torch.uint8, device=dev)
+    ctx.group_decode_attn_fp8(k8, v8, table, lens1, dev_i32(indptr, dev), dev_i32(shared, dev), q, spec.sm_scale, ks, vs, msl, out,
+                              scratch, lse=lse)
+    ctx.check()
+    assert torch.all(torch.isfinite(out.float())) and torch.all(torch.isfinite(lse))
+    del scratch
+    lens = batch.seq_lens_before
+    order = np.argsort(lens, kind="stable")
+    gi = int(np.argmax(shared))
+    pick = sorted({int(order[0]), int(order[-1]), int(order[len(order) // 2]), int(indptr[gi]), int(indptr[gi + 1] - 1), 77})
+    b8 = dataclasses.replace(batch)
+    b8.k_pool, b8.v_pool = k8, v8                         # codes after the GPU append
+    post = W.extract_trajs(b8, pick)
+    sel = torch.tensor(pick, device=dev)
+    ref_o, ref_l = oracle.decode_attn_fp8(post.k_pool.numpy(), post.v_pool.numpy(), post.page_table, post.seq_lens_before + 1,
+                                          W.bf16_to_u16(q[sel]), spec.sm_scale, ks, vs)
+    assert_attn_close(out[sel], ref_o, spec.name + " fp8")
+    assert_lse_close(lse[sel], ref_l, spec.name + " fp8")
+    ctx.close()
+
+
 def run_fp8_group_case(spec, seed, group_size, fraction, device, ks=0.03, vs=0.02):
     """The group call over fp8 pools: the cache is the oracle's quantisation of the bf16 recipe (members alias the same
     prefix pages, so they hold the same codes), the new token goes through the quantising append; expected values are
