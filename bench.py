@@ -529,6 +529,144 @@ def reduce_over_ranks(dist, device, maxima, sums):
     return t.tolist(), u.tolist()
 
 
+# ---- KV hand-off between two workers (Sec. 6.3: with prefill/decode disaggregation a trajectory's cache moves to another
+# worker; Sec. 6.1: a trajectory resumes elsewhere).  Sender: rollart_kv_gather into contiguous rows; the rows cross to the
+# receiver's own buffer (torch.distributed send / recv: NCCL between GPUs, no peer pointer is handed to any kernel);
+# receiver: rollart_pages_reserve + rollart_kv_append onto its own pages.
+
+def handoff_plan(lens):
+    """indptr of the contiguous hand-off buffer for trajectories of these lengths (int32 [n + 1])"""
+    indptr = np.concatenate([[0], np.cumsum(np.asarray(lens, dtype=np.int64))])
+    if indptr[-1] >= 2 ** 31:
+        raise ValueError("too many rows for one hand-off")
+    return indptr.astype(np.int32)
+
+
+def handoff_bytes(total_rows: int, num_kv_heads: int, head_dim: int, elem_bytes: int = 2) -> int:
+    """bytes that cross between the workers: K and V rows"""
+    return 2 * int(total_rows) * num_kv_heads * head_dim * elem_bytes
+
+
+def handoff_send(dist, dst: int, lens, k_rows: torch.Tensor, v_rows: torch.Tensor) -> int:
+    """Sender side: the lengths first (the receiver sizes its buffers from them), then the K and the V rows."""
+    dev = k_rows.device
+    lens_t = torch.as_tensor(np.asarray(lens, dtype=np.int32), device=dev)
+    dist.send(torch.tensor([lens_t.numel()], dtype=torch.int32, device=dev), dst)
+    dist.send(lens_t, dst)
+    dist.send(k_rows, dst)
+    dist.send(v_rows, dst)
+    return k_rows.numel() * k_rows.element_size() + v_rows.numel() * v_rows.element_size()
+
+
+def handoff_recv(dist, src: int, device, num_kv_heads: int, head_dim: int, dtype=torch.bfloat16):
+    """Receiver side: (lens, indptr, k_rows, v_rows) in the receiver's own memory."""
+    n = torch.zeros(1, dtype=torch.int32, device=device)
+    dist.recv(n, src)
+    lens_t = torch.zeros(int(n.item()), dtype=torch.int32, device=device)
+    dist.recv(lens_t, src)
+    lens = lens_t.cpu().numpy()
+    indptr = handoff_plan(lens)
+    k_rows = torch.empty(int(indptr[-1]), num_kv_heads, head_dim, dtype=dtype, device=device)
+    v_rows = torch.empty_like(k_rows)
+    dist.recv(k_rows, src)
+    dist.recv(v_rows, src)
+    return lens, indptr, k_rows, v_rows
+
+
+def run_handoff(args, dist, rank: int, world: int, device):
+    """`--handoff`: world size 2 = sender (rank 0) and receiver (rank 1); world size 1 = both roles on one GPU with the
+    transfer left out (a check of everything but the wire).  The received cache must serve a decode call with the
+    sender's bits."""
+    from paper_2512_22560_b200 import rollart
+    spec = W.CONFIGS[args.config]
+    i32 = lambda a: torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).to(device)
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    times, moved, check = {}, 0, None
+    k_rows = v_rows = lens = indptr = q = ref_out = None
+    if rank == 0:
+        b = W.make_batch(spec, seed=args.seed, device=device)
+        lens = b.seq_lens_before
+        indptr = handoff_plan(lens)
+        table, d_lens = i32(b.page_table), i32(lens)
+        ctx = rollart.Context(device.index or 0, rollart.workspace_size(spec.num_traj, spec.num_q_heads, spec.num_kv_heads, int(lens.max())))
+        k_rows = torch.empty(int(indptr[-1]), spec.num_kv_heads, spec.head_dim, dtype=torch.bfloat16, device=device)
+        v_rows = torch.empty_like(k_rows)
+        a, z = ev(), ev()
+        ctx.kv_gather(b.k_pool, b.v_pool, table, d_lens, i32(indptr), k_rows, v_rows)          # warm-up
+        a.record()
+        ctx.kv_gather(b.k_pool, b.v_pool, table, d_lens, i32(indptr), k_rows, v_rows)
+        z.record()
+        q = b.q_new[torch.from_numpy(b.decode_rows(np.arange(spec.num_traj))).to(device)].contiguous()
+        ref_out = torch.empty_like(q)
+        ctx.decode_attn(b.k_pool, b.v_pool, table, d_lens, q, spec.sm_scale, int(lens.max()), ref_out)
+        ctx.check()
+        times["gather_ms"] = a.elapsed_time(z)
+        if world == 2:
+            torch.cuda.synchronize(device)
+            t0 = time.perf_counter()
+            moved = handoff_send(dist, 1, lens, k_rows, v_rows)
+            dist.send(q, 1)
+            dist.send(ref_out, 1)
+            torch.cuda.synchronize(device)
+            times["transfer_ms"] = (time.perf_counter() - t0) * 1e3
+        ctx.close()
+        del b
+    if rank == world - 1:
+        if world == 2:
+            torch.cuda.synchronize(device)
+            t0 = time.perf_counter()
+            lens, indptr, k_rows, v_rows = handoff_recv(dist, 0, device, spec.num_kv_heads, spec.head_dim)
+            torch.cuda.synchronize(device)
+            times["transfer_ms"] = (time.perf_counter() - t0) * 1e3
+            q = torch.empty(len(lens), spec.num_q_heads, spec.head_dim, dtype=torch.bfloat16, device=device)
+            ref_out = torch.empty_like(q)
+            dist.recv(q, 0)
+            dist.recv(ref_out, 0)
+        # the receiver's own pool and bookkeeping: every page free, every row empty
+        P = spec.page_size
+        pages = (np.asarray(lens, dtype=np.int64) + P - 1) // P
+        num_pages, max_pages, T = int(pages.sum()) + 8, int(pages.max()), len(lens)
+        k_pool = torch.zeros(num_pages, spec.num_kv_heads, P, spec.head_dim, dtype=torch.bfloat16, device=device)
+        v_pool = torch.zeros_like(k_pool)
+        free = torch.arange(num_pages, dtype=torch.int32, device=device)
+        cnt = torch.tensor([num_pages], dtype=torch.int32, device=device)
+        table = torch.full((T, max_pages), -1, dtype=torch.int32, device=device)
+        lens0, lens1 = torch.zeros(T, dtype=torch.int32, device=device), torch.zeros(T, dtype=torch.int32, device=device)
+        ctx = rollart.Context(device.index or 0, rollart.workspace_size(T, spec.num_q_heads, spec.num_kv_heads, int(max(lens))))
+        a, z = ev(), ev()
+        a.record()
+        ctx.pages_reserve(free, cnt, P, table, lens0, i32(lens))
+        ctx.kv_append(k_pool, v_pool, table, lens0, i32(indptr), k_rows, v_rows, seq_lens_out=lens1)
+        z.record()
+        out = torch.empty_like(q)
+        ctx.decode_attn(k_pool, v_pool, table, lens1, q, spec.sm_scale, int(max(lens)), out)
+        ctx.check()
+        times["reserve_append_ms"] = a.elapsed_time(z)
+        check = bool(torch.equal(out.view(torch.int16), ref_out.view(torch.int16)))
+        ctx.close()
+    keys = ["gather_ms", "transfer_ms", "reserve_append_ms"]
+    (t_max), _ = reduce_over_ranks(dist, device, [times.get(k, 0.0) for k in keys], [0])
+    ok = torch.tensor([1.0 if check in (None, True) else 0.0], dtype=torch.float64, device=device)
+    if dist is not None:
+        dist.all_reduce(ok, op=dist.ReduceOp.MIN)
+    if rank == 0:
+        total_rows = int(indptr[-1])
+        nbytes = handoff_bytes(total_rows, spec.num_kv_heads, spec.head_dim)
+        line = {"workload": spec.name + " (KV hand-off: gather -> transfer -> reserve + append)", "n_gpus": world,
+                "trajectories": int(len(lens)), "rows": total_rows, "bytes_moved": nbytes if world == 2 else 0,
+                "decode_over_received_cache_bit_identical": bool(ok.item() == 1.0)}
+        line.update({k: v for k, v in zip(keys, t_max)})
+        if world == 2 and t_max[1] > 0:
+            line["transfer_gbs"] = nbytes / (t_max[1] * 1e-3) / 1e9
+        else:
+            line["note"] = "one GPU: sender and receiver roles on the same device, no transfer"
+        print(json.dumps(line))
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+    return 0
+
+
 def run_reference(args):
     """`--impl reference`: the CPU oracle on a bounded sample per step (rank 0 only)."""
     rank = int(os.environ.get("RANK", "0"))
@@ -568,6 +706,7 @@ def main():
     ap.add_argument("--chunk", action="store_true", help="time only the observation-chunk half of --config (for profiling)")
     ap.add_argument("--shrink", type=int, default=1, help="with --chunk: divide context lengths by this (small profiling case)")
     ap.add_argument("--fp8", action="store_true", help="time only the fp8-pool decode step of --config (for profiling)")
+    ap.add_argument("--handoff", action="store_true", help="KV hand-off between two workers (--gpus 2) or both roles on one GPU")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
@@ -589,6 +728,10 @@ def main():
         dist.init_process_group("nccl", device_id=device)
 
     spec = W.CONFIGS[args.config]
+    if args.handoff:
+        if world > 2:
+            raise SystemExit("--handoff runs on 1 or 2 GPUs")
+        return run_handoff(args, dist, rank, world, device)
     if args.chunk:
         if args.shrink > 1:
             spec = W.shrink(spec, max(2, spec.num_traj // args.shrink), args.shrink)
