@@ -75,7 +75,7 @@ constexpr int kOffXMl = kOffFatal + 8;                     // [stream][row]: (m,
 constexpr int kSmemUsed = kOffXMl + 2 * kRows * 8;
 constexpr int kSmemBytes = kSmemUsed + 1024;               // + slack for the 1024-byte alignment
 static_assert(kSmemBytes <= 227 * 1024, "one block must fit an SM");
-static_assert((kMaxItems + 1) * 4 <= kStages * kStageBytes, "the tile prefix is staged in the KV stages");
+static_assert((kMaxItems + 1) * 4 + kMaxItems * 16 <= kStages * kStageBytes, "the tile prefix and the item table are staged in the KV stages");
 static_assert(kStages % 2 == 0, "K tiles and V tiles alternate in the ring");
 
 constexpr int kTmemCols = 512;             // S buffer b at columns b * 128; stream w's P over the first 32 columns of its half (64 w ..) of the S buffer
@@ -146,14 +146,37 @@ chunk_attn_pair_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_co
     auto bar_odone = [&](int w, int b) { return bars + 8u * (2 + 3 * kStages + 6 + 2 * w + b); };
     const uint32_t peer_abort = map_to_cta(smem_u32(smem + kOffAbort), rank ^ 1u);
 
-    // ---- which (item, kv head, pair of M-tiles) is this cluster?  pairs per item -> prefix -> search ----
+    // ---- set-up that does not depend on the unit, first: it overlaps the loads of the item table below ----
+    // barriers (one per thread), Q zero fill (rows beyond tpt * g are never written by the copy), tensor memory
+    if (threadIdx.x < kNumBars) {
+        const int i = static_cast<int>(threadIdx.x);
+        uint32_t count = 1;                                                      // q_full, full, empty, s_full, o_done
+        if (i == 1 || (i >= 2 + 2 * kStages && i < 2 + 3 * kStages)) count = 2;  // q_ready, ready: one arrival per CTA
+        else if (i >= 2 + 3 * kStages + 2 && i < 2 + 3 * kStages + 6) count = 8; // p_full: 4 warps x 2 CTAs
+        mbar_init(bars + 8u * i, count);
+    }
+    if (threadIdx.x == 0) {
+        *s_abort = 0;
+        // an earlier block ran out of patience: the leader's reading of the flag decides for the pair
+        s_fatal[0] = *reinterpret_cast<volatile int *>(&prm.status->fatal) != 0 ? 1 : 0;
+    }
+    for (int i = threadIdx.x; i < kTileQ / 16; i += kThreads) reinterpret_cast<uint4 *>(smem + kOffQ)[i] = make_uint4(0, 0, 0, 0);
+    if (warp == 0) tmem_alloc_pair(smem_u32(smem + kOffTmemSlot), kTmemCols);
+
+    // ---- which (item, kv head, pair of M-tiles) is this cluster?  pairs per item -> prefix -> search.  The same pass
+    //      keeps every item's rows, trajectory and length in shared memory, so that the unit's geometry below needs no
+    //      further (dependent) global loads ----
+    int *s_item = s_prefix + (kMaxItems + 1);             // [item][4]: first row, rows, trajectory, length (-1: invalid trajectory)
     for (int i = threadIdx.x; i < prm.n_items; i += kThreads) {
-        const int n = __ldg(prm.q_indptr + i + 1) - __ldg(prm.q_indptr + i);
+        const int q0 = __ldg(prm.q_indptr + i), n = __ldg(prm.q_indptr + i + 1) - q0;
+        const int t = prm.traj_ids ? __ldg(prm.traj_ids + i) : i + prm.item_offset;
+        s_item[4 * i] = q0; s_item[4 * i + 1] = n; s_item[4 * i + 2] = t;
+        s_item[4 * i + 3] = (t >= 0 && t < prm.num_traj) ? __ldg(prm.seq_lens + t) : -1;
         s_prefix[i + 1] = n > 0 ? (n + 2 * tpt - 1) / (2 * tpt) : 0;
     }
     if (threadIdx.x == 0) s_prefix[0] = 0;
     __syncthreads();
-    if (warp == 0) {        // inclusive scan of the pair counts, in place
+    if (warp == 1) {        // inclusive scan of the pair counts, in place (warp 0 is allocating tensor memory)
         const int per = (prm.n_items + 31) / 32;
         const int a = min(prm.n_items, lane * per), b = min(prm.n_items, a + per);
         int sum = 0;
@@ -183,63 +206,40 @@ chunk_attn_pair_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_co
         head = rem / np;
         pair = np - 1 - (rem - head * np);      // later M-tiles see more keys: start the longest ones first
     }
-    __syncthreads();                 // everyone has read the prefix: the KV stages are free again
-    // Every exit before the pair's first common barrier depends on the unit alone, so both CTAs take it or neither.
-    if (unit >= total_units) return;
 
-    // ---- geometry of this unit ----
-    const int q_row0 = __ldg(prm.q_indptr + item);
-    const int n_chunk = __ldg(prm.q_indptr + item + 1) - q_row0;
-    const int t = prm.traj_ids ? __ldg(prm.traj_ids + item) : item + prm.item_offset;
-    int L = 0;
-    bool bad = false;
-    if (q_row0 < 0 || n_chunk < 0 || static_cast<long long>(q_row0) + n_chunk > prm.total_q) {
-        bad = true;                  // q_indptr does not describe rows of q
-        if (threadIdx.x == 0 && rank == 0) report(prm.status, ROLLART_ERR_BOUNDS, q_row0, 3);
-    } else if (t < 0 || t >= prm.num_traj) {
-        bad = true;
-        if (threadIdx.x == 0 && rank == 0) report(prm.status, ROLLART_ERR_BOUNDS, t, 3);
-    } else {
-        L = __ldg(prm.seq_lens + t);
-        if (L < 0 || L > prm.max_seq_len || n_chunk > L) {
-            bad = true;
-            if (threadIdx.x == 0 && rank == 0) report(prm.status, ROLLART_ERR_BOUNDS, L, 3);
+    // ---- geometry of this unit.  Whether the pair has work depends on the unit alone, so both CTAs decide alike ----
+    bool active = unit < total_units;
+    const int q_row0 = s_item[4 * item], n_chunk = s_item[4 * item + 1], t = s_item[4 * item + 2];
+    int L = s_item[4 * item + 3];
+    if (active) {
+        int bad_value = 0;
+        bool bad = false;
+        if (q_row0 < 0 || n_chunk < 0 || static_cast<long long>(q_row0) + n_chunk > prm.total_q) { bad = true; bad_value = q_row0; }   // q_indptr does not describe rows of q
+        else if (t < 0 || t >= prm.num_traj) { bad = true; bad_value = t; }
+        else if (L < 0 || L > prm.max_seq_len || n_chunk > L) { bad = true; bad_value = L; }
+        if (bad) {
+            if (threadIdx.x == 0 && rank == 0) report(prm.status, ROLLART_ERR_BOUNDS, bad_value, 3);
+            active = false;
         }
     }
-    if (bad) return;                 // the same in both CTAs, before any barrier or tensor-memory use
+    if (!active) L = 0;
     const int prior = L - n_chunk;
     const int first_tok = (2 * pair + static_cast<int>(rank)) * tpt;       // first chunk token of this CTA's M-tile
     const int toks = max(0, min(tpt, n_chunk - first_tok));                // its live tokens (the second CTA may have none)
     const int pair_toks_end = min(n_chunk, (2 * pair + 2) * tpt);          // one past the pair's last live token
     const int nmax = (prior + pair_toks_end + kKeys - 1) / kKeys;          // key tiles of the pair (>= 1)
     const int min_count = min(L, prior + first_tok + 1);                   // keys the CTA's first row sees
-    const int32_t *table_row = prm.page_table + static_cast<long long>(t) * prm.max_pages;
+    const int32_t *table_row = prm.page_table + static_cast<long long>(active ? t : 0) * prm.max_pages;
 
-    // ---- set-up: barriers, status exchange, Q zero fill, tensor memory ----
-    if (threadIdx.x == 0) {
-        mbar_init(bar_qfull, 1);
-        mbar_init(bar_qready, 2);
-        for (int s = 0; s < kStages; ++s) { mbar_init(bar_full(s), 1); mbar_init(bar_empty(s), 1); mbar_init(bar_ready(s), 2); }
-        for (int b = 0; b < 2; ++b) {
-            mbar_init(bar_sfull(b), 1);
-            for (int w = 0; w < 2; ++w) { mbar_init(bar_odone(w, b), 1); mbar_init(bar_pfull(w, b), 8); }   // 4 warps x 2 CTAs
-        }
-        *s_abort = 0;
-        // an earlier block ran out of patience: the leader's reading of the flag decides for the pair
-        s_fatal[0] = *reinterpret_cast<volatile int *>(&prm.status->fatal) != 0 ? 1 : 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
-    // rows beyond tpt * g are never written by the copy
-    for (int i = threadIdx.x; i < kTileQ / 16; i += kThreads) reinterpret_cast<uint4 *>(smem + kOffQ)[i] = make_uint4(0, 0, 0, 0);
-    fence_proxy_async();
-    if (warp == 0) tmem_alloc_pair(smem_u32(smem + kOffTmemSlot), kTmemCols);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    fence_proxy_async();             // the zeroed Q rows are ordered before the copy that lands beside them
     tc_fence_before();
-    __syncthreads();
+    __syncthreads();                 // everyone has read the tables: the KV stages are free again
     cluster_sync_all();              // both CTAs' barriers exist before anything arrives on them
     tc_fence_after();
     const uint32_t tmem = *s_tmem;
     // (the leader stays resident until the pair's last common barrier, so its shared memory may be read here)
-    const bool run = ld_cluster_u32(map_to_cta(smem_u32(smem + kOffFatal), 0)) == 0u;
+    const bool run = active && ld_cluster_u32(map_to_cta(smem_u32(smem + kOffFatal), 0)) == 0u;
 
     if (!run) {
         // fall through to the common exit
