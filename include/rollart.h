@@ -433,6 +433,16 @@ rollart_status rollart_decode_attn_noalloc(int device, const rollart_kv_pool *po
                                            int32_t num_q_heads, float sm_scale, void *out, float *lse,
                                            int32_t *device_status, void *stream, char *err_buf, size_t err_len);
 
+/*
+ * Diagnostic of the bounded waits (no counterpart in the paper).  Every in-kernel wait of this library (on a copy, on
+ * the tensor core, on another role of the block) polls with a limit of about a second; when the limit runs out the
+ * kernel records ROLLART_ERR_TIMEOUT, stops waiting and runs to its end, so a fault elsewhere cannot hang the GPU.
+ * This call enqueues one thread block whose only thread waits, with that same bounded wait, on a barrier nothing
+ * arrives at: it returns after about a second of GPU time and the next rollart_check returns ROLLART_ERR_TIMEOUT
+ * (and clears it); the context is usable afterwards.  For health checks and for testing the error path.
+ */
+rollart_status rollart_selftest_bounded_wait(rollart_ctx *ctx, void *stream);
+
 /* Synchronises `stream`, then returns and clears the device status word: ROLLART_OK, or the
  * first device-side error recorded since the last check (ROLLART_ERR_BOUNDS / _TIMEOUT), or
  * ROLLART_ERR_CUDA if the stream itself reports an error. */

@@ -603,6 +603,19 @@ chunk_attn_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constan
     }
 }
 
+// Diagnostic: one thread waits, with the bounded wait every role of the tensor-core kernels uses, on a barrier that
+// nothing arrives at.  The wait gives up when its limit (about a second) runs out and records ROLLART_ERR_TIMEOUT.
+__global__ void bounded_wait_selftest_kernel(DeviceStatus *status) {
+    __shared__ uint64_t bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        mbar_init(smem_u32(&bar), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        mbar_wait(smem_u32(&bar), 0, &abort_flag, status, 15);
+    }
+}
+
 }  // namespace
 
 cudaError_t launch_chunk_attn(const AttnCall &c, cudaStream_t stream, int64_t *launches, bool *too_small) {
@@ -641,6 +654,12 @@ cudaError_t launch_chunk_attn(const AttnCall &c, cudaStream_t stream, int64_t *l
         if (e != cudaSuccess) return e;
     }
     return cudaSuccess;
+}
+
+cudaError_t launch_bounded_wait_selftest(DeviceStatus *status, cudaStream_t stream, int64_t *launches) {
+    bounded_wait_selftest_kernel<<<1, 32, 0, stream>>>(status);
+    ++*launches;
+    return cudaGetLastError();
 }
 
 }  // namespace rollart

@@ -713,6 +713,15 @@ rollart_status rollart_obs_chunk_attn_fp8(rollart_ctx *ctx, const rollart_kv_poo
     return ROLLART_OK;
 }
 
+rollart_status rollart_selftest_bounded_wait(rollart_ctx *ctx, void *stream) {
+    if (!ctx) return ROLLART_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return fail(ctx, ROLLART_ERR_CUDA, "cannot select device %d", ctx->device);
+    cudaError_t e = launch_bounded_wait_selftest(ctx->d_status, static_cast<cudaStream_t>(stream), &ctx->launches);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "bounded-wait self-test launch");
+    return ROLLART_OK;
+}
+
 rollart_status rollart_check(rollart_ctx *ctx, void *stream) {
     if (!ctx) return ROLLART_ERR_INVALID_ARG;
     DeviceGuard guard(ctx->device);

@@ -125,6 +125,8 @@ cudaError_t launch_decode_attn(const AttnCall &c, cudaStream_t stream, int64_t *
 // zeroes the bookkeeping at the head of the workspace after a device-side error
 cudaError_t decode_reset_workspace(void *workspace, size_t bytes, cudaStream_t stream);
 cudaError_t launch_chunk_attn(const AttnCall &c, cudaStream_t stream, int64_t *launches, bool *too_small);
+// diagnostic: a bounded in-kernel wait that must run out (see rollart_selftest_bounded_wait)
+cudaError_t launch_bounded_wait_selftest(DeviceStatus *status, cudaStream_t stream, int64_t *launches);
 // the causal chunk call on CTA pairs (no shared-prefix mode, bf16 output): what launch_chunk_attn runs for such calls
 cudaError_t launch_chunk_attn_pair(const AttnCall &c, cudaStream_t stream, int64_t *launches);
 

@@ -27,7 +27,7 @@ EXPORTS = (
     "rollart_kv_gather_fp8", "rollart_kv_append_fp8_codes", "rollart_obs_chunk_attn_fp8",
     "rollart_obs_chunk_fp8_scratch_size", "rollart_group_decode_attn_fp8",
     "rollart_obs_chunk_fp8_scratch_size_for_pages", "rollart_append_decode_attn_host", "rollart_host_staging_size",
-    "rollart_pages_evict_stale",
+    "rollart_pages_evict_stale", "rollart_selftest_bounded_wait",
 )
 
 
@@ -123,6 +123,8 @@ def load_library() -> ctypes.CDLL:
                                               vp, i32, f32, vp, vp, vp, vp, ctypes.c_char_p, ctypes.c_size_t]
     L.rollart_check.restype = ctypes.c_int
     L.rollart_check.argtypes = [vp, vp]
+    L.rollart_selftest_bounded_wait.restype = ctypes.c_int
+    L.rollart_selftest_bounded_wait.argtypes = [vp, vp]
     L.rollart_last_error.restype = ctypes.c_char_p
     L.rollart_last_error.argtypes = [vp]
     L.rollart_launch_count.restype = i64
@@ -621,6 +623,13 @@ class Context:
             _ptr(q, torch.bfloat16, self.device), hq, float(sm_scale), float(k_scale), float(v_scale),
             _ptr(out, torch.bfloat16, self.device), _ptr(lse, torch.float32, self.device),
             _ptr(scratch, torch.uint8, self.device), scratch.numel(), self._stream(stream))
+        if st != OK:
+            self._raise(st)
+
+    def selftest_bounded_wait(self, stream=None) -> None:
+        """rollart_selftest_bounded_wait: enqueues a wait that must run out (about a second); the next status() / check()
+        reports ERR_TIMEOUT."""
+        st = self._lib.rollart_selftest_bounded_wait(self._h, self._stream(stream))
         if st != OK:
             self._raise(st)
 

@@ -198,3 +198,30 @@ def test_append_and_chunk_attention_replayed_from_a_cuda_graph(cuda_device):
     assert torch.equal(db2.k_pool.view(torch.int16), db.k_pool.view(torch.int16))
     assert torch.equal(lens_after, db.lens_after)
     ctx.close()
+
+
+def test_a_wait_that_runs_out_is_reported_and_the_context_stays_usable(cuda_device):
+    # The bounded wait of the tensor-core kernels on a barrier nothing arrives at: it gives up after about a second, the
+    # status word carries ERR_TIMEOUT, and afterwards the same context computes a chunk call correctly.
+    batch = W.make_batch(W.shrink(W.CONFIGS[4], 4, 32, 16), seed=48)
+    spec = batch.spec
+    ids = batch.chunk_ids
+    rows, q_indptr = batch.chunk_rows()
+    msl = int(batch.seq_lens_after.max())
+    ctx = make_ctx(spec, len(ids), msl)
+    ctx.selftest_bounded_wait()
+    assert ctx.status() == rollart.ERR_TIMEOUT
+    assert "wait" in ctx.last_error()
+    assert ctx.status() == rollart.OK
+    db = DeviceBatch(batch, cuda_device)
+    db.append(ctx)
+    q = db.q_new[torch.from_numpy(rows).to(cuda_device)].contiguous()
+    out = torch.full_like(q, float("nan"))
+    ctx.obs_chunk_attn(db.k_pool, db.v_pool, db.page_table, db.lens_after, dev_i32(q_indptr, cuda_device), q, spec.sm_scale,
+                       msl, out, traj_ids=dev_i32(ids, cuda_device))
+    ctx.check()
+    kp, vp, after = oracle_append(batch)
+    ref_o, _ = oracle.obs_chunk_attn(kp, vp, batch.page_table, after, q_indptr, W.bf16_to_u16(batch.q_new[rows]), spec.sm_scale,
+                                     traj_ids=ids)
+    assert_attn_close(out, ref_o, "chunk call after a reported timeout")
+    ctx.close()
