@@ -1,4 +1,8 @@
-// Observation-chunk attention on the 5th-generation tensor cores (tcgen05 + TMEM).
+// Chunk attention on the 5th-generation tensor cores (tcgen05 + TMEM), one thread block per unit.
+//
+// This is the kernel behind the shared-prefix pass of the group decode call (every row of an item sees exactly the
+// item's first shared_lens keys, no causal mask, fp32 result + lse); plain causal chunks go to the CTA-pair kernel
+// (chunk_attn_pair.cu) through launch_chunk_attn below.  The kernel itself handles both modes.
 //
 // Work unit: (item, kv head, pair of M-tiles).  An M-tile is 128 query rows = floor(128 / g)
 // consecutive chunk tokens x the g query heads that share the kv head, so one K/V read serves all
