@@ -225,3 +225,66 @@ def test_a_wait_that_runs_out_is_reported_and_the_context_stays_usable(cuda_devi
                                      traj_ids=ids)
     assert_attn_close(out, ref_o, "chunk call after a reported timeout")
     ctx.close()
+
+
+def _custom_chunk_batch(P, hq, hkv, prior, n_new, seed, name):
+    spec = dataclasses.replace(W.CONFIGS[4], page_size=P, num_traj=len(prior), num_q_heads=hq, num_kv_heads=hkv, name=name)
+    batch = W.make_layout(spec, seed=seed)
+    batch.seq_lens_before = np.array(prior, np.int32)
+    batch.n_new = np.array(n_new, np.int32)
+    batch.is_chunk[:] = True
+    batch.new_indptr = np.concatenate([[0], np.cumsum(batch.n_new)]).astype(np.int32)
+    pages = (batch.seq_lens_before + batch.n_new + P - 1) // P
+    batch.page_table, batch.num_pages = W.build_page_table(pages.astype(np.int64), 0.3, np.random.default_rng(seed + 1))
+    W.fill_tensors(batch)
+    return batch
+
+
+@pytest.mark.parametrize("P,hq,hkv", [(16, 4, 4), (16, 8, 4), (32, 10, 2), (16, 12, 2), (64, 8, 1), (32, 24, 2), (16, 32, 2)])
+def test_chunk_lengths_around_the_tiles_of_the_pair_kernel(cuda_device, P, hq, hkv):
+    # Group sizes 1, 2, 5, 6, 8, 12, 16 (128 / g tokens per M-tile, with and without padding rows).  Contexts that end
+    # just before, on and just after the 128-key tiles and their 64-key halves (the two key streams of a tile), chunks of
+    # one M-tile or less (the second CTA of the pair has no row), exactly one and exactly two M-tiles, and one token more.
+    g = hq // hkv
+    tpt = 128 // g
+    prior = [0, 0, 63, 64, 65, 127, 128, 129, 191, 192, 200, 255, 256 + 64, 0, 1]
+    n_new = [1, tpt, 1, tpt - 1 if tpt > 1 else 1, tpt + 1, 2 * tpt, 2 * tpt + 1, 3, 1, 2 * tpt - 1 if tpt > 1 else 1, 5 * tpt + 2, 1,
+             tpt, 128 + 3, 127]
+    batch = _custom_chunk_batch(P, hq, hkv, prior, n_new, 21, f"pair_edges_{P}_{hq}_{hkv}")
+    run_chunk_case(batch, cuda_device)
+
+
+def test_chunk_rerun_is_bit_identical(cuda_device):
+    # units are independent and every unit adds its tiles and merges its two key streams in a fixed order
+    batch = W.make_batch(W.shrink(W.CONFIGS[4], 8, 16, 8), seed=49)
+    db, ctx, out, _ = run_chunk_case(batch, cuda_device)
+    spec = batch.spec
+    ids = batch.chunk_ids
+    rows, q_indptr = batch.chunk_rows()
+    msl = int(batch.seq_lens_after.max())
+    q = db.q_new[torch.from_numpy(rows).to(cuda_device)].contiguous()
+    for _ in range(3):
+        again = torch.full_like(q, float("nan"))
+        lse = torch.full((q.shape[0], spec.num_q_heads), float("nan"), device=cuda_device)
+        ctx.obs_chunk_attn(db.k_pool, db.v_pool, db.page_table, db.lens_after, dev_i32(q_indptr, cuda_device), q, spec.sm_scale,
+                           msl, again, lse=lse, traj_ids=dev_i32(ids, cuda_device))
+        ctx.check()
+        assert torch.equal(again.view(torch.int16), out.view(torch.int16))
+    ctx.close()
+
+
+def test_chunk_with_one_stream_towering_over_the_other(cuda_device):
+    # The two halves of every 128-key tile are separate softmax streams merged at the end.  Here the keys of one half are
+    # scaled up (scores far above the other half's, by tile parity and by half), so the streams' reference maxima sit
+    # far apart and the final merge has to weigh one stream down to nothing, or both equally, row by row.
+    P = 16
+    prior = [640, 500, 128]
+    n_new = [70, 33, 130]
+    batch = _custom_chunk_batch(P, 8, 2, prior, n_new, 31, "pair_streams")
+    for t, L in enumerate(prior):
+        for pos in range(L):
+            half, tile = (pos // 64) & 1, pos // 128
+            gain = 40.0 if (half == (tile & 1) and t != 1) or (t == 1 and half == 1) else 1.0
+            pg = int(batch.page_table[t, pos // P])
+            batch.k_pool[pg, :, pos % P, :] = (batch.k_pool[pg, :, pos % P, :].float() * gain).to(torch.bfloat16)
+    run_chunk_case(batch, cuda_device)
