@@ -34,6 +34,7 @@
 // Every wait is a bounded mbarrier poll; a pair in which any wait ran out tells both CTAs and runs to its end.
 #include <cuda.h>
 
+#include <climits>
 #include <type_traits>
 
 #include "rollart_internal.cuh"
@@ -423,8 +424,10 @@ chunk_attn_pair_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_co
             const int live_keys = count - key0 - wg * kCols;    // of this thread's 64 columns, those the row sees
             float rs[4];
             // two copies of the pass, chosen once per tile: the unmasked one carries no compare / select per element
-            auto exp_pass = [&](auto masked_tag, float neg_m) {
+            int poly_top = INT_MIN;     // the largest argument handed to the FMA-pipe exponential (see ex2_poly2)
+            auto exp_pass = [&](auto masked_tag, auto poly_tag, float neg_m) {
                 constexpr bool kMasked = decltype(masked_tag)::value;
+                constexpr bool kPoly = decltype(poly_tag)::value;
                 rs[0] = rs[1] = rs[2] = rs[3] = 0.f;
 #pragma unroll
                 for (int h = 0; h < 2; ++h) {
@@ -433,8 +436,8 @@ chunk_attn_pair_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_co
                     for (int c = 0; c < 32; c += 2) {
                         float x0, x1, p0, p1;
                         fma2(x0, x1, __uint_as_float(sraw[h][c]), __uint_as_float(sraw[h][c + 1]), scale, neg_m);
-                        if (((h * 16 + (c >> 1)) % kPolyOneIn) == kPolyOneIn - 1) {
-                            ex2_poly2(p0, p1, x0, x1);
+                        if (kPoly && ((h * 16 + (c >> 1)) % kPolyOneIn) == kPolyOneIn - 1) {
+                            ex2_poly2(p0, p1, x0, x1, poly_top);
                         } else {
                             p0 = ex2(x0);
                             p1 = ex2(x1);
@@ -459,8 +462,9 @@ chunk_attn_pair_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_co
             float rsum = 0.f, corr = 1.f;
             bool careful = j == 0 || need_mask;
             if (!careful) {
-                rsum = exp_pass(std::false_type{}, -m_ref);
-                careful = __any_sync(0xffffffffu, !(rsum <= kRowSumLimit));   // also true for inf / NaN
+                rsum = exp_pass(std::false_type{}, std::true_type{}, -m_ref);
+                // also true for inf / NaN, and for a score so far above the reference that the FMA-pipe exponential broke
+                careful = __any_sync(0xffffffffu, !(rsum <= kRowSumLimit) || poly_top > kPolyArgTop);
                 if (careful) tmem_wait_st();      // the stores of the abandoned pass land before the new ones
             }
             if (careful) {
@@ -520,7 +524,9 @@ chunk_attn_pair_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_co
                 }
                 m_ref = m_new;
                 // a stream that has not seen a key yet (m_ref = -inf) stores zeros through the masked pass
-                rsum = need_mask ? exp_pass(std::true_type{}, -m_ref) : exp_pass(std::false_type{}, -m_ref);
+                // (every exponential on the special-function unit here: the careful path has no bound on its arguments to rely on)
+                rsum = need_mask ? exp_pass(std::true_type{}, std::false_type{}, -m_ref)
+                                 : exp_pass(std::false_type{}, std::false_type{}, -m_ref);
             }
             l_sum = l_sum * corr + rsum;
             tmem_wait_st();

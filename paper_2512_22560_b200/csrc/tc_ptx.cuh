@@ -155,13 +155,19 @@ __device__ __forceinline__ void fma2v(float &d0, float &d1, float a0, float a1, 
         "fma.rn.f32x2 rd, ra, rb, rc;\n\tmov.b64 {%0, %1}, rd;\n\t}"
         : "=f"(d0), "=f"(d1) : "f"(a0), "f"(a1), "f"(b0), "f"(b1), "f"(c0), "f"(c1));
 }
-// 2^x for a pair of arguments x <= 8 on the FMA pipe.  x = n + f with n = round(x), read from the low mantissa bits
-// of x + 1.5 * 2^23; 2^f on [-0.5, 0.5] by a cubic (relative error 7.5e-5, far below the bf16 rounding of P); n is
-// then added to the exponent field.  Arguments below -126 give 2^-126.
-__device__ __forceinline__ void ex2_poly2(float &p0, float &p1, float x0, float x1) {
+// 2^x for a pair of arguments on the FMA pipe.  x = n + f with n = round(x), read from the low mantissa bits of
+// x + 1.5 * 2^23; 2^f on [-0.5, 0.5] by a cubic (relative error 7.5e-5, far below the bf16 rounding of P); n is then
+// added to the exponent field.  Arguments below -126 give 2^-126.  The result is only valid for arguments below 127
+// (beyond, n runs out of the exponent field) and is no NaN for a NaN argument, so the caller gets the means to tell:
+// `top` is raised to the largest argument seen, compared as a signed integer (any negative argument is below every
+// positive one; a NaN argument, which the clamp turns into the positive canonical NaN, is above every number).  A
+// caller that finds top > kPolyArgTop afterwards must redo these values with ex2().
+constexpr int kPolyArgTop = 0x42FC0000;     // 126.0f
+__device__ __forceinline__ void ex2_poly2(float &p0, float &p1, float x0, float x1, int &top) {
     constexpr float kMagic = 12582912.f;
-    x0 = fmaxf(x0, -126.f);
-    x1 = fmaxf(x1, -126.f);
+    asm("max.NaN.f32 %0, %1, %2;" : "=f"(x0) : "f"(x0), "f"(-126.f));
+    asm("max.NaN.f32 %0, %1, %2;" : "=f"(x1) : "f"(x1), "f"(-126.f));
+    top = __vimax3_s32(top, __float_as_int(x0), __float_as_int(x1));
     float t0, t1, n0, n1, f0, f1, q0, q1;
     fma2v(t0, t1, x0, x1, 1.f, 1.f, kMagic, kMagic);
     fma2v(n0, n1, t0, t1, 1.f, 1.f, -kMagic, -kMagic);

@@ -288,3 +288,72 @@ def test_chunk_with_one_stream_towering_over_the_other(cuda_device):
             pg = int(batch.page_table[t, pos // P])
             batch.k_pool[pg, :, pos % P, :] = (batch.k_pool[pg, :, pos % P, :].float() * gain).to(torch.bfloat16)
     run_chunk_case(batch, cuda_device)
+
+
+def _lone_key_batch(seed, name):
+    P = 16
+    prior = [700, 400, 420, 1000]
+    n_new = [100, 40, 70, 129]
+    batch = _custom_chunk_batch(P, 8, 2, prior, n_new, seed, name)
+    return batch.spec, batch, prior, P
+
+
+# positions inside a 128-key tile: both halves of the tile, first and second half of a thread's columns, odd and even
+_LONE_OFFSETS = (4, 5, 10, 29, 36, 37, 47, 68, 69, 100, 101, 125, 0, 63, 64, 127)
+
+
+def test_chunk_lone_key_towering_over_its_tile(cuda_device):
+    # One key per key tile whose score lies hundreds of log2 units above everything the row has seen, every other
+    # key of the tile far below, and the same for every row (so no neighbouring row raises the alarm for it):
+    # whichever unit takes that column's exponential (the special-function unit or the FMA pipe, whose range ends at
+    # 2^127) has to notice by itself.  The rows become one-hot on the last such key.
+    spec, batch, prior, P = _lone_key_batch(17, "chunk_lone_key")
+    batch.q_new[:, :, 0] = 4.0                                 # every query row has the same component along dim 0 ...
+    for t, L in enumerate(prior):
+        for tile in range(1, (L + 127) // 128):
+            pos = tile * 128 + _LONE_OFFSETS[(tile + 3 * t) % len(_LONE_OFFSETS)]
+            if pos >= L:
+                continue
+            x_log2 = (150.0, 200.0, 400.0, 700.0)[(t + tile) % 4] + 40.0 * tile      # rising: each one towers over the last
+            key = torch.zeros(128)
+            key[0] = x_log2 / (4.0 * spec.sm_scale * 1.4426950408889634)   # ... so this key scores x_log2 log2 units for all of them
+            pg = int(batch.page_table[t, pos // P])
+            batch.k_pool[pg, :, pos % P, :] = key.to(torch.bfloat16)
+    run_chunk_case(batch, cuda_device)
+
+
+def test_chunk_nan_key_reaches_every_row_that_sees_it(cuda_device):
+    # A NaN in one cached key: the rows that see the key are NaN (as the definition gives), wherever the key's
+    # column falls, and no other row is touched.
+    spec, batch, prior, P = _lone_key_batch(19, "chunk_nan_key")
+    ids = batch.chunk_ids
+    rows, q_indptr = batch.chunk_rows()
+    msl = int(batch.seq_lens_after.max())
+    W.poison_dead_slots(batch, batch.seq_lens_before)
+    kp, vp, after = oracle_append(batch)
+    ref_o, _ = oracle.obs_chunk_attn(kp, vp, batch.page_table, after, q_indptr, W.bf16_to_u16(batch.q_new[rows]),
+                                     spec.sm_scale, traj_ids=ids)
+    for trial, off in enumerate((4, 37, 68, 101, 0, 127)):
+        db = DeviceBatch(batch, cuda_device)
+        ctx = make_ctx(spec, len(ids), msl)
+        db.append(ctx)
+        nan_pos = {}
+        for t, L in enumerate(prior):
+            pos = 128 * (1 + (t + trial) % 2) + off
+            nan_pos[t] = pos
+            pg = int(batch.page_table[t, pos // P])
+            db.k_pool[pg, t % 2, pos % P, 7] = float("nan")
+        q = db.q_new[torch.from_numpy(rows).to(cuda_device)].contiguous()
+        out = torch.zeros_like(q)
+        ctx.obs_chunk_attn(db.k_pool, db.v_pool, db.page_table, db.lens_after, dev_i32(q_indptr, cuda_device), q,
+                           spec.sm_scale, msl, out, traj_ids=dev_i32(ids, cuda_device))
+        ctx.check()
+        got = out.float().cpu().numpy()
+        g = spec.num_q_heads // spec.num_kv_heads
+        for i, t in enumerate(ids):
+            a, b = int(q_indptr[i]), int(q_indptr[i + 1])
+            hit = slice((t % 2) * g, (t % 2) * g + g)          # the query heads of the kv head that holds the NaN
+            assert np.isnan(got[a:b, hit]).all(), (off, t)      # every chunk row sees the prior cache
+            other = slice((1 - t % 2) * g, (1 - t % 2) * g + g)
+            assert np.isfinite(got[a:b, other]).all(), (off, t)
+            assert np.allclose(got[a:b, other], ref_o[a:b, other], atol=1e-2, rtol=2e-2), (off, t)
