@@ -69,3 +69,38 @@ def test_random_groups(cuda_device, seed):
     fraction = float(rng.choice([0.0, 0.3, 0.75, 1.0]))
     run_group_case(spec, 50 + seed, group_size, fraction, cuda_device)
     run_fp8_group_case(spec, 50 + seed, group_size, fraction, cuda_device)
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_random_chunks_with_wild_scores(cuda_device, seed):
+    # The chunk half of a random batch with keys whose magnitudes are all over the place: a heavy-tailed gain per key,
+    # runs of 64 loud or quiet keys, and a few keys that score the same enormous value for every row (a constant
+    # component in the queries).  The moving reference max, its rescaling of the accumulator and the checks that guard
+    # both kinds of exponential all get exercised; the results are close to one-hot, so a wrong key would show.
+    import torch
+    batch = random_batch(100 + seed)
+    rng = np.random.default_rng(3000 + seed)
+    P = batch.spec.page_size
+    batch.q_new[:, :, 0] = 3.0
+    for t in range(batch.spec.num_traj):
+        L = int(batch.seq_lens_before[t])
+        if L == 0:
+            continue
+        gain = np.exp(rng.normal(0.0, 1.5, L))
+        for b0 in range(0, L, 64):
+            r = rng.random()
+            if r < 0.15:
+                gain[b0:b0 + 64] *= 30.0
+            elif r < 0.3:
+                gain[b0:b0 + 64] *= 0.01
+        lone = rng.choice(L, size=min(L, int(rng.integers(0, 4))), replace=False)
+        for pos in range(L):
+            pg = int(batch.page_table[t, pos // P])
+            if pos in lone:
+                key = torch.zeros(128)
+                key[0] = float(rng.choice([60.0, 150.0, 300.0, 900.0])) / (3.0 * batch.spec.sm_scale * 1.4426950408889634)
+                batch.k_pool[pg, :, pos % P, :] = key.to(torch.bfloat16)
+            else:
+                batch.k_pool[pg, :, pos % P, :] = (batch.k_pool[pg, :, pos % P, :].float() * float(min(gain[pos], 200.0))).to(torch.bfloat16)
+    _, ctx, _, _ = run_chunk_case(batch, cuda_device)
+    ctx.close()
