@@ -912,7 +912,7 @@ def main():
                     extra["cfg4_mixed_multiturn_chunk_half_fp8_pool"] = {
                         "chunk_attn_ms": t8, "bf16_chunk_attn_ms_sustained": att_sus_ms, "ratio_to_bf16": t8 / att_sus_ms,
                         "tflops": cw.flops / (t8 * 1e-3) / 1e12, "append_ms": a8, "scratch_bytes": need,
-                        "launches": 3, "note": "contexts expanded to bf16 into the scratch pool (pages packed by a plan kernel), then the bf16 kernel"}
+                        "launches": 4, "note": "contexts expanded to bf16 into the scratch pool (pages packed by a plan kernel), then the two bf16 kernels"}
                 except Exception as e:
                     extra["cfg4_mixed_multiturn_chunk_half_fp8_pool"] = {"error": repr(e)}
                 cw.ctx.close()

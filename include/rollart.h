@@ -349,6 +349,12 @@ rollart_status rollart_group_decode_attn_fp8(rollart_ctx *ctx, const rollart_kv_
  * chunk causally including itself.  Same formula, layout of q/out/lse ([total_q][...]) and
  * arithmetic as rollart_decode_attn; n_i = 1 is exactly a decode step.  n_i > L is a
  * ROLLART_ERR_BOUNDS device error for that item.
+ * Per 1024 items the call enqueues a 512-byte clear and two kernels: the first keeps, per query row, the largest
+ * score among the row's first 128 keys as the reference of its exponentials for the whole row; a block of rows in which
+ * some later score lies more than 64 powers of two above that reference (or is not finite) is marked in a bitmap that
+ * belongs to the context and is computed again by the second kernel, which moves its reference as it goes; the other
+ * blocks of the second kernel return at once.  Results do not depend on which kernel produced them beyond rounding.
+ * One chunk call per context may be in flight (the bitmap, like the status word, is the context's).
  */
 rollart_status rollart_obs_chunk_attn(rollart_ctx *ctx, const rollart_kv_pool *pool, const rollart_trajs *trajs,
                                       const int32_t *traj_ids, const int32_t *q_indptr, int32_t n_items,
@@ -373,7 +379,7 @@ rollart_status rollart_obs_chunk_attn(rollart_ctx *ctx, const rollart_kv_pool *p
  *                  nothing; one that turns out smaller than the contexts is a device-side ROLLART_ERR_WORKSPACE:
  *                  the items that do not fit are skipped (their rows of out are not written).
  *   other arguments, errors and arithmetic as for rollart_obs_chunk_attn (bf16 operands: here the exact code values).
- * Launches three kernels.  A code of NaN in a live slot gives NaN results for the rows that see it, as a bf16 NaN would.
+ * Launches four kernels (plan, expansion, and the two of rollart_obs_chunk_attn).  A code of NaN in a live slot gives NaN results for the rows that see it, as a bf16 NaN would.
  */
 size_t rollart_obs_chunk_fp8_scratch_size(int32_t n_items, int32_t num_kv_heads, int32_t page_size, int32_t max_seq_len);
 size_t rollart_obs_chunk_fp8_scratch_size_for_pages(int32_t n_items, int32_t num_kv_heads, int32_t page_size,

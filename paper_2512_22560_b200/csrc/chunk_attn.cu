@@ -89,6 +89,7 @@ struct ChunkParams {
     const int32_t *shared_lens;
     float *out_f32;             // when set, result rows go here in fp32 instead of bf16 to `out`
     const int32_t *item_order;  // NULL, or a permutation of the launch's items: blocks take the items in this order
+    const uint32_t *redo_bits;  // NULL, or kChunkRedoBits bits: only the units marked there (unit mod kChunkRedoBits) are computed
     DeviceStatus *status;
 };
 
@@ -100,6 +101,12 @@ using namespace tc;      // the PTX wrappers and descriptors
 __global__ void __launch_bounds__(kThreads, 1)
 chunk_attn_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant__ CUtensorMap kmap,
                   const __grid_constant__ CUtensorMap vmap, const ChunkParams prm) {
+    // Second pass behind the CTA-pair kernel: only the units it marked (rows that outgrew their fixed reference max)
+    // are computed here, with the same unit numbering; every other block leaves at once.
+    if (prm.redo_bits != nullptr) {
+        const unsigned u = blockIdx.x;
+        if (((__ldg(prm.redo_bits + ((u % kChunkRedoBits) >> 5)) >> (u & 31)) & 1u) == 0u) return;
+    }
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -630,9 +637,13 @@ __global__ void bounded_wait_selftest_kernel(DeviceStatus *status) {
 
 cudaError_t launch_chunk_attn(const AttnCall &c, cudaStream_t stream, int64_t *launches, bool *too_small) {
     (void)too_small;
-    // plain causal chunks run on CTA pairs (chunk_attn_pair.cu); this kernel keeps the shared-prefix mode of the group
-    // decode call (one M-tile per group: a pair would idle its second CTA, and that pass is bound by memory)
-    if (c.shared_lens == nullptr && c.out_f32 == nullptr && c.item_order == nullptr) return launch_chunk_attn_pair(c, stream, launches);
+    // Plain causal chunks run on CTA pairs (chunk_attn_pair.cu), whose rows keep the reference max of their first key
+    // tile; the units in which a row outgrew it are marked in a bitmap and computed again here, by the kernel that
+    // moves its reference max (a launch whose other blocks leave at once).  This kernel also keeps the shared-prefix
+    // mode of the group decode call (one M-tile per group: a pair would idle its second CTA, and that pass is bound by
+    // memory).
+    const bool plain = c.shared_lens == nullptr && c.out_f32 == nullptr && c.item_order == nullptr;
+    if (plain && c.redo_bits == nullptr) return cudaErrorInvalidValue;
     const int hkv = c.pool.num_kv_heads, g = c.num_q_heads / hkv, tpt = kRows / g;
     cudaError_t e = cudaFuncSetAttribute(chunk_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (e != cudaSuccess) return e;
@@ -643,6 +654,12 @@ cudaError_t launch_chunk_attn(const AttnCall &c, cudaStream_t stream, int64_t *l
         return cudaErrorInvalidValue;
     for (int base = 0; base < c.n_items; base += kMaxItems) {
         const int n = c.n_items - base < kMaxItems ? c.n_items - base : kMaxItems;
+        if (plain) {
+            e = cudaMemsetAsync(c.redo_bits, 0, kChunkRedoBits / 8, stream);
+            if (e != cudaSuccess) return e;
+            e = launch_chunk_attn_pair(c, base, n, stream, launches);
+            if (e != cudaSuccess) return e;
+        }
         ChunkParams prm;
         prm.page_table = c.trajs.page_table; prm.seq_lens = c.trajs.seq_lens;
         prm.traj_ids = c.traj_ids ? c.traj_ids + base : nullptr;
@@ -654,6 +671,7 @@ cudaError_t launch_chunk_attn(const AttnCall &c, cudaStream_t stream, int64_t *l
         prm.shared_lens = c.shared_lens ? c.shared_lens + base : nullptr;
         prm.out_f32 = c.out_f32;
         prm.item_order = c.item_order ? c.item_order + base : nullptr;
+        prm.redo_bits = plain ? c.redo_bits : nullptr;
         // an upper bound on the M-tile pairs of these items: every item has at most one ragged pair
         const long long pairs = (static_cast<long long>(c.total_q) + 2 * tpt - 1) / (2 * tpt) + n;
         const long long blocks = pairs * hkv;

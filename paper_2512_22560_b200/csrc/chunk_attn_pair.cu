@@ -7,34 +7,43 @@
 //   S = Q K^T      one MMA of M 256 x N 128 x K 128 for the pair.  Each CTA supplies its own 128 rows of Q and HALF of
 //                  the tile's keys (64) from its own shared memory and receives its 128 x 128 scores in its own tensor
 //                  memory: per MMA step an SM reads 4 KB of Q and 2 KB of K for 64 cycles of math, where one CTA
-//                  alone with 64-key tiles read 6 KB per 32 cycles and was held by its shared-memory port.  Two S
-//                  buffers, so S(j+1) is computed while the softmax of tile j runs.
-//   softmax        two warpgroups per CTA, each with its own KEY STREAM: warpgroup w takes keys 64 w .. 64 w + 63 of
-//                  every tile, one thread per query row: tcgen05.ld its 64 scores, P = exp2(scale * s - m) as packed
-//                  bf16 stored back over the start of its half of the S buffer, row sum.  A stream has its own
-//                  reference max, row sum and O accumulator, so the two warps that share a row (they sit on the same
-//                  SM sub-partition: tensor-memory lanes are tied to warp % 4) never exchange anything while the keys
-//                  stream by; the two streams are merged once, at the end.  After a stream's first tile m is not
-//                  recomputed per tile: the exponentials are taken against the current reference max, and only a row
-//                  sum that explodes (or a masked tile) sends the tile down the careful path (row max, new reference,
-//                  the stream's O rescaled in tensor memory).  One pair of exponentials in kPolyOneIn is evaluated
-//                  on the FMA pipe.
-//   O_w += P_w V   per stream an MMA of M 256 x N 128 x K 64 with the A operand (P) in tensor memory; each CTA supplies
-//                  HALF of V's dims (64) for the keys, straight from the [key][dim] page layout (MN-major B).
+//                  alone with 64-key tiles read 6 KB per 32 cycles and was held by its shared-memory port.  THREE S
+//                  buffers: S(j+3) is issued right behind PV(j), so the chain "P(j) stored -> PV(j) -> S of the tile
+//                  that reuses the buffer -> its softmax" spans three tiles and its signalling latencies stay off the
+//                  critical path (with two buffers they were a quarter of a tile's time).
+//   softmax        two warpgroups per CTA that take the key tiles in turn (warpgroup w the tiles j = w mod 2), one
+//                  thread per query row with all 128 scores of the row: tcgen05.ld in four quarters of 32 columns,
+//                  each load in flight behind the arithmetic of the quarter before; P = exp2(scale * s - m) as packed
+//                  bf16 stored back over the start of the S buffer; row sum.  The two warps of an SM sub-partition work
+//                  on different tiles, so each one's waits fall into the other's arithmetic, and the fixed cost of a
+//                  tile (barrier, fences, hand-over) is paid once per 128 columns.
+//                  The reference m of a row is fixed after the first tile (the max of the row's visible scores there;
+//                  every row sees key 0) and never moves: P and the sums of a row whose later scores are larger just
+//                  carry a larger exponent, which fp32 accumulation and bf16's 8-bit mantissa do not mind.  So there
+//                  is no rescaling of O, one O accumulator serves both warpgroups, and the freed tensor-memory columns
+//                  hold the third S buffer.  A row sum of a tile beyond 2^64 (scores more than ~44 nats above the
+//                  first tile's max, or inf / NaN), or an argument beyond the range of the FMA-pipe exponential,
+//                  marks the unit in a bitmap; marked units are computed again by the single-CTA kernel, which moves
+//                  its reference max, in a launch that follows this one (its other blocks return at once).
+//                  One pair of exponentials in kPolyOneIn is evaluated on the FMA pipe.
+//   O += P V       an MMA of M 256 x N 128 x K 128 with the A operand (P) in tensor memory; each CTA supplies HALF of
+//                  V's dims (64) for the keys, straight from the [key][dim] page layout (MN-major B).
 //
-// Roles per CTA (12 warps): warp 0 copies Q and the CTA's half of every K tile, warp 3 its half of every V tile (TMA,
-// one box per page; page ids fetched 32 at a time, a batch ahead); warp 2 waits for each landed tile, zeroes the V
-// rows of dead keys in the last tile and tells the leader that this CTA's half is ready; warp 1 of the leader (the
-// even CTA) issues every MMA (the whole warp walks the loop so that descriptors are warp-uniform values; one elected
-// lane issues); warps 4-7 and 8-11 are the softmax warpgroups, which also write the result.
+// Roles per CTA (16 warps).  Copies: a TMA copy costs the warp that issues it ~135 cycles whatever its size, and a
+// tile of 16-slot pages needs 12 of them per CTA (4 K pages with both 64-dim halves in one 4-D box, 8 V pages), so they
+// are spread: warps 0 and 15 copy the CTA's half of every K tile (warp 0 also Q), warps 3, 12, 13, 14 its half of
+// every V tile, each at least two pages of a tile (with larger pages fewer of them take part); page ids are fetched 32
+// at a time, a batch ahead.  Warp 2 waits for each landed tile, zeroes the V rows of dead keys in the last tile and
+// tells the leader that this CTA's half is ready; warp 1 of the leader (the even CTA) issues every MMA (the whole
+// warp walks the loop so that descriptors are warp-uniform values; one elected lane issues); warps 4-7 and 8-11 are
+// the softmax warpgroups, which also write the result.
 // Completion of MMAs reaches both CTAs through tcgen05.commit to the barriers of both; all other cross-CTA signals are
 // mbarrier arrivals at the leader.  No load is multicast: each CTA copies what it needs itself.
-// A CTA uses ~194 KB of shared memory (Q 32 KB, 10 K/V stages of 16 KB) and all 512 tensor-memory columns (two S
-// buffers of 128, two O accumulators of 128).
+// A CTA uses ~194 KB of shared memory (Q 32 KB, 6 K stages and 4 V stages of 16 KB) and all 512 tensor-memory columns
+// (three S buffers of 128, one O accumulator of 128).
 // Every wait is a bounded mbarrier poll; a pair in which any wait ran out tells both CTAs and runs to its end.
 #include <cuda.h>
 
-#include <climits>
 #include <type_traits>
 
 #include "rollart_internal.cuh"
@@ -50,37 +59,42 @@ constexpr int kRows = 128;                 // query rows of a CTA (the pair's MM
 constexpr int kKeys = 128;                 // keys per KV tile
 constexpr int kOwnKeys = kKeys / 2;        // keys of a K tile held by one CTA
 constexpr int kOwnDims = kHeadDim / 2;     // dims of a V tile held by one CTA
-constexpr int kStages = 10;                // ring of stages; K(j) and V(j) take alternate slots
-constexpr int kThreads = 384;
-constexpr int kCols = kKeys / 2;           // S columns (keys) of a tile per softmax thread: one key stream per warpgroup
+constexpr int kStagesK = 6;                // ring of K stages: K(j) in stage j % 6 (QK runs three tiles ahead of PV)
+constexpr int kStagesV = 4;                // ring of V stages: V(j) in stage 6 + j % 4
+constexpr int kStages = kStagesK + kStagesV;
+constexpr int kSBufs = 3;                  // S buffers in tensor memory
+constexpr int kSoftmaxGroups = 2;          // softmax warpgroups: group w takes the key tiles j = w (mod 2), whole
+constexpr int kVCopyWarps = 4;             // warps that may share the V copies of a tile (warp 3 and warps 12..14)
+constexpr int kKCopyWarps = 2;             // likewise for the K copies (warp 0 and warp 15)
+constexpr int kThreads = 128 + 128 * kSoftmaxGroups + 32 * (kVCopyWarps - 1) + 32 * (kKCopyWarps - 1);
 constexpr int kMaxItems = kChunkItemsPerLaunch;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
-constexpr float kRescaleThreshold = 8.f;   // log2 units
-constexpr float kRowSumLimit = 16777216.f; // 2^24: a half-row sum above this sends the tile down the careful path
+constexpr float kRowSumLimit = 18446744073709551616.f;   // 2^64: a half-row sum of one tile above this marks the unit for the careful kernel
 constexpr int kPolyOneIn = 3;              // one pair of exponentials in this many goes to the FMA pipe
 
 constexpr int kHalfQ = kRows * 128;        // 16 KB: 128 rows x 64 dims
 constexpr int kTileQ = 2 * kHalfQ;         // [dim half][row][128 B]
 constexpr int kHalfK = kOwnKeys * 128;     // 8 KB: 64 keys x 64 dims
-constexpr int kStageBytes = 2 * kHalfK;    // K: [dim half][key][128 B]; V: [key (128)][128 B = the CTA's 64 dims]
+constexpr int kStageBytes = 2 * kHalfK;    // K: [group of 8 keys][dim half][key in group][128 B]; V: [key (128)][128 B = the CTA's 64 dims]
 static_assert(kStageBytes == kKeys * kOwnDims * 2, "a V half tile fills a stage exactly");
 constexpr int kOffQ = 0;
 constexpr int kOffKV = kOffQ + kTileQ;
 constexpr int kOffBars = kOffKV + kStages * kStageBytes;
-constexpr int kNumBars = 2 + 3 * kStages + 10;  // q_full, q_ready | full, empty, ready per stage | s_full per S buffer | p_full, o_done per key stream and S buffer
+constexpr int kNumBars = 2 + 3 * kStages + 2 * kSBufs + 1;  // q_full, q_ready | full, empty, ready per stage | s_full, p_full per S buffer | o_done
 constexpr int kOffTmemSlot = kOffBars + kNumBars * 8;
 constexpr int kOffAbort = kOffTmemSlot + 8;
 constexpr int kOffFatal = kOffAbort + 8;                   // the leader's reading of the status word's fatal flag
-constexpr int kOffXMl = kOffFatal + 8;                     // [stream][row]: (m, l) of each key stream, for the final merge
-constexpr int kSmemUsed = kOffXMl + 2 * kRows * 8;
+constexpr int kOffXMl = kOffFatal + 8;                     // [row]: the row's reference max; then [warpgroup][row]: the row sums
+constexpr int kSmemUsed = kOffXMl + (1 + kSoftmaxGroups) * kRows * 4;
 constexpr int kSmemBytes = kSmemUsed + 1024;               // + slack for the 1024-byte alignment
 static_assert(kSmemBytes <= 227 * 1024, "one block must fit an SM");
+static_assert(kSoftmaxGroups < kSBufs, "a warpgroup finds the S of its next tile computed while it works on this one");
 static_assert((kMaxItems + 1) * 4 + kMaxItems * 16 <= kStages * kStageBytes, "the tile prefix and the item table are staged in the KV stages");
-static_assert(kStages % 2 == 0, "K tiles and V tiles alternate in the ring");
 
-constexpr int kTmemCols = 512;             // S buffer b at columns b * 128; stream w's P over the first 32 columns of its half (64 w ..) of the S buffer
-constexpr int kTmemO = 256;                // O of stream w at 256 + 128 w
+constexpr int kTmemCols = 512;             // S buffer b at columns b * 128; warpgroup w's P over the first 32 columns of its half (64 w ..) of the S buffer
+constexpr int kTmemO = kSBufs * kKeys;     // O at 384
+constexpr int kRedoBits = kChunkRedoBits;  // units of a launch are marked in a bitmap of this many bits (unit mod kRedoBits)
 
 struct PairParams {
     const int32_t *page_table;
@@ -93,6 +107,7 @@ struct PairParams {
     float *lse;
     float scale_log2;
     float out_scale;            // the result is multiplied by this (the value scale of an fp8 cache expanded to bf16; else 1)
+    uint32_t *redo_bits;        // kRedoBits bits, zero at launch: units whose rows outgrew the fixed reference max
     DeviceStatus *status;
 };
 
@@ -138,22 +153,28 @@ chunk_attn_pair_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_co
     }
     const uint32_t bars = smem_u32(smem + kOffBars);
     const uint32_t bar_qfull = bars, bar_qready = bars + 8u;
-    // ring slot r (K(j) is r = 2j, V(j) is r = 2j + 1) lives in stage r % kStages
+    // K(j) lives in stage j % kStagesK, V(j) in stage kStagesK + j % kStagesV; use u of a stage has parity u & 1
+    auto stage_of = [&](int kv, int j) { return kv == 0 ? j % kStagesK : kStagesK + j % kStagesV; };
+    auto use_of = [&](int kv, int j) { return kv == 0 ? j / kStagesK : j / kStagesV; };
     auto bar_full = [&](int s) { return bars + 8u * (2 + s); };                  // this CTA's copies have landed
     auto bar_empty = [&](int s) { return bars + 8u * (2 + kStages + s); };       // the MMAs that read the stage are done
     auto bar_ready = [&](int s) { return bars + 8u * (2 + 2 * kStages + s); };   // leader: both CTAs' halves are in place
     auto bar_sfull = [&](int b) { return bars + 8u * (2 + 3 * kStages + b); };
-    auto bar_pfull = [&](int w, int b) { return bars + 8u * (2 + 3 * kStages + 2 + 2 * w + b); };   // leader: stream w's P of both CTAs is stored
-    auto bar_odone = [&](int w, int b) { return bars + 8u * (2 + 3 * kStages + 6 + 2 * w + b); };
+    auto bar_pfull = [&](int b) { return bars + 8u * (2 + 3 * kStages + kSBufs + b); };   // leader: P of both CTAs is stored in S buffer b
+    const uint32_t bar_odone = bars + 8u * (2 + 3 * kStages + 2 * kSBufs);      // the last PV of the unit is done
     const uint32_t peer_abort = map_to_cta(smem_u32(smem + kOffAbort), rank ^ 1u);
 
     // ---- set-up that does not depend on the unit, first: it overlaps the loads of the item table below ----
     // barriers (one per thread), Q zero fill (rows beyond tpt * g are never written by the copy), tensor memory
+    const int v_warps = min(kVCopyWarps, max(1, kKeys / P / 2));   // V copy warps in use: at least two pages of a tile each
+    const int k_warps = min(kKCopyWarps, max(1, kOwnKeys / P / 2));
     if (threadIdx.x < kNumBars) {
         const int i = static_cast<int>(threadIdx.x);
         uint32_t count = 1;                                                      // q_full, full, empty, s_full, o_done
         if (i == 1 || (i >= 2 + 2 * kStages && i < 2 + 3 * kStages)) count = 2;  // q_ready, ready: one arrival per CTA
-        else if (i >= 2 + 3 * kStages + 2 && i < 2 + 3 * kStages + 6) count = 8; // p_full: 4 warps x 2 CTAs
+        else if (i >= 2 && i < 2 + kStagesK) count = k_warps;                    // full of a K stage, likewise
+        else if (i >= 2 + kStagesK && i < 2 + kStages) count = v_warps;          // full of a V stage: one arrival (with its bytes) per active V copy warp
+        else if (i >= 2 + 3 * kStages + kSBufs && i < 2 + 3 * kStages + 2 * kSBufs) count = 8;   // p_full: 4 warps x 2 CTAs
         mbar_init(bars + 8u * i, count);
     }
     if (threadIdx.x == 0) {
@@ -244,12 +265,16 @@ chunk_attn_pair_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_co
 
     if (!run) {
         // fall through to the common exit
-    } else if (warp == 0 || warp == 3) {
+    } else if (warp < 4 || warp >= 12) {
+      if (warp == 0 || warp == 3 || warp >= 12) {
         // =============================== copy warps ===============================
-        // Warp 0 brings Q and this CTA's 64 keys of every K tile (two boxes per page: 64 dims each); warp 3 brings its
-        // 64 dims of every V tile (one box per page).  Both use the [rows][128 dims] view of a pool.
-        const int kv = warp == 3 ? 1 : 0;
-        if (kv == 0 && lane == 0) {
+        // Warp 0 brings Q; warps 0 and 15 bring this CTA's 64 keys of every K tile (one box per page: its keys in
+        // groups of 8, both 64-dim halves of a group side by side); warps 3 and 12..14 bring its 64 dims of every V tile
+        // (one box per page, from the [rows][128 dims] view of the pool).  Each warp takes its share of a tile's pages.
+        const int kv = (warp == 0 || warp == 15) ? 0 : 1;
+        const int vpart = kv == 0 ? (warp == 15 ? 1 : 0) : (warp >= 12 ? warp - 11 : 0);   // which part of the tile's pages
+        const int parts = kv == 0 ? k_warps : v_warps;
+        if (warp == 0 && lane == 0) {
             if (toks > 0) {
                 mbar_arrive_expect_tx(bar_qfull, static_cast<uint32_t>(tpt * g) * kRowBytes);
                 const uint32_t dst = smem_u32(smem + kOffQ);
@@ -260,8 +285,9 @@ chunk_attn_pair_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_co
             }
         }
         const int pages_per_tile = kKeys / P;
-        const int my_pages = kv == 0 ? kOwnKeys / P : pages_per_tile;            // boxes this warp issues per tile
-        const int my_first = kv == 0 ? static_cast<int>(rank) * (kOwnKeys / P) : 0;
+        const int my_pages = (kv == 0 ? kOwnKeys / P : pages_per_tile) / parts;  // boxes this warp issues per tile
+        const int my_first = (kv == 0 ? static_cast<int>(rank) * (kOwnKeys / P) : 0) + vpart * my_pages;   // first page of the tile it takes
+        const int dst_first = vpart * my_pages;                                   // ... and where in the stage that page lands
         const int tiles_per_batch = 32 / pages_per_tile;
         const uint32_t box_bytes = static_cast<uint32_t>(P) * 128;                // P rows x 64 dims
         // Page ids are fetched 32 at a time, one per lane, and the next 32 are requested a whole batch ahead, so the
@@ -272,14 +298,14 @@ chunk_attn_pair_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_co
             if (lp * P < L && lp < prm.max_pages) {
                 pg = __ldg(table_row + lp);
                 if (pg < 0 || pg >= prm.num_pages) {
-                    if (kv == 1 && rank == 0) report(prm.status, ROLLART_ERR_BOUNDS, pg, 3);
+                    if (warp == 3 && rank == 0) report(prm.status, ROLLART_ERR_BOUNDS, pg, 3);
                     pg = -1;
                 }
             }
             return pg;
         };
         int ids_cur = load_ids(0), ids_next = load_ids(1);
-        for (int j = 0; j < nmax; ++j) {
+        for (int j = 0; j < (vpart < parts ? nmax : 0); ++j) {
             const int within = j % tiles_per_batch;
             if (j > 0 && within == 0) {
                 if (*s_abort) break;
@@ -289,22 +315,21 @@ chunk_attn_pair_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_co
             int pg = __shfl_sync(0xffffffffu, ids_cur, (within * pages_per_tile + my_first + lane) & 31);
             if (lane >= my_pages) pg = -1;
             const uint32_t nvalid = __popc(__ballot_sync(0xffffffffu, pg >= 0));
-            const int r = 2 * j + kv, stage = r % kStages;
-            pair_wait(bar_empty(stage), ((r / kStages) & 1) ^ 1, s_abort, peer_abort, prm.status, 1 + kv);
+            const int stage = stage_of(kv, j);
+            pair_wait(bar_empty(stage), (use_of(kv, j) & 1) ^ 1, s_abort, peer_abort, prm.status, 1 + kv);
             if (lane == 0) mbar_arrive_expect_tx(bar_full(stage), nvalid * (kv == 0 ? 2u : 1u) * box_bytes);
             __syncwarp();
             if (pg >= 0) {
-                const uint32_t dst = smem_u32(smem + kOffKV + stage * kStageBytes) + lane * box_bytes;
+                const uint32_t dst = smem_u32(smem + kOffKV + stage * kStageBytes) + (dst_first + lane) * (kv == 0 ? 2u : 1u) * box_bytes;
                 const int row = (pg * hkv + head) * P;
                 if (kv == 0) {
-                    tma_load_2d(dst, &kmap, bar_full(stage), 0, row);
-                    tma_load_2d(dst + kHalfK, &kmap, bar_full(stage), 64, row);
+                    tma_load_4d(dst, &kmap, bar_full(stage), 0, 0, 0, row >> 3);   // both halves: 2 box_bytes per page
                 } else {
                     tma_load_2d(dst, &vmap, bar_full(stage), kOwnDims * static_cast<int>(rank), row);
                 }
             }
         }
-    } else if (warp == 2) {
+      } else if (warp == 2) {
         // =============================== stage warp ===============================
         // Waits for this CTA's copies of each ring slot and tells the leader.  In the last V tile the rows of keys at or
         // beyond L (dead slots of the last page, pages that were never copied) are zeroed first: their P is exactly 0,
@@ -313,9 +338,9 @@ chunk_attn_pair_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_co
         pair_wait(bar_qfull, 0, s_abort, peer_abort, prm.status, 5);
         __syncwarp();
         if (lane == 0) mbar_arrive_cluster(leader_qready);
-        for (int r = 0; r < 2 * nmax; ++r) {
-            const int stage = r % kStages;
-            pair_wait(bar_full(stage), (r / kStages) & 1, s_abort, peer_abort, prm.status, 6 + (r & 1));
+        for (int r = 0; r < 2 * nmax; ++r) {       // K(0) V(0) K(1) V(1) ...: the order in which the copies were issued
+            const int stage = stage_of(r & 1, r >> 1);
+            pair_wait(bar_full(stage), use_of(r & 1, r >> 1) & 1, s_abort, peer_abort, prm.status, 6 + (r & 1));
             const int key0 = (r >> 1) * kKeys;
             if ((r & 1) && key0 + kKeys > L) {
                 const uint32_t v_addr = smem_u32(smem + kOffKV + stage * kStageBytes);
@@ -329,11 +354,11 @@ chunk_attn_pair_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_co
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(map_to_cta(bar_ready(stage), 0));
         }
-    } else if (warp == 1) {
+      } else {
         // =============================== MMA warp (leader only) ===============================
-        // One thread issues QK(0) | QK(j+1) PV(j) | ...: S of the next key tile is ready before the softmax of this one
-        // ends.  MMAs run in issue order, which is what protects the reuse of an S buffer (it holds P(j-1) until
-        // PV(j-1), issued before QK(j+1), has read it).
+        // One thread issues QK(0) QK(1) QK(2) | PV(j) QK(j+3) | ...: three S buffers, so S of the next two key tiles
+        // is ready long before the softmax of this one ends.  MMAs run in issue order, which is what protects the
+        // reuse of an S buffer (it holds P(j) until PV(j), issued before QK(j+3), has read it).
         // The whole warp walks the loop (waits, descriptor arithmetic: warp-uniform values, which the compiler can keep
         // in uniform registers, where the MMA instruction takes its operands from); only the MMA and commit
         // instructions themselves are predicated on one elected lane.
@@ -344,236 +369,224 @@ chunk_attn_pair_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_co
             const uint32_t tm = __shfl_sync(0xffffffffu, tmem, 0);
             const uint32_t kv_addr = smem_u32(smem + kOffKV);
             const uint64_t q_desc = smem_desc(smem_u32(smem + kOffQ), 16);
-            auto ready_wait = [&](int r, int where) {
-                pair_wait(bar_ready(r % kStages), (r / kStages) & 1, s_abort, peer_abort, prm.status, where);
-            };
             auto issue_qk = [&](int j) {
-                ready_wait(2 * j, 8);                       // K(j), both halves
+                const int stage = stage_of(0, j);
+                pair_wait(bar_ready(stage), use_of(0, j) & 1, s_abort, peer_abort, prm.status, 8);   // K(j), both halves
                 tc_fence_after();
-                const uint64_t k_desc = smem_desc(kv_addr + ((2 * j) % kStages) * kStageBytes, 16);
-                const uint32_t s_tm = tm + (j & 1) * kKeys;
+                const uint64_t k_desc = smem_desc(kv_addr + stage * kStageBytes, 16, 2048);   // 8-key groups 2 KB apart
+                const uint32_t s_tm = tm + (j % kSBufs) * kKeys;
 #pragma unroll
                 for (int ks = 0; ks < kHeadDim / 16; ++ks) {   // 16 dims per step; the second 64 dims live in the other half
                     const uint64_t qoff = static_cast<uint64_t>(((ks >> 2) * kHalfQ + (ks & 3) * 32) >> 4);
-                    const uint64_t koff = static_cast<uint64_t>(((ks >> 2) * kHalfK + (ks & 3) * 32) >> 4);
+                    const uint64_t koff = static_cast<uint64_t>(((ks >> 2) * 1024 + (ks & 3) * 32) >> 4);
                     if (elected) umma_pair_bf16(s_tm, q_desc + qoff, k_desc + koff, kIdescQK, ks > 0 ? 1u : 0u);
                 }
                 if (elected) {
-                    umma_pair_commit(bar_sfull(j & 1));
-                    umma_pair_commit(bar_empty((2 * j) % kStages));
+                    umma_pair_commit(bar_sfull(j % kSBufs));
+                    umma_pair_commit(bar_empty(stage));
                 }
                 __syncwarp();
             };
             pair_wait(bar_qready, 0, s_abort, peer_abort, prm.status, 9);
-            issue_qk(0);
+            for (int j = 0; j < kSBufs && j < nmax; ++j) issue_qk(j);
             for (int j = 0; j < nmax; ++j) {
-                if (j + 1 < nmax) issue_qk(j + 1);
-                ready_wait(2 * j + 1, 10);                  // V(j), both halves
+                const int stage = stage_of(1, j), sb = j % kSBufs;
+                pair_wait(bar_ready(stage), use_of(1, j) & 1, s_abort, peer_abort, prm.status, 10);   // V(j), both halves
                 // V half tile is [key][128 B]: the 16 keys of step ks start 2 KB further on; 8-key groups are 1 KB apart
-                const uint64_t v_desc = smem_desc(kv_addr + ((2 * j + 1) % kStages) * kStageBytes, 1024);
-                const uint32_t p_tm = tm + (j & 1) * kKeys;
-                const uint32_t acc0 = j > 0 ? 1u : 0u;
+                const uint64_t v_desc = smem_desc(kv_addr + stage * kStageBytes, 1024);
+                const uint32_t p_tm = tm + sb * kKeys;
+                pair_wait(bar_pfull(sb), (j / kSBufs) & 1, s_abort, peer_abort, prm.status, 11);
+                tc_fence_after();
 #pragma unroll
-                for (int w = 0; w < 2; ++w) {               // the two key streams: keys 64 w .. 64 w + 63 of the tile into O_w
-                    pair_wait(bar_pfull(w, j & 1), (j >> 1) & 1, s_abort, peer_abort, prm.status, 11);
-                    tc_fence_after();
-#pragma unroll
-                    for (int ks = 0; ks < kCols / 16; ++ks)     // 16 keys per step: 8 packed columns of P's row
-                        if (elected)
-                            umma_pair_bf16_ts(tm + kTmemO + w * kHeadDim, p_tm + w * kCols + ks * 8,
-                                              v_desc + static_cast<uint64_t>(((w * kCols + ks * 16) * 128) >> 4), kIdescPV,
-                                              ks > 0 ? 1u : acc0);
-                    if (elected) {
-                        if (w == 1) umma_pair_commit(bar_empty((2 * j + 1) % kStages));
-                        umma_pair_commit(bar_odone(w, j & 1));
-                    }
-                    __syncwarp();
+                for (int ks = 0; ks < kKeys / 16; ++ks)       // 16 keys per step: 8 packed columns of P's row
+                    if (elected)
+                        umma_pair_bf16_ts(tm + kTmemO, p_tm + ks * 8, v_desc + static_cast<uint64_t>((ks * 16 * 128) >> 4), kIdescPV,
+                                          (j > 0 || ks > 0) ? 1u : 0u);
+                __syncwarp();
+                if (elected) {
+                    umma_pair_commit(bar_empty(stage));
+                    if (j == nmax - 1) umma_pair_commit(bar_odone);
                 }
+                __syncwarp();
+                if (j + kSBufs < nmax) issue_qk(j + kSBufs);
             }
         }
         __syncwarp();
+      }
     } else {
         // =============================== softmax warpgroups ===============================
-        // Warpgroup w owns key stream w: keys 64 w .. 64 w + 63 of every tile, with its own reference max, row sum and
-        // O accumulator, so the two warps that share a row never have to agree on anything while the keys stream by;
-        // the two streams are merged once, at the end.
+        // Warpgroup w takes the key tiles j = w, w + 2, ...: one thread per query row takes all 128 scores of the row.
+        // The two warps of an SM sub-partition work on different tiles, so each one's waits (for S, for tensor-memory
+        // loads and stores) fall into the arithmetic of the other.
         const int wg = (warp - 4) >> 2;
         const int quarter = warp & 3;                         // tensor-memory lanes 32 * quarter .. + 31 belong to this warp
         const int row = quarter * 32 + lane;
         const uint32_t lane_addr = tmem + (static_cast<uint32_t>(quarter * 32) << 16);
-        const uint32_t s_addr = lane_addr + wg * kCols, o_addr = lane_addr + kTmemO + wg * kHeadDim;
         const int tok_local = row / g, head_local = row - tok_local * g;
         const bool live = tok_local < toks;
         const int count = min(L, prior + first_tok + min(tok_local, max(toks, 1) - 1) + 1);   // keys this row sees (>= 1)
         const float scale = prm.scale_log2;
-        const uint32_t leader_pfull = map_to_cta(bar_pfull(wg, 0), 0);
-        float m_ref = -INFINITY, l_sum = 0.f;
+        const uint32_t leader_pfull = map_to_cta(bar_pfull(0), 0);
+        volatile float *x_m = reinterpret_cast<volatile float *>(smem + kOffXMl);   // [row]
+        volatile float *x_l = x_m + kRows;                                            // [warpgroup][row]
+        float l_sum = 0.f;
+        bool outgrown = false;
+        int poly_top = INT_MIN;             // the largest argument handed to the FMA-pipe exponential (see ex2_poly2)
+        uint32_t sa[32], sb[32];            // two quarters (32 columns each) of the row's scores
 
-        for (int j = 0; j < nmax; ++j) {
-            const int sb = j & 1;
-            const uint32_t sbuf = s_addr + sb * kKeys;
-            pair_wait(bar_sfull(sb), (j >> 1) & 1, s_abort, peer_abort, prm.status, 12);
+        // ---- the row's reference max: the largest visible score of the first tile (every row sees key 0) ----
+        if (wg == 0) {
+            pair_wait(bar_sfull(0), 0, s_abort, peer_abort, prm.status, 12);
             tc_fence_after();
-            uint32_t sraw[2][32];
-            tmem_ld32(sbuf, sraw[0]);
-            tmem_ld32(sbuf + 32, sraw[1]);
-            tmem_wait_ld();
-
-            const int key0 = j * kKeys;
-            const bool need_mask = key0 + kKeys > min_count;    // the same for every thread of the CTA
-            const int live_keys = count - key0 - wg * kCols;    // of this thread's 64 columns, those the row sees
-            float rs[4];
-            // two copies of the pass, chosen once per tile: the unmasked one carries no compare / select per element
-            int poly_top = INT_MIN;     // the largest argument handed to the FMA-pipe exponential (see ex2_poly2)
-            auto exp_pass = [&](auto masked_tag, auto poly_tag, float neg_m) {
-                constexpr bool kMasked = decltype(masked_tag)::value;
-                constexpr bool kPoly = decltype(poly_tag)::value;
-                rs[0] = rs[1] = rs[2] = rs[3] = 0.f;
-#pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    uint32_t packed[16];
-#pragma unroll
-                    for (int c = 0; c < 32; c += 2) {
-                        float x0, x1, p0, p1;
-                        fma2(x0, x1, __uint_as_float(sraw[h][c]), __uint_as_float(sraw[h][c + 1]), scale, neg_m);
-                        if (kPoly && ((h * 16 + (c >> 1)) % kPolyOneIn) == kPolyOneIn - 1) {
-                            ex2_poly2(p0, p1, x0, x1, poly_top);
-                        } else {
-                            p0 = ex2(x0);
-                            p1 = ex2(x1);
-                        }
-                        if constexpr (kMasked) {
-                            p0 = h * 32 + c < live_keys ? p0 : 0.f;
-                            p1 = h * 32 + c + 1 < live_keys ? p1 : 0.f;
-                        }
-                        add2(rs[c & 2], rs[(c & 2) + 1], p0, p1);
-                        packed[c >> 1] = pack_bf16(p0, p1);
-                    }
-                    // P as the next A operand: 32 keys of this row as 16 packed columns at the start of this stream's half of the S buffer
-                    tmem_st16(sbuf + h * 16, packed);
-                }
-                return (rs[0] + rs[1]) + (rs[2] + rs[3]);
-            };
-            // Fast path (every unmasked tile after the first): no max pass.  The exponentials are taken against the
-            // stream's reference max m_ref (the max of some earlier score, so later keys far below it rightly vanish);
-            // keys far above it make the row sum explode, and then (rarely) the tile is redone the careful way below.
-            // Up to that bound P and the sums just carry a larger exponent: fp32 accumulation and the 8-bit mantissa
-            // of bf16 P lose nothing by it.
-            float rsum = 0.f, corr = 1.f;
-            bool careful = j == 0 || need_mask;
-            if (!careful) {
-                rsum = exp_pass(std::false_type{}, std::true_type{}, -m_ref);
-                // also true for inf / NaN, and for a score so far above the reference that the FMA-pipe exponential broke
-                careful = __any_sync(0xffffffffu, !(rsum <= kRowSumLimit) || poly_top > kPolyArgTop);
-                if (careful) tmem_wait_st();      // the stores of the abandoned pass land before the new ones
-            }
-            if (careful) {
-                float rmax;
+            const bool need_mask = kKeys > min_count;
+            float rmax = -INFINITY;
+            auto quarter_max = [&](const uint32_t (&r)[32], int col0) {
                 if (!need_mask) {
-                    // the max of scale * s is scale * (max or min of s): the extreme of the raw scores, 8 chains of 3-input ops
-                    float e[8];
+                    // the max of scale * s is scale * (max or min of s): the extreme of the raw scores by 3-input ops
+                    float e[4];
                     if (scale >= 0.f) {
 #pragma unroll
-                        for (int k = 0; k < 8; ++k) e[k] = max3(__uint_as_float(sraw[0][k]), __uint_as_float(sraw[0][8 + k]), __uint_as_float(sraw[0][16 + k]));
+                        for (int k = 0; k < 4; ++k) e[k] = max3(__uint_as_float(r[k]), __uint_as_float(r[4 + k]), __uint_as_float(r[8 + k]));
 #pragma unroll
-                        for (int k = 0; k < 8; ++k) e[k] = max3(e[k], __uint_as_float(sraw[0][24 + k]), __uint_as_float(sraw[1][k]));
+                        for (int k = 0; k < 4; ++k) e[k] = max3(e[k], __uint_as_float(r[12 + k]), __uint_as_float(r[16 + k]));
 #pragma unroll
-                        for (int k = 0; k < 8; ++k) e[k] = max3(e[k], __uint_as_float(sraw[1][8 + k]), __uint_as_float(sraw[1][16 + k]));
+                        for (int k = 0; k < 4; ++k) e[k] = max3(e[k], __uint_as_float(r[20 + k]), __uint_as_float(r[24 + k]));
 #pragma unroll
-                        for (int k = 0; k < 8; ++k) e[k] = fmaxf(e[k], __uint_as_float(sraw[1][24 + k]));
-                        rmax = max3(max3(e[0], e[1], e[2]), max3(e[3], e[4], e[5]), fmaxf(e[6], e[7])) * scale;
+                        for (int k = 0; k < 4; ++k) e[k] = fmaxf(e[k], __uint_as_float(r[28 + k]));
+                        rmax = fmaxf(rmax, fmaxf(fmaxf(e[0], e[1]), fmaxf(e[2], e[3])) * scale);
                     } else {
 #pragma unroll
-                        for (int k = 0; k < 8; ++k) e[k] = min3(__uint_as_float(sraw[0][k]), __uint_as_float(sraw[0][8 + k]), __uint_as_float(sraw[0][16 + k]));
+                        for (int k = 0; k < 4; ++k) e[k] = min3(__uint_as_float(r[k]), __uint_as_float(r[4 + k]), __uint_as_float(r[8 + k]));
 #pragma unroll
-                        for (int k = 0; k < 8; ++k) e[k] = min3(e[k], __uint_as_float(sraw[0][24 + k]), __uint_as_float(sraw[1][k]));
+                        for (int k = 0; k < 4; ++k) e[k] = min3(e[k], __uint_as_float(r[12 + k]), __uint_as_float(r[16 + k]));
 #pragma unroll
-                        for (int k = 0; k < 8; ++k) e[k] = min3(e[k], __uint_as_float(sraw[1][8 + k]), __uint_as_float(sraw[1][16 + k]));
+                        for (int k = 0; k < 4; ++k) e[k] = min3(e[k], __uint_as_float(r[20 + k]), __uint_as_float(r[24 + k]));
 #pragma unroll
-                        for (int k = 0; k < 8; ++k) e[k] = fminf(e[k], __uint_as_float(sraw[1][24 + k]));
-                        rmax = min3(min3(e[0], e[1], e[2]), min3(e[3], e[4], e[5]), fminf(e[6], e[7])) * scale;
+                        for (int k = 0; k < 4; ++k) e[k] = fminf(e[k], __uint_as_float(r[28 + k]));
+                        rmax = fmaxf(rmax, fminf(fminf(e[0], e[1]), fminf(e[2], e[3])) * scale);
                     }
                 } else {
-                    // masked tile: keys the row does not see are left out (their scores may be anything); a row that sees
-                    // none of this stream's keys keeps rmax = -inf and stores P = 0
-                    rmax = -INFINITY;
+                    // masked tile: keys the row does not see are left out (their scores may be anything)
 #pragma unroll
-                    for (int h = 0; h < 2; ++h)
-#pragma unroll
-                        for (int c = 0; c < 32; ++c)
-                            if (h * 32 + c < live_keys) rmax = fmaxf(rmax, __uint_as_float(sraw[h][c]) * scale);
+                    for (int c = 0; c < 32; ++c)
+                        if (col0 + c < count) rmax = fmaxf(rmax, __uint_as_float(r[c]) * scale);
                 }
-                // the reference max moves only when it has to (first keys of the stream) or when a row outgrew it by 2^8
-                const bool grow = rmax > m_ref + kRescaleThreshold;
-                const float m_new = grow ? rmax : m_ref;
-                corr = grow ? ex2(m_ref - m_new) : 1.f;   // ex2(-inf) = 0 while the stream has seen nothing
-                if (j >= 1 && __any_sync(0xffffffffu, grow)) {
-                    // rare: some row of this warp moved its reference max, so this stream's O (the tiles before this
-                    // one) must be rescaled before PV of this tile; PV of the previous tile has to be finished first
-                    pair_wait(bar_odone(wg, (j - 1) & 1), ((j - 1) >> 1) & 1, s_abort, peer_abort, prm.status, 13);
-                    tc_fence_after();
-#pragma unroll 1
-                    for (int c0 = 0; c0 < kHeadDim; c0 += 16) {
-                        uint32_t oraw[16];
-                        tmem_ld16(o_addr + c0, oraw);
-                        tmem_wait_ld();
+            };
+            const uint32_t s_addr = lane_addr;                // tile 0 is in S buffer 0
+            tmem_ld32(s_addr, sa);
+            tmem_ld32(s_addr + 32, sb);
+            tmem_wait_ld_of(sa);
+            tmem_wait_ld_of(sb);
+            quarter_max(sa, 0);
+            quarter_max(sb, 32);
+            tmem_ld32(s_addr + 64, sa);
+            tmem_ld32(s_addr + 96, sb);
+            tmem_wait_ld_of(sa);
+            tmem_wait_ld_of(sb);
+            quarter_max(sa, 64);
+            quarter_max(sb, 96);
+            x_m[row] = rmax;
+            // (a reference of -inf, +inf or NaN, i.e. scores that are not finite, ends in a row sum that marks the unit)
+        }
+        named_bar_sync(1, 128 * kSoftmaxGroups);              // the other warpgroups take the reference from here
+        const float neg_m = -x_m[row];
+
+        for (int j = wg; j < nmax; j += kSoftmaxGroups) {
+            const int sbuf = j % kSBufs;
+            const uint32_t s_addr = lane_addr + sbuf * kKeys;
+            pair_wait(bar_sfull(sbuf), (j / kSBufs) & 1, s_abort, peer_abort, prm.status, 12);
+            tc_fence_after();
+            const int key0 = j * kKeys;
+            const bool need_mask = key0 + kKeys > min_count;    // the same for every thread of the CTA
+            const int live_keys = count - key0;                 // of this tile's 128 keys, those the row sees
+            float rs[4] = {0.f, 0.f, 0.f, 0.f};
+            // P = exp2(scale * s - m) for 32 keys of the row (quarter q of the tile), packed to bf16: 16 columns at
+            // the start of the S buffer, which the scores of quarter q have left by then.  Two copies of the pass,
+            // chosen once per tile: the unmasked one carries no compare / select.  One pair of exponentials in
+            // kPolyOneIn goes to the FMA pipe.
+            auto exp_pass = [&](auto masked_tag, auto q_tag, const uint32_t (&r)[32]) {
+                constexpr bool kMasked = decltype(masked_tag)::value;
+                constexpr int q = decltype(q_tag)::value;
+                uint32_t packed[16];
 #pragma unroll
-                        for (int c = 0; c < 16; ++c) oraw[c] = __float_as_uint(__uint_as_float(oraw[c]) * corr);
-                        tmem_st16(o_addr + c0, oraw);
+                for (int c = 0; c < 32; c += 2) {
+                    float x0, x1, p0, p1;
+                    fma2(x0, x1, __uint_as_float(r[c]), __uint_as_float(r[c + 1]), scale, neg_m);
+                    if (((q * 16 + (c >> 1)) % kPolyOneIn) == kPolyOneIn - 1) {
+                        ex2_poly2(p0, p1, x0, x1, poly_top);
+                    } else {
+                        p0 = ex2(x0);
+                        p1 = ex2(x1);
                     }
+                    if constexpr (kMasked) {
+                        p0 = q * 32 + c < live_keys ? p0 : 0.f;
+                        p1 = q * 32 + c + 1 < live_keys ? p1 : 0.f;
+                    }
+                    add2(rs[c & 2], rs[(c & 2) + 1], p0, p1);
+                    packed[c >> 1] = pack_bf16(p0, p1);
                 }
-                m_ref = m_new;
-                // a stream that has not seen a key yet (m_ref = -inf) stores zeros through the masked pass
-                // (every exponential on the special-function unit here: the careful path has no bound on its arguments to rely on)
-                rsum = need_mask ? exp_pass(std::true_type{}, std::false_type{}, -m_ref)
-                                 : exp_pass(std::false_type{}, std::false_type{}, -m_ref);
-            }
-            l_sum = l_sum * corr + rsum;
+                tmem_st16(s_addr + q * 16, packed);      // P as the next A operand
+            };
+            auto pass = [&](auto q_tag, const uint32_t (&r)[32]) {
+                if (need_mask) exp_pass(std::true_type{}, q_tag, r); else exp_pass(std::false_type{}, q_tag, r);
+            };
+            // each load stays in flight behind the arithmetic of the quarter before it
+            tmem_ld32(s_addr, sa);
+            tmem_ld32(s_addr + 32, sb);
+            tmem_wait_ld_of(sa);
+            tmem_wait_ld_of(sb);
+            pass(std::integral_constant<int, 0>{}, sa);
+            tmem_ld32(s_addr + 64, sa);
+            pass(std::integral_constant<int, 1>{}, sb);
+            tmem_wait_ld_of(sa);
+            tmem_ld32(s_addr + 96, sb);
+            pass(std::integral_constant<int, 2>{}, sa);
+            tmem_wait_ld_of(sb);
+            pass(std::integral_constant<int, 3>{}, sb);
+            const float rsum = (rs[0] + rs[1]) + (rs[2] + rs[3]);
+            outgrown = outgrown || !(rsum <= kRowSumLimit);       // also true for inf / NaN
+            l_sum += rsum;
             tmem_wait_st();
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive_cluster(leader_pfull + 8u * sb);
+            if (lane == 0) mbar_arrive_cluster(leader_pfull + 8u * sbuf);
         }
 
-        // ---- epilogue: merge the two streams, O / l -> bf16 rows of out; warpgroup w writes dims 64 w .. 64 w + 63 ----
-        pair_wait(bar_odone(0, (nmax - 1) & 1), ((nmax - 1) >> 1) & 1, s_abort, peer_abort, prm.status, 14);
-        pair_wait(bar_odone(1, (nmax - 1) & 1), ((nmax - 1) >> 1) & 1, s_abort, peer_abort, prm.status, 14);
-        tc_fence_after();
-        volatile float *x_ml = reinterpret_cast<volatile float *>(smem + kOffXMl);
-        x_ml[(wg * kRows + row) * 2] = m_ref;
-        x_ml[(wg * kRows + row) * 2 + 1] = l_sum;
-        named_bar_sync(1 + quarter, 64);                      // the two warps that share these rows
-        const float m0 = x_ml[row * 2], l0 = x_ml[row * 2 + 1], m1 = x_ml[(kRows + row) * 2], l1 = x_ml[(kRows + row) * 2 + 1];
-        const float m_all = fmaxf(m0, m1);
-        const float w0 = m0 == -INFINITY ? 0.f : ex2(m0 - m_all), w1 = m1 == -INFINITY ? 0.f : ex2(m1 - m_all);
-        const float l_all = l0 * w0 + l1 * w1;
-        const float inv = l_all > 0.f ? prm.out_scale / l_all : 0.f;
-        const float f0 = w0 * inv, f1 = w1 * inv;
-        const uint32_t o_both = lane_addr + kTmemO + wg * kCols;      // this warpgroup's 64 dims, in O_0; O_1 is 128 columns on
-        const long long orow = (static_cast<long long>(q_row0 + first_tok + tok_local) * prm.num_q_heads + head * g + head_local);
+        // a row that outgrew its reference (or whose scores are not finite): the unit is computed again by the kernel
+        // that moves the reference max
+        outgrown = outgrown || poly_top > kPolyArgTop;
+        if (__any_sync(0xffffffffu, outgrown) && lane == 0)
+            atomicOr(prm.redo_bits + ((unit % kRedoBits) >> 5), 1u << (unit & 31));
+
+        // ---- epilogue: O / l -> bf16 rows of out; warpgroups 0 and 1 write dims 0 .. 63 and 64 .. 127 ----
+        x_l[wg * kRows + row] = l_sum;
+        named_bar_sync(1, 128 * kSoftmaxGroups);
+        if (wg < 2) {
+            pair_wait(bar_odone, 0, s_abort, peer_abort, prm.status, 14);
+            tc_fence_after();
+            const float l_all = x_l[row] + x_l[kRows + row];
+            const float inv = l_all > 0.f ? prm.out_scale / l_all : 0.f;
+            const uint32_t o_addr = lane_addr + kTmemO + wg * 64;
+            const long long orow = (static_cast<long long>(q_row0 + first_tok + tok_local) * prm.num_q_heads + head * g + head_local);
 #pragma unroll 1
-        for (int c0 = 0; c0 < kCols; c0 += 32) {
-            uint32_t oa[32], ob[32];
-            tmem_ld32(o_both + c0, oa);
-            tmem_ld32(o_both + kHeadDim + c0, ob);
-            tmem_wait_ld();
-            if (live) {
-                float ov[32];
+            for (int c0 = 0; c0 < 64; c0 += 32) {
+                tmem_ld32(o_addr + c0, sa);
+                tmem_wait_ld_of(sa);
+                if (live) {
+                    uint4 *dst = reinterpret_cast<uint4 *>(prm.out + orow * kHeadDim + wg * 64 + c0);
 #pragma unroll
-                for (int k = 0; k < 32; ++k) ov[k] = fmaf(__uint_as_float(ob[k]), f1, __uint_as_float(oa[k]) * f0);
-                uint4 *dst = reinterpret_cast<uint4 *>(prm.out + orow * kHeadDim + wg * kCols + c0);
-#pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    uint4 v;
-                    v.x = pack_bf16(ov[8 * k], ov[8 * k + 1]);
-                    v.y = pack_bf16(ov[8 * k + 2], ov[8 * k + 3]);
-                    v.z = pack_bf16(ov[8 * k + 4], ov[8 * k + 5]);
-                    v.w = pack_bf16(ov[8 * k + 6], ov[8 * k + 7]);
-                    dst[k] = v;
+                    for (int k = 0; k < 4; ++k) {
+                        uint4 v;
+                        v.x = pack_bf16(__uint_as_float(sa[8 * k]) * inv, __uint_as_float(sa[8 * k + 1]) * inv);
+                        v.y = pack_bf16(__uint_as_float(sa[8 * k + 2]) * inv, __uint_as_float(sa[8 * k + 3]) * inv);
+                        v.z = pack_bf16(__uint_as_float(sa[8 * k + 4]) * inv, __uint_as_float(sa[8 * k + 5]) * inv);
+                        v.w = pack_bf16(__uint_as_float(sa[8 * k + 6]) * inv, __uint_as_float(sa[8 * k + 7]) * inv);
+                        dst[k] = v;
+                    }
                 }
             }
+            if (live && wg == 0 && prm.lse != nullptr) prm.lse[orow] = l_all > 0.f ? (-neg_m + log2f(l_all)) * kLn2 : -INFINITY;
         }
-        if (live && wg == 0 && prm.lse != nullptr) prm.lse[orow] = l_all > 0.f ? (m_all + log2f(l_all)) * kLn2 : -INFINITY;
     }
 
     // ---- all roles of both CTAs meet (nothing of the pair is in flight any more); the tensor memory goes back ----
@@ -588,35 +601,31 @@ chunk_attn_pair_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_co
 
 }  // namespace
 
-cudaError_t launch_chunk_attn_pair(const AttnCall &c, cudaStream_t stream, int64_t *launches) {
+cudaError_t launch_chunk_attn_pair(const AttnCall &c, int base, int n, cudaStream_t stream, int64_t *launches) {
     const int hkv = c.pool.num_kv_heads, g = c.num_q_heads / hkv, tpt = kRows / g;
     cudaError_t e = cudaFuncSetAttribute(chunk_attn_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (e != cudaSuccess) return e;
     CUtensorMap qmap, kmap, vmap;
     if (!encode_q_map(&qmap, c.q, c.total_q, c.num_q_heads, g) ||
-        !encode_pool_rows(&kmap, c.pool.k, c.pool.num_pages, hkv, c.pool.page_size) ||
+        !encode_pool_groups(&kmap, c.pool.k, c.pool.num_pages, hkv, c.pool.page_size) ||
         !encode_pool_rows(&vmap, c.pool.v, c.pool.num_pages, hkv, c.pool.page_size))
         return cudaErrorInvalidValue;
-    for (int base = 0; base < c.n_items; base += kMaxItems) {
-        const int n = c.n_items - base < kMaxItems ? c.n_items - base : kMaxItems;
-        PairParams prm;
-        prm.page_table = c.trajs.page_table; prm.seq_lens = c.trajs.seq_lens;
-        prm.traj_ids = c.traj_ids ? c.traj_ids + base : nullptr;
-        prm.q_indptr = c.q_indptr + base;
-        prm.max_pages = c.trajs.max_pages; prm.num_traj = c.trajs.num_traj; prm.num_pages = c.pool.num_pages;
-        prm.page_size = c.pool.page_size; prm.num_kv_heads = hkv; prm.num_q_heads = c.num_q_heads; prm.group = g;
-        prm.n_items = n; prm.item_offset = base; prm.max_seq_len = c.max_seq_len; prm.total_q = c.total_q;
-        prm.out = c.out; prm.lse = c.lse; prm.scale_log2 = c.sm_scale * kLog2e; prm.out_scale = c.v_scale; prm.status = c.status;
-        // an upper bound on the M-tile pairs of these items: every item has at most one ragged pair
-        const long long pairs = (static_cast<long long>(c.total_q) + 2 * tpt - 1) / (2 * tpt) + n;
-        const long long blocks = 2 * pairs * hkv;
-        if (blocks > 0x7FFFFFFFLL) return cudaErrorInvalidValue;
-        chunk_attn_pair_kernel<<<static_cast<unsigned>(blocks), kThreads, kSmemBytes, stream>>>(qmap, kmap, vmap, prm);
-        ++*launches;
-        e = cudaGetLastError();
-        if (e != cudaSuccess) return e;
-    }
-    return cudaSuccess;
+    PairParams prm;
+    prm.page_table = c.trajs.page_table; prm.seq_lens = c.trajs.seq_lens;
+    prm.traj_ids = c.traj_ids ? c.traj_ids + base : nullptr;
+    prm.q_indptr = c.q_indptr + base;
+    prm.max_pages = c.trajs.max_pages; prm.num_traj = c.trajs.num_traj; prm.num_pages = c.pool.num_pages;
+    prm.page_size = c.pool.page_size; prm.num_kv_heads = hkv; prm.num_q_heads = c.num_q_heads; prm.group = g;
+    prm.n_items = n; prm.item_offset = base; prm.max_seq_len = c.max_seq_len; prm.total_q = c.total_q;
+    prm.out = c.out; prm.lse = c.lse; prm.scale_log2 = c.sm_scale * kLog2e; prm.out_scale = c.v_scale;
+    prm.redo_bits = c.redo_bits; prm.status = c.status;
+    // an upper bound on the M-tile pairs of these items: every item has at most one ragged pair
+    const long long pairs = (static_cast<long long>(c.total_q) + 2 * tpt - 1) / (2 * tpt) + n;
+    const long long blocks = 2 * pairs * hkv;
+    if (blocks > 0x7FFFFFFFLL) return cudaErrorInvalidValue;
+    chunk_attn_pair_kernel<<<static_cast<unsigned>(blocks), kThreads, kSmemBytes, stream>>>(qmap, kmap, vmap, prm);
+    ++*launches;
+    return cudaGetLastError();
 }
 
 }  // namespace rollart

@@ -13,7 +13,8 @@ struct rollart_ctx {
     int sm_count;
     void *workspace;
     size_t workspace_bytes;
-    DeviceStatus *d_status;
+    DeviceStatus *d_status;  // followed, 256 bytes on, by the chunk calls' bitmap of units to compute again
+    uint32_t *d_redo;
     DeviceStatus *h_status;  // pinned
     int64_t launches;
     TmaCache tma;
@@ -109,6 +110,7 @@ AttnCall make_call(rollart_ctx *ctx, const rollart_kv_pool *pool, const rollart_
     c.shared_lens = nullptr;
     c.out_f32 = nullptr;
     c.item_order = nullptr;
+    c.redo_bits = ctx->d_redo;
     c.fp8 = false;
     c.k_scale = 1.f;
     c.v_scale = 1.f;
@@ -143,8 +145,9 @@ rollart_status rollart_create(rollart_ctx **out, int device, size_t workspace_by
         return ROLLART_ERR_UNSUPPORTED;
     }
     if (e == cudaSuccess) ctx->sm_count = prop.multiProcessorCount;
-    if (e == cudaSuccess) e = cudaMalloc(&ctx->d_status, sizeof(DeviceStatus));
-    if (e == cudaSuccess) e = cudaMemset(ctx->d_status, 0, sizeof(DeviceStatus));
+    if (e == cudaSuccess) e = cudaMalloc(&ctx->d_status, 256 + kChunkRedoBits / 8);
+    if (e == cudaSuccess) e = cudaMemset(ctx->d_status, 0, 256 + kChunkRedoBits / 8);
+    if (e == cudaSuccess) ctx->d_redo = reinterpret_cast<uint32_t *>(reinterpret_cast<char *>(ctx->d_status) + 256);
     if (e == cudaSuccess) e = cudaMallocHost(&ctx->h_status, sizeof(DeviceStatus));
     if (e == cudaSuccess && workspace_bytes) e = cudaMalloc(&ctx->workspace, workspace_bytes);
     if (e == cudaSuccess && workspace_bytes) e = cudaMemset(ctx->workspace, 0, workspace_bytes);

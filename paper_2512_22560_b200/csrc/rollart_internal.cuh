@@ -113,6 +113,7 @@ struct AttnCall {
     const int32_t *shared_lens;   // chunk: per item, every query row of the item sees exactly the first shared_lens[i] keys
     float *out_f32;               // when set the result rows are written here in fp32 instead of bf16 to `out`
     const int32_t *item_order;    // chunk: per batch of kChunkItemsPerLaunch items, the order in which blocks take them
+    uint32_t *redo_bits;          // chunk: kChunkRedoBits bits of the context, the units a second pass has to take
     // fp8 (E4M3) pools (decode and fused append + decode): keys are k_scale * code value, values v_scale * code value.
     // The chunk kernel reads bf16 only; it multiplies its result by v_scale (1 for bf16 pools).
     bool fp8;
@@ -128,7 +129,8 @@ cudaError_t launch_chunk_attn(const AttnCall &c, cudaStream_t stream, int64_t *l
 // diagnostic: a bounded in-kernel wait that must run out (see rollart_selftest_bounded_wait)
 cudaError_t launch_bounded_wait_selftest(DeviceStatus *status, cudaStream_t stream, int64_t *launches);
 // the causal chunk call on CTA pairs (no shared-prefix mode, bf16 output): what launch_chunk_attn runs for such calls
-cudaError_t launch_chunk_attn_pair(const AttnCall &c, cudaStream_t stream, int64_t *launches);
+// items base .. base + n - 1 of the call (at most kChunkItemsPerLaunch), c.redo_bits zeroed on the stream before
+cudaError_t launch_chunk_attn_pair(const AttnCall &c, int base, int n, cudaStream_t stream, int64_t *launches);
 
 // Observation-chunk attention over fp8 pools: the listed trajectories' contexts are expanded to bf16 into a scratch
 // pool (item i owns pages i * pages_per_item ..), with a scratch page table and scratch lengths behind the two pools.
@@ -149,6 +151,7 @@ cudaError_t launch_fp8_pages_to_bf16(const rollart_kv_pool &pool, const rollart_
 
 // items per launch of the chunk kernel (its per-item table lives in shared memory)
 constexpr int kChunkItemsPerLaunch = 1024;
+constexpr int kChunkRedoBits = 4096;      // bitmap of the units of a chunk launch that its second pass computes again
 
 // Group decode helpers.  `prepare` derives, per group, the trajectory whose table row stands for the shared
 // prefix and, per item, the pages to skip; it also checks that the members alias the same pages there.

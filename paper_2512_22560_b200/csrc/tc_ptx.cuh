@@ -121,6 +121,14 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16
 }
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+// The same wait for a load that was left in flight across other work: the registers of that load are named as operands,
+// so that no use of them can be scheduled above the wait.
+__device__ __forceinline__ void tmem_wait_ld_of(uint32_t (&r)[32]) {
+    asm volatile("tcgen05.wait::ld.sync.aligned;"
+                 : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]), "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]), "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]), "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
+                 :
+                 : "memory");
+}
 __device__ __forceinline__ float ex2(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -186,9 +194,9 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 // Shared-memory matrix descriptor of a 128B-swizzled operand tile whose 8-row groups are 1024 B
 // apart (stride byte offset); `lbo` is the distance between 64-element blocks along the
 // contiguous dimension of an MN-major operand (ignored for K-major tiles, where it is set to 16).
-__device__ __forceinline__ uint64_t smem_desc(uint32_t saddr, uint32_t lbo) {
+__device__ __forceinline__ uint64_t smem_desc(uint32_t saddr, uint32_t lbo, uint32_t sbo = 1024u) {
     return static_cast<uint64_t>((saddr & 0x3FFFFu) >> 4) | (static_cast<uint64_t>(lbo >> 4) << 16) |
-           (static_cast<uint64_t>(1024u >> 4) << 32) | (1ull << 46) | (2ull << 61);
+           (static_cast<uint64_t>(sbo >> 4) << 32) | (1ull << 46) | (2ull << 61);
 }
 // Instruction descriptor, kind::f16: fp32 accumulate, bf16 A and B, A K-major, D of m x n (m = 128 for one CTA, 256 for
 // a CTA pair: 128 rows in each CTA's tensor memory).
@@ -310,6 +318,21 @@ inline bool encode_pool_pages(CUtensorMap *map, const void *pool, int num_pages,
     const cuuint64_t dims[4] = {64, static_cast<cuuint64_t>(P), 2, static_cast<cuuint64_t>(num_pages) * hkv};
     const cuuint64_t strides[3] = {kRowBytes, 128, static_cast<cuuint64_t>(P) * kRowBytes};
     const cuuint32_t box[4] = {64, static_cast<cuuint32_t>(P), 2, 1};
+    const cuuint32_t ones[4] = {1, 1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(pool), dims, strides, box, ones,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// pool as [group of 8 rows][half][row in group][64 dims]; one box = the P rows of one (page, head) with both halves,
+// landing as [group][half][8 rows][128 B]: 8-row groups 2 KB apart whatever the page size, the second 64 dims of a
+// group 1 KB after the first.  One copy per page where the [rows][64 dims] view needs two.
+inline bool encode_pool_groups(CUtensorMap *map, const void *pool, int num_pages, int hkv, int P) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn || P % 8 != 0) return false;
+    const cuuint64_t dims[4] = {64, 8, 2, static_cast<cuuint64_t>(num_pages) * hkv * P / 8};
+    const cuuint64_t strides[3] = {kRowBytes, 128, 8 * kRowBytes};
+    const cuuint32_t box[4] = {64, 8, 2, static_cast<cuuint32_t>(P / 8)};
     const cuuint32_t ones[4] = {1, 1, 1, 1};
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(pool), dims, strides, box, ones,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,

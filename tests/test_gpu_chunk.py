@@ -357,3 +357,24 @@ def test_chunk_nan_key_reaches_every_row_that_sees_it(cuda_device):
             other = slice((1 - t % 2) * g, (1 - t % 2) * g + g)
             assert np.isfinite(got[a:b, other]).all(), (off, t)
             assert np.allclose(got[a:b, other], ref_o[a:b, other], atol=1e-2, rtol=2e-2), (off, t)
+
+
+def test_chunk_second_pass_among_thousands_of_units(cuda_device):
+    # More (item, kv head, M-tile pair) units than the bitmap of units to compute again has bits, a few of them with a
+    # key that towers over the rows' reference: those go through the second kernel, their aliases in the bitmap with
+    # them, and every row of every unit has to come out right whichever kernel wrote it last.
+    P, hq, hkv = 16, 8, 8
+    rng = np.random.default_rng(77)
+    T = 700
+    prior = rng.integers(129, 300, T).tolist()
+    n_new = rng.integers(1, 4, T).tolist()
+    batch = _custom_chunk_batch(P, hq, hkv, prior, n_new, 23, "chunk_many_units")
+    assert T * hkv > 4096
+    batch.q_new[:, :, 0] = 4.0
+    for t in range(0, T, 97):
+        pos = 128 + _LONE_OFFSETS[(t // 97) % len(_LONE_OFFSETS)]
+        key = torch.zeros(128)
+        key[0] = 300.0 / (4.0 * batch.spec.sm_scale * 1.4426950408889634)
+        pg = int(batch.page_table[t, pos // P])
+        batch.k_pool[pg, :, pos % P, :] = key.to(torch.bfloat16)
+    run_chunk_case(batch, cuda_device)
