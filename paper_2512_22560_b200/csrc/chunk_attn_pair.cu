@@ -71,7 +71,7 @@ constexpr int kMaxItems = kChunkItemsPerLaunch;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 constexpr float kRowSumLimit = 18446744073709551616.f;   // 2^64: a half-row sum of one tile above this marks the unit for the careful kernel
-constexpr int kPolyOneIn = 3;              // one pair of exponentials in this many goes to the FMA pipe
+constexpr int kPolyOneIn = 8;              // one pair of exponentials in this many goes to the FMA pipe
 
 constexpr int kHalfQ = kRows * 128;        // 16 KB: 128 rows x 64 dims
 constexpr int kTileQ = 2 * kHalfQ;         // [dim half][row][128 B]
