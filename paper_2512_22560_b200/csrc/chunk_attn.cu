@@ -655,7 +655,7 @@ cudaError_t launch_chunk_attn(const AttnCall &c, cudaStream_t stream, int64_t *l
     for (int base = 0; base < c.n_items; base += kMaxItems) {
         const int n = c.n_items - base < kMaxItems ? c.n_items - base : kMaxItems;
         if (plain) {
-            e = cudaMemsetAsync(c.redo_bits, 0, kChunkRedoBits / 8, stream);
+            e = cudaMemsetAsync(c.redo_bits, 0, kChunkRedoBits / 8 + 64, stream);      // the bitmap and, behind it, the pair kernel's unit counter
             if (e != cudaSuccess) return e;
             e = launch_chunk_attn_pair(c, base, n, stream, launches);
             if (e != cudaSuccess) return e;

@@ -13,7 +13,7 @@ struct rollart_ctx {
     int sm_count;
     void *workspace;
     size_t workspace_bytes;
-    DeviceStatus *d_status;  // followed, 256 bytes on, by the chunk calls' bitmap of units to compute again
+    DeviceStatus *d_status;  // followed, 256 bytes on, by the chunk calls' bitmap of units to compute again and their unit counter
     uint32_t *d_redo;
     DeviceStatus *h_status;  // pinned
     int64_t launches;
@@ -145,8 +145,8 @@ rollart_status rollart_create(rollart_ctx **out, int device, size_t workspace_by
         return ROLLART_ERR_UNSUPPORTED;
     }
     if (e == cudaSuccess) ctx->sm_count = prop.multiProcessorCount;
-    if (e == cudaSuccess) e = cudaMalloc(&ctx->d_status, 256 + kChunkRedoBits / 8);
-    if (e == cudaSuccess) e = cudaMemset(ctx->d_status, 0, 256 + kChunkRedoBits / 8);
+    if (e == cudaSuccess) e = cudaMalloc(&ctx->d_status, 256 + kChunkRedoBits / 8 + 64);
+    if (e == cudaSuccess) e = cudaMemset(ctx->d_status, 0, 256 + kChunkRedoBits / 8 + 64);
     if (e == cudaSuccess) ctx->d_redo = reinterpret_cast<uint32_t *>(reinterpret_cast<char *>(ctx->d_status) + 256);
     if (e == cudaSuccess) e = cudaMallocHost(&ctx->h_status, sizeof(DeviceStatus));
     if (e == cudaSuccess && workspace_bytes) e = cudaMalloc(&ctx->workspace, workspace_bytes);

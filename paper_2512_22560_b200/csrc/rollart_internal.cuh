@@ -113,7 +113,7 @@ struct AttnCall {
     const int32_t *shared_lens;   // chunk: per item, every query row of the item sees exactly the first shared_lens[i] keys
     float *out_f32;               // when set the result rows are written here in fp32 instead of bf16 to `out`
     const int32_t *item_order;    // chunk: per batch of kChunkItemsPerLaunch items, the order in which blocks take them
-    uint32_t *redo_bits;          // chunk: kChunkRedoBits bits of the context, the units a second pass has to take
+    uint32_t *redo_bits;          // chunk: kChunkRedoBits bits of the context, the units a second pass has to take; 64 more bytes behind them
     // fp8 (E4M3) pools (decode and fused append + decode): keys are k_scale * code value, values v_scale * code value.
     // The chunk kernel reads bf16 only; it multiplies its result by v_scale (1 for bf16 pools).
     bool fp8;
