@@ -349,7 +349,7 @@ rollart_status rollart_group_decode_attn_fp8(rollart_ctx *ctx, const rollart_kv_
  * chunk causally including itself.  Same formula, layout of q/out/lse ([total_q][...]) and
  * arithmetic as rollart_decode_attn; n_i = 1 is exactly a decode step.  n_i > L is a
  * ROLLART_ERR_BOUNDS device error for that item.
- * Per 1024 items the call enqueues a 512-byte clear and two kernels: the first keeps, per query row, the largest
+ * Per 1024 items the call enqueues a 576-byte clear and two kernels: the first keeps, per query row, the largest
  * score among the row's first 128 keys as the reference of its exponentials for the whole row; a block of rows in which
  * some later score lies more than 64 powers of two above that reference (or is not finite) is marked in a bitmap that
  * belongs to the context and is computed again by the second kernel, which moves its reference as it goes; the other
