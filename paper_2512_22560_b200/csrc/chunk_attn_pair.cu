@@ -79,7 +79,7 @@ constexpr int kThreads = 128 + 128 * kSoftmaxGroups + 32 * (kVCopyWarps - 1) + 3
 constexpr int kMaxItems = kChunkItemsPerLaunch;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
-constexpr float kRowSumLimit = 18446744073709551616.f;   // 2^64: a half-row sum of one tile above this marks the unit for the careful kernel
+constexpr float kRowSumLimit = 18446744073709551616.f;   // 2^64: a row sum of one tile above this marks the unit for the careful kernel
 constexpr int kPolyOneIn = 8;              // one pair of exponentials in this many goes to the FMA pipe
 
 constexpr int kHalfQ = kRows * 128;        // 16 KB: 128 rows x 64 dims
@@ -103,7 +103,7 @@ constexpr int kSmemBytes = kSmemUsed + 1024;               // + slack for the 10
 static_assert(kSmemBytes <= 227 * 1024, "one block must fit an SM");
 static_assert(kSoftmaxGroups < kSBufs, "a warpgroup finds the S of its next tile computed while it works on this one");
 
-constexpr int kTmemCols = 512;             // S buffer b at columns b * 128; warpgroup w's P over the first 32 columns of its half (64 w ..) of the S buffer
+constexpr int kTmemCols = 512;             // S buffer b at columns b * 128; the tile's P (packed bf16) over its first 64 columns
 constexpr int kTmemO = kSBufs * kKeys;     // O at 384
 constexpr int kRedoBits = kChunkRedoBits;  // units of a launch are marked in a bitmap of this many bits (unit mod kRedoBits)
 
@@ -205,9 +205,9 @@ chunk_attn_pair_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_co
     for (int i = threadIdx.x; i < kTileQ / 16; i += kThreads) reinterpret_cast<uint4 *>(smem + kOffQ)[i] = make_uint4(0, 0, 0, 0);
     if (warp == 0) tmem_alloc_pair(smem_u32(smem + kOffTmemSlot), kTmemCols);
 
-    // ---- which (item, kv head, pair of M-tiles) is this cluster?  pairs per item -> prefix -> search.  The same pass
-    //      keeps every item's rows, trajectory and length in shared memory, so that the unit's geometry below needs no
-    //      further (dependent) global loads ----
+    // ---- the tables from which a unit number gives (item, kv head, pair of M-tiles): pairs per item -> prefix (searched
+    //      per unit), and every item's rows, trajectory and length, so that a unit's geometry needs no (dependent)
+    //      global loads ----
     int *s_item = s_prefix + (kMaxItems + 1);             // [item][4]: first row, rows, trajectory, length (-1: invalid trajectory)
     for (int i = threadIdx.x; i < prm.n_items; i += kThreads) {
         const int q0 = __ldg(prm.q_indptr + i), n = __ldg(prm.q_indptr + i + 1) - q0;
@@ -234,9 +234,9 @@ chunk_attn_pair_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_co
     }
     __syncthreads();
     const int total_units = s_prefix[prm.n_items] * hkv;
-    // The pair is persistent: cluster c takes the units c, c + #clusters, ...  Units are numbered (item, head, pair) with
-    // the later (longer) pairs of an (item, head) first, so the pairs re-reading the same keys run at the same time on
-    // neighbouring clusters.  Every role walks the same list and derives a unit's geometry from the tables by itself.
+    // Units are numbered (item, head, pair) with the later (longer) pairs of an (item, head) first, and the persistent
+    // pairs take them in that order, so the pairs re-reading the same keys run at the same time.  Every role walks the
+    // same list of unit numbers and derives a unit's geometry from the tables by itself.
     struct Unit {
         bool active;
         int head, q_row0, n_chunk, t, L, prior, first_tok, toks, nmax, min_count;
@@ -589,7 +589,7 @@ chunk_attn_pair_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_co
             x_m[row] = rmax;
             // (a reference of -inf, +inf or NaN, i.e. scores that are not finite, ends in a row sum that marks the unit)
         }
-        named_bar_sync(1, 128 * kSoftmaxGroups);              // the other warpgroups take the reference from here
+        named_bar_sync(1, 128 * kSoftmaxGroups);              // the other warpgroup takes the reference from here
         const float neg_m = -x_m[row];
 
         for (int j = wg; j < nmax; j += kSoftmaxGroups) {
@@ -659,7 +659,7 @@ chunk_attn_pair_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_co
         if (__any_sync(0xffffffffu, outgrown) && lane == 0)
             atomicOr(prm.redo_bits + ((unit % kRedoBits) >> 5), 1u << (unit & 31));
 
-        // ---- epilogue: O / l -> bf16 rows of out; warpgroups 0 and 1 write dims 0 .. 63 and 64 .. 127 ----
+        // ---- epilogue: O / l -> bf16 rows of out; warpgroup w writes dims 64 w .. 64 w + 63 ----
         x_l[wg * kRows + row] = l_sum;
         named_bar_sync(1, 128 * kSoftmaxGroups);
         {
@@ -730,7 +730,7 @@ cudaError_t launch_chunk_attn_pair(const AttnCall &c, int base, int n, cudaStrea
     // an upper bound on the M-tile pairs of these items: every item has at most one ragged pair
     const long long pairs = (static_cast<long long>(c.total_q) + 2 * tpt - 1) / (2 * tpt) + n;
     if (pairs * hkv > 0x3FFFFFFFLL) return cudaErrorInvalidValue;
-    // persistent pairs: one cluster per two SMs (or fewer, when there are fewer units), each walking its share of the units
+    // persistent pairs: one cluster per two SMs (or fewer, when there are fewer units), taking the units from the counter
     const long long clusters = std::max(1LL, std::min<long long>(pairs * hkv, (c.sm_count > 1 ? c.sm_count : 2) / 2));
     chunk_attn_pair_kernel<<<static_cast<unsigned>(2 * clusters), kThreads, kSmemBytes, stream>>>(qmap, kmap, vmap, prm);
     ++*launches;
