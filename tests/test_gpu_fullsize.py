@@ -226,6 +226,12 @@ def test_full_size_mixed_batch_chunk_sampled_rows(cuda_device):
     qsel = q[torch.from_numpy(q_rows).to(cuda_device)]
     ref_o, _ = oracle.attend_rows(kp, vp, post.page_table, row_traj, row_count, W.bf16_to_u16(qsel), spec.sm_scale)
     assert_attn_close(out[torch.from_numpy(q_rows).to(cuda_device)], ref_o, "cfg4 chunk rows")
+    # the pairs take their units from a counter, in whatever order they finish: the result must not depend on it
+    again = torch.full_like(q, float("nan"))
+    ctx.obs_chunk_attn(db.k_pool, db.v_pool, db.page_table, db.lens_after, dev_i32(q_indptr, cuda_device), q, spec.sm_scale,
+                       msl, again, traj_ids=dev_i32(ids, cuda_device))
+    ctx.check()
+    assert torch.equal(again.view(torch.int16), out.view(torch.int16))
     ctx.close()
 
 
